@@ -1,0 +1,174 @@
+/*
+ * uniql.h -- C ABI of the UniQL inference hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates the linear layers of a model compressed the UniQL way
+ * (arXiv 2512.03383): 4-bit group-quantised weights whose rows / columns were
+ * sorted offline by importance, so that the pruning rate chosen on the device
+ * only TRUNCATES each matrix to its leading sorted channels (Section 3.4,
+ * "Quantization and On-device Adaptive Pruning").  Where the paper unpacks,
+ * slices and re-packs the INT4 tensors whenever the rate changes, here the
+ * kept channels are kernel arguments: nothing is copied or re-packed.
+ * The Q / K projections also apply the rotary embedding to the retained head
+ * dimensions, each surviving pair using the frequency of its ORIGINAL index
+ * (Section 3.2, MHSA paragraph and Figure 3a, "fused RoPE kernel").
+ *
+ * Conventions
+ *  - Pointers are DEVICE pointers unless a comment says "host".  The caller owns
+ *    every buffer; the library never frees or keeps caller memory.
+ *  - All work is enqueued on `stream` (a cudaStream_t passed as void*); no call
+ *    synchronises the device.
+ *  - Every function returns a uniql_status.  Argument errors are detected on the
+ *    host before anything is launched; nothing aborts or throws.
+ *  - There is no CPU fallback: without a usable CUDA device calls return
+ *    UNIQL_ERR_CUDA.
+ *
+ * Weight format (the interchange format; benchmark configuration 1)
+ *  - W is stored in nn.Linear orientation, W[N][K]: N output channels (rows),
+ *    K input channels, y = x W^T.  The paper writes W in R^{D_in x D_out}
+ *    (Section 3.1); this is its transpose.
+ *  - packed_w: uint8 [N][K/2]; byte b of row n holds input channel 2b in its low
+ *    nibble and 2b+1 in its high nibble.  16-byte aligned, K % 128 == 0.
+ *  - scales, zeros: fp16 [N][K/128], one pair per group of 128 consecutive STORED
+ *    input channels:  w(n,k) = scale(n,k/128) * (code(n,k) - zero(n,k/128)).
+ *    The paper's symmetric quantiser (Section 3.4 equation, N=4, group 128) is
+ *    the case code = clamp(round(W/s),-8,7) + 8, zero = 8.  zero may be any
+ *    finite fp16 value.
+ *
+ * Activations: x[M][ldx] and y[M][ldy], fp16 or bf16 (same type for both), COMPACT:
+ * column t of x multiplies the t-th retained input channel, column j of y is the
+ * j-th retained output channel.  Accumulation is fp32, one rounding to the output
+ * type at the end (after the rotary embedding where it applies).
+ */
+#ifndef UNIQL_H_
+#define UNIQL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  UNIQL_OK = 0,
+  UNIQL_ERR_NULL = 1,        /* a required pointer is NULL */
+  UNIQL_ERR_SHAPE = 2,       /* a size is out of range or inconsistent */
+  UNIQL_ERR_ALIGN = 3,       /* a pointer or leading dimension is not aligned as required */
+  UNIQL_ERR_DTYPE = 4,       /* unknown uniql_dtype */
+  UNIQL_ERR_UNSUPPORTED = 5, /* valid request that no kernel of the forced path covers */
+  UNIQL_ERR_WORKSPACE = 6,   /* workspace too small (see uniql_workspace_bytes) */
+  UNIQL_ERR_TIMEOUT = 7,     /* a bounded device-side wait expired */
+  UNIQL_ERR_CUDA = 8         /* a CUDA runtime call failed (sticky errors included) */
+} uniql_status;
+
+typedef enum { UNIQL_F16 = 0, UNIQL_BF16 = 1 } uniql_dtype;
+
+/* Kernel selection, for A/B tests.  AUTO: M <= 16 decode kernel, M >= 64 prefill
+ * (tensor-core) kernel when its alignment rules hold, otherwise the generic kernel. */
+typedef enum { UNIQL_PATH_AUTO = 0, UNIQL_PATH_GENERIC = 1, UNIQL_PATH_DECODE = 2,
+               UNIQL_PATH_PREFILL = 3 } uniql_path;
+
+/* Channel map (host struct, copied by value at call time).
+ * On-device pruning keeps the leading sorted channels of D_int, of every head's
+ * D_hd and of D_s, never of D_h (Section 3.4).  Because heads are concatenated,
+ * "leading channels of every head" is a periodic set; a map is a short list of
+ * such families.  Family f keeps channels start + h*period + i for h < count,
+ * i < keep (STORED coordinates).  The compact order is family after family, block
+ * after block.  Families must be given in increasing, non-overlapping order.
+ *   MLP intermediate, keep k:           {0, k, k, 1}
+ *   V rows / o_proj columns, per head:  {0, D_hd, d', H}
+ *   Q or K rows (symmetric sort, Algorithm 2: idx_sym = [argsort, D_hd/2+argsort],
+ *     so each half head keeps its leading d'/2 rows):  {0, D_hd/2, d'/2, 2H}     */
+#define UNIQL_MAX_FAMILIES 8
+typedef struct { int32_t start, period, keep, count; } uniql_family;
+typedef struct { int32_t n_fam; uniql_family fam[UNIQL_MAX_FAMILIES]; } uniql_chanmap;
+
+/* One weight matrix of a multi-matrix call (host struct; pointers inside are device). */
+typedef struct {
+  const uint8_t* packed_w;      /* [N][K/2] */
+  const void* scales;           /* fp16 [N][K/128] */
+  const void* zeros;            /* fp16 [N][K/128] */
+  const void* bias;             /* activation dtype [N] in STORED coordinates, or NULL */
+  int32_t N;                    /* stored rows */
+  int32_t k_out;                /* used when out_map is NULL: keep the leading k_out rows */
+  const uniql_chanmap* out_map; /* host, or NULL */
+  void* y;                      /* [M][ldy] */
+  int32_t ldy;                  /* elements; >= number of retained rows */
+} uniql_job;
+#define UNIQL_MAX_JOBS 4
+
+int uniql_version(void);                 /* major*10000 + minor*100 + patch */
+const char* uniql_status_string(int status);
+
+/* Force a kernel path for subsequent calls of this process (tests / A-B timing). */
+int uniql_set_path(int path);
+
+/* ---- storage helpers (Section 3.4: 4-bit codes; bit-exact integer work) ----
+ * codes: uint8 [N][K], one code (0..15) per byte.  packed: uint8 [N][K/2].  K even. */
+int uniql_pack_u4(const uint8_t* codes, int64_t N, int64_t K, uint8_t* packed, void* stream);
+int uniql_unpack_u4(const uint8_t* packed, int64_t N, int64_t K, uint8_t* codes, void* stream);
+/* Full de-quantised matrix w[N][K] in `dt` (diagnostic; the hot path never materialises it).
+ * Computed as fp32 scale*(code-zero), rounded once. */
+int uniql_dequant(const uint8_t* packed, const void* scales, const void* zeros, int64_t N, int64_t K,
+                  int dt, void* w, void* stream);
+
+/* ---- workspace ----
+ * The decode kernel may split the input channels over several thread blocks; partial sums
+ * and arrival counters live in a workspace.  Calls without a workspace argument use a
+ * per-device buffer the library allocates at its first use on that device (so the first
+ * call on a device must not happen during stream capture).  A caller-provided workspace
+ * must be 256-byte aligned, at least uniql_workspace_bytes() large, and prepared once by
+ * uniql_workspace_init (zeroes the counters; they return to zero after every call).
+ * Calls that share a workspace must not overlap on the device. */
+size_t uniql_workspace_bytes(int M, int K, int N_total);
+int uniql_workspace_init(void* workspace, size_t bytes, void* stream);
+
+/* ---- the quantised, pruned linear layer (Section 3.4; decode and prefill of Section 5) ----
+ * Simple form: fp16 x[M][k_in], fp16 y[M][k_out], keep the leading k_in input and k_out
+ * output channels of the sorted matrix W[N][K].  k_in, k_out > 0, multiples of 4,
+ * k_in <= K, k_out <= N, M >= 1. */
+int uniql_qlinear(const void* x, const uint8_t* packed_w, const void* scales, const void* zeros,
+                  int M, int K, int N, int k_in, int k_out, void* y, void* stream);
+
+/* General form: dtype, leading dimensions, bias, channel maps (NULL map = leading k).
+ * x and y must be 4-byte aligned with even ldx / ldy; every family's start and keep must be
+ * multiples of 4.  workspace may be NULL (library buffer). */
+int uniql_qlinear_ex(const void* x, int ldx, int dt, const uint8_t* packed_w, const void* scales,
+                     const void* zeros, const void* bias, int M, int K, int N,
+                     const uniql_chanmap* in_map, int k_in, const uniql_chanmap* out_map, int k_out,
+                     void* y, int ldy, void* workspace, size_t ws_bytes, void* stream);
+
+/* Several matrices that share x, M, K and the input map in ONE launch (gate|up, q|k|v).
+ * jobs: host array of n_jobs <= UNIQL_MAX_JOBS entries. */
+int uniql_qlinear_multi(const void* x, int ldx, int dt, int M, int K, const uniql_chanmap* in_map,
+                        int k_in, int n_jobs, const uniql_job* jobs, void* workspace, size_t ws_bytes,
+                        void* stream);
+
+/* ---- fused Q and K projection + rotary embedding on the retained head dims ----
+ * (Section 3.2 MHSA paragraph, Figure 3a; GQA index sharing: Algorithm 6.)
+ * Wq[n_q_heads*head_dim][K] and Wk[n_kv_heads*head_dim][K] are symmetric-sorted per head;
+ * each head keeps head_keep dims: rows [0, head_keep/2) of both of its halves.
+ * q_out[M][n_q_heads*head_keep], k_out[M][n_kv_heads*head_keep]; inside a head the order is
+ * [first-half survivors | second-half survivors].  Compact pair c = (column c, column
+ * c + head_keep/2) of query head h is rotated by angle pos[m] * inv_freq[p] with
+ * p = retained_idx[h / (n_q_heads/n_kv_heads)][c], the ORIGINAL pair index (only half of the
+ * symmetric index vector is stored), inv_freq[p] = theta^(-2p/head_dim) unless a table is
+ * given:  (a, b) -> (a cos - b sin, b cos + a sin), applied to the fp32 accumulators (bias
+ * included) before the single output rounding.
+ *   retained_idx: device int32 [n_kv_heads][head_keep/2], values in [0, head_dim/2)
+ *   pos:          device int32 [M]
+ *   inv_freq:     HOST double [head_dim/2] or NULL
+ * head_dim even, <= 256; head_keep % 4 == 0; n_q_heads % n_kv_heads == 0.
+ * Index values are not range-checked on the host (they live on the device); the kernels
+ * clamp them into [0, head_dim/2). */
+int uniql_qk_rope_proj(const void* x, int ldx, int dt, const uint8_t* wq, const void* sq,
+                       const void* zq, const uint8_t* wk, const void* sk, const void* zk,
+                       const void* bq, const void* bk, int M, int K, int n_q_heads, int n_kv_heads,
+                       int head_dim, int head_keep, const int32_t* retained_idx, const int32_t* pos,
+                       double theta, const double* inv_freq, void* q_out, int ldq, void* k_out,
+                       int ldk, void* workspace, size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* UNIQL_H_ */

@@ -1,0 +1,243 @@
+// Host side of the C ABI: argument validation, channel-map compilation, workspace handling
+// and the dispatch by M between the decode, prefill and generic kernels.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "common.cuh"
+
+using namespace uniql;
+
+namespace {
+
+int g_path = UNIQL_PATH_AUTO;
+
+constexpr int kMaxDevices = 64;
+constexpr size_t kLibWorkspaceBytes = (size_t)96 << 20;
+void* g_ws[kMaxDevices] = {nullptr};
+std::mutex g_ws_mutex;
+
+// Per-device library workspace, allocated (and its counters zeroed) at first use.
+int lib_workspace(void** ws, size_t* bytes, cudaStream_t stream) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return UNIQL_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_ws_mutex);
+  if (!g_ws[dev]) {
+    void* p = nullptr;
+    if (cudaMalloc(&p, kLibWorkspaceBytes) != cudaSuccess) { cudaGetLastError(); return UNIQL_ERR_CUDA; }
+    if (cudaMemset(p, 0, kLibWorkspaceBytes) != cudaSuccess) { cudaFree(p); return UNIQL_ERR_CUDA; }
+    g_ws[dev] = p;
+  }
+  (void)stream;
+  *ws = g_ws[dev];
+  *bytes = kLibWorkspaceBytes;
+  return UNIQL_OK;
+}
+
+// Validate a caller map against a dimension of size D and compile it.
+int compile_map(const uniql_chanmap* src, int k_lead, int D, ChanMap* out) {
+  memset(out, 0, sizeof(*out));
+  if (!src) {
+    if (k_lead <= 0 || k_lead > D) return UNIQL_ERR_SHAPE;
+    out->n_fam = 1;
+    out->fam[0] = Fam{0, k_lead, k_lead, 1};
+    out->base[0] = 0;
+    out->total = k_lead;
+    return UNIQL_OK;
+  }
+  if (src->n_fam < 1 || src->n_fam > kMaxFam) return UNIQL_ERR_SHAPE;
+  int64_t prev_end = 0, total = 0;
+  for (int f = 0; f < src->n_fam; ++f) {
+    const uniql_family& a = src->fam[f];
+    if (a.start < 0 || a.keep <= 0 || a.count <= 0 || a.period <= 0) return UNIQL_ERR_SHAPE;
+    if (a.count > 1 && a.period < a.keep) return UNIQL_ERR_SHAPE;
+    int64_t end = (int64_t)a.start + (int64_t)(a.count - 1) * a.period + a.keep;
+    if (a.start < prev_end || end > D) return UNIQL_ERR_SHAPE;
+    prev_end = end;
+    out->fam[f] = Fam{a.start, a.period, a.keep, a.count};
+    out->base[f] = (int)total;
+    total += (int64_t)a.keep * a.count;
+  }
+  if (total > D) return UNIQL_ERR_SHAPE;
+  out->n_fam = src->n_fam;
+  out->total = (int)total;
+  return UNIQL_OK;
+}
+
+int check_common(const void* x, int ldx, int dt, int M, int K) {
+  if (!x) return UNIQL_ERR_NULL;
+  if (dt != UNIQL_F16 && dt != UNIQL_BF16) return UNIQL_ERR_DTYPE;
+  if (M < 1 || K < kGroup || (K % kGroup) != 0 || ldx < 1) return UNIQL_ERR_SHAPE;
+  if (((uintptr_t)x) & 1) return UNIQL_ERR_ALIGN;
+  return UNIQL_OK;
+}
+
+int check_weight(const uint8_t* w, const void* s, const void* z, int N) {
+  if (!w || !s || !z) return UNIQL_ERR_NULL;
+  if (N < 1) return UNIQL_ERR_SHAPE;
+  if ((((uintptr_t)w) & 15) || (((uintptr_t)s) & 1) || (((uintptr_t)z) & 1)) return UNIQL_ERR_ALIGN;
+  return UNIQL_OK;
+}
+
+int dispatch(const Params& p, void* workspace, size_t ws_bytes, void* stream) {
+  if (cudaPeekAtLastError() != cudaSuccess) return UNIQL_ERR_CUDA;
+  LaunchCfg cfg{workspace, ws_bytes, (cudaStream_t)stream};
+  int path = g_path;
+  bool dec_ok = p.M <= 16 && decode_supported(p);
+  bool pre_ok = p.M >= 64 && prefill_supported(p);
+  if (path == UNIQL_PATH_AUTO) path = dec_ok ? UNIQL_PATH_DECODE : (pre_ok ? UNIQL_PATH_PREFILL : UNIQL_PATH_GENERIC);
+  if (path == UNIQL_PATH_DECODE) {
+    if (!(p.M <= 16 && decode_supported(p))) return UNIQL_ERR_UNSUPPORTED;
+    if (!cfg.workspace) {
+      int rc = lib_workspace(&cfg.workspace, &cfg.ws_bytes, cfg.stream);
+      if (rc != UNIQL_OK) return rc;
+    }
+    return launch_decode(p, cfg);
+  }
+  if (path == UNIQL_PATH_PREFILL) {
+    if (!prefill_supported(p)) return UNIQL_ERR_UNSUPPORTED;
+    return launch_prefill(p, cfg);
+  }
+  return launch_generic(p, cfg);
+}
+
+}  // namespace
+
+extern "C" int uniql_version(void) { return 100; }
+
+extern "C" const char* uniql_status_string(int s) {
+  switch (s) {
+    case UNIQL_OK: return "ok";
+    case UNIQL_ERR_NULL: return "null pointer";
+    case UNIQL_ERR_SHAPE: return "bad shape";
+    case UNIQL_ERR_ALIGN: return "bad alignment";
+    case UNIQL_ERR_DTYPE: return "bad dtype";
+    case UNIQL_ERR_UNSUPPORTED: return "unsupported on the forced path";
+    case UNIQL_ERR_WORKSPACE: return "workspace too small";
+    case UNIQL_ERR_TIMEOUT: return "device-side wait timed out";
+    case UNIQL_ERR_CUDA: return "CUDA error";
+    default: return "unknown status";
+  }
+}
+
+extern "C" int uniql_set_path(int path) {
+  if (path < UNIQL_PATH_AUTO || path > UNIQL_PATH_PREFILL) return UNIQL_ERR_SHAPE;
+  g_path = path;
+  return UNIQL_OK;
+}
+
+extern "C" size_t uniql_workspace_bytes(int M, int K, int N_total) {
+  if (M < 1 || K < 1 || N_total < 1) return 0;
+  return decode_workspace_bytes(M, K, N_total);
+}
+
+extern "C" int uniql_workspace_init(void* workspace, size_t bytes, void* stream) {
+  if (!workspace) return UNIQL_ERR_NULL;
+  if (((uintptr_t)workspace) & 255) return UNIQL_ERR_ALIGN;
+  if (bytes == 0) return UNIQL_ERR_WORKSPACE;
+  return cudaMemsetAsync(workspace, 0, bytes, (cudaStream_t)stream) == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
+}
+
+extern "C" int uniql_qlinear_multi(const void* x, int ldx, int dt, int M, int K, const uniql_chanmap* in_map,
+                                   int k_in, int n_jobs, const uniql_job* jobs, void* workspace,
+                                   size_t ws_bytes, void* stream) {
+  int rc = check_common(x, ldx, dt, M, K);
+  if (rc) return rc;
+  if (!jobs) return UNIQL_ERR_NULL;
+  if (n_jobs < 1 || n_jobs > kMaxJobs) return UNIQL_ERR_SHAPE;
+  if (workspace && (((uintptr_t)workspace) & 255)) return UNIQL_ERR_ALIGN;
+  Params p;
+  memset(&p, 0, sizeof(p));
+  rc = compile_map(in_map, k_in, K, &p.imap);
+  if (rc) return rc;
+  p.x = x; p.ldx = ldx; p.dt = dt; p.M = M; p.K = K; p.k_in = p.imap.total;
+  if (ldx < p.k_in) return UNIQL_ERR_SHAPE;
+  p.n_jobs = n_jobs;
+  for (int j = 0; j < n_jobs; ++j) {
+    const uniql_job& s = jobs[j];
+    rc = check_weight(s.packed_w, s.scales, s.zeros, s.N);
+    if (rc) return rc;
+    if (!s.y) return UNIQL_ERR_NULL;
+    if ((((uintptr_t)s.y) & 1) || (s.bias && (((uintptr_t)s.bias) & 1))) return UNIQL_ERR_ALIGN;
+    JobDev& d = p.job[j];
+    rc = compile_map(s.out_map, s.k_out, s.N, &d.omap);
+    if (rc) return rc;
+    d.w = s.packed_w; d.scales = (const __half*)s.scales; d.zeros = (const __half*)s.zeros;
+    d.bias = s.bias; d.y = s.y; d.ldy = s.ldy; d.N = s.N; d.k_out = d.omap.total;
+    if (s.ldy < d.k_out) return UNIQL_ERR_SHAPE;
+  }
+  return dispatch(p, workspace, ws_bytes, stream);
+}
+
+extern "C" int uniql_qlinear_ex(const void* x, int ldx, int dt, const uint8_t* packed_w, const void* scales,
+                                const void* zeros, const void* bias, int M, int K, int N,
+                                const uniql_chanmap* in_map, int k_in, const uniql_chanmap* out_map,
+                                int k_out, void* y, int ldy, void* workspace, size_t ws_bytes, void* stream) {
+  uniql_job job;
+  memset(&job, 0, sizeof(job));
+  job.packed_w = packed_w; job.scales = scales; job.zeros = zeros; job.bias = bias;
+  job.N = N; job.k_out = k_out; job.out_map = out_map; job.y = y; job.ldy = ldy;
+  return uniql_qlinear_multi(x, ldx, dt, M, K, in_map, k_in, 1, &job, workspace, ws_bytes, stream);
+}
+
+extern "C" int uniql_qlinear(const void* x, const uint8_t* packed_w, const void* scales, const void* zeros,
+                             int M, int K, int N, int k_in, int k_out, void* y, void* stream) {
+  return uniql_qlinear_ex(x, k_in, UNIQL_F16, packed_w, scales, zeros, nullptr, M, K, N, nullptr, k_in,
+                          nullptr, k_out, y, k_out, nullptr, 0, stream);
+}
+
+extern "C" int uniql_qk_rope_proj(const void* x, int ldx, int dt, const uint8_t* wq, const void* sq,
+                                  const void* zq, const uint8_t* wk, const void* sk, const void* zk,
+                                  const void* bq, const void* bk, int M, int K, int n_q_heads,
+                                  int n_kv_heads, int head_dim, int head_keep, const int32_t* retained_idx,
+                                  const int32_t* pos, double theta, const double* inv_freq, void* q_out,
+                                  int ldq, void* k_out, int ldk, void* workspace, size_t ws_bytes,
+                                  void* stream) {
+  int rc = check_common(x, ldx, dt, M, K);
+  if (rc) return rc;
+  if (!retained_idx || !pos || !q_out || !k_out) return UNIQL_ERR_NULL;
+  if (n_q_heads < 1 || n_kv_heads < 1 || (n_q_heads % n_kv_heads) != 0) return UNIQL_ERR_SHAPE;
+  if (head_dim < 2 || (head_dim & 1) || head_dim > 2 * kMaxHalfDim) return UNIQL_ERR_SHAPE;
+  if (head_keep < 2 || (head_keep & 1) || head_keep > head_dim) return UNIQL_ERR_SHAPE;
+  if (!inv_freq && !(theta > 0.0)) return UNIQL_ERR_SHAPE;
+  if (ldx < K) return UNIQL_ERR_SHAPE;   // the hidden dimension D_h is never pruned (Section 3.4)
+  if (ldq < n_q_heads * head_keep || ldk < n_kv_heads * head_keep) return UNIQL_ERR_SHAPE;
+  if ((((uintptr_t)q_out) & 1) || (((uintptr_t)k_out) & 1) || (((uintptr_t)retained_idx) & 3) ||
+      (((uintptr_t)pos) & 3))
+    return UNIQL_ERR_ALIGN;
+  if ((bq && (((uintptr_t)bq) & 1)) || (bk && (((uintptr_t)bk) & 1))) return UNIQL_ERR_ALIGN;
+  if (workspace && (((uintptr_t)workspace) & 255)) return UNIQL_ERR_ALIGN;
+  rc = check_weight(wq, sq, zq, n_q_heads * head_dim);
+  if (rc) return rc;
+  rc = check_weight(wk, sk, zk, n_kv_heads * head_dim);
+  if (rc) return rc;
+
+  Params p;
+  memset(&p, 0, sizeof(p));
+  compile_map(nullptr, K, K, &p.imap);
+  p.x = x; p.ldx = ldx; p.dt = dt; p.M = M; p.K = K; p.k_in = K;
+  p.n_jobs = 2;
+  p.idx = retained_idx; p.pos = pos;
+  for (int i = 0; i < head_dim / 2; ++i)
+    p.inv_freq[i] = inv_freq ? inv_freq[i] : pow(theta, -2.0 * (double)i / (double)head_dim);
+  for (int j = 0; j < 2; ++j) {
+    JobDev& d = p.job[j];
+    int nh = j == 0 ? n_q_heads : n_kv_heads;
+    d.w = j == 0 ? wq : wk;
+    d.scales = (const __half*)(j == 0 ? sq : sk);
+    d.zeros = (const __half*)(j == 0 ? zq : zk);
+    d.bias = j == 0 ? bq : bk;
+    d.y = j == 0 ? q_out : k_out;
+    d.ldy = j == 0 ? ldq : ldk;
+    d.N = nh * head_dim;
+    d.k_out = nh * head_keep;
+    uniql_chanmap hm;
+    hm.n_fam = 1;
+    hm.fam[0] = uniql_family{0, head_dim / 2, head_keep / 2, 2 * nh};
+    compile_map(&hm, 0, d.N, &d.omap);
+    d.rope = RopeDesc{1, nh, j == 0 ? n_q_heads / n_kv_heads : 1, head_dim, head_keep};
+  }
+  return dispatch(p, workspace, ws_bytes, stream);
+}

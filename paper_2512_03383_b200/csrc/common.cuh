@@ -1,0 +1,144 @@
+// Internal structures and device helpers shared by the UniQL kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/uniql.h"
+
+namespace uniql {
+
+constexpr int kGroup = 128;       // quantisation group along the input channels (Section 3.4)
+constexpr int kMaxFam = UNIQL_MAX_FAMILIES;
+constexpr int kMaxJobs = UNIQL_MAX_JOBS;
+constexpr int kMaxHalfDim = 128;  // head_dim/2 <= 128
+
+struct Fam { int start, period, keep, count; };
+
+// A channel map with the compact offset of every family precomputed.
+struct ChanMap {
+  int n_fam;
+  int total;            // number of retained channels
+  Fam fam[kMaxFam];
+  int base[kMaxFam];    // compact index of the family's first channel
+};
+
+// Rotary-embedding description of a job (Section 3.2, fused RoPE with index gather).
+struct RopeDesc {
+  int enabled;
+  int n_heads;      // heads of THIS matrix (query heads for Wq, kv heads for Wk)
+  int rep;          // query heads per kv head (1 for Wk)
+  int head_dim;     // un-pruned D_hd
+  int head_keep;    // retained dims per head (even)
+};
+
+struct JobDev {
+  const uint8_t* w;
+  const __half* scales;
+  const __half* zeros;
+  const void* bias;
+  void* y;
+  int ldy;
+  int N;
+  int k_out;          // retained rows
+  ChanMap omap;       // ignored when rope.enabled (rows follow the half-head rule)
+  RopeDesc rope;
+};
+
+struct Params {
+  const void* x;
+  int ldx;
+  int dt;             // uniql_dtype
+  int M;
+  int K;              // stored input channels
+  int k_in;           // retained input channels
+  ChanMap imap;
+  int n_jobs;
+  JobDev job[kMaxJobs];
+  const int32_t* idx;   // [n_kv_heads][head_keep/2] original pair indices
+  const int32_t* pos;   // [M]
+  double inv_freq[kMaxHalfDim];
+};
+
+// ---------------------------------------------------------------- channel-map arithmetic
+// compact index -> stored index
+__host__ __device__ inline int map_compact_to_stored(const ChanMap& m, int j) {
+  int f = 0;
+  while (f + 1 < m.n_fam && j >= m.base[f + 1]) ++f;
+  int r = j - m.base[f];
+  int h = r / m.fam[f].keep;
+  return m.fam[f].start + h * m.fam[f].period + (r - h * m.fam[f].keep);
+}
+
+// stored index -> compact index, or -1 when the channel is pruned
+__host__ __device__ inline int map_stored_to_compact(const ChanMap& m, int k) {
+  for (int f = 0; f < m.n_fam; ++f) {
+    const Fam& a = m.fam[f];
+    if (k < a.start) return -1;
+    int r = k - a.start;
+    int h = r / a.period;
+    if (h >= a.count) continue;
+    int o = r - h * a.period;
+    return (o < a.keep) ? m.base[f] + h * a.keep + o : -1;
+  }
+  return -1;
+}
+
+// Output row `j` (compact order) of a rope job: head h, half s, position c inside the half.
+// Compact layout per head: [first-half survivors | second-half survivors] (Section 3.2).
+struct RopeRow { int stored; int head; int c; int is_hi; };
+__host__ __device__ inline RopeRow rope_row(const RopeDesc& r, int j) {
+  RopeRow o;
+  int half = r.head_keep >> 1;
+  o.head = j / r.head_keep;
+  int within = j - o.head * r.head_keep;
+  o.is_hi = within >= half;
+  o.c = within - (o.is_hi ? half : 0);
+  o.stored = o.head * r.head_dim + (o.is_hi ? (r.head_dim >> 1) : 0) + o.c;
+  return o;
+}
+
+// ---------------------------------------------------------------- dtype helpers
+template <typename T> struct DT;
+template <> struct DT<__half> {
+  using T2 = __half2;
+  static __device__ inline float to_f(__half v) { return __half2float(v); }
+  static __device__ inline __half from_f(float v) { return __float2half_rn(v); }
+  static __device__ inline float2 to_f2(__half2 v) { return __half22float2(v); }
+};
+template <> struct DT<__nv_bfloat16> {
+  using T2 = __nv_bfloat162;
+  static __device__ inline float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+  static __device__ inline __nv_bfloat16 from_f(float v) { return __float2bfloat16_rn(v); }
+  static __device__ inline float2 to_f2(__nv_bfloat162 v) { return __bfloat1622float2(v); }
+};
+
+// ---------------------------------------------------------------- rotary angle
+// cos / sin of pos * inv_freq.  The product reaches thousands of radians, where an fp32
+// product alone would already be off by ~1e-3 rad; it is formed and reduced modulo 2*pi in
+// fp64, then the fast fp32 intrinsics work on an argument in [-pi, pi].
+__device__ inline void rope_cos_sin(int pos, double inv_freq, float& c, float& s) {
+  double a = (double)pos * inv_freq;
+  const double two_pi = 6.283185307179586476925286766559;
+  const double inv_two_pi = 0.15915494309189533576888376337251;
+  a = fma(-rint(a * inv_two_pi), two_pi, a);
+  float af = (float)a;
+  c = __cosf(af);
+  s = __sinf(af);
+}
+
+// host launchers (one per kernel file) --------------------------------------------------
+struct LaunchCfg {
+  void* workspace;
+  size_t ws_bytes;
+  cudaStream_t stream;
+};
+int launch_generic(const Params& p, const LaunchCfg& cfg);
+int launch_decode(const Params& p, const LaunchCfg& cfg);
+int decode_supported(const Params& p);
+size_t decode_workspace_bytes(int M, int K, int N_total);
+int launch_prefill(const Params& p, const LaunchCfg& cfg);
+int prefill_supported(const Params& p);
+
+}  // namespace uniql

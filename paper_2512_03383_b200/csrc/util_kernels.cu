@@ -1,0 +1,91 @@
+// Storage helpers: nibble pack / unpack (bit-exact integer work) and a diagnostic full
+// de-quantisation.  Memory-bound element-wise kernels with 128-bit accesses where the
+// sizes allow.
+#include "common.cuh"
+
+namespace uniql {
+namespace {
+
+// two codes per byte, even input channel in the low nibble
+__global__ void pack_kernel(const uint8_t* __restrict__ codes, uint8_t* __restrict__ packed, int64_t n_bytes) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (; i < n_bytes; i += stride) {
+    uchar2 c = reinterpret_cast<const uchar2*>(codes)[i];
+    packed[i] = (uint8_t)((c.x & 15) | (c.y << 4));
+  }
+}
+
+__global__ void unpack_kernel(const uint8_t* __restrict__ packed, uint8_t* __restrict__ codes, int64_t n_bytes) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (; i < n_bytes; i += stride) {
+    uint8_t b = packed[i];
+    reinterpret_cast<uchar2*>(codes)[i] = make_uchar2(b & 15, b >> 4);
+  }
+}
+
+template <typename T>
+__global__ void dequant_kernel(const uint8_t* __restrict__ packed, const __half* __restrict__ scales,
+                               const __half* __restrict__ zeros, int64_t N, int64_t K, T* __restrict__ w) {
+  int64_t n_bytes = N * (K / 2);
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  int64_t G = K / kGroup;
+  for (; i < n_bytes; i += stride) {
+    int64_t n = i / (K / 2), b = i - n * (K / 2);
+    int64_t g = (2 * b) / kGroup;
+    float s = __half2float(scales[n * G + g]), z = __half2float(zeros[n * G + g]);
+    uint8_t byte = packed[i];
+    w[n * K + 2 * b] = DT<T>::from_f(s * ((float)(byte & 15) - z));
+    w[n * K + 2 * b + 1] = DT<T>::from_f(s * ((float)(byte >> 4) - z));
+  }
+}
+
+inline int grid_for(int64_t n, int threads) {
+  int64_t b = (n + threads - 1) / threads;
+  if (b < 1) b = 1;
+  if (b > 148 * 16) b = 148 * 16;
+  return (int)b;
+}
+
+}  // namespace
+}  // namespace uniql
+
+using namespace uniql;
+
+extern "C" int uniql_pack_u4(const uint8_t* codes, int64_t N, int64_t K, uint8_t* packed, void* stream) {
+  if (!codes || !packed) return UNIQL_ERR_NULL;
+  if (N < 0 || K < 0 || (K & 1)) return UNIQL_ERR_SHAPE;
+  if (((uintptr_t)codes) & 1) return UNIQL_ERR_ALIGN;
+  int64_t nb = N * (K / 2);
+  if (nb == 0) return UNIQL_OK;
+  pack_kernel<<<grid_for(nb, 256), 256, 0, (cudaStream_t)stream>>>(codes, packed, nb);
+  return cudaGetLastError() == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
+}
+
+extern "C" int uniql_unpack_u4(const uint8_t* packed, int64_t N, int64_t K, uint8_t* codes, void* stream) {
+  if (!codes || !packed) return UNIQL_ERR_NULL;
+  if (N < 0 || K < 0 || (K & 1)) return UNIQL_ERR_SHAPE;
+  if (((uintptr_t)codes) & 1) return UNIQL_ERR_ALIGN;
+  int64_t nb = N * (K / 2);
+  if (nb == 0) return UNIQL_OK;
+  unpack_kernel<<<grid_for(nb, 256), 256, 0, (cudaStream_t)stream>>>(packed, codes, nb);
+  return cudaGetLastError() == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
+}
+
+extern "C" int uniql_dequant(const uint8_t* packed, const void* scales, const void* zeros, int64_t N,
+                             int64_t K, int dt, void* w, void* stream) {
+  if (!packed || !scales || !zeros || !w) return UNIQL_ERR_NULL;
+  if (N < 0 || K < 0 || (K % kGroup)) return UNIQL_ERR_SHAPE;
+  if (dt != UNIQL_F16 && dt != UNIQL_BF16) return UNIQL_ERR_DTYPE;
+  int64_t nb = N * (K / 2);
+  if (nb == 0) return UNIQL_OK;
+  if (dt == UNIQL_F16)
+    dequant_kernel<__half><<<grid_for(nb, 256), 256, 0, (cudaStream_t)stream>>>(
+        packed, (const __half*)scales, (const __half*)zeros, N, K, (__half*)w);
+  else
+    dequant_kernel<__nv_bfloat16><<<grid_for(nb, 256), 256, 0, (cudaStream_t)stream>>>(
+        packed, (const __half*)scales, (const __half*)zeros, N, K, (__nv_bfloat16*)w);
+  return cudaGetLastError() == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
+}

@@ -1,0 +1,299 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element,
+on the same seeded inputs.  Decode (M <= 16) and generic kernels."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import check_output, dev_weight, dev_x
+from paper_2512_03383_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TIGHT = 5e-5     # decode / generic kernels: exact products, fp32 accumulation
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2512_03383_b200 import binding
+    return binding
+
+
+@pytest.fixture(autouse=True)
+def _reset_path(B):
+    yield
+    B.set_path(B.PATH_AUTO)
+    for k in ("UNIQL_DECODE_WK", "UNIQL_DECODE_GS"):
+        os.environ.pop(k, None)
+
+
+def run_ex(B, qw, dw, x32, dtype, in_map, k_in, out_map, k_out, bias=None, ldx_pad=0, ldy_pad=0, workspace=None):
+    packed, wp, ws, wz = dw
+    M = x32.shape[0]
+    n_in = synth.map_size(in_map) if in_map else k_in
+    n_out = synth.map_size(out_map) if out_map else k_out
+    xd = torch.full((M, n_in + ldx_pad), 7.0, device="cuda", dtype=torch.float16 if dtype == "f16" else torch.bfloat16)
+    xd[:, :n_in] = dev_x(x32, dtype)
+    y = torch.full((M, n_out + ldy_pad), -77.0, device="cuda", dtype=xd.dtype)
+    bd = None if bias is None else dev_x(bias.reshape(1, -1), dtype).reshape(-1)
+    B.qlinear_ex(xd, xd.stride(0), wp, ws, wz, bd, M, qw.K, qw.N, in_map, k_in, out_map, k_out, y, y.stride(0),
+                 workspace=workspace)
+    torch.cuda.synchronize()
+    if ldy_pad:
+        assert (y[:, n_out:] == -77.0).all(), "wrote outside the output columns"
+    O = oracle.expand_map(out_map) if out_map else oracle.leading(k_out)
+    I = oracle.expand_map(in_map) if in_map else oracle.leading(k_in)
+    ref = oracle.qlinear(x32, packed, qw.scales, qw.zeros, O, I, bias=bias)
+    return y[:, :n_out], ref
+
+
+# ---------------------------------------------------------------- storage helpers, bit exact
+def test_pack_unpack_dequant_bit_exact(B):
+    rng = np.random.default_rng(21)
+    qw = synth.draw_qweight(rng, 300, 384)
+    packed_ref = oracle.pack_u4(qw.codes)
+    codes_d = torch.from_numpy(qw.codes).cuda()
+    packed_d = torch.empty((300, 192), dtype=torch.uint8, device="cuda")
+    B.pack_u4(codes_d, packed_d)
+    assert np.array_equal(packed_d.cpu().numpy(), packed_ref)
+    allb = torch.arange(256, dtype=torch.uint8, device="cuda").reshape(2, 128).contiguous()
+    out = torch.empty((2, 256), dtype=torch.uint8, device="cuda")
+    B.unpack_u4(allb, out)
+    assert np.array_equal(out.cpu().numpy(), oracle.unpack_u4(allb.cpu().numpy()))
+    back = torch.empty_like(codes_d)
+    B.unpack_u4(packed_d, back)
+    assert torch.equal(back, codes_d)
+    w = torch.empty((300, 384), dtype=torch.float16, device="cuda")
+    B.dequant(packed_d, torch.from_numpy(qw.scales).cuda(), torch.from_numpy(qw.zeros).cuda(), w)
+    ref = oracle.dequant(packed_ref, qw.scales, qw.zeros).astype(np.float16)      # integer zero-points: one rounding
+    assert np.array_equal(w.cpu().numpy().view(np.uint16), ref.view(np.uint16))
+
+
+# ---------------------------------------------------------------- configuration 1 (single linear, seed 0)
+@pytest.fixture(scope="module")
+def config1():
+    rng = np.random.default_rng(0)
+    qw = synth.draw_qweight(rng, 2048, 2048, std=0.02)
+    x = synth.draw_x(rng, 1, 2048, "f16")
+    return qw, dev_weight(qw), x
+
+
+@pytest.mark.parametrize("rate", [1.0, 0.85])
+@pytest.mark.parametrize("path", ["auto", "generic", "decode"])
+def test_config1_simple_api(B, config1, rate, path):
+    qw, dw, x = config1
+    B.set_path({"auto": B.PATH_AUTO, "generic": B.PATH_GENERIC, "decode": B.PATH_DECODE}[path])
+    k = synth.keep_count(rate, 2048)
+    packed, wp, ws, wz = dw
+    xd = dev_x(x[:, :k], "f16")
+    y = torch.zeros((1, k), dtype=torch.float16, device="cuda")
+    B.qlinear(xd, wp, ws, wz, 1, 2048, 2048, k, k, y)
+    torch.cuda.synchronize()
+    ref = oracle.qlinear(x[:, :k], packed, qw.scales, qw.zeros, oracle.leading(k), oracle.leading(k))
+    check_output(y, ref, "f16", TIGHT, "config1 %s keep %.2f" % (path, rate))
+    # the stored oracle samples (tests/golden) agree too
+    gold = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", "config1_oracle.txt")) as f:
+        for ln in f:
+            if ln.startswith("#") or not ln.strip():
+                continue
+            r, kk, j, v = ln.split()
+            if float(r) == rate:
+                gold[int(j)] = float.fromhex(v)
+    for j, v in gold.items():
+        assert abs(float(y[0, j]) - v) <= TIGHT * np.abs(ref).max() + 2.0 ** -11 * abs(v) * 1.01
+
+
+# ---------------------------------------------------------------- M sweep, ragged sizes, both dtypes
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("M", [1, 2, 3, 8, 9, 16, 17, 40])
+def test_m_sweep(B, M, dtype):
+    rng = np.random.default_rng(100 + M)
+    qw = synth.draw_qweight(rng, 200, 640)
+    dw = dev_weight(qw)
+    for (k_in, k_out) in [(640, 200), (548, 172), (8, 4), (132, 17)]:
+        x = synth.draw_x(rng, M, k_in, dtype)
+        y, ref = run_ex(B, qw, dw, x, dtype, None, k_in, None, k_out, ldy_pad=3)
+        check_output(y, ref, dtype, TIGHT, "M=%d %s k=(%d,%d)" % (M, dtype, k_in, k_out))
+
+
+@pytest.mark.parametrize("wk,gs", [(4, 1), (4, 2), (2, 2), (1, 1), (1, 4), (2, 8), (4, 16), (1, 16)])
+@pytest.mark.parametrize("M", [1, 5, 16])
+def test_decode_split_configs(B, wk, gs, M):
+    """Every block shape / split-K factor of the decode kernel gives the same answer."""
+    os.environ["UNIQL_DECODE_WK"], os.environ["UNIQL_DECODE_GS"] = str(wk), str(gs)
+    B.set_path(B.PATH_DECODE)
+    rng = np.random.default_rng(7)
+    qw = synth.draw_qweight(rng, 144, 1536)
+    dw = dev_weight(qw)
+    bias = synth.to_dtype_values(rng.standard_normal(144).astype(np.float32), "f16")
+    for (k_in, k_out) in [(1536, 144), (1300, 100)]:
+        x = synth.draw_x(rng, M, k_in, "f16")
+        y, ref = run_ex(B, qw, dw, x, "f16", None, k_in, None, k_out, bias=bias)
+        check_output(y, ref, "f16", TIGHT, "wk=%d gs=%d M=%d" % (wk, gs, M))
+        y2, _ = run_ex(B, qw, dw, x, "f16", None, k_in, None, k_out, bias=bias)
+        assert torch.equal(y, y2), "run-to-run results differ"
+
+
+def test_caller_workspace(B):
+    os.environ["UNIQL_DECODE_WK"], os.environ["UNIQL_DECODE_GS"] = "1", "2"
+    rng = np.random.default_rng(8)
+    qw = synth.draw_qweight(rng, 96, 1024)
+    dw = dev_weight(qw)
+    nbytes = B.workspace_bytes(4, 1024, 96)
+    assert nbytes > 0
+    ws = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+    off = (-ws.data_ptr()) % 256
+    ws = ws[off:off + nbytes]
+    B.workspace_init(ws)
+    x = synth.draw_x(rng, 4, 1024, "f16")
+    for _ in range(2):      # the counters must be back at zero for the second call
+        y, ref = run_ex(B, qw, dw, x, "f16", None, 1024, None, 96, workspace=ws)
+        check_output(y, ref, "f16", TIGHT, "caller workspace")
+
+
+# ---------------------------------------------------------------- channel maps (per-head pruning)
+@pytest.mark.parametrize("M", [1, 6, 16, 33])
+def test_per_head_maps(B, M):
+    rng = np.random.default_rng(30 + M)
+    qw = synth.draw_qweight(rng, 512, 1024)          # 4 heads of 128 on both sides
+    dw = dev_weight(qw)
+    for keep in (128, 108, 96, 84):
+        out_map = synth.map_per_head(4, 128, keep)                      # V-projection rows
+        in_map = synth.map_per_head(8, 128, keep)                       # o_proj columns
+        x = synth.draw_x(rng, M, synth.map_size(in_map), "f16")
+        y, ref = run_ex(B, qw, dw, x, "f16", in_map, 0, out_map, 0, ldx_pad=5)
+        check_output(y, ref, "f16", TIGHT, "per-head keep %d M=%d" % (keep, M))
+
+
+@pytest.mark.parametrize("M", [1, 16])
+def test_mamba_shaped_maps(B, M):
+    """in_proj rows z|x|B|C|dt with z, x pruned per SSM head; out_proj columns pruned per head."""
+    rng = np.random.default_rng(40)
+    nheads, headdim, d_state = 8, 64, 128
+    d_inner = nheads * headdim
+    rows = 2 * d_inner + 2 * d_state + nheads
+    qin = synth.draw_qweight(rng, rows, 256)
+    qout = synth.draw_qweight(rng, 256, d_inner)
+    din, dout = dev_weight(qin), dev_weight(qout)
+    for keep in (64, 56, 48):
+        om = synth.map_mamba_in_proj(d_inner, headdim, keep, d_state, 1, nheads)
+        x = synth.draw_x(rng, M, 256, "f16")
+        y, ref = run_ex(B, qin, din, x, "f16", None, 256, om, 0)
+        check_output(y, ref, "f16", TIGHT, "mamba in_proj keep %d" % keep)
+        im = synth.map_per_head(nheads, headdim, keep)
+        x2 = synth.draw_x(rng, M, synth.map_size(im), "f16")
+        y2, ref2 = run_ex(B, qout, dout, x2, "f16", im, 0, None, 256)
+        check_output(y2, ref2, "f16", TIGHT, "mamba out_proj keep %d" % keep)
+
+
+def test_noninteger_zero_points_and_symmetric(B):
+    rng = np.random.default_rng(50)
+    qw = synth.draw_qweight(rng, 64, 512, symmetric=True)
+    dw = dev_weight(qw)
+    x = synth.draw_x(rng, 2, 512, "f16")
+    y, ref = run_ex(B, qw, dw, x, "f16", None, 512, None, 64)
+    check_output(y, ref, "f16", TIGHT, "symmetric")
+    qw.zeros[:] = (qw.zeros.astype(np.float32) + rng.uniform(-0.5, 0.5, qw.zeros.shape)).astype(np.float16)
+    dw = dev_weight(qw)
+    for path in (B.PATH_DECODE, B.PATH_GENERIC):
+        B.set_path(path)
+        y, ref = run_ex(B, qw, dw, x, "f16", None, 512, None, 64)
+        check_output(y, ref, "f16", TIGHT, "fractional zero-points")
+
+
+# ---------------------------------------------------------------- gate|up in one launch
+def test_multi_job(B):
+    rng = np.random.default_rng(60)
+    gate, up = synth.draw_qweight(rng, 352, 512), synth.draw_qweight(rng, 352, 512)
+    dg, du = dev_weight(gate), dev_weight(up)
+    for M in (1, 16, 20):
+        x = synth.draw_x(rng, M, 512, "f16")
+        xd = dev_x(x, "f16")
+        k = 300
+        yg = torch.zeros((M, k), dtype=torch.float16, device="cuda")
+        yu = torch.zeros((M, k), dtype=torch.float16, device="cuda")
+        jobs = [dict(packed_w=dg[1], scales=dg[2], zeros=dg[3], N=352, k_out=k, y=yg, ldy=k),
+                dict(packed_w=du[1], scales=du[2], zeros=du[3], N=352, k_out=k, y=yu, ldy=k)]
+        B.qlinear_multi(xd, 512, M, 512, None, 512, jobs)
+        torch.cuda.synchronize()
+        for (q, d, y) in ((gate, dg, yg), (up, du, yu)):
+            ref = oracle.qlinear(x, d[0], q.scales, q.zeros, oracle.leading(k), oracle.leading(512))
+            check_output(y, ref, "f16", TIGHT, "multi M=%d" % M)
+
+
+# ---------------------------------------------------------------- fused Q/K projection + pruned RoPE
+def run_rope(B, rng, M, K, Hq, Hkv, D, keep, theta, dtype, idx_kind="perm", bias=False, inv_freq=None):
+    wq, wk = synth.draw_qweight(rng, Hq * D, K), synth.draw_qweight(rng, Hkv * D, K)
+    dq, dk = dev_weight(wq), dev_weight(wk)
+    x = synth.draw_x(rng, M, K, dtype)
+    pos = synth.draw_pos(rng, M)
+    idx = synth.draw_idx(rng, Hkv, D, keep, kind=idx_kind)
+    bq = bk = None
+    if bias:
+        bq = synth.to_dtype_values(rng.standard_normal(Hq * D).astype(np.float32), dtype)
+        bk = synth.to_dtype_values(rng.standard_normal(Hkv * D).astype(np.float32), dtype)
+    xd = dev_x(x, dtype)
+    tdt = xd.dtype
+    qo = torch.zeros((M, Hq * keep), dtype=tdt, device="cuda")
+    ko = torch.zeros((M, Hkv * keep), dtype=tdt, device="cuda")
+    B.qk_rope_proj(xd, K, dq[1], dq[2], dq[3], dk[1], dk[2], dk[3],
+                   None if bq is None else dev_x(bq.reshape(1, -1), dtype).reshape(-1),
+                   None if bk is None else dev_x(bk.reshape(1, -1), dtype).reshape(-1),
+                   M, K, Hq, Hkv, D, keep, torch.from_numpy(idx).cuda(), torch.from_numpy(pos).cuda(), theta,
+                   inv_freq, qo, Hq * keep, ko, Hkv * keep)
+    torch.cuda.synchronize()
+    out = []
+    for (w, d, nh, b, g) in ((wq, dq, Hq, bq, qo), (wk, dk, Hkv, bk, ko)):
+        O = oracle.expand_map(oracle.qk_halfhead_map(nh, D, keep))
+        acc = oracle.qlinear(x, d[0], w.scales, w.zeros, O, oracle.leading(K), bias=b)
+        ref = oracle.rope(acc, nh, Hkv, D, keep, idx, pos, theta, inv_freq=inv_freq)
+        out.append((g, ref))
+    return out
+
+
+@pytest.mark.parametrize("path", ["auto", "generic"])
+@pytest.mark.parametrize("M", [1, 5, 16, 24])
+@pytest.mark.parametrize("keep", [128, 108, 96, 84])
+def test_qk_rope_small(B, path, M, keep):
+    B.set_path(B.PATH_AUTO if path == "auto" else B.PATH_GENERIC)
+    rng = np.random.default_rng(70 + keep + M)
+    kind = {128: "identity", 108: "perm", 96: "reversed", 84: "perm"}[keep]
+    for (g, ref) in run_rope(B, rng, M, 256, 6, 2, 128, keep, 500000.0, "f16", idx_kind=kind, bias=(keep == 96)):
+        check_output(g, ref, "f16", TIGHT, "rope keep %d M=%d" % (keep, M))
+
+
+def test_qk_rope_bf16_table_and_split(B):
+    rng = np.random.default_rng(71)
+    invf = (1e6 ** (-np.arange(64) / 64.0)) * 0.5          # a caller table (scaled-RoPE variants)
+    os.environ["UNIQL_DECODE_WK"], os.environ["UNIQL_DECODE_GS"] = "2", "1"
+    for (g, ref) in run_rope(B, rng, 3, 512, 4, 4, 128, 108, 1e6, "bf16", inv_freq=invf):
+        check_output(g, ref, "bf16", TIGHT, "rope bf16 table")
+
+
+@pytest.mark.parametrize("M", [1, 16])
+def test_qk_rope_llama_shape(B, M):
+    """Configuration 3 at full layer size: 32 Q / 8 KV heads of 128, hidden 4096, theta 5e5."""
+    rng = np.random.default_rng(3)
+    for keep in (128, 84):
+        for (g, ref) in run_rope(B, rng, M, 4096, 32, 8, 128, keep, 500000.0, "f16"):
+            check_output(g, ref, "f16", TIGHT, "llama q/k keep %d M=%d" % (keep, M))
+
+
+# ---------------------------------------------------------------- configuration 2 at full size (sampled rows of the MLP)
+@pytest.mark.parametrize("M", [1, 16])
+def test_llama_mlp_full_size(B, M):
+    rng = np.random.default_rng(2)
+    gate = synth.random_qweight_fast(rng, 14336, 4096)
+    down = synth.random_qweight_fast(rng, 4096, 14336)
+    dg, dd = dev_weight(gate), dev_weight(down)
+    for rate in (1.0, 0.65):
+        k = synth.keep_count(rate, 14336)
+        x = synth.draw_x(rng, M, 4096, "f16")
+        y, ref = run_ex(B, gate, dg, x, "f16", None, 4096, None, k)
+        check_output(y, ref, "f16", TIGHT, "gate keep %.2f" % rate)
+        h = synth.draw_x(rng, M, k, "f16")
+        y, ref = run_ex(B, down, dd, h, "f16", None, k, None, 4096)
+        check_output(y, ref, "f16", TIGHT, "down keep %.2f" % rate)
