@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the UniQL hot path on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference] [--detail]
+
+Workload (N = 1 and every rank at N > 1): the Llama-3-8B-shaped SwiGLU MLP in decode, the
+configuration the headline metric is quoted on -- hidden 4096, intermediate 14336, uint4 g=128
+weights, batch M = 1, intermediate channels truncated at keep rates 1.0 / 0.85 / 0.75 / 0.65.
+One step = for every keep rate one gate|up launch (two matrices, one launch) and one down launch,
+i.e. the whole decode path (truncation, unpack, de-quantise, contraction) over one batch.
+metric = effective weight GB/s: 0.53125 bytes per RETAINED weight (codes + fp16 scale and zero per
+128) divided by device time.  Each launch reads a different one of four weight copies (375 MB in
+rotation, L2 is 126 MB), so every byte comes from HBM.  Synthetic seeded inputs stand in for the
+paper's checkpoints.  The step is captured in a CUDA graph and replayed, timed with CUDA events.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+HIDDEN, INTER = 4096, 14336
+KEEP_RATES = (1.0, 0.85, 0.75, 0.65)
+BYTES_PER_WEIGHT = 0.5 + 4.0 / 128.0
+N_COPIES = 4
+METRIC = "qlinear effective weight GB/s, Llama-3-8B MLP decode M=1, keep rates 1.0/0.85/0.75/0.65"
+
+
+def keep_count(rate, D):
+    return int(4 * round(rate * D / 4.0))
+
+
+def step_bytes(rates=KEEP_RATES):
+    return sum(BYTES_PER_WEIGHT * 3 * HIDDEN * keep_count(r, INTER) for r in rates)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), float(d["bf16_tflops"]), "measured"
+    except Exception:
+        return 6650.0, 1590.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons while the GPU is under load."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.rows.append((time.time(), ln.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for (t, ln) in self.rows:
+            if t < t0 - 0.05 or t > t1 + 0.15:
+                continue
+            f = [c.strip() for c in ln.split(",")]
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except Exception:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------- CPU oracle leg
+class OracleStep:
+    """The oracle as it stands, on the host cores: one whole MLP step at M=1 (all four keep rates)."""
+
+    def __init__(self):
+        import oracle
+        from paper_2512_03383_b200 import synth
+        self.oracle = oracle
+        rng = np.random.default_rng(0)
+        self.mats = [synth.random_qweight_fast(rng, INTER, HIDDEN), synth.random_qweight_fast(rng, INTER, HIDDEN),
+                     synth.random_qweight_fast(rng, HIDDEN, INTER)]
+        self.pk = [oracle.pack_u4(w.codes) for w in self.mats]
+        self.x = synth.draw_x(rng, 1, HIDDEN, "f16")
+        self.h = synth.draw_x(rng, 1, INTER, "f16")
+        oracle.qlinear(self.x, self.pk[0][:64], self.mats[0].scales[:64], self.mats[0].zeros[:64],
+                       oracle.leading(64), oracle.leading(HIDDEN))
+
+    def step(self):
+        o, (gate, up, down), pk = self.oracle, self.mats, self.pk
+        t0 = time.time()
+        for r in KEEP_RATES:
+            k = keep_count(r, INTER)
+            o.qlinear(self.x, pk[0], gate.scales, gate.zeros, o.leading(k), o.leading(HIDDEN))
+            o.qlinear(self.x, pk[1], up.scales, up.zeros, o.leading(k), o.leading(HIDDEN))
+            o.qlinear(self.h[:, :k], pk[2], down.scales, down.zeros, o.leading(HIDDEN), o.leading(k))
+        return time.time() - t0
+
+    def describe(self, sec, steps):
+        return {"value": step_bytes() / sec / 1e9, "unit": "GB/s", "cores": self.oracle.threads(), "kind": "oracle",
+                "sample": "%d whole steps (gate, up, down at 4 keep rates, M=1; the full workload), "
+                          "%.3f s per step" % (steps, sec)}
+
+
+def oracle_leg(budget_s):
+    """Bounded CPU-baseline sample: whole steps until `budget_s` seconds have passed; best step counts."""
+    o = OracleStep()
+    t0, per = time.time(), []
+    while True:
+        per.append(o.step())
+        if time.time() - t0 > budget_s:
+            break
+    return o.describe(min(per), len(per))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    o = OracleStep()
+    for _ in range(args.warmup):
+        o.step()
+    per = [o.step() for _ in range(args.steps)]
+    sec = sum(per) / len(per)
+    val = step_bytes() / sec / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "llama3-8b-mlp-decode-M1 (BASELINE configs[1])", "keep_rates": list(KEEP_RATES),
+                       "M": 1},
+            "cpu_baseline": o.describe(sec, args.steps),
+            "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+# --------------------------------------------------------------------------------------- GPU leg
+class MlpDecode:
+    """Device-resident weights (N_COPIES rotating copies) and the launches of one step."""
+
+    def __init__(self, B, torch, M, seed=0):
+        from paper_2512_03383_b200 import synth
+        self.B, self.torch, self.M = B, torch, M
+        rng = np.random.default_rng(seed)
+        mats = [synth.random_qweight_fast(rng, INTER, HIDDEN), synth.random_qweight_fast(rng, INTER, HIDDEN),
+                synth.random_qweight_fast(rng, HIDDEN, INTER)]
+        codes_d = [torch.from_numpy(m.codes).cuda() for m in mats]
+        self.copies = []
+        for c in range(N_COPIES):
+            cp = []
+            for m, cd in zip(mats, codes_d):
+                packed = torch.empty((m.N, m.K // 2), dtype=torch.uint8, device="cuda")
+                B.pack_u4(cd, packed)                   # the library's own packer
+                cp.append((packed, torch.from_numpy(m.scales).cuda().clone(), torch.from_numpy(m.zeros).cuda().clone()))
+            self.copies.append(cp)
+        del codes_d
+        self.x_host = torch.from_numpy(synth.draw_x(rng, M, HIDDEN, "f16")).half().pin_memory()
+        self.h_host = torch.from_numpy(synth.draw_x(rng, M, INTER, "f16", outlier_frac=0.0)).half().pin_memory()
+        self.x = self.x_host.cuda()
+        self.h = self.h_host.cuda()
+        self.yg = torch.zeros((M, INTER), dtype=torch.float16, device="cuda")
+        self.yu = torch.zeros((M, INTER), dtype=torch.float16, device="cuda")
+        self.yd = torch.zeros((len(KEEP_RATES), M, HIDDEN), dtype=torch.float16, device="cuda")
+        self.yg_host = torch.zeros((M, INTER), dtype=torch.float16).pin_memory()
+        self.yu_host = torch.zeros((M, INTER), dtype=torch.float16).pin_memory()
+        self.yd_host = torch.zeros((len(KEEP_RATES), M, HIDDEN), dtype=torch.float16).pin_memory()
+        self.launches_per_step = 2 * len(KEEP_RATES)
+        self.turn = 0
+
+    def step(self, e2e=False):
+        B, M = self.B, self.M
+        h2d = d2h = 0
+        for i, r in enumerate(KEEP_RATES):
+            k = keep_count(r, INTER)
+            g, u, d = self.copies[self.turn % N_COPIES]
+            self.turn += 1
+            if e2e:
+                self.x.copy_(self.x_host, non_blocking=True)
+                self.h.copy_(self.h_host, non_blocking=True)
+                h2d += self.x_host.numel() * 2 + self.h_host.numel() * 2
+            jobs = [dict(packed_w=g[0], scales=g[1], zeros=g[2], N=INTER, k_out=k, y=self.yg, ldy=INTER),
+                    dict(packed_w=u[0], scales=u[1], zeros=u[2], N=INTER, k_out=k, y=self.yu, ldy=INTER)]
+            B.qlinear_multi(self.x, HIDDEN, M, HIDDEN, None, HIDDEN, jobs)
+            B.qlinear_ex(self.h, INTER, d[0], d[1], d[2], None, M, INTER, HIDDEN, None, k, None, HIDDEN,
+                         self.yd[i], HIDDEN)
+            if e2e:
+                self.yg_host.copy_(self.yg, non_blocking=True)
+                self.yu_host.copy_(self.yu, non_blocking=True)
+                self.yd_host[i].copy_(self.yd[i], non_blocking=True)
+                d2h += self.yg.numel() * 2 + self.yu.numel() * 2 + self.yd[i].numel() * 2
+        return h2d, d2h
+
+
+def capture(torch, fn):
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        fn()                                     # warm: library workspace, function attributes
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    with torch.cuda.graph(g, stream=s):
+        out = fn()
+    return g, out
+
+
+def time_graph(torch, g, steps, barrier=None):
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    a.record()
+    for _ in range(steps):
+        g.replay()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) * 1e-3
+
+
+def detail_tables(B, torch, steps):
+    """Extra, reported next to the headline: decode at M = 4 and 16 and (when available) prefill."""
+    out = {}
+    hbm, tf, which = measured_peaks()
+    for M in (1, 4, 16):
+        w = MlpDecode(B, torch, M)
+        rows = {}
+        for r in KEEP_RATES:
+            k = keep_count(r, INTER)
+
+            def one(r=r, k=k, w=w):
+                for _ in range(N_COPIES):
+                    g, u, d = w.copies[w.turn % N_COPIES]
+                    w.turn += 1
+                    jobs = [dict(packed_w=g[0], scales=g[1], zeros=g[2], N=INTER, k_out=k, y=w.yg, ldy=INTER),
+                            dict(packed_w=u[0], scales=u[1], zeros=u[2], N=INTER, k_out=k, y=w.yu, ldy=INTER)]
+                    B.qlinear_multi(w.x, HIDDEN, M, HIDDEN, None, HIDDEN, jobs)
+                    B.qlinear_ex(w.h, INTER, d[0], d[1], d[2], None, M, INTER, HIDDEN, None, k, None, HIDDEN,
+                                 w.yd[0], HIDDEN)
+            g, _ = capture(torch, one)
+            for _ in range(5):
+                g.replay()
+            sec = time_graph(torch, g, steps) / (steps * N_COPIES)
+            gbs = BYTES_PER_WEIGHT * 3 * HIDDEN * k / sec / 1e9
+            rows["%.2f" % r] = {"us_per_mlp": round(sec * 1e6, 2), "GBps": round(gbs, 1),
+                                "frac_hbm_%s" % which: round(gbs / hbm, 3), "tokens_per_s_mlp": round(M / sec, 1)}
+        out["decode_M%d" % M] = rows
+        del w
+        torch.cuda.empty_cache()
+    return out
+
+
+def run_ours(args):
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    from paper_2512_03383_b200 import binding as B
+
+    work = MlpDecode(B, torch, 1)
+    graph, _ = capture(torch, work.step)
+    graph_e2e, (h2d, d2h) = capture(torch, lambda: work.step(e2e=True))
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    t_load = time.time()
+    for _ in range(max(args.warmup, 3)):
+        graph.replay()
+    # keep the device under load for a moment so that the sampled clocks are the clocks of the timed region
+    torch.cuda.synchronize()
+    while time.time() - t_load < 0.6:
+        for _ in range(50):
+            graph.replay()
+        torch.cuda.synchronize()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    sec = time_graph(torch, graph, args.steps, barrier)
+    barrier()
+    for _ in range(3):
+        graph_e2e.replay()
+    sec_e2e = time_graph(torch, graph_e2e, args.steps, barrier)
+    t_end = time.time()
+    clocks = sampler.stop(t_load, t_end) if rank == 0 else None
+
+    if dist is not None:
+        t = torch.tensor([sec, sec_e2e], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        sec, sec_e2e = float(t[0]), float(t[1])
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    hbm, tf, which = measured_peaks()
+    total_bytes = step_bytes() * args.steps * world
+    value = total_bytes / sec / 1e9
+    launches = work.launches_per_step * args.steps
+    per_launch_bytes = step_bytes() / work.launches_per_step
+    per_launch_sec = sec / launches
+    achieved = per_launch_bytes / per_launch_sec / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": sec / args.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+        "config": {"workload": "llama3-8b-mlp-decode-M1 (BASELINE configs[1])", "hidden": HIDDEN,
+                   "intermediate": INTER, "keep_rates": list(KEEP_RATES), "M": 1,
+                   "l2": "4 rotating weight copies (375 MB) > 126 MB L2", "parallelism": "replicas x%d" % world,
+                   "timing": "CUDA graph of one step replayed, CUDA events"},
+        "tokens_per_s_mlp": args.steps * len(KEEP_RATES) * world / sec,
+        "gpu_launches": launches,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s", "frac": achieved / hbm,
+                     "traffic": DRAM_TRAFFIC_PER_LAUNCH, "peak_source": which,
+                     "kernel": "decode_kernel<half,1>", "algorithmic_bytes_per_launch": per_launch_bytes,
+                     "frac_of_nominal_8TBs": achieved / 8000.0},
+        "e2e": {"value": step_bytes() * args.steps * world / sec_e2e / 1e9, "unit": "GB/s",
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "note": "activations copied from / results to pinned host memory every launch; weights resident"},
+    }
+    if world == 1:
+        line["cpu_baseline"] = oracle_leg(3.0)
+        if args.detail:
+            line["detail"] = detail_tables(B, torch, max(20, min(args.steps, 200)))
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+# DRAM bytes (read + write) per decode launch from the ncu capture summarised under profiles/; None until taken.
+DRAM_TRAFFIC_PER_LAUNCH = None
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--detail", action="store_true", help="also report M=4/16 and per-keep-rate tables")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps > 50:
+            args.steps, args.warmup = 5, 1       # the oracle runs ~1 s per step
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -123,6 +123,8 @@ def test_m_sweep(B, M, dtype):
 @pytest.mark.parametrize("M", [1, 5, 16])
 def test_decode_split_configs(B, wk, gs, M):
     """Every block shape / split-K factor of the decode kernel gives the same answer."""
+    if wk * gs * (M if M <= 8 else 16) * 260 > 64 * 1024:
+        pytest.skip("staged activations of this forced shape exceed the kernel's shared-memory budget")
     os.environ["UNIQL_DECODE_WK"], os.environ["UNIQL_DECODE_GS"] = str(wk), str(gs)
     B.set_path(B.PATH_DECODE)
     rng = np.random.default_rng(7)
