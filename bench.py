@@ -367,6 +367,31 @@ def run_ours(args):
     return 0
 
 
+def run_case(args):
+    """A few plain (un-graphed) launches of one kernel on a small set-up, for ncu captures:
+    --case decode-gateup | decode-down, with --M and --keep."""
+    import torch
+    from paper_2512_03383_b200 import binding as B
+    torch.cuda.set_device(0)
+    w = MlpDecode(B, torch, args.M)
+    k = keep_count(args.keep, INTER)
+    for _ in range(args.launches):
+        g, u, d = w.copies[w.turn % N_COPIES]
+        w.turn += 1
+        if args.case == "decode-gateup":
+            jobs = [dict(packed_w=g[0], scales=g[1], zeros=g[2], N=INTER, k_out=k, y=w.yg, ldy=INTER),
+                    dict(packed_w=u[0], scales=u[1], zeros=u[2], N=INTER, k_out=k, y=w.yu, ldy=INTER)]
+            B.qlinear_multi(w.x, HIDDEN, args.M, HIDDEN, None, HIDDEN, jobs)
+        elif args.case == "decode-down":
+            B.qlinear_ex(w.h, INTER, d[0], d[1], d[2], None, args.M, INTER, HIDDEN, None, k, None, HIDDEN,
+                         w.yd[0], HIDDEN)
+        else:
+            raise SystemExit("unknown case " + args.case)
+    torch.cuda.synchronize()
+    print("case %s M=%d keep=%.2f: %d launches done" % (args.case, args.M, args.keep, args.launches))
+    return 0
+
+
 # DRAM bytes (read + write) per decode launch from the ncu capture summarised under profiles/; None until taken.
 DRAM_TRAFFIC_PER_LAUNCH = None
 
@@ -378,7 +403,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--detail", action="store_true", help="also report M=4/16 and per-keep-rate tables")
+    ap.add_argument("--case", default=None, help="run a few plain launches of one kernel (for ncu)")
+    ap.add_argument("--M", type=int, default=1)
+    ap.add_argument("--keep", type=float, default=1.0)
+    ap.add_argument("--launches", type=int, default=4)
     args = ap.parse_args()
+    if args.case:
+        return run_case(args)
     if args.impl == "reference":
         if args.steps > 50:
             args.steps, args.warmup = 5, 1       # the oracle runs ~1 s per step

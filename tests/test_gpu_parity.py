@@ -25,7 +25,7 @@ def B():
 def _reset_path(B):
     yield
     B.set_path(B.PATH_AUTO)
-    for k in ("UNIQL_DECODE_WK", "UNIQL_DECODE_GS"):
+    for k in ("UNIQL_DECODE_TPW", "UNIQL_DECODE_GS"):
         os.environ.pop(k, None)
 
 
@@ -119,13 +119,11 @@ def test_m_sweep(B, M, dtype):
         check_output(y, ref, dtype, TIGHT, "M=%d %s k=(%d,%d)" % (M, dtype, k_in, k_out))
 
 
-@pytest.mark.parametrize("wk,gs", [(4, 1), (4, 2), (2, 2), (1, 1), (1, 4), (2, 8), (4, 16), (1, 16)])
+@pytest.mark.parametrize("gs,tpw", [(2, 1), (4, 1), (8, 1), (2, 3), (4, 2), (8, 4), (8, 64)])
 @pytest.mark.parametrize("M", [1, 5, 16])
-def test_decode_split_configs(B, wk, gs, M):
+def test_decode_split_configs(B, gs, tpw, M):
     """Every block shape / split-K factor of the decode kernel gives the same answer."""
-    if wk * gs * (M if M <= 8 else 16) * 260 > 64 * 1024:
-        pytest.skip("staged activations of this forced shape exceed the kernel's shared-memory budget")
-    os.environ["UNIQL_DECODE_WK"], os.environ["UNIQL_DECODE_GS"] = str(wk), str(gs)
+    os.environ["UNIQL_DECODE_GS"], os.environ["UNIQL_DECODE_TPW"] = str(gs), str(tpw)
     B.set_path(B.PATH_DECODE)
     rng = np.random.default_rng(7)
     qw = synth.draw_qweight(rng, 144, 1536)
@@ -134,13 +132,13 @@ def test_decode_split_configs(B, wk, gs, M):
     for (k_in, k_out) in [(1536, 144), (1300, 100)]:
         x = synth.draw_x(rng, M, k_in, "f16")
         y, ref = run_ex(B, qw, dw, x, "f16", None, k_in, None, k_out, bias=bias)
-        check_output(y, ref, "f16", TIGHT, "wk=%d gs=%d M=%d" % (wk, gs, M))
+        check_output(y, ref, "f16", TIGHT, "gs=%d tpw=%d M=%d" % (gs, tpw, M))
         y2, _ = run_ex(B, qw, dw, x, "f16", None, k_in, None, k_out, bias=bias)
         assert torch.equal(y, y2), "run-to-run results differ"
 
 
 def test_caller_workspace(B):
-    os.environ["UNIQL_DECODE_WK"], os.environ["UNIQL_DECODE_GS"] = "1", "2"
+    os.environ["UNIQL_DECODE_GS"] = "2"
     rng = np.random.default_rng(8)
     qw = synth.draw_qweight(rng, 96, 1024)
     dw = dev_weight(qw)
@@ -270,7 +268,7 @@ def test_qk_rope_small(B, path, M, keep):
 def test_qk_rope_bf16_table_and_split(B):
     rng = np.random.default_rng(71)
     invf = (1e6 ** (-np.arange(64) / 64.0)) * 0.5          # a caller table (scaled-RoPE variants)
-    os.environ["UNIQL_DECODE_WK"], os.environ["UNIQL_DECODE_GS"] = "2", "1"
+    os.environ["UNIQL_DECODE_GS"], os.environ["UNIQL_DECODE_TPW"] = "2", "2"
     for (g, ref) in run_rope(B, rng, 3, 512, 4, 4, 128, 108, 1e6, "bf16", inv_freq=invf):
         check_output(g, ref, "bf16", TIGHT, "rope bf16 table")
 
