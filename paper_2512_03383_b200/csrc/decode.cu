@@ -12,10 +12,15 @@
 // which makes the result independent of the activation dtype's mantissa.
 // Truncation to the leading sorted channels (Section 3.4) is pure index arithmetic: pruned rows are
 // never addressed, pruned input channels are either outside the visited groups or meet a zero
-// activation.  A block of four warps owns one k-slice of GS groups (its activations staged once)
-// and walks over 4*tpw row tiles; a warp issues all 2*GS loads of a tile before it touches them,
-// and the other resident warps hide the latency.  k-slices of different blocks meet in a workspace
-// where the last block to arrive adds the partials in slice order (deterministic, no spinning).
+// activation.
+// Scheduling: one persistent block of 16 warps per SM.  All (row tile, k-chunk) units of the launch
+// form one k-fastest sequence that is cut into equal contiguous ranges, one per warp (stream-K), so
+// every SM streams the same number of bytes and nothing is launched in waves.  A warp keeps the loads
+// of its next chunk in flight while it works on the current one, accumulates in registers while it
+// stays on a tile, and when it leaves a tile that other warps also worked on it parks its partial sum
+// in a workspace slot; the last warp to arrive adds the slots in a fixed order (deterministic, no
+// spinning).  When the activations of a block do not fit in shared memory (large M x K) the input
+// channels are split into k-parts with their own blocks.
 // The rotary epilogue (Section 3.2, fused RoPE) needs both members of a rotation pair: in rope mode
 // a 16-row tile is 8 pairs, first-half members in rows 0..7 and their partners in rows 8..15, which
 // is exactly the (r, r+8) row pair a lane owns in the MMA accumulator layout.
@@ -27,25 +32,27 @@
 namespace uniql {
 namespace {
 
-constexpr int NTD = 128;          // threads per block (4 warps)
+constexpr int NW = 16;            // warps per block
+constexpr int NTD = NW * 32;      // threads per block
 constexpr int kMaxSpans = kMaxFam;
-constexpr int kCounterInts = 1 << 16;   // arrival counters at the head of the workspace
+constexpr int kCounterInts = 1 << 16;   // arrival counters (one per row tile) at the head of the workspace
+constexpr int kMaxKParts = 16;
+constexpr size_t kSmemBudget = 200 * 1024;
 
 struct DecodeCfg {
-  int tpw;               // row tiles per warp
-  int n_slices;          // blocks along k
-  int rb_total;
-  int rb_begin[kMaxJobs + 1];
-  int tiles[kMaxJobs];
-  int row_base[kMaxJobs];   // first row of each job in the partial-sum buffer
-  int rows_total;
+  int n_kp, n_rp;        // k-parts x row-parts = blocks
+  int gp;                // visited groups per k-part (the last part may be shorter)
+  int tiles_total;
+  int tile_begin[kMaxJobs + 1];   // first global tile of each job
+  int row_base[kMaxJobs];         // (unused by the kernel; kept for sizing)
   int g_total;           // visited 128-channel groups
   int n_spans;
   int vg_begin[kMaxSpans + 1];  // visit index at which span s starts
   int vg_first[kMaxSpans];      // its first stored group
   int x_vec;             // activations can be staged with 128-bit loads
-  int sz_vec;            // scales / zero-points of a slice can be fetched with one vector load
+  int sz_vec;            // scales / zero-points of a chunk can be fetched with one vector load
   int mp;                // activation rows staged in shared memory
+  int max_slots;         // workspace slots per tile
   int* counters;
   float* partials;
 };
@@ -133,15 +140,6 @@ template <> struct Cvt<__nv_bfloat16> {
   }
 };
 
-// 16-byte unit of the staged activations: activation row m, local group lv, word j, lane chunk c.
-// A row holds GS groups of 256 bytes plus 64 bytes of padding, so that the two rows met by the eight
-// lanes of one 128-bit shared-load phase sit 64 bytes apart modulo 128 (distinct banks), and every
-// (group, word) offset is a compile-time immediate.
-template <int GS>
-__device__ inline int x_unit(int lv, int m, int j, int c) {
-  return m * (GS * 16 + 4) + lv * 16 + j * 4 + c;
-}
-
 // The two weight rows a lane owns in a 16-row tile.
 struct LaneRows {
   int sr0, sr1;      // stored rows (clamped to a valid row when the slot is empty)
@@ -211,52 +209,196 @@ __device__ inline void epilogue(const Params& p, const JobDev& jb, const LaneRow
     }
 }
 
-template <typename T, int MT, int GS>
-__global__ void __launch_bounds__(NTD) decode_kernel(const __grid_constant__ Params p,
-                                                     const __grid_constant__ DecodeCfg c) {
+// ---------------------------------------------------------------------------------------- kernel
+__device__ inline int owner_of(long u, long W, long U) {
+  // the warp whose range [U*w/W, U*(w+1)/W) holds unit u; exact in fp64 for these magnitudes
+  return (int)floor(((double)(u + 1) * (double)W - 1.0) / (double)U);
+}
+
+// A warp leaves tile `tgl`: finish it alone, or park the partial sum in its workspace slot and let the
+// last warp to arrive add all slots in slot order and finish.  Kept out of line: it runs once or twice
+// per warp and would only bloat the streaming loop.  Everything is passed by value so that the caller's
+// accumulators stay in registers.
+constexpr int MT_MAX = 2;
+struct OutVals { float v[MT_MAX][4]; };
+template <typename T, int MT, int CH>
+__device__ __noinline__ void flush_tile(const Params& p, const DecodeCfg& c, int kp, int gw, int tgl, int jl,
+                                        const LaneRows Ll, int lane, const OutVals ov) {
+  const int r = lane >> 2, cq = lane & 3;
+  float out[MT][4];
+#pragma unroll
+  for (int t = 0; t < MT; ++t)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) out[t][i] = ov.v[t][i];
+  const long Wall = (long)c.n_rp * NW;
+  int total = 0, my_slot = 0;
+  for (int q = 0; q < c.n_kp; ++q) {
+    const int Gq = min(c.gp, c.g_total - q * c.gp);
+    const long Cq = (Gq + CH - 1) / CH;
+    const long Uq = (long)c.tiles_total * Cq;
+    const long Wq = Wall < Uq ? Wall : Uq;
+    const int first = owner_of((long)tgl * Cq, Wq, Uq);
+    const int last = owner_of((long)tgl * Cq + Cq - 1, Wq, Uq);
+    if (q == kp) my_slot = total + (gw - first);
+    total += last - first + 1;
+  }
+  if (total == 1) {
+    epilogue<T, MT>(p, p.job[jl], Ll, cq, out);
+    return;
+  }
+  const size_t slot_floats = (size_t)p.M * 16;
+  float* tile_part = c.partials + (size_t)tgl * c.max_slots * slot_floats;
+  float* mine = tile_part + (size_t)my_slot * slot_floats;
+#pragma unroll
+  for (int t = 0; t < MT; ++t)
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int m = 2 * cq + e + 8 * t;
+      if (m >= p.M) continue;
+      __stcg(mine + m * 16 + r, out[t][e]);
+      __stcg(mine + m * 16 + r + 8, out[t][2 + e]);
+    }
+  __threadfence();
+  __syncwarp();
+  int last_arrival = 0;
+  if (lane == 0) last_arrival = atomicAdd(&c.counters[tgl], 1) == total - 1;
+  last_arrival = __shfl_sync(0xffffffffu, last_arrival, 0);
+  if (!last_arrival) return;
+  __threadfence();
+#pragma unroll
+  for (int t = 0; t < MT; ++t)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) out[t][i] = 0.f;
+  for (int s2 = 0; s2 < total; ++s2) {
+    const float* src = tile_part + (size_t)s2 * slot_floats;
+#pragma unroll
+    for (int t = 0; t < MT; ++t)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int m = 2 * cq + e + 8 * t;
+        if (m >= p.M) continue;
+        out[t][e] += __ldcg(src + m * 16 + r);
+        out[t][2 + e] += __ldcg(src + m * 16 + r + 8);
+      }
+  }
+  epilogue<T, MT>(p, p.job[jl], Ll, cq, out);
+  if (lane == 0) c.counters[tgl] = 0;       // ready for the next call
+}
+
+template <typename T, int MT, int CH>
+__global__ void __launch_bounds__(NTD, 1) decode_kernel(const __grid_constant__ Params p,
+                                                        const __grid_constant__ DecodeCfg c) {
   extern __shared__ __align__(16) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int r = lane >> 2, cq = lane & 3;
   const int mp = c.mp;
-  // shared memory: staged activations, mp rows + one all-zero row of (GS*256+64) bytes each, then
-  // the per-group activation sums [GS][8*MT] fp32
-  constexpr int kRowBytes = GS * 256 + 64;
-  uint4* xs = reinterpret_cast<uint4*>(smem);
-  const int xg_off = (mp + 1) * kRowBytes;
+  const int kp = blockIdx.x / c.n_rp, rp = blockIdx.x - kp * c.n_rp;
+  const int v_lo = kp * c.gp;                                   // first visit index of this k-part
+  const int Gk = min(c.gp, c.g_total - v_lo);                   // its groups
+  const int Ck = (Gk + CH - 1) / CH;                            // chunks per tile
+  // shared memory: staged activations, mp rows + one all-zero row of (gp*256+64) bytes each (a group is
+  // 256 bytes; the 64-byte pad puts the two rows met by one 128-bit load phase on distinct banks), then
+  // the per-group activation sums [gp][8*MT] fp32
+  const int row_bytes = c.gp * 256 + 64;
+  const int xg_off = (mp + 1) * row_bytes;
   float* xg = reinterpret_cast<float*>(smem + xg_off);
+  const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
+  const int sg_lo = visit_to_group(c, v_lo);
+  const bool contig = visit_to_group(c, v_lo + Gk - 1) == sg_lo + Gk - 1;   // block-uniform
 
-  const int rb = blockIdx.x;
-  int jn = 0;
-  while (jn + 1 < p.n_jobs && rb >= c.rb_begin[jn + 1]) ++jn;
-  const JobDev& jb = p.job[jn];
-  const int v0 = blockIdx.y * GS;
-  const int nvalid = min(GS, c.g_total - v0);
-  const int sg0 = visit_to_group(c, v0);
-  const bool contig = visit_to_group(c, v0 + nvalid - 1) == sg0 + nvalid - 1;   // block-uniform
+  // ---- this warp's contiguous range of (tile, chunk) units, k fastest
+  const long U = (long)c.tiles_total * Ck;
+  const long Wall = (long)c.n_rp * NW;
+  const long W = Wall < U ? Wall : U;                           // warps that get work
+  const int gw = rp * NW + warp;
+  int ub = 0, ue = 0;
+  if (gw < W) { ub = (int)(U * gw / W); ue = (int)(U * (gw + 1) / W); }
+
+  const int G = p.K / kGroup;
+  auto job_of = [&](int tg) { int j = 0; while (j + 1 < p.n_jobs && tg >= c.tile_begin[j + 1]) ++j; return j; };
+
+  // packed codes of the CH groups of the current chunk (reloaded in place, group by group, with the
+  // next chunk's codes as soon as a group has been consumed) and fp16 scale / zero pairs
+  uint4 w0[CH], w1[CH];
+  uint32_t sc[4][CH / 2], scn[4][CH / 2];   // s(row r), z(row r), s(row r+8), z(row r+8); two groups per word
+
+  auto load_group = [&](int g, const uint8_t* q0, const uint8_t* q1, int chn) {
+    // q0/q1: row pointers already advanced to this lane's 16 bytes of stored group sg_lo (contiguous case)
+    const int gi = chn * CH + g;
+    if (gi < Gk) {
+      const size_t off = (size_t)(contig ? sg_lo + gi : visit_to_group(c, v_lo + gi)) * 64;
+      w0[g] = ldg_stream(q0 + off);
+      w1[g] = ldg_stream(q1 + off);
+    }
+  };
+  auto load_scales = [&](uint32_t (&dst)[4][CH / 2], const JobDev& jb, const LaneRows& L, int chn) {
+    const int g0 = chn * CH;
+    const __half* base[4] = {jb.scales + (size_t)L.sr0 * G, jb.zeros + (size_t)L.sr0 * G,
+                             jb.scales + (size_t)L.sr1 * G, jb.zeros + (size_t)L.sr1 * G};
+    if (c.sz_vec) {     // chunk start is CH-aligned in stored groups and the CH values are contiguous
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if constexpr (CH == 4) {
+          const uint2 v = __ldg(reinterpret_cast<const uint2*>(base[q] + sg_lo + g0));
+          dst[q][0] = v.x; dst[q][1] = v.y;
+        } else {
+          dst[q][0] = __ldg(reinterpret_cast<const uint32_t*>(base[q] + sg_lo + g0));
+        }
+      }
+    } else {
+      const int nv = min(CH, Gk - g0);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+#pragma unroll
+        for (int g = 0; g < CH; g += 2) {
+          const int ga = visit_to_group(c, v_lo + g0 + (g < nv ? g : 0));
+          const int gb = visit_to_group(c, v_lo + g0 + (g + 1 < nv ? g + 1 : 0));
+          const uint32_t lo = __half_as_ushort(__ldg(base[q] + ga));
+          const uint32_t hi = __half_as_ushort(__ldg(base[q] + gb));
+          dst[q][g >> 1] = lo | (hi << 16);
+        }
+    }
+  };
+
+  // the first chunk's loads go out before the activations are staged (they do not depend on them)
+  int tg = 0, ch = 0, jn = 0;
+  LaneRows L;
+  if (ub < ue) {
+    tg = ub / Ck; ch = ub - tg * Ck;
+    jn = job_of(tg);
+    L = resolve_rows(p.job[jn], tg - c.tile_begin[jn], r);
+    const uint8_t* q0 = p.job[jn].w + (size_t)L.sr0 * (p.K / 2) + cq * 16;
+    const uint8_t* q1 = p.job[jn].w + (size_t)L.sr1 * (p.K / 2) + cq * 16;
+#pragma unroll
+    for (int g = 0; g < CH; ++g) load_group(g, q0, q1, ch);
+    load_scales(sc, p.job[jn], L, ch);
+  }
 
   // ---- stage activations: permuted into nibble order, zero where the channel is pruned
   {
     const T* x = reinterpret_cast<const T*>(p.x);
-    for (int i = tid; i < kRowBytes / 16; i += NTD) xs[mp * (kRowBytes / 16) + i] = make_uint4(0, 0, 0, 0);
-    for (int i = tid; i < GS * 8 * MT; i += NTD) xg[i] = 0.f;
+    uint4* xs = reinterpret_cast<uint4*>(smem);
+    const int row_units = row_bytes / 16;
+    for (int i = tid; i < row_units; i += NTD) xs[mp * row_units + i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < c.gp * 8 * MT; i += NTD) xg[i] = 0.f;
     __syncthreads();
     if (c.x_vec) {
       const int start = p.imap.fam[0].start, keep = p.imap.fam[0].keep;
-      const int n_units = GS * mp * 16;
+      const int n_units = Gk * mp * 16;
       for (int u = tid; u < ((n_units + 31) & ~31); u += NTD) {   // whole warps stay in the shuffles
         const bool in_range = u < n_units;
         const int u16 = u & 15, pair = in_range ? u >> 4 : 0;
-        const int m = pair / GS, lv = pair - m * GS;
-        const int ccq = u16 >> 2, j = u16 & 3;
+        const int m = pair / Gk, lv = pair - m * Gk;
         uint4 in = make_uint4(0, 0, 0, 0);
-        if (in_range && lv < nvalid && m < p.M) {
-          const int t0 = (contig ? sg0 + lv : visit_to_group(c, v0 + lv)) * kGroup + 8 * u16 - start;
+        if (in_range && m < p.M) {
+          const int t0 = (contig ? sg_lo + lv : visit_to_group(c, v_lo + lv)) * kGroup + 8 * u16 - start;
           if (t0 >= 0 && t0 < keep) in = *reinterpret_cast<const uint4*>(x + (size_t)m * p.ldx + t0);
         }
         uint4 o;
         o.x = __byte_perm(in.x, in.z, 0x5410); o.y = __byte_perm(in.x, in.z, 0x7632);
         o.z = __byte_perm(in.y, in.w, 0x5410); o.w = __byte_perm(in.y, in.w, 0x7632);
-        if (in_range) xs[x_unit<GS>(lv, m, j, ccq)] = o;
+        // unit (chunk c', word j) of a group sits at byte j*64 + c'*16; u16 = c'*4 + j
+        if (in_range) xs[m * row_units + lv * 16 + (u16 & 3) * 4 + (u16 >> 2)] = o;
         const typename DT<T>::T2* h2 = reinterpret_cast<const typename DT<T>::T2*>(&in);
         float sum = 0.f;
 #pragma unroll
@@ -267,11 +409,11 @@ __global__ void __launch_bounds__(NTD) decode_kernel(const __grid_constant__ Par
       }
     } else {
       T* xh = reinterpret_cast<T*>(smem);
-      const int n_pairs = GS * mp;
-      for (int pair = warp; pair < n_pairs; pair += NTD / 32) {
-        const int m = pair / GS, lv = pair - m * GS;
-        const bool live = lv < nvalid && m < p.M;
-        const int kbase = live ? visit_to_group(c, v0 + lv) * kGroup : 0;
+      const int n_pairs = Gk * mp;
+      for (int pair = warp; pair < n_pairs; pair += NW) {
+        const int m = pair / Gk, lv = pair - m * Gk;
+        const bool live = m < p.M;
+        const int kbase = visit_to_group(c, v_lo + lv) * kGroup;
         float sum = 0.f;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -282,7 +424,7 @@ __global__ void __launch_bounds__(NTD) decode_kernel(const __grid_constant__ Par
             if (t >= 0) val = x[(size_t)m * p.ldx + t];
           }
           const int ccq = i >> 5, j = (i & 31) >> 3, e = i & 7;
-          xh[x_unit<GS>(lv, m, j, ccq) * 8 + 2 * (e & 3) + (e >> 2)] = val;
+          xh[(m * row_units + lv * 16 + j * 4 + ccq) * 8 + 2 * (e & 3) + (e >> 2)] = val;
           sum += DT<T>::to_f(val);
         }
 #pragma unroll
@@ -292,97 +434,51 @@ __global__ void __launch_bounds__(NTD) decode_kernel(const __grid_constant__ Par
     }
   }
   __syncthreads();
+  if (ub >= ue) return;
 
   // per-lane shared-memory address of the B fragments (lanes beyond the staged rows read the zero row)
-  const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
   uint32_t xb_addr[MT];
 #pragma unroll
   for (int t = 0; t < MT; ++t) {
     const int m = r + 8 * t;
-    xb_addr[t] = smem_base + (uint32_t)((m < mp ? m : mp) * kRowBytes + cq * 16);
+    xb_addr[t] = smem_base + (uint32_t)((m < mp ? m : mp) * row_bytes + cq * 16);
   }
   const uint32_t xg_addr = smem_base + (uint32_t)xg_off + (uint32_t)(2 * cq * 4);
 
-  const int G = p.K / kGroup;
-  const int first_tile = (rb - c.rb_begin[jn]) * (4 * c.tpw);
-  const int n_tiles = c.tiles[jn];
-  const size_t part_mstride = (size_t)c.rows_total;
-
-  for (int it = 0; it < c.tpw; ++it) {
-    const int tile = first_tile + it * 4 + warp;
-    if (tile >= n_tiles) break;
-    const LaneRows L = resolve_rows(jb, tile, r);
-    const uint8_t* wrow0 = jb.w + (size_t)L.sr0 * (p.K / 2) + cq * 16;
-    const uint8_t* wrow1 = jb.w + (size_t)L.sr1 * (p.K / 2) + cq * 16;
-
-    // ---- all loads of this tile first
-    uint4 w0[GS], w1[GS];
-    if (contig) {
-      const uint8_t* q0 = wrow0 + (size_t)sg0 * 64;
-      const uint8_t* q1 = wrow1 + (size_t)sg0 * 64;
+  float out[MT][4];
 #pragma unroll
-      for (int g = 0; g < GS; ++g) {
-        if (g < nvalid) {
-          w0[g] = ldg_stream(q0 + g * 64);
-          w1[g] = ldg_stream(q1 + g * 64);
-        } else {
-          w0[g] = make_uint4(0, 0, 0, 0); w1[g] = w0[g];
-        }
-      }
-    } else {
+  for (int t = 0; t < MT; ++t)
 #pragma unroll
-      for (int g = 0; g < GS; ++g) {
-        if (g < nvalid) {
-          const size_t off = (size_t)visit_to_group(c, v0 + g) * 64;
-          w0[g] = ldg_stream(wrow0 + off);
-          w1[g] = ldg_stream(wrow1 + off);
-        } else {
-          w0[g] = make_uint4(0, 0, 0, 0); w1[g] = w0[g];
-        }
+    for (int i = 0; i < 4; ++i) out[t][i] = 0.f;
+
+  // ---- stream the units: while group g of the current chunk is consumed, group g of the next chunk
+  //      is already being fetched into the registers group g-1 has just freed
+  for (int u = ub;; ++u) {
+    const bool has_next = u + 1 < ue;
+    int tg1 = tg, ch1 = ch + 1, jn1 = jn;
+    LaneRows L1 = L;
+    if (ch1 == Ck) { ch1 = 0; tg1 = tg + 1; }
+    const uint8_t* q0 = nullptr;
+    const uint8_t* q1 = nullptr;
+    if (has_next) {
+      if (tg1 != tg) {
+        jn1 = job_of(tg1);
+        L1 = resolve_rows(p.job[jn1], tg1 - c.tile_begin[jn1], r);
       }
+      q0 = p.job[jn1].w + (size_t)L1.sr0 * (p.K / 2) + cq * 16;
+      q1 = p.job[jn1].w + (size_t)L1.sr1 * (p.K / 2) + cq * 16;
+      load_scales(scn, p.job[jn1], L1, ch1);
     }
-    uint32_t sc[4][(GS + 1) / 2];   // packed fp16 pairs: s(row r), z(row r), s(row r+8), z(row r+8)
-    {
-      const __half* base[4] = {jb.scales + (size_t)L.sr0 * G, jb.zeros + (size_t)L.sr0 * G,
-                               jb.scales + (size_t)L.sr1 * G, jb.zeros + (size_t)L.sr1 * G};
-      if (c.sz_vec) {
+    const int g0 = ch * CH;
+    const int nvalid = min(CH, Gk - g0);
+    uint32_t xa[MT];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          if constexpr (GS == 8) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(base[q] + sg0));
-            sc[q][0] = v.x; sc[q][1] = v.y; sc[q][2] = v.z; sc[q][3] = v.w;
-          } else if constexpr (GS == 4) {
-            const uint2 v = __ldg(reinterpret_cast<const uint2*>(base[q] + sg0));
-            sc[q][0] = v.x; sc[q][1] = v.y;
-          } else {
-            sc[q][0] = __ldg(reinterpret_cast<const uint32_t*>(base[q] + sg0));
-          }
-        }
-      } else {
+    for (int t = 0; t < MT; ++t) xa[t] = xb_addr[t] + (uint32_t)(g0 * 256);
+    const uint32_t xga = xg_addr + (uint32_t)(g0 * 8 * MT * 4);
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
-#pragma unroll
-          for (int g = 0; g < GS; g += 2) {
-            const int ga = visit_to_group(c, v0 + (g < nvalid ? g : 0));
-            const int gb = visit_to_group(c, v0 + (g + 1 < nvalid ? g + 1 : 0));
-            const uint32_t lo = __half_as_ushort(__ldg(base[q] + ga));
-            const uint32_t hi = __half_as_ushort(__ldg(base[q] + gb));
-            sc[q][g >> 1] = lo | (hi << 16);
-          }
-      }
-    }
-
-    float out[MT][4];
-#pragma unroll
-    for (int t = 0; t < MT; ++t)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) out[t][i] = 0.f;
-
-#pragma unroll
-    for (int g = 0; g < GS; ++g) {
+    for (int g = 0; g < CH; ++g) {
       if (g < nvalid) {
-        // two accumulators per batch tile keep two independent MMA chains in flight
-        float acc[MT][2][4];
+        float acc[MT][2][4];     // two accumulators per batch tile: two independent MMA chains
         const uint32_t wa[4] = {w0[g].x, w0[g].y, w0[g].z, w0[g].w};
         const uint32_t wb[4] = {w1[g].x, w1[g].y, w1[g].z, w1[g].w};
 #pragma unroll
@@ -392,7 +488,7 @@ __global__ void __launch_bounds__(NTD) decode_kernel(const __grid_constant__ Par
           Cvt<T>::word(wb[j], b);
 #pragma unroll
           for (int t = 0; t < MT; ++t) {
-            const uint4 xb = lds128(xb_addr[t] + (uint32_t)(g * 256 + j * 64));
+            const uint4 xb = lds128(xa[t] + (uint32_t)(g * 256 + j * 64));
             if (j == 0) {
               Cvt<T>::mma0(acc[t][0], a[0], b[0], a[1], b[1], xb.x, xb.y);
               Cvt<T>::mma0(acc[t][1], a[2], b[2], a[3], b[3], xb.z, xb.w);
@@ -402,6 +498,7 @@ __global__ void __launch_bounds__(NTD) decode_kernel(const __grid_constant__ Par
             }
           }
         }
+        if (has_next) load_group(g, q0, q1, ch1);      // the registers of group g are free again
         auto pick = [&](int q) -> float {
           const __half2 h = *reinterpret_cast<const __half2*>(&sc[q][g >> 1]);
           return (g & 1) ? __high2float(h) : __low2float(h);
@@ -410,68 +507,35 @@ __global__ void __launch_bounds__(NTD) decode_kernel(const __grid_constant__ Par
         const float s1 = pick(2), nz1 = 8.f - pick(3);
 #pragma unroll
         for (int t = 0; t < MT; ++t) {
-          const float2 X = lds64f(xg_addr + (uint32_t)((g * 8 * MT + 8 * t) * 4));
+          const float2 X = lds64f(xga + (uint32_t)((g * 8 * MT + 8 * t) * 4));
           out[t][0] = fmaf(s0, fmaf(nz0, X.x, acc[t][0][0] + acc[t][1][0]), out[t][0]);
           out[t][1] = fmaf(s0, fmaf(nz0, X.y, acc[t][0][1] + acc[t][1][1]), out[t][1]);
           out[t][2] = fmaf(s1, fmaf(nz1, X.x, acc[t][0][2] + acc[t][1][2]), out[t][2]);
           out[t][3] = fmaf(s1, fmaf(nz1, X.y, acc[t][0][3] + acc[t][1][3]), out[t][3]);
         }
+      } else if (has_next) {
+        load_group(g, q0, q1, ch1);
       }
     }
-
-    if (c.n_slices == 1) {
-      epilogue<T, MT>(p, jb, L, cq, out);
-    } else {
-      // compact partial sums: [slice][m][row]
-      float* part = c.partials + (size_t)blockIdx.y * p.M * part_mstride + c.row_base[jn];
+    if (!has_next || tg1 != tg) {
+      OutVals ov;
+#pragma unroll
+      for (int t = 0; t < MT_MAX; ++t)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) ov.v[t][i] = t < MT ? out[t < MT ? t : 0][i] : 0.f;
+      flush_tile<T, MT, CH>(p, c, kp, gw, tg, jn, L, lane, ov);
 #pragma unroll
       for (int t = 0; t < MT; ++t)
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const int m = 2 * cq + e + 8 * t;
-          if (m >= p.M) continue;
-          if (L.oc0 >= 0) __stcg(part + (size_t)m * part_mstride + L.oc0, out[t][e]);
-          if (L.oc1 >= 0) __stcg(part + (size_t)m * part_mstride + L.oc1, out[t][2 + e]);
-        }
+        for (int i = 0; i < 4; ++i) out[t][i] = 0.f;
     }
+    if (!has_next) break;
+    tg = tg1; ch = ch1; jn = jn1; L = L1;
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+#pragma unroll
+      for (int i = 0; i < CH / 2; ++i) sc[q][i] = scn[q][i];
   }
-  if (c.n_slices == 1) return;
-
-  // ---- the last block to arrive for this row block sums the slices in order and finishes
-  __shared__ int s_last;
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const int ticket = atomicAdd(&c.counters[rb], 1);
-    s_last = ticket == c.n_slices - 1;
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  for (int it = 0; it < c.tpw; ++it) {
-    const int tile = first_tile + it * 4 + warp;
-    if (tile >= n_tiles) break;
-    const LaneRows L = resolve_rows(jb, tile, r);
-    float out[MT][4];
-#pragma unroll
-    for (int t = 0; t < MT; ++t)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) out[t][i] = 0.f;
-    for (int s = 0; s < c.n_slices; ++s) {
-      const float* part = c.partials + (size_t)s * p.M * part_mstride + c.row_base[jn];
-#pragma unroll
-      for (int t = 0; t < MT; ++t)
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const int m = 2 * cq + e + 8 * t;
-          if (m >= p.M) continue;
-          if (L.oc0 >= 0) out[t][e] += __ldcg(part + (size_t)m * part_mstride + L.oc0);
-          if (L.oc1 >= 0) out[t][2 + e] += __ldcg(part + (size_t)m * part_mstride + L.oc1);
-        }
-    }
-    epilogue<T, MT>(p, jb, L, cq, out);
-  }
-  if (tid == 0) c.counters[rb] = 0;     // ready for the next call
 }
 
 // -------------------------------------------------------------------------------- host side
@@ -510,43 +574,64 @@ void build_spans(const ChanMap& m, DecodeCfg* c) {
   c->g_total = total;
 }
 
-template <typename T, int MT, int GS>
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+      n = v;
+    else
+      n = 148;
+  }
+  return n;
+}
+
+size_t smem_bytes(int mp, int gp, int MT) { return (size_t)(mp + 1) * (gp * 256 + 64) + (size_t)gp * 8 * MT * 4; }
+
+template <typename T, int MT, int CH>
 int launch_t(const Params& p, const DecodeCfg& c, cudaStream_t stream) {
-  size_t smem = (size_t)(c.mp + 1) * (GS * 256 + 64) + (size_t)GS * 8 * MT * 4;
-  auto kern = decode_kernel<T, MT, GS>;
+  const size_t smem = smem_bytes(c.mp, c.gp, MT);
+  auto kern = decode_kernel<T, MT, CH>;
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return UNIQL_ERR_CUDA;
-  dim3 grid(c.rb_total, c.n_slices);
-  kern<<<grid, NTD, smem, stream>>>(p, c);
+  kern<<<c.n_kp * c.n_rp, NTD, smem, stream>>>(p, c);
   return cudaGetLastError() == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
 }
 
-template <typename T>
-int launch_dt(const Params& p, const DecodeCfg& c, int MT, int GS, cudaStream_t stream) {
-  if (MT == 1) {
-    if (GS == 8) return launch_t<T, 1, 8>(p, c, stream);
-    if (GS == 4) return launch_t<T, 1, 4>(p, c, stream);
-    return launch_t<T, 1, 2>(p, c, stream);
+// Worst-case number of workspace slots a tile needs for a given split.
+int slots_needed(int tiles, int g_total, int gp, int n_rp, int CH) {
+  int total = 0;
+  for (int v = 0; v < g_total; v += gp) {
+    const long Gq = (g_total - v) < gp ? (g_total - v) : gp;
+    const long Cq = (Gq + CH - 1) / CH;
+    const long Uq = (long)tiles * Cq;
+    long Wq = (long)n_rp * NW;
+    if (Wq > Uq) Wq = Uq;
+    const long per_warp = Uq / Wq;           // >= 1
+    total += (int)((Cq + per_warp - 1) / per_warp) + 1;
   }
-  if (GS == 8) return launch_t<T, 2, 8>(p, c, stream);
-  if (GS == 4) return launch_t<T, 2, 4>(p, c, stream);
-  return launch_t<T, 2, 2>(p, c, stream);
+  return total;
 }
 
 }  // namespace
 
 int decode_supported(const Params& p) {
   if (p.M < 1 || p.M > 16) return 0;
-  for (int j = 0; j < p.n_jobs; ++j)
+  long tiles = 0;
+  for (int j = 0; j < p.n_jobs; ++j) {
     if (job_tiles(p.job[j]) < 1) return 0;
-  return 1;
+    tiles += job_tiles(p.job[j]);
+  }
+  return tiles <= kCounterInts;
 }
 
 size_t decode_workspace_bytes(int M, int K, int N_total) {
-  // counters + fp32 partial sums [slices][M][rows] for the finest slicing (2 groups per slice)
-  size_t slices = (size_t)(K / kGroup + 1) / 2 + 1;
-  return (size_t)kCounterInts * 4 + slices * (size_t)M * (size_t)N_total * 4;
+  // arrival counters + fp32 partial sums: up to 4 slots of [M][16] per 16-row tile and k-part
+  (void)K;
+  size_t tiles = (size_t)(N_total + 15) / 16 + 8 * kMaxJobs;
+  return (size_t)kCounterInts * 4 + tiles * (4 * kMaxKParts) * (size_t)M * 16 * 4;
 }
 
 int launch_decode(const Params& p, const LaunchCfg& cfg) {
@@ -554,61 +639,56 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   memset(&c, 0, sizeof(c));
   build_spans(p.imap, &c);
   const int MT = p.M <= 8 ? 1 : 2;
+  const int CH = MT == 1 ? 4 : 2;
   c.mp = MT == 1 ? p.M : 16;
   // 128-bit staging: one leading family, everything 8-element aligned
   c.x_vec = p.imap.n_fam == 1 && p.imap.fam[0].count == 1 && (p.imap.fam[0].start % 8) == 0 &&
             (p.imap.fam[0].keep % 8) == 0 && (p.ldx % 8) == 0 && ((((uintptr_t)p.x) & 15) == 0);
-  int rows = 0, tiles_total = 0;
+  int tiles = 0;
   for (int j = 0; j < p.n_jobs; ++j) {
-    c.tiles[j] = job_tiles(p.job[j]);
-    c.row_base[j] = rows;
-    rows += p.job[j].k_out;
-    tiles_total += c.tiles[j];
+    c.tile_begin[j] = tiles;
+    tiles += job_tiles(p.job[j]);
   }
-  c.rows_total = rows;
+  for (int j = p.n_jobs; j <= kMaxJobs; ++j) c.tile_begin[j] = tiles;
+  c.tiles_total = tiles;
+  if (tiles > kCounterInts) return UNIQL_ERR_SHAPE;
 
-  const size_t ws_part = cfg.ws_bytes > (size_t)kCounterInts * 4 ? cfg.ws_bytes - (size_t)kCounterInts * 4 : 0;
-  // ---- block shape: GS groups per k-slice, tpw row tiles per warp
-  const int force_gs = env_int("UNIQL_DECODE_GS", 0), force_tpw = env_int("UNIQL_DECODE_TPW", 0);
-  int GS = MT == 1 ? 8 : 4;
-  if (c.g_total < GS) GS = c.g_total >= 4 ? 4 : 2;
-  if (force_gs == 8 || force_gs == 4 || force_gs == 2) GS = force_gs;
-  int slices = (c.g_total + GS - 1) / GS;
-  while (slices > 1 && (size_t)slices * p.M * rows * 4 > ws_part && GS < 8) {   // coarser slices need less workspace
-    GS *= 2;
-    slices = (c.g_total + GS - 1) / GS;
+  // ---- k-parts: as few as let the staged activations fit in shared memory (gp a multiple of CH)
+  int n_kp = env_int("UNIQL_DECODE_KP", 0);
+  if (n_kp < 1) {
+    n_kp = 1;
+    while (n_kp < kMaxKParts) {
+      int gp = ((c.g_total + n_kp - 1) / n_kp + CH - 1) / CH * CH;
+      if (smem_bytes(c.mp, gp, MT) <= kSmemBudget) break;
+      ++n_kp;
+    }
   }
-  if (slices > 1 && (!cfg.workspace || (size_t)slices * p.M * rows * 4 > ws_part)) return UNIQL_ERR_WORKSPACE;
-  if (slices > 65535) return UNIQL_ERR_SHAPE;
-  // enough blocks to fill the machine a few times over, otherwise as many tiles per warp as possible
-  int tpw = 1;
+  if (n_kp > kMaxKParts) n_kp = kMaxKParts;
+  c.gp = ((c.g_total + n_kp - 1) / n_kp + CH - 1) / CH * CH;
+  c.n_kp = (c.g_total + c.gp - 1) / c.gp;
+  if (smem_bytes(c.mp, c.gp, MT) > 220 * 1024) return UNIQL_ERR_UNSUPPORTED;
+  int n_rp = env_int("UNIQL_DECODE_RP", 0);
+  if (n_rp < 1) n_rp = sm_count() / c.n_kp;
+  if (n_rp < 1) n_rp = 1;
+  c.n_rp = n_rp;
+  c.max_slots = slots_needed(tiles, c.g_total, c.gp, c.n_rp, CH);
   {
-    const long target = 148L * 4 * 4;
-    while (tpw < 8 && (long)((tiles_total + 4 * (tpw * 2) - 1) / (4 * (tpw * 2))) * slices >= target) tpw *= 2;
+    const size_t need = (size_t)kCounterInts * 4 + (size_t)tiles * c.max_slots * p.M * 16 * 4;
+    if (!cfg.workspace || cfg.ws_bytes < need) return UNIQL_ERR_WORKSPACE;
   }
-  if (force_tpw >= 1 && force_tpw <= 64) tpw = force_tpw;
-  c.tpw = tpw;
-  c.n_slices = slices;
-  int rbt = 0;
-  for (int j = 0; j < p.n_jobs; ++j) {
-    c.rb_begin[j] = rbt;
-    rbt += (c.tiles[j] + 4 * tpw - 1) / (4 * tpw);
-  }
-  for (int j = p.n_jobs; j <= kMaxJobs; ++j) c.rb_begin[j] = rbt;
-  c.rb_total = rbt;
-  if (rbt > kCounterInts) return UNIQL_ERR_SHAPE;
-  // vector loads of scales / zero-points: slice starts GS-aligned, contiguous, rows GS-aligned
+  // vector loads of scales / zero-points: every chunk starts CH-aligned in stored groups and is contiguous
   {
     const int G = p.K / kGroup;
-    bool ok = c.n_spans == 1 && (c.vg_first[0] % GS) == 0 && (G % GS) == 0;
+    bool ok = c.n_spans == 1 && (c.vg_first[0] % CH) == 0 && (G % CH) == 0;
     for (int j = 0; j < p.n_jobs && ok; ++j)
       ok = ((((uintptr_t)p.job[j].scales) | ((uintptr_t)p.job[j].zeros)) & 15) == 0;
     c.sz_vec = ok;
   }
   c.counters = reinterpret_cast<int*>(cfg.workspace);
   c.partials = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(cfg.workspace) + (size_t)kCounterInts * 4);
-  if (p.dt == UNIQL_F16) return launch_dt<__half>(p, c, MT, GS, cfg.stream);
-  return launch_dt<__nv_bfloat16>(p, c, MT, GS, cfg.stream);
+  if (p.dt == UNIQL_F16)
+    return MT == 1 ? launch_t<__half, 1, 4>(p, c, cfg.stream) : launch_t<__half, 2, 2>(p, c, cfg.stream);
+  return MT == 1 ? launch_t<__nv_bfloat16, 1, 4>(p, c, cfg.stream) : launch_t<__nv_bfloat16, 2, 2>(p, c, cfg.stream);
 }
 
 }  // namespace uniql

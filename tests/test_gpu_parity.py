@@ -25,7 +25,7 @@ def B():
 def _reset_path(B):
     yield
     B.set_path(B.PATH_AUTO)
-    for k in ("UNIQL_DECODE_TPW", "UNIQL_DECODE_GS"):
+    for k in ("UNIQL_DECODE_KP", "UNIQL_DECODE_RP"):
         os.environ.pop(k, None)
 
 
@@ -119,11 +119,11 @@ def test_m_sweep(B, M, dtype):
         check_output(y, ref, dtype, TIGHT, "M=%d %s k=(%d,%d)" % (M, dtype, k_in, k_out))
 
 
-@pytest.mark.parametrize("gs,tpw", [(2, 1), (4, 1), (8, 1), (2, 3), (4, 2), (8, 4), (8, 64)])
+@pytest.mark.parametrize("kp,rp", [(1, 1), (1, 3), (2, 5), (3, 49), (1, 148), (4, 2), (12, 12)])
 @pytest.mark.parametrize("M", [1, 5, 16])
-def test_decode_split_configs(B, gs, tpw, M):
-    """Every block shape / split-K factor of the decode kernel gives the same answer."""
-    os.environ["UNIQL_DECODE_GS"], os.environ["UNIQL_DECODE_TPW"] = str(gs), str(tpw)
+def test_decode_split_configs(B, kp, rp, M):
+    """Every way of cutting the work (k-parts x blocks per k-part) gives the same answer."""
+    os.environ["UNIQL_DECODE_KP"], os.environ["UNIQL_DECODE_RP"] = str(kp), str(rp)
     B.set_path(B.PATH_DECODE)
     rng = np.random.default_rng(7)
     qw = synth.draw_qweight(rng, 144, 1536)
@@ -132,13 +132,13 @@ def test_decode_split_configs(B, gs, tpw, M):
     for (k_in, k_out) in [(1536, 144), (1300, 100)]:
         x = synth.draw_x(rng, M, k_in, "f16")
         y, ref = run_ex(B, qw, dw, x, "f16", None, k_in, None, k_out, bias=bias)
-        check_output(y, ref, "f16", TIGHT, "gs=%d tpw=%d M=%d" % (gs, tpw, M))
+        check_output(y, ref, "f16", TIGHT, "kp=%d rp=%d M=%d" % (kp, rp, M))
         y2, _ = run_ex(B, qw, dw, x, "f16", None, k_in, None, k_out, bias=bias)
         assert torch.equal(y, y2), "run-to-run results differ"
 
 
 def test_caller_workspace(B):
-    os.environ["UNIQL_DECODE_GS"] = "2"
+    os.environ["UNIQL_DECODE_KP"] = "2"
     rng = np.random.default_rng(8)
     qw = synth.draw_qweight(rng, 96, 1024)
     dw = dev_weight(qw)
@@ -268,7 +268,7 @@ def test_qk_rope_small(B, path, M, keep):
 def test_qk_rope_bf16_table_and_split(B):
     rng = np.random.default_rng(71)
     invf = (1e6 ** (-np.arange(64) / 64.0)) * 0.5          # a caller table (scaled-RoPE variants)
-    os.environ["UNIQL_DECODE_GS"], os.environ["UNIQL_DECODE_TPW"] = "2", "2"
+    os.environ["UNIQL_DECODE_KP"], os.environ["UNIQL_DECODE_RP"] = "2", "7"
     for (g, ref) in run_rope(B, rng, 3, 512, 4, 4, 128, 108, 1e6, "bf16", inv_freq=invf):
         check_output(g, ref, "bf16", TIGHT, "rope bf16 table")
 
