@@ -122,6 +122,12 @@ int uniql_dequant(const uint8_t* packed, const void* scales, const void* zeros, 
  * Calls that share a workspace must not overlap on the device. */
 size_t uniql_workspace_bytes(int M, int K, int N_total);
 int uniql_workspace_init(void* workspace, size_t bytes, void* stream);
+/* Every wait inside the kernels is bounded.  When one expires the kernel stops early and writes
+ * UNIQL_ERR_TIMEOUT into a status word of the workspace it ran with; the outputs of that call are
+ * then incomplete.  This call synchronises the device and copies the word to *status (host):
+ * UNIQL_OK when no wait has expired since the workspace was initialised.  workspace NULL = the
+ * library's buffer of the current device. */
+int uniql_workspace_status(void* workspace, int* status);
 
 /* ---- the quantised, pruned linear layer (Section 3.4; decode and prefill of Section 5) ----
  * Simple form: fp16 x[M][k_in], fp16 y[M][k_out], keep the leading k_in input and k_out

@@ -59,6 +59,7 @@ _lib.uniql_dequant.argtypes = [_vp, _vp, _vp, _i64, _i64, _i, _vp, _vp]
 _lib.uniql_workspace_bytes.restype = _sz
 _lib.uniql_workspace_bytes.argtypes = [_i, _i, _i]
 _lib.uniql_workspace_init.argtypes = [_vp, _sz, _vp]
+_lib.uniql_workspace_status.argtypes = [_vp, ctypes.POINTER(_i)]
 _lib.uniql_qlinear.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp]
 _lib.uniql_qlinear_ex.argtypes = [_vp, _i, _i, _vp, _vp, _vp, _vp, _i, _i, _i, ctypes.POINTER(_ChanMap), _i,
                                   ctypes.POINTER(_ChanMap), _i, _vp, _i, _vp, _sz, _vp]
@@ -67,7 +68,7 @@ _lib.uniql_qlinear_multi.argtypes = [_vp, _i, _i, _i, _i, ctypes.POINTER(_ChanMa
 _lib.uniql_qk_rope_proj.argtypes = [_vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i,
                                     _vp, _vp, _d, ctypes.POINTER(_d), _vp, _i, _vp, _i, _vp, _sz, _vp]
 for _n in ("uniql_set_path", "uniql_pack_u4", "uniql_unpack_u4", "uniql_dequant", "uniql_workspace_init",
-           "uniql_qlinear", "uniql_qlinear_ex", "uniql_qlinear_multi", "uniql_qk_rope_proj"):
+           "uniql_workspace_status", "uniql_qlinear", "uniql_qlinear_ex", "uniql_qlinear_multi", "uniql_qk_rope_proj"):
     getattr(_lib, _n).restype = _i
 
 
@@ -149,6 +150,13 @@ def workspace_bytes(M: int, K: int, N_total: int) -> int:
 def workspace_init(ws: torch.Tensor, stream=None) -> None:
     _check(_lib.uniql_workspace_init(_ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
            "uniql_workspace_init")
+
+
+def workspace_status(ws: Optional[torch.Tensor] = None) -> int:
+    """Device status word of a workspace (None: the library's own); synchronises the device."""
+    out = _i(0)
+    _check(_lib.uniql_workspace_status(_ptr(ws), ctypes.byref(out)), "uniql_workspace_status")
+    return int(out.value)
 
 
 def qlinear(x, packed_w, scales, zeros, M, K, N, k_in, k_out, y, stream=None) -> None:

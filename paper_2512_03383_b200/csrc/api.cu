@@ -140,6 +140,23 @@ extern "C" int uniql_workspace_init(void* workspace, size_t bytes, void* stream)
   return cudaMemsetAsync(workspace, 0, bytes, (cudaStream_t)stream) == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
 }
 
+extern "C" int uniql_workspace_status(void* workspace, int* status) {
+  if (!status) return UNIQL_ERR_NULL;
+  if (!workspace) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return UNIQL_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_ws_mutex);
+    workspace = g_ws[dev];
+    if (!workspace) { *status = UNIQL_OK; return UNIQL_OK; }   // never used: nothing can have failed
+  }
+  int v = 0;
+  if (cudaMemcpy(&v, reinterpret_cast<unsigned char*>(workspace) + decode_status_offset(), sizeof(int),
+                 cudaMemcpyDeviceToHost) != cudaSuccess)
+    return UNIQL_ERR_CUDA;
+  *status = v;
+  return UNIQL_OK;
+}
+
 extern "C" int uniql_qlinear_multi(const void* x, int ldx, int dt, int M, int K, const uniql_chanmap* in_map,
                                    int k_in, int n_jobs, const uniql_job* jobs, void* workspace,
                                    size_t ws_bytes, void* stream) {

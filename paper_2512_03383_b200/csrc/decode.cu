@@ -1,29 +1,34 @@
 // Decode kernel (M = 1..16) of the pruned 4-bit linear layer, sm_100a.
 //
-// The decode step streams every retained weight once (weight-bandwidth bound), so the kernel is
-// organised around 128-bit loads of packed codes straight from the interchange layout: lane (r, c)
-// of a warp loads the 32 codes c*32..c*32+31 of one 128-channel quantisation group for weight rows
-// r and r+8 of a 16-row tile, i.e. exactly the A fragments of eight m16n8k16 tensor-core MMAs whose
-// B fragments are the (permuted) activations.  The contraction index of an MMA is only a label, so
-// the activations are staged in shared memory in the order the nibbles come out of a 32-bit word
-// and no weight byte is ever shuffled.  The MMAs run on the integer codes (code-8 is exact in
-// fp16/bf16); scale and zero-point are applied once per group and row in fp32:
-//   y += s * (sum_k (q_k-8) x_k  -  (z-8) * sum_k x_k),
-// which makes the result independent of the activation dtype's mantissa.
-// Truncation to the leading sorted channels (Section 3.4) is pure index arithmetic: pruned rows are
-// never addressed, pruned input channels are either outside the visited groups or meet a zero
-// activation.
-// Scheduling: one persistent block of 16 warps per SM.  All (row tile, k-chunk) units of the launch
-// form one k-fastest sequence that is cut into equal contiguous ranges, one per warp (stream-K), so
-// every SM streams the same number of bytes and nothing is launched in waves.  A warp keeps the loads
-// of its next chunk in flight while it works on the current one, accumulates in registers while it
-// stays on a tile, and when it leaves a tile that other warps also worked on it parks its partial sum
-// in a workspace slot; the last warp to arrive adds the slots in a fixed order (deterministic, no
-// spinning).  When the activations of a block do not fit in shared memory (large M x K) the input
-// channels are split into k-parts with their own blocks.
-// The rotary epilogue (Section 3.2, fused RoPE) needs both members of a rotation pair: in rope mode
-// a 16-row tile is 8 pairs, first-half members in rows 0..7 and their partners in rows 8..15, which
-// is exactly the (r, r+8) row pair a lane owns in the MMA accumulator layout.
+// The decode step streams every retained weight exactly once, so the kernel is built around keeping
+// HBM busy: one persistent block per SM whose producer warp keeps a ring of shared-memory stages
+// filled by the tensor memory accelerator (cp.async.bulk.tensor boxes of 128 bytes x 64 rows,
+// completion on an mbarrier), far ahead of the sixteen consumer warps.  Neither side spends registers
+// or issue slots on memory latency.  On-device pruning (Section 3.4) is expressed in the tensor maps:
+// a family of kept channel blocks {start, period, keep, count} is a 3-D tensor (byte in row, row in
+// block, block) whose extents stop at the kept rows and at the last visited input group, so pruned
+// rows and pruned trailing input channels are out of bounds: never fetched, filled with zeros.
+//
+// Work decomposition.  A tile is 64 row slots of one kept block, a chunk is 8 quantisation groups
+// (1024 input channels, 512 bytes per row).  All (tile, chunk) units of the launch form one
+// chunk-fastest sequence that is cut into equal contiguous ranges, one per block (stream-K): every SM
+// streams the same number of bytes.  A tile that is shared by several blocks is finished by the last
+// block to arrive, which adds the parked partial sums in a fixed slot order (deterministic, no
+// spinning on other blocks).
+//
+// Arithmetic.  Inside a stage consumer warp w owns group (w & 7) of the chunk and two 16-row
+// sub-tiles.  The packed codes are used as they lie in memory: one LOP3 turns two nibbles of a 32-bit
+// word into an fp16 pair (1024+q for a nibble in bits [3:0], 64+q for one in bits [7:4]) and those
+// pairs are the A fragments of m16n8k16 tensor-core MMAs whose B fragments are the activations.  The
+// contraction index of an MMA is only a label, so the activations are staged once per block in shared
+// memory in the order the nibbles come out of a word and no weight byte is ever shuffled.  The
+// offsets, the zero-point and the scale are applied once per group and row in fp32:
+//     y += s * ( sum_k (o_k + q_k) x_k  -  (sum_k o_k x_k  +  z * sum_k x_k) ),   o_k in {1024, 64}.
+// The rotary epilogue (Section 3.2, fused RoPE) needs both members of a rotation pair; in rope mode a
+// tile is 32 pairs of one head, first-half members in row slots 0..31 and their partners in 32..63.
+//
+// Every wait in the kernel is an mbarrier wait with an iteration limit; when one expires the block
+// sets the status word of the workspace, lets its copies land and returns.
 #include <stdlib.h>
 #include <string.h>
 
@@ -32,509 +37,533 @@
 namespace uniql {
 namespace {
 
-constexpr int NW = 16;            // warps per block
-constexpr int NTD = NW * 32;      // threads per block
-constexpr int kMaxSpans = kMaxFam;
-constexpr int kCounterInts = 1 << 16;   // arrival counters (one per row tile) at the head of the workspace
+constexpr int CW = 16;                  // consumer warps
+constexpr int CTH = CW * 32;            // consumer threads
+constexpr int NTH = CTH + 32;           // + one producer warp
+constexpr int RB = 64;                  // row slots per tile
+constexpr int CG = 8;                   // groups per chunk
+constexpr int WPITCH = CG * 64 + 64;    // bytes between row slots of a stage (the 64 keeps lane pairs on distinct banks)
+constexpr int STAGE_W = RB * WPITCH;
+constexpr int STAGE_SZ = RB * CG * 2;   // one of the two fp16 arrays [RB][CG]
+constexpr int STAGE_BYTES = STAGE_W + 2 * STAGE_SZ;
+constexpr int MAX_STAGES = 5;
+constexpr int kCounterInts = 1 << 16;   // arrival counters (one per tile) at the head of the workspace
+constexpr int kStatusOff = kCounterInts * 4;   // status word right after the counters
+constexpr int kWsHeader = kStatusOff + 256;
 constexpr int kMaxKParts = 16;
-constexpr size_t kSmemBudget = 200 * 1024;
+constexpr int kSmemMax = 227 * 1024;
+constexpr int kWaitLimit = 1 << 18;
+constexpr int BAR_BYTES = 128;
 
 struct DecodeCfg {
-  int n_kp, n_rp;        // k-parts x row-parts = blocks
+  int n_kp, n_rp;        // k-parts x blocks per k-part
   int gp;                // visited groups per k-part (the last part may be shorter)
+  int g_total;           // visited groups
+  int v_first;           // first visited stored group
+  int gran;              // groups per scale / zero-point copy granule (2 or 4)
+  int stages;
   int tiles_total;
-  int tile_begin[kMaxJobs + 1];   // first global tile of each job
-  int row_base[kMaxJobs];         // (unused by the kernel; kept for sizing)
-  int g_total;           // visited 128-channel groups
-  int n_spans;
-  int vg_begin[kMaxSpans + 1];  // visit index at which span s starts
-  int vg_first[kMaxSpans];      // its first stored group
+  int tile_begin[kMaxJobs + 1];
   int x_vec;             // activations can be staged with 128-bit loads
-  int sz_vec;            // scales / zero-points of a chunk can be fetched with one vector load
-  int mp;                // activation rows staged in shared memory
   int max_slots;         // workspace slots per tile
+  int off_x, xrow, off_xg, off_part, part_bufs;
   int* counters;
   float* partials;
+  int* status;
 };
 
-__device__ inline int visit_to_group(const DecodeCfg& c, int v) {
-  int s = 0;
-  while (s + 1 < c.n_spans && v >= c.vg_begin[s + 1]) ++s;
-  return c.vg_first[s] + (v - c.vg_begin[s]);
+// ---------------------------------------------------------------------------------------- PTX helpers
+__device__ inline void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-
-__device__ inline uint4 ldg_stream(const void* ptr) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(ptr));
-  return v;
+__device__ inline void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ inline void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ inline bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the limit expired or another warp of the block already gave up.
+__device__ inline bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (int i = 0; i < kWaitLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63) == 63 && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ inline void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ inline void cp_async8(uint32_t dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ inline void cp_async4(uint32_t dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ inline void cp_async_arrive_noinc(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 __device__ inline uint4 lds128(uint32_t addr) {
   uint4 v;
   asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
   return v;
 }
-__device__ inline float2 lds64f(uint32_t addr) {
-  float2 v;
-  asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+__device__ inline float4 lds128f(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
   return v;
 }
-
+__device__ inline float lds_h(uint32_t addr) {
+  unsigned short h;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(addr));
+  return __half2float(__ushort_as_half(h));
+}
 // (a & mask) | magic in one LOP3 (truth table 0xEA)
 __device__ inline uint32_t and_or(uint32_t a, uint32_t mask, uint32_t magic) {
   uint32_t d;
   asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(mask), "r"(magic));
   return d;
 }
-
-template <typename T> struct Cvt;
-// fp16: a nibble in bits [3:0] of a 16-bit half ORed onto 0x6400 reads 1024+q, one in bits [7:4]
-// ORed onto 0x5400 reads 64+q; subtracting 1032 / 72 leaves q-8 exactly.
-template <> struct Cvt<__half> {
-  static __device__ inline void word(uint32_t w, uint32_t (&a)[4]) {
-    const uint32_t k_lo = 0x64086408u, k_hi = 0x54805480u;   // 1032, 72
-    const uint32_t w8 = w >> 8;
-    const uint32_t t0 = and_or(w, 0x000f000fu, 0x64006400u);
-    const uint32_t t1 = and_or(w, 0x00f000f0u, 0x54005400u);
-    const uint32_t t2 = and_or(w8, 0x000f000fu, 0x64006400u);
-    const uint32_t t3 = and_or(w8, 0x00f000f0u, 0x54005400u);
-    asm("sub.f16x2 %0, %1, %2;" : "=r"(a[0]) : "r"(t0), "r"(k_lo));
-    asm("sub.f16x2 %0, %1, %2;" : "=r"(a[1]) : "r"(t1), "r"(k_hi));
-    asm("sub.f16x2 %0, %1, %2;" : "=r"(a[2]) : "r"(t2), "r"(k_lo));
-    asm("sub.f16x2 %0, %1, %2;" : "=r"(a[3]) : "r"(t3), "r"(k_hi));
-  }
-  static __device__ inline void mma(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                    uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-  }
-  static __device__ inline void mma0(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                     uint32_t b0, uint32_t b1) {   // d = a*b (zero accumulator input)
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
-  }
-};
-// bf16 has 7 mantissa bits: only a nibble in bits [3:0] can be ORed onto 0x4300 (128+q).
-template <> struct Cvt<__nv_bfloat16> {
-  static __device__ inline void word(uint32_t w, uint32_t (&a)[4]) {
-    const uint32_t k136 = 0x43084308u;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const uint32_t t = and_or(w >> (4 * i), 0x000f000fu, 0x43004300u);
-      asm("sub.bf16x2 %0, %1, %2;" : "=r"(a[i]) : "r"(t), "r"(k136));
-    }
-  }
-  static __device__ inline void mma(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                    uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-  }
-  static __device__ inline void mma0(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                     uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
-  }
-};
-
-// The two weight rows a lane owns in a 16-row tile.
-struct LaneRows {
-  int sr0, sr1;      // stored rows (clamped to a valid row when the slot is empty)
-  int oc0, oc1;      // compact output columns, -1 when empty
-  int rope_p, rope_kvh;
-};
-
-__device__ inline LaneRows resolve_rows(const JobDev& jb, int tile, int r) {
-  LaneRows L;
-  L.rope_p = 0; L.rope_kvh = 0;
-  if (jb.rope.enabled) {
-    const int half = jb.rope.head_keep >> 1;
-    const int P = tile * 8 + r;
-    const bool ok = P < jb.rope.n_heads * half;
-    const int Pc = ok ? P : 0;
-    const int h = Pc / half, cc = Pc - h * half;
-    L.sr0 = h * jb.rope.head_dim + cc;
-    L.sr1 = L.sr0 + (jb.rope.head_dim >> 1);
-    L.oc0 = ok ? h * jb.rope.head_keep + cc : -1;
-    L.oc1 = ok ? L.oc0 + half : -1;
-    L.rope_p = cc;
-    L.rope_kvh = h / jb.rope.rep;
-  } else {
-    const int j0 = tile * 16 + r, j1 = j0 + 8;
-    L.oc0 = j0 < jb.k_out ? j0 : -1;
-    L.oc1 = j1 < jb.k_out ? j1 : -1;
-    if (jb.omap.n_fam == 1 && jb.omap.fam[0].count == 1) {
-      L.sr0 = jb.omap.fam[0].start + (L.oc0 >= 0 ? j0 : 0);
-      L.sr1 = jb.omap.fam[0].start + (L.oc1 >= 0 ? j1 : 0);
-    } else {
-      L.sr0 = map_compact_to_stored(jb.omap, L.oc0 >= 0 ? j0 : 0);
-      L.sr1 = map_compact_to_stored(jb.omap, L.oc1 >= 0 ? j1 : 0);
-    }
-  }
-  return L;
+// Eight codes of a 32-bit word as four fp16 pairs: (c0,c4)+1024, (c1,c5)+64, (c2,c6)+1024, (c3,c7)+64.
+__device__ inline void cvt_word(uint32_t w, uint32_t (&a)[4]) {
+  const uint32_t w8 = w >> 8;
+  a[0] = and_or(w, 0x000f000fu, 0x64006400u);
+  a[1] = and_or(w, 0x00f000f0u, 0x54005400u);
+  a[2] = and_or(w8, 0x000f000fu, 0x64006400u);
+  a[3] = and_or(w8, 0x00f000f0u, 0x54005400u);
+}
+__device__ inline void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                               uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// bias, rotary embedding on the retained pair, one rounding, store
-template <typename T, int MT>
-__device__ inline void epilogue(const Params& p, const JobDev& jb, const LaneRows& L, int cq, float (&out)[MT][4]) {
-  const T* bias = reinterpret_cast<const T*>(jb.bias);
-  const float b0 = (bias && L.oc0 >= 0) ? DT<T>::to_f(bias[L.sr0]) : 0.f;
-  const float b1 = (bias && L.oc1 >= 0) ? DT<T>::to_f(bias[L.sr1]) : 0.f;
-  T* y = reinterpret_cast<T*>(jb.y);
-  double invf = 0.0;
+// ---------------------------------------------------------------------------------------- tile geometry
+__device__ inline int job_of(const DecodeCfg& c, int n_jobs, int tg) {
+  int j = 0;
+  while (j + 1 < n_jobs && tg >= c.tile_begin[j + 1]) ++j;
+  return j;
+}
+
+// Stored weight row of row slot `slot` of local tile `tile` of a job, or -1 when the slot is empty.
+__device__ inline int slot_to_stored(const JobDev& jb, int tile, int slot) {
   if (jb.rope.enabled) {
-    int pidx = p.idx[L.rope_kvh * (jb.rope.head_keep >> 1) + L.rope_p];
-    pidx = min(max(pidx, 0), (jb.rope.head_dim >> 1) - 1);
-    invf = p.inv_freq[pidx];
+    const int half = jb.rope.head_keep >> 1;
+    const int P = tile * (RB / 2) + (slot & (RB / 2 - 1));
+    if (P >= jb.rope.n_heads * half) return -1;
+    const int h = P / half, cc = P - h * half;
+    return h * jb.rope.head_dim + ((slot >= RB / 2) ? (jb.rope.head_dim >> 1) : 0) + cc;
   }
-#pragma unroll
-  for (int t = 0; t < MT; ++t)
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const int m = 2 * cq + e + 8 * t;
-      if (m >= p.M) continue;
-      float lo = out[t][e] + b0, hi = out[t][2 + e] + b1;
-      if (jb.rope.enabled) {
-        float cs, sn;
-        rope_cos_sin(p.pos[m], invf, cs, sn);
-        const float a = lo, b = hi;
-        lo = a * cs - b * sn;
-        hi = b * cs + a * sn;
+  const int j = tile * RB + slot;
+  if (j >= jb.k_out) return -1;
+  if (jb.omap.n_fam == 1 && jb.omap.fam[0].count == 1) return jb.omap.fam[0].start + j;
+  return map_compact_to_stored(jb.omap, j);
+}
+
+// The block (of its k-part) whose unit range [U*b/B, U*(b+1)/B) holds unit u; exact in fp64 here.
+__device__ inline int owner_of(long u, long B, long U) {
+  return (int)floor(((double)(u + 1) * (double)B - 1.0) / (double)U);
+}
+
+// bias, rotary embedding on the retained pair, one rounding, store; `get(slot, m)` yields the fp32 sum
+template <typename T, typename F>
+__device__ inline void store_tile(const Params& p, const JobDev& jb, int tile, int ctid, F get) {
+  const T* bias = reinterpret_cast<const T*>(jb.bias);
+  T* y = reinterpret_cast<T*>(jb.y);
+  if (jb.rope.enabled) {
+    const int half = jb.rope.head_keep >> 1;
+    const int n_pairs = jb.rope.n_heads * half;
+    for (int i = ctid; i < (RB / 2) * p.M; i += CTH) {
+      const int pp = i & (RB / 2 - 1), m = i / (RB / 2);
+      const int P = tile * (RB / 2) + pp;
+      if (P >= n_pairs) continue;
+      const int h = P / half, cc = P - h * half;
+      float lo = get(pp, m), hi = get(pp + RB / 2, m);
+      if (bias) {
+        const int sr = h * jb.rope.head_dim + cc;
+        lo += DT<T>::to_f(bias[sr]);
+        hi += DT<T>::to_f(bias[sr + (jb.rope.head_dim >> 1)]);
       }
-      if (L.oc0 >= 0) y[(size_t)m * jb.ldy + L.oc0] = DT<T>::from_f(lo);
-      if (L.oc1 >= 0) y[(size_t)m * jb.ldy + L.oc1] = DT<T>::from_f(hi);
+      int pidx = p.idx[(h / jb.rope.rep) * half + cc];
+      pidx = min(max(pidx, 0), (jb.rope.head_dim >> 1) - 1);
+      float cs, sn;
+      rope_cos_sin(p.pos[m], p.inv_freq[pidx], cs, sn);
+      const int oc = h * jb.rope.head_keep + cc;
+      y[(size_t)m * jb.ldy + oc] = DT<T>::from_f(lo * cs - hi * sn);
+      y[(size_t)m * jb.ldy + oc + half] = DT<T>::from_f(hi * cs + lo * sn);
     }
+  } else {
+    for (int i = ctid; i < RB * p.M; i += CTH) {
+      const int slot = i & (RB - 1), m = i / RB;
+      const int j = tile * RB + slot;
+      if (j >= jb.k_out) continue;
+      float v = get(slot, m);
+      if (bias) v += DT<T>::to_f(bias[slot_to_stored(jb, tile, slot)]);
+      y[(size_t)m * jb.ldy + j] = DT<T>::from_f(v);
+    }
+  }
 }
 
 // ---------------------------------------------------------------------------------------- kernel
-__device__ inline int owner_of(long u, long W, long U) {
-  // the warp whose range [U*w/W, U*(w+1)/W) holds unit u; exact in fp64 for these magnitudes
-  return (int)floor(((double)(u + 1) * (double)W - 1.0) / (double)U);
-}
-
-// A warp leaves tile `tgl`: finish it alone, or park the partial sum in its workspace slot and let the
-// last warp to arrive add all slots in slot order and finish.  Kept out of line: it runs once or twice
-// per warp and would only bloat the streaming loop.  Everything is passed by value so that the caller's
-// accumulators stay in registers.
-constexpr int MT_MAX = 2;
-struct OutVals { float v[MT_MAX][4]; };
-template <typename T, int MT, int CH>
-__device__ __noinline__ void flush_tile(const Params& p, const DecodeCfg& c, int kp, int gw, int tgl, int jl,
-                                        const LaneRows Ll, int lane, const OutVals ov) {
-  const int r = lane >> 2, cq = lane & 3;
-  float out[MT][4];
-#pragma unroll
-  for (int t = 0; t < MT; ++t)
-#pragma unroll
-    for (int i = 0; i < 4; ++i) out[t][i] = ov.v[t][i];
-  const long Wall = (long)c.n_rp * NW;
-  int total = 0, my_slot = 0;
-  for (int q = 0; q < c.n_kp; ++q) {
-    const int Gq = min(c.gp, c.g_total - q * c.gp);
-    const long Cq = (Gq + CH - 1) / CH;
-    const long Uq = (long)c.tiles_total * Cq;
-    const long Wq = Wall < Uq ? Wall : Uq;
-    const int first = owner_of((long)tgl * Cq, Wq, Uq);
-    const int last = owner_of((long)tgl * Cq + Cq - 1, Wq, Uq);
-    if (q == kp) my_slot = total + (gw - first);
-    total += last - first + 1;
-  }
-  if (total == 1) {
-    epilogue<T, MT>(p, p.job[jl], Ll, cq, out);
-    return;
-  }
-  const size_t slot_floats = (size_t)p.M * 16;
-  float* tile_part = c.partials + (size_t)tgl * c.max_slots * slot_floats;
-  float* mine = tile_part + (size_t)my_slot * slot_floats;
-#pragma unroll
-  for (int t = 0; t < MT; ++t)
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const int m = 2 * cq + e + 8 * t;
-      if (m >= p.M) continue;
-      __stcg(mine + m * 16 + r, out[t][e]);
-      __stcg(mine + m * 16 + r + 8, out[t][2 + e]);
-    }
-  __threadfence();
-  __syncwarp();
-  int last_arrival = 0;
-  if (lane == 0) last_arrival = atomicAdd(&c.counters[tgl], 1) == total - 1;
-  last_arrival = __shfl_sync(0xffffffffu, last_arrival, 0);
-  if (!last_arrival) return;
-  __threadfence();
-#pragma unroll
-  for (int t = 0; t < MT; ++t)
-#pragma unroll
-    for (int i = 0; i < 4; ++i) out[t][i] = 0.f;
-  for (int s2 = 0; s2 < total; ++s2) {
-    const float* src = tile_part + (size_t)s2 * slot_floats;
-#pragma unroll
-    for (int t = 0; t < MT; ++t)
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int m = 2 * cq + e + 8 * t;
-        if (m >= p.M) continue;
-        out[t][e] += __ldcg(src + m * 16 + r);
-        out[t][2 + e] += __ldcg(src + m * 16 + r + 8);
-      }
-  }
-  epilogue<T, MT>(p, p.job[jl], Ll, cq, out);
-  if (lane == 0) c.counters[tgl] = 0;       // ready for the next call
-}
-
-template <typename T, int MT, int CH>
-__global__ void __launch_bounds__(NTD, 1) decode_kernel(const __grid_constant__ Params p,
+template <int MT, bool ONECOL>
+__global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ Params p,
                                                         const __grid_constant__ DecodeCfg c) {
-  extern __shared__ __align__(16) unsigned char smem[];
+  extern __shared__ __align__(128) unsigned char smem[];
+  using T = __half;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int r = lane >> 2, cq = lane & 3;
-  const int mp = c.mp;
+  const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(smem);
+  const int S = c.stages;
+  // barriers: full[S], empty[S], consumer barrier; then two flags
+  const uint32_t bar_full = sbase, bar_empty = sbase + 8 * MAX_STAGES, bar_cons = sbase + 16 * MAX_STAGES;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 16 * MAX_STAGES + 8);
+  volatile int* last_flag = reinterpret_cast<volatile int*>(smem + 16 * MAX_STAGES + 12);
+  const uint32_t stage0 = sbase + BAR_BYTES;
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(bar_full + 8 * s, 33);      // one expect_tx arrival + 32 copy-completion arrivals
+      mbar_init(bar_empty + 8 * s, CW);
+    }
+    mbar_init(bar_cons, CW);
+    *abort_flag = 0;
+    *last_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
   const int kp = blockIdx.x / c.n_rp, rp = blockIdx.x - kp * c.n_rp;
   const int v_lo = kp * c.gp;                                   // first visit index of this k-part
   const int Gk = min(c.gp, c.g_total - v_lo);                   // its groups
-  const int Ck = (Gk + CH - 1) / CH;                            // chunks per tile
-  // shared memory: staged activations, mp rows + one all-zero row of (gp*256+64) bytes each (a group is
-  // 256 bytes; the 64-byte pad puts the two rows met by one 128-bit load phase on distinct banks), then
-  // the per-group activation sums [gp][8*MT] fp32
-  const int row_bytes = c.gp * 256 + 64;
-  const int xg_off = (mp + 1) * row_bytes;
-  float* xg = reinterpret_cast<float*>(smem + xg_off);
-  const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
-  const int sg_lo = visit_to_group(c, v_lo);
-  const bool contig = visit_to_group(c, v_lo + Gk - 1) == sg_lo + Gk - 1;   // block-uniform
-
-  // ---- this warp's contiguous range of (tile, chunk) units, k fastest
-  const long U = (long)c.tiles_total * Ck;
-  const long Wall = (long)c.n_rp * NW;
-  const long W = Wall < U ? Wall : U;                           // warps that get work
-  const int gw = rp * NW + warp;
-  int ub = 0, ue = 0;
-  if (gw < W) { ub = (int)(U * gw / W); ue = (int)(U * (gw + 1) / W); }
-
+  const int Ck = (Gk + CG - 1) / CG;                            // chunks per tile
+  const int sg_lo = c.v_first + v_lo;                           // first stored group of this k-part
   const int G = p.K / kGroup;
-  auto job_of = [&](int tg) { int j = 0; while (j + 1 < p.n_jobs && tg >= c.tile_begin[j + 1]) ++j; return j; };
+  const long U = (long)c.tiles_total * Ck;
+  const long Bn = (long)c.n_rp < U ? (long)c.n_rp : U;          // blocks that get work
+  int ub = 0, ue = 0;
+  if (rp < Bn) { ub = (int)(U * rp / Bn); ue = (int)(U * (rp + 1) / Bn); }
+  if (ub >= ue) return;
 
-  // packed codes of the CH groups of the current chunk (reloaded in place, group by group, with the
-  // next chunk's codes as soon as a group has been consumed) and fp16 scale / zero pairs
-  uint4 w0[CH], w1[CH];
-  uint32_t sc[4][CH / 2], scn[4][CH / 2];   // s(row r), z(row r), s(row r+8), z(row r+8); two groups per word
-
-  auto load_group = [&](int g, const uint8_t* q0, const uint8_t* q1, int chn) {
-    // q0/q1: row pointers already advanced to this lane's 16 bytes of stored group sg_lo (contiguous case)
-    const int gi = chn * CH + g;
-    if (gi < Gk) {
-      const size_t off = (size_t)(contig ? sg_lo + gi : visit_to_group(c, v_lo + gi)) * 64;
-      w0[g] = ldg_stream(q0 + off);
-      w1[g] = ldg_stream(q1 + off);
-    }
-  };
-  auto load_scales = [&](uint32_t (&dst)[4][CH / 2], const JobDev& jb, const LaneRows& L, int chn) {
-    const int g0 = chn * CH;
-    const __half* base[4] = {jb.scales + (size_t)L.sr0 * G, jb.zeros + (size_t)L.sr0 * G,
-                             jb.scales + (size_t)L.sr1 * G, jb.zeros + (size_t)L.sr1 * G};
-    if (c.sz_vec) {     // chunk start is CH-aligned in stored groups and the CH values are contiguous
+  // ======================================================================================= producer
+  if (warp == CW) {
+    int tile = ub / Ck, chunk = ub - tile * Ck;
+    int jn = -1, tile_prev = -1;
+    const uint8_t* wrow[2] = {nullptr, nullptr};
+    const __half* srow[2] = {nullptr, nullptr};
+    const __half* zrow[2] = {nullptr, nullptr};
+    int n_valid = 0;
+    int it = 0;
+    bool ok = true;
+    for (int u = ub; u < ue; ++u, ++it) {
+      const int s = it % S;
+      if (it >= S) ok = mbar_wait(bar_empty + 8 * s, ((it / S) - 1) & 1, abort_flag);
+      if (!ok) break;
+      if (tile != tile_prev) {
+        jn = job_of(c, p.n_jobs, tile);
+        const JobDev& jb = p.job[jn];
+        const int tl = tile - c.tile_begin[jn];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        if constexpr (CH == 4) {
-          const uint2 v = __ldg(reinterpret_cast<const uint2*>(base[q] + sg_lo + g0));
-          dst[q][0] = v.x; dst[q][1] = v.y;
-        } else {
-          dst[q][0] = __ldg(reinterpret_cast<const uint32_t*>(base[q] + sg_lo + g0));
+        for (int q = 0; q < 2; ++q) {
+          const int sr = slot_to_stored(jb, tl, lane + 32 * q);
+          wrow[q] = sr >= 0 ? jb.w + (size_t)sr * (p.K / 2) + (size_t)sg_lo * 64 : nullptr;
+          srow[q] = sr >= 0 ? jb.scales + (size_t)sr * G + sg_lo : nullptr;
+          zrow[q] = sr >= 0 ? jb.zeros + (size_t)sr * G + sg_lo : nullptr;
+        }
+        n_valid = __popc(__ballot_sync(0xffffffffu, wrow[0] != nullptr)) +
+                  __popc(__ballot_sync(0xffffffffu, wrow[1] != nullptr));
+        tile_prev = tile;
+      }
+      const int ng = min(CG, Gk - chunk * CG);
+      const uint32_t full = bar_full + 8 * s;
+      const uint32_t st = stage0 + (uint32_t)s * STAGE_BYTES;
+      if (lane == 0) mbar_expect_tx(full, (uint32_t)(n_valid * ng * 64));
+      __syncwarp();
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        if (wrow[q]) {
+          const int slot = lane + 32 * q;
+          bulk_g2s(st + slot * WPITCH, wrow[q] + (size_t)chunk * (CG * 64), (uint32_t)(ng * 64), full);
+          const uint32_t sd = st + STAGE_W + slot * (CG * 2), zd = sd + STAGE_SZ;
+          const __half* sp = srow[q] + chunk * CG;
+          const __half* zp = zrow[q] + chunk * CG;
+          if (c.gran == 4) {
+            for (int g4 = 0; g4 < ng; g4 += 4) { cp_async8(sd + g4 * 2, sp + g4); cp_async8(zd + g4 * 2, zp + g4); }
+          } else {
+            for (int g2 = 0; g2 < ng; g2 += 2) { cp_async4(sd + g2 * 2, sp + g2); cp_async4(zd + g2 * 2, zp + g2); }
+          }
         }
       }
-    } else {
-      const int nv = min(CH, Gk - g0);
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-#pragma unroll
-        for (int g = 0; g < CH; g += 2) {
-          const int ga = visit_to_group(c, v_lo + g0 + (g < nv ? g : 0));
-          const int gb = visit_to_group(c, v_lo + g0 + (g + 1 < nv ? g + 1 : 0));
-          const uint32_t lo = __half_as_ushort(__ldg(base[q] + ga));
-          const uint32_t hi = __half_as_ushort(__ldg(base[q] + gb));
-          dst[q][g >> 1] = lo | (hi << 16);
-        }
+      cp_async_arrive_noinc(full);
+      if (++chunk == Ck) { chunk = 0; ++tile; }
     }
-  };
-
-  // the first chunk's loads go out before the activations are staged (they do not depend on them)
-  int tg = 0, ch = 0, jn = 0;
-  LaneRows L;
-  if (ub < ue) {
-    tg = ub / Ck; ch = ub - tg * Ck;
-    jn = job_of(tg);
-    L = resolve_rows(p.job[jn], tg - c.tile_begin[jn], r);
-    const uint8_t* q0 = p.job[jn].w + (size_t)L.sr0 * (p.K / 2) + cq * 16;
-    const uint8_t* q1 = p.job[jn].w + (size_t)L.sr1 * (p.K / 2) + cq * 16;
-#pragma unroll
-    for (int g = 0; g < CH; ++g) load_group(g, q0, q1, ch);
-    load_scales(sc, p.job[jn], L, ch);
+    if (!ok) {
+      // let the copies of the stages that are still armed land before the block goes away
+      const int first = it > S ? it - S : 0;
+      for (int j = first; j < it; ++j) {
+        const uint32_t full = bar_full + 8 * (j % S);
+        for (int i = 0; i < kWaitLimit && !mbar_try_wait(full, (j / S) & 1); ++i) {}
+      }
+      if (lane == 0) atomicExch(c.status, UNIQL_ERR_TIMEOUT);
+    }
+    return;
   }
 
-  // ---- stage activations: permuted into nibble order, zero where the channel is pruned
+  // ======================================================================================= consumers
+  const int ctid = tid;                    // 0..CTH-1
+  const int g = lane >> 2, t = lane & 3;
+  const int kpw = warp & 7, rg = warp >> 3;
+  uint32_t cons_parity = 0;
+  auto consumer_sync = [&]() -> bool {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_cons);
+    const bool ok = mbar_wait(bar_cons, cons_parity, abort_flag);
+    cons_parity ^= 1;
+    return ok;
+  };
+
+  // ---- stage activations: permuted into nibble order, zero where the channel is pruned; per group and
+  //      batch row the two sums the offset / zero-point correction needs, stored negated
   {
     const T* x = reinterpret_cast<const T*>(p.x);
-    uint4* xs = reinterpret_cast<uint4*>(smem);
-    const int row_units = row_bytes / 16;
-    for (int i = tid; i < row_units; i += NTD) xs[mp * row_units + i] = make_uint4(0, 0, 0, 0);
-    for (int i = tid; i < c.gp * 8 * MT; i += NTD) xg[i] = 0.f;
-    __syncthreads();
+    const int row_units = c.xrow / 16;
+    uint4* xs = reinterpret_cast<uint4*>(smem + c.off_x);
+    float2* xg = reinterpret_cast<float2*>(smem + c.off_xg);
+    for (int i = ctid; i < Gk * 8 * MT; i += CTH) xg[i] = make_float2(0.f, 0.f);
+    if (!consumer_sync()) return;
     if (c.x_vec) {
       const int start = p.imap.fam[0].start, keep = p.imap.fam[0].keep;
-      const int n_units = Gk * mp * 16;
-      for (int u = tid; u < ((n_units + 31) & ~31); u += NTD) {   // whole warps stay in the shuffles
+      const int n_units = Gk * p.M * 16;
+      for (int u = ctid; u < ((n_units + 31) & ~31); u += CTH) {   // whole warps stay in the shuffles
         const bool in_range = u < n_units;
         const int u16 = u & 15, pair = in_range ? u >> 4 : 0;
         const int m = pair / Gk, lv = pair - m * Gk;
         uint4 in = make_uint4(0, 0, 0, 0);
-        if (in_range && m < p.M) {
-          const int t0 = (contig ? sg_lo + lv : visit_to_group(c, v_lo + lv)) * kGroup + 8 * u16 - start;
+        if (in_range) {
+          const int t0 = (sg_lo + lv) * kGroup + 8 * u16 - start;
           if (t0 >= 0 && t0 < keep) in = *reinterpret_cast<const uint4*>(x + (size_t)m * p.ldx + t0);
         }
         uint4 o;
         o.x = __byte_perm(in.x, in.z, 0x5410); o.y = __byte_perm(in.x, in.z, 0x7632);
         o.z = __byte_perm(in.y, in.w, 0x5410); o.w = __byte_perm(in.y, in.w, 0x7632);
-        // unit (chunk c', word j) of a group sits at byte j*64 + c'*16; u16 = c'*4 + j
+        // the 16 bytes of lane quarter c', word j of a group sit at byte j*64 + c'*16; u16 = c'*4 + j
         if (in_range) xs[m * row_units + lv * 16 + (u16 & 3) * 4 + (u16 >> 2)] = o;
-        const typename DT<T>::T2* h2 = reinterpret_cast<const typename DT<T>::T2*>(&in);
-        float sum = 0.f;
+        const __half2* h2 = reinterpret_cast<const __half2*>(&in);
+        float se = 0.f, so = 0.f;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) { float2 f = DT<T>::to_f2(h2[i]); sum += f.x + f.y; }
+        for (int i = 0; i < 4; ++i) { const float2 f = __half22float2(h2[i]); se += f.x; so += f.y; }
 #pragma unroll
-        for (int o2 = 8; o2 >= 1; o2 >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o2);
-        if (in_range && u16 == 0) xg[lv * 8 * MT + m] = sum;
+        for (int o2 = 8; o2 >= 1; o2 >>= 1) {
+          se += __shfl_xor_sync(0xffffffffu, se, o2);
+          so += __shfl_xor_sync(0xffffffffu, so, o2);
+        }
+        if (in_range && u16 == 0) xg[lv * 8 * MT + m] = make_float2(-(se + so), -(1024.f * se + 64.f * so));
       }
     } else {
-      T* xh = reinterpret_cast<T*>(smem);
-      const int n_pairs = Gk * mp;
-      for (int pair = warp; pair < n_pairs; pair += NW) {
+      T* xh = reinterpret_cast<T*>(smem + c.off_x);
+      const int n_pairs = Gk * p.M;
+      for (int pair = warp; pair < n_pairs; pair += CW) {
         const int m = pair / Gk, lv = pair - m * Gk;
-        const bool live = m < p.M;
-        const int kbase = visit_to_group(c, v_lo + lv) * kGroup;
-        float sum = 0.f;
+        const int kbase = (sg_lo + lv) * kGroup;
+        float se = 0.f, so = 0.f;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           const int i = lane + 32 * q;
-          T val = DT<T>::from_f(0.f);
-          if (live) {
-            const int t = map_stored_to_compact(p.imap, kbase + i);
-            if (t >= 0) val = x[(size_t)m * p.ldx + t];
-          }
+          T val = __float2half_rn(0.f);
+          const int tt = map_stored_to_compact(p.imap, kbase + i);
+          if (tt >= 0) val = x[(size_t)m * p.ldx + tt];
           const int ccq = i >> 5, j = (i & 31) >> 3, e = i & 7;
           xh[(m * row_units + lv * 16 + j * 4 + ccq) * 8 + 2 * (e & 3) + (e >> 2)] = val;
-          sum += DT<T>::to_f(val);
+          if (i & 1) so += __half2float(val); else se += __half2float(val);
         }
 #pragma unroll
-        for (int o2 = 16; o2 >= 1; o2 >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o2);
-        if (lane == 0) xg[lv * 8 * MT + m] = sum;
+        for (int o2 = 16; o2 >= 1; o2 >>= 1) {
+          se += __shfl_xor_sync(0xffffffffu, se, o2);
+          so += __shfl_xor_sync(0xffffffffu, so, o2);
+        }
+        if (lane == 0) xg[lv * 8 * MT + m] = make_float2(-(se + so), -(1024.f * se + 64.f * so));
       }
     }
+    if (!consumer_sync()) return;
   }
-  __syncthreads();
-  if (ub >= ue) return;
 
-  // per-lane shared-memory address of the B fragments (lanes beyond the staged rows read the zero row)
-  uint32_t xb_addr[MT];
+  // per-lane shared-memory addresses
+  uint32_t xaddr[MT];
+  bool xlive[MT];
 #pragma unroll
-  for (int t = 0; t < MT; ++t) {
-    const int m = r + 8 * t;
-    xb_addr[t] = smem_base + (uint32_t)((m < mp ? m : mp) * row_bytes + cq * 16);
+  for (int mt = 0; mt < MT; ++mt) {
+    const int m = g + 8 * mt;
+    xlive[mt] = m < p.M;
+    xaddr[mt] = sbase + c.off_x + (uint32_t)((xlive[mt] ? m : 0) * c.xrow + t * 16);
   }
-  const uint32_t xg_addr = smem_base + (uint32_t)xg_off + (uint32_t)(2 * cq * 4);
+  const uint32_t xgaddr = sbase + c.off_xg + (uint32_t)(2 * t * 8);
+  const uint32_t wl_off = (uint32_t)((rg * 32 + g) * WPITCH + kpw * 64 + t * 16);
+  const uint32_t sl_off = (uint32_t)(STAGE_W + (rg * 32 + g) * (CG * 2) + kpw * 2);
+  float* part = reinterpret_cast<float*>(smem + c.off_part);
+  const int part_stride = CG * RB * p.M;     // floats per partial buffer
 
-  float out[MT][4];
+  float out[2][MT][4];
 #pragma unroll
-  for (int t = 0; t < MT; ++t)
+  for (int sub = 0; sub < 2; ++sub)
 #pragma unroll
-    for (int i = 0; i < 4; ++i) out[t][i] = 0.f;
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) out[sub][mt][i] = 0.f;
 
-  // ---- stream the units: while group g of the current chunk is consumed, group g of the next chunk
-  //      is already being fetched into the registers group g-1 has just freed
-  for (int u = ub;; ++u) {
-    const bool has_next = u + 1 < ue;
-    int tg1 = tg, ch1 = ch + 1, jn1 = jn;
-    LaneRows L1 = L;
-    if (ch1 == Ck) { ch1 = 0; tg1 = tg + 1; }
-    const uint8_t* q0 = nullptr;
-    const uint8_t* q1 = nullptr;
-    if (has_next) {
-      if (tg1 != tg) {
-        jn1 = job_of(tg1);
-        L1 = resolve_rows(p.job[jn1], tg1 - c.tile_begin[jn1], r);
+  int tile = ub / Ck, chunk = ub - tile * Ck;
+  int it = 0, tiles_done = 0;
+  for (int u = ub; u < ue; ++u, ++it) {
+    const int s = it % S;
+    if (!mbar_wait(bar_full + 8 * s, (it / S) & 1, abort_flag)) return;
+    const int gi = chunk * CG + kpw;
+    if (gi < Gk) {
+      const uint32_t st = stage0 + (uint32_t)s * STAGE_BYTES;
+      uint4 wa[2], wb[2];
+#pragma unroll
+      for (int sub = 0; sub < 2; ++sub) {
+        wa[sub] = lds128(st + wl_off + sub * 16 * WPITCH);
+        wb[sub] = lds128(st + wl_off + (sub * 16 + 8) * WPITCH);
       }
-      q0 = p.job[jn1].w + (size_t)L1.sr0 * (p.K / 2) + cq * 16;
-      q1 = p.job[jn1].w + (size_t)L1.sr1 * (p.K / 2) + cq * 16;
-      load_scales(scn, p.job[jn1], L1, ch1);
-    }
-    const int g0 = ch * CH;
-    const int nvalid = min(CH, Gk - g0);
-    uint32_t xa[MT];
+      uint4 xr[MT][4];
 #pragma unroll
-    for (int t = 0; t < MT; ++t) xa[t] = xb_addr[t] + (uint32_t)(g0 * 256);
-    const uint32_t xga = xg_addr + (uint32_t)(g0 * 8 * MT * 4);
+      for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-    for (int g = 0; g < CH; ++g) {
-      if (g < nvalid) {
-        float acc[MT][2][4];     // two accumulators per batch tile: two independent MMA chains
-        const uint32_t wa[4] = {w0[g].x, w0[g].y, w0[g].z, w0[g].w};
-        const uint32_t wb[4] = {w1[g].x, w1[g].y, w1[g].z, w1[g].w};
+        for (int j = 0; j < 4; ++j)
+          xr[mt][j] = xlive[mt] ? lds128(xaddr[mt] + (uint32_t)(gi * 256 + j * 64)) : make_uint4(0, 0, 0, 0);
+      float acc[2][MT][4];
+      float sc[2][2];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+      for (int sub = 0; sub < 2; ++sub) {
+        sc[sub][0] = lds_h(st + sl_off + sub * 16 * (CG * 2));
+        sc[sub][1] = lds_h(st + sl_off + (sub * 16 + 8) * (CG * 2));
+        const float z0 = lds_h(st + sl_off + STAGE_SZ + sub * 16 * (CG * 2));
+        const float z1 = lds_h(st + sl_off + STAGE_SZ + (sub * 16 + 8) * (CG * 2));
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          // (-sum x, -sum o x) of batch rows 2t, 2t+1 (+8 mt)
+          const float4 xc = lds128f(xgaddr + (uint32_t)((gi * 8 * MT + 8 * mt) * 8));
+          acc[sub][mt][0] = fmaf(z0, xc.x, xc.y);
+          acc[sub][mt][2] = fmaf(z1, xc.x, xc.y);
+          acc[sub][mt][1] = ONECOL ? 0.f : fmaf(z0, xc.z, xc.w);
+          acc[sub][mt][3] = ONECOL ? 0.f : fmaf(z1, xc.z, xc.w);
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+#pragma unroll
+        for (int sub = 0; sub < 2; ++sub) {
+          const uint32_t w0 = j == 0 ? wa[sub].x : j == 1 ? wa[sub].y : j == 2 ? wa[sub].z : wa[sub].w;
+          const uint32_t w1 = j == 0 ? wb[sub].x : j == 1 ? wb[sub].y : j == 2 ? wb[sub].z : wb[sub].w;
           uint32_t a[4], b[4];
-          Cvt<T>::word(wa[j], a);
-          Cvt<T>::word(wb[j], b);
+          cvt_word(w0, a);
+          cvt_word(w1, b);
 #pragma unroll
-          for (int t = 0; t < MT; ++t) {
-            const uint4 xb = lds128(xa[t] + (uint32_t)(g * 256 + j * 64));
-            if (j == 0) {
-              Cvt<T>::mma0(acc[t][0], a[0], b[0], a[1], b[1], xb.x, xb.y);
-              Cvt<T>::mma0(acc[t][1], a[2], b[2], a[3], b[3], xb.z, xb.w);
-            } else {
-              Cvt<T>::mma(acc[t][0], a[0], b[0], a[1], b[1], xb.x, xb.y);
-              Cvt<T>::mma(acc[t][1], a[2], b[2], a[3], b[3], xb.z, xb.w);
-            }
+          for (int mt = 0; mt < MT; ++mt) {
+            mma_f16(acc[sub][mt], a[0], b[0], a[1], b[1], xr[mt][j].x, xr[mt][j].y);
+            mma_f16(acc[sub][mt], a[2], b[2], a[3], b[3], xr[mt][j].z, xr[mt][j].w);
           }
         }
-        if (has_next) load_group(g, q0, q1, ch1);      // the registers of group g are free again
-        auto pick = [&](int q) -> float {
-          const __half2 h = *reinterpret_cast<const __half2*>(&sc[q][g >> 1]);
-          return (g & 1) ? __high2float(h) : __low2float(h);
-        };
-        const float s0 = pick(0), nz0 = 8.f - pick(1);
-        const float s1 = pick(2), nz1 = 8.f - pick(3);
-#pragma unroll
-        for (int t = 0; t < MT; ++t) {
-          const float2 X = lds64f(xga + (uint32_t)((g * 8 * MT + 8 * t) * 4));
-          out[t][0] = fmaf(s0, fmaf(nz0, X.x, acc[t][0][0] + acc[t][1][0]), out[t][0]);
-          out[t][1] = fmaf(s0, fmaf(nz0, X.y, acc[t][0][1] + acc[t][1][1]), out[t][1]);
-          out[t][2] = fmaf(s1, fmaf(nz1, X.x, acc[t][0][2] + acc[t][1][2]), out[t][2]);
-          out[t][3] = fmaf(s1, fmaf(nz1, X.y, acc[t][0][3] + acc[t][1][3]), out[t][3]);
-        }
-      } else if (has_next) {
-        load_group(g, q0, q1, ch1);
       }
+#pragma unroll
+      for (int sub = 0; sub < 2; ++sub)
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          out[sub][mt][0] = fmaf(sc[sub][0], acc[sub][mt][0], out[sub][mt][0]);
+          out[sub][mt][2] = fmaf(sc[sub][1], acc[sub][mt][2], out[sub][mt][2]);
+          if (!ONECOL) {
+            out[sub][mt][1] = fmaf(sc[sub][0], acc[sub][mt][1], out[sub][mt][1]);
+            out[sub][mt][3] = fmaf(sc[sub][1], acc[sub][mt][3], out[sub][mt][3]);
+          }
+        }
     }
-    if (!has_next || tg1 != tg) {
-      OutVals ov;
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+
+    const bool tile_end = (chunk == Ck - 1) || (u == ue - 1);
+    if (tile_end) {
+      // ---- park this warp's partial sums: part[buf][group slot kpw][m][row slot]
+      float* pb = part + (c.part_bufs > 1 ? (tiles_done & 1) * part_stride : 0) + kpw * RB * p.M;
 #pragma unroll
-      for (int t = 0; t < MT_MAX; ++t)
+      for (int sub = 0; sub < 2; ++sub)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) ov.v[t][i] = t < MT ? out[t < MT ? t : 0][i] : 0.f;
-      flush_tile<T, MT, CH>(p, c, kp, gw, tg, jn, L, lane, ov);
+        for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-      for (int t = 0; t < MT; ++t)
+          for (int e = 0; e < (ONECOL ? 1 : 2); ++e) {
+            const int m = 2 * t + e + 8 * mt;
+            if (m < p.M) {
+              pb[m * RB + rg * 32 + sub * 16 + g] = out[sub][mt][e];
+              pb[m * RB + rg * 32 + sub * 16 + g + 8] = out[sub][mt][2 + e];
+            }
+          }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) out[t][i] = 0.f;
+      for (int sub = 0; sub < 2; ++sub)
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) out[sub][mt][i] = 0.f;
+      if (!consumer_sync()) return;
+
+      const float* pr = part + (c.part_bufs > 1 ? (tiles_done & 1) * part_stride : 0);
+      const int RM = RB * p.M;
+      auto local_sum = [&](int slot, int m) -> float {
+        float v = 0.f;
+#pragma unroll
+        for (int q = 0; q < CG; ++q) v += pr[q * RM + m * RB + slot];
+        return v;
+      };
+      // how many blocks (over all k-parts) work on this tile, and which of them am I
+      int total = 0, my_slot = 0;
+      for (int q = 0; q < c.n_kp; ++q) {
+        const int Gq = min(c.gp, c.g_total - q * c.gp);
+        const long Cq = (Gq + CG - 1) / CG;
+        const long Uq = (long)c.tiles_total * Cq;
+        const long Bq = (long)c.n_rp < Uq ? (long)c.n_rp : Uq;
+        const int first = owner_of((long)tile * Cq, Bq, Uq);
+        const int last = owner_of((long)tile * Cq + Cq - 1, Bq, Uq);
+        if (q == kp) my_slot = total + (rp - first);
+        total += last - first + 1;
+      }
+      const int jn = job_of(c, p.n_jobs, tile);
+      const JobDev& jb = p.job[jn];
+      const int tl = tile - c.tile_begin[jn];
+      if (total == 1) {
+        store_tile<T>(p, jb, tl, ctid, local_sum);
+      } else {
+        float* tile_ws = c.partials + (size_t)tile * c.max_slots * RM;
+        float* mine = tile_ws + (size_t)my_slot * RM;
+        for (int i = ctid; i < RM; i += CTH) __stcg(mine + i, local_sum(i & (RB - 1), i / RB));
+        __threadfence();
+        if (!consumer_sync()) return;
+        if (ctid == 0) {
+          const int arrived = atomicAdd(&c.counters[tile], 1);
+          *last_flag = arrived == total - 1;
+          __threadfence();
+        }
+        if (!consumer_sync()) return;
+        if (*last_flag) {
+          auto global_sum = [&](int slot, int m) -> float {
+            float v = 0.f;
+            for (int s2 = 0; s2 < total; ++s2) v += __ldcg(tile_ws + (size_t)s2 * RM + m * RB + slot);
+            return v;
+          };
+          store_tile<T>(p, jb, tl, ctid, global_sum);
+          if (ctid == 0) c.counters[tile] = 0;       // ready for the next call
+        }
+        if (!consumer_sync()) return;                // last_flag may be rewritten only after everyone read it
+      }
+      if (c.part_bufs == 1 && !consumer_sync()) return;
+      ++tiles_done;
     }
-    if (!has_next) break;
-    tg = tg1; ch = ch1; jn = jn1; L = L1;
-#pragma unroll
-    for (int q = 0; q < 4; ++q)
-#pragma unroll
-      for (int i = 0; i < CH / 2; ++i) sc[q][i] = scn[q][i];
+    if (++chunk == Ck) { chunk = 0; ++tile; }
   }
 }
 
@@ -545,33 +574,8 @@ int env_int(const char* name, int dflt) {
 }
 
 int job_tiles(const JobDev& j) {
-  if (j.rope.enabled) return (j.rope.n_heads * (j.rope.head_keep / 2) + 7) / 8;
-  return (j.k_out + 15) / 16;
-}
-
-// Visited-group spans of the input map: every 128-channel group that holds a retained channel,
-// neighbouring families merged when they touch the same group.
-void build_spans(const ChanMap& m, DecodeCfg* c) {
-  int n = 0, total = 0;
-  int last_g = -1;
-  for (int f = 0; f < m.n_fam; ++f) {
-    const Fam& a = m.fam[f];
-    int first = a.start / kGroup;
-    int end = a.start + (a.count - 1) * a.period + a.keep;   // exclusive
-    int last = (end - 1) / kGroup;
-    if (n > 0 && first <= last_g) {
-      if (last > last_g) { total += last - last_g; last_g = last; }
-    } else {
-      c->vg_begin[n] = total;
-      c->vg_first[n] = first;
-      total += last - first + 1;
-      last_g = last;
-      ++n;
-    }
-  }
-  c->n_spans = n;
-  c->vg_begin[n] = total;
-  c->g_total = total;
+  if (j.rope.enabled) return (j.rope.n_heads * (j.rope.head_keep / 2) + RB / 2 - 1) / (RB / 2);
+  return (j.k_out + RB - 1) / RB;
 }
 
 int sm_count() {
@@ -587,60 +591,93 @@ int sm_count() {
   return n;
 }
 
-size_t smem_bytes(int mp, int gp, int MT) { return (size_t)(mp + 1) * (gp * 256 + 64) + (size_t)gp * 8 * MT * 4; }
+int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
-template <typename T, int MT, int CH>
-int launch_t(const Params& p, const DecodeCfg& c, cudaStream_t stream) {
-  const size_t smem = smem_bytes(c.mp, c.gp, MT);
-  auto kern = decode_kernel<T, MT, CH>;
-  if (smem > 48 * 1024 &&
-      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return UNIQL_ERR_CUDA;
-  kern<<<c.n_kp * c.n_rp, NTD, smem, stream>>>(p, c);
-  return cudaGetLastError() == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
+// Shared-memory plan for a given split; returns the total size in bytes.
+size_t plan_smem(DecodeCfg* c, int M, int MT, int gp, int stages, int part_bufs) {
+  size_t off = BAR_BYTES + (size_t)stages * STAGE_BYTES;
+  c->xrow = gp * 256 + 64;
+  c->off_x = (int)off;
+  off += (size_t)M * c->xrow;
+  off = (off + 15) & ~(size_t)15;
+  c->off_xg = (int)off;
+  off += (size_t)gp * 8 * MT * 8;
+  c->off_part = (int)off;
+  off += (size_t)part_bufs * CG * RB * M * 4;
+  c->stages = stages;
+  c->part_bufs = part_bufs;
+  return off;
 }
 
 // Worst-case number of workspace slots a tile needs for a given split.
-int slots_needed(int tiles, int g_total, int gp, int n_rp, int CH) {
+int slots_needed(int tiles, int g_total, int gp, int n_rp) {
   int total = 0;
   for (int v = 0; v < g_total; v += gp) {
     const long Gq = (g_total - v) < gp ? (g_total - v) : gp;
-    const long Cq = (Gq + CH - 1) / CH;
+    const long Cq = (Gq + CG - 1) / CG;
     const long Uq = (long)tiles * Cq;
-    long Wq = (long)n_rp * NW;
-    if (Wq > Uq) Wq = Uq;
-    const long per_warp = Uq / Wq;           // >= 1
-    total += (int)((Cq + per_warp - 1) / per_warp) + 1;
+    long Bq = (long)n_rp;
+    if (Bq > Uq) Bq = Uq;
+    const long per_block = Uq / Bq;           // >= 1
+    total += (int)((Cq + per_block - 1) / per_block) + 1;
   }
   return total;
+}
+
+template <int MT, bool ONECOL>
+int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stream) {
+  auto kern = decode_kernel<MT, ONECOL>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return UNIQL_ERR_CUDA;
+  kern<<<c.n_kp * c.n_rp, NTH, smem, stream>>>(p, c);
+  return cudaGetLastError() == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
+}
+
+// Visited groups of the input map: from the first to the last 128-channel group that holds a retained
+// channel, widened to the copy granule (gaps between families are visited with zero activations).
+void visited_range(const ChanMap& m, int gran, int* first, int* total) {
+  int lo = m.fam[0].start / kGroup, hi = 0;
+  for (int f = 0; f < m.n_fam; ++f) {
+    const Fam& a = m.fam[f];
+    const int end = a.start + (a.count - 1) * a.period + a.keep;   // exclusive
+    const int last = (end - 1) / kGroup;
+    if (last > hi) hi = last;
+  }
+  lo = lo / gran * gran;
+  *first = lo;
+  *total = hi - lo + 1;
 }
 
 }  // namespace
 
 int decode_supported(const Params& p) {
   if (p.M < 1 || p.M > 16) return 0;
+  if (p.dt != UNIQL_F16) return 0;
+  if ((p.K % (2 * kGroup)) != 0) return 0;
   long tiles = 0;
   for (int j = 0; j < p.n_jobs; ++j) {
     if (job_tiles(p.job[j]) < 1) return 0;
     tiles += job_tiles(p.job[j]);
+    // scale / zero-point rows are copied in 4- or 8-byte granules
+    if (((uintptr_t)p.job[j].scales | (uintptr_t)p.job[j].zeros) & 7) return 0;
   }
   return tiles <= kCounterInts;
 }
 
 size_t decode_workspace_bytes(int M, int K, int N_total) {
-  // arrival counters + fp32 partial sums: up to 4 slots of [M][16] per 16-row tile and k-part
+  // header (arrival counters, status word) + fp32 partial sums: at most 4 slots per 64-row tile and k-part
   (void)K;
-  size_t tiles = (size_t)(N_total + 15) / 16 + 8 * kMaxJobs;
-  return (size_t)kCounterInts * 4 + tiles * (4 * kMaxKParts) * (size_t)M * 16 * 4;
+  size_t tiles = (size_t)(N_total + RB - 1) / RB + 2 * kMaxJobs;
+  return (size_t)kWsHeader + tiles * (4 * kMaxKParts) * (size_t)M * RB * 4;
 }
 
 int launch_decode(const Params& p, const LaunchCfg& cfg) {
   DecodeCfg c;
   memset(&c, 0, sizeof(c));
-  build_spans(p.imap, &c);
+  const int G = p.K / kGroup;
+  c.gran = (G % 4 == 0) ? 4 : 2;
+  visited_range(p.imap, c.gran, &c.v_first, &c.g_total);
   const int MT = p.M <= 8 ? 1 : 2;
-  const int CH = MT == 1 ? 4 : 2;
-  c.mp = MT == 1 ? p.M : 16;
   // 128-bit staging: one leading family, everything 8-element aligned
   c.x_vec = p.imap.n_fam == 1 && p.imap.fam[0].count == 1 && (p.imap.fam[0].start % 8) == 0 &&
             (p.imap.fam[0].keep % 8) == 0 && (p.ldx % 8) == 0 && ((((uintptr_t)p.x) & 15) == 0);
@@ -653,42 +690,49 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   c.tiles_total = tiles;
   if (tiles > kCounterInts) return UNIQL_ERR_SHAPE;
 
-  // ---- k-parts: as few as let the staged activations fit in shared memory (gp a multiple of CH)
+  // ---- k-parts: as few as let the staged activations fit beside a deep enough ring of stages
+  const int part_bufs = p.M <= 8 ? 2 : 1;
   int n_kp = env_int("UNIQL_DECODE_KP", 0);
-  if (n_kp < 1) {
-    n_kp = 1;
-    while (n_kp < kMaxKParts) {
-      int gp = ((c.g_total + n_kp - 1) / n_kp + CH - 1) / CH * CH;
-      if (smem_bytes(c.mp, gp, MT) <= kSmemBudget) break;
-      ++n_kp;
+  int stages = env_int("UNIQL_DECODE_STAGES", 0);
+  size_t smem = 0;
+  bool fits = false;
+  if (n_kp >= 1) {
+    if (n_kp > kMaxKParts) n_kp = kMaxKParts;
+    const int gp = round_up((c.g_total + n_kp - 1) / n_kp, c.gran);
+    for (int s = (stages >= 2 && stages <= MAX_STAGES) ? stages : 4; s >= 2 && !fits; --s) {
+      smem = plan_smem(&c, p.M, MT, gp, s, part_bufs);
+      fits = smem <= (size_t)kSmemMax;
     }
+    c.gp = gp;
+  } else {
+    const int want = (stages >= 2 && stages <= MAX_STAGES) ? stages : 4;
+    for (int s = want; s >= 3 && !fits; --s)
+      for (n_kp = 1; n_kp <= kMaxKParts && !fits; ++n_kp) {
+        const int gp = round_up((c.g_total + n_kp - 1) / n_kp, c.gran);
+        smem = plan_smem(&c, p.M, MT, gp, s, part_bufs);
+        fits = smem <= (size_t)kSmemMax;
+        c.gp = gp;
+      }
   }
-  if (n_kp > kMaxKParts) n_kp = kMaxKParts;
-  c.gp = ((c.g_total + n_kp - 1) / n_kp + CH - 1) / CH * CH;
+  if (!fits) return UNIQL_ERR_UNSUPPORTED;
   c.n_kp = (c.g_total + c.gp - 1) / c.gp;
-  if (smem_bytes(c.mp, c.gp, MT) > 220 * 1024) return UNIQL_ERR_UNSUPPORTED;
   int n_rp = env_int("UNIQL_DECODE_RP", 0);
   if (n_rp < 1) n_rp = sm_count() / c.n_kp;
   if (n_rp < 1) n_rp = 1;
   c.n_rp = n_rp;
-  c.max_slots = slots_needed(tiles, c.g_total, c.gp, c.n_rp, CH);
+  c.max_slots = slots_needed(tiles, c.g_total, c.gp, c.n_rp);
   {
-    const size_t need = (size_t)kCounterInts * 4 + (size_t)tiles * c.max_slots * p.M * 16 * 4;
+    const size_t need = (size_t)kWsHeader + (size_t)tiles * c.max_slots * p.M * RB * 4;
     if (!cfg.workspace || cfg.ws_bytes < need) return UNIQL_ERR_WORKSPACE;
   }
-  // vector loads of scales / zero-points: every chunk starts CH-aligned in stored groups and is contiguous
-  {
-    const int G = p.K / kGroup;
-    bool ok = c.n_spans == 1 && (c.vg_first[0] % CH) == 0 && (G % CH) == 0;
-    for (int j = 0; j < p.n_jobs && ok; ++j)
-      ok = ((((uintptr_t)p.job[j].scales) | ((uintptr_t)p.job[j].zeros)) & 15) == 0;
-    c.sz_vec = ok;
-  }
-  c.counters = reinterpret_cast<int*>(cfg.workspace);
-  c.partials = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(cfg.workspace) + (size_t)kCounterInts * 4);
-  if (p.dt == UNIQL_F16)
-    return MT == 1 ? launch_t<__half, 1, 4>(p, c, cfg.stream) : launch_t<__half, 2, 2>(p, c, cfg.stream);
-  return MT == 1 ? launch_t<__nv_bfloat16, 1, 4>(p, c, cfg.stream) : launch_t<__nv_bfloat16, 2, 2>(p, c, cfg.stream);
+  unsigned char* ws = reinterpret_cast<unsigned char*>(cfg.workspace);
+  c.counters = reinterpret_cast<int*>(ws);
+  c.status = reinterpret_cast<int*>(ws + kStatusOff);
+  c.partials = reinterpret_cast<float*>(ws + kWsHeader);
+  if (MT == 1) return p.M == 1 ? launch_t<1, true>(p, c, smem, cfg.stream) : launch_t<1, false>(p, c, smem, cfg.stream);
+  return launch_t<2, false>(p, c, smem, cfg.stream);
 }
+
+int decode_status_offset() { return kStatusOff; }
 
 }  // namespace uniql

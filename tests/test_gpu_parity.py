@@ -12,7 +12,11 @@ from paper_2512_03383_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
-TIGHT = 5e-5     # decode / generic kernels: exact products, fp32 accumulation
+# Decode / generic kernels: exact products, fp32 accumulation.  The decode kernel feeds the tensor
+# cores the codes with their conversion offsets (1024+q, 64+q) and removes the offsets per group in
+# fp32, so each group's accumulator is about 1000 times larger than its useful part and its fp32
+# rounding (2^-24 relative) shows up as roughly 1e-4 of the output scale: a tenth of the 2e-3 bar.
+TIGHT = 2e-4
 
 
 @pytest.fixture(scope="module")
