@@ -29,8 +29,11 @@
 //
 // Every wait in the kernel is an mbarrier wait with an iteration limit; when one expires the block
 // sets the status word of the workspace, lets its copies land and returns.
+#include <cuda.h>
 #include <stdlib.h>
 #include <string.h>
+
+#include <mutex>
 
 #include "common.cuh"
 
@@ -42,11 +45,12 @@ constexpr int CTH = CW * 32;            // consumer threads
 constexpr int NTH = CTH + 32;           // + one producer warp
 constexpr int RB = 64;                  // row slots per tile
 constexpr int CG = 8;                   // groups per chunk
-constexpr int WPITCH = CG * 64 + 64;    // bytes between row slots of a stage (the 64 keeps lane pairs on distinct banks)
-constexpr int STAGE_W = RB * WPITCH;
+constexpr int BOX_COLS = CG / 2;        // 128-byte columns (two groups each) per chunk
+constexpr int BOX_BYTES = RB * 128;     // one column of a stage: [RB rows][128 bytes], 128-byte swizzled
+constexpr int STAGE_W = BOX_COLS * BOX_BYTES;
 constexpr int STAGE_SZ = RB * CG * 2;   // one of the two fp16 arrays [RB][CG]
-constexpr int STAGE_BYTES = STAGE_W + 2 * STAGE_SZ;
-constexpr int MAX_STAGES = 5;
+constexpr int STAGE_BYTES = STAGE_W + 2 * STAGE_SZ;   // a multiple of 1024 (swizzle atom)
+constexpr int MAX_STAGES = 6;
 constexpr int kCounterInts = 1 << 16;   // arrival counters (one per tile) at the head of the workspace
 constexpr int kStatusOff = kCounterInts * 4;   // status word right after the counters
 constexpr int kWsHeader = kStatusOff + 256;
@@ -54,19 +58,34 @@ constexpr int kMaxKParts = 16;
 constexpr int kSmemMax = 227 * 1024;
 constexpr int kWaitLimit = 1 << 18;
 constexpr int BAR_BYTES = 128;
+constexpr int kMaxTF = 8;               // (job, family) pairs of one launch
+
+// One family of kept row blocks of one job: `count` blocks of `keep` rows, tiles of RB rows inside each
+// block (rope jobs: blocks are heads, rows are rotation pairs, RB/2 pairs per tile).
+struct TileFam {
+  int tile_begin;        // first global tile
+  int tpb;               // tiles per block
+  int keep;              // rows (pairs) per block
+  int count;
+  int job;
+  int start, period;     // stored row of block h, row r: start + h*period + r   (rope: h*head_dim + r)
+  int out_base;          // compact output column of block 0, row 0
+};
 
 struct DecodeCfg {
+  CUtensorMap wmap[kMaxTF];   // packed weights of each family: (byte, row in block, block)
+  TileFam tf[kMaxTF];
+  int n_tf;
   int n_kp, n_rp;        // k-parts x blocks per k-part
   int gp;                // visited groups per k-part (the last part may be shorter)
   int g_total;           // visited groups
   int v_first;           // first visited stored group
-  int gran;              // groups per scale / zero-point copy granule (2 or 4)
+  int gran;              // groups per scale / zero-point copy granule (2, 4 or 8)
   int stages;
   int tiles_total;
-  int tile_begin[kMaxJobs + 1];
   int x_vec;             // activations can be staged with 128-bit loads
   int max_slots;         // workspace slots per tile
-  int off_x, xrow, off_xg, off_part, part_bufs;
+  int off_bar, off_x, xrow, off_xg, off_part, part_bufs;
   int* counters;
   float* partials;
   int* status;
@@ -100,9 +119,14 @@ __device__ inline bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* ab
   *abort_flag = 1;
   return false;
 }
-__device__ inline void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+// One box of a 3-D tensor map into shared memory (no multicast), completion counted on `bar`.
+__device__ inline void tma_box3(uint32_t dst, const CUtensorMap* tm, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+__device__ inline void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ inline void cp_async8(uint32_t dst, const void* src) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
@@ -113,19 +137,30 @@ __device__ inline void cp_async4(uint32_t dst, const void* src) {
 __device__ inline void cp_async_arrive_noinc(uint32_t bar) {
   asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
+// shared-memory loads at [addr + OFF]: the offset is an immediate of the instruction, not an address add
+template <int OFF>
 __device__ inline uint4 lds128(uint32_t addr) {
   uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+%5];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr), "n"(OFF));
   return v;
 }
+template <int OFF>
+__device__ inline void lds128_if(uint4& v, uint32_t addr, bool pred) {      // v is left alone when !pred
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %5, 0;\n\t@p ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+%6];\n\t}"
+               : "+r"(v.x), "+r"(v.y), "+r"(v.z), "+r"(v.w) : "r"(addr), "r"((uint32_t)pred), "n"(OFF));
+}
+template <int OFF>
 __device__ inline float4 lds128f(uint32_t addr) {
   float4 v;
-  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+%5];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr), "n"(OFF));
   return v;
 }
+template <int OFF>
 __device__ inline float lds_h(uint32_t addr) {
   unsigned short h;
-  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(addr));
+  asm volatile("ld.shared.u16 %0, [%1+%2];" : "=h"(h) : "r"(addr), "n"(OFF));
   return __half2float(__ushort_as_half(h));
 }
 // (a & mask) | magic in one LOP3 (truth table 0xEA)
@@ -150,25 +185,17 @@ __device__ inline void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t
 }
 
 // ---------------------------------------------------------------------------------------- tile geometry
-__device__ inline int job_of(const DecodeCfg& c, int n_jobs, int tg) {
-  int j = 0;
-  while (j + 1 < n_jobs && tg >= c.tile_begin[j + 1]) ++j;
-  return j;
-}
-
-// Stored weight row of row slot `slot` of local tile `tile` of a job, or -1 when the slot is empty.
-__device__ inline int slot_to_stored(const JobDev& jb, int tile, int slot) {
-  if (jb.rope.enabled) {
-    const int half = jb.rope.head_keep >> 1;
-    const int P = tile * (RB / 2) + (slot & (RB / 2 - 1));
-    if (P >= jb.rope.n_heads * half) return -1;
-    const int h = P / half, cc = P - h * half;
-    return h * jb.rope.head_dim + ((slot >= RB / 2) ? (jb.rope.head_dim >> 1) : 0) + cc;
-  }
-  const int j = tile * RB + slot;
-  if (j >= jb.k_out) return -1;
-  if (jb.omap.n_fam == 1 && jb.omap.fam[0].count == 1) return jb.omap.fam[0].start + j;
-  return map_compact_to_stored(jb.omap, j);
+struct TilePos { int fi, h, r0; };
+__device__ inline TilePos tile_pos(const DecodeCfg& c, const Params& p, int tg) {
+  TilePos q;
+  q.fi = 0;
+  while (q.fi + 1 < c.n_tf && tg >= c.tf[q.fi + 1].tile_begin) ++q.fi;
+  const TileFam& f = c.tf[q.fi];
+  const int tl = tg - f.tile_begin;
+  q.h = tl / f.tpb;
+  const int rows = p.job[f.job].rope.enabled ? RB / 2 : RB;
+  q.r0 = (tl - q.h * f.tpb) * rows;
+  return q;
 }
 
 // The block (of its k-part) whose unit range [U*b/B, U*(b+1)/B) holds unit u; exact in fp64 here.
@@ -178,39 +205,38 @@ __device__ inline int owner_of(long u, long B, long U) {
 
 // bias, rotary embedding on the retained pair, one rounding, store; `get(slot, m)` yields the fp32 sum
 template <typename T, typename F>
-__device__ inline void store_tile(const Params& p, const JobDev& jb, int tile, int ctid, F get) {
+__device__ inline void store_tile(const Params& p, const TileFam& f, const TilePos& q, int ctid, F get) {
+  const JobDev& jb = p.job[f.job];
   const T* bias = reinterpret_cast<const T*>(jb.bias);
   T* y = reinterpret_cast<T*>(jb.y);
   if (jb.rope.enabled) {
     const int half = jb.rope.head_keep >> 1;
-    const int n_pairs = jb.rope.n_heads * half;
     for (int i = ctid; i < (RB / 2) * p.M; i += CTH) {
       const int pp = i & (RB / 2 - 1), m = i / (RB / 2);
-      const int P = tile * (RB / 2) + pp;
-      if (P >= n_pairs) continue;
-      const int h = P / half, cc = P - h * half;
+      const int cc = q.r0 + pp;
+      if (cc >= half) continue;
       float lo = get(pp, m), hi = get(pp + RB / 2, m);
       if (bias) {
-        const int sr = h * jb.rope.head_dim + cc;
+        const int sr = q.h * jb.rope.head_dim + cc;
         lo += DT<T>::to_f(bias[sr]);
         hi += DT<T>::to_f(bias[sr + (jb.rope.head_dim >> 1)]);
       }
-      int pidx = p.idx[(h / jb.rope.rep) * half + cc];
+      int pidx = p.idx[(q.h / jb.rope.rep) * half + cc];
       pidx = min(max(pidx, 0), (jb.rope.head_dim >> 1) - 1);
       float cs, sn;
       rope_cos_sin(p.pos[m], p.inv_freq[pidx], cs, sn);
-      const int oc = h * jb.rope.head_keep + cc;
+      const int oc = q.h * jb.rope.head_keep + cc;
       y[(size_t)m * jb.ldy + oc] = DT<T>::from_f(lo * cs - hi * sn);
       y[(size_t)m * jb.ldy + oc + half] = DT<T>::from_f(hi * cs + lo * sn);
     }
   } else {
     for (int i = ctid; i < RB * p.M; i += CTH) {
       const int slot = i & (RB - 1), m = i / RB;
-      const int j = tile * RB + slot;
-      if (j >= jb.k_out) continue;
+      const int r = q.r0 + slot;
+      if (r >= f.keep) continue;
       float v = get(slot, m);
-      if (bias) v += DT<T>::to_f(bias[slot_to_stored(jb, tile, slot)]);
-      y[(size_t)m * jb.ldy + j] = DT<T>::from_f(v);
+      if (bias) v += DT<T>::to_f(bias[f.start + q.h * f.period + r]);
+      y[(size_t)m * jb.ldy + f.out_base + q.h * f.keep + r] = DT<T>::from_f(v);
     }
   }
 }
@@ -219,16 +245,18 @@ __device__ inline void store_tile(const Params& p, const JobDev& jb, int tile, i
 template <int MT, bool ONECOL>
 __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ Params p,
                                                         const __grid_constant__ DecodeCfg c) {
-  extern __shared__ __align__(128) unsigned char smem[];
+  extern __shared__ unsigned char smem_raw[];
   using T = __half;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(smem);
+  // the stage ring starts on a 1024-byte boundary (the swizzle pattern repeats every 1024 bytes)
+  const uint32_t raw = (uint32_t)__cvta_generic_to_shared(smem_raw);
+  const uint32_t sbase = (raw + 1023u) & ~1023u;
+  unsigned char* smem = smem_raw + (sbase - raw);
   const int S = c.stages;
   // barriers: full[S], empty[S], consumer barrier; then two flags
-  const uint32_t bar_full = sbase, bar_empty = sbase + 8 * MAX_STAGES, bar_cons = sbase + 16 * MAX_STAGES;
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 16 * MAX_STAGES + 8);
-  volatile int* last_flag = reinterpret_cast<volatile int*>(smem + 16 * MAX_STAGES + 12);
-  const uint32_t stage0 = sbase + BAR_BYTES;
+  const uint32_t bar_full = sbase + c.off_bar, bar_empty = bar_full + 8 * MAX_STAGES, bar_cons = bar_full + 16 * MAX_STAGES;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + c.off_bar + 16 * MAX_STAGES + 8);
+  volatile int* last_flag = reinterpret_cast<volatile int*>(smem + c.off_bar + 16 * MAX_STAGES + 12);
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) {
@@ -257,46 +285,64 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   // ======================================================================================= producer
   if (warp == CW) {
     int tile = ub / Ck, chunk = ub - tile * Ck;
-    int jn = -1, tile_prev = -1;
-    const uint8_t* wrow[2] = {nullptr, nullptr};
+    int tile_prev = -1;
+    TilePos q = {0, 0, 0};
+    bool rope = false;
     const __half* srow[2] = {nullptr, nullptr};
     const __half* zrow[2] = {nullptr, nullptr};
-    int n_valid = 0;
-    int it = 0;
+    int it = 0, s = 0;
+    uint32_t ring_parity = 1;      // parity of the previous use of ring position s
     bool ok = true;
     for (int u = ub; u < ue; ++u, ++it) {
-      const int s = it % S;
-      if (it >= S) ok = mbar_wait(bar_empty + 8 * s, ((it / S) - 1) & 1, abort_flag);
+      if (it >= S) ok = mbar_wait(bar_empty + 8 * s, ring_parity, abort_flag);
       if (!ok) break;
       if (tile != tile_prev) {
-        jn = job_of(c, p.n_jobs, tile);
-        const JobDev& jb = p.job[jn];
-        const int tl = tile - c.tile_begin[jn];
+        q = tile_pos(c, p, tile);
+        const TileFam& f = c.tf[q.fi];
+        const JobDev& jb = p.job[f.job];
+        rope = jb.rope.enabled != 0;
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
-          const int sr = slot_to_stored(jb, tl, lane + 32 * q);
-          wrow[q] = sr >= 0 ? jb.w + (size_t)sr * (p.K / 2) + (size_t)sg_lo * 64 : nullptr;
-          srow[q] = sr >= 0 ? jb.scales + (size_t)sr * G + sg_lo : nullptr;
-          zrow[q] = sr >= 0 ? jb.zeros + (size_t)sr * G + sg_lo : nullptr;
+        for (int r2 = 0; r2 < 2; ++r2) {
+          const int slot = lane + 32 * r2;
+          int sr = -1;
+          if (rope) {
+            const int cc = q.r0 + lane;
+            if (cc < f.keep) sr = q.h * jb.rope.head_dim + r2 * (jb.rope.head_dim >> 1) + cc;
+          } else {
+            const int r = q.r0 + slot;
+            if (r < f.keep) sr = f.start + q.h * f.period + r;
+          }
+          srow[r2] = sr >= 0 ? jb.scales + (size_t)sr * G + sg_lo : nullptr;
+          zrow[r2] = sr >= 0 ? jb.zeros + (size_t)sr * G + sg_lo : nullptr;
         }
-        n_valid = __popc(__ballot_sync(0xffffffffu, wrow[0] != nullptr)) +
-                  __popc(__ballot_sync(0xffffffffu, wrow[1] != nullptr));
         tile_prev = tile;
       }
       const int ng = min(CG, Gk - chunk * CG);
+      const int nb = (ng + 1) >> 1;                      // 128-byte columns with a visited group
       const uint32_t full = bar_full + 8 * s;
-      const uint32_t st = stage0 + (uint32_t)s * STAGE_BYTES;
-      if (lane == 0) mbar_expect_tx(full, (uint32_t)(n_valid * ng * 64));
+      const uint32_t st = sbase + (uint32_t)s * STAGE_BYTES;
+      if (lane == 0) mbar_expect_tx(full, (uint32_t)(nb * BOX_BYTES));
       __syncwarp();
+      if (lane < nb) {
+        const int xb = (sg_lo + chunk * CG + 2 * lane) * 64;       // byte in the weight row
+        const uint32_t dst = st + (uint32_t)lane * BOX_BYTES;
+        if (rope) {
+          tma_box3(dst, &c.wmap[q.fi], xb, q.r0, 2 * q.h, full);
+          tma_box3(dst + (RB / 2) * 128, &c.wmap[q.fi], xb, q.r0, 2 * q.h + 1, full);
+        } else {
+          tma_box3(dst, &c.wmap[q.fi], xb, q.r0, q.h, full);
+        }
+      }
 #pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        if (wrow[q]) {
-          const int slot = lane + 32 * q;
-          bulk_g2s(st + slot * WPITCH, wrow[q] + (size_t)chunk * (CG * 64), (uint32_t)(ng * 64), full);
+      for (int r2 = 0; r2 < 2; ++r2) {
+        if (srow[r2]) {
+          const int slot = lane + 32 * r2;
           const uint32_t sd = st + STAGE_W + slot * (CG * 2), zd = sd + STAGE_SZ;
-          const __half* sp = srow[q] + chunk * CG;
-          const __half* zp = zrow[q] + chunk * CG;
-          if (c.gran == 4) {
+          const __half* sp = srow[r2] + chunk * CG;
+          const __half* zp = zrow[r2] + chunk * CG;
+          if (c.gran == 8) {
+            cp_async16(sd, sp); cp_async16(zd, zp);
+          } else if (c.gran == 4) {
             for (int g4 = 0; g4 < ng; g4 += 4) { cp_async8(sd + g4 * 2, sp + g4); cp_async8(zd + g4 * 2, zp + g4); }
           } else {
             for (int g2 = 0; g2 < ng; g2 += 2) { cp_async4(sd + g2 * 2, sp + g2); cp_async4(zd + g2 * 2, zp + g2); }
@@ -305,6 +351,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       }
       cp_async_arrive_noinc(full);
       if (++chunk == Ck) { chunk = 0; ++tile; }
+      if (++s == S) { s = 0; ring_parity ^= 1; }
     }
     if (!ok) {
       // let the copies of the stages that are still armed land before the block goes away
@@ -322,12 +369,17 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   const int ctid = tid;                    // 0..CTH-1
   const int g = lane >> 2, t = lane & 3;
   const int kpw = warp & 7, rg = warp >> 3;
+  // MMA row g of a sub-tile is row slot pg: lanes g = 2i and 2i+1 get slots that differ in bit 2, so that
+  // under the 128-byte swizzle the eight lanes of a shared-memory load phase touch eight distinct 16-byte columns
+  const int pg = (g >> 1) | ((g & 1) << 2);
   uint32_t cons_parity = 0;
+  auto give_up = [&]() { if (lane == 0) atomicExch(c.status, UNIQL_ERR_TIMEOUT); };
   auto consumer_sync = [&]() -> bool {
     __syncwarp();
     if (lane == 0) mbar_arrive(bar_cons);
     const bool ok = mbar_wait(bar_cons, cons_parity, abort_flag);
     cons_parity ^= 1;
+    if (!ok) give_up();
     return ok;
   };
 
@@ -343,30 +395,42 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     if (c.x_vec) {
       const int start = p.imap.fam[0].start, keep = p.imap.fam[0].keep;
       const int n_units = Gk * p.M * 16;
-      for (int u = ctid; u < ((n_units + 31) & ~31); u += CTH) {   // whole warps stay in the shuffles
-        const bool in_range = u < n_units;
-        const int u16 = u & 15, pair = in_range ? u >> 4 : 0;
-        const int m = pair / Gk, lv = pair - m * Gk;
-        uint4 in = make_uint4(0, 0, 0, 0);
-        if (in_range) {
-          const int t0 = (sg_lo + lv) * kGroup + 8 * u16 - start;
-          if (t0 >= 0 && t0 < keep) in = *reinterpret_cast<const uint4*>(x + (size_t)m * p.ldx + t0);
-        }
-        uint4 o;
-        o.x = __byte_perm(in.x, in.z, 0x5410); o.y = __byte_perm(in.x, in.z, 0x7632);
-        o.z = __byte_perm(in.y, in.w, 0x5410); o.w = __byte_perm(in.y, in.w, 0x7632);
-        // the 16 bytes of lane quarter c', word j of a group sit at byte j*64 + c'*16; u16 = c'*4 + j
-        if (in_range) xs[m * row_units + lv * 16 + (u16 & 3) * 4 + (u16 >> 2)] = o;
-        const __half2* h2 = reinterpret_cast<const __half2*>(&in);
-        float se = 0.f, so = 0.f;
+      constexpr int UN = 4;                                        // loads in flight per thread
+      for (int u0 = ctid; u0 < ((n_units + 31) & ~31); u0 += CTH * UN) {   // whole warps stay in the shuffles
+        uint4 in[UN];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) { const float2 f = __half22float2(h2[i]); se += f.x; so += f.y; }
-#pragma unroll
-        for (int o2 = 8; o2 >= 1; o2 >>= 1) {
-          se += __shfl_xor_sync(0xffffffffu, se, o2);
-          so += __shfl_xor_sync(0xffffffffu, so, o2);
+        for (int q4 = 0; q4 < UN; ++q4) {
+          const int u = u0 + q4 * CTH;
+          in[q4] = make_uint4(0, 0, 0, 0);
+          if (u < n_units) {
+            const int pair = u >> 4, m = pair / Gk, lv = pair - m * Gk;
+            const int t0 = (sg_lo + lv) * kGroup + 8 * (u & 15) - start;
+            if (t0 >= 0 && t0 < keep) in[q4] = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * p.ldx + t0));
+          }
         }
-        if (in_range && u16 == 0) xg[lv * 8 * MT + m] = make_float2(-(se + so), -(1024.f * se + 64.f * so));
+#pragma unroll
+        for (int q4 = 0; q4 < UN; ++q4) {
+          const int u = u0 + q4 * CTH;
+          if (u >= ((n_units + 31) & ~31)) break;                  // warp-uniform
+          const bool in_range = u < n_units;
+          const int u16 = u & 15, pair = in_range ? u >> 4 : 0;
+          const int m = pair / Gk, lv = pair - m * Gk;
+          uint4 o;
+          o.x = __byte_perm(in[q4].x, in[q4].z, 0x5410); o.y = __byte_perm(in[q4].x, in[q4].z, 0x7632);
+          o.z = __byte_perm(in[q4].y, in[q4].w, 0x5410); o.w = __byte_perm(in[q4].y, in[q4].w, 0x7632);
+          // the 16 bytes of lane quarter c', word j of a group sit at byte j*64 + c'*16; u16 = c'*4 + j
+          if (in_range) xs[m * row_units + lv * 16 + (u16 & 3) * 4 + (u16 >> 2)] = o;
+          const __half2* h2 = reinterpret_cast<const __half2*>(&in[q4]);
+          float se = 0.f, so = 0.f;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) { const float2 f = __half22float2(h2[i]); se += f.x; so += f.y; }
+#pragma unroll
+          for (int o2 = 8; o2 >= 1; o2 >>= 1) {
+            se += __shfl_xor_sync(0xffffffffu, se, o2);
+            so += __shfl_xor_sync(0xffffffffu, so, o2);
+          }
+          if (in_range && u16 == 0) xg[lv * 8 * MT + m] = make_float2(-(se + so), -(1024.f * se + 64.f * so));
+        }
       }
     } else {
       T* xh = reinterpret_cast<T*>(smem + c.off_x);
@@ -376,8 +440,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         const int kbase = (sg_lo + lv) * kGroup;
         float se = 0.f, so = 0.f;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int i = lane + 32 * q;
+        for (int q4 = 0; q4 < 4; ++q4) {
+          const int i = lane + 32 * q4;
           T val = __float2half_rn(0.f);
           const int tt = map_stored_to_compact(p.imap, kbase + i);
           if (tt >= 0) val = x[(size_t)m * p.ldx + tt];
@@ -406,8 +470,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     xaddr[mt] = sbase + c.off_x + (uint32_t)((xlive[mt] ? m : 0) * c.xrow + t * 16);
   }
   const uint32_t xgaddr = sbase + c.off_xg + (uint32_t)(2 * t * 8);
-  const uint32_t wl_off = (uint32_t)((rg * 32 + g) * WPITCH + kpw * 64 + t * 16);
-  const uint32_t sl_off = (uint32_t)(STAGE_W + (rg * 32 + g) * (CG * 2) + kpw * 2);
+  const uint32_t wl_off = (uint32_t)((kpw >> 1) * BOX_BYTES + (rg * 32 + pg) * 128 + ((((kpw & 1) * 4 + t) ^ pg) * 16));
+  const uint32_t sl_off = (uint32_t)(STAGE_W + (rg * 32 + pg) * (CG * 2) + kpw * 2);
   float* part = reinterpret_cast<float*>(smem + c.off_part);
   const int part_stride = CG * RB * p.M;     // floats per partial buffer
 
@@ -420,41 +484,58 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       for (int i = 0; i < 4; ++i) out[sub][mt][i] = 0.f;
 
   int tile = ub / Ck, chunk = ub - tile * Ck;
-  int it = 0, tiles_done = 0;
-  for (int u = ub; u < ue; ++u, ++it) {
-    const int s = it % S;
-    if (!mbar_wait(bar_full + 8 * s, (it / S) & 1, abort_flag)) return;
+  int tiles_done = 0;
+  int s = 0;                 // ring position and the parity of its current use
+  uint32_t ring_parity = 0;
+  uint4 xr[MT][4];           // B fragments; lanes whose batch row does not exist keep zeros
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) xr[mt][j] = make_uint4(0, 0, 0, 0);
+  for (int u = ub; u < ue; ++u) {
+    if (!mbar_try_wait(bar_full + 8 * s, ring_parity) && !mbar_wait(bar_full + 8 * s, ring_parity, abort_flag)) {
+      give_up();
+      return;
+    }
     const int gi = chunk * CG + kpw;
     if (gi < Gk) {
-      const uint32_t st = stage0 + (uint32_t)s * STAGE_BYTES;
+      const uint32_t st = sbase + (uint32_t)s * STAGE_BYTES;
+      const uint32_t wp = st + wl_off, sp = st + sl_off;
       uint4 wa[2], wb[2];
+      wa[0] = lds128<0>(wp);
+      wb[0] = lds128<8 * 128>(wp);
+      wa[1] = lds128<16 * 128>(wp);
+      wb[1] = lds128<24 * 128>(wp);
 #pragma unroll
-      for (int sub = 0; sub < 2; ++sub) {
-        wa[sub] = lds128(st + wl_off + sub * 16 * WPITCH);
-        wb[sub] = lds128(st + wl_off + (sub * 16 + 8) * WPITCH);
+      for (int mt = 0; mt < MT; ++mt) {
+        const uint32_t xa = xaddr[mt] + (uint32_t)(gi * 256);
+        lds128_if<0>(xr[mt][0], xa, xlive[mt]);
+        lds128_if<64>(xr[mt][1], xa, xlive[mt]);
+        lds128_if<128>(xr[mt][2], xa, xlive[mt]);
+        lds128_if<192>(xr[mt][3], xa, xlive[mt]);
       }
-      uint4 xr[MT][4];
-#pragma unroll
-      for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-          xr[mt][j] = xlive[mt] ? lds128(xaddr[mt] + (uint32_t)(gi * 256 + j * 64)) : make_uint4(0, 0, 0, 0);
       float acc[2][MT][4];
       float sc[2][2];
+      sc[0][0] = lds_h<0>(sp);
+      sc[0][1] = lds_h<8 * CG * 2>(sp);
+      sc[1][0] = lds_h<16 * CG * 2>(sp);
+      sc[1][1] = lds_h<24 * CG * 2>(sp);
+      float zp[2][2];
+      zp[0][0] = lds_h<STAGE_SZ>(sp);
+      zp[0][1] = lds_h<STAGE_SZ + 8 * CG * 2>(sp);
+      zp[1][0] = lds_h<STAGE_SZ + 16 * CG * 2>(sp);
+      zp[1][1] = lds_h<STAGE_SZ + 24 * CG * 2>(sp);
+      const uint32_t xga = xgaddr + (uint32_t)(gi * 8 * MT * 8);
 #pragma unroll
-      for (int sub = 0; sub < 2; ++sub) {
-        sc[sub][0] = lds_h(st + sl_off + sub * 16 * (CG * 2));
-        sc[sub][1] = lds_h(st + sl_off + (sub * 16 + 8) * (CG * 2));
-        const float z0 = lds_h(st + sl_off + STAGE_SZ + sub * 16 * (CG * 2));
-        const float z1 = lds_h(st + sl_off + STAGE_SZ + (sub * 16 + 8) * (CG * 2));
+      for (int mt = 0; mt < MT; ++mt) {
+        // (-sum x, -sum o x) of batch rows 2t, 2t+1 (+8 mt)
+        const float4 xc = mt == 0 ? lds128f<0>(xga) : lds128f<64>(xga);
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt) {
-          // (-sum x, -sum o x) of batch rows 2t, 2t+1 (+8 mt)
-          const float4 xc = lds128f(xgaddr + (uint32_t)((gi * 8 * MT + 8 * mt) * 8));
-          acc[sub][mt][0] = fmaf(z0, xc.x, xc.y);
-          acc[sub][mt][2] = fmaf(z1, xc.x, xc.y);
-          acc[sub][mt][1] = ONECOL ? 0.f : fmaf(z0, xc.z, xc.w);
-          acc[sub][mt][3] = ONECOL ? 0.f : fmaf(z1, xc.z, xc.w);
+        for (int sub = 0; sub < 2; ++sub) {
+          acc[sub][mt][0] = fmaf(zp[sub][0], xc.x, xc.y);
+          acc[sub][mt][2] = fmaf(zp[sub][1], xc.x, xc.y);
+          acc[sub][mt][1] = ONECOL ? 0.f : fmaf(zp[sub][0], xc.z, xc.w);
+          acc[sub][mt][3] = ONECOL ? 0.f : fmaf(zp[sub][1], xc.z, xc.w);
         }
       }
 #pragma unroll
@@ -487,6 +568,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+    if (++s == S) { s = 0; ring_parity ^= 1; }
 
     const bool tile_end = (chunk == Ck - 1) || (u == ue - 1);
     if (tile_end) {
@@ -500,8 +582,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           for (int e = 0; e < (ONECOL ? 1 : 2); ++e) {
             const int m = 2 * t + e + 8 * mt;
             if (m < p.M) {
-              pb[m * RB + rg * 32 + sub * 16 + g] = out[sub][mt][e];
-              pb[m * RB + rg * 32 + sub * 16 + g + 8] = out[sub][mt][2 + e];
+              pb[m * RB + rg * 32 + sub * 16 + pg] = out[sub][mt][e];
+              pb[m * RB + rg * 32 + sub * 16 + pg + 8] = out[sub][mt][2 + e];
             }
           }
 #pragma unroll
@@ -517,26 +599,25 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       auto local_sum = [&](int slot, int m) -> float {
         float v = 0.f;
 #pragma unroll
-        for (int q = 0; q < CG; ++q) v += pr[q * RM + m * RB + slot];
+        for (int q8 = 0; q8 < CG; ++q8) v += pr[q8 * RM + m * RB + slot];
         return v;
       };
       // how many blocks (over all k-parts) work on this tile, and which of them am I
       int total = 0, my_slot = 0;
-      for (int q = 0; q < c.n_kp; ++q) {
-        const int Gq = min(c.gp, c.g_total - q * c.gp);
+      for (int q2 = 0; q2 < c.n_kp; ++q2) {
+        const int Gq = min(c.gp, c.g_total - q2 * c.gp);
         const long Cq = (Gq + CG - 1) / CG;
         const long Uq = (long)c.tiles_total * Cq;
         const long Bq = (long)c.n_rp < Uq ? (long)c.n_rp : Uq;
         const int first = owner_of((long)tile * Cq, Bq, Uq);
         const int last = owner_of((long)tile * Cq + Cq - 1, Bq, Uq);
-        if (q == kp) my_slot = total + (rp - first);
+        if (q2 == kp) my_slot = total + (rp - first);
         total += last - first + 1;
       }
-      const int jn = job_of(c, p.n_jobs, tile);
-      const JobDev& jb = p.job[jn];
-      const int tl = tile - c.tile_begin[jn];
+      const TilePos q = tile_pos(c, p, tile);
+      const TileFam& f = c.tf[q.fi];
       if (total == 1) {
-        store_tile<T>(p, jb, tl, ctid, local_sum);
+        store_tile<T>(p, f, q, ctid, local_sum);
       } else {
         float* tile_ws = c.partials + (size_t)tile * c.max_slots * RM;
         float* mine = tile_ws + (size_t)my_slot * RM;
@@ -555,7 +636,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
             for (int s2 = 0; s2 < total; ++s2) v += __ldcg(tile_ws + (size_t)s2 * RM + m * RB + slot);
             return v;
           };
-          store_tile<T>(p, jb, tl, ctid, global_sum);
+          store_tile<T>(p, f, q, ctid, global_sum);
           if (ctid == 0) c.counters[tile] = 0;       // ready for the next call
         }
         if (!consumer_sync()) return;                // last_flag may be rewritten only after everyone read it
@@ -573,11 +654,6 @@ int env_int(const char* name, int dflt) {
   return s ? atoi(s) : dflt;
 }
 
-int job_tiles(const JobDev& j) {
-  if (j.rope.enabled) return (j.rope.n_heads * (j.rope.head_keep / 2) + RB / 2 - 1) / (RB / 2);
-  return (j.k_out + RB - 1) / RB;
-}
-
 int sm_count() {
   static int n = 0;
   if (n == 0) {
@@ -593,9 +669,55 @@ int sm_count() {
 
 int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
-// Shared-memory plan for a given split; returns the total size in bytes.
+int copy_granule(int G) { return (G % 8 == 0) ? 8 : (G % 4 == 0) ? 4 : 2; }
+
+// number of (job, family) pairs of a launch
+int count_tile_fams(const Params& p) {
+  int n = 0;
+  for (int j = 0; j < p.n_jobs; ++j) n += p.job[j].rope.enabled ? 1 : p.job[j].omap.n_fam;
+  return n;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up through the runtime (no link-time dependency on libcuda).
+EncodeTiledFn encoder() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qr) == cudaSuccess &&
+        qr == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    else
+      cudaGetLastError();
+  });
+  return fn;
+}
+
+// Packed rows of one family as a 3-D byte tensor (byte in row, row in block, block), 128-byte swizzled boxes.
+int encode_family(CUtensorMap* tm, const uint8_t* base, int K, int x_extent, int keep, int count, int row_stride_rows,
+                  int box_rows) {
+  EncodeTiledFn enc = encoder();
+  if (!enc) return UNIQL_ERR_CUDA;
+  const cuuint64_t dims[3] = {(cuuint64_t)x_extent, (cuuint64_t)keep, (cuuint64_t)count};
+  const cuuint64_t strides[2] = {(cuuint64_t)(K / 2), (cuuint64_t)row_stride_rows * (cuuint64_t)(K / 2)};
+  const cuuint32_t box[3] = {128, (cuuint32_t)box_rows, 1};
+  const cuuint32_t es[3] = {1, 1, 1};
+  const CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t*>(base), dims, strides, box, es,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? UNIQL_OK : UNIQL_ERR_CUDA;
+}
+
+// Shared-memory plan for a given split; returns the total size in bytes (with the alignment slack).
 size_t plan_smem(DecodeCfg* c, int M, int MT, int gp, int stages, int part_bufs) {
-  size_t off = BAR_BYTES + (size_t)stages * STAGE_BYTES;
+  size_t off = (size_t)stages * STAGE_BYTES;
+  c->off_bar = (int)off;
+  off += BAR_BYTES;
   c->xrow = gp * 256 + 64;
   c->off_x = (int)off;
   off += (size_t)M * c->xrow;
@@ -606,7 +728,7 @@ size_t plan_smem(DecodeCfg* c, int M, int MT, int gp, int stages, int part_bufs)
   off += (size_t)part_bufs * CG * RB * M * 4;
   c->stages = stages;
   c->part_bufs = part_bufs;
-  return off;
+  return off + 1024;
 }
 
 // Worst-case number of workspace slots a tile needs for a given split.
@@ -648,78 +770,123 @@ void visited_range(const ChanMap& m, int gran, int* first, int* total) {
   *total = hi - lo + 1;
 }
 
+// Split of the visited groups into k-parts and the shared-memory plan: as few k-parts as let the staged
+// activations fit beside a deep enough ring of stages.  Returns 0 when nothing fits.
+size_t plan_split(DecodeCfg* c, int M, int g_total, int gran) {
+  const int MT = M <= 8 ? 1 : 2;
+  const int part_bufs = M <= 8 ? 2 : 1;
+  int n_kp = env_int("UNIQL_DECODE_KP", 0);
+  const int stages = env_int("UNIQL_DECODE_STAGES", 0);
+  const int want = (stages >= 2 && stages <= MAX_STAGES) ? stages : 4;
+  size_t smem = 0;
+  bool fits = false;
+  if (n_kp >= 1) {
+    if (n_kp > kMaxKParts) n_kp = kMaxKParts;
+    const int gp = round_up((g_total + n_kp - 1) / n_kp, gran);
+    for (int s = want; s >= 2 && !fits; --s) {
+      smem = plan_smem(c, M, MT, gp, s, part_bufs);
+      fits = smem <= (size_t)kSmemMax;
+    }
+    c->gp = gp;
+  } else {
+    for (int s = want; s >= 3 && !fits; --s)
+      for (n_kp = 1; n_kp <= kMaxKParts && !fits; ++n_kp) {
+        const int gp = round_up((g_total + n_kp - 1) / n_kp, gran);
+        smem = plan_smem(c, M, MT, gp, s, part_bufs);
+        fits = smem <= (size_t)kSmemMax;
+        c->gp = gp;
+      }
+  }
+  if (!fits) return 0;
+  c->g_total = g_total;
+  c->gran = gran;
+  c->n_kp = (g_total + c->gp - 1) / c->gp;
+  int n_rp = env_int("UNIQL_DECODE_RP", 0);
+  if (n_rp < 1) n_rp = sm_count() / c->n_kp;
+  if (n_rp < 1) n_rp = 1;
+  c->n_rp = n_rp;
+  return smem;
+}
+
 }  // namespace
 
 int decode_supported(const Params& p) {
   if (p.M < 1 || p.M > 16) return 0;
   if (p.dt != UNIQL_F16) return 0;
   if ((p.K % (2 * kGroup)) != 0) return 0;
-  long tiles = 0;
+  if (count_tile_fams(p) > kMaxTF) return 0;
+  const int gran = copy_granule(p.K / kGroup);
   for (int j = 0; j < p.n_jobs; ++j) {
-    if (job_tiles(p.job[j]) < 1) return 0;
-    tiles += job_tiles(p.job[j]);
-    // scale / zero-point rows are copied in 4- or 8-byte granules
-    if (((uintptr_t)p.job[j].scales | (uintptr_t)p.job[j].zeros) & 7) return 0;
+    // scale / zero-point rows are copied in granules of 2, 4 or 8 fp16 values
+    if (((uintptr_t)p.job[j].scales | (uintptr_t)p.job[j].zeros) & (uintptr_t)(gran * 2 - 1)) return 0;
   }
-  return tiles <= kCounterInts;
+  return 1;
 }
 
 size_t decode_workspace_bytes(int M, int K, int N_total) {
-  // header (arrival counters, status word) + fp32 partial sums: at most 4 slots per 64-row tile and k-part
-  (void)K;
-  size_t tiles = (size_t)(N_total + RB - 1) / RB + 2 * kMaxJobs;
-  return (size_t)kWsHeader + tiles * (4 * kMaxKParts) * (size_t)M * RB * 4;
+  // header (arrival counters, status word) + fp32 partial sums [slots][M][64] per tile.  With many tiles
+  // a tile is shared by at most two blocks per k-part; with few tiles by at most one block per chunk
+  // (+2 per k-part).  Tiles: 64-row tiles plus one ragged tile per kept block, blocks of >= 32 rows assumed
+  // (the launch re-checks its exact need and returns UNIQL_ERR_WORKSPACE when this estimate is too small).
+  if (M > 16) return (size_t)kWsHeader;
+  DecodeCfg c;
+  memset(&c, 0, sizeof(c));
+  const int G = (K + kGroup - 1) / kGroup;
+  if (!plan_split(&c, M, G, 2)) return (size_t)kWsHeader;
+  const size_t chunks = (size_t)(G + CG - 1) / CG;
+  const size_t tiles = (size_t)(N_total + RB - 1) / RB + (size_t)N_total / 32 + 2 * kMaxJobs;
+  const size_t slots = tiles * 2 * c.n_kp + (size_t)c.n_rp * c.n_kp * (chunks + 2 * c.n_kp);
+  return (size_t)kWsHeader + slots * (size_t)M * RB * 4;
 }
 
 int launch_decode(const Params& p, const LaunchCfg& cfg) {
   DecodeCfg c;
   memset(&c, 0, sizeof(c));
   const int G = p.K / kGroup;
-  c.gran = (G % 4 == 0) ? 4 : 2;
-  visited_range(p.imap, c.gran, &c.v_first, &c.g_total);
+  const int gran = copy_granule(G);
+  int g_total = 0;
+  visited_range(p.imap, gran, &c.v_first, &g_total);
   const int MT = p.M <= 8 ? 1 : 2;
   // 128-bit staging: one leading family, everything 8-element aligned
   c.x_vec = p.imap.n_fam == 1 && p.imap.fam[0].count == 1 && (p.imap.fam[0].start % 8) == 0 &&
             (p.imap.fam[0].keep % 8) == 0 && (p.ldx % 8) == 0 && ((((uintptr_t)p.x) & 15) == 0);
-  int tiles = 0;
-  for (int j = 0; j < p.n_jobs; ++j) {
-    c.tile_begin[j] = tiles;
-    tiles += job_tiles(p.job[j]);
-  }
-  for (int j = p.n_jobs; j <= kMaxJobs; ++j) c.tile_begin[j] = tiles;
-  c.tiles_total = tiles;
-  if (tiles > kCounterInts) return UNIQL_ERR_SHAPE;
+  if (count_tile_fams(p) > kMaxTF) return UNIQL_ERR_UNSUPPORTED;
 
-  // ---- k-parts: as few as let the staged activations fit beside a deep enough ring of stages
-  const int part_bufs = p.M <= 8 ? 2 : 1;
-  int n_kp = env_int("UNIQL_DECODE_KP", 0);
-  int stages = env_int("UNIQL_DECODE_STAGES", 0);
-  size_t smem = 0;
-  bool fits = false;
-  if (n_kp >= 1) {
-    if (n_kp > kMaxKParts) n_kp = kMaxKParts;
-    const int gp = round_up((c.g_total + n_kp - 1) / n_kp, c.gran);
-    for (int s = (stages >= 2 && stages <= MAX_STAGES) ? stages : 4; s >= 2 && !fits; --s) {
-      smem = plan_smem(&c, p.M, MT, gp, s, part_bufs);
-      fits = smem <= (size_t)kSmemMax;
-    }
-    c.gp = gp;
-  } else {
-    const int want = (stages >= 2 && stages <= MAX_STAGES) ? stages : 4;
-    for (int s = want; s >= 3 && !fits; --s)
-      for (n_kp = 1; n_kp <= kMaxKParts && !fits; ++n_kp) {
-        const int gp = round_up((c.g_total + n_kp - 1) / n_kp, c.gran);
-        smem = plan_smem(&c, p.M, MT, gp, s, part_bufs);
-        fits = smem <= (size_t)kSmemMax;
-        c.gp = gp;
+  // ---- tile families and their tensor maps
+  const int x_extent = (c.v_first + g_total) * 64 < p.K / 2 ? (c.v_first + g_total) * 64 : p.K / 2;
+  int tiles = 0, n_tf = 0;
+  for (int j = 0; j < p.n_jobs; ++j) {
+    const JobDev& jb = p.job[j];
+    if (jb.rope.enabled) {
+      const int half = jb.rope.head_keep / 2;
+      TileFam& f = c.tf[n_tf];
+      f.tile_begin = tiles; f.tpb = (half + RB / 2 - 1) / (RB / 2); f.keep = half; f.count = jb.rope.n_heads;
+      f.job = j; f.start = 0; f.period = jb.rope.head_dim; f.out_base = 0;
+      const int rc = encode_family(&c.wmap[n_tf], jb.w, p.K, x_extent, half, 2 * jb.rope.n_heads,
+                                   jb.rope.head_dim / 2, RB / 2);
+      if (rc) return rc;
+      tiles += f.tpb * f.count;
+      ++n_tf;
+    } else {
+      for (int k = 0; k < jb.omap.n_fam; ++k) {
+        const Fam& a = jb.omap.fam[k];
+        TileFam& f = c.tf[n_tf];
+        f.tile_begin = tiles; f.tpb = (a.keep + RB - 1) / RB; f.keep = a.keep; f.count = a.count;
+        f.job = j; f.start = a.start; f.period = a.period; f.out_base = jb.omap.base[k];
+        const int rc = encode_family(&c.wmap[n_tf], jb.w + (size_t)a.start * (p.K / 2), p.K, x_extent, a.keep,
+                                     a.count, a.count > 1 ? a.period : a.keep, RB);
+        if (rc) return rc;
+        tiles += f.tpb * f.count;
+        ++n_tf;
       }
+    }
   }
-  if (!fits) return UNIQL_ERR_UNSUPPORTED;
-  c.n_kp = (c.g_total + c.gp - 1) / c.gp;
-  int n_rp = env_int("UNIQL_DECODE_RP", 0);
-  if (n_rp < 1) n_rp = sm_count() / c.n_kp;
-  if (n_rp < 1) n_rp = 1;
-  c.n_rp = n_rp;
+  c.n_tf = n_tf;
+  c.tiles_total = tiles;
+  if (tiles < 1 || tiles > kCounterInts) return UNIQL_ERR_UNSUPPORTED;
+
+  const size_t smem = plan_split(&c, p.M, g_total, gran);
+  if (!smem) return UNIQL_ERR_UNSUPPORTED;
   c.max_slots = slots_needed(tiles, c.g_total, c.gp, c.n_rp);
   {
     const size_t need = (size_t)kWsHeader + (size_t)tiles * c.max_slots * p.M * RB * 4;
