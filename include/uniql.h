@@ -136,6 +136,27 @@ int uniql_workspace_status(void* workspace, int* status);
 int uniql_qlinear(const void* x, const uint8_t* packed_w, const void* scales, const void* zeros,
                   int M, int K, int N, int k_in, int k_out, void* y, void* stream);
 
+/* The same layer for callers that cannot allocate device memory (no counterpart in the paper: this
+ * is a property of the library, not of the method).  Think of a serving process whose device memory
+ * was handed out completely at start-up, a real-time loop in which cudaMalloc could stall on the
+ * driver, or a sandbox in which the call is forbidden.  Nothing is allocated here, by this library or
+ * by anything it calls: the scratch memory of the decode kernel is a fixed array of
+ * UNIQL_NOALLOC_SCRATCH_BYTES inside the library's device image (every GPU that loads the library
+ * carries it until the process ends).
+ *  - Arguments as uniql_qlinear (fp16, leading k_in x k_out block); decode only: M <= 16, else
+ *    UNIQL_ERR_UNSUPPORTED.  A problem whose split-K partial sums do not fit the fixed array returns
+ *    UNIQL_ERR_WORKSPACE and launches nothing.  The need is 256 KB plus roughly 512 bytes per 64
+ *    retained rows and batch row (more when large M * K splits the input channels over several
+ *    groups of thread blocks); the Llama-3-8B MLP matrices fit for every M <= 16.
+ *  - The first call on a device looks up the array's device address (once per device, with that
+ *    device current); make that first call outside any stream capture.
+ *  - All calls share the one array, and it keeps what the previous call left: each call clears the
+ *    part that must start at zero on `stream` before it launches.  Two calls that may overlap on the
+ *    GPU (different streams without ordering between them) race on it: order them. */
+#define UNIQL_NOALLOC_SCRATCH_BYTES (8u << 20)
+int uniql_qlinear_noalloc(const void* x, const uint8_t* packed_w, const void* scales, const void* zeros,
+                          int M, int K, int N, int k_in, int k_out, void* y, void* stream);
+
 /* General form: dtype, leading dimensions, bias, channel maps (NULL map = leading k).
  * x and y must be 4-byte aligned with even ldx / ldy; every family's start and keep must be
  * multiples of 4.  workspace may be NULL (library buffer). */

@@ -61,6 +61,7 @@ _lib.uniql_workspace_bytes.argtypes = [_i, _i, _i]
 _lib.uniql_workspace_init.argtypes = [_vp, _sz, _vp]
 _lib.uniql_workspace_status.argtypes = [_vp, ctypes.POINTER(_i)]
 _lib.uniql_qlinear.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp]
+_lib.uniql_qlinear_noalloc.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp]
 _lib.uniql_qlinear_ex.argtypes = [_vp, _i, _i, _vp, _vp, _vp, _vp, _i, _i, _i, ctypes.POINTER(_ChanMap), _i,
                                   ctypes.POINTER(_ChanMap), _i, _vp, _i, _vp, _sz, _vp]
 _lib.uniql_qlinear_multi.argtypes = [_vp, _i, _i, _i, _i, ctypes.POINTER(_ChanMap), _i, _i,
@@ -68,7 +69,7 @@ _lib.uniql_qlinear_multi.argtypes = [_vp, _i, _i, _i, _i, ctypes.POINTER(_ChanMa
 _lib.uniql_qk_rope_proj.argtypes = [_vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i,
                                     _vp, _vp, _d, ctypes.POINTER(_d), _vp, _i, _vp, _i, _vp, _sz, _vp]
 for _n in ("uniql_set_path", "uniql_pack_u4", "uniql_unpack_u4", "uniql_dequant", "uniql_workspace_init",
-           "uniql_workspace_status", "uniql_qlinear", "uniql_qlinear_ex", "uniql_qlinear_multi", "uniql_qk_rope_proj"):
+           "uniql_workspace_status", "uniql_qlinear", "uniql_qlinear_noalloc", "uniql_qlinear_ex", "uniql_qlinear_multi", "uniql_qk_rope_proj"):
     getattr(_lib, _n).restype = _i
 
 
@@ -162,6 +163,13 @@ def workspace_status(ws: Optional[torch.Tensor] = None) -> int:
 def qlinear(x, packed_w, scales, zeros, M, K, N, k_in, k_out, y, stream=None) -> None:
     _check(_lib.uniql_qlinear(_ptr(x), _ptr(packed_w), _ptr(scales), _ptr(zeros), M, K, N, k_in, k_out, _ptr(y),
                               _stream(stream)), "uniql_qlinear")
+
+
+def qlinear_noalloc(x, packed_w, scales, zeros, M, K, N, k_in, k_out, y, stream=None) -> None:
+    """uniql_qlinear for callers that must not allocate device memory: the kernel's scratch is a fixed
+    array inside the library (decode sizes only, M <= 16)."""
+    _check(_lib.uniql_qlinear_noalloc(_ptr(x), _ptr(packed_w), _ptr(scales), _ptr(zeros), M, K, N, k_in, k_out,
+                                      _ptr(y), _stream(stream)), "uniql_qlinear_noalloc")
 
 
 def qlinear_ex(x, ldx, packed_w, scales, zeros, bias, M, K, N, in_map, k_in, out_map, k_out, y, ldy,

@@ -139,6 +139,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg);
 int decode_supported(const Params& p);
 size_t decode_workspace_bytes(int M, int K, int N_total);
 int decode_status_offset();   // byte offset of the device status word inside a workspace
+size_t decode_workspace_header_bytes();   // counters + status word: the part that must start at zero
 int launch_prefill(const Params& p, const LaunchCfg& cfg);
 int prefill_supported(const Params& p);
 

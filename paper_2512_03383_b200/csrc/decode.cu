@@ -901,5 +901,6 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
 }
 
 int decode_status_offset() { return kStatusOff; }
+size_t decode_workspace_header_bytes() { return (size_t)kWsHeader; }
 
 }  // namespace uniql
