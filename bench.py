@@ -219,7 +219,20 @@ class MlpDecode:
         return h2d, d2h
 
 
-def capture(torch, fn):
+class Eager:
+    """Stand-in for a captured graph that launches the step directly (profiler launch lists:
+    ncu could not launch this kernel as a node of a replayed graph on this pool)."""
+
+    def __init__(self, fn):
+        self.fn = fn
+
+    def replay(self):
+        self.fn()
+
+
+def capture(torch, fn, eager=False):
+    if eager:
+        return Eager(fn), fn()
     g = torch.cuda.CUDAGraph()
     s = torch.cuda.Stream()
     s.wait_stream(torch.cuda.current_stream())
@@ -292,8 +305,8 @@ def run_ours(args):
     from paper_2512_03383_b200 import binding as B
 
     work = MlpDecode(B, torch, 1)
-    graph, _ = capture(torch, work.step)
-    graph_e2e, (h2d, d2h) = capture(torch, lambda: work.step(e2e=True))
+    graph, _ = capture(torch, work.step, args.no_graph)
+    graph_e2e, (h2d, d2h) = capture(torch, lambda: work.step(e2e=True), args.no_graph)
 
     sampler = ClockSampler(local)
     if rank == 0:
@@ -345,12 +358,13 @@ def run_ours(args):
         "config": {"workload": "llama3-8b-mlp-decode-M1 (BASELINE configs[1])", "hidden": HIDDEN,
                    "intermediate": INTER, "keep_rates": list(KEEP_RATES), "M": 1,
                    "l2": "4 rotating weight copies (375 MB) > 126 MB L2", "parallelism": "replicas x%d" % world,
-                   "timing": "CUDA graph of one step replayed, CUDA events"},
+                   "timing": ("eager launches (profiling mode, host-bound: not a bench value), CUDA events" if args.no_graph
+                              else "CUDA graph of one step replayed, CUDA events")},
         "tokens_per_s_mlp": args.steps * len(KEEP_RATES) * world / sec,
         "gpu_launches": launches,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s", "frac": achieved / hbm,
-                     "traffic": DRAM_TRAFFIC_PER_LAUNCH, "peak_source": which,
+                     "traffic": None if DRAM_TRAFFIC_RATIO is None else DRAM_TRAFFIC_RATIO * per_launch_bytes, "peak_source": which,
                      "kernel": "decode_kernel<half,1>", "algorithmic_bytes_per_launch": per_launch_bytes,
                      "frac_of_nominal_8TBs": achieved / 8000.0},
         "e2e": {"value": step_bytes() * args.steps * world / sec_e2e / 1e9, "unit": "GB/s",
@@ -392,8 +406,11 @@ def run_case(args):
     return 0
 
 
-# DRAM bytes (read + write) per decode launch from the ncu capture summarised under profiles/; None until taken.
-DRAM_TRAFFIC_PER_LAUNCH = None
+# DRAM bytes (read + write) per algorithmic byte of a decode launch, from the ncu capture summarised in
+# profiles/decode_kernel_llama3_gateup_m1.md (62.47 MB read + 0.15 MB written for 62.39 MB of retained weights);
+# traffic grows in proportion to the retained weights, so the per-launch average of the step is scaled from it.
+# None once the kernel has changed since the capture.
+DRAM_TRAFFIC_RATIO = 62.62 / 62.39
 
 
 def main():
@@ -402,6 +419,8 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-graph", action="store_true",
+                    help="launch eagerly instead of replaying a CUDA graph (for profiler launch lists only)")
     ap.add_argument("--detail", action="store_true", help="also report M=4/16 and per-keep-rate tables")
     ap.add_argument("--case", default=None, help="run a few plain launches of one kernel (for ncu)")
     ap.add_argument("--M", type=int, default=1)
