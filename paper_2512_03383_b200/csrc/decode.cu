@@ -197,6 +197,15 @@ __device__ inline TilePos tile_pos(const DecodeCfg& c, const Params& p, int tg) 
   q.r0 = (tl - q.h * f.tpb) * rows;
   return q;
 }
+// position of the next tile (tiles are numbered block after block, family after family)
+__device__ inline void next_tile(const DecodeCfg& c, const Params& p, TilePos& q) {
+  const TileFam& f = c.tf[q.fi];
+  q.r0 += p.job[f.job].rope.enabled ? RB / 2 : RB;
+  if (q.r0 >= f.keep) {
+    q.r0 = 0;
+    if (++q.h == f.count) { q.h = 0; ++q.fi; }
+  }
+}
 
 // The block (of its k-part) whose unit range [U*b/B, U*(b+1)/B) holds unit u; exact in fp64 here.
 __device__ inline int owner_of(long u, long B, long U) {
@@ -297,7 +306,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       if (it >= S) ok = mbar_wait(bar_empty + 8 * s, ring_parity, abort_flag);
       if (!ok) break;
       if (tile != tile_prev) {
-        q = tile_pos(c, p, tile);
+        if (tile_prev < 0) q = tile_pos(c, p, tile); else next_tile(c, p, q);
         const TileFam& f = c.tf[q.fi];
         const JobDev& jb = p.job[f.job];
         rope = jb.rope.enabled != 0;
@@ -484,6 +493,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       for (int i = 0; i < 4; ++i) out[sub][mt][i] = 0.f;
 
   int tile = ub / Ck, chunk = ub - tile * Ck;
+  TilePos q = tile_pos(c, p, tile);
   int tiles_done = 0;
   int s = 0;                 // ring position and the parity of its current use
   uint32_t ring_parity = 0;
@@ -602,9 +612,12 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         for (int q8 = 0; q8 < CG; ++q8) v += pr[q8 * RM + m * RB + slot];
         return v;
       };
-      // how many blocks (over all k-parts) work on this tile, and which of them am I
+      // how many blocks (over all k-parts) work on this tile, and which of them am I; a tile whose
+      // chunks all lie in this block's range (the usual case) needs none of that arithmetic
       int total = 0, my_slot = 0;
-      for (int q2 = 0; q2 < c.n_kp; ++q2) {
+      const bool whole_here = c.n_kp == 1 && tile * Ck >= ub && tile * Ck + Ck <= ue;
+      if (whole_here) total = 1;
+      for (int q2 = 0; q2 < (whole_here ? 0 : c.n_kp); ++q2) {
         const int Gq = min(c.gp, c.g_total - q2 * c.gp);
         const long Cq = (Gq + CG - 1) / CG;
         const long Uq = (long)c.tiles_total * Cq;
@@ -614,7 +627,6 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         if (q2 == kp) my_slot = total + (rp - first);
         total += last - first + 1;
       }
-      const TilePos q = tile_pos(c, p, tile);
       const TileFam& f = c.tf[q.fi];
       if (total == 1) {
         store_tile<T>(p, f, q, ctid, local_sum);
@@ -644,7 +656,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       if (c.part_bufs == 1 && !consumer_sync()) return;
       ++tiles_done;
     }
-    if (++chunk == Ck) { chunk = 0; ++tile; }
+    if (++chunk == Ck) { chunk = 0; ++tile; next_tile(c, p, q); }
   }
 }
 
