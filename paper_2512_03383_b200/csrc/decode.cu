@@ -3,18 +3,19 @@
 // The decode step streams every retained weight exactly once, so the kernel is built around keeping
 // HBM busy: one persistent block per SM whose producer warp keeps a ring of shared-memory stages
 // filled by the tensor memory accelerator (cp.async.bulk.tensor boxes of 128 bytes x 64 rows,
-// completion on an mbarrier), far ahead of the sixteen consumer warps.  Neither side spends registers
-// or issue slots on memory latency.  On-device pruning (Section 3.4) is expressed in the tensor maps:
+// completion on an mbarrier), far ahead of the sixteen consumer warps, and whose two epilogue warps
+// finish tiles (reduction over the consumer warps, bias, rotary embedding, store) behind them.  No
+// role spends registers or issue slots on another role's latency.  On-device pruning (Section 3.4) is expressed in the tensor maps:
 // a family of kept channel blocks {start, period, keep, count} is a 3-D tensor (byte in row, row in
 // block, block) whose extents stop at the kept rows and at the last visited input group, so pruned
 // rows and pruned trailing input channels are out of bounds: never fetched, filled with zeros.
 //
 // Work decomposition.  A tile is 64 row slots of one kept block, a chunk is 8 quantisation groups
-// (1024 input channels, 512 bytes per row).  All (tile, chunk) units of the launch form one
-// chunk-fastest sequence that is cut into equal contiguous ranges, one per block (stream-K): every SM
-// streams the same number of bytes.  A tile that is shared by several blocks is finished by the last
-// block to arrive, which adds the parked partial sums in a fixed slot order (deterministic, no
-// spinning on other blocks).
+// (1024 input channels, 512 bytes per row).  Every block first takes the same number of whole tiles;
+// the (tile, chunk) units of the tiles left over form one chunk-fastest sequence that is cut into equal
+// contiguous ranges, one per block (stream-K), so every SM streams the same number of bytes.  A tile
+// that is shared by several blocks is finished by the last block to arrive, which adds the parked
+// partial sums in a fixed slot order (deterministic, no spinning on other blocks).
 //
 // Arithmetic.  Inside a stage consumer warp w owns group (w & 7) of the chunk and two 16-row
 // sub-tiles.  The packed codes are used as they lie in memory: one LOP3 turns two nibbles of a 32-bit
@@ -42,7 +43,9 @@ namespace {
 
 constexpr int CW = 16;                  // consumer warps
 constexpr int CTH = CW * 32;            // consumer threads
-constexpr int NTH = CTH + 32;           // + one producer warp
+constexpr int EW = 2;                   // epilogue warps
+constexpr int ETH = EW * 32;
+constexpr int NTH = CTH + 32 + ETH;     // consumers + one producer warp + epilogue warps
 constexpr int RB = 64;                  // row slots per tile
 constexpr int CG = 8;                   // groups per chunk
 constexpr int BOX_COLS = CG / 2;        // 128-byte columns (two groups each) per chunk
@@ -57,7 +60,7 @@ constexpr int kWsHeader = kStatusOff + 256;
 constexpr int kMaxKParts = 16;
 constexpr int kSmemMax = 227 * 1024;
 constexpr int kWaitLimit = 1 << 18;
-constexpr int BAR_BYTES = 128;
+constexpr int BAR_BYTES = 256;
 constexpr int kMaxTF = 8;               // (job, family) pairs of one launch
 
 // One family of kept row blocks of one job: `count` blocks of `keep` rows, tiles of RB rows inside each
@@ -214,13 +217,13 @@ __device__ inline int owner_of(long u, long B, long U) {
 
 // bias, rotary embedding on the retained pair, one rounding, store; `get(slot, m)` yields the fp32 sum
 template <typename T, typename F>
-__device__ inline void store_tile(const Params& p, const TileFam& f, const TilePos& q, int ctid, F get) {
+__device__ inline void store_tile(const Params& p, const TileFam& f, const TilePos& q, int etid, F get) {
   const JobDev& jb = p.job[f.job];
   const T* bias = reinterpret_cast<const T*>(jb.bias);
   T* y = reinterpret_cast<T*>(jb.y);
   if (jb.rope.enabled) {
     const int half = jb.rope.head_keep >> 1;
-    for (int i = ctid; i < (RB / 2) * p.M; i += CTH) {
+    for (int i = etid; i < (RB / 2) * p.M; i += ETH) {
       const int pp = i & (RB / 2 - 1), m = i / (RB / 2);
       const int cc = q.r0 + pp;
       if (cc >= half) continue;
@@ -239,7 +242,7 @@ __device__ inline void store_tile(const Params& p, const TileFam& f, const TileP
       y[(size_t)m * jb.ldy + oc + half] = DT<T>::from_f(hi * cs + lo * sn);
     }
   } else {
-    for (int i = ctid; i < RB * p.M; i += CTH) {
+    for (int i = etid; i < RB * p.M; i += ETH) {
       const int slot = i & (RB - 1), m = i / RB;
       const int r = q.r0 + slot;
       if (r >= f.keep) continue;
@@ -249,6 +252,50 @@ __device__ inline void store_tile(const Params& p, const TileFam& f, const TileP
     }
   }
 }
+
+// ---------------------------------------------------------------------------------------- work split
+// Units of one block of k-part `kp`: first `base` whole tiles (all chunks), then a contiguous range of
+// the chunk-fastest unit sequence of the R tiles that are left over after every block took its share.
+struct Work {
+  int Ck;            // chunks per tile in this k-part
+  int n1;            // units of the whole-tile phase (base * Ck)
+  int tile1;         // first whole tile
+  int tail_tile0;    // first left-over tile (n_rp * base)
+  int tb, te;        // tail unit range [tb, te) in the left-over sequence
+  int n_units;
+};
+__device__ inline Work block_work(const DecodeCfg& c, int Ck, int rp) {
+  Work w;
+  w.Ck = Ck;
+  const int base = c.tiles_total / c.n_rp;
+  const int R = c.tiles_total - base * c.n_rp;
+  const long Ut = (long)R * Ck;
+  const long Bt = (long)c.n_rp < Ut ? (long)c.n_rp : Ut;      // blocks that get tail units
+  w.n1 = base * Ck;
+  w.tile1 = rp * base;
+  w.tail_tile0 = c.n_rp * base;
+  w.tb = w.te = 0;
+  if (rp < Bt) { w.tb = (int)(Ut * rp / Bt); w.te = (int)(Ut * (rp + 1) / Bt); }
+  w.n_units = w.n1 + (w.te - w.tb);
+  return w;
+}
+// (tile, chunk) of block-local unit i, walked in order
+struct UnitIter {
+  int tile, chunk;
+  __device__ inline void start(const Work& w) {
+    if (w.n1 > 0) { tile = w.tile1; chunk = 0; }
+    else { tile = w.tail_tile0 + w.tb / w.Ck; chunk = w.tb - (w.tb / w.Ck) * w.Ck; }
+  }
+  // returns true when the position jumped (phase switch), i.e. the tile position must be recomputed
+  __device__ inline bool advance(const Work& w, int i_next) {
+    if (i_next == w.n1 && w.n1 > 0) {
+      tile = w.tail_tile0 + w.tb / w.Ck; chunk = w.tb - (w.tb / w.Ck) * w.Ck;
+      return true;
+    }
+    if (++chunk == w.Ck) { chunk = 0; ++tile; }
+    return false;
+  }
+};
 
 // ---------------------------------------------------------------------------------------- kernel
 template <int MT, bool ONECOL>
@@ -262,10 +309,12 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   const uint32_t sbase = (raw + 1023u) & ~1023u;
   unsigned char* smem = smem_raw + (sbase - raw);
   const int S = c.stages;
-  // barriers: full[S], empty[S], consumer barrier; then two flags
-  const uint32_t bar_full = sbase + c.off_bar, bar_empty = bar_full + 8 * MAX_STAGES, bar_cons = bar_full + 16 * MAX_STAGES;
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + c.off_bar + 16 * MAX_STAGES + 8);
-  volatile int* last_flag = reinterpret_cast<volatile int*>(smem + c.off_bar + 16 * MAX_STAGES + 12);
+  // barriers: full[S], empty[S], consumer barrier, epilogue barrier, partials full[2] / free[2]; then flags
+  const uint32_t bar_full = sbase + c.off_bar, bar_empty = bar_full + 8 * MAX_STAGES;
+  const uint32_t bar_cons = bar_full + 16 * MAX_STAGES, bar_epi = bar_cons + 8;
+  const uint32_t bar_pfull = bar_cons + 16, bar_pfree = bar_cons + 32;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + c.off_bar + 16 * MAX_STAGES + 48);
+  volatile int* last_flag = reinterpret_cast<volatile int*>(smem + c.off_bar + 16 * MAX_STAGES + 52);
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) {
@@ -273,6 +322,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       mbar_init(bar_empty + 8 * s, CW);
     }
     mbar_init(bar_cons, CW);
+    mbar_init(bar_epi, EW);
+    for (int b = 0; b < 2; ++b) { mbar_init(bar_pfull + 8 * b, CW); mbar_init(bar_pfree + 8 * b, EW); }
     *abort_flag = 0;
     *last_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -282,19 +333,17 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   const int kp = blockIdx.x / c.n_rp, rp = blockIdx.x - kp * c.n_rp;
   const int v_lo = kp * c.gp;                                   // first visit index of this k-part
   const int Gk = min(c.gp, c.g_total - v_lo);                   // its groups
-  const int Ck = (Gk + CG - 1) / CG;                            // chunks per tile
   const int sg_lo = c.v_first + v_lo;                           // first stored group of this k-part
   const int G = p.K / kGroup;
-  const long U = (long)c.tiles_total * Ck;
-  const long Bn = (long)c.n_rp < U ? (long)c.n_rp : U;          // blocks that get work
-  int ub = 0, ue = 0;
-  if (rp < Bn) { ub = (int)(U * rp / Bn); ue = (int)(U * (rp + 1) / Bn); }
-  if (ub >= ue) return;
+  const Work wk = block_work(c, (Gk + CG - 1) / CG, rp);
+  if (wk.n_units == 0) return;
 
   // ======================================================================================= producer
   if (warp == CW) {
-    int tile = ub / Ck, chunk = ub - tile * Ck;
+    UnitIter ui;
+    ui.start(wk);
     int tile_prev = -1;
+    bool jumped = true;
     TilePos q = {0, 0, 0};
     bool rope = false;
     const __half* srow[2] = {nullptr, nullptr};
@@ -302,11 +351,12 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     int it = 0, s = 0;
     uint32_t ring_parity = 1;      // parity of the previous use of ring position s
     bool ok = true;
-    for (int u = ub; u < ue; ++u, ++it) {
+    for (; it < wk.n_units; ++it) {
       if (it >= S) ok = mbar_wait(bar_empty + 8 * s, ring_parity, abort_flag);
       if (!ok) break;
-      if (tile != tile_prev) {
-        if (tile_prev < 0) q = tile_pos(c, p, tile); else next_tile(c, p, q);
+      if (ui.tile != tile_prev) {
+        if (jumped) q = tile_pos(c, p, ui.tile); else next_tile(c, p, q);
+        jumped = false;
         const TileFam& f = c.tf[q.fi];
         const JobDev& jb = p.job[f.job];
         rope = jb.rope.enabled != 0;
@@ -324,8 +374,9 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           srow[r2] = sr >= 0 ? jb.scales + (size_t)sr * G + sg_lo : nullptr;
           zrow[r2] = sr >= 0 ? jb.zeros + (size_t)sr * G + sg_lo : nullptr;
         }
-        tile_prev = tile;
+        tile_prev = ui.tile;
       }
+      const int chunk = ui.chunk;
       const int ng = min(CG, Gk - chunk * CG);
       const int nb = (ng + 1) >> 1;                      // 128-byte columns with a visited group
       const uint32_t full = bar_full + 8 * s;
@@ -359,7 +410,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         }
       }
       cp_async_arrive_noinc(full);
-      if (++chunk == Ck) { chunk = 0; ++tile; }
+      if (it + 1 < wk.n_units && ui.advance(wk, it + 1)) jumped = true;
       if (++s == S) { s = 0; ring_parity ^= 1; }
     }
     if (!ok) {
@@ -370,6 +421,105 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         for (int i = 0; i < kWaitLimit && !mbar_try_wait(full, (j / S) & 1); ++i) {}
       }
       if (lane == 0) atomicExch(c.status, UNIQL_ERR_TIMEOUT);
+    }
+    return;
+  }
+
+  float* part = reinterpret_cast<float*>(smem + c.off_part);
+  const int RM = RB * p.M;
+  const int part_stride = CG * RM;           // floats per partial buffer
+
+  // ======================================================================================= epilogue
+  // Finishes the block's tiles in order, behind the consumers: sums the eight parked group partials of
+  // every (row slot, batch row), then stores the tile, or parks the sum for the block that finishes it.
+  if (warp > CW) {
+    const int etid = tid - (CW + 1) * 32;
+    uint32_t epi_parity = 0;
+    auto give_up = [&]() { if (lane == 0) atomicExch(c.status, UNIQL_ERR_TIMEOUT); };
+    auto epi_sync = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_epi);
+      const bool ok = mbar_wait(bar_epi, epi_parity, abort_flag);
+      epi_parity ^= 1;
+      if (!ok) give_up();
+      return ok;
+    };
+    UnitIter ui;
+    ui.start(wk);
+    TilePos q = tile_pos(c, p, ui.tile);
+    int tiles_done = 0;
+    for (int i = 0; i < wk.n_units; ++i) {
+      const bool tile_end = (ui.chunk == wk.Ck - 1) || (i == wk.n_units - 1);
+      if (tile_end) {
+        const int buf = c.part_bufs > 1 ? (tiles_done & 1) : 0;
+        const int use = c.part_bufs > 1 ? (tiles_done >> 1) : tiles_done;
+        if (!mbar_wait(bar_pfull + 8 * buf, use & 1, abort_flag)) { give_up(); return; }
+        const float* pr = part + buf * part_stride;
+        auto local_sum = [&](int slot, int m) -> float {
+          float v = 0.f;
+#pragma unroll
+          for (int q8 = 0; q8 < CG; ++q8) v += pr[q8 * RM + m * RB + slot];
+          return v;
+        };
+        const int tile = ui.tile;
+        const TileFam& f = c.tf[q.fi];
+        // how many blocks (over all k-parts) work on this tile, and which of them am I
+        int total = 0, my_slot = 0;
+        const bool tail = tile >= wk.tail_tile0;
+        if (c.n_kp == 1 && !tail) {
+          total = 1;
+        } else {
+          const int base = c.tiles_total / c.n_rp;
+          const int R = c.tiles_total - base * c.n_rp;
+          for (int q2 = 0; q2 < c.n_kp; ++q2) {
+            int n_here = 1, first = rp;                      // a whole tile: one block per k-part
+            if (tail) {
+              const int Gq = min(c.gp, c.g_total - q2 * c.gp);
+              const long Cq = (Gq + CG - 1) / CG;
+              const long Ut = (long)R * Cq;
+              const long Bt = (long)c.n_rp < Ut ? (long)c.n_rp : Ut;
+              const long t0 = (long)(tile - wk.tail_tile0) * Cq;
+              first = owner_of(t0, Bt, Ut);
+              n_here = owner_of(t0 + Cq - 1, Bt, Ut) - first + 1;
+            }
+            if (q2 == kp) my_slot = total + (rp - first);
+            total += n_here;
+          }
+        }
+        if (total == 1) {
+          store_tile<T>(p, f, q, etid, local_sum);
+        } else {
+          float* tile_ws = c.partials + (size_t)tile * c.max_slots * RM;
+          float* mine = tile_ws + (size_t)my_slot * RM;
+          for (int j = etid; j < RM; j += ETH) __stcg(mine + j, local_sum(j & (RB - 1), j / RB));
+          __threadfence();
+          if (!epi_sync()) return;
+          if (etid == 0) {
+            const int arrived = atomicAdd(&c.counters[tile], 1);
+            *last_flag = arrived == total - 1;
+            __threadfence();
+          }
+          if (!epi_sync()) return;
+          if (*last_flag) {
+            auto global_sum = [&](int slot, int m) -> float {
+              float v = 0.f;
+              for (int s2 = 0; s2 < total; ++s2) v += __ldcg(tile_ws + (size_t)s2 * RM + m * RB + slot);
+              return v;
+            };
+            store_tile<T>(p, f, q, etid, global_sum);
+            if (etid == 0) c.counters[tile] = 0;       // ready for the next call
+          }
+          if (!epi_sync()) return;                     // last_flag may be rewritten only after everyone read it
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_pfree + 8 * buf);
+        ++tiles_done;
+      }
+      if (i + 1 < wk.n_units) {
+        const int tile_before = ui.tile;
+        if (ui.advance(wk, i + 1)) q = tile_pos(c, p, ui.tile);
+        else if (ui.tile != tile_before) next_tile(c, p, q);
+      }
     }
     return;
   }
@@ -481,8 +631,6 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   const uint32_t xgaddr = sbase + c.off_xg + (uint32_t)(2 * t * 8);
   const uint32_t wl_off = (uint32_t)((kpw >> 1) * BOX_BYTES + (rg * 32 + pg) * 128 + ((((kpw & 1) * 4 + t) ^ pg) * 16));
   const uint32_t sl_off = (uint32_t)(STAGE_W + (rg * 32 + pg) * (CG * 2) + kpw * 2);
-  float* part = reinterpret_cast<float*>(smem + c.off_part);
-  const int part_stride = CG * RB * p.M;     // floats per partial buffer
 
   float out[2][MT][4];
 #pragma unroll
@@ -492,8 +640,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
 #pragma unroll
       for (int i = 0; i < 4; ++i) out[sub][mt][i] = 0.f;
 
-  int tile = ub / Ck, chunk = ub - tile * Ck;
-  TilePos q = tile_pos(c, p, tile);
+  UnitIter ui;
+  ui.start(wk);
   int tiles_done = 0;
   int s = 0;                 // ring position and the parity of its current use
   uint32_t ring_parity = 0;
@@ -502,12 +650,12 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
     for (int j = 0; j < 4; ++j) xr[mt][j] = make_uint4(0, 0, 0, 0);
-  for (int u = ub; u < ue; ++u) {
+  for (int i = 0; i < wk.n_units; ++i) {
     if (!mbar_try_wait(bar_full + 8 * s, ring_parity) && !mbar_wait(bar_full + 8 * s, ring_parity, abort_flag)) {
       give_up();
       return;
     }
-    const int gi = chunk * CG + kpw;
+    const int gi = ui.chunk * CG + kpw;
     if (gi < Gk) {
       const uint32_t st = sbase + (uint32_t)s * STAGE_BYTES;
       const uint32_t wp = st + wl_off, sp = st + sl_off;
@@ -580,10 +728,13 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     if (lane == 0) mbar_arrive(bar_empty + 8 * s);
     if (++s == S) { s = 0; ring_parity ^= 1; }
 
-    const bool tile_end = (chunk == Ck - 1) || (u == ue - 1);
+    const bool tile_end = (ui.chunk == wk.Ck - 1) || (i == wk.n_units - 1);
     if (tile_end) {
-      // ---- park this warp's partial sums: part[buf][group slot kpw][m][row slot]
-      float* pb = part + (c.part_bufs > 1 ? (tiles_done & 1) * part_stride : 0) + kpw * RB * p.M;
+      // ---- park this warp's partial sums for the epilogue warps: part[buf][group slot kpw][m][row slot]
+      const int buf = c.part_bufs > 1 ? (tiles_done & 1) : 0;
+      const int use = c.part_bufs > 1 ? (tiles_done >> 1) : tiles_done;
+      if (use > 0 && !mbar_wait(bar_pfree + 8 * buf, (use - 1) & 1, abort_flag)) { give_up(); return; }
+      float* pb = part + buf * part_stride + kpw * RM;
 #pragma unroll
       for (int sub = 0; sub < 2; ++sub)
 #pragma unroll
@@ -601,62 +752,12 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-          for (int i = 0; i < 4; ++i) out[sub][mt][i] = 0.f;
-      if (!consumer_sync()) return;
-
-      const float* pr = part + (c.part_bufs > 1 ? (tiles_done & 1) * part_stride : 0);
-      const int RM = RB * p.M;
-      auto local_sum = [&](int slot, int m) -> float {
-        float v = 0.f;
-#pragma unroll
-        for (int q8 = 0; q8 < CG; ++q8) v += pr[q8 * RM + m * RB + slot];
-        return v;
-      };
-      // how many blocks (over all k-parts) work on this tile, and which of them am I; a tile whose
-      // chunks all lie in this block's range (the usual case) needs none of that arithmetic
-      int total = 0, my_slot = 0;
-      const bool whole_here = c.n_kp == 1 && tile * Ck >= ub && tile * Ck + Ck <= ue;
-      if (whole_here) total = 1;
-      for (int q2 = 0; q2 < (whole_here ? 0 : c.n_kp); ++q2) {
-        const int Gq = min(c.gp, c.g_total - q2 * c.gp);
-        const long Cq = (Gq + CG - 1) / CG;
-        const long Uq = (long)c.tiles_total * Cq;
-        const long Bq = (long)c.n_rp < Uq ? (long)c.n_rp : Uq;
-        const int first = owner_of((long)tile * Cq, Bq, Uq);
-        const int last = owner_of((long)tile * Cq + Cq - 1, Bq, Uq);
-        if (q2 == kp) my_slot = total + (rp - first);
-        total += last - first + 1;
-      }
-      const TileFam& f = c.tf[q.fi];
-      if (total == 1) {
-        store_tile<T>(p, f, q, ctid, local_sum);
-      } else {
-        float* tile_ws = c.partials + (size_t)tile * c.max_slots * RM;
-        float* mine = tile_ws + (size_t)my_slot * RM;
-        for (int i = ctid; i < RM; i += CTH) __stcg(mine + i, local_sum(i & (RB - 1), i / RB));
-        __threadfence();
-        if (!consumer_sync()) return;
-        if (ctid == 0) {
-          const int arrived = atomicAdd(&c.counters[tile], 1);
-          *last_flag = arrived == total - 1;
-          __threadfence();
-        }
-        if (!consumer_sync()) return;
-        if (*last_flag) {
-          auto global_sum = [&](int slot, int m) -> float {
-            float v = 0.f;
-            for (int s2 = 0; s2 < total; ++s2) v += __ldcg(tile_ws + (size_t)s2 * RM + m * RB + slot);
-            return v;
-          };
-          store_tile<T>(p, f, q, ctid, global_sum);
-          if (ctid == 0) c.counters[tile] = 0;       // ready for the next call
-        }
-        if (!consumer_sync()) return;                // last_flag may be rewritten only after everyone read it
-      }
-      if (c.part_bufs == 1 && !consumer_sync()) return;
+          for (int i2 = 0; i2 < 4; ++i2) out[sub][mt][i2] = 0.f;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_pfull + 8 * buf);
       ++tiles_done;
     }
-    if (++chunk == Ck) { chunk = 0; ++tile; next_tile(c, p, q); }
+    if (i + 1 < wk.n_units) ui.advance(wk, i + 1);
   }
 }
 
@@ -743,16 +844,19 @@ size_t plan_smem(DecodeCfg* c, int M, int MT, int gp, int stages, int part_bufs)
   return off + 1024;
 }
 
-// Worst-case number of workspace slots a tile needs for a given split.
+// Worst-case number of workspace slots a tile needs for a given split: one per k-part for a whole tile,
+// one per block that shares it for a left-over tile.
 int slots_needed(int tiles, int g_total, int gp, int n_rp) {
   int total = 0;
+  const int base = tiles / n_rp;
+  const long R = tiles - (long)base * n_rp;
   for (int v = 0; v < g_total; v += gp) {
     const long Gq = (g_total - v) < gp ? (g_total - v) : gp;
     const long Cq = (Gq + CG - 1) / CG;
-    const long Uq = (long)tiles * Cq;
-    long Bq = (long)n_rp;
-    if (Bq > Uq) Bq = Uq;
-    const long per_block = Uq / Bq;           // >= 1
+    const long Ut = R * Cq;
+    if (Ut == 0) { total += 1; continue; }
+    const long Bt = (long)n_rp < Ut ? (long)n_rp : Ut;
+    const long per_block = Ut / Bt;           // >= 1
     total += (int)((Cq + per_block - 1) / per_block) + 1;
   }
   return total;
