@@ -3,7 +3,7 @@
 // The decode step streams every retained weight exactly once, so the kernel is built around keeping
 // HBM busy: one persistent block per SM whose producer warp keeps a ring of shared-memory stages
 // filled by the tensor memory accelerator (cp.async.bulk.tensor boxes of 128 bytes x 64 rows,
-// completion on an mbarrier), far ahead of the sixteen consumer warps, and whose two epilogue warps
+// completion on an mbarrier), far ahead of the sixteen consumer warps, and whose epilogue warps
 // finish tiles (reduction over the consumer warps, bias, rotary embedding, store) behind them.  No
 // role spends registers or issue slots on another role's latency.  On-device pruning (Section 3.4) is expressed in the tensor maps:
 // a family of kept channel blocks {start, period, keep, count} is a 3-D tensor (byte in row, row in
@@ -43,7 +43,7 @@ namespace {
 
 constexpr int CW = 16;                  // consumer warps
 constexpr int CTH = CW * 32;            // consumer threads
-constexpr int EW = 2;                   // epilogue warps
+constexpr int EW = 4;                   // epilogue warps
 constexpr int ETH = EW * 32;
 constexpr int NTH = CTH + 32 + ETH;     // consumers + one producer warp + epilogue warps
 constexpr int RB = 64;                  // row slots per tile
@@ -492,9 +492,10 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           float* tile_ws = c.partials + (size_t)tile * c.max_slots * RM;
           float* mine = tile_ws + (size_t)my_slot * RM;
           for (int j = etid; j < RM; j += ETH) __stcg(mine + j, local_sum(j & (RB - 1), j / RB));
-          __threadfence();
           if (!epi_sync()) return;
           if (etid == 0) {
+            __threadfence();                           // orders the whole group's parked sums (observed through
+                                                       // the barrier) before the arrival count
             const int arrived = atomicAdd(&c.counters[tile], 1);
             *last_flag = arrived == total - 1;
             __threadfence();
@@ -905,8 +906,8 @@ size_t plan_split(DecodeCfg* c, int M, int g_total, int gran) {
     }
     c->gp = gp;
   } else {
-    for (int s = want; s >= 3 && !fits; --s)
-      for (n_kp = 1; n_kp <= kMaxKParts && !fits; ++n_kp) {
+    for (n_kp = 1; n_kp <= kMaxKParts && !fits; ++n_kp)
+      for (int s = want; s >= 3 && !fits; --s) {
         const int gp = round_up((g_total + n_kp - 1) / n_kp, gran);
         smem = plan_smem(c, M, MT, gp, s, part_bufs);
         fits = smem <= (size_t)kSmemMax;
