@@ -98,6 +98,10 @@ int dispatch(const Params& p, void* workspace, size_t ws_bytes, void* stream) {
   }
   if (path == UNIQL_PATH_PREFILL) {
     if (!prefill_supported(p)) return UNIQL_ERR_UNSUPPORTED;
+    if (!cfg.workspace) {      // only the status word of the workspace is used
+      int rc = lib_workspace(&cfg.workspace, &cfg.ws_bytes, cfg.stream);
+      if (rc != UNIQL_OK) return rc;
+    }
     return launch_prefill(p, cfg);
   }
   return launch_generic(p, cfg);

@@ -1,6 +1,532 @@
-// Prefill kernel (M >= 64): placeholder until the tcgen05 path lands.
+// Prefill kernel (M >= 64 tokens) of the pruned 4-bit linear layer, sm_100a: a dense contraction on
+// the fifth-generation tensor cores (tcgen05.mma, accumulators in tensor memory).
+//
+// Orientation.  The packed weights are four times smaller than the activations, so the weight side
+// takes the MMA's M dimension (128 retained weight rows per tile, de-quantised once per tile and
+// k-block) and the tokens its N dimension (up to 256 per tile): D[row][token] += W[row][k] x[token][k].
+//
+// Roles inside a block (one persistent block per SM, tiles taken round-robin):
+//   warp 0       TMA producer: one box [64 k x BN tokens] of activations per stage (128-byte swizzle)
+//   warp 1       allocates tensor memory; one lane issues the MMAs of a stage (4 x K=16) and commits
+//                them to the stage's "empty" barrier and, at the end of a tile, to "accumulator full"
+//   warps 4..7   epilogue: tcgen05.ld the fp32 accumulators (warp w owns TMEM lanes 32(w-4)..),
+//                transpose through shared memory, bias, rotary embedding on the retained pair
+//                (Section 3.2), one rounding, coalesced stores; two accumulator buffers of 256 columns
+//                let the epilogue of tile i overlap the MMAs of tile i+1
+//   warps 8..15  de-quantisers: thread (row, half) converts 32 codes of its weight row per k-block --
+//                nibbles to fp16 by magic number, (q-8) exact, then s*(q-8) + s*(8-z) in fp32, one
+//                rounding to fp16 -- and writes them into the A-operand stage in the
+//                canonical K-major 128-byte-swizzled layout; the packed codes of the next two k-blocks
+//                are already in registers
+// On-device pruning (Section 3.4) is index arithmetic: tile rows are compact output channels mapped to
+// stored rows per thread; the input side is the leading k_in channels (the TMA tensor ends at k_in, so
+// the tail of the last k-block is zero activations).
+// bf16 activations: bf16 weights would carry 2^-9 relative rounding error each, which alone spends the
+// 2e-3 error budget; instead the de-quantisers convert the activation tile to fp16 in place (exact in
+// fp16's range, saturating beyond) and both operands are fp16.
+//
+// Every mbarrier wait is bounded; on expiry the block raises a flag, every role leaves its loop, the
+// status word of the workspace is set, tensor memory is released and the block returns.
+#include <cuda.h>
+#include <string.h>
+
+#include <mutex>
+#include <type_traits>
+
 #include "common.cuh"
+
 namespace uniql {
-int prefill_supported(const Params&) { return 0; }
-int launch_prefill(const Params&, const LaunchCfg&) { return UNIQL_ERR_UNSUPPORTED; }
+namespace {
+
+constexpr int BMW = 128;            // weight rows per tile (MMA M)
+constexpr int BK = 64;              // k per stage: 128 bytes of fp16 / bf16, one swizzle row
+constexpr int MAXBN = 256;          // tokens per tile (MMA N), at most
+constexpr int PSTAGES = 4;
+constexpr int A_BYTES = BMW * BK * 2;        // 16 KB
+constexpr int B_BYTES = MAXBN * BK * 2;      // 32 KB
+constexpr int PSTAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int EPI_TOK = 32;                  // tokens per epilogue pass
+constexpr int STG_BYTES = EPI_TOK * BMW * 4; // fp32 staging [token][row]
+constexpr int NWARPS = 16;
+constexpr int PTH = NWARPS * 32;
+constexpr int DQ_WARP0 = 8, DQ_WARPS = 8;
+constexpr int EPI_WARP0 = 4;
+constexpr int kPWait = 1 << 20;
+constexpr int kMaxPJobs = kMaxJobs;
+
+struct PrefillCfg {
+  CUtensorMap xmap;          // activations: (k, token), box 64 x BN, 128-byte swizzle
+  int bn;                    // tokens per tile: 64, 128 or 256
+  int n_ttiles;              // token tiles
+  int wtile_begin[kMaxPJobs + 1];   // first weight tile of each job
+  int n_tiles;               // weight tiles (all jobs) x token tiles
+  int n_kb;                  // k-blocks of 64 (k_in rounded up)
+  uint32_t idesc;
+  int* status;
+};
+
+// ---------------------------------------------------------------------------------------- PTX
+__device__ inline void pmbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ inline void pmbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ inline void pmbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ inline bool pmbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ inline bool pmbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (int i = 0; i < kPWait; ++i) {
+    if (pmbar_try(bar, parity)) return true;
+    if ((i & 63) == 63 && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ inline void tma_box2(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ inline void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ inline void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ inline void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ inline void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ inline void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// D[tmem] (+)= A[smem desc] * B[smem desc]; accumulate == 0 overwrites D
+__device__ inline void umma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives on `bar` when all MMAs issued so far by this thread have completed
+__device__ inline void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ inline void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ inline void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ inline void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 fp16/bf16), 128-byte
+// swizzle: 8-row groups 1024 bytes apart (stride byte offset), leading byte offset unused (1),
+// descriptor version 1 (sm_100), layout type 2 (SWIZZLE_128B).
+__device__ inline uint64_t smem_desc_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+__device__ inline uint32_t pand_or(uint32_t a, uint32_t mask, uint32_t magic) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(mask), "r"(magic));
+  return d;
+}
+
+// ---------------------------------------------------------------------------------------- tile rows
+// Row r (0..127) of local weight tile `tl` of a job: stored weight row, or -1 when the row is empty.
+// Rope jobs: rows 0..63 are the first-half members of 64 rotation pairs, rows 64..127 their partners.
+struct RowInfo { int stored; int out_col; int pair_c; int head; };
+__device__ inline RowInfo tile_row(const JobDev& jb, int tl, int r) {
+  RowInfo o;
+  o.stored = -1; o.out_col = -1; o.pair_c = 0; o.head = 0;
+  if (jb.rope.enabled) {
+    const int half = jb.rope.head_keep >> 1;
+    const int P = tl * (BMW / 2) + (r & (BMW / 2 - 1));
+    if (P >= jb.rope.n_heads * half) return o;
+    const int h = P / half, cc = P - h * half, hi = r >> 6;
+    o.stored = h * jb.rope.head_dim + hi * (jb.rope.head_dim >> 1) + cc;
+    o.out_col = h * jb.rope.head_keep + hi * half + cc;
+    o.pair_c = cc; o.head = h;
+  } else {
+    const int j = tl * BMW + r;
+    if (j >= jb.k_out) return o;
+    o.stored = (jb.omap.n_fam == 1 && jb.omap.fam[0].count == 1) ? jb.omap.fam[0].start + j
+                                                                  : map_compact_to_stored(jb.omap, j);
+    o.out_col = j;
+  }
+  return o;
+}
+__device__ inline int job_tiles_p(const JobDev& j) {
+  if (j.rope.enabled) return (j.rope.n_heads * (j.rope.head_keep / 2) + BMW / 2 - 1) / (BMW / 2);
+  return (j.k_out + BMW - 1) / BMW;
+}
+
+// Two bf16 values of a word as two fp16 values (exact for magnitudes in fp16's normal range, which
+// holds LLM activations; larger magnitudes saturate at +-65504 instead of becoming infinite).
+__device__ inline uint32_t bf16x2_to_f16x2(uint32_t w) {
+  uint32_t d;
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(__uint_as_float(w & 0xffff0000u)), "f"(__uint_as_float(w << 16)));
+  return d;
+}
+
+// Eight codes of one 32-bit word, in input-channel order, as eight fp16 values packed in a uint4:
+// byte b -> (1024 + c_even, 64 + c_odd) as an fp16 pair (one PRMT, one LOP3), minus (1032, 72) = the
+// exact (c-8) pair, then s*(c-8) + s*(8-z) in fp32 and one rounding.
+__device__ inline uint4 dequant_word(uint32_t w, float s, float cz) {
+  uint32_t o[4];
+#pragma unroll
+  for (int b = 0; b < 4; ++b) {
+    const uint32_t t = __byte_perm(w, 0u, 0x4040u + 0x0101u * b);
+    const uint32_t v = pand_or(t, 0x00f0000fu, 0x54006400u);
+    const __half2 h2 = __hsub2(*reinterpret_cast<const __half2*>(&v), __halves2half2(__ushort_as_half(0x6408), __ushort_as_half(0x5480)));
+    const float2 f = __half22float2(h2);
+    const float w0 = fmaf(f.x, s, cz), w1 = fmaf(f.y, s, cz);
+    const __half2 r = __floats2half2_rn(w0, w1);
+    o[b] = *reinterpret_cast<const uint32_t*>(&r);
+  }
+  return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// ---------------------------------------------------------------------------------------- kernel
+template <typename T>
+__global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__ Params p,
+                                                         const __grid_constant__ PrefillCfg c) {
+  extern __shared__ unsigned char psmem_raw[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t raw = (uint32_t)__cvta_generic_to_shared(psmem_raw);
+  const uint32_t sbase = (raw + 1023u) & ~1023u;           // swizzled tiles need 1024-byte alignment
+  unsigned char* smem = psmem_raw + (sbase - raw);
+  const uint32_t stg = sbase + PSTAGES * PSTAGE_BYTES;     // fp32 staging [32 tokens][128 rows]
+  float* stg_p = reinterpret_cast<float*>(smem + PSTAGES * PSTAGE_BYTES);
+  const uint32_t bars = stg + STG_BYTES;
+  const uint32_t full_a = bars, full_b = bars + 8 * PSTAGES, empty = bars + 16 * PSTAGES;
+  const uint32_t acc_full = bars + 24 * PSTAGES, acc_empty = acc_full + 16, epi_bar = acc_full + 32;
+  unsigned char* misc = smem + PSTAGES * PSTAGE_BYTES + STG_BYTES + 24 * PSTAGES + 40;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
+
+  if (tid == 0) {
+    for (int s = 0; s < PSTAGES; ++s) {
+      pmbar_init(full_a + 8 * s, DQ_WARPS);
+      pmbar_init(full_b + 8 * s, 1);
+      pmbar_init(empty + 8 * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) { pmbar_init(acc_full + 8 * b, 1); pmbar_init(acc_empty + 8 * b, 4); }
+    pmbar_init(epi_bar, 4);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {                      // the whole tensor memory of the SM: two accumulators of 256 columns
+    tmem_alloc((uint32_t)__cvta_generic_to_shared(const_cast<uint32_t*>(tmem_slot)), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int n_wtiles = c.wtile_begin[p.n_jobs];
+  auto job_of_wt = [&](int wt) { int j = 0; while (j + 1 < p.n_jobs && wt >= c.wtile_begin[j + 1]) ++j; return j; };
+  bool failed = false;
+
+  if (warp == 0) {
+    // ===================================================================== activations by TMA
+    if (lane == 0) {
+      int s = 0; uint32_t par = 1; int it = 0;
+      for (int t = blockIdx.x; t < c.n_tiles && !failed; t += gridDim.x) {
+        const int tt = t % c.n_ttiles;
+        for (int kb = 0; kb < c.n_kb; ++kb, ++it) {
+          if (it >= PSTAGES && !pmbar_wait(empty + 8 * s, par, abort_flag)) { failed = true; break; }
+          const uint32_t fb = full_b + 8 * s;
+          pmbar_expect_tx(fb, (uint32_t)(c.bn * BK * 2));
+          tma_box2(sbase + s * PSTAGE_BYTES + A_BYTES, &c.xmap, kb * BK, tt * c.bn, fb);
+          if (++s == PSTAGES) { s = 0; par ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ===================================================================== MMA issue
+    if (lane == 0) {
+      int s = 0; uint32_t par = 0; int tcount = 0;
+      for (int t = blockIdx.x; t < c.n_tiles && !failed; t += gridDim.x, ++tcount) {
+        const int buf = tcount & 1;
+        if (tcount >= 2 && !pmbar_wait(acc_empty + 8 * buf, ((tcount >> 1) - 1) & 1, abort_flag)) { failed = true; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MAXBN);
+        for (int kb = 0; kb < c.n_kb; ++kb) {
+          // (bf16: the de-quantisers waited for the activation tile themselves and converted it)
+          if (!pmbar_wait(full_a + 8 * s, par, abort_flag) ||
+              (!std::is_same<T, __nv_bfloat16>::value && !pmbar_wait(full_b + 8 * s, par, abort_flag))) { failed = true; break; }
+          tc_fence_after();
+          const uint64_t adesc = smem_desc_sw128(sbase + s * PSTAGE_BYTES);
+          const uint64_t bdesc = smem_desc_sw128(sbase + s * PSTAGE_BYTES + A_BYTES);
+#pragma unroll
+          for (int k16 = 0; k16 < BK / 16; ++k16)       // 32 bytes along K per MMA: +2 in the address field
+            umma_f16(d_tmem, adesc + 2 * k16, bdesc + 2 * k16, c.idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+          umma_commit(empty + 8 * s);                   // the stage is free once these MMAs have read it
+          if (++s == PSTAGES) { s = 0; par ^= 1; }
+        }
+        if (failed) break;
+        umma_commit(acc_full + 8 * buf);
+      }
+    }
+  } else if (warp >= DQ_WARP0) {
+    // ===================================================================== de-quantisers
+    const int dt = tid - DQ_WARP0 * 32;
+    const int r = dt >> 1, hf = dt & 1;
+    const int G = p.K / kGroup;
+    int s = 0; uint32_t par = 1; int it = 0;
+    for (int t = blockIdx.x; t < c.n_tiles && !failed; t += gridDim.x) {
+      const int wt = t / c.n_ttiles;
+      const int jn = job_of_wt(wt);
+      const JobDev& jb = p.job[jn];
+      const RowInfo ri = tile_row(jb, wt - c.wtile_begin[jn], r);
+      const bool live = ri.stored >= 0;
+      const uint8_t* wrow = jb.w + (size_t)(live ? ri.stored : 0) * (p.K / 2) + hf * 16;
+      const __half* srow = jb.scales + (size_t)(live ? ri.stored : 0) * G;
+      const __half* zrow = jb.zeros + (size_t)(live ? ri.stored : 0) * G;
+      // codes and scale / zero-point of the next two k-blocks are kept in registers
+      uint4 q0 = make_uint4(0, 0, 0, 0), q1 = q0;
+      float s0 = 0.f, z0 = 0.f, s1 = 0.f, z1 = 0.f;
+      if (live) {
+        q0 = __ldg(reinterpret_cast<const uint4*>(wrow));
+        s0 = __half2float(__ldg(srow)); z0 = __half2float(__ldg(zrow));
+        if (c.n_kb > 1) {
+          q1 = __ldg(reinterpret_cast<const uint4*>(wrow + 32));
+          s1 = __half2float(__ldg(srow + 0)); z1 = __half2float(__ldg(zrow + 0));
+        }
+      }
+      const uint32_t row_off = (uint32_t)(r * 128);
+      for (int kb = 0; kb < c.n_kb; ++kb, ++it) {
+        uint4 q2 = make_uint4(0, 0, 0, 0);
+        float s2 = 0.f, z2 = 0.f;
+        if (live && kb + 2 < c.n_kb) {
+          q2 = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)(kb + 2) * 32));
+          s2 = __half2float(__ldg(srow + ((kb + 2) >> 1))); z2 = __half2float(__ldg(zrow + ((kb + 2) >> 1)));
+        }
+        if (it >= PSTAGES && !pmbar_wait(empty + 8 * s, par, abort_flag)) { failed = true; break; }
+        const uint32_t a_st = sbase + s * PSTAGE_BYTES + row_off;
+        const float cz = (8.f - z0) * s0;
+        const uint32_t qw[4] = {q0.x, q0.y, q0.z, q0.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint4 o = live ? dequant_word(qw[j], s0, cz) : make_uint4(0, 0, 0, 0);
+          const uint32_t a = a_st + (uint32_t)((((hf * 4 + j) ^ (r & 7))) * 16);
+          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w) : "memory");
+        }
+        if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+          // bf16 activations: the tensor cores run on fp16 (8 more mantissa bits for the weights than bf16
+          // would leave them); the activation tile that TMA delivered is converted in place
+          if (!pmbar_wait(full_b + 8 * s, par ^ 1, abort_flag)) { failed = true; break; }
+          const uint32_t b_st = sbase + s * PSTAGE_BYTES + A_BYTES;
+          for (int ci = dt; ci < c.bn * 8; ci += DQ_WARPS * 32) {
+            uint32_t v0, v1, v2, v3;
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(b_st + ci * 16));
+            v0 = bf16x2_to_f16x2(v0); v1 = bf16x2_to_f16x2(v1); v2 = bf16x2_to_f16x2(v2); v3 = bf16x2_to_f16x2(v3);
+            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(b_st + ci * 16), "r"(v0), "r"(v1), "r"(v2), "r"(v3) : "memory");
+          }
+        }
+        fence_async_smem();            // generic-proxy writes must be visible to the tensor core (async proxy)
+        __syncwarp();
+        if (lane == 0) pmbar_arrive(full_a + 8 * s);
+        q0 = q1; s0 = s1; z0 = z1;
+        q1 = q2; s1 = s2; z1 = z2;
+        if (++s == PSTAGES) { s = 0; par ^= 1; }
+      }
+    }
+  } else if (warp >= EPI_WARP0) {
+    // ===================================================================== epilogue
+    const int q = warp - EPI_WARP0;                 // TMEM lanes 32q .. 32q+31
+    const int etid = tid - EPI_WARP0 * 32;          // 0..127 = tile row handled in the store phase
+    uint32_t epar = 0;
+    auto epi_sync = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) pmbar_arrive(epi_bar);
+      const bool ok = pmbar_wait(epi_bar, epar, abort_flag);
+      epar ^= 1;
+      return ok;
+    };
+    int tcount = 0;
+    for (int t = blockIdx.x; t < c.n_tiles && !failed; t += gridDim.x, ++tcount) {
+      const int buf = tcount & 1;
+      const int wt = t / c.n_ttiles, tt = t - wt * c.n_ttiles;
+      const int jn = job_of_wt(wt);
+      const JobDev& jb = p.job[jn];
+      const int tl = wt - c.wtile_begin[jn];
+      T* y = reinterpret_cast<T*>(jb.y);
+      const T* bias = reinterpret_cast<const T*>(jb.bias);
+      const bool rope = jb.rope.enabled != 0;
+      // store phase: non-rope: this thread owns tile row etid; rope: pair (etid & 63), tokens of parity etid >> 6
+      const RowInfo ri = tile_row(jb, tl, rope ? (etid & 63) : etid);
+      float b_lo = 0.f, b_hi = 0.f;
+      double invf = 0.0;
+      if (ri.stored >= 0) {
+        if (bias) {
+          b_lo = DT<T>::to_f(bias[ri.stored]);
+          if (rope) b_hi = DT<T>::to_f(bias[ri.stored + (jb.rope.head_dim >> 1)]);
+        }
+        if (rope) {
+          const int half = jb.rope.head_keep >> 1;
+          int pidx = p.idx[(ri.head / jb.rope.rep) * half + ri.pair_c];
+          pidx = min(max(pidx, 0), (jb.rope.head_dim >> 1) - 1);
+          invf = p.inv_freq[pidx];
+        }
+      }
+      if (!pmbar_wait(acc_full + 8 * buf, (tcount >> 1) & 1, abort_flag)) { failed = true; break; }
+      tc_fence_after();
+      for (int ch = 0; ch < c.bn / EPI_TOK && !failed; ++ch) {
+        uint32_t v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * MAXBN + ch * EPI_TOK), v);
+        tmem_ld_wait();
+        // staging[token][row]: lanes are consecutive rows
+#pragma unroll
+        for (int k = 0; k < 32; ++k) stg_p[k * BMW + 32 * q + lane] = __uint_as_float(v[k]);
+        if (!epi_sync()) { failed = true; break; }
+        const int m0 = tt * c.bn + ch * EPI_TOK;
+        if (ri.stored >= 0) {
+          if (rope) {
+            const int half = jb.rope.head_keep >> 1;
+            for (int k = etid >> 6; k < EPI_TOK; k += 2) {
+              const int m = m0 + k;
+              if (m >= p.M) break;
+              const float lo = stg_p[k * BMW + (etid & 63)] + b_lo, hi = stg_p[k * BMW + 64 + (etid & 63)] + b_hi;
+              float cs, sn;
+              rope_cos_sin(p.pos[m], invf, cs, sn);
+              y[(size_t)m * jb.ldy + ri.out_col] = DT<T>::from_f(lo * cs - hi * sn);
+              y[(size_t)m * jb.ldy + ri.out_col + half] = DT<T>::from_f(hi * cs + lo * sn);
+            }
+          } else {
+            for (int k = 0; k < EPI_TOK; ++k) {
+              const int m = m0 + k;
+              if (m >= p.M) break;
+              y[(size_t)m * jb.ldy + ri.out_col] = DT<T>::from_f(stg_p[k * BMW + etid] + b_lo);
+            }
+          }
+        }
+        if (!epi_sync()) { failed = true; break; }       // staging is rewritten by the next pass
+      }
+      if (failed) break;
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) pmbar_arrive(acc_empty + 8 * buf);
+    }
+  }
+
+  if (failed && lane == 0) atomicExch(c.status, UNIQL_ERR_TIMEOUT);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, 512);
+}
+
+// -------------------------------------------------------------------------------- host side
+typedef CUresult (*PEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+PEncodeFn p_encoder() {
+  static PEncodeFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qr) == cudaSuccess &&
+        qr == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<PEncodeFn>(ptr);
+    else
+      cudaGetLastError();
+  });
+  return fn;
+}
+
+int p_sm_count() {
+  int dev = 0, v = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess &&
+      cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+    return v;
+  return 148;
+}
+
+int host_job_tiles(const JobDev& j) {
+  if (j.rope.enabled) return (j.rope.n_heads * (j.rope.head_keep / 2) + BMW / 2 - 1) / (BMW / 2);
+  return (j.k_out + BMW - 1) / BMW;
+}
+
+template <typename T>
+int launch_pt(const Params& p, const PrefillCfg& c, int grid, cudaStream_t stream) {
+  const size_t smem = 1024 + (size_t)PSTAGES * PSTAGE_BYTES + STG_BYTES + 512;
+  auto kern = prefill_kernel<T>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return UNIQL_ERR_CUDA;
+  kern<<<grid, PTH, smem, stream>>>(p, c);
+  return cudaGetLastError() == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
+}
+
+}  // namespace
+
+// The tensor-core path takes: the leading k_in input channels (the hidden dimension D_h is never pruned,
+// D_int is pruned as a leading block: Section 3.4), any output map, both activation types.
+int prefill_supported(const Params& p) {
+  if (p.M < 17) return 0;
+  if (p.dt != UNIQL_F16 && p.dt != UNIQL_BF16) return 0;
+  if (p.imap.n_fam != 1 || p.imap.fam[0].count != 1 || p.imap.fam[0].start != 0) return 0;
+  if ((p.ldx % 8) != 0 || (((uintptr_t)p.x) & 15) != 0) return 0;       // TMA: 16-byte base and row pitch
+  if ((p.K % kGroup) != 0) return 0;
+  return 1;
+}
+
+int launch_prefill(const Params& p, const LaunchCfg& cfg) {
+  PEncodeFn enc = p_encoder();
+  if (!enc) return UNIQL_ERR_CUDA;
+  if (!cfg.workspace) return UNIQL_ERR_WORKSPACE;
+  PrefillCfg c;
+  memset(&c, 0, sizeof(c));
+  c.bn = p.M <= 64 ? 64 : (p.M <= 128 ? 128 : 256);
+  c.n_ttiles = (p.M + c.bn - 1) / c.bn;
+  int wt = 0;
+  for (int j = 0; j < p.n_jobs; ++j) { c.wtile_begin[j] = wt; wt += host_job_tiles(p.job[j]); }
+  for (int j = p.n_jobs; j <= kMaxPJobs; ++j) c.wtile_begin[j] = wt;
+  c.n_tiles = wt * c.n_ttiles;
+  if (c.n_tiles < 1) return UNIQL_ERR_SHAPE;
+  c.n_kb = (p.k_in + BK - 1) / BK;
+  const uint32_t fmt = 0u;      // both operands fp16 (bf16 activations are converted in shared memory)
+  // instruction descriptor: fp32 accumulate, A and B of the activation type, both K-major, N = bn, M = 128
+  c.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(c.bn >> 3) << 17) | ((uint32_t)(BMW >> 4) << 24);
+  c.status = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(cfg.workspace) + decode_status_offset());
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)p.k_in, (cuuint64_t)p.M};
+    const cuuint64_t strides[1] = {(cuuint64_t)p.ldx * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)c.bn};
+    const cuuint32_t es[2] = {1, 1};
+    const CUresult r = enc(&c.xmap, p.dt == UNIQL_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16,
+                           2, const_cast<void*>(p.x), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return UNIQL_ERR_CUDA;
+  }
+  const int sms = p_sm_count();
+  const int grid = c.n_tiles < sms ? c.n_tiles : sms;
+  return p.dt == UNIQL_BF16 ? launch_pt<__nv_bfloat16>(p, c, grid, cfg.stream) : launch_pt<__half>(p, c, grid, cfg.stream);
+}
+
 }  // namespace uniql
