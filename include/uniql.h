@@ -120,6 +120,10 @@ int uniql_dequant(const uint8_t* packed, const void* scales, const void* zeros, 
  * must be 256-byte aligned, at least uniql_workspace_bytes() large, and prepared once by
  * uniql_workspace_init (zeroes the counters; they return to zero after every call).
  * Calls that share a workspace must not overlap on the device. */
+/* For M > 16 (tensor-core path) the workspace only carries the status word and, for bf16 activations,
+ * an fp16 copy of x (M x K x 2 bytes): the tensor cores run on fp16 operands, because weights rounded
+ * to bf16 would alone spend the 2e-3 error budget; bf16 magnitudes beyond 65504 saturate.  When the
+ * workspace is too small for the copy the tiles are converted inside the kernel (same result, slower). */
 size_t uniql_workspace_bytes(int M, int K, int N_total);
 int uniql_workspace_init(void* workspace, size_t bytes, void* stream);
 /* Every wait inside the kernels is bounded.  When one expires the kernel stops early and writes

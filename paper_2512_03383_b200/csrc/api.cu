@@ -134,7 +134,7 @@ extern "C" int uniql_set_path(int path) {
 
 extern "C" size_t uniql_workspace_bytes(int M, int K, int N_total) {
   if (M < 1 || K < 1 || N_total < 1) return 0;
-  return decode_workspace_bytes(M, K, N_total);
+  return M <= 16 ? decode_workspace_bytes(M, K, N_total) : prefill_workspace_bytes(M, K);
 }
 
 extern "C" int uniql_workspace_init(void* workspace, size_t bytes, void* stream) {

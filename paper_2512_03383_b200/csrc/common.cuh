@@ -142,5 +142,6 @@ int decode_status_offset();   // byte offset of the device status word inside a 
 size_t decode_workspace_header_bytes();   // counters + status word: the part that must start at zero
 int launch_prefill(const Params& p, const LaunchCfg& cfg);
 int prefill_supported(const Params& p);
+size_t prefill_workspace_bytes(int M, int K);
 
 }  // namespace uniql

@@ -28,6 +28,7 @@
 // Every mbarrier wait is bounded; on expiry the block raises a flag, every role leaves its loop, the
 // status word of the workspace is set, tensor memory is released and the block returns.
 #include <cuda.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <mutex>
@@ -208,7 +209,36 @@ __device__ inline uint4 dequant_word(uint32_t w, float s, float cz) {
 }
 
 // ---------------------------------------------------------------------------------------- kernel
-template <typename T>
+// bf16 activations -> fp16 copy in the workspace, once per call (every weight tile re-reads the tile of
+// activations, so converting there would repeat the work once per 128 weight rows).
+__global__ void x_to_f16_kernel(const __nv_bfloat16* __restrict__ x, int ldx, int M, int k_in, __half* __restrict__ o, int ldo) {
+  const int units = ldo / 8;                         // 16-byte units per output row (ldo is a multiple of 8)
+  const long total = (long)M * units;
+  for (long i = (long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
+    const int m = (int)(i / units), u = (int)(i - (long)m * units);
+    const __nv_bfloat16* src = x + (size_t)m * ldx + u * 8;
+    uint32_t w[4];
+    if (u * 8 + 8 <= k_in && ((ldx & 7) == 0) && ((((uintptr_t)x) & 15) == 0)) {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(src));
+      w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int k0 = u * 8 + 2 * e;
+        const uint32_t lo = k0 < k_in ? __bfloat16_as_ushort(src[2 * e]) : 0u;
+        const uint32_t hi = k0 + 1 < k_in ? __bfloat16_as_ushort(src[2 * e + 1]) : 0u;
+        w[e] = lo | (hi << 16);
+      }
+    }
+    uint4 r;
+    r.x = bf16x2_to_f16x2(w[0]); r.y = bf16x2_to_f16x2(w[1]); r.z = bf16x2_to_f16x2(w[2]); r.w = bf16x2_to_f16x2(w[3]);
+    *reinterpret_cast<uint4*>(o + (size_t)m * ldo + u * 8) = r;
+  }
+}
+
+// T: activation / output type.  CONV: the activation tiles arrive as bf16 and are converted to fp16 in
+// shared memory by the de-quantisers (used when the workspace cannot hold a converted copy).
+template <typename T, bool CONV>
 __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__ Params p,
                                                          const __grid_constant__ PrefillCfg c) {
   extern __shared__ unsigned char psmem_raw[];
@@ -276,7 +306,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         for (int kb = 0; kb < c.n_kb; ++kb) {
           // (bf16: the de-quantisers waited for the activation tile themselves and converted it)
           if (!pmbar_wait(full_a + 8 * s, par, abort_flag) ||
-              (!std::is_same<T, __nv_bfloat16>::value && !pmbar_wait(full_b + 8 * s, par, abort_flag))) { failed = true; break; }
+              (!CONV && !pmbar_wait(full_b + 8 * s, par, abort_flag))) { failed = true; break; }
           tc_fence_after();
           const uint64_t adesc = smem_desc_sw128(sbase + s * PSTAGE_BYTES);
           const uint64_t bdesc = smem_desc_sw128(sbase + s * PSTAGE_BYTES + A_BYTES);
@@ -334,7 +364,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
           const uint32_t a = a_st + (uint32_t)((((hf * 4 + j) ^ (r & 7))) * 16);
           asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w) : "memory");
         }
-        if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+        if constexpr (CONV) {
           // bf16 activations: the tensor cores run on fp16 (8 more mantissa bits for the weights than bf16
           // would leave them); the activation tile that TMA delivered is converted in place
           if (!pmbar_wait(full_b + 8 * s, par ^ 1, abort_flag)) { failed = true; break; }
@@ -472,10 +502,10 @@ int host_job_tiles(const JobDev& j) {
   return (j.k_out + BMW - 1) / BMW;
 }
 
-template <typename T>
+template <typename T, bool CONV>
 int launch_pt(const Params& p, const PrefillCfg& c, int grid, cudaStream_t stream) {
   const size_t smem = 1024 + (size_t)PSTAGES * PSTAGE_BYTES + STG_BYTES + 512;
-  auto kern = prefill_kernel<T>;
+  auto kern = prefill_kernel<T, CONV>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return UNIQL_ERR_CUDA;
   kern<<<grid, PTH, smem, stream>>>(p, c);
@@ -513,20 +543,50 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   // instruction descriptor: fp32 accumulate, A and B of the activation type, both K-major, N = bn, M = 128
   c.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(c.bn >> 3) << 17) | ((uint32_t)(BMW >> 4) << 24);
   c.status = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(cfg.workspace) + decode_status_offset());
+  // bf16 activations: fp16 copy in the workspace when it fits (else converted tile by tile in the kernel)
+  const void* xsrc = p.x;
+  int ldxs = p.ldx;
+  bool conv_in_kernel = false;
+  if (p.dt == UNIQL_BF16) {
+    const int ldo = (p.k_in + 7) / 8 * 8;
+    const size_t off = (decode_workspace_header_bytes() + 255) & ~(size_t)255;
+    const size_t need = off + (size_t)p.M * ldo * 2;
+    const char* force = getenv("UNIQL_PREFILL_CONVERT");
+    if (cfg.ws_bytes >= need && !(force && force[0] == 'k')) {
+      __half* x16 = reinterpret_cast<__half*>(reinterpret_cast<unsigned char*>(cfg.workspace) + off);
+      const long units = (long)p.M * (ldo / 8);
+      long blocks = (units + 255) / 256;
+      if (blocks > 148 * 8) blocks = 148 * 8;
+      x_to_f16_kernel<<<(int)blocks, 256, 0, cfg.stream>>>(reinterpret_cast<const __nv_bfloat16*>(p.x), p.ldx, p.M, p.k_in, x16, ldo);
+      if (cudaGetLastError() != cudaSuccess) return UNIQL_ERR_CUDA;
+      xsrc = x16;
+      ldxs = ldo;
+    } else {
+      conv_in_kernel = true;
+    }
+  }
   {
     const cuuint64_t dims[2] = {(cuuint64_t)p.k_in, (cuuint64_t)p.M};
-    const cuuint64_t strides[1] = {(cuuint64_t)p.ldx * 2};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldxs * 2};
     const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)c.bn};
     const cuuint32_t es[2] = {1, 1};
-    const CUresult r = enc(&c.xmap, p.dt == UNIQL_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16,
-                           2, const_cast<void*>(p.x), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    const CUresult r = enc(&c.xmap, conv_in_kernel ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16,
+                           2, const_cast<void*>(xsrc), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return UNIQL_ERR_CUDA;
   }
   const int sms = p_sm_count();
   const int grid = c.n_tiles < sms ? c.n_tiles : sms;
-  return p.dt == UNIQL_BF16 ? launch_pt<__nv_bfloat16>(p, c, grid, cfg.stream) : launch_pt<__half>(p, c, grid, cfg.stream);
+  if (p.dt == UNIQL_BF16)
+    return conv_in_kernel ? launch_pt<__nv_bfloat16, true>(p, c, grid, cfg.stream)
+                          : launch_pt<__nv_bfloat16, false>(p, c, grid, cfg.stream);
+  return launch_pt<__half, false>(p, c, grid, cfg.stream);
+}
+
+size_t prefill_workspace_bytes(int M, int K) {
+  // status word (shared header) + room for the fp16 copy of bf16 activations
+  return ((decode_workspace_header_bytes() + 255) & ~(size_t)255) + (size_t)M * ((K + 7) / 8 * 8) * 2;
 }
 
 }  // namespace uniql

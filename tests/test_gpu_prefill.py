@@ -89,6 +89,21 @@ def test_prefill_qk_rope(B, M, keep, dtype):
         check_output(g, ref, dtype, TOL[dtype], "prefill rope keep %d M=%d %s" % (keep, M, dtype))
 
 
+def test_prefill_bf16_converted_in_kernel(B, monkeypatch):
+    """The fallback for workspaces too small for an fp16 copy of the activations: tiles are converted in
+    shared memory.  Same result as the copy-first path, bit for bit."""
+    B.set_path(B.PATH_PREFILL)
+    rng = np.random.default_rng(650)
+    qw = synth.draw_qweight(rng, 300, 768)
+    dw = dev_weight(qw)
+    x = synth.draw_x(rng, 300, 652, "bf16")
+    y1, ref = run_ex(B, qw, dw, x, "bf16", None, 652, None, 256, ldx_pad=4)
+    monkeypatch.setenv("UNIQL_PREFILL_CONVERT", "kernel")
+    y2, _ = run_ex(B, qw, dw, x, "bf16", None, 652, None, 256, ldx_pad=4)
+    check_output(y2, ref, "bf16", TOL["bf16"], "bf16 converted in kernel")
+    assert torch.equal(y1, y2)
+
+
 def test_prefill_multi_job(B):
     rng = np.random.default_rng(800)
     gate, up = synth.draw_qweight(rng, 352, 512), synth.draw_qweight(rng, 352, 512)
