@@ -375,18 +375,90 @@ def run_ours(args):
         line["cpu_baseline"] = oracle_leg(3.0)
         if args.detail:
             line["detail"] = detail_tables(B, torch, max(20, min(args.steps, 200)))
+            line["detail"].update(prefill_tables(B, torch))
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
     return 0
 
 
+QWEN_HIDDEN, QWEN_INTER = 3584, 18944
+
+
+class QwenPrefill:
+    """Qwen2.5-7B-shaped gate (output rows pruned) and down (input columns pruned) projections, bf16."""
+
+    def __init__(self, B, torch, M, seed=0):
+        from paper_2512_03383_b200 import synth
+        self.B, self.torch, self.M = B, torch, M
+        rng = np.random.default_rng(seed)
+        self.w = {}
+        for name, N, K in (("gate", QWEN_INTER, QWEN_HIDDEN), ("down", QWEN_HIDDEN, QWEN_INTER)):
+            m = synth.random_qweight_fast(rng, N, K)
+            cd = torch.from_numpy(m.codes).cuda()
+            packed = torch.empty((N, K // 2), dtype=torch.uint8, device="cuda")
+            B.pack_u4(cd, packed)
+            self.w[name] = (packed, torch.from_numpy(m.scales).cuda(), torch.from_numpy(m.zeros).cuda(), N, K)
+            del cd
+        self.x = torch.randn((M, QWEN_HIDDEN), device="cuda").to(torch.bfloat16)
+        self.h = torch.randn((M, QWEN_INTER), device="cuda").to(torch.bfloat16)
+        self.yg = torch.zeros((M, QWEN_INTER), dtype=torch.bfloat16, device="cuda")
+        self.yd = torch.zeros((M, QWEN_HIDDEN), dtype=torch.bfloat16, device="cuda")
+
+    def gate(self, rate):
+        k = keep_count(rate, QWEN_INTER)
+        pw, s, z, N, K = self.w["gate"]
+        self.B.qlinear_ex(self.x, QWEN_HIDDEN, pw, s, z, None, self.M, K, N, None, K, None, k, self.yg, QWEN_INTER)
+        return 2.0 * self.M * K * k
+
+    def down(self, rate):
+        k = keep_count(rate, QWEN_INTER)
+        pw, s, z, N, K = self.w["down"]
+        self.B.qlinear_ex(self.h, QWEN_INTER, pw, s, z, None, self.M, K, N, None, k, None, N, self.yd, QWEN_HIDDEN)
+        return 2.0 * self.M * k * N
+
+
+def prefill_tables(B, torch):
+    """Tensor-core path: TFLOP/s of Qwen2.5-7B gate / down at M = 512, 2048 per keep rate (bf16)."""
+    hbm, tf, which = measured_peaks()
+    out = {}
+    for M in (512, 2048):
+        q = QwenPrefill(B, torch, M)
+        for name, fn in (("gate", q.gate), ("down", q.down)):
+            rows = {}
+            for r in (1.0, 0.85, 0.65):
+                for _ in range(3):
+                    flops = fn(r)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                a.record()
+                for _ in range(10):
+                    fn(r)
+                b.record()
+                torch.cuda.synchronize()
+                sec = a.elapsed_time(b) * 1e-3 / 10
+                rows["%.2f" % r] = {"us": round(sec * 1e6, 1), "TFLOPs": round(flops / sec / 1e12, 1),
+                                    "frac_bf16_%s" % which: round(flops / sec / 1e12 / tf, 3),
+                                    "tokens_per_s": round(M / sec, 1)}
+            out["prefill_qwen_%s_M%d" % (name, M)] = rows
+        del q
+        torch.cuda.empty_cache()
+    return out
+
+
 def run_case(args):
     """A few plain (un-graphed) launches of one kernel on a small set-up, for ncu captures:
-    --case decode-gateup | decode-down, with --M and --keep."""
+    --case decode-gateup | decode-down | prefill-gate | prefill-down, with --M and --keep."""
     import torch
     from paper_2512_03383_b200 import binding as B
     torch.cuda.set_device(0)
+    if args.case.startswith("prefill"):
+        q = QwenPrefill(B, torch, args.M)
+        for _ in range(args.launches):
+            (q.gate if args.case == "prefill-gate" else q.down)(args.keep)
+        torch.cuda.synchronize()
+        print("case %s M=%d keep=%.2f: %d launches done" % (args.case, args.M, args.keep, args.launches))
+        return 0
     w = MlpDecode(B, torch, args.M)
     k = keep_count(args.keep, INTER)
     for _ in range(args.launches):

@@ -14,8 +14,8 @@
 //                (Section 3.2), one rounding, coalesced stores; two accumulator buffers of 256 columns
 //                let the epilogue of tile i overlap the MMAs of tile i+1
 //   warps 8..15  de-quantisers: thread (row, half) converts 32 codes of its weight row per k-block --
-//                nibbles to fp16 by magic number, (q-8) exact, then s*(q-8) + s*(8-z) in fp32, one
-//                rounding to fp16 -- and writes them into the A-operand stage in the
+//                nibbles to fp16 by magic number, (q-8) exact, then one fp16 FMA (q-8)*s + fp16(s*(8-z))
+//                -- and writes them into the A-operand stage in the
 //                canonical K-major 128-byte-swizzled layout; the packed codes of the next two k-blocks
 //                are already in registers
 // On-device pruning (Section 3.4) is index arithmetic: tile rows are compact output channels mapped to
@@ -192,23 +192,22 @@ __device__ inline uint32_t bf16x2_to_f16x2(uint32_t w) {
 
 // Eight codes of one 32-bit word, in input-channel order, as eight fp16 values packed in a uint4:
 // byte b -> (1024 + c_even, 64 + c_odd) as an fp16 pair (one PRMT, one LOP3), minus (1032, 72) = the
-// exact (c-8) pair, then s*(c-8) + s*(8-z) in fp32 and one rounding.
-__device__ inline uint4 dequant_word(uint32_t w, float s, float cz) {
+// exact (c-8) pair, then one fp16 FMA per pair: (c-8)*s + cz with cz = fp16(s*(8-z)).  s is the stored
+// fp16 scale itself, (c-8)*s + cz is rounded once; the only other error is the rounding of cz (2^-12
+// of at most 8 s, shared by the 128 weights of a group).
+__device__ inline uint4 dequant_word(uint32_t w, __half2 s2, __half2 cz2) {
   uint32_t o[4];
+  const __half2 off = __halves2half2(__ushort_as_half(0x6408), __ushort_as_half(0x5480));
 #pragma unroll
   for (int b = 0; b < 4; ++b) {
     const uint32_t t = __byte_perm(w, 0u, 0x4040u + 0x0101u * b);
     const uint32_t v = pand_or(t, 0x00f0000fu, 0x54006400u);
-    const __half2 h2 = __hsub2(*reinterpret_cast<const __half2*>(&v), __halves2half2(__ushort_as_half(0x6408), __ushort_as_half(0x5480)));
-    const float2 f = __half22float2(h2);
-    const float w0 = fmaf(f.x, s, cz), w1 = fmaf(f.y, s, cz);
-    const __half2 r = __floats2half2_rn(w0, w1);
+    const __half2 r = __hfma2(__hsub2(*reinterpret_cast<const __half2*>(&v), off), s2, cz2);
     o[b] = *reinterpret_cast<const uint32_t*>(&r);
   }
   return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
-// ---------------------------------------------------------------------------------------- kernel
 // bf16 activations -> fp16 copy in the workspace, once per call (every weight tile re-reads the tile of
 // activations, so converting there would repeat the work once per 128 weight rows).
 __global__ void x_to_f16_kernel(const __nv_bfloat16* __restrict__ x, int ldx, int M, int k_in, __half* __restrict__ o, int ldo) {
@@ -337,30 +336,31 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
       const __half* zrow = jb.zeros + (size_t)(live ? ri.stored : 0) * G;
       // codes and scale / zero-point of the next two k-blocks are kept in registers
       uint4 q0 = make_uint4(0, 0, 0, 0), q1 = q0;
-      float s0 = 0.f, z0 = 0.f, s1 = 0.f, z1 = 0.f;
+      __half s0 = __ushort_as_half(0), z0 = s0, s1 = s0, z1 = s0;
       if (live) {
         q0 = __ldg(reinterpret_cast<const uint4*>(wrow));
-        s0 = __half2float(__ldg(srow)); z0 = __half2float(__ldg(zrow));
+        s0 = __ldg(srow); z0 = __ldg(zrow);
         if (c.n_kb > 1) {
           q1 = __ldg(reinterpret_cast<const uint4*>(wrow + 32));
-          s1 = __half2float(__ldg(srow + 0)); z1 = __half2float(__ldg(zrow + 0));
+          s1 = s0; z1 = z0;
         }
       }
       const uint32_t row_off = (uint32_t)(r * 128);
       for (int kb = 0; kb < c.n_kb; ++kb, ++it) {
         uint4 q2 = make_uint4(0, 0, 0, 0);
-        float s2 = 0.f, z2 = 0.f;
+        __half s2 = s1, z2 = z1;
         if (live && kb + 2 < c.n_kb) {
           q2 = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)(kb + 2) * 32));
-          s2 = __half2float(__ldg(srow + ((kb + 2) >> 1))); z2 = __half2float(__ldg(zrow + ((kb + 2) >> 1)));
+          s2 = __ldg(srow + ((kb + 2) >> 1)); z2 = __ldg(zrow + ((kb + 2) >> 1));
         }
         if (it >= PSTAGES && !pmbar_wait(empty + 8 * s, par, abort_flag)) { failed = true; break; }
         const uint32_t a_st = sbase + s * PSTAGE_BYTES + row_off;
-        const float cz = (8.f - z0) * s0;
+        const __half2 sh2 = __half2half2(s0);
+        const __half2 cz2 = __float2half2_rn((8.f - __half2float(z0)) * __half2float(s0));
         const uint32_t qw[4] = {q0.x, q0.y, q0.z, q0.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const uint4 o = live ? dequant_word(qw[j], s0, cz) : make_uint4(0, 0, 0, 0);
+          const uint4 o = live ? dequant_word(qw[j], sh2, cz2) : make_uint4(0, 0, 0, 0);
           const uint32_t a = a_st + (uint32_t)((((hf * 4 + j) ^ (r & 7))) * 16);
           asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w) : "memory");
         }
