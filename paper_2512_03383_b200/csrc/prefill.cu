@@ -13,7 +13,7 @@
 //                transpose through shared memory, bias, rotary embedding on the retained pair
 //                (Section 3.2), one rounding, coalesced stores; two accumulator buffers of 256 columns
 //                let the epilogue of tile i overlap the MMAs of tile i+1
-//   warps 8..15  de-quantisers: thread (row, half) converts 32 codes of its weight row per k-block --
+//   warps 8..23  de-quantisers (two teams of eight warps on alternate stages): thread (row, half) converts 32 codes of its weight row per k-block --
 //                nibbles to fp16 by magic number, (q-8) exact, then one fp16 FMA (q-8)*s + fp16(s*(8-z))
 //                -- and writes them into the A-operand stage in the
 //                canonical K-major 128-byte-swizzled layout; the packed codes of the next two k-blocks
@@ -48,9 +48,9 @@ constexpr int B_BYTES = MAXBN * BK * 2;      // 32 KB
 constexpr int PSTAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int EPI_TOK = 32;                  // tokens per epilogue pass
 constexpr int STG_BYTES = EPI_TOK * BMW * 4; // fp32 staging [token][row]
-constexpr int NWARPS = 16;
+constexpr int NWARPS = 24;
 constexpr int PTH = NWARPS * 32;
-constexpr int DQ_WARP0 = 8, DQ_WARPS = 8;
+constexpr int DQ_WARP0 = 8, DQ_WARPS = 8;      // two teams of DQ_WARPS warps: even and odd stages
 constexpr int EPI_WARP0 = 4;
 constexpr int kPWait = 1 << 20;
 constexpr int kMaxPJobs = kMaxJobs;
@@ -85,9 +85,11 @@ __device__ inline bool pmbar_try(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-__device__ inline bool pmbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// `relaxed`: sleep between polls (roles that run several stages ahead and must not steal issue slots)
+__device__ inline bool pmbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool relaxed = false) {
   for (int i = 0; i < kPWait; ++i) {
     if (pmbar_try(bar, parity)) return true;
+    if (relaxed) __nanosleep(200);
     if ((i & 63) == 63 && *abort_flag) return false;
   }
   *abort_flag = 1;
@@ -285,7 +287,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
       for (int t = blockIdx.x; t < c.n_tiles && !failed; t += gridDim.x) {
         const int tt = t % c.n_ttiles;
         for (int kb = 0; kb < c.n_kb; ++kb, ++it) {
-          if (it >= PSTAGES && !pmbar_wait(empty + 8 * s, par, abort_flag)) { failed = true; break; }
+          if (it >= PSTAGES && !pmbar_wait(empty + 8 * s, par, abort_flag, true)) { failed = true; break; }
           const uint32_t fb = full_b + 8 * s;
           pmbar_expect_tx(fb, (uint32_t)(c.bn * BK * 2));
           tma_box2(sbase + s * PSTAGE_BYTES + A_BYTES, &c.xmap, kb * BK, tt * c.bn, fb);
@@ -321,11 +323,18 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
     }
   } else if (warp >= DQ_WARP0) {
     // ===================================================================== de-quantisers
-    const int dt = tid - DQ_WARP0 * 32;
+    // Two teams of eight warps take alternate stages, so that each warp has two stage periods for the
+    // conversion of one stage and the schedulers always find a ready warp.
+    const int team = (warp - DQ_WARP0) / DQ_WARPS;
+    const int dt = tid - (DQ_WARP0 + team * DQ_WARPS) * 32;
     const int r = dt >> 1, hf = dt & 1;
     const int G = p.K / kGroup;
-    int s = 0; uint32_t par = 1; int it = 0;
-    for (int t = blockIdx.x; t < c.n_tiles && !failed; t += gridDim.x) {
+    const uint32_t row_off = (uint32_t)(r * 128);
+    uint32_t col_off[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) col_off[j] = (uint32_t)(((hf * 4 + j) ^ (r & 7)) * 16);
+    int it0 = 0;                       // stage iterations before this tile
+    for (int t = blockIdx.x; t < c.n_tiles && !failed; t += gridDim.x, it0 += c.n_kb) {
       const int wt = t / c.n_ttiles;
       const int jn = job_of_wt(wt);
       const JobDev& jb = p.job[jn];
@@ -334,26 +343,31 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
       const uint8_t* wrow = jb.w + (size_t)(live ? ri.stored : 0) * (p.K / 2) + hf * 16;
       const __half* srow = jb.scales + (size_t)(live ? ri.stored : 0) * G;
       const __half* zrow = jb.zeros + (size_t)(live ? ri.stored : 0) * G;
-      // codes and scale / zero-point of the next two k-blocks are kept in registers
+      const int kb0 = ((it0 & 1) == team) ? 0 : 1;
+      // codes and scale / zero-point of this team's next two k-blocks are kept in registers
       uint4 q0 = make_uint4(0, 0, 0, 0), q1 = q0;
       __half s0 = __ushort_as_half(0), z0 = s0, s1 = s0, z1 = s0;
       if (live) {
-        q0 = __ldg(reinterpret_cast<const uint4*>(wrow));
-        s0 = __ldg(srow); z0 = __ldg(zrow);
-        if (c.n_kb > 1) {
-          q1 = __ldg(reinterpret_cast<const uint4*>(wrow + 32));
-          s1 = s0; z1 = z0;
+        if (kb0 < c.n_kb) {
+          q0 = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)kb0 * 32));
+          s0 = __ldg(srow + (kb0 >> 1)); z0 = __ldg(zrow + (kb0 >> 1));
+        }
+        if (kb0 + 2 < c.n_kb) {
+          q1 = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)(kb0 + 2) * 32));
+          s1 = __ldg(srow + ((kb0 + 2) >> 1)); z1 = __ldg(zrow + ((kb0 + 2) >> 1));
         }
       }
-      const uint32_t row_off = (uint32_t)(r * 128);
-      for (int kb = 0; kb < c.n_kb; ++kb, ++it) {
+      for (int kb = kb0; kb < c.n_kb; kb += 2) {
+        const int it = it0 + kb;
+        const int s = it & (PSTAGES - 1);
+        const uint32_t use = (uint32_t)(it / PSTAGES);
         uint4 q2 = make_uint4(0, 0, 0, 0);
         __half s2 = s1, z2 = z1;
-        if (live && kb + 2 < c.n_kb) {
-          q2 = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)(kb + 2) * 32));
-          s2 = __ldg(srow + ((kb + 2) >> 1)); z2 = __ldg(zrow + ((kb + 2) >> 1));
+        if (live && kb + 4 < c.n_kb) {
+          q2 = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)(kb + 4) * 32));
+          s2 = __ldg(srow + ((kb + 4) >> 1)); z2 = __ldg(zrow + ((kb + 4) >> 1));
         }
-        if (it >= PSTAGES && !pmbar_wait(empty + 8 * s, par, abort_flag)) { failed = true; break; }
+        if (it >= PSTAGES && !pmbar_wait(empty + 8 * s, (use - 1) & 1, abort_flag)) { failed = true; break; }
         const uint32_t a_st = sbase + s * PSTAGE_BYTES + row_off;
         const __half2 sh2 = __half2half2(s0);
         const __half2 cz2 = __float2half2_rn((8.f - __half2float(z0)) * __half2float(s0));
@@ -361,13 +375,12 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const uint4 o = live ? dequant_word(qw[j], sh2, cz2) : make_uint4(0, 0, 0, 0);
-          const uint32_t a = a_st + (uint32_t)((((hf * 4 + j) ^ (r & 7))) * 16);
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w) : "memory");
+          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a_st + col_off[j]), "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w) : "memory");
         }
         if constexpr (CONV) {
           // bf16 activations: the tensor cores run on fp16 (8 more mantissa bits for the weights than bf16
           // would leave them); the activation tile that TMA delivered is converted in place
-          if (!pmbar_wait(full_b + 8 * s, par ^ 1, abort_flag)) { failed = true; break; }
+          if (!pmbar_wait(full_b + 8 * s, use & 1, abort_flag)) { failed = true; break; }
           const uint32_t b_st = sbase + s * PSTAGE_BYTES + A_BYTES;
           for (int ci = dt; ci < c.bn * 8; ci += DQ_WARPS * 32) {
             uint32_t v0, v1, v2, v3;
@@ -381,7 +394,6 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         if (lane == 0) pmbar_arrive(full_a + 8 * s);
         q0 = q1; s0 = s1; z0 = z1;
         q1 = q2; s1 = s2; z1 = z2;
-        if (++s == PSTAGES) { s = 0; par ^= 1; }
       }
     }
   } else if (warp >= EPI_WARP0) {
