@@ -254,8 +254,8 @@ __device__ inline void store_tile(const Params& p, const TileFam& f, const TileP
 }
 
 // ---------------------------------------------------------------------------------------- work split
-// Units of one block of k-part `kp`: first `base` whole tiles (all chunks), then a contiguous range of
-// the chunk-fastest unit sequence of the R tiles that are left over after every block took its share.
+// Units of one block of k-part `kp`: `base` whole tiles (all chunks) and a contiguous range of the
+// chunk-fastest unit sequence of the R tiles that are left over after every block took its share.
 struct Work {
   int Ck;            // chunks per tile in this k-part
   int n1;            // units of the whole-tile phase (base * Ck)
@@ -279,21 +279,27 @@ __device__ inline Work block_work(const DecodeCfg& c, int Ck, int rp) {
   w.n_units = w.n1 + (w.te - w.tb);
   return w;
 }
-// (tile, chunk) of block-local unit i, walked in order
+// (tile, chunk) of block-local unit i, walked in order.  The share of the left-over tiles comes first:
+// its hand-over between blocks (parked sums, arrival count, final reduction by the last block) then
+// overlaps the streaming of the whole tiles instead of trailing the kernel.
 struct UnitIter {
   int tile, chunk;
   __device__ inline void start(const Work& w) {
-    if (w.n1 > 0) { tile = w.tile1; chunk = 0; }
-    else { tile = w.tail_tile0 + w.tb / w.Ck; chunk = w.tb - (w.tb / w.Ck) * w.Ck; }
+    if (w.te > w.tb) { tile = w.tail_tile0 + w.tb / w.Ck; chunk = w.tb - (w.tb / w.Ck) * w.Ck; }
+    else { tile = w.tile1; chunk = 0; }
   }
   // returns true when the position jumped (phase switch), i.e. the tile position must be recomputed
   __device__ inline bool advance(const Work& w, int i_next) {
-    if (i_next == w.n1 && w.n1 > 0) {
-      tile = w.tail_tile0 + w.tb / w.Ck; chunk = w.tb - (w.tb / w.Ck) * w.Ck;
+    if (i_next == w.te - w.tb && w.te > w.tb) {
+      tile = w.tile1; chunk = 0;
       return true;
     }
     if (++chunk == w.Ck) { chunk = 0; ++tile; }
     return false;
+  }
+  // unit i is the block's last unit of its tile
+  __device__ inline bool tile_end(const Work& w, int i) const {
+    return chunk == w.Ck - 1 || i == w.n_units - 1 || i == w.te - w.tb - 1;
   }
 };
 
@@ -449,7 +455,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     TilePos q = tile_pos(c, p, ui.tile);
     int tiles_done = 0;
     for (int i = 0; i < wk.n_units; ++i) {
-      const bool tile_end = (ui.chunk == wk.Ck - 1) || (i == wk.n_units - 1);
+      const bool tile_end = ui.tile_end(wk, i);
       if (tile_end) {
         const int buf = c.part_bufs > 1 ? (tiles_done & 1) : 0;
         const int use = c.part_bufs > 1 ? (tiles_done >> 1) : tiles_done;
@@ -729,7 +735,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     if (lane == 0) mbar_arrive(bar_empty + 8 * s);
     if (++s == S) { s = 0; ring_parity ^= 1; }
 
-    const bool tile_end = (ui.chunk == wk.Ck - 1) || (i == wk.n_units - 1);
+    const bool tile_end = ui.tile_end(wk, i);
     if (tile_end) {
       // ---- park this warp's partial sums for the epilogue warps: part[buf][group slot kpw][m][row slot]
       const int buf = c.part_bufs > 1 ? (tiles_done & 1) : 0;
