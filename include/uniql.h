@@ -21,6 +21,13 @@
  *    host before anything is launched; nothing aborts or throws.
  *  - There is no CPU fallback: without a usable CUDA device calls return
  *    UNIQL_ERR_CUDA.
+ *  - Decode launches (M <= 16) carry the programmatic-stream-serialization attribute: back-to-back
+ *    decode calls on one stream overlap their launch set-up and weight prefetch with the tail of the
+ *    preceding one, while everything that can depend on the preceding kernel (activations, outputs,
+ *    workspace, bias, positions, indices) is touched only after it has completed.  Packed weights,
+ *    scales and zero-points must not be written by a decode call's immediate predecessor on the stream
+ *    unless that predecessor is a plain kernel (which completes before its successor starts).
+ *    UNIQL_PDL=0 in the environment turns the attribute off.
  *
  * Weight format (the interchange format; benchmark configuration 1)
  *  - W is stored in nn.Linear orientation, W[N][K]: N output channels (rows),

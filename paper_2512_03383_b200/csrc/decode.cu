@@ -342,6 +342,9 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   const int sg_lo = c.v_first + v_lo;                           // first stored group of this k-part
   const int G = p.K / kGroup;
   const Work wk = block_work(c, (Gk + CG - 1) / CG, rp);
+  // Programmatic dependent launch: the next kernel of the stream may be set up while this one runs (its
+  // blocks still need this block's resources, so they start as blocks here exit) ...
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (wk.n_units == 0) return;
 
   // ======================================================================================= producer
@@ -454,6 +457,10 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     ui.start(wk);
     TilePos q = tile_pos(c, p, ui.tile);
     int tiles_done = 0;
+    // ... and this kernel may have been started before its predecessor finished: outputs, workspace, bias,
+    // positions and indices are touched only after the predecessor is complete (the producer warp does not
+    // wait: weights, scales and zero-points are not produced by a preceding decode launch)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int i = 0; i < wk.n_units; ++i) {
       const bool tile_end = ui.tile_end(wk, i);
       if (tile_end) {
@@ -552,6 +559,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   // ---- stage activations: permuted into nibble order, zero where the channel is pruned; per group and
   //      batch row the two sums the offset / zero-point correction needs, stored negated
   {
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // the activations may come from the preceding kernel
     const T* x = reinterpret_cast<const T*>(p.x);
     const int row_units = c.xrow / 16;
     uint4* xs = reinterpret_cast<uint4*>(smem + c.off_x);
@@ -874,8 +882,19 @@ int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stre
   auto kern = decode_kernel<MT, ONECOL>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return UNIQL_ERR_CUDA;
-  kern<<<c.n_kp * c.n_rp, NTH, smem, stream>>>(p, c);
-  return cudaGetLastError() == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
+  cudaLaunchConfig_t lc;
+  memset(&lc, 0, sizeof(lc));
+  lc.gridDim = dim3(c.n_kp * c.n_rp);
+  lc.blockDim = dim3(NTH);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr;
+  lc.numAttrs = env_int("UNIQL_PDL", 1) ? 1 : 0;
+  if (cudaLaunchKernelEx(&lc, kern, p, c) != cudaSuccess) { cudaGetLastError(); return UNIQL_ERR_CUDA; }
+  return UNIQL_OK;
 }
 
 // Visited groups of the input map: from the first to the last 128-channel group that holds a retained
