@@ -290,6 +290,20 @@ def detail_tables(B, torch, steps):
     return out
 
 
+def max_over_ranks(dist, torch, values, device):
+    """Replicas share nothing on the data path; the job's time is the slowest rank's (weak scaling)."""
+    if dist is None:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_value(bytes_per_rank_step, steps, world, sec):
+    """Aggregate metric over all replicas: bytes every rank processed, divided by the slowest rank's time."""
+    return bytes_per_rank_step * steps * world / sec / 1e9
+
+
 def run_ours(args):
     import torch
     rank = int(os.environ.get("RANK", "0"))
@@ -334,10 +348,7 @@ def run_ours(args):
     t_end = time.time()
     clocks = sampler.stop(t_load, t_end) if rank == 0 else None
 
-    if dist is not None:
-        t = torch.tensor([sec, sec_e2e], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        sec, sec_e2e = float(t[0]), float(t[1])
+    sec, sec_e2e = max_over_ranks(dist, torch, [sec, sec_e2e], "cuda")
 
     if rank != 0:
         if dist is not None:
@@ -345,8 +356,7 @@ def run_ours(args):
         return 0
 
     hbm, tf, which = measured_peaks()
-    total_bytes = step_bytes() * args.steps * world
-    value = total_bytes / sec / 1e9
+    value = whole_job_value(step_bytes(), args.steps, world, sec)
     launches = work.launches_per_step * args.steps
     per_launch_bytes = step_bytes() / work.launches_per_step
     per_launch_sec = sec / launches
@@ -367,7 +377,7 @@ def run_ours(args):
                      "traffic": None if DRAM_TRAFFIC_RATIO is None else DRAM_TRAFFIC_RATIO * per_launch_bytes, "peak_source": which,
                      "kernel": "decode_kernel<half,1>", "algorithmic_bytes_per_launch": per_launch_bytes,
                      "frac_of_nominal_8TBs": achieved / 8000.0},
-        "e2e": {"value": step_bytes() * args.steps * world / sec_e2e / 1e9, "unit": "GB/s",
+        "e2e": {"value": whole_job_value(step_bytes(), args.steps, world, sec_e2e), "unit": "GB/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "note": "activations copied from / results to pinned host memory every launch; weights resident"},
     }
