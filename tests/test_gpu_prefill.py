@@ -120,3 +120,96 @@ def test_prefill_multi_job(B):
     for (q, d, y) in ((gate, dg, yg), (up, du, yu)):
         ref = oracle.qlinear(x, d[0], q.scales, q.zeros, oracle.leading(k), oracle.leading(512))
         check_output(y, ref, "bf16", TOL["bf16"], "multi")
+
+
+# ---------------------------------------------------------------- full benchmark sizes, sampled token rows
+def _sampled_rows(M):
+    rows = sorted(set([0, 1, 31, 32, 63, 64, 127, 128, 255, 256, M // 2, M - 2, M - 1]))
+    return [r for r in rows if 0 <= r < M]
+
+
+@pytest.mark.parametrize("M", [512, 2048])
+def test_qwen_gate_down_full_size_sampled(B, M):
+    """Configuration 4 (Qwen2.5-7B-shaped MLP in prefill, bf16) in the launch configuration of the bench:
+    sampled token rows of the full output against the oracle."""
+    rng = np.random.default_rng(4)
+    gate = synth.random_qweight_fast(rng, 18944, 3584)
+    dg = dev_weight(gate)
+    for rate in (1.0, 0.65):
+        k = synth.keep_count(rate, 18944)
+        x = synth.draw_x(rng, M, 3584, "bf16")
+        xd = dev_x(x, "bf16")
+        y = torch.zeros((M, k), dtype=torch.bfloat16, device="cuda")
+        B.qlinear_ex(xd, 3584, dg[1], dg[2], dg[3], None, M, 3584, 18944, None, 3584, None, k, y, k)
+        torch.cuda.synchronize()
+        rows = _sampled_rows(M)
+        ref = oracle.qlinear(x, dg[0], gate.scales, gate.zeros, oracle.leading(k), oracle.leading(3584), rows=rows)
+        check_output(y[rows], ref, "bf16", TOL["bf16"], "qwen gate keep %.2f M=%d" % (rate, M))
+    del dg
+    down = synth.random_qweight_fast(rng, 3584, 18944)
+    dd = dev_weight(down)
+    for rate in (1.0, 0.65):
+        k = synth.keep_count(rate, 18944)
+        h = synth.draw_x(rng, M, k, "bf16")
+        hd = dev_x(h, "bf16")
+        y = torch.zeros((M, 3584), dtype=torch.bfloat16, device="cuda")
+        B.qlinear_ex(hd, k, dd[1], dd[2], dd[3], None, M, 18944, 3584, None, k, None, 3584, y, 3584)
+        torch.cuda.synchronize()
+        rows = _sampled_rows(M)[::2]
+        ref = oracle.qlinear(h, dd[0], down.scales, down.zeros, oracle.leading(3584), oracle.leading(k), rows=rows)
+        check_output(y[rows], ref, "bf16", TOL["bf16"], "qwen down keep %.2f M=%d" % (rate, M))
+    assert B.workspace_status() == 0
+
+
+def test_qwen_qk_rope_full_size_sampled(B):
+    """Configuration 4's attention projections with the fused pruned RoPE at M = 512 (theta 1e6, 28 Q / 4 KV heads)."""
+    rng = np.random.default_rng(44)
+    M, K, Hq, Hkv, D, theta = 512, 3584, 28, 4, 128, 1e6
+    wq, wk = synth.random_qweight_fast(rng, Hq * D, K), synth.random_qweight_fast(rng, Hkv * D, K)
+    dq, dk = dev_weight(wq), dev_weight(wk)
+    x = synth.draw_x(rng, M, K, "bf16")
+    xd = dev_x(x, "bf16")
+    pos = synth.draw_pos(rng, M)
+    rows = _sampled_rows(M)
+    for keep in (128, 84):
+        idx = synth.draw_idx(rng, Hkv, D, keep)
+        qo = torch.zeros((M, Hq * keep), dtype=torch.bfloat16, device="cuda")
+        ko = torch.zeros((M, Hkv * keep), dtype=torch.bfloat16, device="cuda")
+        B.qk_rope_proj(xd, K, dq[1], dq[2], dq[3], dk[1], dk[2], dk[3], None, None, M, K, Hq, Hkv, D, keep,
+                       torch.from_numpy(idx).cuda(), torch.from_numpy(pos).cuda(), theta, None, qo, Hq * keep, ko,
+                       Hkv * keep)
+        torch.cuda.synchronize()
+        for (w, d, nh, g) in ((wq, dq, Hq, qo), (wk, dk, Hkv, ko)):
+            O = oracle.expand_map(oracle.qk_halfhead_map(nh, D, keep))
+            acc = oracle.qlinear(x, d[0], w.scales, w.zeros, O, oracle.leading(K), rows=rows)
+            ref = oracle.rope(acc, nh, Hkv, D, keep, idx, pos[rows], theta)
+            check_output(g[rows], ref, "bf16", TOL["bf16"], "qwen q/k rope keep %d" % keep)
+
+
+@pytest.mark.parametrize("M", [1, 1024])
+def test_mamba2_full_size(B, M):
+    """Configuration 5: Mamba2-2.7B in_proj [10576 x 2560] (z, x rows pruned per SSM head) and out_proj
+    [2560 x 5120] (columns pruned per head), fp16; decode at M = 1, prefill / generic at M = 1024 (sampled rows)."""
+    rng = np.random.default_rng(5)
+    nheads, headdim, d_state, d_inner = 80, 64, 128, 5120
+    qin = synth.random_qweight_fast(rng, 10576, 2560)
+    qout = synth.random_qweight_fast(rng, 2560, d_inner)
+    din, dout = dev_weight(qin), dev_weight(qout)
+    rows = _sampled_rows(M)
+    for keep in (64, 48):
+        om = synth.map_mamba_in_proj(d_inner, headdim, keep, d_state, 1, nheads)
+        n_out = synth.map_size(om)
+        x = synth.draw_x(rng, M, 2560, "f16")
+        y = torch.zeros((M, n_out), dtype=torch.float16, device="cuda")
+        B.qlinear_ex(dev_x(x, "f16"), 2560, din[1], din[2], din[3], None, M, 2560, 10576, None, 2560, om, 0, y, n_out)
+        torch.cuda.synchronize()
+        ref = oracle.qlinear(x, din[0], qin.scales, qin.zeros, oracle.expand_map(om), oracle.leading(2560), rows=rows)
+        check_output(y[rows], ref, "f16", TOL["f16"], "mamba in_proj keep %d M=%d" % (keep, M))
+        im = synth.map_per_head(nheads, headdim, keep)
+        n_in = synth.map_size(im)
+        h = synth.draw_x(rng, M, n_in, "f16")
+        y2 = torch.zeros((M, 2560), dtype=torch.float16, device="cuda")
+        B.qlinear_ex(dev_x(h, "f16"), n_in, dout[1], dout[2], dout[3], None, M, d_inner, 2560, im, 0, None, 2560, y2, 2560)
+        torch.cuda.synchronize()
+        ref2 = oracle.qlinear(h, dout[0], qout.scales, qout.zeros, oracle.leading(2560), oracle.expand_map(im), rows=rows)
+        check_output(y2[rows], ref2, "f16", TOL["f16"], "mamba out_proj keep %d M=%d" % (keep, M))
