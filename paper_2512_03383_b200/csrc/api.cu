@@ -15,7 +15,7 @@ namespace {
 int g_path = UNIQL_PATH_AUTO;
 
 constexpr int kMaxDevices = 64;
-constexpr size_t kLibWorkspaceBytes = (size_t)96 << 20;
+constexpr size_t kLibWorkspaceBytes = (size_t)192 << 20;
 void* g_ws[kMaxDevices] = {nullptr};
 std::mutex g_ws_mutex;
 

@@ -63,8 +63,55 @@ struct PrefillCfg {
   int n_tiles;               // weight tiles (all jobs) x token tiles
   int n_kb;                  // k-blocks of 64 (k_in rounded up)
   uint32_t idesc;
+  int streamk;               // 1: contiguous ranges of (tile, k-block) units per block; 0: whole tiles round-robin
   int* status;
+  int* counters;             // stream-K: arrivals per tile
+  float* partials;           // stream-K: two slots of [bn tokens][128 rows] fp32 per block
 };
+
+// Work of a block as a sequence of segments (tile, k-blocks [kb0, kb1)): whole tiles t = b, b + grid, ...
+// With stream-K only for as many rounds as fill every block; the k-blocks of the tiles left over are then
+// cut into equal contiguous ranges, one per block, so that the last round keeps every SM busy however few
+// tiles remain.  Blocks stay in step along k (few distinct k offsets are alive at a time, which keeps the
+// activation slices in L2).  A left-over tile is finished by the last of its blocks to arrive (fp32 partial
+// tiles in the workspace, added in block order).
+struct Seg { int tile, kb0, kb1, tail_idx; };     // tail_idx: -1 whole-tile round, else index among the block's tail segments
+struct SegIter {
+  long u, ue;
+  int t, t_end, n_kb, step, tail_tile0, n_tail_seg;
+  __device__ inline void init(const PrefillCfg& c, int b, int grid) {
+    n_kb = c.n_kb; step = grid; t = b; n_tail_seg = 0;
+    const int base = c.streamk ? c.n_tiles / grid : (c.n_tiles + grid - 1) / grid;
+    t_end = c.streamk ? base * grid : c.n_tiles;
+    tail_tile0 = base * grid;
+    u = ue = 0;
+    if (c.streamk) {
+      const long Ut = (long)(c.n_tiles - tail_tile0) * c.n_kb;
+      const long Bt = grid < Ut ? grid : Ut;
+      if (b < Bt) { u = Ut * b / Bt; ue = Ut * (b + 1) / Bt; }
+    }
+  }
+  __device__ inline bool next(Seg& sg) {
+    if (t < t_end) {
+      sg.tile = t; sg.kb0 = 0; sg.kb1 = n_kb; sg.tail_idx = -1;
+      t += step;
+      return true;
+    }
+    if (u >= ue) return false;
+    const int tt = (int)(u / n_kb);
+    sg.tile = tail_tile0 + tt;
+    sg.kb0 = (int)(u - (long)tt * n_kb);
+    const long len = (n_kb - sg.kb0) < (ue - u) ? (n_kb - sg.kb0) : (ue - u);
+    sg.kb1 = sg.kb0 + (int)len;
+    sg.tail_idx = n_tail_seg++;
+    u += len;
+    return true;
+  }
+};
+// block whose range [U*b/B, U*(b+1)/B) of the left-over units holds unit u (exact in fp64 for these magnitudes)
+__device__ inline int sk_owner(long u, long B, long U) {
+  return (int)floor(((double)(u + 1) * (double)B - 1.0) / (double)U);
+}
 
 // ---------------------------------------------------------------------------------------- PTX
 __device__ inline void pmbar_init(uint32_t bar, uint32_t count) {
@@ -284,9 +331,11 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
     // ===================================================================== activations by TMA
     if (lane == 0) {
       int s = 0; uint32_t par = 1; int it = 0;
-      for (int t = blockIdx.x; t < c.n_tiles && !failed; t += gridDim.x) {
-        const int tt = t % c.n_ttiles;
-        for (int kb = 0; kb < c.n_kb; ++kb, ++it) {
+      SegIter si; si.init(c, blockIdx.x, gridDim.x);
+      Seg sg;
+      while (!failed && si.next(sg)) {
+        const int tt = sg.tile % c.n_ttiles;
+        for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
           if (it >= PSTAGES && !pmbar_wait(empty + 8 * s, par, abort_flag, true)) { failed = true; break; }
           const uint32_t fb = full_b + 8 * s;
           pmbar_expect_tx(fb, (uint32_t)(c.bn * BK * 2));
@@ -299,12 +348,14 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
     // ===================================================================== MMA issue
     if (lane == 0) {
       int s = 0; uint32_t par = 0; int tcount = 0;
-      for (int t = blockIdx.x; t < c.n_tiles && !failed; t += gridDim.x, ++tcount) {
+      SegIter si; si.init(c, blockIdx.x, gridDim.x);
+      Seg sg;
+      for (; !failed && si.next(sg); ++tcount) {
         const int buf = tcount & 1;
         if (tcount >= 2 && !pmbar_wait(acc_empty + 8 * buf, ((tcount >> 1) - 1) & 1, abort_flag)) { failed = true; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MAXBN);
-        for (int kb = 0; kb < c.n_kb; ++kb) {
+        for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
           // (bf16: the de-quantisers waited for the activation tile themselves and converted it)
           if (!pmbar_wait(full_a + 8 * s, par, abort_flag) ||
               (!CONV && !pmbar_wait(full_b + 8 * s, par, abort_flag))) { failed = true; break; }
@@ -313,7 +364,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
           const uint64_t bdesc = smem_desc_sw128(sbase + s * PSTAGE_BYTES + A_BYTES);
 #pragma unroll
           for (int k16 = 0; k16 < BK / 16; ++k16)       // 32 bytes along K per MMA: +2 in the address field
-            umma_f16(d_tmem, adesc + 2 * k16, bdesc + 2 * k16, c.idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+            umma_f16(d_tmem, adesc + 2 * k16, bdesc + 2 * k16, c.idesc, (kb > sg.kb0 || k16 > 0) ? 1u : 0u);
           umma_commit(empty + 8 * s);                   // the stage is free once these MMAs have read it
           if (++s == PSTAGES) { s = 0; par ^= 1; }
         }
@@ -333,9 +384,12 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
     uint32_t col_off[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) col_off[j] = (uint32_t)(((hf * 4 + j) ^ (r & 7)) * 16);
-    int it0 = 0;                       // stage iterations before this tile
-    for (int t = blockIdx.x; t < c.n_tiles && !failed; t += gridDim.x, it0 += c.n_kb) {
-      const int wt = t / c.n_ttiles;
+    int done = 0;                      // stage iterations before this segment
+    SegIter si; si.init(c, blockIdx.x, gridDim.x);
+    Seg sg;
+    for (; !failed && si.next(sg); done += sg.kb1 - sg.kb0) {
+      const int it0 = done - sg.kb0;   // stage iteration of k-block kb of this segment = it0 + kb
+      const int wt = sg.tile / c.n_ttiles;
       const int jn = job_of_wt(wt);
       const JobDev& jb = p.job[jn];
       const RowInfo ri = tile_row(jb, wt - c.wtile_begin[jn], r);
@@ -343,27 +397,27 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
       const uint8_t* wrow = jb.w + (size_t)(live ? ri.stored : 0) * (p.K / 2) + hf * 16;
       const __half* srow = jb.scales + (size_t)(live ? ri.stored : 0) * G;
       const __half* zrow = jb.zeros + (size_t)(live ? ri.stored : 0) * G;
-      const int kb0 = ((it0 & 1) == team) ? 0 : 1;
+      const int kb0 = ((done & 1) == team) ? sg.kb0 : sg.kb0 + 1;
       // codes and scale / zero-point of this team's next two k-blocks are kept in registers
       uint4 q0 = make_uint4(0, 0, 0, 0), q1 = q0;
       __half s0 = __ushort_as_half(0), z0 = s0, s1 = s0, z1 = s0;
       if (live) {
-        if (kb0 < c.n_kb) {
+        if (kb0 < sg.kb1) {
           q0 = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)kb0 * 32));
           s0 = __ldg(srow + (kb0 >> 1)); z0 = __ldg(zrow + (kb0 >> 1));
         }
-        if (kb0 + 2 < c.n_kb) {
+        if (kb0 + 2 < sg.kb1) {
           q1 = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)(kb0 + 2) * 32));
           s1 = __ldg(srow + ((kb0 + 2) >> 1)); z1 = __ldg(zrow + ((kb0 + 2) >> 1));
         }
       }
-      for (int kb = kb0; kb < c.n_kb; kb += 2) {
+      for (int kb = kb0; kb < sg.kb1; kb += 2) {
         const int it = it0 + kb;
         const int s = it & (PSTAGES - 1);
         const uint32_t use = (uint32_t)(it / PSTAGES);
         uint4 q2 = make_uint4(0, 0, 0, 0);
         __half s2 = s1, z2 = z1;
-        if (live && kb + 4 < c.n_kb) {
+        if (live && kb + 4 < sg.kb1) {
           q2 = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)(kb + 4) * 32));
           s2 = __ldg(srow + ((kb + 4) >> 1)); z2 = __ldg(zrow + ((kb + 4) >> 1));
         }
@@ -408,9 +462,13 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
       epar ^= 1;
       return ok;
     };
+    volatile int* last_flag = reinterpret_cast<volatile int*>(misc + 8);
     int tcount = 0;
-    for (int t = blockIdx.x; t < c.n_tiles && !failed; t += gridDim.x, ++tcount) {
+    SegIter si; si.init(c, blockIdx.x, gridDim.x);
+    Seg sg;
+    for (; !failed && si.next(sg); ++tcount) {
       const int buf = tcount & 1;
+      const int t = sg.tile;
       const int wt = t / c.n_ttiles, tt = t - wt * c.n_ttiles;
       const int jn = job_of_wt(wt);
       const JobDev& jb = p.job[jn];
@@ -434,43 +492,98 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
           invf = p.inv_freq[pidx];
         }
       }
-      if (!pmbar_wait(acc_full + 8 * buf, (tcount >> 1) & 1, abort_flag)) { failed = true; break; }
-      tc_fence_after();
-      for (int ch = 0; ch < c.bn / EPI_TOK && !failed; ++ch) {
-        uint32_t v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * MAXBN + ch * EPI_TOK), v);
-        tmem_ld_wait();
-        // staging[token][row]: lanes are consecutive rows
-#pragma unroll
-        for (int k = 0; k < 32; ++k) stg_p[k * BMW + 32 * q + lane] = __uint_as_float(v[k]);
-        if (!epi_sync()) { failed = true; break; }
+      // bias, rotary embedding, rounding and store of the 32 tokens that sit in the staging tile
+      auto store_chunk = [&](int ch) {
         const int m0 = tt * c.bn + ch * EPI_TOK;
-        if (ri.stored >= 0) {
-          if (rope) {
-            const int half = jb.rope.head_keep >> 1;
-            for (int k = etid >> 6; k < EPI_TOK; k += 2) {
-              const int m = m0 + k;
-              if (m >= p.M) break;
-              const float lo = stg_p[k * BMW + (etid & 63)] + b_lo, hi = stg_p[k * BMW + 64 + (etid & 63)] + b_hi;
-              float cs, sn;
-              rope_cos_sin(p.pos[m], invf, cs, sn);
-              y[(size_t)m * jb.ldy + ri.out_col] = DT<T>::from_f(lo * cs - hi * sn);
-              y[(size_t)m * jb.ldy + ri.out_col + half] = DT<T>::from_f(hi * cs + lo * sn);
-            }
-          } else {
-            for (int k = 0; k < EPI_TOK; ++k) {
-              const int m = m0 + k;
-              if (m >= p.M) break;
-              y[(size_t)m * jb.ldy + ri.out_col] = DT<T>::from_f(stg_p[k * BMW + etid] + b_lo);
-            }
+        if (ri.stored < 0) return;
+        if (rope) {
+          const int half = jb.rope.head_keep >> 1;
+          for (int k = etid >> 6; k < EPI_TOK; k += 2) {
+            const int m = m0 + k;
+            if (m >= p.M) break;
+            const float lo = stg_p[k * BMW + (etid & 63)] + b_lo, hi = stg_p[k * BMW + 64 + (etid & 63)] + b_hi;
+            float cs, sn;
+            rope_cos_sin(p.pos[m], invf, cs, sn);
+            y[(size_t)m * jb.ldy + ri.out_col] = DT<T>::from_f(lo * cs - hi * sn);
+            y[(size_t)m * jb.ldy + ri.out_col + half] = DT<T>::from_f(hi * cs + lo * sn);
+          }
+        } else {
+          for (int k = 0; k < EPI_TOK; ++k) {
+            const int m = m0 + k;
+            if (m >= p.M) break;
+            y[(size_t)m * jb.ldy + ri.out_col] = DT<T>::from_f(stg_p[k * BMW + etid] + b_lo);
           }
         }
-        if (!epi_sync()) { failed = true; break; }       // staging is rewritten by the next pass
+      };
+      if (!pmbar_wait(acc_full + 8 * buf, (tcount >> 1) & 1, abort_flag)) { failed = true; break; }
+      tc_fence_after();
+      const uint32_t t_acc = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * MAXBN);
+      const int row = 32 * q + lane;
+      if (sg.kb0 == 0 && sg.kb1 == c.n_kb) {
+        // ---- the whole contraction of this tile ran here
+        for (int ch = 0; ch < c.bn / EPI_TOK && !failed; ++ch) {
+          uint32_t v[32];
+          tmem_ld32(t_acc + (uint32_t)(ch * EPI_TOK), v);
+          tmem_ld_wait();
+          // staging[token][row]: lanes are consecutive rows
+#pragma unroll
+          for (int k = 0; k < 32; ++k) stg_p[k * BMW + row] = __uint_as_float(v[k]);
+          if (!epi_sync()) { failed = true; break; }
+          store_chunk(ch);
+          if (!epi_sync()) { failed = true; break; }       // staging is rewritten by the next pass
+        }
+        if (failed) break;
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) pmbar_arrive(acc_empty + 8 * buf);
+      } else {
+        // ---- a part of the contraction (stream-K): park the fp32 partial tile [token][row]; the last of the
+        //      tile's blocks to arrive adds the parts in block order and finishes the tile
+        const size_t slot_f = (size_t)c.bn * BMW;
+        float* mine = c.partials + (size_t)(2 * blockIdx.x + (sg.tail_idx == 0 ? 0 : 1)) * slot_f;
+        for (int ch = 0; ch < c.bn / EPI_TOK; ++ch) {
+          uint32_t v[32];
+          tmem_ld32(t_acc + (uint32_t)(ch * EPI_TOK), v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int k = 0; k < 32; ++k) __stcg(mine + (size_t)(ch * EPI_TOK + k) * BMW + row, __uint_as_float(v[k]));
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) pmbar_arrive(acc_empty + 8 * buf);      // the accumulator is free for the next segment
+        __threadfence();
+        if (!epi_sync()) { failed = true; break; }
+        const int T0 = (c.n_tiles / (int)gridDim.x) * (int)gridDim.x;          // first left-over tile
+        const long U = (long)(c.n_tiles - T0) * c.n_kb, Bn = (long)gridDim.x < U ? (long)gridDim.x : U;
+        const long tu = (long)(t - T0) * c.n_kb;                               // the tile's first left-over unit
+        const int first = sk_owner(tu, Bn, U), last = sk_owner(tu + c.n_kb - 1, Bn, U);
+        if (etid == 0) {
+          const int arrived = atomicAdd(&c.counters[t], 1);
+          *last_flag = arrived == last - first;
+          __threadfence();
+        }
+        if (!epi_sync()) { failed = true; break; }
+        if (*last_flag) {
+          for (int ch = 0; ch < c.bn / EPI_TOK && !failed; ++ch) {
+            float acc[32];
+#pragma unroll
+            for (int k = 0; k < 32; ++k) acc[k] = 0.f;
+            for (int j = first; j <= last; ++j) {
+              // block j's part of this tile sits in its first slot when its left-over range starts inside the tile
+              const int sj = (U * j / Bn >= tu) ? 0 : 1;
+              const float* src = c.partials + (size_t)(2 * j + sj) * slot_f + (size_t)(ch * EPI_TOK) * BMW + row;
+#pragma unroll
+              for (int k = 0; k < 32; ++k) acc[k] += __ldcg(src + (size_t)k * BMW);
+            }
+#pragma unroll
+            for (int k = 0; k < 32; ++k) stg_p[k * BMW + row] = acc[k];
+            if (!epi_sync()) { failed = true; break; }
+            store_chunk(ch);
+            if (!epi_sync()) { failed = true; break; }
+          }
+          if (etid == 0) c.counters[t] = 0;              // ready for the next call
+        }
       }
-      if (failed) break;
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) pmbar_arrive(acc_empty + 8 * buf);
     }
   }
 
@@ -555,13 +668,22 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   // instruction descriptor: fp32 accumulate, A and B of the activation type, both K-major, N = bn, M = 128
   c.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(c.bn >> 3) << 17) | ((uint32_t)(BMW >> 4) << 24);
   c.status = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(cfg.workspace) + decode_status_offset());
+  const int sms = p_sm_count();
+  int grid = c.n_tiles < sms ? c.n_tiles : sms;
+  if (const char* g = getenv("UNIQL_PREFILL_GRID")) {          // tests: odd splits on small problems
+    const int v = atoi(g);
+    if (v >= 1 && v <= sms) grid = v;
+  }
+  // workspace: [header: counters, status][fp16 copy of bf16 activations][stream-K partial tiles]
+  size_t ws_used = (decode_workspace_header_bytes() + 255) & ~(size_t)255;
+  c.counters = reinterpret_cast<int*>(cfg.workspace);
   // bf16 activations: fp16 copy in the workspace when it fits (else converted tile by tile in the kernel)
   const void* xsrc = p.x;
   int ldxs = p.ldx;
   bool conv_in_kernel = false;
   if (p.dt == UNIQL_BF16) {
     const int ldo = (p.k_in + 7) / 8 * 8;
-    const size_t off = (decode_workspace_header_bytes() + 255) & ~(size_t)255;
+    const size_t off = ws_used;
     const size_t need = off + (size_t)p.M * ldo * 2;
     const char* force = getenv("UNIQL_PREFILL_CONVERT");
     if (cfg.ws_bytes >= need && !(force && force[0] == 'k')) {
@@ -573,8 +695,25 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
       if (cudaGetLastError() != cudaSuccess) return UNIQL_ERR_CUDA;
       xsrc = x16;
       ldxs = ldo;
+      ws_used = (need + 255) & ~(size_t)255;
     } else {
       conv_in_kernel = true;
+    }
+  }
+  // stream-K for the last round when whole tiles would leave many SMs idle in it, the share of every block
+  // is long enough to amortise the hand-over of a partial tile, and the partial tiles fit in the workspace
+  {
+    int g2 = sms;
+    if (const char* g = getenv("UNIQL_PREFILL_GRID")) { const int v = atoi(g); if (v >= 1 && v <= sms) g2 = v; }
+    const int left = c.n_tiles % g2;
+    const long share = left ? (long)left * c.n_kb / g2 : 0;            // k-blocks per block in the last round
+    const size_t need = ws_used + (size_t)2 * g2 * c.bn * BMW * 4;
+    const char* force = getenv("UNIQL_PREFILL_STREAMK");
+    const bool want = force ? (force[0] == '1') : (left != 0 && left * 10 < g2 * 9 && share >= 48);
+    if (want && left != 0 && cfg.ws_bytes >= need && c.n_tiles <= (1 << 16)) {
+      c.streamk = 1;
+      c.partials = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(cfg.workspace) + ws_used);
+      grid = g2;
     }
   }
   {
@@ -588,8 +727,6 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return UNIQL_ERR_CUDA;
   }
-  const int sms = p_sm_count();
-  const int grid = c.n_tiles < sms ? c.n_tiles : sms;
   if (p.dt == UNIQL_BF16)
     return conv_in_kernel ? launch_pt<__nv_bfloat16, true>(p, c, grid, cfg.stream)
                           : launch_pt<__nv_bfloat16, false>(p, c, grid, cfg.stream);
@@ -597,8 +734,9 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
 }
 
 size_t prefill_workspace_bytes(int M, int K) {
-  // status word (shared header) + room for the fp16 copy of bf16 activations
-  return ((decode_workspace_header_bytes() + 255) & ~(size_t)255) + (size_t)M * ((K + 7) / 8 * 8) * 2;
+  // status word and counters (shared header) + room for the fp16 copy of bf16 activations + stream-K partial tiles
+  return ((decode_workspace_header_bytes() + 255) & ~(size_t)255) + (size_t)M * ((K + 7) / 8 * 8) * 2 + 256 +
+         (size_t)2 * 148 * MAXBN * BMW * 4;
 }
 
 }  // namespace uniql

@@ -104,6 +104,27 @@ def test_prefill_bf16_converted_in_kernel(B, monkeypatch):
     assert torch.equal(y1, y2)
 
 
+@pytest.mark.parametrize("grid", [1, 3, 5, 7, 11])
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+def test_prefill_stream_k(B, monkeypatch, grid, dtype):
+    """Stream-K: blocks take contiguous ranges of (tile, k-block) units; tiles cut by a range boundary are
+    finished by the last block to arrive.  Every split gives the same answer, bit for bit, run after run."""
+    B.set_path(B.PATH_PREFILL)
+    monkeypatch.setenv("UNIQL_PREFILL_STREAMK", "1")
+    monkeypatch.setenv("UNIQL_PREFILL_GRID", str(grid))
+    rng = np.random.default_rng(900 + grid)
+    qw = synth.draw_qweight(rng, 300, 1024)
+    dw = dev_weight(qw)
+    x = synth.draw_x(rng, 300, 1024, dtype)                      # 3 weight tiles x 2 token tiles, 16 k-blocks
+    y, ref = run_ex(B, qw, dw, x, dtype, None, 1024, None, 300)
+    check_output(y, ref, dtype, TOL[dtype], "stream-K grid %d" % grid)
+    y2, _ = run_ex(B, qw, dw, x, dtype, None, 1024, None, 300)
+    assert torch.equal(y, y2)
+    for (g, r) in run_rope(B, rng, 200, 512, 6, 2, 128, 84, 5e5, dtype):
+        check_output(g, r, dtype, TOL[dtype], "stream-K rope grid %d" % grid)
+    assert B.workspace_status() == 0
+
+
 def test_prefill_multi_job(B):
     rng = np.random.default_rng(800)
     gate, up = synth.draw_qweight(rng, 352, 512), synth.draw_qweight(rng, 352, 512)
