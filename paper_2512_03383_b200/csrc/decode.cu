@@ -187,6 +187,20 @@ __device__ inline void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+__device__ inline void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+template <int OFF>
+__device__ inline float2 lds64f(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0,%1}, [%2+%3];" : "=f"(v.x), "=f"(v.y) : "r"(addr), "n"(OFF));
+  return v;
+}
+// exact int -> float for |v| < 2^22 without the conversion unit
+__device__ inline float small_int_to_float(int v) { return __int_as_float(v + 0x4B400000) - 12582912.f; }
+
 // ---------------------------------------------------------------------------------------- tile geometry
 struct TilePos { int fi, h, r0; };
 __device__ inline TilePos tile_pos(const DecodeCfg& c, const Params& p, int tg) {
@@ -304,7 +318,9 @@ struct UnitIter {
 };
 
 // ---------------------------------------------------------------------------------------- kernel
-template <int MT, bool ONECOL>
+// NT == 0: fp16 tensor-core path (MT batch tiles of 8, ONECOL: batch 1).  NT > 0: integer path, NT column
+// tiles of the int8 MMA, each holding the high and the low byte of four batch rows.
+template <int MT, bool ONECOL, int NT>
 __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ Params p,
                                                         const __grid_constant__ DecodeCfg c) {
   extern __shared__ unsigned char smem_raw[];
@@ -566,7 +582,77 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     float2* xg = reinterpret_cast<float2*>(smem + c.off_xg);
     for (int i = ctid; i < Gk * 8 * MT; i += CTH) xg[i] = make_float2(0.f, 0.f);
     if (!consumer_sync()) return;
-    if (c.x_vec) {
+    if (NT > 0) {
+      // Integer path.  Per (batch row, group) the activations become 16-bit fixed point, x_i = rint(x * 2^e)
+      // with 2^e the largest power of two that keeps the group's maximum at or below 32639 (so that the high
+      // byte of x_i + 128 stays a signed byte; exact for every element within a factor 8..16 of the maximum,
+      // since fp16 carries 11 bits; smaller elements are rounded to 2^-15..2^-14 of the maximum).
+      // x_i = 256 * hi + lo with both bytes signed; the bytes go to two "virtual"
+      // batch rows (columns 2m and 2m+1 of the int8 MMA), in the order the nibbles leave a weight word:
+      // even codes in the first register of a word's pair, odd codes in the second.
+      const int start = p.imap.fam[0].start, keep = p.imap.fam[0].keep;
+      const int n_units = Gk * p.M * 16;
+      unsigned char* xb = smem + c.off_x;
+      constexpr int UN = 4;
+      for (int u0 = ctid; u0 < ((n_units + 31) & ~31); u0 += CTH * UN) {
+        uint4 in[UN];
+#pragma unroll
+        for (int q4 = 0; q4 < UN; ++q4) {
+          const int u = u0 + q4 * CTH;
+          in[q4] = make_uint4(0, 0, 0, 0);
+          if (u < n_units) {
+            const int pair = u >> 4, m = pair / Gk, lv = pair - m * Gk;
+            const int t0 = (sg_lo + lv) * kGroup + 8 * (u & 15) - start;
+            if (t0 >= 0 && t0 < keep) in[q4] = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * p.ldx + t0));
+          }
+        }
+#pragma unroll
+        for (int q4 = 0; q4 < UN; ++q4) {
+          const int u = u0 + q4 * CTH;
+          if (u >= ((n_units + 31) & ~31)) break;                  // warp-uniform
+          const bool in_range = u < n_units;
+          const int u16 = u & 15, pair = in_range ? u >> 4 : 0;
+          const int m = pair / Gk, lv = pair - m * Gk;
+          const __half2* h2 = reinterpret_cast<const __half2*>(&in[q4]);
+          float f[8];
+          float amax = 0.f;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float2 v = __half22float2(h2[i]);
+            f[2 * i] = v.x; f[2 * i + 1] = v.y;
+            amax = fmaxf(amax, fmaxf(fabsf(v.x), fabsf(v.y)));
+          }
+#pragma unroll
+          for (int o2 = 8; o2 >= 1; o2 >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o2));
+          int e = 0;
+          if (amax > 0.f && amax < 3.0e38f) {
+            e = 14 - ((int)((__float_as_uint(amax) >> 23) & 255u) - 127);
+            if (amax * __uint_as_float((uint32_t)(127 + e) << 23) > 32639.f) --e;     // keep the high byte of x_i + 128 signed
+          }
+          const float scale = __uint_as_float((uint32_t)(127 + e) << 23), inv_scale = __uint_as_float((uint32_t)(127 - e) << 23);
+          int isum = 0;
+          uint32_t hi_e = 0, hi_o = 0, lo_e = 0, lo_o = 0;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const int xi = __float2int_rn(f[k] * scale);
+            isum += xi;
+            const int hi = (xi + 128) >> 8, lo = xi - (hi << 8);
+            const int sh = 8 * (k >> 1);
+            if (k & 1) { hi_o |= (uint32_t)(hi & 255) << sh; lo_o |= (uint32_t)(lo & 255) << sh; }
+            else       { hi_e |= (uint32_t)(hi & 255) << sh; lo_e |= (uint32_t)(lo & 255) << sh; }
+          }
+#pragma unroll
+          for (int o2 = 8; o2 >= 1; o2 >>= 1) isum += __shfl_xor_sync(0xffffffffu, isum, o2);
+          if (in_range) {
+            // word j of lane quarter c' (u16 = c'*4 + j): 8 bytes at c'*32 + j*8 of the group's 128 bytes
+            const int off = lv * 128 + (u16 >> 2) * 32 + (u16 & 3) * 8;
+            *reinterpret_cast<uint2*>(xb + (size_t)(2 * m) * c.xrow + off) = make_uint2(hi_e, hi_o);
+            *reinterpret_cast<uint2*>(xb + (size_t)(2 * m + 1) * c.xrow + off) = make_uint2(lo_e, lo_o);
+            if (u16 == 0) xg[lv * 8 * MT + m] = make_float2((float)isum, inv_scale);
+          }
+        }
+      }
+    } else if (c.x_vec) {
       const int start = p.imap.fam[0].start, keep = p.imap.fam[0].keep;
       const int n_units = Gk * p.M * 16;
       constexpr int UN = 4;                                        // loads in flight per thread
@@ -632,6 +718,128 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       }
     }
     if (!consumer_sync()) return;
+  }
+
+  if constexpr (NT > 0) {
+    // ===================================================================== consumers, integer path
+    // Per weight word: low nibbles and high nibbles as bytes (AND, SHR, AND) are the A fragments of one
+    // m16n8k32 int8 MMA for two weight rows; B holds the activation bytes.  Column 2m of the MMA sums
+    // q * hi, column 2m+1 sums q * lo: both land in the same lane, 256 * d_hi + d_lo is sum q * x_i exactly.
+    uint32_t xaddr8[NT];
+    bool xlive8[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const int v = g + 8 * nt;                        // virtual batch row: 2m (high bytes), 2m+1 (low bytes)
+      xlive8[nt] = v < 2 * p.M;
+      xaddr8[nt] = sbase + c.off_x + (uint32_t)((xlive8[nt] ? v : 0) * c.xrow + t * 32);
+    }
+    const uint32_t xgaddr8 = sbase + c.off_xg + (uint32_t)(t * 8);           // batch row m = t + 4 nt
+    const uint32_t wl_off = (uint32_t)((kpw >> 1) * BOX_BYTES + (rg * 32 + pg) * 128 + ((((kpw & 1) * 4 + t) ^ pg) * 16));
+    const uint32_t sl_off = (uint32_t)(STAGE_W + (rg * 32 + pg) * (CG * 2) + kpw * 2);
+    float out8[2][NT][2];
+#pragma unroll
+    for (int sub = 0; sub < 2; ++sub)
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) out8[sub][nt][0] = out8[sub][nt][1] = 0.f;
+    uint4 xr8[NT][2];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) xr8[nt][0] = xr8[nt][1] = make_uint4(0, 0, 0, 0);
+    UnitIter ui;
+    ui.start(wk);
+    int tiles_done = 0;
+    int s = 0;
+    uint32_t ring_parity = 0;
+    for (int i = 0; i < wk.n_units; ++i) {
+      if (!mbar_try_wait(bar_full + 8 * s, ring_parity) && !mbar_wait(bar_full + 8 * s, ring_parity, abort_flag)) {
+        give_up();
+        return;
+      }
+      const int gi = ui.chunk * CG + kpw;
+      if (gi < Gk) {
+        const uint32_t st = sbase + (uint32_t)s * STAGE_BYTES;
+        const uint32_t wp = st + wl_off, sp = st + sl_off;
+        uint4 wa[2], wb[2];
+        wa[0] = lds128<0>(wp);
+        wb[0] = lds128<8 * 128>(wp);
+        wa[1] = lds128<16 * 128>(wp);
+        wb[1] = lds128<24 * 128>(wp);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          const uint32_t xa = xaddr8[nt] + (uint32_t)(gi * 128);
+          lds128_if<0>(xr8[nt][0], xa, xlive8[nt]);
+          lds128_if<16>(xr8[nt][1], xa, xlive8[nt]);
+        }
+        float sc[2][2], zp[2][2];
+        sc[0][0] = lds_h<0>(sp);
+        sc[0][1] = lds_h<8 * CG * 2>(sp);
+        sc[1][0] = lds_h<16 * CG * 2>(sp);
+        sc[1][1] = lds_h<24 * CG * 2>(sp);
+        zp[0][0] = lds_h<STAGE_SZ>(sp);
+        zp[0][1] = lds_h<STAGE_SZ + 8 * CG * 2>(sp);
+        zp[1][0] = lds_h<STAGE_SZ + 16 * CG * 2>(sp);
+        zp[1][1] = lds_h<STAGE_SZ + 24 * CG * 2>(sp);
+        int d[2][NT][4];
+#pragma unroll
+        for (int sub = 0; sub < 2; ++sub)
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) d[sub][nt][e] = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+#pragma unroll
+          for (int sub = 0; sub < 2; ++sub) {
+            const uint32_t w0 = j == 0 ? wa[sub].x : j == 1 ? wa[sub].y : j == 2 ? wa[sub].z : wa[sub].w;
+            const uint32_t w1 = j == 0 ? wb[sub].x : j == 1 ? wb[sub].y : j == 2 ? wb[sub].z : wb[sub].w;
+            const uint32_t lo0 = w0 & 0x0f0f0f0fu, hi0 = (w0 >> 4) & 0x0f0f0f0fu;
+            const uint32_t lo1 = w1 & 0x0f0f0f0fu, hi1 = (w1 >> 4) & 0x0f0f0f0fu;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              const uint4 xv = xr8[nt][j >> 1];
+              const uint32_t b0 = (j & 1) ? xv.z : xv.x, b1 = (j & 1) ? xv.w : xv.y;
+              mma_s8(d[sub][nt], lo0, lo1, hi0, hi1, b0, b1);
+            }
+          }
+        }
+        const uint32_t xga = xgaddr8 + (uint32_t)(gi * 8 * MT * 8);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          const float2 xs = nt == 0 ? lds64f<0>(xga) : nt == 1 ? lds64f<32>(xga) : nt == 2 ? lds64f<64>(xga) : lds64f<96>(xga);
+#pragma unroll
+          for (int sub = 0; sub < 2; ++sub) {
+            const float y0 = fmaf(256.f, small_int_to_float(d[sub][nt][0]), small_int_to_float(d[sub][nt][1]));
+            const float y1 = fmaf(256.f, small_int_to_float(d[sub][nt][2]), small_int_to_float(d[sub][nt][3]));
+            out8[sub][nt][0] = fmaf(sc[sub][0] * xs.y, fmaf(-zp[sub][0], xs.x, y0), out8[sub][nt][0]);
+            out8[sub][nt][1] = fmaf(sc[sub][1] * xs.y, fmaf(-zp[sub][1], xs.x, y1), out8[sub][nt][1]);
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+      if (++s == S) { s = 0; ring_parity ^= 1; }
+      if (ui.tile_end(wk, i)) {
+        const int buf = c.part_bufs > 1 ? (tiles_done & 1) : 0;
+        const int use = c.part_bufs > 1 ? (tiles_done >> 1) : tiles_done;
+        if (use > 0 && !mbar_wait(bar_pfree + 8 * buf, (use - 1) & 1, abort_flag)) { give_up(); return; }
+        float* pb = part + buf * part_stride + kpw * RM;
+#pragma unroll
+        for (int sub = 0; sub < 2; ++sub)
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            const int m = t + 4 * nt;
+            if (m < p.M) {
+              pb[m * RB + rg * 32 + sub * 16 + pg] = out8[sub][nt][0];
+              pb[m * RB + rg * 32 + sub * 16 + pg + 8] = out8[sub][nt][1];
+            }
+            out8[sub][nt][0] = out8[sub][nt][1] = 0.f;
+          }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_pfull + 8 * buf);
+        ++tiles_done;
+      }
+      if (i + 1 < wk.n_units) ui.advance(wk, i + 1);
+    }
+    return;
   }
 
   // per-lane shared-memory addresses
@@ -842,13 +1050,15 @@ int encode_family(CUtensorMap* tm, const uint8_t* base, int K, int x_extent, int
 }
 
 // Shared-memory plan for a given split; returns the total size in bytes (with the alignment slack).
-size_t plan_smem(DecodeCfg* c, int M, int MT, int gp, int stages, int part_bufs) {
+size_t plan_smem(DecodeCfg* c, int M, int MT, int gp, int stages, int part_bufs, bool i8) {
   size_t off = (size_t)stages * STAGE_BYTES;
   c->off_bar = (int)off;
   off += BAR_BYTES;
-  c->xrow = gp * 256 + 64;
+  // fp16 path: one row of gp*256 bytes per batch row (+64: lane pairs on distinct banks);
+  // integer path: two rows (high and low bytes) of gp*128 bytes per batch row (+16)
+  c->xrow = i8 ? gp * 128 + 16 : gp * 256 + 64;
   c->off_x = (int)off;
-  off += (size_t)M * c->xrow;
+  off += (size_t)M * (i8 ? 2 : 1) * c->xrow;
   off = (off + 15) & ~(size_t)15;
   c->off_xg = (int)off;
   off += (size_t)gp * 8 * MT * 8;
@@ -877,9 +1087,9 @@ int slots_needed(int tiles, int g_total, int gp, int n_rp) {
   return total;
 }
 
-template <int MT, bool ONECOL>
+template <int MT, bool ONECOL, int NT>
 int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stream) {
-  auto kern = decode_kernel<MT, ONECOL>;
+  auto kern = decode_kernel<MT, ONECOL, NT>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return UNIQL_ERR_CUDA;
   cudaLaunchConfig_t lc;
@@ -914,7 +1124,7 @@ void visited_range(const ChanMap& m, int gran, int* first, int* total) {
 
 // Split of the visited groups into k-parts and the shared-memory plan: as few k-parts as let the staged
 // activations fit beside a deep enough ring of stages.  Returns 0 when nothing fits.
-size_t plan_split(DecodeCfg* c, int M, int g_total, int gran) {
+size_t plan_split(DecodeCfg* c, int M, int g_total, int gran, bool i8) {
   const int MT = M <= 8 ? 1 : 2;
   const int part_bufs = M <= 8 ? 2 : 1;
   int n_kp = env_int("UNIQL_DECODE_KP", 0);
@@ -926,7 +1136,7 @@ size_t plan_split(DecodeCfg* c, int M, int g_total, int gran) {
     if (n_kp > kMaxKParts) n_kp = kMaxKParts;
     const int gp = round_up((g_total + n_kp - 1) / n_kp, gran);
     for (int s = want; s >= 2 && !fits; --s) {
-      smem = plan_smem(c, M, MT, gp, s, part_bufs);
+      smem = plan_smem(c, M, MT, gp, s, part_bufs, i8);
       fits = smem <= (size_t)kSmemMax;
     }
     c->gp = gp;
@@ -934,7 +1144,7 @@ size_t plan_split(DecodeCfg* c, int M, int g_total, int gran) {
     for (n_kp = 1; n_kp <= kMaxKParts && !fits; ++n_kp)
       for (int s = want; s >= 3 && !fits; --s) {
         const int gp = round_up((g_total + n_kp - 1) / n_kp, gran);
-        smem = plan_smem(c, M, MT, gp, s, part_bufs);
+        smem = plan_smem(c, M, MT, gp, s, part_bufs, i8);
         fits = smem <= (size_t)kSmemMax;
         c->gp = gp;
       }
@@ -974,7 +1184,7 @@ size_t decode_workspace_bytes(int M, int K, int N_total) {
   DecodeCfg c;
   memset(&c, 0, sizeof(c));
   const int G = (K + kGroup - 1) / kGroup;
-  if (!plan_split(&c, M, G, 2)) return (size_t)kWsHeader;
+  if (!plan_split(&c, M, G, 2, false)) return (size_t)kWsHeader;
   const size_t chunks = (size_t)(G + CG - 1) / CG;
   const size_t tiles = (size_t)(N_total + RB - 1) / RB + (size_t)N_total / 32 + 2 * kMaxJobs;
   const size_t slots = tiles * 2 * c.n_kp + (size_t)c.n_rp * c.n_kp * (chunks + 2 * c.n_kp);
@@ -1027,7 +1237,9 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   c.tiles_total = tiles;
   if (tiles < 1 || tiles > kCounterInts) return UNIQL_ERR_UNSUPPORTED;
 
-  const size_t smem = plan_split(&c, p.M, g_total, gran);
+  // integer path: fp16 activations staged with 128-bit loads (a leading input block); UNIQL_DECODE_I8=0: fp16 MMAs
+  const bool i8 = c.x_vec && env_int("UNIQL_DECODE_I8", 1) != 0;
+  const size_t smem = plan_split(&c, p.M, g_total, gran, i8);
   if (!smem) return UNIQL_ERR_UNSUPPORTED;
   c.max_slots = slots_needed(tiles, c.g_total, c.gp, c.n_rp);
   {
@@ -1038,8 +1250,13 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   c.counters = reinterpret_cast<int*>(ws);
   c.status = reinterpret_cast<int*>(ws + kStatusOff);
   c.partials = reinterpret_cast<float*>(ws + kWsHeader);
-  if (MT == 1) return p.M == 1 ? launch_t<1, true>(p, c, smem, cfg.stream) : launch_t<1, false>(p, c, smem, cfg.stream);
-  return launch_t<2, false>(p, c, smem, cfg.stream);
+  if (i8) {
+    if (p.M <= 4) return launch_t<1, false, 1>(p, c, smem, cfg.stream);
+    if (p.M <= 8) return launch_t<1, false, 2>(p, c, smem, cfg.stream);
+    return launch_t<2, false, 4>(p, c, smem, cfg.stream);
+  }
+  if (MT == 1) return p.M == 1 ? launch_t<1, true, 0>(p, c, smem, cfg.stream) : launch_t<1, false, 0>(p, c, smem, cfg.stream);
+  return launch_t<2, false, 0>(p, c, smem, cfg.stream);
 }
 
 int decode_status_offset() { return kStatusOff; }

@@ -12,11 +12,13 @@ from paper_2512_03383_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
-# Decode / generic kernels: exact products, fp32 accumulation.  The decode kernel feeds the tensor
-# cores the codes with their conversion offsets (1024+q, 64+q) and removes the offsets per group in
-# fp32, so each group's accumulator is about 1000 times larger than its useful part and its fp32
-# rounding (2^-24 relative) shows up as roughly 1e-4 of the output scale: a tenth of the 2e-3 bar.
-TIGHT = 2e-4
+# Decode / generic kernels.  Products and sums are exact or fp32; what the decode kernel adds is the
+# representation of the activations: for fp16 inputs it runs on int8 tensor-core MMAs over 16-bit fixed-point
+# activations (per batch row and 128-channel group, scaled to the group's maximum), so elements far below
+# their group's maximum are rounded to 2^-15..2^-14 of that maximum.  With the x20 outlier channels of the
+# synthetic inputs and short rows (K = 256) this reaches 2..3e-4 of the output scale; long rows average it
+# down (measured 3e-5 at K = 4096).  Held to 4e-4, a fifth of the 2e-3 bar.
+TIGHT = 4e-4
 
 
 @pytest.fixture(scope="module")
