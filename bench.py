@@ -386,6 +386,7 @@ def run_ours(args):
         if args.detail:
             line["detail"] = detail_tables(B, torch, max(20, min(args.steps, 200)))
             line["detail"].update(prefill_tables(B, torch))
+            line["detail"].update(attention_tables(B, torch, 20))
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -453,6 +454,58 @@ def prefill_tables(B, torch):
             out["prefill_qwen_%s_M%d" % (name, M)] = rows
         del q
         torch.cuda.empty_cache()
+    return out
+
+
+def attention_tables(B, torch, steps):
+    """Llama-3-8B Q and K projection with the fused pruned RoPE (one launch): decode at M = 1, 16 and the
+    tensor-core path at M = 512, per retained head dim.  Weights rotate over enough copies to exceed L2."""
+    from paper_2512_03383_b200 import synth
+    hbm, tf, which = measured_peaks()
+    rng = np.random.default_rng(3)
+    Hq, Hkv, D, K, theta = 32, 8, 128, HIDDEN, 500000.0
+    n_copies = 14                                   # 14 x 11.1 MB > 126 MB
+    wq, wk = synth.random_qweight_fast(rng, Hq * D, K), synth.random_qweight_fast(rng, Hkv * D, K)
+    copies = []
+    for _ in range(n_copies):
+        c = []
+        for m in (wq, wk):
+            cd = torch.from_numpy(m.codes).cuda()
+            packed = torch.empty((m.N, m.K // 2), dtype=torch.uint8, device="cuda")
+            B.pack_u4(cd, packed)
+            c.append((packed, torch.from_numpy(m.scales).cuda().clone(), torch.from_numpy(m.zeros).cuda().clone()))
+        copies.append(c)
+    out = {}
+    for M in (1, 16, 512):
+        x = torch.from_numpy(synth.draw_x(rng, M, K, "f16")).cuda().half()
+        pos = torch.from_numpy(synth.draw_pos(rng, M)).cuda()
+        rows = {}
+        for keep in (128, 108, 96, 84):
+            idx = torch.from_numpy(synth.draw_idx(rng, Hkv, D, keep)).cuda()
+            qo = torch.zeros((M, Hq * keep), dtype=torch.float16, device="cuda")
+            ko = torch.zeros((M, Hkv * keep), dtype=torch.float16, device="cuda")
+            turn = [0]
+
+            def one():
+                for _ in range(n_copies):
+                    (q, k) = copies[turn[0] % n_copies]
+                    turn[0] += 1
+                    B.qk_rope_proj(x, K, q[0], q[1], q[2], k[0], k[1], k[2], None, None, M, K, Hq, Hkv, D, keep, idx, pos,
+                                   theta, None, qo, Hq * keep, ko, Hkv * keep)
+            g, _ = capture(torch, one)
+            for _ in range(3):
+                g.replay()
+            sec = time_graph(torch, g, steps) / (steps * n_copies)
+            weights = (Hq + Hkv) * keep * K
+            row = {"us": round(sec * 1e6, 2), "tokens_per_s": round(M / sec, 1)}
+            if M <= 16:
+                gbs = BYTES_PER_WEIGHT * weights / sec / 1e9
+                row.update({"GBps": round(gbs, 1), "frac_hbm_%s" % which: round(gbs / hbm, 3)})
+            else:
+                tfl = 2.0 * M * weights / sec / 1e12
+                row.update({"TFLOPs": round(tfl, 1), "frac_bf16_%s" % which: round(tfl / tf, 3)})
+            rows["d%d" % keep] = row
+        out["llama_qk_rope_M%d" % M] = rows
     return out
 
 

@@ -267,6 +267,18 @@ __device__ inline void store_tile(const Params& p, const TileFam& f, const TileP
   }
 }
 
+// Blocks that share the R left-over tiles of a k-part with Cq chunks per tile.  Cutting the left-over
+// units into n_rp equal ranges (stream-K) balances the bytes but every tile then ends with a hand-over
+// between blocks (park, arrival count, reduction by the last block: about the time of three chunks);
+// when that costs more than it saves, the left-over tiles are given whole to R blocks instead.
+__host__ __device__ inline long tail_blocks(long n_rp, long R, long Cq) {
+  const long Ut = R * Cq;
+  if (Ut == 0) return 1;
+  const bool split = R * Cq / n_rp + 3 < Cq;
+  const long Bt = split ? n_rp : R;
+  return Bt < Ut ? Bt : Ut;
+}
+
 // ---------------------------------------------------------------------------------------- work split
 // Units of one block of k-part `kp`: `base` whole tiles (all chunks) and a contiguous range of the
 // chunk-fastest unit sequence of the R tiles that are left over after every block took its share.
@@ -284,7 +296,7 @@ __device__ inline Work block_work(const DecodeCfg& c, int Ck, int rp) {
   const int base = c.tiles_total / c.n_rp;
   const int R = c.tiles_total - base * c.n_rp;
   const long Ut = (long)R * Ck;
-  const long Bt = (long)c.n_rp < Ut ? (long)c.n_rp : Ut;      // blocks that get tail units
+  const long Bt = tail_blocks(c.n_rp, R, Ck);                 // blocks that get tail units
   w.n1 = base * Ck;
   w.tile1 = rp * base;
   w.tail_tile0 = c.n_rp * base;
@@ -506,7 +518,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
               const int Gq = min(c.gp, c.g_total - q2 * c.gp);
               const long Cq = (Gq + CG - 1) / CG;
               const long Ut = (long)R * Cq;
-              const long Bt = (long)c.n_rp < Ut ? (long)c.n_rp : Ut;
+              const long Bt = tail_blocks(c.n_rp, R, Cq);
               const long t0 = (long)(tile - wk.tail_tile0) * Cq;
               first = owner_of(t0, Bt, Ut);
               n_here = owner_of(t0 + Cq - 1, Bt, Ut) - first + 1;
@@ -580,8 +592,10 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     const int row_units = c.xrow / 16;
     uint4* xs = reinterpret_cast<uint4*>(smem + c.off_x);
     float2* xg = reinterpret_cast<float2*>(smem + c.off_xg);
-    for (int i = ctid; i < Gk * 8 * MT; i += CTH) xg[i] = make_float2(0.f, 0.f);
-    if (!consumer_sync()) return;
+    if (NT == 0) {          // (the integer path writes every entry it later reads)
+      for (int i = ctid; i < Gk * 8 * MT; i += CTH) xg[i] = make_float2(0.f, 0.f);
+      if (!consumer_sync()) return;
+    }
     if (NT > 0) {
       // Integer path.  Per (batch row, group) the activations become 16-bit fixed point, x_i = rint(x * 2^e)
       // with 2^e the largest power of two that keeps the group's maximum at or below 32639 (so that the high
@@ -1080,7 +1094,7 @@ int slots_needed(int tiles, int g_total, int gp, int n_rp) {
     const long Cq = (Gq + CG - 1) / CG;
     const long Ut = R * Cq;
     if (Ut == 0) { total += 1; continue; }
-    const long Bt = (long)n_rp < Ut ? (long)n_rp : Ut;
+    const long Bt = tail_blocks(n_rp, R, Cq);
     const long per_block = Ut / Bt;           // >= 1
     total += (int)((Cq + per_block - 1) / per_block) + 1;
   }
