@@ -343,12 +343,11 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   const uint32_t sbase = (raw + 1023u) & ~1023u;
   unsigned char* smem = smem_raw + (sbase - raw);
   const int S = c.stages;
-  // barriers: full[S], empty[S], consumer barrier, epilogue barrier, partials full[2] / free[2]; then flags
+  // barriers: full[S], empty[S], consumer barrier, (spare), partials full[2] / free[2]; then the abort flag
   const uint32_t bar_full = sbase + c.off_bar, bar_empty = bar_full + 8 * MAX_STAGES;
   const uint32_t bar_cons = bar_full + 16 * MAX_STAGES, bar_epi = bar_cons + 8;
   const uint32_t bar_pfull = bar_cons + 16, bar_pfree = bar_cons + 32;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + c.off_bar + 16 * MAX_STAGES + 48);
-  volatile int* last_flag = reinterpret_cast<volatile int*>(smem + c.off_bar + 16 * MAX_STAGES + 52);
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) {
@@ -359,7 +358,6 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     mbar_init(bar_epi, EW);
     for (int b = 0; b < 2; ++b) { mbar_init(bar_pfull + 8 * b, CW); mbar_init(bar_pfree + 8 * b, EW); }
     *abort_flag = 0;
-    *last_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -471,16 +469,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   // every (row slot, batch row), then stores the tile, or parks the sum for the block that finishes it.
   if (warp > CW) {
     const int etid = tid - (CW + 1) * 32;
-    uint32_t epi_parity = 0;
     auto give_up = [&]() { if (lane == 0) atomicExch(c.status, UNIQL_ERR_TIMEOUT); };
-    auto epi_sync = [&]() -> bool {
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_epi);
-      const bool ok = mbar_wait(bar_epi, epi_parity, abort_flag);
-      epi_parity ^= 1;
-      if (!ok) give_up();
-      return ok;
-    };
     UnitIter ui;
     ui.start(wk);
     TilePos q = tile_pos(c, p, ui.tile);
@@ -530,28 +519,39 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         if (total == 1) {
           store_tile<T>(p, f, q, etid, local_sum);
         } else {
+          // Hand-over without block-wide barriers: every epilogue warp owns the same output items in all
+          // blocks (item i belongs to warp (i / 32) % EW), parks the sums of its items, counts its own
+          // arrival, and the last warp of its kind to arrive finishes its items.
           float* tile_ws = c.partials + (size_t)tile * c.max_slots * RM;
           float* mine = tile_ws + (size_t)my_slot * RM;
-          for (int j = etid; j < RM; j += ETH) __stcg(mine + j, local_sum(j & (RB - 1), j / RB));
-          if (!epi_sync()) return;
-          if (etid == 0) {
-            __threadfence();                           // orders the whole group's parked sums (observed through
-                                                       // the barrier) before the arrival count
-            const int arrived = atomicAdd(&c.counters[tile], 1);
-            *last_flag = arrived == total - 1;
+          const bool rope = p.job[f.job].rope.enabled != 0;
+          if (rope) {
+            for (int j = etid; j < (RB / 2) * p.M; j += ETH) {
+              const int pp = j & (RB / 2 - 1), m = j / (RB / 2);
+              __stcg(mine + m * RB + pp, local_sum(pp, m));
+              __stcg(mine + m * RB + pp + RB / 2, local_sum(pp + RB / 2, m));
+            }
+          } else {
+            for (int j = etid; j < RM; j += ETH) __stcg(mine + j, local_sum(j & (RB - 1), j / RB));
+          }
+          __threadfence();
+          __syncwarp();
+          int last_w = 0;
+          int* cnt = c.counters + tile * EW + (warp - CW - 1);
+          if (lane == 0) {
+            last_w = atomicAdd(cnt, 1) == total - 1;
             __threadfence();
           }
-          if (!epi_sync()) return;
-          if (*last_flag) {
+          last_w = __shfl_sync(0xffffffffu, last_w, 0);
+          if (last_w) {
             auto global_sum = [&](int slot, int m) -> float {
               float v = 0.f;
               for (int s2 = 0; s2 < total; ++s2) v += __ldcg(tile_ws + (size_t)s2 * RM + m * RB + slot);
               return v;
             };
             store_tile<T>(p, f, q, etid, global_sum);
-            if (etid == 0) c.counters[tile] = 0;       // ready for the next call
+            if (lane == 0) *cnt = 0;                   // ready for the next call
           }
-          if (!epi_sync()) return;                     // last_flag may be rewritten only after everyone read it
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_pfree + 8 * buf);
@@ -592,6 +592,12 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     const int row_units = c.xrow / 16;
     uint4* xs = reinterpret_cast<uint4*>(smem + c.off_x);
     float2* xg = reinterpret_cast<float2*>(smem + c.off_xg);
+    // Groups this block needs: all visited groups, or, for a block that only holds a short run of left-over
+    // units (K-heavy matrices), the chunks of that run.
+    int ch0 = 0, n_ch = wk.Ck;
+    if (wk.n1 == 0 && wk.te - wk.tb < wk.Ck) { ch0 = wk.tb % wk.Ck; n_ch = wk.te - wk.tb; }
+    const int Gn = n_ch * CG;
+    auto needed_group = [&](int gn) { int ch = ch0 + gn / CG; if (ch >= wk.Ck) ch -= wk.Ck; return ch * CG + (gn & (CG - 1)); };
     if (NT == 0) {          // (the integer path writes every entry it later reads)
       for (int i = ctid; i < Gk * 8 * MT; i += CTH) xg[i] = make_float2(0.f, 0.f);
       if (!consumer_sync()) return;
@@ -605,7 +611,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       // batch rows (columns 2m and 2m+1 of the int8 MMA), in the order the nibbles leave a weight word:
       // even codes in the first register of a word's pair, odd codes in the second.
       const int start = p.imap.fam[0].start, keep = p.imap.fam[0].keep;
-      const int n_units = Gk * p.M * 16;
+      const int n_units = Gn * p.M * 16;
       unsigned char* xb = smem + c.off_x;
       constexpr int UN = 4;
       for (int u0 = ctid; u0 < ((n_units + 31) & ~31); u0 += CTH * UN) {
@@ -615,18 +621,18 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           const int u = u0 + q4 * CTH;
           in[q4] = make_uint4(0, 0, 0, 0);
           if (u < n_units) {
-            const int pair = u >> 4, m = pair / Gk, lv = pair - m * Gk;
+            const int pair = u >> 4, m = pair / Gn, lv = needed_group(pair - m * Gn);
             const int t0 = (sg_lo + lv) * kGroup + 8 * (u & 15) - start;
-            if (t0 >= 0 && t0 < keep) in[q4] = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * p.ldx + t0));
+            if (lv < Gk && t0 >= 0 && t0 < keep) in[q4] = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * p.ldx + t0));
           }
         }
 #pragma unroll
         for (int q4 = 0; q4 < UN; ++q4) {
           const int u = u0 + q4 * CTH;
           if (u >= ((n_units + 31) & ~31)) break;                  // warp-uniform
-          const bool in_range = u < n_units;
-          const int u16 = u & 15, pair = in_range ? u >> 4 : 0;
-          const int m = pair / Gk, lv = pair - m * Gk;
+          const int u16 = u & 15, pair = u < n_units ? u >> 4 : 0;
+          const int m = pair / Gn, lv = needed_group(pair - m * Gn);
+          const bool in_range = u < n_units && lv < Gk;
           const __half2* h2 = reinterpret_cast<const __half2*>(&in[q4]);
           float f[8];
           float amax = 0.f;
@@ -668,7 +674,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       }
     } else if (c.x_vec) {
       const int start = p.imap.fam[0].start, keep = p.imap.fam[0].keep;
-      const int n_units = Gk * p.M * 16;
+      const int n_units = Gn * p.M * 16;
       constexpr int UN = 4;                                        // loads in flight per thread
       for (int u0 = ctid; u0 < ((n_units + 31) & ~31); u0 += CTH * UN) {   // whole warps stay in the shuffles
         uint4 in[UN];
@@ -677,18 +683,18 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           const int u = u0 + q4 * CTH;
           in[q4] = make_uint4(0, 0, 0, 0);
           if (u < n_units) {
-            const int pair = u >> 4, m = pair / Gk, lv = pair - m * Gk;
+            const int pair = u >> 4, m = pair / Gn, lv = needed_group(pair - m * Gn);
             const int t0 = (sg_lo + lv) * kGroup + 8 * (u & 15) - start;
-            if (t0 >= 0 && t0 < keep) in[q4] = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * p.ldx + t0));
+            if (lv < Gk && t0 >= 0 && t0 < keep) in[q4] = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * p.ldx + t0));
           }
         }
 #pragma unroll
         for (int q4 = 0; q4 < UN; ++q4) {
           const int u = u0 + q4 * CTH;
           if (u >= ((n_units + 31) & ~31)) break;                  // warp-uniform
-          const bool in_range = u < n_units;
-          const int u16 = u & 15, pair = in_range ? u >> 4 : 0;
-          const int m = pair / Gk, lv = pair - m * Gk;
+          const int u16 = u & 15, pair = u < n_units ? u >> 4 : 0;
+          const int m = pair / Gn, lv = needed_group(pair - m * Gn);
+          const bool in_range = u < n_units && lv < Gk;
           uint4 o;
           o.x = __byte_perm(in[q4].x, in[q4].z, 0x5410); o.y = __byte_perm(in[q4].x, in[q4].z, 0x7632);
           o.z = __byte_perm(in[q4].y, in[q4].w, 0x5410); o.w = __byte_perm(in[q4].y, in[q4].w, 0x7632);
@@ -1249,7 +1255,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   }
   c.n_tf = n_tf;
   c.tiles_total = tiles;
-  if (tiles < 1 || tiles > kCounterInts) return UNIQL_ERR_UNSUPPORTED;
+  if (tiles < 1 || tiles * EW > kCounterInts) return UNIQL_ERR_UNSUPPORTED;
 
   // integer path: fp16 activations staged with 128-bit loads (a leading input block); UNIQL_DECODE_I8=0: fp16 MMAs
   const bool i8 = c.x_vec && env_int("UNIQL_DECODE_I8", 1) != 0;
