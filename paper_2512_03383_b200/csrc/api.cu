@@ -2,6 +2,7 @@
 // and the dispatch by M between the decode, prefill and generic kernels.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <mutex>
@@ -93,6 +94,25 @@ int dispatch(const Params& p, void* workspace, size_t ws_bytes, void* stream) {
     if (!cfg.workspace) {
       int rc = lib_workspace(&cfg.workspace, &cfg.ws_bytes, cfg.stream);
       if (rc != UNIQL_OK) return rc;
+    }
+    // Batches of 9..16: the staged activations of 16 rows do not fit beside the stage ring, which would
+    // force the input channels to be split over two groups of blocks and every tile through a hand-over.
+    // Two launches over half the batch each re-read the weights but run more than twice as fast
+    // (UNIQL_DECODE_SPLIT_BATCH=0: one launch).
+    static const bool split_batch = []{ const char* e = getenv("UNIQL_DECODE_SPLIT_BATCH"); return !(e && e[0] == '0'); }();
+    if (p.M > 8 && split_batch) {
+      const int m1 = (p.M + 1) / 2;
+      const size_t esz = 2;                               // fp16 / bf16
+      Params a = p, b = p;
+      a.M = m1;
+      b.M = p.M - m1;
+      b.x = reinterpret_cast<const unsigned char*>(p.x) + (size_t)m1 * p.ldx * esz;
+      b.pos = p.pos ? p.pos + m1 : nullptr;
+      for (int j = 0; j < p.n_jobs; ++j)
+        b.job[j].y = reinterpret_cast<unsigned char*>(p.job[j].y) + (size_t)m1 * p.job[j].ldy * esz;
+      int rc = launch_decode(a, cfg);
+      if (rc != UNIQL_OK) return rc;
+      return launch_decode(b, cfg);
     }
     return launch_decode(p, cfg);
   }
