@@ -206,6 +206,30 @@ int uniql_qk_rope_proj(const void* x, int ldx, int dt, const uint8_t* wq, const 
                        double theta, const double* inv_freq, void* q_out, int ldq, void* k_out,
                        int ldk, void* workspace, size_t ws_bytes, void* stream);
 
+/* ---- SwiGLU MLP block at decode:  y = ( silu(x Wg^T) * (x Wu^T) ) Wd^T ----
+ * (Section 3.1, the MLP block f_MLP(X) = (sigma(X W_g) . X W_u) W_d with sigma(t) = t / (1 + exp(-t)),
+ * the gate of the Llama / Qwen blocks the paper compresses; Section 3.4: after sorting, pruning the
+ * intermediate dimension keeps the leading k_int channels.)
+ * Stored matrices: Wg, Wu [inter][hidden] and Wd [hidden][inter] packed as for uniql_qlinear, scales /
+ * zeros [rows][cols/128] fp16.  Used: rows [0, k_int) of Wg and Wu, columns [0, k_int) of Wd.
+ *   x [M][ldx] fp16 (hidden columns),  h [M][ldh] fp16 (k_int columns: the gated activations, rounded to
+ *   fp16 once; written by the call, valid on return),  y [M][ldy] fp16 (hidden columns).
+ * fuse = 1: ONE launch (gate|up tiles, a grid-wide barrier with a bounded wait, down tiles; weights of the
+ *   down projection are prefetched across the barrier); UNIQL_ERR_UNSUPPORTED when M > 8 or the staged
+ *   activations do not fit in shared memory.  fuse = 0: two launches (gate|up with the gated product as
+ *   epilogue, then down).  fuse = -1: the faster of the two on this hardware (two launches: the boundary
+ *   between dependent launches costs less than the grid-wide barrier).  M in 9..16 runs as two halves.
+ * Limits: fp16; 1 <= M <= 16; hidden, inter multiples of 256; k_int a multiple of 8; ldx, ldh multiples of 8;
+ * x and h 16-byte aligned.  Other shapes: UNIQL_ERR_UNSUPPORTED (compose uniql_qlinear_multi calls).
+ * workspace: NULL (library buffer) or uniql_mlp_workspace_bytes(M, hidden, inter) bytes, zeroed once by
+ * uniql_workspace_init; after a UNIQL_ERR_TIMEOUT status it must be zeroed again before reuse. */
+size_t uniql_mlp_workspace_bytes(int M, int hidden, int inter);
+int uniql_mlp_swiglu_decode(const void* x, int ldx, const uint8_t* wg, const void* sg, const void* zg,
+                            const uint8_t* wu, const void* su, const void* zu, const uint8_t* wd,
+                            const void* sd, const void* zd, int M, int hidden, int inter, int k_int,
+                            void* h, int ldh, void* y, int ldy, int fuse, void* workspace,
+                            size_t ws_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

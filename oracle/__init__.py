@@ -51,6 +51,7 @@ def _load():
                                               vp, i64, vp, i64, vp, i64, vp]
         _lib.uniql_oracle_rope.argtypes = [vp, i64, i64, i64, i64, i64, vp, vp,
                                            ctypes.c_double, vp, vp]
+        _lib.uniql_oracle_swiglu.argtypes = [vp, vp, i64, vp]
     return _lib
 
 
@@ -174,3 +175,33 @@ def qk_halfhead_map(n_heads: int, head_dim: int, head_keep: int) -> list:
     head_keep dims per head: the leading head_keep/2 rows of every half head
     (Algorithm 2: idx_sym = [argsort, D_hd/2 + argsort], so pairs stay intact)."""
     return [(0, head_dim // 2, head_keep // 2, 2 * n_heads)]
+
+
+def swiglu(g, u) -> np.ndarray:
+    """silu(g) * u element by element in fp64 (MLP block of Section 3.1, SiLU gate)."""
+    gd, ud = _f64(g), _f64(u)
+    assert gd.shape == ud.shape
+    out = np.empty_like(gd)
+    rc = _load().uniql_oracle_swiglu(_p(gd), _p(ud), gd.size, _p(out))
+    if rc:
+        raise ValueError("swiglu: bad argument (rc=%d)" % rc)
+    return out
+
+
+def mlp_swiglu(x, wg, sg, zg, wu, su, zu, wd, sd, zd, k_int: int,
+               out_rows: Optional[Sequence[int]] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """The pruned SwiGLU MLP block, one call of the oracle per step:
+    g = x Wg[:k_int]^T, u = x Wu[:k_int]^T, h = silu(g) * u, y = fp16(h) Wd[:, :k_int]^T.
+    The gated activations are a stored fp16 tensor of the model, so they are rounded to
+    fp16 (a type conversion, no arithmetic) before the down projection.
+    Returns (h in fp64 before that rounding, y in fp64); `out_rows` samples output channels of y."""
+    hidden = 2 * np.asarray(wg).shape[1]
+    O, I = leading(k_int), leading(hidden)
+    g = qlinear(x, wg, sg, zg, O, I)
+    u = qlinear(x, wu, su, zu, O, I)
+    h = swiglu(g, u)
+    h16 = h.astype(np.float16).astype(np.float64)
+    n_out = np.asarray(wd).shape[0]
+    Od = leading(n_out) if out_rows is None else np.ascontiguousarray(out_rows, dtype=np.int32)
+    y = qlinear(h16, wd, sd, zd, Od, leading(k_int))
+    return h, y

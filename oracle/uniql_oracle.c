@@ -148,3 +148,14 @@ int uniql_oracle_rope(const double* in, int64_t R, int64_t n_heads, int64_t n_kv
       }
   return 0;
 }
+
+/* ---- gated activation of the MLP block -------------------------------------------------
+ * Section 3.1 writes the MLP block as f_MLP(X) = (sigma(X W_g) (.) X W_u) W_d.  Reading taken
+ * here: sigma is the SiLU gate of the Llama / Qwen blocks the paper compresses,
+ * sigma(t) = t * logistic(t) = t / (1 + exp(-t)), applied element by element.
+ * g, u, h: n fp64 values each;  h[i] = sigma(g[i]) * u[i]. */
+int uniql_oracle_swiglu(const double* g, const double* u, int64_t n, double* h) {
+  if (n < 0) return 1;
+  for (int64_t i = 0; i < n; ++i) h[i] = g[i] / (1.0 + exp(-g[i])) * u[i];
+  return 0;
+}

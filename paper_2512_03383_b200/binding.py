@@ -61,6 +61,10 @@ _lib.uniql_workspace_bytes.argtypes = [_i, _i, _i]
 _lib.uniql_workspace_init.argtypes = [_vp, _sz, _vp]
 _lib.uniql_workspace_status.argtypes = [_vp, ctypes.POINTER(_i)]
 _lib.uniql_qlinear.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp]
+_lib.uniql_mlp_workspace_bytes.restype = _sz
+_lib.uniql_mlp_workspace_bytes.argtypes = [_i, _i, _i]
+_lib.uniql_mlp_swiglu_decode.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i,
+                                         _vp, _i, _vp, _i, _i, _vp, _sz, _vp]
 _lib.uniql_qlinear_noalloc.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp]
 _lib.uniql_qlinear_ex.argtypes = [_vp, _i, _i, _vp, _vp, _vp, _vp, _i, _i, _i, ctypes.POINTER(_ChanMap), _i,
                                   ctypes.POINTER(_ChanMap), _i, _vp, _i, _vp, _sz, _vp]
@@ -69,7 +73,8 @@ _lib.uniql_qlinear_multi.argtypes = [_vp, _i, _i, _i, _i, ctypes.POINTER(_ChanMa
 _lib.uniql_qk_rope_proj.argtypes = [_vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i,
                                     _vp, _vp, _d, ctypes.POINTER(_d), _vp, _i, _vp, _i, _vp, _sz, _vp]
 for _n in ("uniql_set_path", "uniql_pack_u4", "uniql_unpack_u4", "uniql_dequant", "uniql_workspace_init",
-           "uniql_workspace_status", "uniql_qlinear", "uniql_qlinear_noalloc", "uniql_qlinear_ex", "uniql_qlinear_multi", "uniql_qk_rope_proj"):
+           "uniql_workspace_status", "uniql_qlinear", "uniql_qlinear_noalloc", "uniql_qlinear_ex", "uniql_qlinear_multi", "uniql_qk_rope_proj",
+           "uniql_mlp_swiglu_decode"):
     getattr(_lib, _n).restype = _i
 
 
@@ -213,3 +218,18 @@ def qk_rope_proj(x, ldx, wq, sq, zq, wk, sk, zk, bq, bk, M, K, n_q_heads, n_kv_h
                                    _ptr(bq), _ptr(bk), M, K, n_q_heads, n_kv_heads, head_dim, head_keep,
                                    _ptr(retained_idx), _ptr(pos), float(theta), f, _ptr(q_out), ldq, _ptr(k_out),
                                    ldk, _ptr(workspace), ws_bytes, _stream(stream)), "uniql_qk_rope_proj")
+
+
+def mlp_workspace_bytes(M: int, hidden: int, inter: int) -> int:
+    return int(_lib.uniql_mlp_workspace_bytes(M, hidden, inter))
+
+
+def mlp_swiglu_decode(x, ldx, wg, sg, zg, wu, su, zu, wd, sd, zd, M, hidden, inter, k_int, h, ldh, y, ldy,
+                      fuse=-1, workspace=None, stream=None) -> None:
+    if x.dtype != torch.float16 or h.dtype != torch.float16 or y.dtype != torch.float16:
+        raise TypeError("uniql_mlp_swiglu_decode computes in fp16")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.uniql_mlp_swiglu_decode(_ptr(x), ldx, _ptr(wg), _ptr(sg), _ptr(zg), _ptr(wu), _ptr(su), _ptr(zu),
+                                        _ptr(wd), _ptr(sd), _ptr(zd), M, hidden, inter, k_int, _ptr(h), ldh,
+                                        _ptr(y), ldy, int(fuse), _ptr(workspace), ws_bytes, _stream(stream)),
+           "uniql_mlp_swiglu_decode")

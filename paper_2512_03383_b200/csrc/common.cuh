@@ -140,6 +140,21 @@ int decode_supported(const Params& p);
 size_t decode_workspace_bytes(int M, int K, int N_total);
 int decode_status_offset();   // byte offset of the device status word inside a workspace
 size_t decode_workspace_header_bytes();   // counters + status word: the part that must start at zero
+// SwiGLU MLP at decode (Section 3.1: y = (silu(x Wg^T) * (x Wu^T)) Wd^T with the trailing `inter - k_int`
+// sorted intermediate channels pruned): leading k_int rows of Wg, Wu and leading k_int columns of Wd.
+struct MlpDecode {
+  const void* x; int ldx;      // [M][hidden] fp16
+  int M, hidden, inter, k_int;
+  const uint8_t *wg, *wu, *wd; // packed [inter][hidden/2], [inter][hidden/2], [hidden][inter/2]
+  const __half *sg, *zg, *su, *zu, *sd, *zd;
+  void* h; int ldh;            // [M][k_int] fp16: the gated activations (written, then read)
+  void* y; int ldy;            // [M][hidden] fp16
+};
+// fuse != 0: both products in one launch (UNIQL_ERR_UNSUPPORTED when the shapes do not allow it);
+// fuse == 0: two launches.
+int launch_mlp_decode(const MlpDecode& d, int fuse, const LaunchCfg& cfg);
+int mlp_decode_supported(const MlpDecode& d);
+size_t mlp_decode_workspace_bytes(int M, int hidden, int inter);
 int launch_prefill(const Params& p, const LaunchCfg& cfg);
 int prefill_supported(const Params& p);
 size_t prefill_workspace_bytes(int M, int K);

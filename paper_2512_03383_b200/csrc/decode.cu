@@ -56,10 +56,12 @@ constexpr int STAGE_BYTES = STAGE_W + 2 * STAGE_SZ;   // a multiple of 1024 (swi
 constexpr int MAX_STAGES = 6;
 constexpr int kCounterInts = 1 << 16;   // arrival counters (one per tile) at the head of the workspace
 constexpr int kStatusOff = kCounterInts * 4;   // status word right after the counters
+constexpr int kGridSyncOff = kStatusOff + 64;   // the two counters of the barrier between phases
 constexpr int kWsHeader = kStatusOff + 256;
 constexpr int kMaxKParts = 16;
 constexpr int kSmemMax = 227 * 1024;
 constexpr int kWaitLimit = 1 << 18;
+constexpr int kGridWaitLimit = 1 << 21;   // polls (40 ns apart) of the barrier between the phases of a fused launch
 constexpr int BAR_BYTES = 256;
 constexpr int kMaxTF = 8;               // (job, family) pairs of one launch
 
@@ -73,16 +75,33 @@ struct TileFam {
   int job;
   int start, period;     // stored row of block h, row r: start + h*period + r   (rope: h*head_dim + r)
   int out_base;          // compact output column of block 0, row 0
+  int mode;              // kPlain, kRope (32 rotation pairs per tile) or kSwiglu (32 gate rows + 32 up rows)
+  int job2;              // kSwiglu: the job of the up projection (`job` is the gate projection)
+};
+enum { kPlain = 0, kRope = 1, kSwiglu = 2 };
+__host__ __device__ inline int tile_rows(const TileFam& f) { return f.mode == kPlain ? RB : RB / 2; }
+
+// One matrix product of a launch.  A plain launch has one phase; the fused SwiGLU MLP has two (gate|up,
+// then down on the activations the first phase wrote), separated by a grid-wide barrier.
+struct Phase {
+  const void* x;         // activations [M][ldx]
+  long long ldx;
+  int K;                 // stored input channels of the phase's matrices
+  int start, keep;       // leading input family (128-bit staging)
+  int g_total, v_first;  // visited groups and the first of them
+  int tile0, tiles;      // global tiles [tile0, tile0 + tiles)
 };
 
 struct DecodeCfg {
   CUtensorMap wmap[kMaxTF];   // packed weights of each family: (byte, row in block, block)
+  CUtensorMap wmap_up;        // kSwiglu family: the up projection (wmap[] holds the gate projection)
   TileFam tf[kMaxTF];
+  Phase ph[2];
+  int n_ph;
   int n_tf;
   int n_kp, n_rp;        // k-parts x blocks per k-part
   int gp;                // visited groups per k-part (the last part may be shorter)
-  int g_total;           // visited groups
-  int v_first;           // first visited stored group
+  int g_total;           // visited groups (largest phase)
   int gran;              // groups per scale / zero-point copy granule (2, 4 or 8)
   int stages;
   int tiles_total;
@@ -92,6 +111,7 @@ struct DecodeCfg {
   int* counters;
   float* partials;
   int* status;
+  int* grid_sync;        // two ints: epilogue warps that finished phase 0, blocks that saw all of them
 };
 
 // ---------------------------------------------------------------------------------------- PTX helpers
@@ -210,14 +230,13 @@ __device__ inline TilePos tile_pos(const DecodeCfg& c, const Params& p, int tg) 
   const TileFam& f = c.tf[q.fi];
   const int tl = tg - f.tile_begin;
   q.h = tl / f.tpb;
-  const int rows = p.job[f.job].rope.enabled ? RB / 2 : RB;
-  q.r0 = (tl - q.h * f.tpb) * rows;
+  q.r0 = (tl - q.h * f.tpb) * tile_rows(f);
   return q;
 }
 // position of the next tile (tiles are numbered block after block, family after family)
 __device__ inline void next_tile(const DecodeCfg& c, const Params& p, TilePos& q) {
   const TileFam& f = c.tf[q.fi];
-  q.r0 += p.job[f.job].rope.enabled ? RB / 2 : RB;
+  q.r0 += tile_rows(f);
   if (q.r0 >= f.keep) {
     q.r0 = 0;
     if (++q.h == f.count) { q.h = 0; ++q.fi; }
@@ -235,7 +254,18 @@ __device__ inline void store_tile(const Params& p, const TileFam& f, const TileP
   const JobDev& jb = p.job[f.job];
   const T* bias = reinterpret_cast<const T*>(jb.bias);
   T* y = reinterpret_cast<T*>(jb.y);
-  if (jb.rope.enabled) {
+  if (f.mode == kSwiglu) {
+    // slots 0..31 hold the gate rows, slots 32..63 the up rows of the same channels:
+    // h = g * sigmoid(g) * u, rounded once (MLP block of Section 3.1 with the SiLU gate)
+    for (int i = etid; i < (RB / 2) * p.M; i += ETH) {
+      const int pp = i & (RB / 2 - 1), m = i / (RB / 2);
+      const int cc = q.r0 + pp;
+      if (cc >= f.keep) continue;
+      const float gt = get(pp, m), up = get(pp + RB / 2, m);
+      const float hv = gt / (1.f + __expf(-gt)) * up;
+      y[(size_t)m * jb.ldy + f.out_base + cc] = DT<T>::from_f(hv);
+    }
+  } else if (jb.rope.enabled) {
     const int half = jb.rope.head_keep >> 1;
     for (int i = etid; i < (RB / 2) * p.M; i += ETH) {
       const int pp = i & (RB / 2 - 1), m = i / (RB / 2);
@@ -290,20 +320,37 @@ struct Work {
   int tb, te;        // tail unit range [tb, te) in the left-over sequence
   int n_units;
 };
-__device__ inline Work block_work(const DecodeCfg& c, int Ck, int rp) {
+__device__ inline Work block_work(int n_rp, int tile0, int tiles, int Ck, int rp) {
   Work w;
   w.Ck = Ck;
-  const int base = c.tiles_total / c.n_rp;
-  const int R = c.tiles_total - base * c.n_rp;
+  const int base = tiles / n_rp;
+  const int R = tiles - base * n_rp;
   const long Ut = (long)R * Ck;
-  const long Bt = tail_blocks(c.n_rp, R, Ck);                 // blocks that get tail units
+  const long Bt = tail_blocks(n_rp, R, Ck);                   // blocks that get tail units
   w.n1 = base * Ck;
-  w.tile1 = rp * base;
-  w.tail_tile0 = c.n_rp * base;
+  w.tile1 = tile0 + rp * base;
+  w.tail_tile0 = tile0 + n_rp * base;
   w.tb = w.te = 0;
   if (rp < Bt) { w.tb = (int)(Ut * rp / Bt); w.te = (int)(Ut * (rp + 1) / Bt); }
   w.n_units = w.n1 + (w.te - w.tb);
   return w;
+}
+// What block (kp, rp) does in one phase.
+struct PhaseCtx {
+  int Gk;            // groups of this k-part
+  int sg_lo;         // its first stored group
+  int G;             // groups per stored row
+  Work wk;
+};
+__device__ inline PhaseCtx phase_ctx(const DecodeCfg& c, int ph, int kp, int rp) {
+  const Phase& P = c.ph[ph];
+  PhaseCtx k;
+  const int v_lo = kp * c.gp;                                   // first visit index of this k-part
+  k.Gk = min(c.gp, P.g_total - v_lo);
+  k.sg_lo = P.v_first + v_lo;
+  k.G = P.K / kGroup;
+  k.wk = block_work(c.n_rp, P.tile0, P.tiles, (k.Gk + CG - 1) / CG, rp);
+  return k;
 }
 // (tile, chunk) of block-local unit i, walked in order.  The share of the left-over tiles comes first:
 // its hand-over between blocks (parked sums, arrival count, final reduction by the last block) then
@@ -332,7 +379,8 @@ struct UnitIter {
 // ---------------------------------------------------------------------------------------- kernel
 // NT == 0: fp16 tensor-core path (MT batch tiles of 8, ONECOL: batch 1).  NT > 0: integer path, NT column
 // tiles of the int8 MMA, each holding the high and the low byte of four batch rows.
-template <int MT, bool ONECOL, int NT>
+// NPH: phases (2: the fused SwiGLU MLP, integer path only).
+template <int MT, bool ONECOL, int NT, int NPH>
 __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ Params p,
                                                         const __grid_constant__ DecodeCfg c) {
   extern __shared__ unsigned char smem_raw[];
@@ -363,90 +411,99 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   __syncthreads();
 
   const int kp = blockIdx.x / c.n_rp, rp = blockIdx.x - kp * c.n_rp;
-  const int v_lo = kp * c.gp;                                   // first visit index of this k-part
-  const int Gk = min(c.gp, c.g_total - v_lo);                   // its groups
-  const int sg_lo = c.v_first + v_lo;                           // first stored group of this k-part
-  const int G = p.K / kGroup;
-  const Work wk = block_work(c, (Gk + CG - 1) / CG, rp);
   // Programmatic dependent launch: the next kernel of the stream may be set up while this one runs (its
   // blocks still need this block's resources, so they start as blocks here exit) ...
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (wk.n_units == 0) return;
+  if (NPH == 1 && phase_ctx(c, 0, kp, rp).wk.n_units == 0) return;
 
   // ======================================================================================= producer
+  // The ring runs on across phases: the weights of the next phase are fetched while the grid-wide barrier
+  // between the phases is still being crossed (weights, scales and zero-points are never produced in here).
   if (warp == CW) {
-    UnitIter ui;
-    ui.start(wk);
-    int tile_prev = -1;
-    bool jumped = true;
-    TilePos q = {0, 0, 0};
-    bool rope = false;
-    const __half* srow[2] = {nullptr, nullptr};
-    const __half* zrow[2] = {nullptr, nullptr};
     int it = 0, s = 0;
     uint32_t ring_parity = 1;      // parity of the previous use of ring position s
     bool ok = true;
-    for (; it < wk.n_units; ++it) {
-      if (it >= S) ok = mbar_wait(bar_empty + 8 * s, ring_parity, abort_flag);
-      if (!ok) break;
-      if (ui.tile != tile_prev) {
-        if (jumped) q = tile_pos(c, p, ui.tile); else next_tile(c, p, q);
-        jumped = false;
-        const TileFam& f = c.tf[q.fi];
-        const JobDev& jb = p.job[f.job];
-        rope = jb.rope.enabled != 0;
+    for (int ph = 0; ph < NPH && ok; ++ph) {
+      const PhaseCtx pc = phase_ctx(c, ph, kp, rp);
+      const Work& wk = pc.wk;
+      const int Gk = pc.Gk, sg_lo = pc.sg_lo, G = pc.G;
+      if (wk.n_units == 0) continue;
+      UnitIter ui;
+      ui.start(wk);
+      int tile_prev = -1;
+      bool jumped = true;
+      TilePos q = {0, 0, 0};
+      int mode = kPlain;
+      const __half* srow[2] = {nullptr, nullptr};
+      const __half* zrow[2] = {nullptr, nullptr};
+      for (int iu = 0; iu < wk.n_units; ++iu, ++it) {
+        if (it >= S) ok = mbar_wait(bar_empty + 8 * s, ring_parity, abort_flag);
+        if (!ok) break;
+        if (ui.tile != tile_prev) {
+          if (jumped) q = tile_pos(c, p, ui.tile); else next_tile(c, p, q);
+          jumped = false;
+          const TileFam& f = c.tf[q.fi];
+          mode = f.mode;
+#pragma unroll
+          for (int r2 = 0; r2 < 2; ++r2) {
+            const JobDev& jb = p.job[(mode == kSwiglu && r2) ? f.job2 : f.job];
+            const int slot = lane + 32 * r2;
+            int sr = -1;
+            if (mode == kRope) {
+              const int cc = q.r0 + lane;
+              if (cc < f.keep) sr = q.h * jb.rope.head_dim + r2 * (jb.rope.head_dim >> 1) + cc;
+            } else if (mode == kSwiglu) {
+              const int cc = q.r0 + lane;
+              if (cc < f.keep) sr = f.start + cc;
+            } else {
+              const int r = q.r0 + slot;
+              if (r < f.keep) sr = f.start + q.h * f.period + r;
+            }
+            srow[r2] = sr >= 0 ? jb.scales + (size_t)sr * G + sg_lo : nullptr;
+            zrow[r2] = sr >= 0 ? jb.zeros + (size_t)sr * G + sg_lo : nullptr;
+          }
+          tile_prev = ui.tile;
+        }
+        const int chunk = ui.chunk;
+        const int ng = min(CG, Gk - chunk * CG);
+        const int nb = (ng + 1) >> 1;                      // 128-byte columns with a visited group
+        const uint32_t full = bar_full + 8 * s;
+        const uint32_t st = sbase + (uint32_t)s * STAGE_BYTES;
+        if (lane == 0) mbar_expect_tx(full, (uint32_t)(nb * BOX_BYTES));
+        __syncwarp();
+        if (lane < nb) {
+          const int xb = (sg_lo + chunk * CG + 2 * lane) * 64;       // byte in the weight row
+          const uint32_t dst = st + (uint32_t)lane * BOX_BYTES;
+          if (mode == kRope) {
+            tma_box3(dst, &c.wmap[q.fi], xb, q.r0, 2 * q.h, full);
+            tma_box3(dst + (RB / 2) * 128, &c.wmap[q.fi], xb, q.r0, 2 * q.h + 1, full);
+          } else if (mode == kSwiglu) {
+            tma_box3(dst, &c.wmap[q.fi], xb, q.r0, 0, full);
+            tma_box3(dst + (RB / 2) * 128, &c.wmap_up, xb, q.r0, 0, full);
+          } else {
+            tma_box3(dst, &c.wmap[q.fi], xb, q.r0, q.h, full);
+          }
+        }
 #pragma unroll
         for (int r2 = 0; r2 < 2; ++r2) {
-          const int slot = lane + 32 * r2;
-          int sr = -1;
-          if (rope) {
-            const int cc = q.r0 + lane;
-            if (cc < f.keep) sr = q.h * jb.rope.head_dim + r2 * (jb.rope.head_dim >> 1) + cc;
-          } else {
-            const int r = q.r0 + slot;
-            if (r < f.keep) sr = f.start + q.h * f.period + r;
-          }
-          srow[r2] = sr >= 0 ? jb.scales + (size_t)sr * G + sg_lo : nullptr;
-          zrow[r2] = sr >= 0 ? jb.zeros + (size_t)sr * G + sg_lo : nullptr;
-        }
-        tile_prev = ui.tile;
-      }
-      const int chunk = ui.chunk;
-      const int ng = min(CG, Gk - chunk * CG);
-      const int nb = (ng + 1) >> 1;                      // 128-byte columns with a visited group
-      const uint32_t full = bar_full + 8 * s;
-      const uint32_t st = sbase + (uint32_t)s * STAGE_BYTES;
-      if (lane == 0) mbar_expect_tx(full, (uint32_t)(nb * BOX_BYTES));
-      __syncwarp();
-      if (lane < nb) {
-        const int xb = (sg_lo + chunk * CG + 2 * lane) * 64;       // byte in the weight row
-        const uint32_t dst = st + (uint32_t)lane * BOX_BYTES;
-        if (rope) {
-          tma_box3(dst, &c.wmap[q.fi], xb, q.r0, 2 * q.h, full);
-          tma_box3(dst + (RB / 2) * 128, &c.wmap[q.fi], xb, q.r0, 2 * q.h + 1, full);
-        } else {
-          tma_box3(dst, &c.wmap[q.fi], xb, q.r0, q.h, full);
-        }
-      }
-#pragma unroll
-      for (int r2 = 0; r2 < 2; ++r2) {
-        if (srow[r2]) {
-          const int slot = lane + 32 * r2;
-          const uint32_t sd = st + STAGE_W + slot * (CG * 2), zd = sd + STAGE_SZ;
-          const __half* sp = srow[r2] + chunk * CG;
-          const __half* zp = zrow[r2] + chunk * CG;
-          if (c.gran == 8) {
-            cp_async16(sd, sp); cp_async16(zd, zp);
-          } else if (c.gran == 4) {
-            for (int g4 = 0; g4 < ng; g4 += 4) { cp_async8(sd + g4 * 2, sp + g4); cp_async8(zd + g4 * 2, zp + g4); }
-          } else {
-            for (int g2 = 0; g2 < ng; g2 += 2) { cp_async4(sd + g2 * 2, sp + g2); cp_async4(zd + g2 * 2, zp + g2); }
+          if (srow[r2]) {
+            const int slot = lane + 32 * r2;
+            const uint32_t sd = st + STAGE_W + slot * (CG * 2), zd = sd + STAGE_SZ;
+            const __half* sp = srow[r2] + chunk * CG;
+            const __half* zp = zrow[r2] + chunk * CG;
+            if (c.gran == 8) {
+              cp_async16(sd, sp); cp_async16(zd, zp);
+            } else if (c.gran == 4) {
+              for (int g4 = 0; g4 < ng; g4 += 4) { cp_async8(sd + g4 * 2, sp + g4); cp_async8(zd + g4 * 2, zp + g4); }
+            } else {
+              for (int g2 = 0; g2 < ng; g2 += 2) { cp_async4(sd + g2 * 2, sp + g2); cp_async4(zd + g2 * 2, zp + g2); }
+            }
           }
         }
+        cp_async_arrive_noinc(full);
+        if (iu + 1 < wk.n_units && ui.advance(wk, iu + 1)) jumped = true;
+        if (++s == S) { s = 0; ring_parity ^= 1; }
       }
-      cp_async_arrive_noinc(full);
-      if (it + 1 < wk.n_units && ui.advance(wk, it + 1)) jumped = true;
-      if (++s == S) { s = 0; ring_parity ^= 1; }
     }
     if (!ok) {
       // let the copies of the stages that are still armed land before the block goes away
@@ -470,97 +527,111 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   if (warp > CW) {
     const int etid = tid - (CW + 1) * 32;
     auto give_up = [&]() { if (lane == 0) atomicExch(c.status, UNIQL_ERR_TIMEOUT); };
-    UnitIter ui;
-    ui.start(wk);
-    TilePos q = tile_pos(c, p, ui.tile);
     int tiles_done = 0;
     // ... and this kernel may have been started before its predecessor finished: outputs, workspace, bias,
     // positions and indices are touched only after the predecessor is complete (the producer warp does not
     // wait: weights, scales and zero-points are not produced by a preceding decode launch)
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    for (int i = 0; i < wk.n_units; ++i) {
-      const bool tile_end = ui.tile_end(wk, i);
-      if (tile_end) {
-        const int buf = c.part_bufs > 1 ? (tiles_done & 1) : 0;
-        const int use = c.part_bufs > 1 ? (tiles_done >> 1) : tiles_done;
-        if (!mbar_wait(bar_pfull + 8 * buf, use & 1, abort_flag)) { give_up(); return; }
-        const float* pr = part + buf * part_stride;
-        auto local_sum = [&](int slot, int m) -> float {
-          float v = 0.f;
-#pragma unroll
-          for (int q8 = 0; q8 < CG; ++q8) v += pr[q8 * RM + m * RB + slot];
-          return v;
-        };
-        const int tile = ui.tile;
-        const TileFam& f = c.tf[q.fi];
-        // how many blocks (over all k-parts) work on this tile, and which of them am I
-        int total = 0, my_slot = 0;
-        const bool tail = tile >= wk.tail_tile0;
-        if (c.n_kp == 1 && !tail) {
-          total = 1;
-        } else {
-          const int base = c.tiles_total / c.n_rp;
-          const int R = c.tiles_total - base * c.n_rp;
-          for (int q2 = 0; q2 < c.n_kp; ++q2) {
-            int n_here = 1, first = rp;                      // a whole tile: one block per k-part
-            if (tail) {
-              const int Gq = min(c.gp, c.g_total - q2 * c.gp);
-              const long Cq = (Gq + CG - 1) / CG;
-              const long Ut = (long)R * Cq;
-              const long Bt = tail_blocks(c.n_rp, R, Cq);
-              const long t0 = (long)(tile - wk.tail_tile0) * Cq;
-              first = owner_of(t0, Bt, Ut);
-              n_here = owner_of(t0 + Cq - 1, Bt, Ut) - first + 1;
-            }
-            if (q2 == kp) my_slot = total + (rp - first);
-            total += n_here;
-          }
-        }
-        if (total == 1) {
-          store_tile<T>(p, f, q, etid, local_sum);
-        } else {
-          // Hand-over without block-wide barriers: every epilogue warp owns the same output items in all
-          // blocks (item i belongs to warp (i / 32) % EW), parks the sums of its items, counts its own
-          // arrival, and the last warp of its kind to arrive finishes its items.
-          float* tile_ws = c.partials + (size_t)tile * c.max_slots * RM;
-          float* mine = tile_ws + (size_t)my_slot * RM;
-          const bool rope = p.job[f.job].rope.enabled != 0;
-          if (rope) {
-            for (int j = etid; j < (RB / 2) * p.M; j += ETH) {
-              const int pp = j & (RB / 2 - 1), m = j / (RB / 2);
-              __stcg(mine + m * RB + pp, local_sum(pp, m));
-              __stcg(mine + m * RB + pp + RB / 2, local_sum(pp + RB / 2, m));
-            }
-          } else {
-            for (int j = etid; j < RM; j += ETH) __stcg(mine + j, local_sum(j & (RB - 1), j / RB));
-          }
-          __threadfence();
-          __syncwarp();
-          int last_w = 0;
-          int* cnt = c.counters + tile * EW + (warp - CW - 1);
-          if (lane == 0) {
-            last_w = atomicAdd(cnt, 1) == total - 1;
-            __threadfence();
-          }
-          last_w = __shfl_sync(0xffffffffu, last_w, 0);
-          if (last_w) {
-            auto global_sum = [&](int slot, int m) -> float {
-              float v = 0.f;
-              for (int s2 = 0; s2 < total; ++s2) v += __ldcg(tile_ws + (size_t)s2 * RM + m * RB + slot);
-              return v;
-            };
-            store_tile<T>(p, f, q, etid, global_sum);
-            if (lane == 0) *cnt = 0;                   // ready for the next call
-          }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_pfree + 8 * buf);
-        ++tiles_done;
+    for (int ph = 0; ph < NPH; ++ph) {
+      const PhaseCtx pc = phase_ctx(c, ph, kp, rp);
+      const Work& wk = pc.wk;
+      const Phase& P = c.ph[ph];
+      UnitIter ui;
+      TilePos q = {0, 0, 0};
+      if (wk.n_units > 0) {
+        ui.start(wk);
+        q = tile_pos(c, p, ui.tile);
       }
-      if (i + 1 < wk.n_units) {
-        const int tile_before = ui.tile;
-        if (ui.advance(wk, i + 1)) q = tile_pos(c, p, ui.tile);
-        else if (ui.tile != tile_before) next_tile(c, p, q);
+      for (int i = 0; i < wk.n_units; ++i) {
+        const bool tile_end = ui.tile_end(wk, i);
+        if (tile_end) {
+          const int buf = c.part_bufs > 1 ? (tiles_done & 1) : 0;
+          const int use = c.part_bufs > 1 ? (tiles_done >> 1) : tiles_done;
+          if (!mbar_wait(bar_pfull + 8 * buf, use & 1, abort_flag)) { give_up(); return; }
+          const float* pr = part + buf * part_stride;
+          auto local_sum = [&](int slot, int m) -> float {
+            float v = 0.f;
+#pragma unroll
+            for (int q8 = 0; q8 < CG; ++q8) v += pr[q8 * RM + m * RB + slot];
+            return v;
+          };
+          const int tile = ui.tile;
+          const TileFam& f = c.tf[q.fi];
+          // how many blocks (over all k-parts) work on this tile, and which of them am I
+          int total = 0, my_slot = 0;
+          const bool tail = tile >= wk.tail_tile0;
+          if (c.n_kp == 1 && !tail) {
+            total = 1;
+          } else {
+            const int base = P.tiles / c.n_rp;
+            const int R = P.tiles - base * c.n_rp;
+            for (int q2 = 0; q2 < c.n_kp; ++q2) {
+              int n_here = 1, first = rp;                      // a whole tile: one block per k-part
+              if (tail) {
+                const int Gq = min(c.gp, P.g_total - q2 * c.gp);
+                const long Cq = (Gq + CG - 1) / CG;
+                const long Ut = (long)R * Cq;
+                const long Bt = tail_blocks(c.n_rp, R, Cq);
+                const long t0 = (long)(tile - wk.tail_tile0) * Cq;
+                first = owner_of(t0, Bt, Ut);
+                n_here = owner_of(t0 + Cq - 1, Bt, Ut) - first + 1;
+              }
+              if (q2 == kp) my_slot = total + (rp - first);
+              total += n_here;
+            }
+          }
+          if (total == 1) {
+            store_tile<T>(p, f, q, etid, local_sum);
+          } else {
+            // Hand-over without block-wide barriers: every epilogue warp owns the same output items in all
+            // blocks (item i belongs to warp (i / 32) % EW), parks the sums of its items, counts its own
+            // arrival, and the last warp of its kind to arrive finishes its items.
+            float* tile_ws = c.partials + (size_t)tile * c.max_slots * RM;
+            float* mine = tile_ws + (size_t)my_slot * RM;
+            if (f.mode != kPlain) {
+              for (int j = etid; j < (RB / 2) * p.M; j += ETH) {
+                const int pp = j & (RB / 2 - 1), m = j / (RB / 2);
+                __stcg(mine + m * RB + pp, local_sum(pp, m));
+                __stcg(mine + m * RB + pp + RB / 2, local_sum(pp + RB / 2, m));
+              }
+            } else {
+              for (int j = etid; j < RM; j += ETH) __stcg(mine + j, local_sum(j & (RB - 1), j / RB));
+            }
+            __threadfence();
+            __syncwarp();
+            int last_w = 0;
+            int* cnt = c.counters + tile * EW + (warp - CW - 1);
+            if (lane == 0) {
+              last_w = atomicAdd(cnt, 1) == total - 1;
+              __threadfence();
+            }
+            last_w = __shfl_sync(0xffffffffu, last_w, 0);
+            if (last_w) {
+              auto global_sum = [&](int slot, int m) -> float {
+                float v = 0.f;
+                for (int s2 = 0; s2 < total; ++s2) v += __ldcg(tile_ws + (size_t)s2 * RM + m * RB + slot);
+                return v;
+              };
+              store_tile<T>(p, f, q, etid, global_sum);
+              if (lane == 0) *cnt = 0;                   // ready for the next call
+            }
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_pfree + 8 * buf);
+          ++tiles_done;
+        }
+        if (i + 1 < wk.n_units) {
+          const int tile_before = ui.tile;
+          if (ui.advance(wk, i + 1)) q = tile_pos(c, p, ui.tile);
+          else if (ui.tile != tile_before) next_tile(c, p, q);
+        }
+      }
+      if (NPH > 1 && ph + 1 < NPH) {
+        // this warp's outputs of the phase (tiles it stored, sums it parked) are complete and visible:
+        // count it at the grid-wide barrier the consumers of every block wait on before the next phase
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) atomicAdd(c.grid_sync, 1);
       }
     }
     return;
@@ -586,9 +657,16 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
 
   // ---- stage activations: permuted into nibble order, zero where the channel is pruned; per group and
   //      batch row the two sums the offset / zero-point correction needs, stored negated
-  {
-    asm volatile("griddepcontrol.wait;" ::: "memory");       // the activations may come from the preceding kernel
-    const T* x = reinterpret_cast<const T*>(p.x);
+  auto stage_x = [&](int ph, const PhaseCtx& pc) -> bool {
+    const Phase& P = c.ph[ph];
+    const Work& wk = pc.wk;
+    const int Gk = pc.Gk, sg_lo = pc.sg_lo;
+    const T* x = reinterpret_cast<const T*>(P.x);
+    const long long ldx = P.ldx;
+    // activations a previous phase of this launch wrote are read past the non-coherent cache
+    auto load16 = [&](const T* ptr) -> uint4 {
+      return (NPH > 1 && ph > 0) ? __ldcg(reinterpret_cast<const uint4*>(ptr)) : __ldg(reinterpret_cast<const uint4*>(ptr));
+    };
     const int row_units = c.xrow / 16;
     uint4* xs = reinterpret_cast<uint4*>(smem + c.off_x);
     float2* xg = reinterpret_cast<float2*>(smem + c.off_xg);
@@ -600,7 +678,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     auto needed_group = [&](int gn) { int ch = ch0 + gn / CG; if (ch >= wk.Ck) ch -= wk.Ck; return ch * CG + (gn & (CG - 1)); };
     if (NT == 0) {          // (the integer path writes every entry it later reads)
       for (int i = ctid; i < Gk * 8 * MT; i += CTH) xg[i] = make_float2(0.f, 0.f);
-      if (!consumer_sync()) return;
+      if (!consumer_sync()) return false;
     }
     if (NT > 0) {
       // Integer path.  Per (batch row, group) the activations become 16-bit fixed point, x_i = rint(x * 2^e)
@@ -610,7 +688,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       // x_i = 256 * hi + lo with both bytes signed; the bytes go to two "virtual"
       // batch rows (columns 2m and 2m+1 of the int8 MMA), in the order the nibbles leave a weight word:
       // even codes in the first register of a word's pair, odd codes in the second.
-      const int start = p.imap.fam[0].start, keep = p.imap.fam[0].keep;
+      const int start = P.start, keep = P.keep;
       const int n_units = Gn * p.M * 16;
       unsigned char* xb = smem + c.off_x;
       constexpr int UN = 4;
@@ -623,7 +701,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           if (u < n_units) {
             const int pair = u >> 4, m = pair / Gn, lv = needed_group(pair - m * Gn);
             const int t0 = (sg_lo + lv) * kGroup + 8 * (u & 15) - start;
-            if (lv < Gk && t0 >= 0 && t0 < keep) in[q4] = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * p.ldx + t0));
+            if (lv < Gk && t0 >= 0 && t0 < keep) in[q4] = load16(x + (size_t)m * ldx + t0);
           }
         }
 #pragma unroll
@@ -673,7 +751,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         }
       }
     } else if (c.x_vec) {
-      const int start = p.imap.fam[0].start, keep = p.imap.fam[0].keep;
+      const int start = P.start, keep = P.keep;
       const int n_units = Gn * p.M * 16;
       constexpr int UN = 4;                                        // loads in flight per thread
       for (int u0 = ctid; u0 < ((n_units + 31) & ~31); u0 += CTH * UN) {   // whole warps stay in the shuffles
@@ -685,7 +763,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           if (u < n_units) {
             const int pair = u >> 4, m = pair / Gn, lv = needed_group(pair - m * Gn);
             const int t0 = (sg_lo + lv) * kGroup + 8 * (u & 15) - start;
-            if (lv < Gk && t0 >= 0 && t0 < keep) in[q4] = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * p.ldx + t0));
+            if (lv < Gk && t0 >= 0 && t0 < keep) in[q4] = load16(x + (size_t)m * ldx + t0);
           }
         }
 #pragma unroll
@@ -724,7 +802,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           const int i = lane + 32 * q4;
           T val = __float2half_rn(0.f);
           const int tt = map_stored_to_compact(p.imap, kbase + i);
-          if (tt >= 0) val = x[(size_t)m * p.ldx + tt];
+          if (tt >= 0) val = x[(size_t)m * ldx + tt];
           const int ccq = i >> 5, j = (i & 31) >> 3, e = i & 7;
           xh[(m * row_units + lv * 16 + j * 4 + ccq) * 8 + 2 * (e & 3) + (e >> 2)] = val;
           if (i & 1) so += __half2float(val); else se += __half2float(val);
@@ -737,8 +815,10 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         if (lane == 0) xg[lv * 8 * MT + m] = make_float2(-(se + so), -(1024.f * se + 64.f * so));
       }
     }
-    if (!consumer_sync()) return;
-  }
+    if (!consumer_sync()) return false;
+    return true;
+  };
+  asm volatile("griddepcontrol.wait;" ::: "memory");       // the activations may come from the preceding kernel
 
   if constexpr (NT > 0) {
     // ===================================================================== consumers, integer path
@@ -764,11 +844,46 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     uint4 xr8[NT][2];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) xr8[nt][0] = xr8[nt][1] = make_uint4(0, 0, 0, 0);
-    UnitIter ui;
-    ui.start(wk);
     int tiles_done = 0;
     int s = 0;
     uint32_t ring_parity = 0;
+    for (int ph = 0; ph < NPH; ++ph) {
+    const PhaseCtx pc = phase_ctx(c, ph, kp, rp);
+    const Work& wk = pc.wk;
+    const int Gk = pc.Gk;
+    if (NPH > 1 && ph > 0) {
+      // Grid-wide barrier: the activations of this phase are complete once every epilogue warp of the grid
+      // has counted itself in.  One thread polls (bounded), the consumer barrier releases the others; the
+      // last block to see the full count clears both counters for the next launch.
+      if (warp == 0 && lane == 0) {
+        const int target = (int)gridDim.x * EW;
+        bool seen = false;
+        for (int i = 0; i < kGridWaitLimit && !seen; ++i) {
+          int v;
+          asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(c.grid_sync) : "memory");
+          seen = v >= target;
+          if (!seen) {
+            if (*abort_flag) break;
+            __nanosleep(40);
+          }
+        }
+        if (seen) {
+          __threadfence();
+          if (atomicAdd(c.grid_sync + 1, 1) == (int)gridDim.x - 1) {
+            c.grid_sync[0] = 0;
+            c.grid_sync[1] = 0;
+            __threadfence();
+          }
+        } else {
+          *abort_flag = 1;
+        }
+      }
+      if (!consumer_sync()) return;
+    }
+    if (wk.n_units == 0) continue;
+    if (!stage_x(ph, pc)) return;
+    UnitIter ui;
+    ui.start(wk);
     for (int i = 0; i < wk.n_units; ++i) {
       if (!mbar_try_wait(bar_full + 8 * s, ring_parity) && !mbar_wait(bar_full + 8 * s, ring_parity, abort_flag)) {
         give_up();
@@ -859,9 +974,15 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       }
       if (i + 1 < wk.n_units) ui.advance(wk, i + 1);
     }
+    }   // phases
     return;
   }
 
+  // ===================================================================== consumers, fp16 path (one phase)
+  const PhaseCtx pc = phase_ctx(c, 0, kp, rp);
+  const Work& wk = pc.wk;
+  const int Gk = pc.Gk;
+  if (!stage_x(0, pc)) return;
   // per-lane shared-memory addresses
   uint32_t xaddr[MT];
   bool xlive[MT];
@@ -1107,9 +1228,9 @@ int slots_needed(int tiles, int g_total, int gp, int n_rp) {
   return total;
 }
 
-template <int MT, bool ONECOL, int NT>
+template <int MT, bool ONECOL, int NT, int NPH>
 int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stream) {
-  auto kern = decode_kernel<MT, ONECOL, NT>;
+  auto kern = decode_kernel<MT, ONECOL, NT, NPH>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return UNIQL_ERR_CUDA;
   cudaLaunchConfig_t lc;
@@ -1119,10 +1240,17 @@ int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stre
   lc.dynamicSmemBytes = smem;
   lc.stream = stream;
   cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  if (NPH > 1) {
+    // the blocks of a fused launch wait on one another: all of them must be resident at once
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    lc.numAttrs = 1;
+  } else {
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.numAttrs = env_int("UNIQL_PDL", 1) ? 1 : 0;
+  }
   lc.attrs = attr;
-  lc.numAttrs = env_int("UNIQL_PDL", 1) ? 1 : 0;
   if (cudaLaunchKernelEx(&lc, kern, p, c) != cudaSuccess) { cudaGetLastError(); return UNIQL_ERR_CUDA; }
   return UNIQL_OK;
 }
@@ -1216,8 +1344,8 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   memset(&c, 0, sizeof(c));
   const int G = p.K / kGroup;
   const int gran = copy_granule(G);
-  int g_total = 0;
-  visited_range(p.imap, gran, &c.v_first, &g_total);
+  int g_total = 0, v_first = 0;
+  visited_range(p.imap, gran, &v_first, &g_total);
   const int MT = p.M <= 8 ? 1 : 2;
   // 128-bit staging: one leading family, everything 8-element aligned
   c.x_vec = p.imap.n_fam == 1 && p.imap.fam[0].count == 1 && (p.imap.fam[0].start % 8) == 0 &&
@@ -1225,7 +1353,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   if (count_tile_fams(p) > kMaxTF) return UNIQL_ERR_UNSUPPORTED;
 
   // ---- tile families and their tensor maps
-  const int x_extent = (c.v_first + g_total) * 64 < p.K / 2 ? (c.v_first + g_total) * 64 : p.K / 2;
+  const int x_extent = (v_first + g_total) * 64 < p.K / 2 ? (v_first + g_total) * 64 : p.K / 2;
   int tiles = 0, n_tf = 0;
   for (int j = 0; j < p.n_jobs; ++j) {
     const JobDev& jb = p.job[j];
@@ -1233,7 +1361,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
       const int half = jb.rope.head_keep / 2;
       TileFam& f = c.tf[n_tf];
       f.tile_begin = tiles; f.tpb = (half + RB / 2 - 1) / (RB / 2); f.keep = half; f.count = jb.rope.n_heads;
-      f.job = j; f.start = 0; f.period = jb.rope.head_dim; f.out_base = 0;
+      f.job = j; f.start = 0; f.period = jb.rope.head_dim; f.out_base = 0; f.mode = kRope; f.job2 = j;
       const int rc = encode_family(&c.wmap[n_tf], jb.w, p.K, x_extent, half, 2 * jb.rope.n_heads,
                                    jb.rope.head_dim / 2, RB / 2);
       if (rc) return rc;
@@ -1244,7 +1372,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
         const Fam& a = jb.omap.fam[k];
         TileFam& f = c.tf[n_tf];
         f.tile_begin = tiles; f.tpb = (a.keep + RB - 1) / RB; f.keep = a.keep; f.count = a.count;
-        f.job = j; f.start = a.start; f.period = a.period; f.out_base = jb.omap.base[k];
+        f.job = j; f.start = a.start; f.period = a.period; f.out_base = jb.omap.base[k]; f.mode = kPlain; f.job2 = j;
         const int rc = encode_family(&c.wmap[n_tf], jb.w + (size_t)a.start * (p.K / 2), p.K, x_extent, a.keep,
                                      a.count, a.count > 1 ? a.period : a.keep, RB);
         if (rc) return rc;
@@ -1255,6 +1383,14 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   }
   c.n_tf = n_tf;
   c.tiles_total = tiles;
+  c.n_ph = 1;
+  {
+    Phase& P = c.ph[0];
+    P.x = p.x; P.ldx = p.ldx; P.K = p.K;
+    P.start = p.imap.fam[0].start; P.keep = p.imap.fam[0].keep;
+    P.g_total = g_total; P.v_first = v_first;
+    P.tile0 = 0; P.tiles = tiles;
+  }
   if (tiles < 1 || tiles * EW > kCounterInts) return UNIQL_ERR_UNSUPPORTED;
 
   // integer path: fp16 activations staged with 128-bit loads (a leading input block); UNIQL_DECODE_I8=0: fp16 MMAs
@@ -1270,13 +1406,125 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   c.counters = reinterpret_cast<int*>(ws);
   c.status = reinterpret_cast<int*>(ws + kStatusOff);
   c.partials = reinterpret_cast<float*>(ws + kWsHeader);
+  c.grid_sync = reinterpret_cast<int*>(ws + kGridSyncOff);
   if (i8) {
-    if (p.M <= 4) return launch_t<1, false, 1>(p, c, smem, cfg.stream);
-    if (p.M <= 8) return launch_t<1, false, 2>(p, c, smem, cfg.stream);
-    return launch_t<2, false, 4>(p, c, smem, cfg.stream);
+    if (p.M <= 4) return launch_t<1, false, 1, 1>(p, c, smem, cfg.stream);
+    if (p.M <= 8) return launch_t<1, false, 2, 1>(p, c, smem, cfg.stream);
+    return launch_t<2, false, 4, 1>(p, c, smem, cfg.stream);
   }
-  if (MT == 1) return p.M == 1 ? launch_t<1, true, 0>(p, c, smem, cfg.stream) : launch_t<1, false, 0>(p, c, smem, cfg.stream);
-  return launch_t<2, false, 0>(p, c, smem, cfg.stream);
+  if (MT == 1)
+    return p.M == 1 ? launch_t<1, true, 0, 1>(p, c, smem, cfg.stream) : launch_t<1, false, 0, 1>(p, c, smem, cfg.stream);
+  return launch_t<2, false, 0, 1>(p, c, smem, cfg.stream);
+}
+
+// ---------------------------------------------------------------------------------------- SwiGLU MLP
+int mlp_decode_supported(const MlpDecode& d) {
+  if (d.M < 1 || d.M > 16) return 0;
+  if (d.hidden < 2 * kGroup || d.inter < 2 * kGroup) return 0;
+  if ((d.hidden % (2 * kGroup)) != 0 || (d.inter % (2 * kGroup)) != 0) return 0;
+  if (d.k_int < 8 || d.k_int > d.inter || (d.k_int % 8) != 0) return 0;
+  if ((d.ldx % 8) != 0 || (d.ldh % 8) != 0 || d.ldx < d.hidden || d.ldh < d.k_int || d.ldy < d.hidden) return 0;
+  if ((((uintptr_t)d.x) | ((uintptr_t)d.h)) & 15) return 0;
+  const int ga = copy_granule(d.hidden / kGroup), gb = copy_granule(d.inter / kGroup);
+  if ((((uintptr_t)d.sg) | ((uintptr_t)d.zg) | ((uintptr_t)d.su) | ((uintptr_t)d.zu)) & (uintptr_t)(ga * 2 - 1)) return 0;
+  if ((((uintptr_t)d.sd) | ((uintptr_t)d.zd)) & (uintptr_t)(gb * 2 - 1)) return 0;
+  return 1;
+}
+
+size_t mlp_decode_workspace_bytes(int M, int hidden, int inter) {
+  const size_t a = decode_workspace_bytes(M, hidden, 2 * inter);
+  const size_t b = decode_workspace_bytes(M, inter, hidden);
+  return a + b;      // the fused launch numbers the tiles of both products in one sequence
+}
+
+namespace {
+
+// Phases [first, first + count) of the MLP (0: gate|up with the gated product as epilogue, 1: down) in one launch.
+int launch_mlp_phases(const MlpDecode& d, int first, int count, const LaunchCfg& cfg) {
+  Params p;
+  memset(&p, 0, sizeof(p));
+  p.x = first == 0 ? d.x : d.h;
+  p.ldx = first == 0 ? d.ldx : d.ldh;
+  p.dt = UNIQL_F16;
+  p.M = d.M;
+  p.K = first == 0 ? d.hidden : d.inter;
+  p.k_in = first == 0 ? d.hidden : d.k_int;
+  p.n_jobs = 3;
+  JobDev& jg = p.job[0];
+  JobDev& ju = p.job[1];
+  JobDev& jd = p.job[2];
+  jg.w = d.wg; jg.scales = d.sg; jg.zeros = d.zg; jg.y = d.h; jg.ldy = d.ldh; jg.N = d.inter; jg.k_out = d.k_int;
+  ju.w = d.wu; ju.scales = d.su; ju.zeros = d.zu; ju.y = d.h; ju.ldy = d.ldh; ju.N = d.inter; ju.k_out = d.k_int;
+  jd.w = d.wd; jd.scales = d.sd; jd.zeros = d.zd; jd.y = d.y; jd.ldy = d.ldy; jd.N = d.hidden; jd.k_out = d.hidden;
+
+  DecodeCfg c;
+  memset(&c, 0, sizeof(c));
+  c.x_vec = 1;
+  c.n_ph = count;
+  int tiles = 0, n_tf = 0, g_max = 0, gran = 8;
+  for (int ph = first; ph < first + count; ++ph) {
+    Phase& P = c.ph[ph - first];
+    TileFam& f = c.tf[n_tf];
+    f.tile_begin = tiles; f.count = 1; f.start = 0; f.out_base = 0;
+    P.tile0 = tiles; P.v_first = 0;
+    int rc;
+    if (ph == 0) {
+      P.x = d.x; P.ldx = d.ldx; P.K = d.hidden; P.start = 0; P.keep = d.hidden; P.g_total = d.hidden / kGroup;
+      f.mode = kSwiglu; f.job = 0; f.job2 = 1; f.keep = d.k_int; f.period = d.inter;
+      f.tpb = (d.k_int + RB / 2 - 1) / (RB / 2);
+      rc = encode_family(&c.wmap[n_tf], d.wg, d.hidden, d.hidden / 2, d.k_int, 1, d.k_int, RB / 2);
+      if (!rc) rc = encode_family(&c.wmap_up, d.wu, d.hidden, d.hidden / 2, d.k_int, 1, d.k_int, RB / 2);
+    } else {
+      P.x = d.h; P.ldx = d.ldh; P.K = d.inter; P.start = 0; P.keep = d.k_int;
+      P.g_total = (d.k_int + kGroup - 1) / kGroup;
+      f.mode = kPlain; f.job = 2; f.job2 = 2; f.keep = d.hidden; f.period = d.hidden;
+      f.tpb = (d.hidden + RB - 1) / RB;
+      const int x_extent = P.g_total * 64 < d.inter / 2 ? P.g_total * 64 : d.inter / 2;
+      rc = encode_family(&c.wmap[n_tf], d.wd, d.inter, x_extent, d.hidden, 1, d.hidden, RB);
+    }
+    if (rc) return rc;
+    P.tiles = f.tpb;
+    tiles += f.tpb;
+    ++n_tf;
+    if (P.g_total > g_max) g_max = P.g_total;
+    const int gr = copy_granule(P.K / kGroup);
+    if (gr < gran) gran = gr;
+  }
+  c.n_tf = n_tf;
+  c.tiles_total = tiles;
+  if (tiles < 1 || tiles * EW > kCounterInts) return UNIQL_ERR_UNSUPPORTED;
+
+  const size_t smem = plan_split(&c, d.M, g_max, gran, true);
+  if (!smem) return UNIQL_ERR_UNSUPPORTED;
+  if (count > 1 && (c.n_kp != 1 || d.M > 8)) return UNIQL_ERR_UNSUPPORTED;
+  c.max_slots = 0;
+  for (int i = 0; i < count; ++i) {
+    const int sl = slots_needed(c.ph[i].tiles, c.ph[i].g_total, c.gp, c.n_rp);
+    if (sl > c.max_slots) c.max_slots = sl;
+  }
+  const size_t need = (size_t)kWsHeader + (size_t)tiles * c.max_slots * d.M * RB * 4;
+  if (!cfg.workspace || cfg.ws_bytes < need) return UNIQL_ERR_WORKSPACE;
+  unsigned char* ws = reinterpret_cast<unsigned char*>(cfg.workspace);
+  c.counters = reinterpret_cast<int*>(ws);
+  c.status = reinterpret_cast<int*>(ws + kStatusOff);
+  c.partials = reinterpret_cast<float*>(ws + kWsHeader);
+  c.grid_sync = reinterpret_cast<int*>(ws + kGridSyncOff);
+  if (count > 1) {
+    if (d.M <= 4) return launch_t<1, false, 1, 2>(p, c, smem, cfg.stream);
+    return launch_t<1, false, 2, 2>(p, c, smem, cfg.stream);
+  }
+  if (d.M <= 4) return launch_t<1, false, 1, 1>(p, c, smem, cfg.stream);
+  if (d.M <= 8) return launch_t<1, false, 2, 1>(p, c, smem, cfg.stream);
+  return launch_t<2, false, 4, 1>(p, c, smem, cfg.stream);
+}
+
+}  // namespace
+
+int launch_mlp_decode(const MlpDecode& d, int fuse, const LaunchCfg& cfg) {
+  if (!mlp_decode_supported(d)) return UNIQL_ERR_UNSUPPORTED;
+  if (fuse) return launch_mlp_phases(d, 0, 2, cfg);
+  const int rc = launch_mlp_phases(d, 0, 1, cfg);
+  return rc ? rc : launch_mlp_phases(d, 1, 1, cfg);
 }
 
 int decode_status_offset() { return kStatusOff; }

@@ -1,6 +1,7 @@
 """Pins for the CPU oracle: it is checked against things other than itself --
 an integer reference, exact rational arithmetic, numpy's dense matmul, the
 textbook rotary embedding, invariants and closed forms.  CPU only."""
+import math
 from fractions import Fraction
 
 import numpy as np
@@ -267,3 +268,58 @@ def test_sorted_truncated_projection_matches_rope_on_original_then_gather():
 def test_rope_rejects_bad_arguments():
     with pytest.raises(ValueError):
         oracle.rope(np.zeros((1, 2)), 1, 1, 4, 2, np.array([[2]], dtype=np.int32), [0], 10.0)
+
+
+# ------------------------------------------------------------------ gated MLP block (Section 3.1)
+def test_swiglu_closed_forms_and_library_logistic():
+    from scipy.special import expit                       # the library's logistic function
+    # literal values: silu(0) = 0, silu(ln 3) = ln 3 * 3/4, silu(-ln 3) = -ln 3 / 4
+    ln3 = math.log(3.0)
+    g = np.array([0.0, ln3, -ln3, 1.0])
+    u = np.array([5.0, 2.0, -4.0, 1.0])
+    h = oracle.swiglu(g, u)
+    assert h[0] == 0.0
+    assert abs(h[1] - 2.0 * ln3 * 0.75) < 1e-15
+    assert abs(h[2] - ln3) < 1e-15                        # (-ln3/4) * (-4)
+    assert abs(h[3] - 1.0 / (1.0 + math.exp(-1.0))) < 1e-15
+    rng = np.random.default_rng(11)
+    g = rng.normal(0, 4, 4096)
+    u = rng.normal(0, 2, 4096)
+    h = oracle.swiglu(g, u)
+    assert np.allclose(h, g * expit(g) * u, rtol=1e-13, atol=1e-300)
+    # silu(t) - silu(-t) = t (logistic(t) + logistic(-t) = 1): fails for any other gate such as sigmoid or gelu
+    one = np.ones_like(g)
+    assert np.allclose(oracle.swiglu(g, one) - oracle.swiglu(-g, one), g, rtol=0, atol=1e-14)
+    # linear in u, the gate acts on g only (a swapped operand order fails here)
+    assert np.allclose(oracle.swiglu(g, 3.0 * u), 3.0 * h, rtol=1e-15)
+    assert not np.allclose(oracle.swiglu(u, g), h)
+    # saturation: silu(t) -> t for large t, -> 0 for very negative t, without overflow
+    big = oracle.swiglu(np.array([800.0, -800.0]), np.array([1.0, 1.0]))
+    assert big[0] == 800.0 and big[1] == 0.0 and np.isfinite(big).all()
+
+
+def test_mlp_swiglu_equals_dense_definition():
+    from scipy.special import expit
+    rng = np.random.default_rng(12)
+    hidden, inter, k_int, M = 256, 384, 200, 3
+    qg, pg = _small_q(rng, inter, hidden)
+    qu, pu = _small_q(rng, inter, hidden)
+    qd, pd = _small_q(rng, hidden, inter)
+    x = synth.draw_x(rng, M, hidden, "f16", outlier_frac=0.02)
+    Wg = oracle.dequant(pg, qg.scales, qg.zeros)
+    Wu = oracle.dequant(pu, qu.scales, qu.zeros)
+    Wd = oracle.dequant(pd, qd.scales, qd.zeros)
+    xd = x.astype(np.float64)
+    gd = xd @ Wg[:k_int].T
+    hd = gd * expit(gd) * (xd @ Wu[:k_int].T)
+    h, y = oracle.mlp_swiglu(x, pg, qg.scales, qg.zeros, pu, qu.scales, qu.zeros, pd, qd.scales, qd.zeros, k_int)
+    assert h.shape == (M, k_int) and y.shape == (M, hidden)
+    assert np.allclose(h, hd, rtol=1e-11, atol=1e-13)
+    # the down projection sees the fp16-rounded activations and only the kept columns of Wd
+    yd = hd.astype(np.float16).astype(np.float64) @ Wd[:, :k_int].T
+    assert np.allclose(y, yd, rtol=1e-11, atol=1e-12)
+    # pruning the intermediate channels is not a no-op here
+    assert not np.allclose(yd, hd.astype(np.float16).astype(np.float64)[:, :k_int - 8] @ Wd[:, :k_int - 8].T)
+    ys = oracle.mlp_swiglu(x, pg, qg.scales, qg.zeros, pu, qu.scales, qu.zeros, pd, qd.scales, qd.zeros, k_int,
+                           out_rows=[5, 77, 255])[1]
+    assert np.array_equal(ys, y[:, [5, 77, 255]])
