@@ -75,10 +75,11 @@ struct TileFam {
   int job;
   int start, period;     // stored row of block h, row r: start + h*period + r   (rope: h*head_dim + r)
   int out_base;          // compact output column of block 0, row 0
-  int mode;              // kPlain, kRope (32 rotation pairs per tile) or kSwiglu (32 gate rows + 32 up rows)
+  int mode;              // kPlain, kNarrow (32 rows x 16 groups), kRope (32 rotation pairs per tile) or
+                         // kSwiglu (32 gate rows + 32 up rows)
   int job2;              // kSwiglu: the job of the up projection (`job` is the gate projection)
 };
-enum { kPlain = 0, kRope = 1, kSwiglu = 2 };
+enum { kPlain = 0, kRope = 1, kSwiglu = 2, kNarrow = 3 };
 __host__ __device__ inline int tile_rows(const TileFam& f) { return f.mode == kPlain ? RB : RB / 2; }
 
 // One matrix product of a launch.  A plain launch has one phase; the fused SwiGLU MLP has two (gate|up,
@@ -103,6 +104,8 @@ struct DecodeCfg {
   int gp;                // visited groups per k-part (the last part may be shorter)
   int g_total;           // visited groups (largest phase)
   int gran;              // groups per scale / zero-point copy granule (2, 4 or 8)
+  int cgz;               // groups per chunk: CG, or 2 * CG when the tiles are narrow (all families kNarrow:
+                         // row slots 32..63 of a stage then hold the same 32 rows, eight groups further on)
   int stages;
   int tiles_total;
   int x_vec;             // activations can be staged with 128-bit loads
@@ -265,6 +268,15 @@ __device__ inline void store_tile(const Params& p, const TileFam& f, const TileP
       const float hv = gt / (1.f + __expf(-gt)) * up;
       y[(size_t)m * jb.ldy + f.out_base + cc] = DT<T>::from_f(hv);
     }
+  } else if (f.mode == kNarrow) {
+    for (int i = etid; i < (RB / 2) * p.M; i += ETH) {
+      const int pp = i & (RB / 2 - 1), m = i / (RB / 2);
+      const int r = q.r0 + pp;
+      if (r >= f.keep) continue;
+      float v = get(pp, m) + get(pp + RB / 2, m);          // the two halves of the chunk's groups
+      if (bias) v += DT<T>::to_f(bias[f.start + q.h * f.period + r]);
+      y[(size_t)m * jb.ldy + f.out_base + q.h * f.keep + r] = DT<T>::from_f(v);
+    }
   } else if (jb.rope.enabled) {
     const int half = jb.rope.head_keep >> 1;
     for (int i = etid; i < (RB / 2) * p.M; i += ETH) {
@@ -301,11 +313,11 @@ __device__ inline void store_tile(const Params& p, const TileFam& f, const TileP
 // units into n_rp equal ranges (stream-K) balances the bytes but every tile then ends with a hand-over
 // between blocks (park, arrival count, reduction by the last block: about the time of three chunks);
 // when that costs more than it saves, the left-over tiles are given whole to R blocks instead.
-__host__ __device__ inline long tail_blocks(long n_rp, long R, long Cq) {
-  const long Ut = R * Cq;
+__host__ __device__ inline int tail_blocks(int n_rp, int R, int Cq) {
+  const int Ut = R * Cq;
   if (Ut == 0) return 1;
-  const bool split = R * Cq / n_rp + 3 < Cq;
-  const long Bt = split ? n_rp : R;
+  const bool split = Ut / n_rp + 3 < Cq;
+  const int Bt = split ? n_rp : R;
   return Bt < Ut ? Bt : Ut;
 }
 
@@ -325,13 +337,15 @@ __device__ inline Work block_work(int n_rp, int tile0, int tiles, int Ck, int rp
   w.Ck = Ck;
   const int base = tiles / n_rp;
   const int R = tiles - base * n_rp;
-  const long Ut = (long)R * Ck;
-  const long Bt = tail_blocks(n_rp, R, Ck);                   // blocks that get tail units
+  // 32-bit arithmetic (64-bit divisions are slow and this is on every warp's way to its first unit):
+  // the host checks n_rp * n_rp * Ck < 2^31
+  const unsigned Ut = (unsigned)(R * Ck);
+  const unsigned Bt = (unsigned)tail_blocks(n_rp, R, Ck);     // blocks that get tail units
   w.n1 = base * Ck;
   w.tile1 = tile0 + rp * base;
   w.tail_tile0 = tile0 + n_rp * base;
   w.tb = w.te = 0;
-  if (rp < Bt) { w.tb = (int)(Ut * rp / Bt); w.te = (int)(Ut * (rp + 1) / Bt); }
+  if ((unsigned)rp < Bt) { w.tb = (int)(Ut * (unsigned)rp / Bt); w.te = (int)(Ut * (unsigned)(rp + 1) / Bt); }
   w.n_units = w.n1 + (w.te - w.tb);
   return w;
 }
@@ -349,7 +363,7 @@ __device__ inline PhaseCtx phase_ctx(const DecodeCfg& c, int ph, int kp, int rp)
   k.Gk = min(c.gp, P.g_total - v_lo);
   k.sg_lo = P.v_first + v_lo;
   k.G = P.K / kGroup;
-  k.wk = block_work(c.n_rp, P.tile0, P.tiles, (k.Gk + CG - 1) / CG, rp);
+  k.wk = block_work(c.n_rp, P.tile0, P.tiles, (k.Gk + c.cgz - 1) / c.cgz, rp);
   return k;
 }
 // (tile, chunk) of block-local unit i, walked in order.  The share of the left-over tiles comes first:
@@ -414,7 +428,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   // Programmatic dependent launch: the next kernel of the stream may be set up while this one runs (its
   // blocks still need this block's resources, so they start as blocks here exit) ...
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (NPH == 1 && phase_ctx(c, 0, kp, rp).wk.n_units == 0) return;
+  const PhaseCtx pc0 = phase_ctx(c, 0, kp, rp);
+  if (NPH == 1 && pc0.wk.n_units == 0) return;
 
   // ======================================================================================= producer
   // The ring runs on across phases: the weights of the next phase are fetched while the grid-wide barrier
@@ -424,7 +439,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     uint32_t ring_parity = 1;      // parity of the previous use of ring position s
     bool ok = true;
     for (int ph = 0; ph < NPH && ok; ++ph) {
-      const PhaseCtx pc = phase_ctx(c, ph, kp, rp);
+      const PhaseCtx pc = (NPH == 1 || ph == 0) ? pc0 : phase_ctx(c, ph, kp, rp);
       const Work& wk = pc.wk;
       const int Gk = pc.Gk, sg_lo = pc.sg_lo, G = pc.G;
       if (wk.n_units == 0) continue;
@@ -455,26 +470,35 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
             } else if (mode == kSwiglu) {
               const int cc = q.r0 + lane;
               if (cc < f.keep) sr = f.start + cc;
+            } else if (mode == kNarrow) {
+              const int r = q.r0 + lane;
+              if (r < f.keep) sr = f.start + q.h * f.period + r;
             } else {
               const int r = q.r0 + slot;
               if (r < f.keep) sr = f.start + q.h * f.period + r;
             }
-            srow[r2] = sr >= 0 ? jb.scales + (size_t)sr * G + sg_lo : nullptr;
-            zrow[r2] = sr >= 0 ? jb.zeros + (size_t)sr * G + sg_lo : nullptr;
+            const int gsh = mode == kNarrow ? r2 * CG : 0;       // the second half of a narrow chunk
+            srow[r2] = sr >= 0 ? jb.scales + (size_t)sr * G + sg_lo + gsh : nullptr;
+            zrow[r2] = sr >= 0 ? jb.zeros + (size_t)sr * G + sg_lo + gsh : nullptr;
           }
           tile_prev = ui.tile;
         }
         const int chunk = ui.chunk;
-        const int ng = min(CG, Gk - chunk * CG);
-        const int nb = (ng + 1) >> 1;                      // 128-byte columns with a visited group
+        const int ng_all = min(c.cgz, Gk - chunk * c.cgz);  // visited groups of the unit
+        const int ng = min(CG, ng_all), ng2 = ng_all - ng;  // ... in row slots 0..31 (all 64 unless narrow) / 32..63
+        const int nb = (ng + 1) >> 1, nb2 = (ng2 + 1) >> 1; // 128-byte columns with a visited group
         const uint32_t full = bar_full + 8 * s;
         const uint32_t st = sbase + (uint32_t)s * STAGE_BYTES;
-        if (lane == 0) mbar_expect_tx(full, (uint32_t)(nb * BOX_BYTES));
+        if (lane == 0)
+          mbar_expect_tx(full, mode == kNarrow ? (uint32_t)((nb + nb2) * (BOX_BYTES / 2)) : (uint32_t)(nb * BOX_BYTES));
         __syncwarp();
         if (lane < nb) {
-          const int xb = (sg_lo + chunk * CG + 2 * lane) * 64;       // byte in the weight row
+          const int xb = (sg_lo + chunk * c.cgz + 2 * lane) * 64;    // byte in the weight row
           const uint32_t dst = st + (uint32_t)lane * BOX_BYTES;
-          if (mode == kRope) {
+          if (mode == kNarrow) {
+            tma_box3(dst, &c.wmap[q.fi], xb, q.r0, q.h, full);
+            if (lane < nb2) tma_box3(dst + (RB / 2) * 128, &c.wmap[q.fi], xb + CG * 64, q.r0, q.h, full);
+          } else if (mode == kRope) {
             tma_box3(dst, &c.wmap[q.fi], xb, q.r0, 2 * q.h, full);
             tma_box3(dst + (RB / 2) * 128, &c.wmap[q.fi], xb, q.r0, 2 * q.h + 1, full);
           } else if (mode == kSwiglu) {
@@ -486,17 +510,18 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         }
 #pragma unroll
         for (int r2 = 0; r2 < 2; ++r2) {
-          if (srow[r2]) {
+          const int ngr = (mode == kNarrow && r2) ? ng2 : ng;      // groups of this half of the row slots
+          if (srow[r2] && ngr > 0) {
             const int slot = lane + 32 * r2;
             const uint32_t sd = st + STAGE_W + slot * (CG * 2), zd = sd + STAGE_SZ;
-            const __half* sp = srow[r2] + chunk * CG;
-            const __half* zp = zrow[r2] + chunk * CG;
+            const __half* sp = srow[r2] + chunk * c.cgz;
+            const __half* zp = zrow[r2] + chunk * c.cgz;
             if (c.gran == 8) {
               cp_async16(sd, sp); cp_async16(zd, zp);
             } else if (c.gran == 4) {
-              for (int g4 = 0; g4 < ng; g4 += 4) { cp_async8(sd + g4 * 2, sp + g4); cp_async8(zd + g4 * 2, zp + g4); }
+              for (int g4 = 0; g4 < ngr; g4 += 4) { cp_async8(sd + g4 * 2, sp + g4); cp_async8(zd + g4 * 2, zp + g4); }
             } else {
-              for (int g2 = 0; g2 < ng; g2 += 2) { cp_async4(sd + g2 * 2, sp + g2); cp_async4(zd + g2 * 2, zp + g2); }
+              for (int g2 = 0; g2 < ngr; g2 += 2) { cp_async4(sd + g2 * 2, sp + g2); cp_async4(zd + g2 * 2, zp + g2); }
             }
           }
         }
@@ -533,7 +558,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     // wait: weights, scales and zero-points are not produced by a preceding decode launch)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int ph = 0; ph < NPH; ++ph) {
-      const PhaseCtx pc = phase_ctx(c, ph, kp, rp);
+      const PhaseCtx pc = (NPH == 1 || ph == 0) ? pc0 : phase_ctx(c, ph, kp, rp);
       const Work& wk = pc.wk;
       const Phase& P = c.ph[ph];
       UnitIter ui;
@@ -569,9 +594,9 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
               int n_here = 1, first = rp;                      // a whole tile: one block per k-part
               if (tail) {
                 const int Gq = min(c.gp, P.g_total - q2 * c.gp);
-                const long Cq = (Gq + CG - 1) / CG;
+                const long Cq = (Gq + c.cgz - 1) / c.cgz;
                 const long Ut = (long)R * Cq;
-                const long Bt = tail_blocks(c.n_rp, R, Cq);
+                const long Bt = tail_blocks(c.n_rp, R, (int)Cq);
                 const long t0 = (long)(tile - wk.tail_tile0) * Cq;
                 first = owner_of(t0, Bt, Ut);
                 n_here = owner_of(t0 + Cq - 1, Bt, Ut) - first + 1;
@@ -644,6 +669,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   // MMA row g of a sub-tile is row slot pg: lanes g = 2i and 2i+1 get slots that differ in bit 2, so that
   // under the 128-byte swizzle the eight lanes of a shared-memory load phase touch eight distinct 16-byte columns
   const int pg = (g >> 1) | ((g & 1) << 2);
+  // group of the chunk this warp works on: narrow tiles put eight more groups of the same rows in slots 32..63
+  const int g_first = c.cgz > CG ? rg * CG + kpw : kpw;
   uint32_t cons_parity = 0;
   auto give_up = [&]() { if (lane == 0) atomicExch(c.status, UNIQL_ERR_TIMEOUT); };
   auto consumer_sync = [&]() -> bool {
@@ -674,8 +701,9 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     // units (K-heavy matrices), the chunks of that run.
     int ch0 = 0, n_ch = wk.Ck;
     if (wk.n1 == 0 && wk.te - wk.tb < wk.Ck) { ch0 = wk.tb % wk.Ck; n_ch = wk.te - wk.tb; }
-    const int Gn = n_ch * CG;
-    auto needed_group = [&](int gn) { int ch = ch0 + gn / CG; if (ch >= wk.Ck) ch -= wk.Ck; return ch * CG + (gn & (CG - 1)); };
+    const int cgz = c.cgz, cg_sh = c.cgz > CG ? 4 : 3;
+    const int Gn = n_ch * cgz;
+    auto needed_group = [&](int gn) { int ch = ch0 + (gn >> cg_sh); if (ch >= wk.Ck) ch -= wk.Ck; return (ch << cg_sh) + (gn & (cgz - 1)); };
     if (NT == 0) {          // (the integer path writes every entry it later reads)
       for (int i = ctid; i < Gk * 8 * MT; i += CTH) xg[i] = make_float2(0.f, 0.f);
       if (!consumer_sync()) return false;
@@ -848,7 +876,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     int s = 0;
     uint32_t ring_parity = 0;
     for (int ph = 0; ph < NPH; ++ph) {
-    const PhaseCtx pc = phase_ctx(c, ph, kp, rp);
+    const PhaseCtx pc = (NPH == 1 || ph == 0) ? pc0 : phase_ctx(c, ph, kp, rp);
     const Work& wk = pc.wk;
     const int Gk = pc.Gk;
     if (NPH > 1 && ph > 0) {
@@ -889,7 +917,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         give_up();
         return;
       }
-      const int gi = ui.chunk * CG + kpw;
+      const int gi = ui.chunk * c.cgz + g_first;
       if (gi < Gk) {
         const uint32_t st = sbase + (uint32_t)s * STAGE_BYTES;
         const uint32_t wp = st + wl_off, sp = st + sl_off;
@@ -979,7 +1007,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   }
 
   // ===================================================================== consumers, fp16 path (one phase)
-  const PhaseCtx pc = phase_ctx(c, 0, kp, rp);
+  const PhaseCtx& pc = pc0;
   const Work& wk = pc.wk;
   const int Gk = pc.Gk;
   if (!stage_x(0, pc)) return;
@@ -1019,7 +1047,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       give_up();
       return;
     }
-    const int gi = ui.chunk * CG + kpw;
+    const int gi = ui.chunk * c.cgz + g_first;
     if (gi < Gk) {
       const uint32_t st = sbase + (uint32_t)s * STAGE_BYTES;
       const uint32_t wp = st + wl_off, sp = st + sl_off;
@@ -1212,20 +1240,29 @@ size_t plan_smem(DecodeCfg* c, int M, int MT, int gp, int stages, int part_bufs,
 
 // Worst-case number of workspace slots a tile needs for a given split: one per k-part for a whole tile,
 // one per block that shares it for a left-over tile.
-int slots_needed(int tiles, int g_total, int gp, int n_rp) {
+int slots_needed(int tiles, int g_total, int gp, int n_rp, int cgz) {
   int total = 0;
   const int base = tiles / n_rp;
   const long R = tiles - (long)base * n_rp;
   for (int v = 0; v < g_total; v += gp) {
     const long Gq = (g_total - v) < gp ? (g_total - v) : gp;
-    const long Cq = (Gq + CG - 1) / CG;
+    const long Cq = (Gq + cgz - 1) / cgz;
     const long Ut = R * Cq;
     if (Ut == 0) { total += 1; continue; }
-    const long Bt = tail_blocks(n_rp, R, Cq);
+    const long Bt = tail_blocks(n_rp, (int)R, (int)Cq);
     const long per_block = Ut / Bt;           // >= 1
     total += (int)((Cq + per_block - 1) / per_block) + 1;
   }
   return total;
+}
+
+// Time of the slowest block, in units (one stage of the ring), for `tiles` tiles of Ck units over n_rp blocks:
+// whole tiles, then the left-over tiles either cut into equal ranges (plus the hand-over) or given whole.
+long schedule_cost(long tiles, long Ck, long n_rp) {
+  const long base = tiles / n_rp, R = tiles - base * n_rp;
+  if (R == 0) return base * Ck;
+  const bool split = R * Ck / n_rp + 3 < Ck;                 // the rule of tail_blocks()
+  return base * Ck + (split ? (R * Ck + n_rp - 1) / n_rp + 3 : Ck);
 }
 
 template <int MT, bool ONECOL, int NT, int NPH>
@@ -1305,6 +1342,8 @@ size_t plan_split(DecodeCfg* c, int M, int g_total, int gran, bool i8) {
   if (n_rp < 1) n_rp = sm_count() / c->n_kp;
   if (n_rp < 1) n_rp = 1;
   c->n_rp = n_rp;
+  // the kernel cuts the left-over units with 32-bit products of at most n_rp * n_rp * (chunks per tile)
+  if ((long long)n_rp * n_rp * ((c->gp + CG - 1) / CG) >= (1ll << 31)) return 0;
   return smem;
 }
 
@@ -1352,6 +1391,39 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
             (p.imap.fam[0].keep % 8) == 0 && (p.ldx % 8) == 0 && ((((uintptr_t)p.x) & 15) == 0);
   if (count_tile_fams(p) > kMaxTF) return UNIQL_ERR_UNSUPPORTED;
 
+  // integer path: fp16 activations staged with 128-bit loads (a leading input block); UNIQL_DECODE_I8=0: fp16 MMAs
+  const bool i8 = c.x_vec && env_int("UNIQL_DECODE_I8", 1) != 0;
+  const size_t smem = plan_split(&c, p.M, g_total, gran, i8);
+  if (!smem) return UNIQL_ERR_UNSUPPORTED;
+
+  // ---- narrow tiles (32 rows x 16 groups) when the schedule they give is shorter: matrices with fewer
+  //      64-row tiles than blocks then run without a hand-over between blocks (UNIQL_DECODE_NARROW=0/1 forces)
+  bool narrow = false;
+  {
+    bool all_plain = true;
+    long t64 = 0, t32 = 0;
+    for (int j = 0; j < p.n_jobs; ++j) {
+      const JobDev& jb = p.job[j];
+      if (jb.rope.enabled) { all_plain = false; continue; }
+      for (int k = 0; k < jb.omap.n_fam; ++k) {
+        const Fam& a = jb.omap.fam[k];
+        t64 += (long)((a.keep + RB - 1) / RB) * a.count;
+        t32 += (long)((a.keep + RB / 2 - 1) / (RB / 2)) * a.count;
+      }
+    }
+    if (all_plain) {
+      const int Gk0 = g_total < c.gp ? g_total : c.gp;
+      // (only where there are fewer wide tiles than blocks and the input channels are not split: measured,
+      //  the smaller boxes of the narrow tiles cost more than a better balance of many tiles gains)
+      narrow = c.n_kp == 1 && t64 < c.n_rp &&
+               schedule_cost(t32, (Gk0 + 2 * CG - 1) / (2 * CG), c.n_rp) < schedule_cost(t64, (Gk0 + CG - 1) / CG, c.n_rp);
+      const int force = env_int("UNIQL_DECODE_NARROW", -1);
+      if (force == 0) narrow = false;
+      if (force == 1) narrow = true;
+    }
+  }
+  c.cgz = narrow ? 2 * CG : CG;
+
   // ---- tile families and their tensor maps
   const int x_extent = (v_first + g_total) * 64 < p.K / 2 ? (v_first + g_total) * 64 : p.K / 2;
   int tiles = 0, n_tf = 0;
@@ -1368,13 +1440,15 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
       tiles += f.tpb * f.count;
       ++n_tf;
     } else {
+      const int rows = narrow ? RB / 2 : RB;
       for (int k = 0; k < jb.omap.n_fam; ++k) {
         const Fam& a = jb.omap.fam[k];
         TileFam& f = c.tf[n_tf];
-        f.tile_begin = tiles; f.tpb = (a.keep + RB - 1) / RB; f.keep = a.keep; f.count = a.count;
-        f.job = j; f.start = a.start; f.period = a.period; f.out_base = jb.omap.base[k]; f.mode = kPlain; f.job2 = j;
+        f.tile_begin = tiles; f.tpb = (a.keep + rows - 1) / rows; f.keep = a.keep; f.count = a.count;
+        f.job = j; f.start = a.start; f.period = a.period; f.out_base = jb.omap.base[k];
+        f.mode = narrow ? kNarrow : kPlain; f.job2 = j;
         const int rc = encode_family(&c.wmap[n_tf], jb.w + (size_t)a.start * (p.K / 2), p.K, x_extent, a.keep,
-                                     a.count, a.count > 1 ? a.period : a.keep, RB);
+                                     a.count, a.count > 1 ? a.period : a.keep, rows);
         if (rc) return rc;
         tiles += f.tpb * f.count;
         ++n_tf;
@@ -1392,12 +1466,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
     P.tile0 = 0; P.tiles = tiles;
   }
   if (tiles < 1 || tiles * EW > kCounterInts) return UNIQL_ERR_UNSUPPORTED;
-
-  // integer path: fp16 activations staged with 128-bit loads (a leading input block); UNIQL_DECODE_I8=0: fp16 MMAs
-  const bool i8 = c.x_vec && env_int("UNIQL_DECODE_I8", 1) != 0;
-  const size_t smem = plan_split(&c, p.M, g_total, gran, i8);
-  if (!smem) return UNIQL_ERR_UNSUPPORTED;
-  c.max_slots = slots_needed(tiles, c.g_total, c.gp, c.n_rp);
+  c.max_slots = slots_needed(tiles, c.g_total, c.gp, c.n_rp, c.cgz);
   {
     const size_t need = (size_t)kWsHeader + (size_t)tiles * c.max_slots * p.M * RB * 4;
     if (!cfg.workspace || cfg.ws_bytes < need) return UNIQL_ERR_WORKSPACE;
@@ -1461,7 +1530,30 @@ int launch_mlp_phases(const MlpDecode& d, int first, int count, const LaunchCfg&
   memset(&c, 0, sizeof(c));
   c.x_vec = 1;
   c.n_ph = count;
-  int tiles = 0, n_tf = 0, g_max = 0, gran = 8;
+  int g_max = 0, gran = 8;
+  for (int ph = first; ph < first + count; ++ph) {
+    const int g_total = ph == 0 ? d.hidden / kGroup : (d.k_int + kGroup - 1) / kGroup;
+    if (g_total > g_max) g_max = g_total;
+    const int gr = copy_granule((ph == 0 ? d.hidden : d.inter) / kGroup);
+    if (gr < gran) gran = gr;
+  }
+  const size_t smem = plan_split(&c, d.M, g_max, gran, true);
+  if (!smem) return UNIQL_ERR_UNSUPPORTED;
+  if (count > 1 && (c.n_kp != 1 || d.M > 8)) return UNIQL_ERR_UNSUPPORTED;
+  // the down projection on its own: narrow tiles under the same rule as any plain launch
+  bool narrow = false;
+  if (first == 1 && count == 1) {
+    const int Gk0 = g_max < c.gp ? g_max : c.gp;
+    narrow = c.n_kp == 1 && (d.hidden + RB - 1) / RB < c.n_rp &&
+             schedule_cost((d.hidden + RB / 2 - 1) / (RB / 2), (Gk0 + 2 * CG - 1) / (2 * CG), c.n_rp) <
+                 schedule_cost((d.hidden + RB - 1) / RB, (Gk0 + CG - 1) / CG, c.n_rp);
+    const int force = env_int("UNIQL_DECODE_NARROW", -1);
+    if (force == 0) narrow = false;
+    if (force == 1) narrow = true;
+  }
+  c.cgz = narrow ? 2 * CG : CG;
+
+  int tiles = 0, n_tf = 0;
   for (int ph = first; ph < first + count; ++ph) {
     Phase& P = c.ph[ph - first];
     TileFam& f = c.tf[n_tf];
@@ -1477,29 +1569,23 @@ int launch_mlp_phases(const MlpDecode& d, int first, int count, const LaunchCfg&
     } else {
       P.x = d.h; P.ldx = d.ldh; P.K = d.inter; P.start = 0; P.keep = d.k_int;
       P.g_total = (d.k_int + kGroup - 1) / kGroup;
-      f.mode = kPlain; f.job = 2; f.job2 = 2; f.keep = d.hidden; f.period = d.hidden;
-      f.tpb = (d.hidden + RB - 1) / RB;
+      const int rows = narrow ? RB / 2 : RB;
+      f.mode = narrow ? kNarrow : kPlain; f.job = 2; f.job2 = 2; f.keep = d.hidden; f.period = d.hidden;
+      f.tpb = (d.hidden + rows - 1) / rows;
       const int x_extent = P.g_total * 64 < d.inter / 2 ? P.g_total * 64 : d.inter / 2;
-      rc = encode_family(&c.wmap[n_tf], d.wd, d.inter, x_extent, d.hidden, 1, d.hidden, RB);
+      rc = encode_family(&c.wmap[n_tf], d.wd, d.inter, x_extent, d.hidden, 1, d.hidden, rows);
     }
     if (rc) return rc;
     P.tiles = f.tpb;
     tiles += f.tpb;
     ++n_tf;
-    if (P.g_total > g_max) g_max = P.g_total;
-    const int gr = copy_granule(P.K / kGroup);
-    if (gr < gran) gran = gr;
   }
   c.n_tf = n_tf;
   c.tiles_total = tiles;
   if (tiles < 1 || tiles * EW > kCounterInts) return UNIQL_ERR_UNSUPPORTED;
-
-  const size_t smem = plan_split(&c, d.M, g_max, gran, true);
-  if (!smem) return UNIQL_ERR_UNSUPPORTED;
-  if (count > 1 && (c.n_kp != 1 || d.M > 8)) return UNIQL_ERR_UNSUPPORTED;
   c.max_slots = 0;
   for (int i = 0; i < count; ++i) {
-    const int sl = slots_needed(c.ph[i].tiles, c.ph[i].g_total, c.gp, c.n_rp);
+    const int sl = slots_needed(c.ph[i].tiles, c.ph[i].g_total, c.gp, c.n_rp, c.cgz);
     if (sl > c.max_slots) c.max_slots = sl;
   }
   const size_t need = (size_t)kWsHeader + (size_t)tiles * c.max_slots * d.M * RB * 4;

@@ -31,7 +31,7 @@ def B():
 def _reset_path(B):
     yield
     B.set_path(B.PATH_AUTO)
-    for k in ("UNIQL_DECODE_KP", "UNIQL_DECODE_RP"):
+    for k in ("UNIQL_DECODE_KP", "UNIQL_DECODE_RP", "UNIQL_DECODE_NARROW"):
         os.environ.pop(k, None)
 
 
@@ -141,6 +141,35 @@ def test_decode_split_configs(B, kp, rp, M):
         check_output(y, ref, "f16", TIGHT, "kp=%d rp=%d M=%d" % (kp, rp, M))
         y2, _ = run_ex(B, qw, dw, x, "f16", None, k_in, None, k_out, bias=bias)
         assert torch.equal(y, y2), "run-to-run results differ"
+
+
+@pytest.mark.parametrize("narrow", [0, 1])
+@pytest.mark.parametrize("kp,rp", [(0, 0), (1, 1), (1, 7), (2, 5), (3, 49)])
+@pytest.mark.parametrize("M", [1, 4, 7, 16])
+def test_tile_shapes(B, narrow, kp, rp, M):
+    """Wide tiles (64 rows x 8 groups) and narrow tiles (32 rows x 16 groups) give the same answer for every
+    split: ragged row counts, group counts that leave the second half of a narrow chunk empty or short,
+    several families, bias, and both activation paths (128-bit staging and the generic one)."""
+    os.environ["UNIQL_DECODE_NARROW"] = str(narrow)
+    if kp:
+        os.environ["UNIQL_DECODE_KP"], os.environ["UNIQL_DECODE_RP"] = str(kp), str(rp)
+    B.set_path(B.PATH_DECODE)
+    rng = np.random.default_rng(70 + M)
+    for (N, K, k_in, k_out) in [(200, 2304, 2304, 200), (200, 2304, 1100, 77), (96, 256, 256, 96), (70, 3328, 3072, 33)]:
+        qw = synth.draw_qweight(rng, N, K)
+        dw = dev_weight(qw)
+        bias = synth.to_dtype_values(rng.standard_normal(N).astype(np.float32), "f16")
+        x = synth.draw_x(rng, M, k_in, "f16")
+        y, ref = run_ex(B, qw, dw, x, "f16", None, k_in, None, k_out, bias=bias, ldy_pad=3)
+        check_output(y, ref, "f16", TIGHT, "narrow=%d kp=%d rp=%d M=%d %s" % (narrow, kp, rp, M, (N, K, k_in, k_out)))
+    qw = synth.draw_qweight(rng, 512, 1024)
+    dw = dev_weight(qw)
+    for keep in (128, 108, 84):
+        out_map = synth.map_per_head(4, 128, keep)
+        in_map = synth.map_per_head(8, 128, keep)
+        x = synth.draw_x(rng, M, synth.map_size(in_map), "f16")
+        y, ref = run_ex(B, qw, dw, x, "f16", in_map, 0, out_map, 0)
+        check_output(y, ref, "f16", TIGHT, "narrow=%d per-head keep %d M=%d" % (narrow, keep, M))
 
 
 def test_caller_workspace(B):
