@@ -541,11 +541,12 @@ def run_case(args):
     return 0
 
 
-# DRAM bytes (read + write) per algorithmic byte of a decode launch, from the ncu capture summarised in
-# profiles/decode_kernel_llama3_gateup_m1.md (62.48 MB read + 0.11 MB written for 62.39 MB of retained weights);
-# traffic grows in proportion to the retained weights, so the per-launch average of the step is scaled from it.
-# None once the kernel has changed since the capture.
-DRAM_TRAFFIC_RATIO = 62.59 / 62.39
+# DRAM bytes (read + write) per algorithmic byte of a decode launch, from the ncu captures summarised in
+# profiles/decode_kernel_llama3_gateup_m1.md (62.49 MB read + 0.07 MB written for 62.39 MB of retained weights)
+# and profiles/decode_kernel_llama3_down_m1.md (31.31 MB for 31.20 MB); traffic grows in proportion to the
+# retained weights, so the per-launch average of the step is scaled from the two.
+# None once the kernel has changed since the captures.
+DRAM_TRAFFIC_RATIO = (62.56 + 31.31) / (62.39 + 31.20)
 
 
 def main():

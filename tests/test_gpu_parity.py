@@ -145,7 +145,7 @@ def test_decode_split_configs(B, kp, rp, M):
 
 @pytest.mark.parametrize("narrow", [0, 1])
 @pytest.mark.parametrize("kp,rp", [(0, 0), (1, 1), (1, 7), (2, 5), (3, 49)])
-@pytest.mark.parametrize("M", [1, 4, 7, 16])
+@pytest.mark.parametrize("M", [1, 2, 4, 7, 16])
 def test_tile_shapes(B, narrow, kp, rp, M):
     """Wide tiles (64 rows x 8 groups) and narrow tiles (32 rows x 16 groups) give the same answer for every
     split: ragged row counts, group counts that leave the second half of a narrow chunk empty or short,
