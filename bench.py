@@ -285,7 +285,34 @@ def detail_tables(B, torch, steps):
             rows["%.2f" % r] = {"us_per_mlp": round(sec * 1e6, 2), "GBps": round(gbs, 1),
                                 "frac_hbm_%s" % which: round(gbs / hbm, 3), "tokens_per_s_mlp": round(M / sec, 1)}
         out["decode_M%d" % M] = rows
-        del w
+        # the MLP block through its own entry point: gate|up with the gated product as epilogue, then down
+        # (two launches), and both products in one launch where the shapes allow it
+        hbuf = torch.zeros((M, INTER), dtype=torch.float16, device="cuda")
+        for fuse, name in ((0, "mlp_swiglu_two_launches_M%d" % M), (1, "mlp_swiglu_one_launch_M%d" % M)):
+            rows = {}
+            for r in KEEP_RATES:
+                k = keep_count(r, INTER) // 8 * 8
+
+                def one(k=k, w=w, fuse=fuse):
+                    for _ in range(N_COPIES):
+                        g, u, d = w.copies[w.turn % N_COPIES]
+                        w.turn += 1
+                        B.mlp_swiglu_decode(w.x, HIDDEN, g[0], g[1], g[2], u[0], u[1], u[2], d[0], d[1], d[2], M,
+                                            HIDDEN, INTER, k, hbuf, INTER, w.yd[0], HIDDEN, fuse=fuse)
+                try:
+                    g, _ = capture(torch, one)
+                except RuntimeError as e:                      # one launch: M > 8, or the activations do not fit
+                    rows["%.2f" % r] = {"unsupported": str(e)[:80]}
+                    torch.cuda.synchronize()
+                    continue
+                for _ in range(5):
+                    g.replay()
+                sec = time_graph(torch, g, steps) / (steps * N_COPIES)
+                gbs = BYTES_PER_WEIGHT * 3 * HIDDEN * k / sec / 1e9
+                rows["%.2f" % r] = {"us_per_mlp": round(sec * 1e6, 2), "GBps": round(gbs, 1),
+                                    "frac_hbm_%s" % which: round(gbs / hbm, 3)}
+            out[name] = rows
+        del w, hbuf
         torch.cuda.empty_cache()
     return out
 
