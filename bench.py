@@ -491,12 +491,13 @@ def attention_tables(B, torch, steps):
     hbm, tf, which = measured_peaks()
     rng = np.random.default_rng(3)
     Hq, Hkv, D, K, theta = 32, 8, 128, HIDDEN, 500000.0
-    n_copies = 14                                   # 14 x 11.1 MB > 126 MB
+    n_copies = 12                                   # 12 x 13.4 MB (q, k, v) > 126 MB
     wq, wk = synth.random_qweight_fast(rng, Hq * D, K), synth.random_qweight_fast(rng, Hkv * D, K)
+    wv = synth.random_qweight_fast(rng, Hkv * D, K)
     copies = []
     for _ in range(n_copies):
         c = []
-        for m in (wq, wk):
+        for m in (wq, wk, wv):
             cd = torch.from_numpy(m.codes).cuda()
             packed = torch.empty((m.N, m.K // 2), dtype=torch.uint8, device="cuda")
             B.pack_u4(cd, packed)
@@ -515,7 +516,7 @@ def attention_tables(B, torch, steps):
 
             def one():
                 for _ in range(n_copies):
-                    (q, k) = copies[turn[0] % n_copies]
+                    (q, k, _v) = copies[turn[0] % n_copies]
                     turn[0] += 1
                     B.qk_rope_proj(x, K, q[0], q[1], q[2], k[0], k[1], k[2], None, None, M, K, Hq, Hkv, D, keep, idx, pos,
                                    theta, None, qo, Hq * keep, ko, Hkv * keep)
@@ -532,6 +533,31 @@ def attention_tables(B, torch, steps):
                 tfl = 2.0 * M * weights / sec / 1e12
                 row.update({"TFLOPs": round(tfl, 1), "frac_bf16_%s" % which: round(tfl / tf, 3)})
             rows["d%d" % keep] = row
+            # Q, K and V in one launch, against the Q|K launch followed by a V launch
+            vo = torch.zeros((M, Hkv * keep), dtype=torch.float16, device="cuda")
+            vmap = synth.map_per_head(Hkv, D, keep)
+
+            def one_qkv():
+                for _ in range(n_copies):
+                    (q, k, v) = copies[turn[0] % n_copies]
+                    turn[0] += 1
+                    B.qkv_rope_proj(x, K, q[0], q[1], q[2], k[0], k[1], k[2], v[0], v[1], v[2], None, None, None, M, K,
+                                    Hq, Hkv, D, keep, keep, idx, pos, theta, None, qo, Hq * keep, ko, Hkv * keep, vo,
+                                    Hkv * keep)
+
+            def two_launches():
+                for _ in range(n_copies):
+                    (q, k, v) = copies[turn[0] % n_copies]
+                    turn[0] += 1
+                    B.qk_rope_proj(x, K, q[0], q[1], q[2], k[0], k[1], k[2], None, None, M, K, Hq, Hkv, D, keep, idx, pos,
+                                   theta, None, qo, Hq * keep, ko, Hkv * keep)
+                    B.qlinear_ex(x, K, v[0], v[1], v[2], None, M, K, Hkv * D, None, K, vmap, 0, vo, Hkv * keep)
+            for name, fn in (("qkv_one_launch", one_qkv), ("qk_then_v", two_launches)):
+                g, _ = capture(torch, fn)
+                for _ in range(3):
+                    g.replay()
+                sec = time_graph(torch, g, steps) / (steps * n_copies)
+                rows["d%d" % keep][name + "_us"] = round(sec * 1e6, 2)
         out["llama_qk_rope_M%d" % M] = rows
     return out
 

@@ -206,6 +206,21 @@ int uniql_qk_rope_proj(const void* x, int ldx, int dt, const uint8_t* wq, const 
                        double theta, const double* inv_freq, void* q_out, int ldq, void* k_out,
                        int ldk, void* workspace, size_t ws_bytes, void* stream);
 
+/* ---- Q, K and V projections of one attention block in ONE launch ----
+ * (Section 3.2, MHSA paragraph: the weights of a head form the groups {W_q, W_k}, sorted symmetrically and
+ * rotated, and {W_v, W_o}, sorted per head without the symmetry constraint.)  As uniql_qk_rope_proj, plus
+ * Wv[n_kv_heads*head_dim][K] as a third matrix of the same launch: every key-value head keeps its leading
+ * v_keep rows, no rotation, v_out[M][n_kv_heads*v_keep] (row h*v_keep + r = stored row h*head_dim + r).
+ * v_keep a multiple of 4, 4 <= v_keep <= head_dim; bv optional.  All three share x, so x is staged once and
+ * the three weight matrices stream through one launch. */
+int uniql_qkv_rope_proj(const void* x, int ldx, int dt, const uint8_t* wq, const void* sq, const void* zq,
+                        const uint8_t* wk, const void* sk, const void* zk, const uint8_t* wv,
+                        const void* sv, const void* zv, const void* bq, const void* bk, const void* bv,
+                        int M, int K, int n_q_heads, int n_kv_heads, int head_dim, int head_keep,
+                        int v_keep, const int32_t* retained_idx, const int32_t* pos, double theta,
+                        const double* inv_freq, void* q_out, int ldq, void* k_out, int ldk, void* v_out,
+                        int ldv, void* workspace, size_t ws_bytes, void* stream);
+
 /* ---- SwiGLU MLP block at decode:  y = ( silu(x Wg^T) * (x Wu^T) ) Wd^T ----
  * (Section 3.1, the MLP block f_MLP(X) = (sigma(X W_g) . X W_u) W_d with sigma(t) = t / (1 + exp(-t)),
  * the gate of the Llama / Qwen blocks the paper compresses; Section 3.4: after sorting, pruning the

@@ -61,6 +61,9 @@ _lib.uniql_workspace_bytes.argtypes = [_i, _i, _i]
 _lib.uniql_workspace_init.argtypes = [_vp, _sz, _vp]
 _lib.uniql_workspace_status.argtypes = [_vp, ctypes.POINTER(_i)]
 _lib.uniql_qlinear.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp]
+_lib.uniql_qkv_rope_proj.argtypes = [_vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i,
+                                     _i, _i, _i, _i, _vp, _vp, _d, ctypes.POINTER(_d), _vp, _i, _vp, _i, _vp, _i,
+                                     _vp, _sz, _vp]
 _lib.uniql_mlp_workspace_bytes.restype = _sz
 _lib.uniql_mlp_workspace_bytes.argtypes = [_i, _i, _i]
 _lib.uniql_mlp_swiglu_decode.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i,
@@ -74,7 +77,7 @@ _lib.uniql_qk_rope_proj.argtypes = [_vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _
                                     _vp, _vp, _d, ctypes.POINTER(_d), _vp, _i, _vp, _i, _vp, _sz, _vp]
 for _n in ("uniql_set_path", "uniql_pack_u4", "uniql_unpack_u4", "uniql_dequant", "uniql_workspace_init",
            "uniql_workspace_status", "uniql_qlinear", "uniql_qlinear_noalloc", "uniql_qlinear_ex", "uniql_qlinear_multi", "uniql_qk_rope_proj",
-           "uniql_mlp_swiglu_decode"):
+           "uniql_mlp_swiglu_decode", "uniql_qkv_rope_proj"):
     getattr(_lib, _n).restype = _i
 
 
@@ -233,3 +236,17 @@ def mlp_swiglu_decode(x, ldx, wg, sg, zg, wu, su, zu, wd, sd, zd, M, hidden, int
                                         _ptr(wd), _ptr(sd), _ptr(zd), M, hidden, inter, k_int, _ptr(h), ldh,
                                         _ptr(y), ldy, int(fuse), _ptr(workspace), ws_bytes, _stream(stream)),
            "uniql_mlp_swiglu_decode")
+
+
+def qkv_rope_proj(x, ldx, wq, sq, zq, wk, sk, zk, wv, sv, zv, bq, bk, bv, M, K, n_q_heads, n_kv_heads, head_dim,
+                  head_keep, v_keep, retained_idx, pos, theta, inv_freq, q_out, ldq, k_out, ldk, v_out, ldv,
+                  workspace=None, stream=None) -> None:
+    f = None
+    if inv_freq is not None:
+        f = (ctypes.c_double * len(inv_freq))(*[float(v) for v in inv_freq])
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.uniql_qkv_rope_proj(_ptr(x), ldx, _dt(x), _ptr(wq), _ptr(sq), _ptr(zq), _ptr(wk), _ptr(sk), _ptr(zk),
+                                    _ptr(wv), _ptr(sv), _ptr(zv), _ptr(bq), _ptr(bk), _ptr(bv), M, K, n_q_heads,
+                                    n_kv_heads, head_dim, head_keep, v_keep, _ptr(retained_idx), _ptr(pos),
+                                    float(theta), f, _ptr(q_out), ldq, _ptr(k_out), ldk, _ptr(v_out), ldv,
+                                    _ptr(workspace), ws_bytes, _stream(stream)), "uniql_qkv_rope_proj")

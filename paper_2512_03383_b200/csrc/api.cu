@@ -229,13 +229,16 @@ extern "C" int uniql_qlinear(const void* x, const uint8_t* packed_w, const void*
                           nullptr, k_out, y, k_out, nullptr, 0, stream);
 }
 
-extern "C" int uniql_qk_rope_proj(const void* x, int ldx, int dt, const uint8_t* wq, const void* sq,
-                                  const void* zq, const uint8_t* wk, const void* sk, const void* zk,
-                                  const void* bq, const void* bk, int M, int K, int n_q_heads,
-                                  int n_kv_heads, int head_dim, int head_keep, const int32_t* retained_idx,
-                                  const int32_t* pos, double theta, const double* inv_freq, void* q_out,
-                                  int ldq, void* k_out, int ldk, void* workspace, size_t ws_bytes,
-                                  void* stream) {
+namespace {
+
+// Q and K projections with the rotary epilogue and, when wv is given, the V projection (plain rows, the
+// leading v_keep of every key-value head) as a third job of the same launch.
+int qkv_rope_impl(const void* x, int ldx, int dt, const uint8_t* wq, const void* sq, const void* zq,
+                  const uint8_t* wk, const void* sk, const void* zk, const uint8_t* wv, const void* sv,
+                  const void* zv, const void* bq, const void* bk, const void* bv, int M, int K, int n_q_heads,
+                  int n_kv_heads, int head_dim, int head_keep, int v_keep, const int32_t* retained_idx,
+                  const int32_t* pos, double theta, const double* inv_freq, void* q_out, int ldq, void* k_out,
+                  int ldk, void* v_out, int ldv, void* workspace, size_t ws_bytes, void* stream) {
   int rc = check_common(x, ldx, dt, M, K);
   if (rc) return rc;
   if (!retained_idx || !pos || !q_out || !k_out) return UNIQL_ERR_NULL;
@@ -254,12 +257,19 @@ extern "C" int uniql_qk_rope_proj(const void* x, int ldx, int dt, const uint8_t*
   if (rc) return rc;
   rc = check_weight(wk, sk, zk, n_kv_heads * head_dim);
   if (rc) return rc;
+  if (wv) {
+    if (!v_out) return UNIQL_ERR_NULL;
+    if (v_keep < 1 || v_keep > head_dim || ldv < n_kv_heads * v_keep) return UNIQL_ERR_SHAPE;
+    if ((((uintptr_t)v_out) & 1) || (bv && (((uintptr_t)bv) & 1))) return UNIQL_ERR_ALIGN;
+    rc = check_weight(wv, sv, zv, n_kv_heads * head_dim);
+    if (rc) return rc;
+  }
 
   Params p;
   memset(&p, 0, sizeof(p));
   compile_map(nullptr, K, K, &p.imap);
   p.x = x; p.ldx = ldx; p.dt = dt; p.M = M; p.K = K; p.k_in = K;
-  p.n_jobs = 2;
+  p.n_jobs = wv ? 3 : 2;
   p.idx = retained_idx; p.pos = pos;
   for (int i = 0; i < head_dim / 2; ++i)
     p.inv_freq[i] = inv_freq ? inv_freq[i] : pow(theta, -2.0 * (double)i / (double)head_dim);
@@ -280,7 +290,46 @@ extern "C" int uniql_qk_rope_proj(const void* x, int ldx, int dt, const uint8_t*
     compile_map(&hm, 0, d.N, &d.omap);
     d.rope = RopeDesc{1, nh, j == 0 ? n_q_heads / n_kv_heads : 1, head_dim, head_keep};
   }
+  if (wv) {
+    JobDev& d = p.job[2];
+    d.w = wv; d.scales = (const __half*)sv; d.zeros = (const __half*)zv; d.bias = bv;
+    d.y = v_out; d.ldy = ldv; d.N = n_kv_heads * head_dim;
+    uniql_chanmap hm;
+    hm.n_fam = 1;
+    hm.fam[0] = uniql_family{0, head_dim, v_keep, n_kv_heads};
+    rc = compile_map(&hm, 0, d.N, &d.omap);
+    if (rc) return rc;
+    d.k_out = d.omap.total;
+  }
   return dispatch(p, workspace, ws_bytes, stream);
+}
+
+}  // namespace
+
+extern "C" int uniql_qk_rope_proj(const void* x, int ldx, int dt, const uint8_t* wq, const void* sq,
+                                  const void* zq, const uint8_t* wk, const void* sk, const void* zk,
+                                  const void* bq, const void* bk, int M, int K, int n_q_heads,
+                                  int n_kv_heads, int head_dim, int head_keep, const int32_t* retained_idx,
+                                  const int32_t* pos, double theta, const double* inv_freq, void* q_out,
+                                  int ldq, void* k_out, int ldk, void* workspace, size_t ws_bytes,
+                                  void* stream) {
+  return qkv_rope_impl(x, ldx, dt, wq, sq, zq, wk, sk, zk, nullptr, nullptr, nullptr, bq, bk, nullptr, M, K,
+                       n_q_heads, n_kv_heads, head_dim, head_keep, 0, retained_idx, pos, theta, inv_freq, q_out,
+                       ldq, k_out, ldk, nullptr, 0, workspace, ws_bytes, stream);
+}
+
+extern "C" int uniql_qkv_rope_proj(const void* x, int ldx, int dt, const uint8_t* wq, const void* sq,
+                                   const void* zq, const uint8_t* wk, const void* sk, const void* zk,
+                                   const uint8_t* wv, const void* sv, const void* zv, const void* bq,
+                                   const void* bk, const void* bv, int M, int K, int n_q_heads, int n_kv_heads,
+                                   int head_dim, int head_keep, int v_keep, const int32_t* retained_idx,
+                                   const int32_t* pos, double theta, const double* inv_freq, void* q_out,
+                                   int ldq, void* k_out, int ldk, void* v_out, int ldv, void* workspace,
+                                   size_t ws_bytes, void* stream) {
+  if (!wv) return UNIQL_ERR_NULL;
+  return qkv_rope_impl(x, ldx, dt, wq, sq, zq, wk, sk, zk, wv, sv, zv, bq, bk, bv, M, K, n_q_heads, n_kv_heads,
+                       head_dim, head_keep, v_keep, retained_idx, pos, theta, inv_freq, q_out, ldq, k_out, ldk,
+                       v_out, ldv, workspace, ws_bytes, stream);
 }
 
 extern "C" size_t uniql_mlp_workspace_bytes(int M, int hidden, int inter) {

@@ -260,7 +260,8 @@ def test_multi_job(B):
 
 
 # ---------------------------------------------------------------- fused Q/K projection + pruned RoPE
-def run_rope(B, rng, M, K, Hq, Hkv, D, keep, theta, dtype, idx_kind="perm", bias=False, inv_freq=None):
+def run_rope(B, rng, M, K, Hq, Hkv, D, keep, theta, dtype, idx_kind="perm", bias=False, inv_freq=None, v_keep=None):
+    """Q and K projection with the rotary epilogue; with v_keep also the V projection in the same launch."""
     wq, wk = synth.draw_qweight(rng, Hq * D, K), synth.draw_qweight(rng, Hkv * D, K)
     dq, dk = dev_weight(wq), dev_weight(wk)
     x = synth.draw_x(rng, M, K, dtype)
@@ -274,13 +275,27 @@ def run_rope(B, rng, M, K, Hq, Hkv, D, keep, theta, dtype, idx_kind="perm", bias
     tdt = xd.dtype
     qo = torch.zeros((M, Hq * keep), dtype=tdt, device="cuda")
     ko = torch.zeros((M, Hkv * keep), dtype=tdt, device="cuda")
-    B.qk_rope_proj(xd, K, dq[1], dq[2], dq[3], dk[1], dk[2], dk[3],
-                   None if bq is None else dev_x(bq.reshape(1, -1), dtype).reshape(-1),
-                   None if bk is None else dev_x(bk.reshape(1, -1), dtype).reshape(-1),
-                   M, K, Hq, Hkv, D, keep, torch.from_numpy(idx).cuda(), torch.from_numpy(pos).cuda(), theta,
-                   inv_freq, qo, Hq * keep, ko, Hkv * keep)
+    bqd = None if bq is None else dev_x(bq.reshape(1, -1), dtype).reshape(-1)
+    bkd = None if bk is None else dev_x(bk.reshape(1, -1), dtype).reshape(-1)
+    if v_keep is None:
+        B.qk_rope_proj(xd, K, dq[1], dq[2], dq[3], dk[1], dk[2], dk[3], bqd, bkd,
+                       M, K, Hq, Hkv, D, keep, torch.from_numpy(idx).cuda(), torch.from_numpy(pos).cuda(), theta,
+                       inv_freq, qo, Hq * keep, ko, Hkv * keep)
+    else:
+        wv = synth.draw_qweight(rng, Hkv * D, K)
+        dv = dev_weight(wv)
+        bv = synth.to_dtype_values(rng.standard_normal(Hkv * D).astype(np.float32), dtype) if bias else None
+        vo = torch.full((M, Hkv * v_keep + 3), -9.0, dtype=tdt, device="cuda")
+        B.qkv_rope_proj(xd, K, dq[1], dq[2], dq[3], dk[1], dk[2], dk[3], dv[1], dv[2], dv[3], bqd, bkd,
+                        None if bv is None else dev_x(bv.reshape(1, -1), dtype).reshape(-1),
+                        M, K, Hq, Hkv, D, keep, v_keep, torch.from_numpy(idx).cuda(), torch.from_numpy(pos).cuda(),
+                        theta, inv_freq, qo, Hq * keep, ko, Hkv * keep, vo, vo.stride(0))
     torch.cuda.synchronize()
     out = []
+    if v_keep is not None:
+        assert (vo[:, Hkv * v_keep:] == -9.0).all(), "wrote outside the V columns"
+        Ov = oracle.expand_map(synth.map_per_head(Hkv, D, v_keep))
+        out.append((vo[:, :Hkv * v_keep], oracle.qlinear(x, dv[0], wv.scales, wv.zeros, Ov, oracle.leading(K), bias=bv)))
     for (w, d, nh, b, g) in ((wq, dq, Hq, bq, qo), (wk, dk, Hkv, bk, ko)):
         O = oracle.expand_map(oracle.qk_halfhead_map(nh, D, keep))
         acc = oracle.qlinear(x, d[0], w.scales, w.zeros, O, oracle.leading(K), bias=b)
@@ -300,6 +315,19 @@ def test_qk_rope_small(B, path, M, keep):
         check_output(g, ref, "f16", TIGHT, "rope keep %d M=%d" % (keep, M))
 
 
+@pytest.mark.parametrize("path", ["auto", "generic"])
+@pytest.mark.parametrize("M", [1, 5, 16, 24, 160])
+@pytest.mark.parametrize("keep,v_keep", [(128, 128), (108, 96), (84, 108), (96, 4)])
+def test_qkv_one_launch(B, path, M, keep, v_keep):
+    """V rides in the launch of Q and K: plain rows beside rotated pairs, its own keep count per head."""
+    B.set_path(B.PATH_AUTO if path == "auto" else B.PATH_GENERIC)
+    rng = np.random.default_rng(170 + keep + M)
+    tol = TIGHT if M < 64 else 5e-4          # M >= 64 takes the tensor-core path (weights rounded to fp16)
+    for dtype in (("f16", "bf16") if M in (5, 160) else ("f16",)):
+        for (g, ref) in run_rope(B, rng, M, 256, 6, 2, 128, keep, 500000.0, dtype, bias=(keep == 96), v_keep=v_keep):
+            check_output(g, ref, dtype, tol, "qkv keep %d/%d M=%d %s" % (keep, v_keep, M, dtype))
+
+
 def test_qk_rope_bf16_table_and_split(B):
     rng = np.random.default_rng(71)
     invf = (1e6 ** (-np.arange(64) / 64.0)) * 0.5          # a caller table (scaled-RoPE variants)
@@ -315,6 +343,8 @@ def test_qk_rope_llama_shape(B, M):
     for keep in (128, 84):
         for (g, ref) in run_rope(B, rng, M, 4096, 32, 8, 128, keep, 500000.0, "f16"):
             check_output(g, ref, "f16", TIGHT, "llama q/k keep %d M=%d" % (keep, M))
+    for (g, ref) in run_rope(B, rng, M, 4096, 32, 8, 128, 96, 500000.0, "f16", v_keep=108):
+        check_output(g, ref, "f16", TIGHT, "llama q/k/v M=%d" % M)
 
 
 # ---------------------------------------------------------------- configuration 2 at full size (sampled rows of the MLP)
