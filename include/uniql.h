@@ -119,6 +119,14 @@ int uniql_unpack_u4(const uint8_t* packed, int64_t N, int64_t K, uint8_t* codes,
 int uniql_dequant(const uint8_t* packed, const void* scales, const void* zeros, int64_t N, int64_t K,
                   int dt, void* w, void* stream);
 
+/* 4-bit embedding table (Section 3.4 applies 4-bit quantisation to the embedding and output layers too):
+ * out[m][0..K) = scale * (code - zero) of table row ids[m], in `dt`, rounded once; the output layer
+ * (lm_head) is uniql_qlinear on a [V][K] matrix.  packed [V][K/2], scales / zeros fp16 [V][K/128];
+ * ids device int32 [M], M <= 65535; out [M][ldo], ldo >= K.  An id outside [0, V) gives a row of zeros and,
+ * when bad_id (device int, may be NULL) is given, sets *bad_id = 1; nothing is read out of bounds. */
+int uniql_embed_rows(const uint8_t* packed, const void* scales, const void* zeros, int64_t V, int64_t K,
+                     const int32_t* ids, int64_t M, int dt, void* out, int64_t ldo, int* bad_id, void* stream);
+
 /* ---- workspace ----
  * The decode kernel may split the input channels over several thread blocks; partial sums
  * and arrival counters live in a workspace.  Calls without a workspace argument use a
@@ -222,7 +230,7 @@ int uniql_qkv_rope_proj(const void* x, int ldx, int dt, const uint8_t* wq, const
                         int ldv, void* workspace, size_t ws_bytes, void* stream);
 
 /* ---- SwiGLU MLP block at decode:  y = ( silu(x Wg^T) * (x Wu^T) ) Wd^T ----
- * (Section 3.1, the MLP block f_MLP(X) = (sigma(X W_g) . X W_u) W_d with sigma(t) = t / (1 + exp(-t)),
+ * (Section 3.2, MLP paragraph: f_MLP(X) = (sigma(X W_g) . X W_u) W_d with sigma(t) = t / (1 + exp(-t)),
  * the gate of the Llama / Qwen blocks the paper compresses; Section 3.4: after sorting, pruning the
  * intermediate dimension keeps the leading k_int channels.)
  * Stored matrices: Wg, Wu [inter][hidden] and Wd [hidden][inter] packed as for uniql_qlinear, scales /

@@ -178,7 +178,7 @@ def qk_halfhead_map(n_heads: int, head_dim: int, head_keep: int) -> list:
 
 
 def swiglu(g, u) -> np.ndarray:
-    """silu(g) * u element by element in fp64 (MLP block of Section 3.1, SiLU gate)."""
+    """silu(g) * u element by element in fp64 (MLP paragraph of Section 3.2, SiLU gate)."""
     gd, ud = _f64(g), _f64(u)
     assert gd.shape == ud.shape
     out = np.empty_like(gd)

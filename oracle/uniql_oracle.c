@@ -150,7 +150,7 @@ int uniql_oracle_rope(const double* in, int64_t R, int64_t n_heads, int64_t n_kv
 }
 
 /* ---- gated activation of the MLP block -------------------------------------------------
- * Section 3.1 writes the MLP block as f_MLP(X) = (sigma(X W_g) (.) X W_u) W_d.  Reading taken
+ * Section 3.2 (MLP paragraph) writes the MLP block as f_MLP(X) = (sigma(X W_g) (.) X W_u) W_d.  Reading taken
  * here: sigma is the SiLU gate of the Llama / Qwen blocks the paper compresses,
  * sigma(t) = t * logistic(t) = t / (1 + exp(-t)), applied element by element.
  * g, u, h: n fp64 values each;  h[i] = sigma(g[i]) * u[i]. */

@@ -64,6 +64,7 @@ _lib.uniql_qlinear.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp]
 _lib.uniql_qkv_rope_proj.argtypes = [_vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i,
                                      _i, _i, _i, _i, _vp, _vp, _d, ctypes.POINTER(_d), _vp, _i, _vp, _i, _vp, _i,
                                      _vp, _sz, _vp]
+_lib.uniql_embed_rows.argtypes = [_vp, _vp, _vp, _i64, _i64, _vp, _i64, _i, _vp, _i64, _vp, _vp]
 _lib.uniql_mlp_workspace_bytes.restype = _sz
 _lib.uniql_mlp_workspace_bytes.argtypes = [_i, _i, _i]
 _lib.uniql_mlp_swiglu_decode.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i,
@@ -77,7 +78,7 @@ _lib.uniql_qk_rope_proj.argtypes = [_vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _
                                     _vp, _vp, _d, ctypes.POINTER(_d), _vp, _i, _vp, _i, _vp, _sz, _vp]
 for _n in ("uniql_set_path", "uniql_pack_u4", "uniql_unpack_u4", "uniql_dequant", "uniql_workspace_init",
            "uniql_workspace_status", "uniql_qlinear", "uniql_qlinear_noalloc", "uniql_qlinear_ex", "uniql_qlinear_multi", "uniql_qk_rope_proj",
-           "uniql_mlp_swiglu_decode", "uniql_qkv_rope_proj"):
+           "uniql_mlp_swiglu_decode", "uniql_qkv_rope_proj", "uniql_embed_rows"):
     getattr(_lib, _n).restype = _i
 
 
@@ -250,3 +251,9 @@ def qkv_rope_proj(x, ldx, wq, sq, zq, wk, sk, zk, wv, sv, zv, bq, bk, bv, M, K, 
                                     n_kv_heads, head_dim, head_keep, v_keep, _ptr(retained_idx), _ptr(pos),
                                     float(theta), f, _ptr(q_out), ldq, _ptr(k_out), ldk, _ptr(v_out), ldv,
                                     _ptr(workspace), ws_bytes, _stream(stream)), "uniql_qkv_rope_proj")
+
+
+def embed_rows(packed, scales, zeros, ids, out, bad_id=None, stream=None) -> None:
+    V, K = packed.shape[0], packed.shape[1] * 2
+    _check(_lib.uniql_embed_rows(_ptr(packed), _ptr(scales), _ptr(zeros), V, K, _ptr(ids), ids.numel(), _dt(out),
+                                 _ptr(out), out.stride(0), _ptr(bad_id), _stream(stream)), "uniql_embed_rows")

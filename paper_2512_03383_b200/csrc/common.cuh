@@ -140,7 +140,7 @@ int decode_supported(const Params& p);
 size_t decode_workspace_bytes(int M, int K, int N_total);
 int decode_status_offset();   // byte offset of the device status word inside a workspace
 size_t decode_workspace_header_bytes();   // counters + status word: the part that must start at zero
-// SwiGLU MLP at decode (Section 3.1: y = (silu(x Wg^T) * (x Wu^T)) Wd^T with the trailing `inter - k_int`
+// SwiGLU MLP at decode (Section 3.2, MLP paragraph: y = (silu(x Wg^T) * (x Wu^T)) Wd^T with the trailing `inter - k_int`
 // sorted intermediate channels pruned): leading k_int rows of Wg, Wu and leading k_int columns of Wd.
 struct MlpDecode {
   const void* x; int ldx;      // [M][hidden] fp16

@@ -259,7 +259,7 @@ __device__ inline void store_tile(const Params& p, const TileFam& f, const TileP
   T* y = reinterpret_cast<T*>(jb.y);
   if (f.mode == kSwiglu) {
     // slots 0..31 hold the gate rows, slots 32..63 the up rows of the same channels:
-    // h = g * sigmoid(g) * u, rounded once (MLP block of Section 3.1 with the SiLU gate)
+    // h = g * sigmoid(g) * u, rounded once (MLP paragraph of Section 3.2, SiLU gate)
     for (int i = etid; i < (RB / 2) * p.M; i += ETH) {
       const int pp = i & (RB / 2 - 1), m = i / (RB / 2);
       const int cc = q.r0 + pp;

@@ -42,6 +42,39 @@ __global__ void dequant_kernel(const uint8_t* __restrict__ packed, const __half*
   }
 }
 
+// Rows ids[m] of a 4-bit table, de-quantised: one block per (token, slice of the row), a thread per packed
+// 32-bit word (eight channels, one 16-byte store).
+template <typename T>
+__global__ void embed_kernel(const uint8_t* __restrict__ packed, const __half* __restrict__ scales,
+                             const __half* __restrict__ zeros, int64_t V, int64_t K, const int32_t* __restrict__ ids,
+                             T* __restrict__ out, int64_t ldo, int* __restrict__ bad) {
+  const int64_t m = blockIdx.y;
+  int64_t row = ids[m];
+  const bool in_range = row >= 0 && row < V;
+  if (!in_range) {
+    if (bad && threadIdx.x == 0 && blockIdx.x == 0) atomicExch(bad, 1);
+    row = 0;                                   // the output row is zero-filled below
+  }
+  const int64_t words = K / 8, G = K / kGroup;
+  const uint32_t* wrow = reinterpret_cast<const uint32_t*>(packed + row * (K / 2));
+  for (int64_t w = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; w < words; w += (int64_t)gridDim.x * blockDim.x) {
+    const uint32_t q = in_range ? __ldg(wrow + w) : 0u;
+    const int64_t g = (w * 8) / kGroup;
+    const float s = in_range ? __half2float(scales[row * G + g]) : 0.f;
+    const float z = __half2float(zeros[row * G + g]);
+    __align__(16) T v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = DT<T>::from_f(s * ((float)((q >> (4 * e)) & 15u) - z));
+    T* o = out + m * ldo + w * 8;
+    if ((reinterpret_cast<uintptr_t>(o) & 15) == 0) {
+      *reinterpret_cast<uint4*>(o) = *reinterpret_cast<const uint4*>(v);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) o[e] = v[e];
+    }
+  }
+}
+
 inline int grid_for(int64_t n, int threads) {
   int64_t b = (n + threads - 1) / threads;
   if (b < 1) b = 1;
@@ -87,5 +120,28 @@ extern "C" int uniql_dequant(const uint8_t* packed, const void* scales, const vo
   else
     dequant_kernel<__nv_bfloat16><<<grid_for(nb, 256), 256, 0, (cudaStream_t)stream>>>(
         packed, (const __half*)scales, (const __half*)zeros, N, K, (__nv_bfloat16*)w);
+  return cudaGetLastError() == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
+}
+
+extern "C" int uniql_embed_rows(const uint8_t* packed, const void* scales, const void* zeros, int64_t V, int64_t K,
+                                const int32_t* ids, int64_t M, int dt, void* out, int64_t ldo, int* bad_id,
+                                void* stream) {
+  if (!packed || !scales || !zeros || !ids || !out) return UNIQL_ERR_NULL;
+  if (V < 1 || K < kGroup || (K % kGroup) || M < 0 || ldo < K) return UNIQL_ERR_SHAPE;
+  if (M > 65535) return UNIQL_ERR_SHAPE;
+  if (dt != UNIQL_F16 && dt != UNIQL_BF16) return UNIQL_ERR_DTYPE;
+  if ((((uintptr_t)packed) & 3) || (((uintptr_t)ids) & 3) || (((uintptr_t)out) & 1) || (bad_id && (((uintptr_t)bad_id) & 3)))
+    return UNIQL_ERR_ALIGN;
+  if (M == 0) return UNIQL_OK;
+  const int threads = 128;
+  int bx = (int)((K / 8 + threads - 1) / threads);
+  if (bx > 64) bx = 64;
+  dim3 grid(bx, (unsigned)M);
+  if (dt == UNIQL_F16)
+    embed_kernel<__half><<<grid, threads, 0, (cudaStream_t)stream>>>(packed, (const __half*)scales, (const __half*)zeros,
+                                                                      V, K, ids, (__half*)out, ldo, bad_id);
+  else
+    embed_kernel<__nv_bfloat16><<<grid, threads, 0, (cudaStream_t)stream>>>(
+        packed, (const __half*)scales, (const __half*)zeros, V, K, ids, (__nv_bfloat16*)out, ldo, bad_id);
   return cudaGetLastError() == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
 }

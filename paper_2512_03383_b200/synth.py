@@ -174,11 +174,18 @@ def map_qk_halfheads(n_heads: int, head_dim: int, head_keep: int) -> List[Family
 
 
 def map_mamba_in_proj(d_inner: int, headdim: int, head_keep: int, d_state: int, ngroups: int,
-                      nheads: int) -> List[Family]:
-    """Mamba2 in_proj rows in the order z, x, B, C, dt; z and x pruned per SSM head."""
-    bc_dt = 2 * ngroups * d_state + nheads
+                      nheads: int, state_keep: Optional[int] = None) -> List[Family]:
+    """Mamba2 in_proj rows in the order z, x, B, C, dt; z and x pruned per SSM head.  With state_keep the
+    state dimension D_s is pruned too: every group of B and of C keeps its leading state_keep rows."""
+    if state_keep is None or state_keep == d_state:
+        bc_dt = 2 * ngroups * d_state + nheads
+        return [(0, headdim, head_keep, nheads), (d_inner, headdim, head_keep, nheads),
+                (2 * d_inner, bc_dt, bc_dt, 1)]
+    b0 = 2 * d_inner
+    c0 = b0 + ngroups * d_state
+    dt0 = c0 + ngroups * d_state
     return [(0, headdim, head_keep, nheads), (d_inner, headdim, head_keep, nheads),
-            (2 * d_inner, bc_dt, bc_dt, 1)]
+            (b0, d_state, state_keep, ngroups), (c0, d_state, state_keep, ngroups), (dt0, nheads, nheads, 1)]
 
 
 def map_size(fams: List[Family]) -> int:

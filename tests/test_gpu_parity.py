@@ -224,6 +224,27 @@ def test_mamba_shaped_maps(B, M):
         check_output(y2, ref2, "f16", TIGHT, "mamba out_proj keep %d" % keep)
 
 
+@pytest.mark.parametrize("M", [1, 16, 200])
+@pytest.mark.parametrize("ngroups,nheads", [(1, 8), (2, 16)])
+def test_mamba_state_dimension_pruning(B, M, ngroups, nheads):
+    """D_s pruning (Section 3.2, SSM paragraph: B and C are sorted along the state dimension per group): in_proj
+    rows z|x|B|C|dt with z, x pruned per head and every group of B and C cut to its leading state_keep rows.
+    ngroups > 1 is the layout of the hybrid models (several B/C groups shared by blocks of heads)."""
+    rng = np.random.default_rng(45 + M + ngroups)
+    headdim, d_state = 64, 128
+    d_inner = nheads * headdim
+    rows = 2 * d_inner + 2 * ngroups * d_state + nheads
+    qin = synth.draw_qweight(rng, rows, 256)
+    din = dev_weight(qin)
+    dtype = "f16" if M <= 16 else "bf16"
+    for keep, sk in ((64, 96), (48, 64), (56, 128), (64, 4)):
+        om = synth.map_mamba_in_proj(d_inner, headdim, keep, d_state, ngroups, nheads, state_keep=sk)
+        assert synth.map_size(om) == 2 * nheads * keep + 2 * ngroups * sk + nheads
+        x = synth.draw_x(rng, M, 256, dtype)
+        y, ref = run_ex(B, qin, din, x, dtype, None, 256, om, 0)
+        check_output(y, ref, dtype, TIGHT if M <= 16 else 5e-4, "mamba in_proj keep %d state %d M=%d" % (keep, sk, M))
+
+
 def test_noninteger_zero_points_and_symmetric(B):
     rng = np.random.default_rng(50)
     qw = synth.draw_qweight(rng, 64, 512, symmetric=True)

@@ -270,7 +270,7 @@ def test_rope_rejects_bad_arguments():
         oracle.rope(np.zeros((1, 2)), 1, 1, 4, 2, np.array([[2]], dtype=np.int32), [0], 10.0)
 
 
-# ------------------------------------------------------------------ gated MLP block (Section 3.1)
+# ------------------------------------------------------------------ gated MLP block (Section 3.2, MLP paragraph)
 def test_swiglu_closed_forms_and_library_logistic():
     from scipy.special import expit                       # the library's logistic function
     # literal values: silu(0) = 0, silu(ln 3) = ln 3 * 3/4, silu(-ln 3) = -ln 3 / 4
