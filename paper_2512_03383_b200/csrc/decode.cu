@@ -88,7 +88,8 @@ struct Phase {
   const void* x;         // activations [M][ldx]
   long long ldx;
   int K;                 // stored input channels of the phase's matrices
-  int start, keep;       // leading input family (128-bit staging)
+  int start, keep;       // the input family (128-bit staging): head h keeps [start + h*period, +keep)
+  int period, count;     // count = 1: a leading block
   int g_total, v_first;  // visited groups and the first of them
   int tile0, tiles;      // global tiles [tile0, tile0 + tiles)
 };
@@ -690,6 +691,14 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     const int Gk = pc.Gk, sg_lo = pc.sg_lo;
     const T* x = reinterpret_cast<const T*>(P.x);
     const long long ldx = P.ldx;
+    // stored channel (a multiple of 8) -> compact activation column, or -1 when the channel is pruned
+    auto compact_of = [&](int ch) -> int {
+      int r = ch - P.start;
+      if (r < 0) return -1;
+      int h = 0;
+      if (P.count > 1) { h = r / P.period; r -= h * P.period; if (h >= P.count) return -1; }
+      return r < P.keep ? h * P.keep + r : -1;
+    };
     // activations a previous phase of this launch wrote are read past the non-coherent cache
     auto load16 = [&](const T* ptr) -> uint4 {
       return (NPH > 1 && ph > 0) ? __ldcg(reinterpret_cast<const uint4*>(ptr)) : __ldg(reinterpret_cast<const uint4*>(ptr));
@@ -716,7 +725,6 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       // x_i = 256 * hi + lo with both bytes signed; the bytes go to two "virtual"
       // batch rows (columns 2m and 2m+1 of the int8 MMA), in the order the nibbles leave a weight word:
       // even codes in the first register of a word's pair, odd codes in the second.
-      const int start = P.start, keep = P.keep;
       const int n_units = Gn * p.M * 16;
       unsigned char* xb = smem + c.off_x;
       constexpr int UN = 4;
@@ -728,8 +736,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           in[q4] = make_uint4(0, 0, 0, 0);
           if (u < n_units) {
             const int pair = u >> 4, m = pair / Gn, lv = needed_group(pair - m * Gn);
-            const int t0 = (sg_lo + lv) * kGroup + 8 * (u & 15) - start;
-            if (lv < Gk && t0 >= 0 && t0 < keep) in[q4] = load16(x + (size_t)m * ldx + t0);
+            const int t0 = compact_of((sg_lo + lv) * kGroup + 8 * (u & 15));
+            if (lv < Gk && t0 >= 0) in[q4] = load16(x + (size_t)m * ldx + t0);
           }
         }
 #pragma unroll
@@ -779,7 +787,6 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         }
       }
     } else if (c.x_vec) {
-      const int start = P.start, keep = P.keep;
       const int n_units = Gn * p.M * 16;
       constexpr int UN = 4;                                        // loads in flight per thread
       for (int u0 = ctid; u0 < ((n_units + 31) & ~31); u0 += CTH * UN) {   // whole warps stay in the shuffles
@@ -790,8 +797,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           in[q4] = make_uint4(0, 0, 0, 0);
           if (u < n_units) {
             const int pair = u >> 4, m = pair / Gn, lv = needed_group(pair - m * Gn);
-            const int t0 = (sg_lo + lv) * kGroup + 8 * (u & 15) - start;
-            if (lv < Gk && t0 >= 0 && t0 < keep) in[q4] = load16(x + (size_t)m * ldx + t0);
+            const int t0 = compact_of((sg_lo + lv) * kGroup + 8 * (u & 15));
+            if (lv < Gk && t0 >= 0) in[q4] = load16(x + (size_t)m * ldx + t0);
           }
         }
 #pragma unroll
@@ -1387,8 +1394,9 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   visited_range(p.imap, gran, &v_first, &g_total);
   const int MT = p.M <= 8 ? 1 : 2;
   // 128-bit staging: one leading family, everything 8-element aligned
-  c.x_vec = p.imap.n_fam == 1 && p.imap.fam[0].count == 1 && (p.imap.fam[0].start % 8) == 0 &&
-            (p.imap.fam[0].keep % 8) == 0 && (p.ldx % 8) == 0 && ((((uintptr_t)p.x) & 15) == 0);
+  c.x_vec = p.imap.n_fam == 1 && (p.imap.fam[0].start % 8) == 0 && (p.imap.fam[0].keep % 8) == 0 &&
+            (p.imap.fam[0].count == 1 || (p.imap.fam[0].period % 8) == 0) && (p.ldx % 8) == 0 &&
+            ((((uintptr_t)p.x) & 15) == 0);
   if (count_tile_fams(p) > kMaxTF) return UNIQL_ERR_UNSUPPORTED;
 
   // integer path: fp16 activations staged with 128-bit loads (a leading input block); UNIQL_DECODE_I8=0: fp16 MMAs
@@ -1462,6 +1470,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
     Phase& P = c.ph[0];
     P.x = p.x; P.ldx = p.ldx; P.K = p.K;
     P.start = p.imap.fam[0].start; P.keep = p.imap.fam[0].keep;
+    P.period = p.imap.fam[0].period; P.count = p.imap.fam[0].count;
     P.g_total = g_total; P.v_first = v_first;
     P.tile0 = 0; P.tiles = tiles;
   }
@@ -1562,12 +1571,13 @@ int launch_mlp_phases(const MlpDecode& d, int first, int count, const LaunchCfg&
     int rc;
     if (ph == 0) {
       P.x = d.x; P.ldx = d.ldx; P.K = d.hidden; P.start = 0; P.keep = d.hidden; P.g_total = d.hidden / kGroup;
+      P.period = d.hidden; P.count = 1;
       f.mode = kSwiglu; f.job = 0; f.job2 = 1; f.keep = d.k_int; f.period = d.inter;
       f.tpb = (d.k_int + RB / 2 - 1) / (RB / 2);
       rc = encode_family(&c.wmap[n_tf], d.wg, d.hidden, d.hidden / 2, d.k_int, 1, d.k_int, RB / 2);
       if (!rc) rc = encode_family(&c.wmap_up, d.wu, d.hidden, d.hidden / 2, d.k_int, 1, d.k_int, RB / 2);
     } else {
-      P.x = d.h; P.ldx = d.ldh; P.K = d.inter; P.start = 0; P.keep = d.k_int;
+      P.x = d.h; P.ldx = d.ldh; P.K = d.inter; P.start = 0; P.keep = d.k_int; P.period = d.inter; P.count = 1;
       P.g_total = (d.k_int + kGroup - 1) / kGroup;
       const int rows = narrow ? RB / 2 : RB;
       f.mode = narrow ? kNarrow : kPlain; f.job = 2; f.job2 = 2; f.keep = d.hidden; f.period = d.hidden;

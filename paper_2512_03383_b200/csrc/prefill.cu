@@ -61,7 +61,9 @@ struct PrefillCfg {
   int n_ttiles;              // token tiles
   int wtile_begin[kMaxPJobs + 1];   // first weight tile of each job
   int n_tiles;               // weight tiles (all jobs) x token tiles
-  int n_kb;                  // k-blocks of 64 (k_in rounded up)
+  int n_kb;                  // visited k-blocks of 64: kept blocks of every head, head after head
+  int km_start, km_period;   // input map in k-blocks: first stored block of head 0, stored blocks per head
+  int km_kbh, km_keep;       // kept k-blocks per head (the last may be partly kept), kept channels per head
   uint32_t idesc;
   int streamk;               // 1: contiguous ranges of (tile, k-block) units per block; 0: whole tiles round-robin
   int* status;
@@ -75,6 +77,21 @@ struct PrefillCfg {
 // tiles remain.  Blocks stay in step along k (few distinct k offsets are alive at a time, which keeps the
 // activation slices in L2).  A left-over tile is finished by the last of its blocks to arrive (fp32 partial
 // tiles in the workspace, added in block order).
+// Visited k-block v of the input map -> stored k-block, first compact activation column, kept channels in it.
+// One family {start, period, keep, count}: head h keeps channels [0, keep) of its period; a leading block is
+// the case count = 1.  The activation box of a partly kept block also covers the first columns of the next
+// head: the de-quantisers write zeros for the pruned channels of the block, so those columns do not count.
+struct KBlock { int stored, xcol, valid; };
+__device__ inline KBlock kblock_of(const PrefillCfg& c, int v) {
+  int h = 0, r = v;
+  if (v >= c.km_kbh) { h = v / c.km_kbh; r = v - h * c.km_kbh; }
+  KBlock k;
+  k.stored = c.km_start + h * c.km_period + r;
+  k.xcol = h * c.km_keep + r * BK;
+  k.valid = min(BK, c.km_keep - r * BK);
+  return k;
+}
+
 struct Seg { int tile, kb0, kb1, tail_idx; };     // tail_idx: -1 whole-tile round, else index among the block's tail segments
 struct SegIter {
   long u, ue;
@@ -339,7 +356,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
           if (it >= PSTAGES && !pmbar_wait(empty + 8 * s, par, abort_flag, true)) { failed = true; break; }
           const uint32_t fb = full_b + 8 * s;
           pmbar_expect_tx(fb, (uint32_t)(c.bn * BK * 2));
-          tma_box2(sbase + s * PSTAGE_BYTES + A_BYTES, &c.xmap, kb * BK, tt * c.bn, fb);
+          tma_box2(sbase + s * PSTAGE_BYTES + A_BYTES, &c.xmap, kblock_of(c, kb).xcol, tt * c.bn, fb);
           if (++s == PSTAGES) { s = 0; par ^= 1; }
         }
       }
@@ -401,15 +418,17 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
       // codes and scale / zero-point of this team's next two k-blocks are kept in registers
       uint4 q0 = make_uint4(0, 0, 0, 0), q1 = q0;
       __half s0 = __ushort_as_half(0), z0 = s0, s1 = s0, z1 = s0;
+      int v0 = 0, v1 = 0;              // kept channels of the k-blocks held in q0 / q1
+      // codes, scale and zero-point of visited k-block v of this thread's row; `valid` channels of it are kept
+      auto fetch = [&](int v, uint4& q, __half& sc, __half& zr, int& valid) {
+        const KBlock kbk = kblock_of(c, v);
+        valid = kbk.valid;
+        q = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)kbk.stored * 32));
+        sc = __ldg(srow + (kbk.stored >> 1)); zr = __ldg(zrow + (kbk.stored >> 1));
+      };
       if (live) {
-        if (kb0 < sg.kb1) {
-          q0 = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)kb0 * 32));
-          s0 = __ldg(srow + (kb0 >> 1)); z0 = __ldg(zrow + (kb0 >> 1));
-        }
-        if (kb0 + 2 < sg.kb1) {
-          q1 = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)(kb0 + 2) * 32));
-          s1 = __ldg(srow + ((kb0 + 2) >> 1)); z1 = __ldg(zrow + ((kb0 + 2) >> 1));
-        }
+        if (kb0 < sg.kb1) fetch(kb0, q0, s0, z0, v0);
+        if (kb0 + 2 < sg.kb1) fetch(kb0 + 2, q1, s1, z1, v1);
       }
       for (int kb = kb0; kb < sg.kb1; kb += 2) {
         const int it = it0 + kb;
@@ -417,10 +436,8 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         const uint32_t use = (uint32_t)(it / PSTAGES);
         uint4 q2 = make_uint4(0, 0, 0, 0);
         __half s2 = s1, z2 = z1;
-        if (live && kb + 4 < sg.kb1) {
-          q2 = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)(kb + 4) * 32));
-          s2 = __ldg(srow + ((kb + 4) >> 1)); z2 = __ldg(zrow + ((kb + 4) >> 1));
-        }
+        int v2 = 0;
+        if (live && kb + 4 < sg.kb1) fetch(kb + 4, q2, s2, z2, v2);
         if (it >= PSTAGES && !pmbar_wait(empty + 8 * s, (use - 1) & 1, abort_flag)) { failed = true; break; }
         const uint32_t a_st = sbase + s * PSTAGE_BYTES + row_off;
         const __half2 sh2 = __half2half2(s0);
@@ -428,7 +445,8 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         const uint32_t qw[4] = {q0.x, q0.y, q0.z, q0.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const uint4 o = live ? dequant_word(qw[j], sh2, cz2) : make_uint4(0, 0, 0, 0);
+          // (eight channels per word; keep counts are multiples of eight, so a word is kept or pruned whole)
+          const uint4 o = (live && hf * 32 + j * 8 < v0) ? dequant_word(qw[j], sh2, cz2) : make_uint4(0, 0, 0, 0);
           asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a_st + col_off[j]), "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w) : "memory");
         }
         if constexpr (CONV) {
@@ -446,8 +464,8 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         fence_async_smem();            // generic-proxy writes must be visible to the tensor core (async proxy)
         __syncwarp();
         if (lane == 0) pmbar_arrive(full_a + 8 * s);
-        q0 = q1; s0 = s1; z0 = z1;
-        q1 = q2; s1 = s2; z1 = z2;
+        q0 = q1; s0 = s1; z0 = z1; v0 = v1;
+        q1 = q2; s1 = s2; z1 = z2; v1 = v2;
       }
     }
   } else if (warp >= EPI_WARP0) {
@@ -640,11 +658,20 @@ int launch_pt(const Params& p, const PrefillCfg& c, int grid, cudaStream_t strea
 }  // namespace
 
 // The tensor-core path takes: the leading k_in input channels (the hidden dimension D_h is never pruned,
-// D_int is pruned as a leading block: Section 3.4), any output map, both activation types.
+// D_int is pruned as a leading block: Section 3.4) or one family of per-head kept blocks (the input side of
+// o_proj / out_proj: heads on 64-channel boundaries, keep a multiple of 8), any output map, both activation types.
 int prefill_supported(const Params& p) {
   if (p.M < 17) return 0;
   if (p.dt != UNIQL_F16 && p.dt != UNIQL_BF16) return 0;
-  if (p.imap.n_fam != 1 || p.imap.fam[0].count != 1 || p.imap.fam[0].start != 0) return 0;
+  if (p.imap.n_fam != 1) return 0;
+  {
+    const Fam& a = p.imap.fam[0];
+    if (a.count == 1) {
+      if (a.start != 0) return 0;
+    } else if ((a.start % BK) != 0 || (a.period % BK) != 0 || (a.keep % 8) != 0) {
+      return 0;                    // per-head input maps: heads on k-block boundaries, 16-byte activation boxes
+    }
+  }
   if ((p.ldx % 8) != 0 || (((uintptr_t)p.x) & 15) != 0) return 0;       // TMA: 16-byte base and row pitch
   if ((p.K % kGroup) != 0) return 0;
   return 1;
@@ -663,7 +690,14 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   for (int j = p.n_jobs; j <= kMaxPJobs; ++j) c.wtile_begin[j] = wt;
   c.n_tiles = wt * c.n_ttiles;
   if (c.n_tiles < 1) return UNIQL_ERR_SHAPE;
-  c.n_kb = (p.k_in + BK - 1) / BK;
+  {
+    const Fam& a = p.imap.fam[0];
+    c.km_start = a.start / BK;
+    c.km_period = a.count > 1 ? a.period / BK : 0;
+    c.km_keep = a.keep;
+    c.km_kbh = (a.keep + BK - 1) / BK;
+    c.n_kb = c.km_kbh * a.count;
+  }
   const uint32_t fmt = 0u;      // both operands fp16 (bf16 activations are converted in shared memory)
   // instruction descriptor: fp32 accumulate, A and B of the activation type, both K-major, N = bn, M = 128
   c.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(c.bn >> 3) << 17) | ((uint32_t)(BMW >> 4) << 24);

@@ -201,6 +201,17 @@ def test_per_head_maps(B, M):
         x = synth.draw_x(rng, M, synth.map_size(in_map), "f16")
         y, ref = run_ex(B, qw, dw, x, "f16", in_map, 0, out_map, 0, ldx_pad=5)
         check_output(y, ref, "f16", TIGHT, "per-head keep %d M=%d" % (keep, M))
+    # keep counts and a row pitch in multiples of 8: the 128-bit staging (integer path at M <= 16) maps every
+    # eight-channel unit through the head structure
+    for (hd, keep) in ((128, 96), (128, 104), (128, 64), (64, 8), (256, 200)):
+        in_map = synth.map_per_head(1024 // hd, hd, keep)
+        x = synth.draw_x(rng, M, synth.map_size(in_map), "f16")
+        y, ref = run_ex(B, qw, dw, x, "f16", in_map, 0, None, 512, ldx_pad=8)
+        check_output(y, ref, "f16", TIGHT, "per-head keep %d of %d M=%d" % (keep, hd, M))
+    in_map = [(256, 128, 96, 5)]                    # first head not at channel 0
+    x = synth.draw_x(rng, M, synth.map_size(in_map), "f16")
+    y, ref = run_ex(B, qw, dw, x, "f16", in_map, 0, None, 512)
+    check_output(y, ref, "f16", TIGHT, "offset per-head map M=%d" % M)
 
 
 @pytest.mark.parametrize("M", [1, 16])

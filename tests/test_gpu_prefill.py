@@ -104,6 +104,40 @@ def test_prefill_bf16_converted_in_kernel(B, monkeypatch):
     assert torch.equal(y1, y2)
 
 
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("M", [64, 200])
+@pytest.mark.parametrize("grid", [0, 3])
+def test_prefill_per_head_input_maps(B, monkeypatch, M, dtype, grid):
+    """The input side of o_proj / out_proj: every head keeps its leading channels.  Heads of 128 and of 64
+    channels; keep counts that end a head on a k-block boundary (128, 64), inside its second block (104, 96),
+    inside its first (40, 8): a partly kept block reads the next head's activations against zero weights."""
+    B.set_path(B.PATH_PREFILL)
+    if grid:
+        monkeypatch.setenv("UNIQL_PREFILL_STREAMK", "1")
+        monkeypatch.setenv("UNIQL_PREFILL_GRID", str(grid))
+    rng = np.random.default_rng(950 + M)
+    qw = synth.draw_qweight(rng, 200, 1024)
+    dw = dev_weight(qw)
+    for (hd, keep) in ((128, 128), (128, 104), (128, 96), (128, 64), (128, 40), (64, 64), (64, 48), (64, 8)):
+        im = synth.map_per_head(1024 // hd, hd, keep)
+        x = synth.draw_x(rng, M, synth.map_size(im), dtype)
+        y, ref = run_ex(B, qw, dw, x, dtype, im, 0, None, 200, ldx_pad=8)
+        check_output(y, ref, dtype, TOL[dtype], "per-head input map %d/%d M=%d" % (keep, hd, M))
+    # a map whose first head does not start at channel 0, with per-head output rows as well
+    im = [(256, 128, 96, 5)]
+    om = synth.map_per_head(3, 64, 56)
+    x = synth.draw_x(rng, M, synth.map_size(im), dtype)
+    y, ref = run_ex(B, qw, dw, x, dtype, im, 0, om, 0, ldx_pad=8)
+    check_output(y, ref, dtype, TOL[dtype], "offset per-head input map")
+    assert B.workspace_status() == 0
+    # not on the tensor-core path: keep counts that are not multiples of 8 (the call falls back to the generic kernel)
+    B.set_path(B.PATH_AUTO)
+    im = synth.map_per_head(8, 128, 108)
+    x = synth.draw_x(rng, M, synth.map_size(im), dtype)
+    y, ref = run_ex(B, qw, dw, x, dtype, im, 0, None, 200)
+    check_output(y, ref, dtype, TOL[dtype], "keep 108 via auto")
+
+
 @pytest.mark.parametrize("grid", [1, 3, 5, 7, 11])
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
 def test_prefill_stream_k(B, monkeypatch, grid, dtype):
