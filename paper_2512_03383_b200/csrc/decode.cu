@@ -116,6 +116,14 @@ struct DecodeCfg {
   float* partials;
   int* status;
   int* grid_sync;        // two ints: epilogue warps that finished phase 0, blocks that saw all of them
+  // Streamed activations (rows too long to stage whole beside the ring): a small kernel quantises x once
+  // into the layout the consumers read, [group][virtual row][128 bytes] plus (integer sum, 2^-e) per (group,
+  // batch row), and every stage of the ring carries the eight groups of its unit beside the weights.
+  int x_stream;
+  int stage_bytes;       // STAGE_BYTES, plus vr * CG * 128 + 1024 when the activations are streamed
+  int vr;                // virtual rows per group in a stage: 8 (up to four batch rows) or 16
+  const float2* xg_glob; // [group][8] (integer sum, 2^-e)
+  CUtensorMap xmap;      // quantised activations: (byte in line, virtual row, group), 128-byte swizzle
 };
 
 // ---------------------------------------------------------------------------------------- PTX helpers
@@ -151,6 +159,11 @@ __device__ inline void tma_box3(uint32_t dst, const CUtensorMap* tm, int x, int 
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
       ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+// contiguous bytes (a multiple of 16, both sides 16-byte aligned) into shared memory, counted on `bar`
+__device__ inline void bulk_copy(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 __device__ inline void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -224,6 +237,86 @@ __device__ inline float2 lds64f(uint32_t addr) {
 }
 // exact int -> float for |v| < 2^22 without the conversion unit
 __device__ inline float small_int_to_float(int v) { return __int_as_float(v + 0x4B400000) - 12582912.f; }
+
+// Sixteen consecutive lanes hold the 128 activations of one (batch row, group), eight each (`in`): 16-bit fixed
+// point against the group's maximum, x_i = rint(x * 2^e) = 256 * hi + lo with both bytes signed.  Returns this
+// lane's bytes in the order the nibbles leave a weight word (even codes first), the group's integer sum and
+// 2^-e.  Every lane of the warp must call it (shuffles over the sixteen lanes).
+__device__ inline void quantise16(const uint4& in, uint2& hi2, uint2& lo2, int& isum_out, float& inv_scale_out) {
+  const __half2* h2 = reinterpret_cast<const __half2*>(&in);
+  float f[8];
+  float amax = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 v = __half22float2(h2[i]);
+    f[2 * i] = v.x; f[2 * i + 1] = v.y;
+    amax = fmaxf(amax, fmaxf(fabsf(v.x), fabsf(v.y)));
+  }
+#pragma unroll
+  for (int o2 = 8; o2 >= 1; o2 >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o2));
+  int e = 0;
+  if (amax > 0.f && amax < 3.0e38f) {
+    e = 14 - ((int)((__float_as_uint(amax) >> 23) & 255u) - 127);
+    if (amax * __uint_as_float((uint32_t)(127 + e) << 23) > 32639.f) --e;     // keep the high byte of x_i + 128 signed
+  }
+  const float scale = __uint_as_float((uint32_t)(127 + e) << 23), inv_scale = __uint_as_float((uint32_t)(127 - e) << 23);
+  int isum = 0;
+  uint32_t hi_e = 0, hi_o = 0, lo_e = 0, lo_o = 0;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const int xi = __float2int_rn(f[k] * scale);
+    isum += xi;
+    const int hi = (xi + 128) >> 8, lo = xi - (hi << 8);
+    const int sh = 8 * (k >> 1);
+    if (k & 1) { hi_o |= (uint32_t)(hi & 255) << sh; lo_o |= (uint32_t)(lo & 255) << sh; }
+    else       { hi_e |= (uint32_t)(hi & 255) << sh; lo_e |= (uint32_t)(lo & 255) << sh; }
+  }
+#pragma unroll
+  for (int o2 = 8; o2 >= 1; o2 >>= 1) isum += __shfl_xor_sync(0xffffffffu, isum, o2);
+  hi2 = make_uint2(hi_e, hi_o);
+  lo2 = make_uint2(lo_e, lo_o);
+  isum_out = isum;
+  inv_scale_out = inv_scale;
+}
+
+// stored input channel (a multiple of 8) -> compact activation column, or -1 when the channel is pruned
+__device__ inline int compact_channel(const Phase& P, int ch) {
+  int r = ch - P.start;
+  if (r < 0) return -1;
+  int h = 0;
+  if (P.count > 1) { h = r / P.period; r -= h * P.period; if (h >= P.count) return -1; }
+  return r < P.keep ? h * P.keep + r : -1;
+}
+
+// Quantises the activations of one launch once (streamed mode): half-warp (batch row m, visited group lv).
+// Rows m >= M of the vr / 2 row slots are written as zeros.
+__global__ void __launch_bounds__(256) xquant_kernel(const Phase P, int M, int vr, int g_total, unsigned char* xq,
+                                                     float2* xg) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");            // x may come from the preceding kernel
+  const int rows = vr >> 1;
+  const int n_units = g_total * rows * 16;
+  const __half* x = reinterpret_cast<const __half*>(P.x);
+  for (int u = blockIdx.x * blockDim.x + threadIdx.x; u < ((n_units + 31) & ~31); u += gridDim.x * blockDim.x) {
+    const int u16 = u & 15, pair = u < n_units ? u >> 4 : 0;
+    const int lv = pair / rows, m = pair - lv * rows;
+    uint4 in = make_uint4(0, 0, 0, 0);
+    if (u < n_units && m < M) {
+      const int t0 = compact_channel(P, (P.v_first + lv) * kGroup + 8 * u16);
+      if (t0 >= 0) in = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * P.ldx + t0));
+    }
+    uint2 hi2, lo2;
+    int isum;
+    float inv_scale;
+    quantise16(in, hi2, lo2, isum, inv_scale);
+    if (u < n_units) {
+      const int off = (u16 >> 2) * 32 + (u16 & 3) * 8;
+      *reinterpret_cast<uint2*>(xq + ((size_t)lv * vr + 2 * m) * 128 + off) = hi2;
+      *reinterpret_cast<uint2*>(xq + ((size_t)lv * vr + 2 * m + 1) * 128 + off) = lo2;
+      if (u16 == 0) xg[lv * 8 + m] = make_float2((float)isum, inv_scale);
+    }
+  }
+}
 
 // ---------------------------------------------------------------------------------------- tile geometry
 struct TilePos { int fi, h, r0; };
@@ -439,6 +532,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     int it = 0, s = 0;
     uint32_t ring_parity = 1;      // parity of the previous use of ring position s
     bool ok = true;
+    // streamed activations are written by the kernel launched just before this one
+    if (NPH == 1 && c.x_stream) asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int ph = 0; ph < NPH && ok; ++ph) {
       const PhaseCtx pc = (NPH == 1 || ph == 0) ? pc0 : phase_ctx(c, ph, kp, rp);
       const Work& wk = pc.wk;
@@ -489,10 +584,16 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         const int ng = min(CG, ng_all), ng2 = ng_all - ng;  // ... in row slots 0..31 (all 64 unless narrow) / 32..63
         const int nb = (ng + 1) >> 1, nb2 = (ng2 + 1) >> 1; // 128-byte columns with a visited group
         const uint32_t full = bar_full + 8 * s;
-        const uint32_t st = sbase + (uint32_t)s * STAGE_BYTES;
+        const uint32_t st = sbase + (uint32_t)s * (uint32_t)c.stage_bytes;
+        const uint32_t xbytes = (NPH == 1 && c.x_stream) ? (uint32_t)(c.vr * CG * 128 + CG * 64) : 0u;
         if (lane == 0)
-          mbar_expect_tx(full, mode == kNarrow ? (uint32_t)((nb + nb2) * (BOX_BYTES / 2)) : (uint32_t)(nb * BOX_BYTES));
+          mbar_expect_tx(full, xbytes + (mode == kNarrow ? (uint32_t)((nb + nb2) * (BOX_BYTES / 2)) : (uint32_t)(nb * BOX_BYTES)));
         __syncwarp();
+        if (xbytes && lane == 31) {
+          const int lv0 = chunk * CG;                                // (one k-part, wide tiles)
+          tma_box3(st + STAGE_BYTES, &c.xmap, 0, 0, lv0, full);
+          bulk_copy(st + STAGE_BYTES + (uint32_t)(c.vr * CG * 128), c.xg_glob + (size_t)lv0 * 8, CG * 64, full);
+        }
         if (lane < nb) {
           const int xb = (sg_lo + chunk * c.cgz + 2 * lane) * 64;    // byte in the weight row
           const uint32_t dst = st + (uint32_t)lane * BOX_BYTES;
@@ -691,14 +792,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     const int Gk = pc.Gk, sg_lo = pc.sg_lo;
     const T* x = reinterpret_cast<const T*>(P.x);
     const long long ldx = P.ldx;
-    // stored channel (a multiple of 8) -> compact activation column, or -1 when the channel is pruned
-    auto compact_of = [&](int ch) -> int {
-      int r = ch - P.start;
-      if (r < 0) return -1;
-      int h = 0;
-      if (P.count > 1) { h = r / P.period; r -= h * P.period; if (h >= P.count) return -1; }
-      return r < P.keep ? h * P.keep + r : -1;
-    };
+    auto compact_of = [&](int ch) -> int { return compact_channel(P, ch); };
     // activations a previous phase of this launch wrote are read past the non-coherent cache
     auto load16 = [&](const T* ptr) -> uint4 {
       return (NPH > 1 && ph > 0) ? __ldcg(reinterpret_cast<const uint4*>(ptr)) : __ldg(reinterpret_cast<const uint4*>(ptr));
@@ -747,41 +841,15 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           const int u16 = u & 15, pair = u < n_units ? u >> 4 : 0;
           const int m = pair / Gn, lv = needed_group(pair - m * Gn);
           const bool in_range = u < n_units && lv < Gk;
-          const __half2* h2 = reinterpret_cast<const __half2*>(&in[q4]);
-          float f[8];
-          float amax = 0.f;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float2 v = __half22float2(h2[i]);
-            f[2 * i] = v.x; f[2 * i + 1] = v.y;
-            amax = fmaxf(amax, fmaxf(fabsf(v.x), fabsf(v.y)));
-          }
-#pragma unroll
-          for (int o2 = 8; o2 >= 1; o2 >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o2));
-          int e = 0;
-          if (amax > 0.f && amax < 3.0e38f) {
-            e = 14 - ((int)((__float_as_uint(amax) >> 23) & 255u) - 127);
-            if (amax * __uint_as_float((uint32_t)(127 + e) << 23) > 32639.f) --e;     // keep the high byte of x_i + 128 signed
-          }
-          const float scale = __uint_as_float((uint32_t)(127 + e) << 23), inv_scale = __uint_as_float((uint32_t)(127 - e) << 23);
-          int isum = 0;
-          uint32_t hi_e = 0, hi_o = 0, lo_e = 0, lo_o = 0;
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const int xi = __float2int_rn(f[k] * scale);
-            isum += xi;
-            const int hi = (xi + 128) >> 8, lo = xi - (hi << 8);
-            const int sh = 8 * (k >> 1);
-            if (k & 1) { hi_o |= (uint32_t)(hi & 255) << sh; lo_o |= (uint32_t)(lo & 255) << sh; }
-            else       { hi_e |= (uint32_t)(hi & 255) << sh; lo_e |= (uint32_t)(lo & 255) << sh; }
-          }
-#pragma unroll
-          for (int o2 = 8; o2 >= 1; o2 >>= 1) isum += __shfl_xor_sync(0xffffffffu, isum, o2);
+          uint2 hi2, lo2;
+          int isum;
+          float inv_scale;
+          quantise16(in[q4], hi2, lo2, isum, inv_scale);
           if (in_range) {
             // word j of lane quarter c' (u16 = c'*4 + j): 8 bytes at c'*32 + j*8 of the group's 128 bytes
             const int off = lv * 128 + (u16 >> 2) * 32 + (u16 & 3) * 8;
-            *reinterpret_cast<uint2*>(xb + (size_t)(2 * m) * c.xrow + off) = make_uint2(hi_e, hi_o);
-            *reinterpret_cast<uint2*>(xb + (size_t)(2 * m + 1) * c.xrow + off) = make_uint2(lo_e, lo_o);
+            *reinterpret_cast<uint2*>(xb + (size_t)(2 * m) * c.xrow + off) = hi2;
+            *reinterpret_cast<uint2*>(xb + (size_t)(2 * m + 1) * c.xrow + off) = lo2;
             if (u16 == 0) xg[lv * 8 * MT + m] = make_float2((float)isum, inv_scale);
           }
         }
@@ -869,6 +937,17 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       xaddr8[nt] = sbase + c.off_x + (uint32_t)((xlive8[nt] ? v : 0) * c.xrow + t * 32);
     }
     const uint32_t xgaddr8 = sbase + c.off_xg + (uint32_t)(t * 8);           // batch row m = t + 4 nt
+    // streamed activations: line (group kpw, virtual row v) of the stage, its 16-byte chunks XOR-ed with v & 7
+    const bool xstream = NPH == 1 && c.x_stream != 0;
+    uint32_t xs0[NT], xs1[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const int v = g + 8 * nt;
+      const uint32_t line = (uint32_t)(STAGE_BYTES + (kpw * c.vr + (v < c.vr ? v : 0)) * 128);
+      xs0[nt] = line + (uint32_t)(((2 * t) ^ (v & 7)) * 16);
+      xs1[nt] = line + (uint32_t)(((2 * t + 1) ^ (v & 7)) * 16);
+    }
+    const uint32_t xsg = (uint32_t)(STAGE_BYTES + c.vr * CG * 128 + kpw * 64 + t * 8);
     const uint32_t wl_off = (uint32_t)((kpw >> 1) * BOX_BYTES + (rg * 32 + pg) * 128 + ((((kpw & 1) * 4 + t) ^ pg) * 16));
     const uint32_t sl_off = (uint32_t)(STAGE_W + (rg * 32 + pg) * (CG * 2) + kpw * 2);
     float out8[2][NT][2];
@@ -916,7 +995,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       if (!consumer_sync()) return;
     }
     if (wk.n_units == 0) continue;
-    if (!stage_x(ph, pc)) return;
+    if (!xstream && !stage_x(ph, pc)) return;
     UnitIter ui;
     ui.start(wk);
     for (int i = 0; i < wk.n_units; ++i) {
@@ -926,7 +1005,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       }
       const int gi = ui.chunk * c.cgz + g_first;
       if (gi < Gk) {
-        const uint32_t st = sbase + (uint32_t)s * STAGE_BYTES;
+        const uint32_t st = sbase + (uint32_t)s * (uint32_t)c.stage_bytes;
         const uint32_t wp = st + wl_off, sp = st + sl_off;
         uint4 wa[2], wb[2];
         wa[0] = lds128<0>(wp);
@@ -936,8 +1015,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
           const uint32_t xa = xaddr8[nt] + (uint32_t)(gi * 128);
-          lds128_if<0>(xr8[nt][0], xa, xlive8[nt]);
-          lds128_if<16>(xr8[nt][1], xa, xlive8[nt]);
+          lds128_if<0>(xr8[nt][0], xstream ? st + xs0[nt] : xa, xlive8[nt]);
+          lds128_if<0>(xr8[nt][1], xstream ? st + xs1[nt] : xa + 16, xlive8[nt]);
         }
         float sc[2][2], zp[2][2];
         sc[0][0] = lds_h<0>(sp);
@@ -971,7 +1050,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
             }
           }
         }
-        const uint32_t xga = xgaddr8 + (uint32_t)(gi * 8 * MT * 8);
+        const uint32_t xga = xstream ? st + xsg : xgaddr8 + (uint32_t)(gi * 8 * MT * 8);
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
           const float2 xs = nt == 0 ? lds64f<0>(xga) : nt == 1 ? lds64f<32>(xga) : nt == 2 ? lds64f<64>(xga) : lds64f<96>(xga);
@@ -1056,7 +1135,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     }
     const int gi = ui.chunk * c.cgz + g_first;
     if (gi < Gk) {
-      const uint32_t st = sbase + (uint32_t)s * STAGE_BYTES;
+      const uint32_t st = sbase + (uint32_t)s * (uint32_t)c.stage_bytes;
       const uint32_t wp = st + wl_off, sp = st + sl_off;
       uint4 wa[2], wb[2];
       wa[0] = lds128<0>(wp);
@@ -1354,6 +1433,37 @@ size_t plan_split(DecodeCfg* c, int M, int g_total, int gran, bool i8) {
   return smem;
 }
 
+// Shared-memory plan with streamed activations: no staged copy of x, every stage carries the unit's eight
+// groups of quantised activations.  One k-part.  Returns 0 when nothing fits.
+size_t plan_stream(DecodeCfg* c, int M, int g_total, int gran) {
+  c->vr = M <= 4 ? 8 : 16;
+  c->stage_bytes = STAGE_BYTES + c->vr * CG * 128 + 1024;
+  const int tries[4][2] = {{4, 2}, {4, 1}, {3, 2}, {3, 1}};
+  for (int i = 0; i < 4; ++i) {
+    const int stages = tries[i][0], part_bufs = tries[i][1];
+    size_t off = (size_t)stages * c->stage_bytes;
+    c->off_bar = (int)off;
+    off += BAR_BYTES;
+    c->off_x = c->off_xg = (int)off;
+    c->xrow = 0;
+    c->off_part = (int)off;
+    off += (size_t)part_bufs * CG * RB * M * 4;
+    if (off + 1024 > (size_t)kSmemMax) continue;
+    c->stages = stages;
+    c->part_bufs = part_bufs;
+    c->gp = round_up(g_total, gran);
+    c->g_total = g_total;
+    c->gran = gran;
+    c->n_kp = 1;
+    int n_rp = env_int("UNIQL_DECODE_RP", 0);
+    if (n_rp < 1) n_rp = sm_count();
+    c->n_rp = n_rp;
+    if ((long long)n_rp * n_rp * ((c->gp + CG - 1) / CG) >= (1ll << 31)) return 0;
+    return off + 1024;
+  }
+  return 0;
+}
+
 }  // namespace
 
 int decode_supported(const Params& p) {
@@ -1382,7 +1492,8 @@ size_t decode_workspace_bytes(int M, int K, int N_total) {
   const size_t chunks = (size_t)(G + CG - 1) / CG;
   const size_t tiles = (size_t)(N_total + RB - 1) / RB + (size_t)N_total / 32 + 2 * kMaxJobs;
   const size_t slots = tiles * 2 * c.n_kp + (size_t)c.n_rp * c.n_kp * (chunks + 2 * c.n_kp);
-  return (size_t)kWsHeader + slots * (size_t)M * RB * 4;
+  // (+ the quantised activations of the streamed mode: 16 virtual rows of 128 bytes and 64 bytes per group)
+  return (size_t)kWsHeader + slots * (size_t)M * RB * 4 + (size_t)round_up(G, CG) * (16 * 128 + 64) + 512;
 }
 
 int launch_decode(const Params& p, const LaunchCfg& cfg) {
@@ -1401,7 +1512,24 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
 
   // integer path: fp16 activations staged with 128-bit loads (a leading input block); UNIQL_DECODE_I8=0: fp16 MMAs
   const bool i8 = c.x_vec && env_int("UNIQL_DECODE_I8", 1) != 0;
-  const size_t smem = plan_split(&c, p.M, g_total, gran, i8);
+  // Streamed activations for rows too long to stage whole beside the ring (which would otherwise split the input
+  // channels over several groups of blocks and hand every tile over); UNIQL_DECODE_XSTREAM=0/1 forces.  Where the
+  // staged copy fits the quantising kernel in front costs more than the staging it saves (measured 3.5 us).
+  size_t smem = 0;
+  c.stage_bytes = STAGE_BYTES;
+  {
+    const int force = env_int("UNIQL_DECODE_XSTREAM", -1);
+    if (i8 && p.M <= 8 && force != 0) {
+      DecodeCfg t = c;
+      const size_t s0 = plan_split(&t, p.M, g_total, gran, true);
+      if (force == 1 || !s0 || t.n_kp > 1) {
+        smem = plan_stream(&c, p.M, g_total, gran);
+        c.x_stream = smem != 0;
+        if (!smem) c.stage_bytes = STAGE_BYTES;
+      }
+    }
+  }
+  if (!c.x_stream) smem = plan_split(&c, p.M, g_total, gran, i8);
   if (!smem) return UNIQL_ERR_UNSUPPORTED;
 
   // ---- narrow tiles (32 rows x 16 groups) when the schedule they give is shorter: matrices with fewer
@@ -1419,7 +1547,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
         t32 += (long)((a.keep + RB / 2 - 1) / (RB / 2)) * a.count;
       }
     }
-    if (all_plain) {
+    if (all_plain && !c.x_stream) {
       const int Gk0 = g_total < c.gp ? g_total : c.gp;
       // (only where there are fewer wide tiles than blocks and the input channels are not split: measured,
       //  the smaller boxes of the narrow tiles cost more than a better balance of many tiles gains)
@@ -1476,15 +1604,49 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   }
   if (tiles < 1 || tiles * EW > kCounterInts) return UNIQL_ERR_UNSUPPORTED;
   c.max_slots = slots_needed(tiles, c.g_total, c.gp, c.n_rp, c.cgz);
-  {
-    const size_t need = (size_t)kWsHeader + (size_t)tiles * c.max_slots * p.M * RB * 4;
-    if (!cfg.workspace || cfg.ws_bytes < need) return UNIQL_ERR_WORKSPACE;
+  size_t need = (size_t)kWsHeader + (size_t)tiles * c.max_slots * p.M * RB * 4;
+  size_t xq_off = 0, xg_off = 0;
+  const int g_pad = round_up(g_total, CG);
+  if (c.x_stream) {
+    xq_off = (need + 255) & ~(size_t)255;
+    xg_off = xq_off + (size_t)g_pad * c.vr * 128;
+    need = xg_off + (size_t)g_pad * 64;
   }
+  if (!cfg.workspace || cfg.ws_bytes < need) return UNIQL_ERR_WORKSPACE;
   unsigned char* ws = reinterpret_cast<unsigned char*>(cfg.workspace);
   c.counters = reinterpret_cast<int*>(ws);
   c.status = reinterpret_cast<int*>(ws + kStatusOff);
   c.partials = reinterpret_cast<float*>(ws + kWsHeader);
   c.grid_sync = reinterpret_cast<int*>(ws + kGridSyncOff);
+  if (c.x_stream) {
+    EncodeTiledFn enc = encoder();
+    if (!enc) return UNIQL_ERR_CUDA;
+    const cuuint64_t dims[3] = {128, (cuuint64_t)c.vr, (cuuint64_t)g_pad};
+    const cuuint64_t strides[2] = {128, (cuuint64_t)c.vr * 128};
+    const cuuint32_t box[3] = {128, (cuuint32_t)c.vr, (cuuint32_t)CG};
+    const cuuint32_t es[3] = {1, 1, 1};
+    if (enc(&c.xmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, ws + xq_off, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return UNIQL_ERR_CUDA;
+    c.xg_glob = reinterpret_cast<const float2*>(ws + xg_off);
+    // the activations are quantised once, by a small kernel in front of the streaming one
+    cudaLaunchConfig_t lc;
+    memset(&lc, 0, sizeof(lc));
+    const int units = g_total * (c.vr / 2) * 16;
+    lc.gridDim = dim3((units + 255) / 256);
+    lc.blockDim = dim3(256);
+    lc.stream = cfg.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = env_int("UNIQL_PDL", 1) ? 1 : 0;
+    if (cudaLaunchKernelEx(&lc, xquant_kernel, c.ph[0], p.M, c.vr, g_total, ws + xq_off,
+                           reinterpret_cast<float2*>(ws + xg_off)) != cudaSuccess) {
+      cudaGetLastError();
+      return UNIQL_ERR_CUDA;
+    }
+  }
   if (i8) {
     if (p.M <= 4) return launch_t<1, false, 1, 1>(p, c, smem, cfg.stream);
     if (p.M <= 8) return launch_t<1, false, 2, 1>(p, c, smem, cfg.stream);
@@ -1539,6 +1701,7 @@ int launch_mlp_phases(const MlpDecode& d, int first, int count, const LaunchCfg&
   memset(&c, 0, sizeof(c));
   c.x_vec = 1;
   c.n_ph = count;
+  c.stage_bytes = STAGE_BYTES;
   int g_max = 0, gran = 8;
   for (int ph = first; ph < first + count; ++ph) {
     const int g_total = ph == 0 ? d.hidden / kGroup : (d.k_int + kGroup - 1) / kGroup;

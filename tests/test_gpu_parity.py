@@ -31,7 +31,7 @@ def B():
 def _reset_path(B):
     yield
     B.set_path(B.PATH_AUTO)
-    for k in ("UNIQL_DECODE_KP", "UNIQL_DECODE_RP", "UNIQL_DECODE_NARROW"):
+    for k in ("UNIQL_DECODE_KP", "UNIQL_DECODE_RP", "UNIQL_DECODE_NARROW", "UNIQL_DECODE_XSTREAM"):
         os.environ.pop(k, None)
 
 
@@ -170,6 +170,39 @@ def test_tile_shapes(B, narrow, kp, rp, M):
         x = synth.draw_x(rng, M, synth.map_size(in_map), "f16")
         y, ref = run_ex(B, qw, dw, x, "f16", in_map, 0, out_map, 0)
         check_output(y, ref, "f16", TIGHT, "narrow=%d per-head keep %d M=%d" % (narrow, keep, M))
+
+
+@pytest.mark.parametrize("stream", [0, 1])
+@pytest.mark.parametrize("rp", [0, 1, 7])
+@pytest.mark.parametrize("M", [1, 3, 4, 5, 6, 8, 13, 16])
+def test_streamed_activations(B, stream, rp, M):
+    """Activations quantised once by a small kernel and carried through the ring beside the weights (the default
+    where a staged copy of x does not fit beside the ring) against the block-wide staging: the same results for plain, ragged and per-head shapes,
+    several matrices in one launch and the rotary epilogue."""
+    os.environ["UNIQL_DECODE_XSTREAM"] = str(stream)
+    if rp:
+        os.environ["UNIQL_DECODE_RP"] = str(rp)
+    B.set_path(B.PATH_DECODE)
+    rng = np.random.default_rng(80 + M)
+    for (N, K, k_in, k_out) in [(200, 2304, 2304, 200), (200, 2304, 1096, 77), (96, 256, 256, 96), (70, 3328, 3072, 33)]:
+        qw = synth.draw_qweight(rng, N, K)
+        dw = dev_weight(qw)
+        bias = synth.to_dtype_values(rng.standard_normal(N).astype(np.float32), "f16")
+        x = synth.draw_x(rng, M, k_in, "f16")
+        y, ref = run_ex(B, qw, dw, x, "f16", None, k_in, None, k_out, bias=bias, ldy_pad=3)
+        check_output(y, ref, "f16", TIGHT, "stream=%d rp=%d M=%d %s" % (stream, rp, M, (N, K, k_in, k_out)))
+        y2, _ = run_ex(B, qw, dw, x, "f16", None, k_in, None, k_out, bias=bias, ldy_pad=3)
+        assert torch.equal(y, y2), "run-to-run results differ"
+    qw = synth.draw_qweight(rng, 512, 1024)
+    dw = dev_weight(qw)
+    for keep in (128, 96, 40):
+        in_map = synth.map_per_head(8, 128, keep)
+        x = synth.draw_x(rng, M, synth.map_size(in_map), "f16")
+        y, ref = run_ex(B, qw, dw, x, "f16", in_map, 0, synth.map_per_head(4, 128, 108), 0)
+        check_output(y, ref, "f16", TIGHT, "stream=%d per-head keep %d M=%d" % (stream, keep, M))
+    for (g, ref) in run_rope(B, rng, M, 512, 6, 2, 128, 96, 500000.0, "f16", bias=True, v_keep=104):
+        check_output(g, ref, "f16", TIGHT, "stream=%d q/k/v M=%d" % (stream, M))
+    assert B.workspace_status() == 0
 
 
 def test_caller_workspace(B):
