@@ -487,8 +487,8 @@ struct UnitIter {
 // ---------------------------------------------------------------------------------------- kernel
 // NT == 0: fp16 tensor-core path (MT batch tiles of 8, ONECOL: batch 1).  NT > 0: integer path, NT column
 // tiles of the int8 MMA, each holding the high and the low byte of four batch rows.
-// NPH: phases (2: the fused SwiGLU MLP, integer path only).
-template <int MT, bool ONECOL, int NT, int NPH>
+// NPH: phases (2: the fused SwiGLU MLP, integer path only).  XS: activations streamed through the ring.
+template <int MT, bool ONECOL, int NT, int NPH, bool XS>
 __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ Params p,
                                                         const __grid_constant__ DecodeCfg c) {
   extern __shared__ unsigned char smem_raw[];
@@ -533,7 +533,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     uint32_t ring_parity = 1;      // parity of the previous use of ring position s
     bool ok = true;
     // streamed activations are written by the kernel launched just before this one
-    if (NPH == 1 && c.x_stream) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (XS) asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int ph = 0; ph < NPH && ok; ++ph) {
       const PhaseCtx pc = (NPH == 1 || ph == 0) ? pc0 : phase_ctx(c, ph, kp, rp);
       const Work& wk = pc.wk;
@@ -584,8 +584,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         const int ng = min(CG, ng_all), ng2 = ng_all - ng;  // ... in row slots 0..31 (all 64 unless narrow) / 32..63
         const int nb = (ng + 1) >> 1, nb2 = (ng2 + 1) >> 1; // 128-byte columns with a visited group
         const uint32_t full = bar_full + 8 * s;
-        const uint32_t st = sbase + (uint32_t)s * (uint32_t)c.stage_bytes;
-        const uint32_t xbytes = (NPH == 1 && c.x_stream) ? (uint32_t)(c.vr * CG * 128 + CG * 64) : 0u;
+        const uint32_t st = sbase + (uint32_t)s * (XS ? (uint32_t)c.stage_bytes : (uint32_t)STAGE_BYTES);
+        const uint32_t xbytes = XS ? (uint32_t)(c.vr * CG * 128 + CG * 64) : 0u;
         if (lane == 0)
           mbar_expect_tx(full, xbytes + (mode == kNarrow ? (uint32_t)((nb + nb2) * (BOX_BYTES / 2)) : (uint32_t)(nb * BOX_BYTES)));
         __syncwarp();
@@ -792,7 +792,14 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     const int Gk = pc.Gk, sg_lo = pc.sg_lo;
     const T* x = reinterpret_cast<const T*>(P.x);
     const long long ldx = P.ldx;
-    auto compact_of = [&](int ch) -> int { return compact_channel(P, ch); };
+    // stored channel (a multiple of 8) -> compact activation column, or -1 when the channel is pruned
+    const int m_start = P.start, m_keep = P.keep;
+    const bool m_heads = P.count > 1;
+    auto compact_of = [&](int ch) -> int {
+      if (m_heads) return compact_channel(P, ch);
+      const int r = ch - m_start;
+      return (r >= 0 && r < m_keep) ? r : -1;
+    };
     // activations a previous phase of this launch wrote are read past the non-coherent cache
     auto load16 = [&](const T* ptr) -> uint4 {
       return (NPH > 1 && ph > 0) ? __ldcg(reinterpret_cast<const uint4*>(ptr)) : __ldg(reinterpret_cast<const uint4*>(ptr));
@@ -938,7 +945,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     }
     const uint32_t xgaddr8 = sbase + c.off_xg + (uint32_t)(t * 8);           // batch row m = t + 4 nt
     // streamed activations: line (group kpw, virtual row v) of the stage, its 16-byte chunks XOR-ed with v & 7
-    const bool xstream = NPH == 1 && c.x_stream != 0;
+    constexpr bool xstream = XS;
     uint32_t xs0[NT], xs1[NT];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -1005,7 +1012,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       }
       const int gi = ui.chunk * c.cgz + g_first;
       if (gi < Gk) {
-        const uint32_t st = sbase + (uint32_t)s * (uint32_t)c.stage_bytes;
+        const uint32_t st = sbase + (uint32_t)s * (XS ? (uint32_t)c.stage_bytes : (uint32_t)STAGE_BYTES);
         const uint32_t wp = st + wl_off, sp = st + sl_off;
         uint4 wa[2], wb[2];
         wa[0] = lds128<0>(wp);
@@ -1135,7 +1142,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     }
     const int gi = ui.chunk * c.cgz + g_first;
     if (gi < Gk) {
-      const uint32_t st = sbase + (uint32_t)s * (uint32_t)c.stage_bytes;
+      const uint32_t st = sbase + (uint32_t)s * (uint32_t)STAGE_BYTES;
       const uint32_t wp = st + wl_off, sp = st + sl_off;
       uint4 wa[2], wb[2];
       wa[0] = lds128<0>(wp);
@@ -1351,9 +1358,9 @@ long schedule_cost(long tiles, long Ck, long n_rp) {
   return base * Ck + (split ? (R * Ck + n_rp - 1) / n_rp + 3 : Ck);
 }
 
-template <int MT, bool ONECOL, int NT, int NPH>
+template <int MT, bool ONECOL, int NT, int NPH, bool XS = false>
 int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stream) {
-  auto kern = decode_kernel<MT, ONECOL, NT, NPH>;
+  auto kern = decode_kernel<MT, ONECOL, NT, NPH, XS>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return UNIQL_ERR_CUDA;
   cudaLaunchConfig_t lc;
@@ -1646,6 +1653,10 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
       cudaGetLastError();
       return UNIQL_ERR_CUDA;
     }
+  }
+  if (c.x_stream) {
+    if (p.M <= 4) return launch_t<1, false, 1, 1, true>(p, c, smem, cfg.stream);
+    return launch_t<1, false, 2, 1, true>(p, c, smem, cfg.stream);
   }
   if (i8) {
     if (p.M <= 4) return launch_t<1, false, 1, 1>(p, c, smem, cfg.stream);
