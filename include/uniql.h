@@ -70,8 +70,10 @@ typedef enum {
 
 typedef enum { UNIQL_F16 = 0, UNIQL_BF16 = 1 } uniql_dtype;
 
-/* Kernel selection, for A/B tests.  AUTO: M <= 16 decode kernel, M >= 64 prefill
- * (tensor-core) kernel when its alignment rules hold, otherwise the generic kernel. */
+/* Kernel selection, for A/B tests.  AUTO: fp16 batches of M <= 16 take the decode kernel; everything
+ * else (M > 16, bf16) the tensor-core (prefill) kernel when its alignment rules hold (activations 16-byte
+ * aligned with a row pitch that is a multiple of 8, input map a leading block or one family of per-head
+ * blocks on 64-channel boundaries with keep % 8 == 0), otherwise the generic kernel. */
 typedef enum { UNIQL_PATH_AUTO = 0, UNIQL_PATH_GENERIC = 1, UNIQL_PATH_DECODE = 2,
                UNIQL_PATH_PREFILL = 3 } uniql_path;
 

@@ -87,7 +87,10 @@ int dispatch(const Params& p, void* workspace, size_t ws_bytes, void* stream) {
   LaunchCfg cfg{workspace, ws_bytes, (cudaStream_t)stream};
   int path = g_path;
   bool dec_ok = p.M <= 16 && decode_supported(p);
-  bool pre_ok = p.M >= 64 && prefill_supported(p);
+  // every batch the decode kernel does not take (more than 16 rows, bf16) goes to the tensor cores when the maps
+  // allow it: at 17..63 rows the generic kernel measured 13 to 26 times slower (930 us against 71 us for the
+  // Llama-3-8B gate|up at M = 17)
+  bool pre_ok = prefill_supported(p);
   if (path == UNIQL_PATH_AUTO) path = dec_ok ? UNIQL_PATH_DECODE : (pre_ok ? UNIQL_PATH_PREFILL : UNIQL_PATH_GENERIC);
   if (path == UNIQL_PATH_DECODE) {
     if (!(p.M <= 16 && decode_supported(p))) return UNIQL_ERR_UNSUPPORTED;

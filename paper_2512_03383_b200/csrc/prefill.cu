@@ -1,4 +1,5 @@
-// Prefill kernel (M >= 64 tokens) of the pruned 4-bit linear layer, sm_100a: a dense contraction on
+// Prefill kernel (every batch the decode kernel does not take: more than 16 rows, bf16) of the pruned 4-bit
+// linear layer, sm_100a: a dense contraction on
 // the fifth-generation tensor cores (tcgen05.mma, accumulators in tensor memory).
 //
 // Orientation.  The packed weights are four times smaller than the activations, so the weight side
@@ -661,7 +662,7 @@ int launch_pt(const Params& p, const PrefillCfg& c, int grid, cudaStream_t strea
 // D_int is pruned as a leading block: Section 3.4) or one family of per-head kept blocks (the input side of
 // o_proj / out_proj: heads on 64-channel boundaries, keep a multiple of 8), any output map, both activation types.
 int prefill_supported(const Params& p) {
-  if (p.M < 17) return 0;
+  if (p.M < 1) return 0;
   if (p.dt != UNIQL_F16 && p.dt != UNIQL_BF16) return 0;
   if (p.imap.n_fam != 1) return 0;
   {
