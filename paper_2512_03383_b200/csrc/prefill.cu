@@ -304,7 +304,8 @@ __global__ void x_to_f16_kernel(const __nv_bfloat16* __restrict__ x, int ldx, in
 
 // T: activation / output type.  CONV: the activation tiles arrive as bf16 and are converted to fp16 in
 // shared memory by the de-quantisers (used when the workspace cannot hold a converted copy).
-template <typename T, bool CONV>
+// HEADS: the input map is a family of per-head blocks (else a leading block).
+template <typename T, bool CONV, bool HEADS>
 __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__ Params p,
                                                          const __grid_constant__ PrefillCfg c) {
   extern __shared__ unsigned char psmem_raw[];
@@ -357,7 +358,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
           if (it >= PSTAGES && !pmbar_wait(empty + 8 * s, par, abort_flag, true)) { failed = true; break; }
           const uint32_t fb = full_b + 8 * s;
           pmbar_expect_tx(fb, (uint32_t)(c.bn * BK * 2));
-          tma_box2(sbase + s * PSTAGE_BYTES + A_BYTES, &c.xmap, kblock_of(c, kb).xcol, tt * c.bn, fb);
+          tma_box2(sbase + s * PSTAGE_BYTES + A_BYTES, &c.xmap, HEADS ? kblock_of(c, kb).xcol : kb * BK, tt * c.bn, fb);
           if (++s == PSTAGES) { s = 0; par ^= 1; }
         }
       }
@@ -403,6 +404,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
 #pragma unroll
     for (int j = 0; j < 4; ++j) col_off[j] = (uint32_t)(((hf * 4 + j) ^ (r & 7)) * 16);
     int done = 0;                      // stage iterations before this segment
+    constexpr bool heads = HEADS;
     SegIter si; si.init(c, blockIdx.x, gridDim.x);
     Seg sg;
     for (; !failed && si.next(sg); done += sg.kb1 - sg.kb0) {
@@ -419,17 +421,17 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
       // codes and scale / zero-point of this team's next two k-blocks are kept in registers
       uint4 q0 = make_uint4(0, 0, 0, 0), q1 = q0;
       __half s0 = __ushort_as_half(0), z0 = s0, s1 = s0, z1 = s0;
-      int v0 = 0, v1 = 0;              // kept channels of the k-blocks held in q0 / q1
       // codes, scale and zero-point of visited k-block v of this thread's row; `valid` channels of it are kept
-      auto fetch = [&](int v, uint4& q, __half& sc, __half& zr, int& valid) {
-        const KBlock kbk = kblock_of(c, v);
-        valid = kbk.valid;
-        q = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)kbk.stored * 32));
-        sc = __ldg(srow + (kbk.stored >> 1)); zr = __ldg(zrow + (kbk.stored >> 1));
+      // (a leading block needs no mask: the activation tensor map ends at k_in, so the tail of its last k-block
+      //  meets zeros)
+      auto fetch = [&](int v, uint4& q, __half& sc, __half& zr) {
+        const int stored = heads ? kblock_of(c, v).stored : v;
+        q = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)stored * 32));
+        sc = __ldg(srow + (stored >> 1)); zr = __ldg(zrow + (stored >> 1));
       };
       if (live) {
-        if (kb0 < sg.kb1) fetch(kb0, q0, s0, z0, v0);
-        if (kb0 + 2 < sg.kb1) fetch(kb0 + 2, q1, s1, z1, v1);
+        if (kb0 < sg.kb1) fetch(kb0, q0, s0, z0);
+        if (kb0 + 2 < sg.kb1) fetch(kb0 + 2, q1, s1, z1);
       }
       for (int kb = kb0; kb < sg.kb1; kb += 2) {
         const int it = it0 + kb;
@@ -437,17 +439,17 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         const uint32_t use = (uint32_t)(it / PSTAGES);
         uint4 q2 = make_uint4(0, 0, 0, 0);
         __half s2 = s1, z2 = z1;
-        int v2 = 0;
-        if (live && kb + 4 < sg.kb1) fetch(kb + 4, q2, s2, z2, v2);
+        if (live && kb + 4 < sg.kb1) fetch(kb + 4, q2, s2, z2);
         if (it >= PSTAGES && !pmbar_wait(empty + 8 * s, (use - 1) & 1, abort_flag)) { failed = true; break; }
         const uint32_t a_st = sbase + s * PSTAGE_BYTES + row_off;
         const __half2 sh2 = __half2half2(s0);
         const __half2 cz2 = __float2half2_rn((8.f - __half2float(z0)) * __half2float(s0));
         const uint32_t qw[4] = {q0.x, q0.y, q0.z, q0.w};
+        const int v0 = heads ? kblock_of(c, kb).valid : BK;        // kept channels of this k-block
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           // (eight channels per word; keep counts are multiples of eight, so a word is kept or pruned whole)
-          const uint4 o = (live && hf * 32 + j * 8 < v0) ? dequant_word(qw[j], sh2, cz2) : make_uint4(0, 0, 0, 0);
+          const uint4 o = (live && (!HEADS || hf * 32 + j * 8 < v0)) ? dequant_word(qw[j], sh2, cz2) : make_uint4(0, 0, 0, 0);
           asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a_st + col_off[j]), "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w) : "memory");
         }
         if constexpr (CONV) {
@@ -465,8 +467,8 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         fence_async_smem();            // generic-proxy writes must be visible to the tensor core (async proxy)
         __syncwarp();
         if (lane == 0) pmbar_arrive(full_a + 8 * s);
-        q0 = q1; s0 = s1; z0 = z1; v0 = v1;
-        q1 = q2; s1 = s2; z1 = z2; v1 = v2;
+        q0 = q1; s0 = s1; z0 = z1;
+        q1 = q2; s1 = s2; z1 = z2;
       }
     }
   } else if (warp >= EPI_WARP0) {
@@ -646,14 +648,18 @@ int host_job_tiles(const JobDev& j) {
   return (j.k_out + BMW - 1) / BMW;
 }
 
-template <typename T, bool CONV>
-int launch_pt(const Params& p, const PrefillCfg& c, int grid, cudaStream_t stream) {
+template <typename T, bool CONV, bool HEADS>
+int launch_pth(const Params& p, const PrefillCfg& c, int grid, cudaStream_t stream) {
   const size_t smem = 1024 + (size_t)PSTAGES * PSTAGE_BYTES + STG_BYTES + 512;
-  auto kern = prefill_kernel<T, CONV>;
+  auto kern = prefill_kernel<T, CONV, HEADS>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return UNIQL_ERR_CUDA;
   kern<<<grid, PTH, smem, stream>>>(p, c);
   return cudaGetLastError() == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
+}
+template <typename T, bool CONV>
+int launch_pt(const Params& p, const PrefillCfg& c, int grid, cudaStream_t stream) {
+  return c.km_period != 0 ? launch_pth<T, CONV, true>(p, c, grid, stream) : launch_pth<T, CONV, false>(p, c, grid, stream);
 }
 
 }  // namespace
