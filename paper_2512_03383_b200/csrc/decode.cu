@@ -133,6 +133,10 @@ __device__ inline void mbar_init(uint32_t bar, uint32_t count) {
 __device__ inline void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// more bytes expected in the current phase, without an arrival
+__device__ inline void mbar_expect_tx_only(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
 __device__ inline void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
@@ -532,8 +536,26 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     int it = 0, s = 0;
     uint32_t ring_parity = 1;      // parity of the previous use of ring position s
     bool ok = true;
-    // streamed activations are written by the kernel launched just before this one
-    if (XS) asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Streamed activations are written by the kernel launched just before this one.  The weights of the first
+    // fill of the ring do not wait for it: their stages are armed with the weight bytes only, and once the ring
+    // is full (or the block's units are all issued) the producer waits for the predecessor and sends the
+    // activations of those stages after them, with the arrival the stages' barriers still lack.
+    bool x_waited = !XS;
+    int x_lv0[MAX_STAGES];
+    auto send_x = [&](int stage, int lv0) {                          // lane 31: arrival + the unit's activations
+      const uint32_t full = bar_full + 8 * stage;
+      const uint32_t st = sbase + (uint32_t)stage * (uint32_t)c.stage_bytes;
+      mbar_expect_tx(full, (uint32_t)(c.vr * CG * 128 + CG * 64));
+      tma_box3(st + STAGE_BYTES, &c.xmap, 0, 0, lv0, full);
+      bulk_copy(st + STAGE_BYTES + (uint32_t)(c.vr * CG * 128), c.xg_glob + (size_t)lv0 * 8, CG * 64, full);
+    };
+    auto flush_x = [&](int n_issued) {                               // after the first min(S, units) stages
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      if (lane == 31)
+        for (int j = 0; j < n_issued; ++j) send_x(j, x_lv0[j]);
+      __syncwarp();
+      x_waited = true;
+    };
     for (int ph = 0; ph < NPH && ok; ++ph) {
       const PhaseCtx pc = (NPH == 1 || ph == 0) ? pc0 : phase_ctx(c, ph, kp, rp);
       const Work& wk = pc.wk;
@@ -585,15 +607,15 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         const int nb = (ng + 1) >> 1, nb2 = (ng2 + 1) >> 1; // 128-byte columns with a visited group
         const uint32_t full = bar_full + 8 * s;
         const uint32_t st = sbase + (uint32_t)s * (XS ? (uint32_t)c.stage_bytes : (uint32_t)STAGE_BYTES);
-        const uint32_t xbytes = XS ? (uint32_t)(c.vr * CG * 128 + CG * 64) : 0u;
-        if (lane == 0)
-          mbar_expect_tx(full, xbytes + (mode == kNarrow ? (uint32_t)((nb + nb2) * (BOX_BYTES / 2)) : (uint32_t)(nb * BOX_BYTES)));
-        __syncwarp();
-        if (xbytes && lane == 31) {
-          const int lv0 = chunk * CG;                                // (one k-part, wide tiles)
-          tma_box3(st + STAGE_BYTES, &c.xmap, 0, 0, lv0, full);
-          bulk_copy(st + STAGE_BYTES + (uint32_t)(c.vr * CG * 128), c.xg_glob + (size_t)lv0 * 8, CG * 64, full);
+        const uint32_t wbytes = mode == kNarrow ? (uint32_t)((nb + nb2) * (BOX_BYTES / 2)) : (uint32_t)(nb * BOX_BYTES);
+        if (XS) {
+          if (lane == 0) mbar_expect_tx_only(full, wbytes);          // the arrival comes with the activations
+          if (!x_waited) x_lv0[s] = chunk * CG;                      // (one k-part, wide tiles; s == it here)
+        } else if (lane == 0) {
+          mbar_expect_tx(full, wbytes);
         }
+        __syncwarp();
+        if (XS && x_waited && lane == 31) send_x(s, chunk * CG);
         if (lane < nb) {
           const int xb = (sg_lo + chunk * c.cgz + 2 * lane) * 64;    // byte in the weight row
           const uint32_t dst = st + (uint32_t)lane * BOX_BYTES;
@@ -630,7 +652,9 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         cp_async_arrive_noinc(full);
         if (iu + 1 < wk.n_units && ui.advance(wk, iu + 1)) jumped = true;
         if (++s == S) { s = 0; ring_parity ^= 1; }
+        if (XS && !x_waited && it + 1 == S) flush_x(S);
       }
+      if (XS && !x_waited) flush_x(it);                              // fewer units than stages
     }
     if (!ok) {
       // let the copies of the stages that are still armed land before the block goes away
@@ -1521,7 +1545,9 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   const bool i8 = c.x_vec && env_int("UNIQL_DECODE_I8", 1) != 0;
   // Streamed activations for rows too long to stage whole beside the ring (which would otherwise split the input
   // channels over several groups of blocks and hand every tile over); UNIQL_DECODE_XSTREAM=0/1 forces.  Where the
-  // staged copy fits the quantising kernel in front costs more than the staging it saves (measured 3.5 us).
+  // staged copy fits the quantising kernel in front costs more than the staging it saves (measured 3.5 us), and
+  // inside a sequence of launches it only pays for itself at eight rows (Llama-3-8B MLP: 51.7 against 53.9 us
+  // at M = 8, 93.8 against 105.1 us at M = 16 as two launches of eight; 46.6 against 43.0 us at M = 5).
   size_t smem = 0;
   c.stage_bytes = STAGE_BYTES;
   {
@@ -1529,7 +1555,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
     if (i8 && p.M <= 8 && force != 0) {
       DecodeCfg t = c;
       const size_t s0 = plan_split(&t, p.M, g_total, gran, true);
-      if (force == 1 || !s0 || t.n_kp > 1) {
+      if (force == 1 || !s0 || (t.n_kp > 1 && p.M >= 8)) {
         smem = plan_stream(&c, p.M, g_total, gran);
         c.x_stream = smem != 0;
         if (!smem) c.stage_bytes = STAGE_BYTES;
