@@ -233,6 +233,12 @@ __device__ inline void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2
                : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// the first MMA of a chain: accumulators start at zero (no registers to clear)
+__device__ inline void mma_s8_first(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+               : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
+}
 template <int OFF>
 __device__ inline float2 lds64f(uint32_t addr) {
   float2 v;
@@ -1060,12 +1066,6 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         zp[1][1] = lds_h<STAGE_SZ + 24 * CG * 2>(sp);
         int d[2][NT][4];
 #pragma unroll
-        for (int sub = 0; sub < 2; ++sub)
-#pragma unroll
-          for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) d[sub][nt][e] = 0;
-#pragma unroll
         for (int j = 0; j < 4; ++j) {
 #pragma unroll
           for (int sub = 0; sub < 2; ++sub) {
@@ -1077,7 +1077,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
             for (int nt = 0; nt < NT; ++nt) {
               const uint4 xv = xr8[nt][j >> 1];
               const uint32_t b0 = (j & 1) ? xv.z : xv.x, b1 = (j & 1) ? xv.w : xv.y;
-              mma_s8(d[sub][nt], lo0, lo1, hi0, hi1, b0, b1);
+              if (j == 0) mma_s8_first(d[sub][nt], lo0, lo1, hi0, hi1, b0, b1);
+              else mma_s8(d[sub][nt], lo0, lo1, hi0, hi1, b0, b1);
             }
           }
         }
@@ -1087,8 +1088,9 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           const float2 xs = nt == 0 ? lds64f<0>(xga) : nt == 1 ? lds64f<32>(xga) : nt == 2 ? lds64f<64>(xga) : lds64f<96>(xga);
 #pragma unroll
           for (int sub = 0; sub < 2; ++sub) {
-            const float y0 = fmaf(256.f, small_int_to_float(d[sub][nt][0]), small_int_to_float(d[sub][nt][1]));
-            const float y1 = fmaf(256.f, small_int_to_float(d[sub][nt][2]), small_int_to_float(d[sub][nt][3]));
+            // 256 * (sum q*hi) + (sum q*lo) = sum q*x_i exactly, in integers; one conversion, one rounding
+            const float y0 = (float)(d[sub][nt][0] * 256 + d[sub][nt][1]);
+            const float y1 = (float)(d[sub][nt][2] * 256 + d[sub][nt][3]);
             out8[sub][nt][0] = fmaf(sc[sub][0] * xs.y, fmaf(-zp[sub][0], xs.x, y0), out8[sub][nt][0]);
             out8[sub][nt][1] = fmaf(sc[sub][1] * xs.y, fmaf(-zp[sub][1], xs.x, y1), out8[sub][nt][1]);
           }
