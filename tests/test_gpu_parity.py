@@ -205,6 +205,26 @@ def test_streamed_activations(B, stream, rp, M):
     assert B.workspace_status() == 0
 
 
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("M", [1, 7, 16, 17, 70])
+def test_tiny_and_ragged_shapes(B, M, dtype):
+    """Degenerate sizes through the automatic dispatch: one group, one row, keep counts of 4, a single kept
+    input channel block, outputs narrower than a tile."""
+    rng = np.random.default_rng(300 + M)
+    for (N, K, k_in, k_out) in [(1, 128, 128, 1), (5, 128, 4, 4), (64, 256, 256, 64), (3, 256, 8, 3), (130, 384, 384, 129),
+                                (257, 128, 124, 257)]:
+        qw = synth.draw_qweight(rng, N, K)
+        dw = dev_weight(qw)
+        x = synth.draw_x(rng, M, k_in, dtype)
+        y, ref = run_ex(B, qw, dw, x, dtype, None, k_in, None, k_out, ldy_pad=1)
+        check_output(y, ref, dtype, 5e-4, "tiny %s M=%d %s" % ((N, K, k_in, k_out), M, dtype))
+    for bad in ((0, 128), (128, 0)):                     # nothing kept: an error, not a launch
+        qw = synth.draw_qweight(rng, 8, 128)
+        dw = dev_weight(qw)
+        with pytest.raises(RuntimeError):
+            run_ex(B, qw, dw, synth.draw_x(rng, M, 128, dtype), dtype, None, bad[0], None, min(bad[1], 8))
+
+
 def test_caller_workspace(B):
     os.environ["UNIQL_DECODE_KP"] = "2"
     rng = np.random.default_rng(8)
