@@ -65,6 +65,20 @@ constexpr int kGridWaitLimit = 1 << 21;   // polls (40 ns apart) of the barrier 
 constexpr int BAR_BYTES = 256;
 constexpr int kMaxTF = 8;               // (job, family) pairs of one launch
 
+// Division by a divisor the host knows: q = floor(x / d) = umulhi(x, m) with m = floor(2^32 / d) + 1, exact for
+// x * d < 2^32 (the host passes m = 0 when that cannot be promised or d = 1: then the plain division is used).
+// Integer divisions take about a hundred cycles and several sit on every warp's way to its first unit.
+struct FastDiv { unsigned d, m; };
+__host__ inline FastDiv fast_div(unsigned d, unsigned long long x_max) {
+  FastDiv f;
+  f.d = d ? d : 1;
+  f.m = (f.d > 1 && x_max * f.d < (1ull << 32)) ? (unsigned)((1ull << 32) / f.d + 1) : 0u;
+  return f;
+}
+__device__ inline int div_by(int x, const FastDiv& f) {
+  return f.m ? (int)__umulhi((unsigned)x, f.m) : (f.d == 1 ? x : (int)((unsigned)x / f.d));
+}
+
 // One family of kept row blocks of one job: `count` blocks of `keep` rows, tiles of RB rows inside each
 // block (rope jobs: blocks are heads, rows are rotation pairs, RB/2 pairs per tile).
 struct TileFam {
@@ -78,6 +92,7 @@ struct TileFam {
   int mode;              // kPlain, kNarrow (32 rows x 16 groups), kRope (32 rotation pairs per tile) or
                          // kSwiglu (32 gate rows + 32 up rows)
   int job2;              // kSwiglu: the job of the up projection (`job` is the gate projection)
+  FastDiv by_tpb;        // division by tpb
 };
 enum { kPlain = 0, kRope = 1, kSwiglu = 2, kNarrow = 3 };
 __host__ __device__ inline int tile_rows(const TileFam& f) { return f.mode == kPlain ? RB : RB / 2; }
@@ -92,6 +107,11 @@ struct Phase {
   int period, count;     // count = 1: a leading block
   int g_total, v_first;  // visited groups and the first of them
   int tile0, tiles;      // global tiles [tile0, tile0 + tiles)
+  // the split of the tiles over the blocks, worked out on the host (integer divisions are slow and sit on
+  // every warp's way to its first unit): whole tiles per block, left-over tiles, and for a full k-part its
+  // groups, chunks per tile and the number of blocks that share the left-over units
+  int base, R, gk0, ck0, bt0;
+  FastDiv by_ck0, by_bt0;
 };
 
 struct DecodeCfg {
@@ -336,7 +356,7 @@ __device__ inline TilePos tile_pos(const DecodeCfg& c, const Params& p, int tg) 
   while (q.fi + 1 < c.n_tf && tg >= c.tf[q.fi + 1].tile_begin) ++q.fi;
   const TileFam& f = c.tf[q.fi];
   const int tl = tg - f.tile_begin;
-  q.h = tl / f.tpb;
+  q.h = div_by(tl, f.by_tpb);
   q.r0 = (tl - q.h * f.tpb) * tile_rows(f);
   return q;
 }
@@ -435,21 +455,21 @@ struct Work {
   int tail_tile0;    // first left-over tile (n_rp * base)
   int tb, te;        // tail unit range [tb, te) in the left-over sequence
   int n_units;
+  FastDiv by_ck;     // division by Ck
 };
-__device__ inline Work block_work(int n_rp, int tile0, int tiles, int Ck, int rp) {
+__device__ inline Work block_work(int n_rp, int tile0, int base, int R, int Ck, int Bt_, int rp, const FastDiv& by_ck,
+                                  const FastDiv& by_bt) {
   Work w;
   w.Ck = Ck;
-  const int base = tiles / n_rp;
-  const int R = tiles - base * n_rp;
-  // 32-bit arithmetic (64-bit divisions are slow and this is on every warp's way to its first unit):
-  // the host checks n_rp * n_rp * Ck < 2^31
+  w.by_ck = by_ck;
+  // 32-bit arithmetic (64-bit divisions are slow): the host checks n_rp * n_rp * Ck < 2^31
   const unsigned Ut = (unsigned)(R * Ck);
-  const unsigned Bt = (unsigned)tail_blocks(n_rp, R, Ck);     // blocks that get tail units
+  const unsigned Bt = (unsigned)Bt_;                          // blocks that get tail units
   w.n1 = base * Ck;
   w.tile1 = tile0 + rp * base;
   w.tail_tile0 = tile0 + n_rp * base;
   w.tb = w.te = 0;
-  if ((unsigned)rp < Bt) { w.tb = (int)(Ut * (unsigned)rp / Bt); w.te = (int)(Ut * (unsigned)(rp + 1) / Bt); }
+  if ((unsigned)rp < Bt) { w.tb = div_by((int)(Ut * (unsigned)rp), by_bt); w.te = div_by((int)(Ut * (unsigned)(rp + 1)), by_bt); }
   w.n_units = w.n1 + (w.te - w.tb);
   return w;
 }
@@ -467,7 +487,15 @@ __device__ inline PhaseCtx phase_ctx(const DecodeCfg& c, int ph, int kp, int rp)
   k.Gk = min(c.gp, P.g_total - v_lo);
   k.sg_lo = P.v_first + v_lo;
   k.G = P.K / kGroup;
-  k.wk = block_work(c.n_rp, P.tile0, P.tiles, (k.Gk + c.cgz - 1) / c.cgz, rp);
+  int Ck = P.ck0, Bt = P.bt0;
+  FastDiv by_ck = P.by_ck0, by_bt = P.by_bt0;
+  if (k.Gk != P.gk0) {                                          // a shorter last k-part
+    Ck = (k.Gk + c.cgz - 1) / c.cgz;
+    Bt = tail_blocks(c.n_rp, P.R, Ck);
+    by_ck.d = (unsigned)Ck; by_ck.m = 0;
+    by_bt.d = (unsigned)Bt; by_bt.m = 0;
+  }
+  k.wk = block_work(c.n_rp, P.tile0, P.base, P.R, Ck, Bt, rp, by_ck, by_bt);
   return k;
 }
 // (tile, chunk) of block-local unit i, walked in order.  The share of the left-over tiles comes first:
@@ -476,7 +504,7 @@ __device__ inline PhaseCtx phase_ctx(const DecodeCfg& c, int ph, int kp, int rp)
 struct UnitIter {
   int tile, chunk;
   __device__ inline void start(const Work& w) {
-    if (w.te > w.tb) { tile = w.tail_tile0 + w.tb / w.Ck; chunk = w.tb - (w.tb / w.Ck) * w.Ck; }
+    if (w.te > w.tb) { const int t = div_by(w.tb, w.by_ck); tile = w.tail_tile0 + t; chunk = w.tb - t * w.Ck; }
     else { tile = w.tile1; chunk = 0; }
   }
   // returns true when the position jumped (phase switch), i.e. the tile position must be recomputed
@@ -528,7 +556,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   }
   __syncthreads();
 
-  const int kp = blockIdx.x / c.n_rp, rp = blockIdx.x - kp * c.n_rp;
+  int kp = 0, rp = (int)blockIdx.x;
+  if (c.n_kp > 1) { kp = rp / c.n_rp; rp -= kp * c.n_rp; }
   // Programmatic dependent launch: the next kernel of the stream may be set up while this one runs (its
   // blocks still need this block's resources, so they start as blocks here exit) ...
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -720,8 +749,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           if (c.n_kp == 1 && !tail) {
             total = 1;
           } else {
-            const int base = P.tiles / c.n_rp;
-            const int R = P.tiles - base * c.n_rp;
+            const int R = P.R;
             for (int q2 = 0; q2 < c.n_kp; ++q2) {
               int n_here = 1, first = rp;                      // a whole tile: one block per k-part
               if (tail) {
@@ -843,6 +871,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     if (wk.n1 == 0 && wk.te - wk.tb < wk.Ck) { ch0 = wk.tb % wk.Ck; n_ch = wk.te - wk.tb; }
     const int cgz = c.cgz, cg_sh = c.cgz > CG ? 4 : 3;
     const int Gn = n_ch * cgz;
+    // batch row of (row, group) pair number `pair` = pair / Gn, without the division (at most 15 steps)
+    auto row_of = [&](int pair) { int m = 0; while (pair >= Gn) { pair -= Gn; ++m; } return m; };
     auto needed_group = [&](int gn) { int ch = ch0 + (gn >> cg_sh); if (ch >= wk.Ck) ch -= wk.Ck; return (ch << cg_sh) + (gn & (cgz - 1)); };
     if (NT == 0) {          // (the integer path writes every entry it later reads)
       for (int i = ctid; i < Gk * 8 * MT; i += CTH) xg[i] = make_float2(0.f, 0.f);
@@ -866,7 +896,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           const int u = u0 + q4 * CTH;
           in[q4] = make_uint4(0, 0, 0, 0);
           if (u < n_units) {
-            const int pair = u >> 4, m = pair / Gn, lv = needed_group(pair - m * Gn);
+            const int pair = u >> 4, m = row_of(pair), lv = needed_group(pair - m * Gn);
             const int t0 = compact_of((sg_lo + lv) * kGroup + 8 * (u & 15));
             if (lv < Gk && t0 >= 0) in[q4] = load16(x + (size_t)m * ldx + t0);
           }
@@ -876,7 +906,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           const int u = u0 + q4 * CTH;
           if (u >= ((n_units + 31) & ~31)) break;                  // warp-uniform
           const int u16 = u & 15, pair = u < n_units ? u >> 4 : 0;
-          const int m = pair / Gn, lv = needed_group(pair - m * Gn);
+          const int m = row_of(pair), lv = needed_group(pair - m * Gn);
           const bool in_range = u < n_units && lv < Gk;
           uint2 hi2, lo2;
           int isum;
@@ -901,7 +931,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           const int u = u0 + q4 * CTH;
           in[q4] = make_uint4(0, 0, 0, 0);
           if (u < n_units) {
-            const int pair = u >> 4, m = pair / Gn, lv = needed_group(pair - m * Gn);
+            const int pair = u >> 4, m = row_of(pair), lv = needed_group(pair - m * Gn);
             const int t0 = compact_of((sg_lo + lv) * kGroup + 8 * (u & 15));
             if (lv < Gk && t0 >= 0) in[q4] = load16(x + (size_t)m * ldx + t0);
           }
@@ -911,7 +941,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           const int u = u0 + q4 * CTH;
           if (u >= ((n_units + 31) & ~31)) break;                  // warp-uniform
           const int u16 = u & 15, pair = u < n_units ? u >> 4 : 0;
-          const int m = pair / Gn, lv = needed_group(pair - m * Gn);
+          const int m = row_of(pair), lv = needed_group(pair - m * Gn);
           const bool in_range = u < n_units && lv < Gk;
           uint4 o;
           o.x = __byte_perm(in[q4].x, in[q4].z, 0x5410); o.y = __byte_perm(in[q4].x, in[q4].z, 0x7632);
@@ -1384,6 +1414,18 @@ long schedule_cost(long tiles, long Ck, long n_rp) {
   return base * Ck + (split ? (R * Ck + n_rp - 1) / n_rp + 3 : Ck);
 }
 
+// the host's part of the work split of one phase (see Phase)
+void fill_split(const DecodeCfg& c, Phase* P) {
+  P->base = P->tiles / c.n_rp;
+  P->R = P->tiles - P->base * c.n_rp;
+  P->gk0 = P->g_total < c.gp ? P->g_total : c.gp;
+  P->ck0 = (P->gk0 + c.cgz - 1) / c.cgz;
+  P->bt0 = tail_blocks(c.n_rp, P->R, P->ck0);
+  const unsigned long long ut = (unsigned long long)P->R * P->ck0;
+  P->by_ck0 = fast_div((unsigned)P->ck0, ut);
+  P->by_bt0 = fast_div((unsigned)P->bt0, ut * (unsigned long long)c.n_rp);
+}
+
 template <int MT, bool ONECOL, int NT, int NPH, bool XS = false>
 int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stream) {
   auto kern = decode_kernel<MT, ONECOL, NT, NPH, XS>;
@@ -1628,6 +1670,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   }
   c.n_tf = n_tf;
   c.tiles_total = tiles;
+  for (int i = 0; i < n_tf; ++i) c.tf[i].by_tpb = fast_div((unsigned)c.tf[i].tpb, (unsigned long long)tiles);
   c.n_ph = 1;
   {
     Phase& P = c.ph[0];
@@ -1636,6 +1679,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
     P.period = p.imap.fam[0].period; P.count = p.imap.fam[0].count;
     P.g_total = g_total; P.v_first = v_first;
     P.tile0 = 0; P.tiles = tiles;
+    fill_split(c, &P);
   }
   if (tiles < 1 || tiles * EW > kCounterInts) return UNIQL_ERR_UNSUPPORTED;
   c.max_slots = slots_needed(tiles, c.g_total, c.gp, c.n_rp, c.cgz);
@@ -1794,8 +1838,10 @@ int launch_mlp_phases(const MlpDecode& d, int first, int count, const LaunchCfg&
   }
   c.n_tf = n_tf;
   c.tiles_total = tiles;
+  for (int i = 0; i < n_tf; ++i) c.tf[i].by_tpb = fast_div((unsigned)c.tf[i].tpb, (unsigned long long)tiles);
   if (tiles < 1 || tiles * EW > kCounterInts) return UNIQL_ERR_UNSUPPORTED;
   c.max_slots = 0;
+  for (int i = 0; i < count; ++i) fill_split(c, &c.ph[i]);
   for (int i = 0; i < count; ++i) {
     const int sl = slots_needed(c.ph[i].tiles, c.ph[i].g_total, c.gp, c.n_rp, c.cgz);
     if (sl > c.max_slots) c.max_slots = sl;
