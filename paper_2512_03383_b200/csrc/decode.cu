@@ -370,9 +370,10 @@ __device__ inline void next_tile(const DecodeCfg& c, const Params& p, TilePos& q
   }
 }
 
-// The block (of its k-part) whose unit range [U*b/B, U*(b+1)/B) holds unit u; exact in fp64 here.
-__device__ inline int owner_of(long u, long B, long U) {
-  return (int)floor(((double)(u + 1) * (double)B - 1.0) / (double)U);
+// The block (of its k-part) whose unit range [U*b/B, U*(b+1)/B) holds unit u: floor(((u + 1) * B - 1) / U), in
+// 32-bit integers (the host checks U * B < 2^31).
+__device__ inline int owner_of(int u, int B, int U) {
+  return (int)(((unsigned)(u + 1) * (unsigned)B - 1u) / (unsigned)U);
 }
 
 // bias, rotary embedding on the retained pair, one rounding, store; `get(slot, m)` yields the fp32 sum
@@ -754,10 +755,10 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
               int n_here = 1, first = rp;                      // a whole tile: one block per k-part
               if (tail) {
                 const int Gq = min(c.gp, P.g_total - q2 * c.gp);
-                const long Cq = (Gq + c.cgz - 1) / c.cgz;
-                const long Ut = (long)R * Cq;
-                const long Bt = tail_blocks(c.n_rp, R, (int)Cq);
-                const long t0 = (long)(tile - wk.tail_tile0) * Cq;
+                const int Cq = Gq == P.gk0 ? P.ck0 : (Gq + c.cgz - 1) / c.cgz;
+                const int Ut = R * Cq;
+                const int Bt = Gq == P.gk0 ? P.bt0 : tail_blocks(c.n_rp, R, Cq);
+                const int t0 = (tile - wk.tail_tile0) * Cq;
                 first = owner_of(t0, Bt, Ut);
                 n_here = owner_of(t0 + Cq - 1, Bt, Ut) - first + 1;
               }
