@@ -290,17 +290,20 @@ __device__ inline void quantise16(const uint4& in, uint2& hi2, uint2& lo2, int& 
     if (amax * __uint_as_float((uint32_t)(127 + e) << 23) > 32639.f) --e;     // keep the high byte of x_i + 128 signed
   }
   const float scale = __uint_as_float((uint32_t)(127 + e) << 23), inv_scale = __uint_as_float((uint32_t)(127 - e) << 23);
-  int isum = 0;
-  uint32_t hi_e = 0, hi_o = 0, lo_e = 0, lo_o = 0;
+  // t_k = x_i + 128 through the float adder: x * 2^e + (1.5 * 2^23 + 128) is rounded to an integer (nearest even,
+  // as rint) whose low mantissa bits are t_k.  Byte 1 of t_k is hi, byte 0 of t_k xor 0x80 is lo; the bytes are
+  // gathered with byte permutes.
+  int tk[8];
+  int isum = -8 * 128;
 #pragma unroll
   for (int k = 0; k < 8; ++k) {
-    const int xi = __float2int_rn(f[k] * scale);
-    isum += xi;
-    const int hi = (xi + 128) >> 8, lo = xi - (hi << 8);
-    const int sh = 8 * (k >> 1);
-    if (k & 1) { hi_o |= (uint32_t)(hi & 255) << sh; lo_o |= (uint32_t)(lo & 255) << sh; }
-    else       { hi_e |= (uint32_t)(hi & 255) << sh; lo_e |= (uint32_t)(lo & 255) << sh; }
+    tk[k] = __float_as_int(fmaf(f[k], scale, 12582912.f + 128.f)) - 0x4B400000;
+    isum += tk[k];
   }
+  const uint32_t hi_e = __byte_perm(__byte_perm(tk[0], tk[2], 0x0051), __byte_perm(tk[4], tk[6], 0x0051), 0x5410);
+  const uint32_t hi_o = __byte_perm(__byte_perm(tk[1], tk[3], 0x0051), __byte_perm(tk[5], tk[7], 0x0051), 0x5410);
+  const uint32_t lo_e = __byte_perm(__byte_perm(tk[0], tk[2], 0x0040), __byte_perm(tk[4], tk[6], 0x0040), 0x5410) ^ 0x80808080u;
+  const uint32_t lo_o = __byte_perm(__byte_perm(tk[1], tk[3], 0x0040), __byte_perm(tk[5], tk[7], 0x0040), 0x5410) ^ 0x80808080u;
 #pragma unroll
   for (int o2 = 8; o2 >= 1; o2 >>= 1) isum += __shfl_xor_sync(0xffffffffu, isum, o2);
   hi2 = make_uint2(hi_e, hi_o);
