@@ -611,11 +611,17 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       for (int iu = 0; iu < wk.n_units; ++iu, ++it) {
         if (it >= S) ok = mbar_wait(bar_empty + 8 * s, ring_parity, abort_flag);
         if (!ok) break;
-        if (ui.tile != tile_prev) {
+        const bool new_tile = ui.tile != tile_prev;
+        if (new_tile) {
           if (jumped) q = tile_pos(c, p, ui.tile); else next_tile(c, p, q);
           jumped = false;
+          mode = c.tf[q.fi].mode;
+          tile_prev = ui.tile;
+        }
+        // (the rows of scales and zero-points of a new tile are worked out after its first weight boxes are on
+        //  their way: they need several more dependent reads of the kernel parameters)
+        auto setup_rows = [&]() {
           const TileFam& f = c.tf[q.fi];
-          mode = f.mode;
 #pragma unroll
           for (int r2 = 0; r2 < 2; ++r2) {
             const JobDev& jb = p.job[(mode == kSwiglu && r2) ? f.job2 : f.job];
@@ -638,8 +644,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
             srow[r2] = sr >= 0 ? jb.scales + (size_t)sr * G + sg_lo + gsh : nullptr;
             zrow[r2] = sr >= 0 ? jb.zeros + (size_t)sr * G + sg_lo + gsh : nullptr;
           }
-          tile_prev = ui.tile;
-        }
+        };
         const int chunk = ui.chunk;
         const int ng_all = min(c.cgz, Gk - chunk * c.cgz);  // visited groups of the unit
         const int ng = min(CG, ng_all), ng2 = ng_all - ng;  // ... in row slots 0..31 (all 64 unless narrow) / 32..63
@@ -671,6 +676,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
             tma_box3(dst, &c.wmap[q.fi], xb, q.r0, q.h, full);
           }
         }
+        if (new_tile) setup_rows();
 #pragma unroll
         for (int r2 = 0; r2 < 2; ++r2) {
           const int ngr = (mode == kNarrow && r2) ? ng2 : ng;      // groups of this half of the row slots
