@@ -242,6 +242,30 @@ def test_caller_workspace(B):
         check_output(y, ref, "f16", TIGHT, "caller workspace")
 
 
+@pytest.mark.parametrize("M,N,K", [(8, 4096, 14336), (16, 4096, 14336), (4, 4096, 14336), (1, 28672, 4096), (8, 1024, 8192)])
+def test_caller_workspace_is_large_enough_at_model_sizes(B, M, N, K):
+    """uniql_workspace_bytes() covers what the launch needs at full layer sizes, including the quantised copy of the
+    activations that long rows at eight batch rows stream through the ring (sampled output columns)."""
+    rng = np.random.default_rng(400 + M)
+    qw = synth.random_qweight_fast(rng, N, K)
+    packed, wp, ws_, wz = dev_weight(qw)
+    nbytes = B.workspace_bytes(M, K, N)
+    ws = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+    off = (-ws.data_ptr()) % 256
+    ws = ws[off:off + nbytes]
+    B.workspace_init(ws)
+    x = synth.draw_x(rng, M, K, "f16", outlier_frac=0.005)
+    xd = dev_x(x, "f16")
+    y = torch.zeros((M, N), dtype=torch.float16, device="cuda")
+    for _ in range(2):
+        B.qlinear_ex(xd, K, wp, ws_, wz, None, M, K, N, None, K, None, N, y, N, workspace=ws)
+        torch.cuda.synchronize()
+        assert B.workspace_status(ws) == 0
+    cols = np.unique(np.concatenate([[0, 63, 64, N - 1], rng.integers(0, N, 200)])).astype(np.int32)
+    ref = oracle.qlinear(x, packed, qw.scales, qw.zeros, cols, oracle.leading(K))
+    check_output(y[:, torch.from_numpy(cols.astype(np.int64)).cuda()], ref, "f16", TIGHT, "caller workspace M=%d" % M)
+
+
 # ---------------------------------------------------------------- channel maps (per-head pruning)
 @pytest.mark.parametrize("M", [1, 6, 16, 33])
 def test_per_head_maps(B, M):
