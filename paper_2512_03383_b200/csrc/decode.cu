@@ -1439,8 +1439,19 @@ void fill_split(const DecodeCfg& c, Phase* P) {
 template <int MT, bool ONECOL, int NT, int NPH, bool XS = false>
 int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stream) {
   auto kern = decode_kernel<MT, ONECOL, NT, NPH, XS>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return UNIQL_ERR_CUDA;
+  {
+    // the shared-memory limit of this instance is raised once per device (the call costs about a microsecond)
+    static std::mutex mu;
+    static bool done[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return UNIQL_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (dev < 0 || dev >= 64 || !done[dev]) {
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax) != cudaSuccess)
+        return UNIQL_ERR_CUDA;
+      if (dev >= 0 && dev < 64) done[dev] = true;
+    }
+  }
   cudaLaunchConfig_t lc;
   memset(&lc, 0, sizeof(lc));
   lc.gridDim = dim3(c.n_kp * c.n_rp);
