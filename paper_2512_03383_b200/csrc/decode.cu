@@ -139,6 +139,8 @@ struct DecodeCfg {
   // Streamed activations (rows too long to stage whole beside the ring): a small kernel quantises x once
   // into the layout the consumers read, [group][virtual row][128 bytes] plus (integer sum, 2^-e) per (group,
   // batch row), and every stage of the ring carries the eight groups of its unit beside the weights.
+  int x_cluster;         // blocks run as clusters of two that share the staging of the activations: each quantises
+                         // half of the (row, group) pairs and writes them into both blocks' shared memory
   int x_stream;
   int stage_bytes;       // STAGE_BYTES, plus vr * CG * 128 + 1024 when the activations are streamed
   int vr;                // virtual rows per group in a stage: 8 (up to four batch rows) or 16
@@ -165,6 +167,33 @@ __device__ inline bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// ---- cluster of two (shared staging of the activations)
+__device__ inline uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// address of `addr` (shared memory of this block) in block `rank` of the cluster
+__device__ inline uint32_t peer_addr(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ inline void st_peer_v2(uint32_t addr, uint32_t a, uint32_t b) {
+  asm volatile("st.shared::cluster.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(a), "r"(b) : "memory");
+}
+__device__ inline void mbar_arrive_peer(uint32_t addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(addr) : "memory");
+}
+__device__ inline bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
@@ -553,13 +582,16 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       mbar_init(bar_empty + 8 * s, CW);
     }
     mbar_init(bar_cons, CW);
-    mbar_init(bar_epi, EW);
+    mbar_init(bar_epi, c.x_cluster ? 2 * CW : EW);        // shared staging: the consumer warps of both blocks arrive
     for (int b = 0; b < 2; ++b) { mbar_init(bar_pfull + 8 * b, CW); mbar_init(bar_pfree + 8 * b, EW); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
 
+  // shared staging: every thread of the pair arrives at the cluster barrier once its block's barriers exist; the
+  // consumer warps wait for it before they first touch the other block's shared memory
+  if (c.x_cluster) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   int kp = 0, rp = (int)blockIdx.x;
   if (c.n_kp > 1) { kp = rp / c.n_rp; rp -= kp * c.n_rp; }
   // Programmatic dependent launch: the next kernel of the stream may be set up while this one runs (its
@@ -896,8 +928,19 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       // x_i = 256 * hi + lo with both bytes signed; the bytes go to two "virtual"
       // batch rows (columns 2m and 2m+1 of the int8 MMA), in the order the nibbles leave a weight word:
       // even codes in the first register of a word's pair, odd codes in the second.
-      const int n_units = Gn * p.M * 16;
+      // Shared staging (clusters of two): this block quantises the pairs of its own parity and writes them into
+      // both blocks' shared memory (same layout, same offsets); the other block does the same for the rest.
+      const bool xc = NPH == 1 && !XS && c.x_cluster != 0;
+      const int crank = xc ? (int)cluster_rank() : 0, csh = xc ? 1 : 0;
+      const int n_pairs = Gn * p.M;
+      const int n_units = ((n_pairs - crank + csh) >> csh) * 16;     // units of this block's pairs
       unsigned char* xb = smem + c.off_x;
+      uint32_t px = 0, pxg = 0;                                      // the other block's x and xg regions
+      if (xc) {
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // its barriers exist
+        px = peer_addr(sbase + (uint32_t)c.off_x, (uint32_t)(crank ^ 1));
+        pxg = peer_addr(sbase + (uint32_t)c.off_xg, (uint32_t)(crank ^ 1));
+      }
       constexpr int UN = 4;
       for (int u0 = ctid; u0 < ((n_units + 31) & ~31); u0 += CTH * UN) {
         uint4 in[UN];
@@ -906,7 +949,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           const int u = u0 + q4 * CTH;
           in[q4] = make_uint4(0, 0, 0, 0);
           if (u < n_units) {
-            const int pair = u >> 4, m = row_of(pair), lv = needed_group(pair - m * Gn);
+            const int pair = ((u >> 4) << csh) + crank, m = row_of(pair), lv = needed_group(pair - m * Gn);
             const int t0 = compact_of((sg_lo + lv) * kGroup + 8 * (u & 15));
             if (lv < Gk && t0 >= 0) in[q4] = load16(x + (size_t)m * ldx + t0);
           }
@@ -915,7 +958,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         for (int q4 = 0; q4 < UN; ++q4) {
           const int u = u0 + q4 * CTH;
           if (u >= ((n_units + 31) & ~31)) break;                  // warp-uniform
-          const int u16 = u & 15, pair = u < n_units ? u >> 4 : 0;
+          const int u16 = u & 15, pair = u < n_units ? ((u >> 4) << csh) + crank : 0;
           const int m = row_of(pair), lv = needed_group(pair - m * Gn);
           const bool in_range = u < n_units && lv < Gk;
           uint2 hi2, lo2;
@@ -928,8 +971,32 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
             *reinterpret_cast<uint2*>(xb + (size_t)(2 * m) * c.xrow + off) = hi2;
             *reinterpret_cast<uint2*>(xb + (size_t)(2 * m + 1) * c.xrow + off) = lo2;
             if (u16 == 0) xg[lv * 8 * MT + m] = make_float2((float)isum, inv_scale);
+            if (xc) {
+              st_peer_v2(px + (uint32_t)((2 * m) * c.xrow + off), hi2.x, hi2.y);
+              st_peer_v2(px + (uint32_t)((2 * m + 1) * c.xrow + off), lo2.x, lo2.y);
+              if (u16 == 0) st_peer_v2(pxg + (uint32_t)((lv * 8 * MT + m) * 8), (uint32_t)__float_as_int((float)isum),
+                                       (uint32_t)__float_as_int(inv_scale));
+            }
           }
         }
+      }
+      if (xc) {
+        // both halves are in place once the sixteen consumer warps of each block have arrived at this block's
+        // barrier (bounded wait; the other block cannot leave before it has seen this block's arrivals, and this
+        // block writes nothing into it after them)
+        __syncwarp();
+        if (lane == 0) {
+          asm volatile("fence.acq_rel.cluster;" ::: "memory");
+          mbar_arrive(bar_epi);
+          mbar_arrive_peer(peer_addr(bar_epi, (uint32_t)(crank ^ 1)));
+        }
+        bool ok = false;
+        for (int i = 0; i < kWaitLimit && !ok; ++i) {
+          ok = mbar_try_wait_cluster(bar_epi, 0);
+          if (!ok && (i & 63) == 63 && *abort_flag) break;
+        }
+        if (!ok) { *abort_flag = 1; give_up(); return false; }
+        return true;
       }
     } else if (c.x_vec) {
       const int n_units = Gn * p.M * 16;
@@ -1458,7 +1525,8 @@ int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stre
   lc.blockDim = dim3(NTH);
   lc.dynamicSmemBytes = smem;
   lc.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
+  lc.attrs = attr;
   if (NPH > 1) {
     // the blocks of a fused launch wait on one another: all of them must be resident at once
     attr[0].id = cudaLaunchAttributeCooperative;
@@ -1469,9 +1537,30 @@ int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stre
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.numAttrs = env_int("UNIQL_PDL", 1) ? 1 : 0;
   }
-  lc.attrs = attr;
-  if (cudaLaunchKernelEx(&lc, kern, p, c) != cudaSuccess) { cudaGetLastError(); return UNIQL_ERR_CUDA; }
-  return UNIQL_OK;
+  DecodeCfg cc = c;
+  if (cc.x_cluster) {
+    // clusters of two (shared staging): only when every pair can be resident at once, else plain blocks
+    attr[lc.numAttrs].id = cudaLaunchAttributeClusterDimension;
+    attr[lc.numAttrs].val.clusterDim.x = 2;
+    attr[lc.numAttrs].val.clusterDim.y = 1;
+    attr[lc.numAttrs].val.clusterDim.z = 1;
+    ++lc.numAttrs;
+    int n_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&n_clusters, kern, &lc) != cudaSuccess || n_clusters * 2 < (int)lc.gridDim.x) {
+      cudaGetLastError();
+      --lc.numAttrs;
+      cc.x_cluster = 0;
+    }
+  }
+  if (cudaLaunchKernelEx(&lc, kern, p, cc) == cudaSuccess) return UNIQL_OK;
+  cudaGetLastError();
+  if (cc.x_cluster) {                    // the launch as clusters was refused: plain blocks
+    --lc.numAttrs;
+    cc.x_cluster = 0;
+    if (cudaLaunchKernelEx(&lc, kern, p, cc) == cudaSuccess) return UNIQL_OK;
+    cudaGetLastError();
+  }
+  return UNIQL_ERR_CUDA;
 }
 
 // Visited groups of the input map: from the first to the last 128-channel group that holds a retained
@@ -1701,6 +1790,16 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
     P.g_total = g_total; P.v_first = v_first;
     P.tile0 = 0; P.tiles = tiles;
     fill_split(c, &P);
+    // Shared staging in clusters of two: integer path, activations staged whole by every block (no k-split, no
+    // streaming, no block that stages only the chunks of a short run), blocks paired so that both have work or
+    // neither has.  UNIQL_DECODE_XCLUSTER=0 turns it off.
+    const bool all_stage_everything = P.base > 0 || P.R == 0 || (P.R * P.ck0) / P.bt0 >= P.ck0;
+    const bool pairs_alike = P.base > 0 || (P.bt0 % 2) == 0;
+    // Launching as clusters delays the start of the blocks (pairs of free SMs are needed, measured 1.5 - 2 us on the
+    // small launches), so it is used where the staging is long: eight or more 16-byte units per thread.
+    const int force_xc = env_int("UNIQL_DECODE_XCLUSTER", -1);
+    c.x_cluster = i8 && !c.x_stream && c.n_kp == 1 && (c.n_rp % 2) == 0 && p.M <= 8 && all_stage_everything &&
+                  pairs_alike && force_xc != 0 && (force_xc == 1 || g_total * p.M >= 256);
   }
   if (tiles < 1 || tiles * EW > kCounterInts) return UNIQL_ERR_UNSUPPORTED;
   c.max_slots = slots_needed(tiles, c.g_total, c.gp, c.n_rp, c.cgz);

@@ -31,7 +31,7 @@ def B():
 def _reset_path(B):
     yield
     B.set_path(B.PATH_AUTO)
-    for k in ("UNIQL_DECODE_KP", "UNIQL_DECODE_RP", "UNIQL_DECODE_NARROW", "UNIQL_DECODE_XSTREAM"):
+    for k in ("UNIQL_DECODE_KP", "UNIQL_DECODE_RP", "UNIQL_DECODE_NARROW", "UNIQL_DECODE_XSTREAM", "UNIQL_DECODE_XCLUSTER"):
         os.environ.pop(k, None)
 
 
@@ -223,6 +223,37 @@ def test_tiny_and_ragged_shapes(B, M, dtype):
         dw = dev_weight(qw)
         with pytest.raises(RuntimeError):
             run_ex(B, qw, dw, synth.draw_x(rng, M, 128, dtype), dtype, None, bad[0], None, min(bad[1], 8))
+
+
+@pytest.mark.parametrize("xc", [0, 1])
+@pytest.mark.parametrize("rp", [0, 2, 6])
+@pytest.mark.parametrize("M", [1, 3, 4, 8, 16])
+def test_shared_staging_in_clusters(B, xc, rp, M):
+    """Blocks launched as clusters of two, each quantising half of the activations into both blocks' shared memory
+    (used by default where the staging is long), against every block staging everything."""
+    os.environ["UNIQL_DECODE_XCLUSTER"] = str(xc)
+    if rp:
+        os.environ["UNIQL_DECODE_RP"] = str(rp)
+    B.set_path(B.PATH_DECODE)
+    rng = np.random.default_rng(500 + M)
+    for (N, K, k_in, k_out) in [(300, 1024, 1024, 300), (200, 2304, 1096, 77), (96, 256, 256, 96), (640, 3328, 3072, 600)]:
+        qw = synth.draw_qweight(rng, N, K)
+        dw = dev_weight(qw)
+        bias = synth.to_dtype_values(rng.standard_normal(N).astype(np.float32), "f16")
+        x = synth.draw_x(rng, M, k_in, "f16")
+        y, ref = run_ex(B, qw, dw, x, "f16", None, k_in, None, k_out, bias=bias, ldy_pad=3)
+        check_output(y, ref, "f16", TIGHT, "xc=%d rp=%d M=%d %s" % (xc, rp, M, (N, K, k_in, k_out)))
+        y2, _ = run_ex(B, qw, dw, x, "f16", None, k_in, None, k_out, bias=bias, ldy_pad=3)
+        assert torch.equal(y, y2), "run-to-run results differ"
+    qw = synth.draw_qweight(rng, 512, 1024)
+    dw = dev_weight(qw)
+    in_map = synth.map_per_head(8, 128, 96)
+    x = synth.draw_x(rng, M, synth.map_size(in_map), "f16")
+    y, ref = run_ex(B, qw, dw, x, "f16", in_map, 0, synth.map_per_head(4, 128, 108), 0)
+    check_output(y, ref, "f16", TIGHT, "xc=%d per-head M=%d" % (xc, M))
+    for (g, ref) in run_rope(B, rng, M, 512, 6, 2, 128, 96, 500000.0, "f16", bias=True, v_keep=104):
+        check_output(g, ref, "f16", TIGHT, "xc=%d q/k/v M=%d" % (xc, M))
+    assert B.workspace_status() == 0
 
 
 def test_caller_workspace(B):
