@@ -559,7 +559,8 @@ struct UnitIter {
 // NT == 0: fp16 tensor-core path (MT batch tiles of 8, ONECOL: batch 1).  NT > 0: integer path, NT column
 // tiles of the int8 MMA, each holding the high and the low byte of four batch rows.
 // NPH: phases (2: the fused SwiGLU MLP, integer path only).  XS: activations streamed through the ring.
-template <int MT, bool ONECOL, int NT, int NPH, bool XS>
+// XC: blocks are launched as clusters of two that share the staging of the activations.
+template <int MT, bool ONECOL, int NT, int NPH, bool XS, bool XC>
 __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ Params p,
                                                         const __grid_constant__ DecodeCfg c) {
   extern __shared__ unsigned char smem_raw[];
@@ -582,7 +583,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       mbar_init(bar_empty + 8 * s, CW);
     }
     mbar_init(bar_cons, CW);
-    mbar_init(bar_epi, c.x_cluster ? 2 * CW : EW);        // shared staging: the consumer warps of both blocks arrive
+    mbar_init(bar_epi, XC ? 2 * CW : EW);        // shared staging: the consumer warps of both blocks arrive
     for (int b = 0; b < 2; ++b) { mbar_init(bar_pfull + 8 * b, CW); mbar_init(bar_pfree + 8 * b, EW); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -591,7 +592,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
 
   // shared staging: every thread of the pair arrives at the cluster barrier once its block's barriers exist; the
   // consumer warps wait for it before they first touch the other block's shared memory
-  if (c.x_cluster) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  if (XC) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   int kp = 0, rp = (int)blockIdx.x;
   if (c.n_kp > 1) { kp = rp / c.n_rp; rp -= kp * c.n_rp; }
   // Programmatic dependent launch: the next kernel of the stream may be set up while this one runs (its
@@ -930,7 +931,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       // even codes in the first register of a word's pair, odd codes in the second.
       // Shared staging (clusters of two): this block quantises the pairs of its own parity and writes them into
       // both blocks' shared memory (same layout, same offsets); the other block does the same for the rest.
-      const bool xc = NPH == 1 && !XS && c.x_cluster != 0;
+      constexpr bool xc = XC;
       const int crank = xc ? (int)cluster_rank() : 0, csh = xc ? 1 : 0;
       const int n_pairs = Gn * p.M;
       const int n_units = ((n_pairs - crank + csh) >> csh) * 16;     // units of this block's pairs
@@ -1503,9 +1504,9 @@ void fill_split(const DecodeCfg& c, Phase* P) {
   P->by_bt0 = fast_div((unsigned)P->bt0, ut * (unsigned long long)c.n_rp);
 }
 
-template <int MT, bool ONECOL, int NT, int NPH, bool XS = false>
+template <int MT, bool ONECOL, int NT, int NPH, bool XS = false, bool XC = false>
 int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stream) {
-  auto kern = decode_kernel<MT, ONECOL, NT, NPH, XS>;
+  auto kern = decode_kernel<MT, ONECOL, NT, NPH, XS, XC>;
   {
     // the shared-memory limit of this instance is raised once per device (the call costs about a microsecond)
     static std::mutex mu;
@@ -1538,7 +1539,7 @@ int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stre
     lc.numAttrs = env_int("UNIQL_PDL", 1) ? 1 : 0;
   }
   DecodeCfg cc = c;
-  if (cc.x_cluster) {
+  if (XC) {
     // clusters of two (shared staging): only when every pair can be resident at once, else plain blocks
     attr[lc.numAttrs].id = cudaLaunchAttributeClusterDimension;
     attr[lc.numAttrs].val.clusterDim.x = 2;
@@ -1548,19 +1549,12 @@ int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stre
     int n_clusters = 0;
     if (cudaOccupancyMaxActiveClusters(&n_clusters, kern, &lc) != cudaSuccess || n_clusters * 2 < (int)lc.gridDim.x) {
       cudaGetLastError();
-      --lc.numAttrs;
-      cc.x_cluster = 0;
+      return UNIQL_ERR_UNSUPPORTED;        // the caller launches plain blocks instead
     }
   }
   if (cudaLaunchKernelEx(&lc, kern, p, cc) == cudaSuccess) return UNIQL_OK;
   cudaGetLastError();
-  if (cc.x_cluster) {                    // the launch as clusters was refused: plain blocks
-    --lc.numAttrs;
-    cc.x_cluster = 0;
-    if (cudaLaunchKernelEx(&lc, kern, p, cc) == cudaSuccess) return UNIQL_OK;
-    cudaGetLastError();
-  }
-  return UNIQL_ERR_CUDA;
+  return XC ? UNIQL_ERR_UNSUPPORTED : UNIQL_ERR_CUDA;
 }
 
 // Visited groups of the input map: from the first to the last 128-channel group that holds a retained
@@ -1849,6 +1843,12 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   if (c.x_stream) {
     if (p.M <= 4) return launch_t<1, false, 1, 1, true>(p, c, smem, cfg.stream);
     return launch_t<1, false, 2, 1, true>(p, c, smem, cfg.stream);
+  }
+  if (i8 && c.x_cluster) {
+    const int rc = p.M <= 4 ? launch_t<1, false, 1, 1, false, true>(p, c, smem, cfg.stream)
+                            : launch_t<1, false, 2, 1, false, true>(p, c, smem, cfg.stream);
+    if (rc != UNIQL_ERR_UNSUPPORTED) return rc;
+    c.x_cluster = 0;                       // clusters cannot all be resident, or the launch was refused
   }
   if (i8) {
     if (p.M <= 4) return launch_t<1, false, 1, 1>(p, c, smem, cfg.stream);
