@@ -571,6 +571,10 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   const uint32_t sbase = (raw + 1023u) & ~1023u;
   unsigned char* smem = smem_raw + (sbase - raw);
   const int S = c.stages;
+  // XS / XC say what this instance can do; whether a launch streams its activations or shares their staging is a
+  // flag of the launch (batches of five to eight rows always take the same instance: alternating between two
+  // kernel functions costs about 1.5 us per switch)
+  const bool xs_on = XS && c.x_stream != 0, xc_on = XC && c.x_cluster != 0;
   // barriers: full[S], empty[S], consumer barrier, (spare), partials full[2] / free[2]; then the abort flag
   const uint32_t bar_full = sbase + c.off_bar, bar_empty = bar_full + 8 * MAX_STAGES;
   const uint32_t bar_cons = bar_full + 16 * MAX_STAGES, bar_epi = bar_cons + 8;
@@ -583,7 +587,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       mbar_init(bar_empty + 8 * s, CW);
     }
     mbar_init(bar_cons, CW);
-    mbar_init(bar_epi, XC ? 2 * CW : EW);        // shared staging: the consumer warps of both blocks arrive
+    mbar_init(bar_epi, xc_on ? 2 * CW : EW);        // shared staging: the consumer warps of both blocks arrive
     for (int b = 0; b < 2; ++b) { mbar_init(bar_pfull + 8 * b, CW); mbar_init(bar_pfree + 8 * b, EW); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -592,7 +596,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
 
   // shared staging: every thread of the pair arrives at the cluster barrier once its block's barriers exist; the
   // consumer warps wait for it before they first touch the other block's shared memory
-  if (XC) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  if (xc_on) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   int kp = 0, rp = (int)blockIdx.x;
   if (c.n_kp > 1) { kp = rp / c.n_rp; rp -= kp * c.n_rp; }
   // Programmatic dependent launch: the next kernel of the stream may be set up while this one runs (its
@@ -612,7 +616,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     // fill of the ring do not wait for it: their stages are armed with the weight bytes only, and once the ring
     // is full (or the block's units are all issued) the producer waits for the predecessor and sends the
     // activations of those stages after them, with the arrival the stages' barriers still lack.
-    bool x_waited = !XS;
+    bool x_waited = !xs_on;
     int x_lv0[MAX_STAGES];
     auto send_x = [&](int stage, int lv0) {                          // lane 31: arrival + the unit's activations
       const uint32_t full = bar_full + 8 * stage;
@@ -683,16 +687,16 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         const int ng = min(CG, ng_all), ng2 = ng_all - ng;  // ... in row slots 0..31 (all 64 unless narrow) / 32..63
         const int nb = (ng + 1) >> 1, nb2 = (ng2 + 1) >> 1; // 128-byte columns with a visited group
         const uint32_t full = bar_full + 8 * s;
-        const uint32_t st = sbase + (uint32_t)s * (XS ? (uint32_t)c.stage_bytes : (uint32_t)STAGE_BYTES);
+        const uint32_t st = sbase + (uint32_t)s * (xs_on ? (uint32_t)c.stage_bytes : (uint32_t)STAGE_BYTES);
         const uint32_t wbytes = mode == kNarrow ? (uint32_t)((nb + nb2) * (BOX_BYTES / 2)) : (uint32_t)(nb * BOX_BYTES);
-        if (XS) {
+        if (xs_on) {
           if (lane == 0) mbar_expect_tx_only(full, wbytes);          // the arrival comes with the activations
           if (!x_waited) x_lv0[s] = chunk * CG;                      // (one k-part, wide tiles; s == it here)
         } else if (lane == 0) {
           mbar_expect_tx(full, wbytes);
         }
         __syncwarp();
-        if (XS && x_waited && lane == 31) send_x(s, chunk * CG);
+        if (xs_on && x_waited && lane == 31) send_x(s, chunk * CG);
         if (lane < nb) {
           const int xb = (sg_lo + chunk * c.cgz + 2 * lane) * 64;    // byte in the weight row
           const uint32_t dst = st + (uint32_t)lane * BOX_BYTES;
@@ -730,9 +734,9 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
         cp_async_arrive_noinc(full);
         if (iu + 1 < wk.n_units && ui.advance(wk, iu + 1)) jumped = true;
         if (++s == S) { s = 0; ring_parity ^= 1; }
-        if (XS && !x_waited && it + 1 == S) flush_x(S);
+        if (xs_on && !x_waited && it + 1 == S) flush_x(S);
       }
-      if (XS && !x_waited) flush_x(it);                              // fewer units than stages
+      if (xs_on && !x_waited) flush_x(it);                              // fewer units than stages
     }
     if (!ok) {
       // let the copies of the stages that are still armed land before the block goes away
@@ -931,7 +935,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       // even codes in the first register of a word's pair, odd codes in the second.
       // Shared staging (clusters of two): this block quantises the pairs of its own parity and writes them into
       // both blocks' shared memory (same layout, same offsets); the other block does the same for the rest.
-      constexpr bool xc = XC;
+      const bool xc = xc_on;
       const int crank = xc ? (int)cluster_rank() : 0, csh = xc ? 1 : 0;
       const int n_pairs = Gn * p.M;
       const int n_units = ((n_pairs - crank + csh) >> csh) * 16;     // units of this block's pairs
@@ -1083,7 +1087,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     }
     const uint32_t xgaddr8 = sbase + c.off_xg + (uint32_t)(t * 8);           // batch row m = t + 4 nt
     // streamed activations: line (group kpw, virtual row v) of the stage, its 16-byte chunks XOR-ed with v & 7
-    constexpr bool xstream = XS;
+    const bool xstream = xs_on;
     uint32_t xs0[NT], xs1[NT];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -1150,7 +1154,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       }
       const int gi = ui.chunk * c.cgz + g_first;
       if (gi < Gk) {
-        const uint32_t st = sbase + (uint32_t)s * (XS ? (uint32_t)c.stage_bytes : (uint32_t)STAGE_BYTES);
+        const uint32_t st = sbase + (uint32_t)s * (xs_on ? (uint32_t)c.stage_bytes : (uint32_t)STAGE_BYTES);
         const uint32_t wp = st + wl_off, sp = st + sl_off;
         uint4 wa[2], wb[2];
         wa[0] = lds128<0>(wp);
@@ -1539,7 +1543,8 @@ int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stre
     lc.numAttrs = env_int("UNIQL_PDL", 1) ? 1 : 0;
   }
   DecodeCfg cc = c;
-  if (XC) {
+  const bool as_clusters = XC && c.x_cluster != 0;
+  if (as_clusters) {
     // clusters of two (shared staging): only when every pair can be resident at once, else plain blocks
     attr[lc.numAttrs].id = cudaLaunchAttributeClusterDimension;
     attr[lc.numAttrs].val.clusterDim.x = 2;
@@ -1554,7 +1559,7 @@ int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stre
   }
   if (cudaLaunchKernelEx(&lc, kern, p, cc) == cudaSuccess) return UNIQL_OK;
   cudaGetLastError();
-  return XC ? UNIQL_ERR_UNSUPPORTED : UNIQL_ERR_CUDA;
+  return as_clusters ? UNIQL_ERR_UNSUPPORTED : UNIQL_ERR_CUDA;
 }
 
 // Visited groups of the input map: from the first to the last 128-channel group that holds a retained
@@ -1790,10 +1795,12 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
     const bool all_stage_everything = P.base > 0 || P.R == 0 || (P.R * P.ck0) / P.bt0 >= P.ck0;
     const bool pairs_alike = P.base > 0 || (P.bt0 % 2) == 0;
     // Launching as clusters delays the start of the blocks (pairs of free SMs are needed, measured 1.5 - 2 us on the
-    // small launches), so it is used where the staging is long: eight or more 16-byte units per thread.
+    // small launches), so it is used where the staging is long: seven or eight rows and eight or more 16-byte units
+    // per thread (smaller batches would alternate between two kernel functions within a layer, which costs more
+    // than the staging saved).
     const int force_xc = env_int("UNIQL_DECODE_XCLUSTER", -1);
     c.x_cluster = i8 && !c.x_stream && c.n_kp == 1 && (c.n_rp % 2) == 0 && p.M <= 8 && all_stage_everything &&
-                  pairs_alike && force_xc != 0 && (force_xc == 1 || g_total * p.M >= 256);
+                  pairs_alike && force_xc != 0 && (force_xc == 1 || (p.M >= 7 && g_total * p.M >= 256));
   }
   if (tiles < 1 || tiles * EW > kCounterInts) return UNIQL_ERR_UNSUPPORTED;
   c.max_slots = slots_needed(tiles, c.g_total, c.gp, c.n_rp, c.cgz);
@@ -1840,19 +1847,23 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
       return UNIQL_ERR_CUDA;
     }
   }
-  if (c.x_stream) {
-    if (p.M <= 4) return launch_t<1, false, 1, 1, true>(p, c, smem, cfg.stream);
-    return launch_t<1, false, 2, 1, true>(p, c, smem, cfg.stream);
+  if (i8 && p.M > 4 && p.M <= 8) {
+    // five to eight rows: one instance that can stream and share, whatever this launch does
+    int rc = launch_t<1, false, 2, 1, true, true>(p, c, smem, cfg.stream);
+    if (rc == UNIQL_ERR_UNSUPPORTED && c.x_cluster) {      // clusters cannot all be resident, or were refused
+      c.x_cluster = 0;
+      rc = launch_t<1, false, 2, 1, true, true>(p, c, smem, cfg.stream);
+    }
+    return rc;
   }
-  if (i8 && c.x_cluster) {
-    const int rc = p.M <= 4 ? launch_t<1, false, 1, 1, false, true>(p, c, smem, cfg.stream)
-                            : launch_t<1, false, 2, 1, false, true>(p, c, smem, cfg.stream);
+  if (c.x_stream) return launch_t<1, false, 1, 1, true>(p, c, smem, cfg.stream);      // (M <= 4: rows too long to stage)
+  if (i8 && c.x_cluster) {                                                           // (M <= 4: forced only)
+    const int rc = launch_t<1, false, 1, 1, false, true>(p, c, smem, cfg.stream);
     if (rc != UNIQL_ERR_UNSUPPORTED) return rc;
-    c.x_cluster = 0;                       // clusters cannot all be resident, or the launch was refused
+    c.x_cluster = 0;
   }
   if (i8) {
     if (p.M <= 4) return launch_t<1, false, 1, 1>(p, c, smem, cfg.stream);
-    if (p.M <= 8) return launch_t<1, false, 2, 1>(p, c, smem, cfg.stream);
     return launch_t<2, false, 4, 1>(p, c, smem, cfg.stream);
   }
   if (MT == 1)
@@ -1978,7 +1989,7 @@ int launch_mlp_phases(const MlpDecode& d, int first, int count, const LaunchCfg&
     return launch_t<1, false, 2, 2>(p, c, smem, cfg.stream);
   }
   if (d.M <= 4) return launch_t<1, false, 1, 1>(p, c, smem, cfg.stream);
-  if (d.M <= 8) return launch_t<1, false, 2, 1>(p, c, smem, cfg.stream);
+  if (d.M <= 8) return launch_t<1, false, 2, 1, true, true>(p, c, smem, cfg.stream);
   return launch_t<2, false, 4, 1>(p, c, smem, cfg.stream);
 }
 
