@@ -1989,7 +1989,18 @@ int launch_mlp_phases(const MlpDecode& d, int first, int count, const LaunchCfg&
     return launch_t<1, false, 2, 2>(p, c, smem, cfg.stream);
   }
   if (d.M <= 4) return launch_t<1, false, 1, 1>(p, c, smem, cfg.stream);
-  if (d.M <= 8) return launch_t<1, false, 2, 1, true, true>(p, c, smem, cfg.stream);
+  if (d.M <= 8) {
+    // shared staging under the rule of the plain launches (every block of the gate|up launch has whole tiles)
+    const Phase& P = c.ph[0];
+    const int force_xc = env_int("UNIQL_DECODE_XCLUSTER", -1);
+    c.x_cluster = c.n_kp == 1 && (c.n_rp % 2) == 0 && P.base > 0 && force_xc != 0 && d.M >= 7 && P.g_total * d.M >= 256;
+    int rc = launch_t<1, false, 2, 1, true, true>(p, c, smem, cfg.stream);
+    if (rc == UNIQL_ERR_UNSUPPORTED && c.x_cluster) {
+      c.x_cluster = 0;
+      rc = launch_t<1, false, 2, 1, true, true>(p, c, smem, cfg.stream);
+    }
+    return rc;
+  }
   return launch_t<2, false, 4, 1>(p, c, smem, cfg.stream);
 }
 
@@ -1999,7 +2010,18 @@ int launch_mlp_decode(const MlpDecode& d, int fuse, const LaunchCfg& cfg) {
   if (!mlp_decode_supported(d)) return UNIQL_ERR_UNSUPPORTED;
   if (fuse) return launch_mlp_phases(d, 0, 2, cfg);
   const int rc = launch_mlp_phases(d, 0, 1, cfg);
-  return rc ? rc : launch_mlp_phases(d, 1, 1, cfg);
+  if (rc) return rc;
+  // the down projection is an ordinary launch on h (leading k_int input channels, all hidden outputs): it takes
+  // the narrow tiles, the streamed or shared staging of the plain path as they apply
+  Params p;
+  memset(&p, 0, sizeof(p));
+  p.x = d.h; p.ldx = d.ldh; p.dt = UNIQL_F16; p.M = d.M; p.K = d.inter; p.k_in = d.k_int;
+  p.imap.n_fam = 1; p.imap.total = d.k_int; p.imap.fam[0] = Fam{0, d.k_int, d.k_int, 1}; p.imap.base[0] = 0;
+  p.n_jobs = 1;
+  JobDev& jd = p.job[0];
+  jd.w = d.wd; jd.scales = d.sd; jd.zeros = d.zd; jd.y = d.y; jd.ldy = d.ldy; jd.N = d.hidden; jd.k_out = d.hidden;
+  jd.omap.n_fam = 1; jd.omap.total = d.hidden; jd.omap.fam[0] = Fam{0, d.hidden, d.hidden, 1}; jd.omap.base[0] = 0;
+  return launch_decode(p, cfg);
 }
 
 int decode_status_offset() { return kStatusOff; }
