@@ -275,7 +275,7 @@ int qkv_rope_impl(const void* x, int ldx, int dt, const uint8_t* wq, const void*
   p.n_jobs = wv ? 3 : 2;
   p.idx = retained_idx; p.pos = pos;
   for (int i = 0; i < head_dim / 2; ++i)
-    p.inv_freq[i] = inv_freq ? inv_freq[i] : pow(theta, -2.0 * (double)i / (double)head_dim);
+    p.rope_turn[i] = rope_turn_of(inv_freq ? inv_freq[i] : pow(theta, -2.0 * (double)i / (double)head_dim));
   for (int j = 0; j < 2; ++j) {
     JobDev& d = p.job[j];
     int nh = j == 0 ? n_q_heads : n_kv_heads;

@@ -58,7 +58,7 @@ struct Params {
   JobDev job[kMaxJobs];
   const int32_t* idx;   // [n_kv_heads][head_keep/2] original pair indices
   const int32_t* pos;   // [M]
-  double inv_freq[kMaxHalfDim];
+  unsigned long long rope_turn[kMaxHalfDim];   // frac(inv_freq / 2 pi) * 2^64, per original pair
 };
 
 // ---------------------------------------------------------------- channel-map arithmetic
@@ -116,14 +116,21 @@ template <> struct DT<__nv_bfloat16> {
 
 // ---------------------------------------------------------------- rotary angle
 // cos / sin of pos * inv_freq.  The product reaches thousands of radians, where an fp32
-// product alone would already be off by ~1e-3 rad; it is formed and reduced modulo 2*pi in
-// fp64, then the fast fp32 intrinsics work on an argument in [-pi, pi].
-__device__ inline void rope_cos_sin(int pos, double inv_freq, float& c, float& s) {
-  double a = (double)pos * inv_freq;
-  const double two_pi = 6.283185307179586476925286766559;
-  const double inv_two_pi = 0.15915494309189533576888376337251;
-  a = fma(-rint(a * inv_two_pi), two_pi, a);
-  float af = (float)a;
+// product alone would already be off by ~1e-3 rad.  The host therefore passes each frequency
+// as a 64-bit fixed-point fraction of a turn (turn = frac(inv_freq / 2 pi) * 2^64): the
+// integer product pos * turn wraps modulo one turn by itself, exactly, and its upper 32 bits,
+// read as a signed number, are the reduced angle in [-1/2, 1/2) turns with 2^-32 resolution.
+// The fast fp32 intrinsics then work on an argument in [-pi, pi).  (fp64 arithmetic here cost
+// the 64 x 256 angles of one tensor-core tile about as much time as the tile's main loop.)
+__host__ inline unsigned long long rope_turn_of(double inv_freq) {
+  long double t = (long double)inv_freq / 6.283185307179586476925286766559L;
+  t -= floorl(t);
+  const long double scaled = t * 18446744073709551616.0L;
+  return scaled >= 18446744073709551615.0L ? ~0ull : (unsigned long long)scaled;
+}
+__device__ inline void rope_cos_sin(int pos, unsigned long long turn, float& c, float& s) {
+  const unsigned long long a = (unsigned long long)(long long)pos * turn;
+  const float af = (float)(int)(a >> 32) * (6.283185307179586476925286766559f / 4294967296.f);
   c = __cosf(af);
   s = __sinf(af);
 }

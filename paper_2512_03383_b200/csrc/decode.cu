@@ -449,7 +449,7 @@ __device__ inline void store_tile(const Params& p, const TileFam& f, const TileP
       int pidx = p.idx[(q.h / jb.rope.rep) * half + cc];
       pidx = min(max(pidx, 0), (jb.rope.head_dim >> 1) - 1);
       float cs, sn;
-      rope_cos_sin(p.pos[m], p.inv_freq[pidx], cs, sn);
+      rope_cos_sin(p.pos[m], p.rope_turn[pidx], cs, sn);
       const int oc = q.h * jb.rope.head_keep + cc;
       y[(size_t)m * jb.ldy + oc] = DT<T>::from_f(lo * cs - hi * sn);
       y[(size_t)m * jb.ldy + oc + half] = DT<T>::from_f(hi * cs + lo * sn);

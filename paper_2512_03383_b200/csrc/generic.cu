@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(NT) generic_kernel(const __grid_constant__ Par
       int pidx = p.idx[s_kvh[c] * half + s_pp[c]];
       pidx = min(max(pidx, 0), (jb.rope.head_dim >> 1) - 1);
       float cs, sn;
-      rope_cos_sin(p.pos[m], p.inv_freq[pidx], cs, sn);
+      rope_cos_sin(p.pos[m], p.rope_turn[pidx], cs, sn);
       float a = tile_out[mm][c], b = tile_out[mm][c + BN / 2];
       y[(size_t)m * jb.ldy + s_out[c]] = DT<T>::from_f(a * cs - b * sn);
       y[(size_t)m * jb.ldy + s_out[c + BN / 2]] = DT<T>::from_f(b * cs + a * sn);

@@ -10,10 +10,12 @@
 //   warp 0       TMA producer: one box [64 k x BN tokens] of activations per stage (128-byte swizzle)
 //   warp 1       allocates tensor memory; one lane issues the MMAs of a stage (4 x K=16) and commits
 //                them to the stage's "empty" barrier and, at the end of a tile, to "accumulator full"
-//   warps 4..7   epilogue: tcgen05.ld the fp32 accumulators (warp w owns TMEM lanes 32(w-4)..),
-//                transpose through shared memory, bias, rotary embedding on the retained pair
-//                (Section 3.2), one rounding, coalesced stores; two accumulator buffers of 256 columns
-//                let the epilogue of tile i overlap the MMAs of tile i+1
+//   warps 4..7   epilogue: tcgen05.ld the fp32 accumulators (warp w owns TMEM lanes 32(w-4).., a lane
+//                is a tile row and holds 32 tokens of it per pass), bias, rotary embedding on the
+//                retained pair (Section 3.2; the pair's two rows are neighbouring lanes and swap
+//                values by shuffle), one rounding, stores of 32 consecutive outputs of a token per
+//                warp; two accumulator buffers of 256 columns let the epilogue of tile i overlap
+//                the MMAs of tile i+1
 //   warps 8..23  de-quantisers (two teams of eight warps on alternate stages): thread (row, half) converts 32 codes of its weight row per k-block --
 //                nibbles to fp16 by magic number, (q-8) exact, then one fp16 FMA (q-8)*s + fp16(s*(8-z))
 //                -- and writes them into the A-operand stage in the
@@ -48,7 +50,6 @@ constexpr int A_BYTES = BMW * BK * 2;        // 16 KB
 constexpr int B_BYTES = MAXBN * BK * 2;      // 32 KB
 constexpr int PSTAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int EPI_TOK = 32;                  // tokens per epilogue pass
-constexpr int STG_BYTES = EPI_TOK * BMW * 4; // fp32 staging [token][row]
 constexpr int NWARPS = 24;
 constexpr int PTH = NWARPS * 32;
 constexpr int DQ_WARP0 = 8, DQ_WARPS = 8;      // two teams of DQ_WARPS warps: even and odd stages
@@ -69,15 +70,18 @@ struct PrefillCfg {
   int streamk;               // 1: contiguous ranges of (tile, k-block) units per block; 0: whole tiles round-robin
   int* status;
   int* counters;             // stream-K: arrivals per tile
-  float* partials;           // stream-K: two slots of [bn tokens][128 rows] fp32 per block
+  float* partials;           // stream-K: one accumulation tile [bn tokens][128 rows] fp32 per left-over tile
 };
 
 // Work of a block as a sequence of segments (tile, k-blocks [kb0, kb1)): whole tiles t = b, b + grid, ...
-// With stream-K only for as many rounds as fill every block; the k-blocks of the tiles left over are then
-// cut into equal contiguous ranges, one per block, so that the last round keeps every SM busy however few
-// tiles remain.  Blocks stay in step along k (few distinct k offsets are alive at a time, which keeps the
-// activation slices in L2).  A left-over tile is finished by the last of its blocks to arrive (fp32 partial
-// tiles in the workspace, added in block order).
+// With stream-K only for as many rounds as fill every block; the k-blocks of the tiles left over are
+// cut into equal contiguous ranges, one per block, so that every SM stays busy however few tiles remain.
+// A block runs its range of the split tiles FIRST: handing over the partial tile and finishing the split
+// tiles then overlap the main loop of the whole tiles that follow instead of standing at the kernel's end.  Blocks stay in step along k (few distinct k offsets are alive at a time, which keeps the
+// activation slices in L2).  Every block adds its fp32 partial tile to the tile's accumulation buffer in the
+// workspace (reductions done in L2); the last of the tile's blocks to arrive reads the sum
+// and finishes the tile.  With more than two blocks on a tile the order of the additions, and so the last
+// bit of the fp32 sum, depends on the order of arrival.
 // Visited k-block v of the input map -> stored k-block, first compact activation column, kept channels in it.
 // One family {start, period, keep, count}: head h keeps channels [0, keep) of its period; a leading block is
 // the case count = 1.  The activation box of a partly kept block also covers the first columns of the next
@@ -93,12 +97,12 @@ __device__ inline KBlock kblock_of(const PrefillCfg& c, int v) {
   return k;
 }
 
-struct Seg { int tile, kb0, kb1, tail_idx; };     // tail_idx: -1 whole-tile round, else index among the block's tail segments
+struct Seg { int tile, kb0, kb1; };
 struct SegIter {
   long u, ue;
-  int t, t_end, n_kb, step, tail_tile0, n_tail_seg;
+  int t, t_end, n_kb, step, tail_tile0;
   __device__ inline void init(const PrefillCfg& c, int b, int grid) {
-    n_kb = c.n_kb; step = grid; t = b; n_tail_seg = 0;
+    n_kb = c.n_kb; step = grid; t = b;
     const int base = c.streamk ? c.n_tiles / grid : (c.n_tiles + grid - 1) / grid;
     t_end = c.streamk ? base * grid : c.n_tiles;
     tail_tile0 = base * grid;
@@ -110,20 +114,21 @@ struct SegIter {
     }
   }
   __device__ inline bool next(Seg& sg) {
+    if (u < ue) {
+      const int tt = (int)(u / n_kb);
+      sg.tile = tail_tile0 + tt;
+      sg.kb0 = (int)(u - (long)tt * n_kb);
+      const long len = (n_kb - sg.kb0) < (ue - u) ? (n_kb - sg.kb0) : (ue - u);
+      sg.kb1 = sg.kb0 + (int)len;
+      u += len;
+      return true;
+    }
     if (t < t_end) {
-      sg.tile = t; sg.kb0 = 0; sg.kb1 = n_kb; sg.tail_idx = -1;
+      sg.tile = t; sg.kb0 = 0; sg.kb1 = n_kb;
       t += step;
       return true;
     }
-    if (u >= ue) return false;
-    const int tt = (int)(u / n_kb);
-    sg.tile = tail_tile0 + tt;
-    sg.kb0 = (int)(u - (long)tt * n_kb);
-    const long len = (n_kb - sg.kb0) < (ue - u) ? (n_kb - sg.kb0) : (ue - u);
-    sg.kb1 = sg.kb0 + (int)len;
-    sg.tail_idx = n_tail_seg++;
-    u += len;
-    return true;
+    return false;
   }
 };
 // block whose range [U*b/B, U*(b+1)/B) of the left-over units holds unit u (exact in fp64 for these magnitudes)
@@ -222,16 +227,17 @@ __device__ inline uint32_t pand_or(uint32_t a, uint32_t mask, uint32_t magic) {
 
 // ---------------------------------------------------------------------------------------- tile rows
 // Row r (0..127) of local weight tile `tl` of a job: stored weight row, or -1 when the row is empty.
-// Rope jobs: rows 0..63 are the first-half members of 64 rotation pairs, rows 64..127 their partners.
+// Rope jobs: rows 2i and 2i + 1 are the two members of rotation pair i (first-half member, then its partner),
+// so that the two sit in neighbouring lanes of the epilogue warp that rotates them.
 struct RowInfo { int stored; int out_col; int pair_c; int head; };
 __device__ inline RowInfo tile_row(const JobDev& jb, int tl, int r) {
   RowInfo o;
   o.stored = -1; o.out_col = -1; o.pair_c = 0; o.head = 0;
   if (jb.rope.enabled) {
     const int half = jb.rope.head_keep >> 1;
-    const int P = tl * (BMW / 2) + (r & (BMW / 2 - 1));
+    const int P = tl * (BMW / 2) + (r >> 1);
     if (P >= jb.rope.n_heads * half) return o;
-    const int h = P / half, cc = P - h * half, hi = r >> 6;
+    const int h = P / half, cc = P - h * half, hi = r & 1;
     o.stored = h * jb.rope.head_dim + hi * (jb.rope.head_dim >> 1) + cc;
     o.out_col = h * jb.rope.head_keep + hi * half + cc;
     o.pair_c = cc; o.head = h;
@@ -313,12 +319,10 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
   const uint32_t raw = (uint32_t)__cvta_generic_to_shared(psmem_raw);
   const uint32_t sbase = (raw + 1023u) & ~1023u;           // swizzled tiles need 1024-byte alignment
   unsigned char* smem = psmem_raw + (sbase - raw);
-  const uint32_t stg = sbase + PSTAGES * PSTAGE_BYTES;     // fp32 staging [32 tokens][128 rows]
-  float* stg_p = reinterpret_cast<float*>(smem + PSTAGES * PSTAGE_BYTES);
-  const uint32_t bars = stg + STG_BYTES;
+  const uint32_t bars = sbase + PSTAGES * PSTAGE_BYTES;
   const uint32_t full_a = bars, full_b = bars + 8 * PSTAGES, empty = bars + 16 * PSTAGES;
   const uint32_t acc_full = bars + 24 * PSTAGES, acc_empty = acc_full + 16, epi_bar = acc_full + 32;
-  unsigned char* misc = smem + PSTAGES * PSTAGE_BYTES + STG_BYTES + 24 * PSTAGES + 40;
+  unsigned char* misc = smem + PSTAGES * PSTAGE_BYTES + 24 * PSTAGES + 40;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
 
@@ -497,42 +501,52 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
       T* y = reinterpret_cast<T*>(jb.y);
       const T* bias = reinterpret_cast<const T*>(jb.bias);
       const bool rope = jb.rope.enabled != 0;
-      // store phase: non-rope: this thread owns tile row etid; rope: pair (etid & 63), tokens of parity etid >> 6
-      const RowInfo ri = tile_row(jb, tl, rope ? (etid & 63) : etid);
-      float b_lo = 0.f, b_hi = 0.f;
-      double invf = 0.0;
+      // this thread owns tile row etid (= its TMEM lane); a rope pair sits in lanes 2i, 2i + 1
+      const RowInfo ri = tile_row(jb, tl, etid);
+      float b_own = 0.f;
+      unsigned long long turn = 0;
       if (ri.stored >= 0) {
-        if (bias) {
-          b_lo = DT<T>::to_f(bias[ri.stored]);
-          if (rope) b_hi = DT<T>::to_f(bias[ri.stored + (jb.rope.head_dim >> 1)]);
-        }
+        if (bias) b_own = DT<T>::to_f(bias[ri.stored]);
         if (rope) {
           const int half = jb.rope.head_keep >> 1;
           int pidx = p.idx[(ri.head / jb.rope.rep) * half + ri.pair_c];
           pidx = min(max(pidx, 0), (jb.rope.head_dim >> 1) - 1);
-          invf = p.inv_freq[pidx];
+          turn = p.rope_turn[pidx];
         }
       }
-      // bias, rotary embedding, rounding and store of the 32 tokens that sit in the staging tile
-      auto store_chunk = [&](int ch) {
-        const int m0 = tt * c.bn + ch * EPI_TOK;
-        if (ri.stored < 0) return;
+      // bias, rotary embedding, rounding and store of 32 tokens of this row (all lanes of the warp call it)
+      auto store_chunk = [&](int tok0, const auto& val) {
+        constexpr int NV = (int)(sizeof(val) / sizeof(float));
+        const int m0 = tt * c.bn + tok0;
         if (rope) {
+          // the even lane of a pair rotates the even tokens, the odd lane the odd ones: one exchange hands
+          // each the other member's value of its token, and it stores both rotated members
+          const bool second = (lane & 1) != 0;
           const int half = jb.rope.head_keep >> 1;
-          for (int k = etid >> 6; k < EPI_TOK; k += 2) {
-            const int m = m0 + k;
-            if (m >= p.M) break;
-            const float lo = stg_p[k * BMW + (etid & 63)] + b_lo, hi = stg_p[k * BMW + 64 + (etid & 63)] + b_hi;
-            float cs, sn;
-            rope_cos_sin(p.pos[m], invf, cs, sn);
-            y[(size_t)m * jb.ldy + ri.out_col] = DT<T>::from_f(lo * cs - hi * sn);
-            y[(size_t)m * jb.ldy + ri.out_col + half] = DT<T>::from_f(hi * cs + lo * sn);
+          const float b_other = __shfl_xor_sync(0xffffffffu, b_own, 1);
+          const float b_lo = second ? b_other : b_own, b_hi = second ? b_own : b_other;
+          T* y_lo = y + (ri.out_col - (second ? half : 0));
+#pragma unroll
+          for (int k = 0; k < NV; k += 2) {
+            if (m0 + k >= p.M) break;
+            const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
+            const int m = m0 + k + (second ? 1 : 0);
+            const float lo = (second ? got : val[k]) + b_lo, hi = (second ? val[k + 1] : got) + b_hi;
+            if (ri.stored >= 0 && m < p.M) {
+              float cs, sn;
+              rope_cos_sin(p.pos[m], turn, cs, sn);
+              y_lo[(size_t)m * jb.ldy] = DT<T>::from_f(fmaf(-hi, sn, lo * cs));
+              y_lo[(size_t)m * jb.ldy + half] = DT<T>::from_f(fmaf(lo, sn, hi * cs));
+            }
           }
         } else {
-          for (int k = 0; k < EPI_TOK; ++k) {
+          if (ri.stored < 0) return;
+          T* yr = y + ri.out_col;
+#pragma unroll
+          for (int k = 0; k < NV; ++k) {
             const int m = m0 + k;
             if (m >= p.M) break;
-            y[(size_t)m * jb.ldy + ri.out_col] = DT<T>::from_f(stg_p[k * BMW + etid] + b_lo);
+            yr[(size_t)m * jb.ldy] = DT<T>::from_f(val[k] + b_own);
           }
         }
       };
@@ -542,65 +556,63 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
       const int row = 32 * q + lane;
       if (sg.kb0 == 0 && sg.kb1 == c.n_kb) {
         // ---- the whole contraction of this tile ran here
-        for (int ch = 0; ch < c.bn / EPI_TOK && !failed; ++ch) {
-          uint32_t v[32];
-          tmem_ld32(t_acc + (uint32_t)(ch * EPI_TOK), v);
-          tmem_ld_wait();
-          // staging[token][row]: lanes are consecutive rows
-#pragma unroll
-          for (int k = 0; k < 32; ++k) stg_p[k * BMW + row] = __uint_as_float(v[k]);
-          if (!epi_sync()) { failed = true; break; }
-          store_chunk(ch);
-          if (!epi_sync()) { failed = true; break; }       // staging is rewritten by the next pass
-        }
-        if (failed) break;
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) pmbar_arrive(acc_empty + 8 * buf);
-      } else {
-        // ---- a part of the contraction (stream-K): park the fp32 partial tile [token][row]; the last of the
-        //      tile's blocks to arrive adds the parts in block order and finishes the tile
-        const size_t slot_f = (size_t)c.bn * BMW;
-        float* mine = c.partials + (size_t)(2 * blockIdx.x + (sg.tail_idx == 0 ? 0 : 1)) * slot_f;
         for (int ch = 0; ch < c.bn / EPI_TOK; ++ch) {
           uint32_t v[32];
           tmem_ld32(t_acc + (uint32_t)(ch * EPI_TOK), v);
           tmem_ld_wait();
+          float val[32];
 #pragma unroll
-          for (int k = 0; k < 32; ++k) __stcg(mine + (size_t)(ch * EPI_TOK + k) * BMW + row, __uint_as_float(v[k]));
+          for (int k = 0; k < 32; ++k) val[k] = __uint_as_float(v[k]);
+          store_chunk(ch * EPI_TOK, val);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) pmbar_arrive(acc_empty + 8 * buf);
+      } else {
+        // ---- a part of the contraction (stream-K): the fp32 partial tile is added (reductions done in L2, a
+        //      warp covers 32 consecutive rows of a token) to the tile's accumulation buffer [token][row] in the
+        //      workspace (zero at launch); the last of the tile's blocks to arrive reads the sum and finishes the tile
+        const size_t slot_f = (size_t)c.bn * BMW;
+        const int T0 = (c.n_tiles / (int)gridDim.x) * (int)gridDim.x;          // first left-over tile
+        float* sum = c.partials + (size_t)(t - T0) * slot_f;
+        for (int ch = 0; ch < c.bn / EPI_TOK; ++ch) {
+          uint32_t v[32];
+          tmem_ld32(t_acc + (uint32_t)(ch * EPI_TOK), v);
+          tmem_ld_wait();
+          float* dst = sum + (size_t)(ch * EPI_TOK) * BMW + row;
+#pragma unroll
+          for (int k = 0; k < 32; ++k) atomicAdd(dst + (size_t)k * BMW, __uint_as_float(v[k]));
         }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) pmbar_arrive(acc_empty + 8 * buf);      // the accumulator is free for the next segment
-        __threadfence();
+        __threadfence();                                       // this thread's additions are done before ...
         if (!epi_sync()) { failed = true; break; }
-        const int T0 = (c.n_tiles / (int)gridDim.x) * (int)gridDim.x;          // first left-over tile
         const long U = (long)(c.n_tiles - T0) * c.n_kb, Bn = (long)gridDim.x < U ? (long)gridDim.x : U;
         const long tu = (long)(t - T0) * c.n_kb;                               // the tile's first left-over unit
         const int first = sk_owner(tu, Bn, U), last = sk_owner(tu + c.n_kb - 1, Bn, U);
         if (etid == 0) {
-          const int arrived = atomicAdd(&c.counters[t], 1);
+          const int arrived = atomicAdd(&c.counters[t], 1);    // ... the block's arrival shows
           *last_flag = arrived == last - first;
           __threadfence();
         }
         if (!epi_sync()) { failed = true; break; }
         if (*last_flag) {
-          for (int ch = 0; ch < c.bn / EPI_TOK && !failed; ++ch) {
-            float acc[32];
+          // 16 tokens at a time: the loads of the next 16 are in flight while these are rotated and stored
+          const float* src = sum + row;
+          float nxt[16];
 #pragma unroll
-            for (int k = 0; k < 32; ++k) acc[k] = 0.f;
-            for (int j = first; j <= last; ++j) {
-              // block j's part of this tile sits in its first slot when its left-over range starts inside the tile
-              const int sj = (U * j / Bn >= tu) ? 0 : 1;
-              const float* src = c.partials + (size_t)(2 * j + sj) * slot_f + (size_t)(ch * EPI_TOK) * BMW + row;
+          for (int k = 0; k < 16; ++k) nxt[k] = __ldcg(src + (size_t)k * BMW);
+          for (int tk = 0; tk < c.bn; tk += 16) {
+            float val[16];
 #pragma unroll
-              for (int k = 0; k < 32; ++k) acc[k] += __ldcg(src + (size_t)k * BMW);
+            for (int k = 0; k < 16; ++k) val[k] = nxt[k];
+            if (tk + 16 < c.bn) {
+              const float* nx = src + (size_t)(tk + 16) * BMW;
+#pragma unroll
+              for (int k = 0; k < 16; ++k) nxt[k] = __ldcg(nx + (size_t)k * BMW);
             }
-#pragma unroll
-            for (int k = 0; k < 32; ++k) stg_p[k * BMW + row] = acc[k];
-            if (!epi_sync()) { failed = true; break; }
-            store_chunk(ch);
-            if (!epi_sync()) { failed = true; break; }
+            store_chunk(tk, val);
           }
           if (etid == 0) c.counters[t] = 0;              // ready for the next call
         }
@@ -650,7 +662,7 @@ int host_job_tiles(const JobDev& j) {
 
 template <typename T, bool CONV, bool HEADS>
 int launch_pth(const Params& p, const PrefillCfg& c, int grid, cudaStream_t stream) {
-  const size_t smem = 1024 + (size_t)PSTAGES * PSTAGE_BYTES + STG_BYTES + 512;
+  const size_t smem = 1024 + (size_t)PSTAGES * PSTAGE_BYTES + 512;
   auto kern = prefill_kernel<T, CONV, HEADS>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return UNIQL_ERR_CUDA;
@@ -748,12 +760,14 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
     if (const char* g = getenv("UNIQL_PREFILL_GRID")) { const int v = atoi(g); if (v >= 1 && v <= sms) g2 = v; }
     const int left = c.n_tiles % g2;
     const long share = left ? (long)left * c.n_kb / g2 : 0;            // k-blocks per block in the last round
-    const size_t need = ws_used + (size_t)2 * g2 * c.bn * BMW * 4;
+    const size_t sums = (size_t)left * c.bn * BMW * 4;                 // one fp32 tile per left-over tile
+    const size_t need = ws_used + sums;
     const char* force = getenv("UNIQL_PREFILL_STREAMK");
     const bool want = force ? (force[0] == '1') : (left != 0 && left * 10 < g2 * 9 && share >= 48);
     if (want && left != 0 && cfg.ws_bytes >= need && c.n_tiles <= (1 << 16)) {
       c.streamk = 1;
       c.partials = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(cfg.workspace) + ws_used);
+      if (cudaMemsetAsync(c.partials, 0, sums, cfg.stream) != cudaSuccess) return UNIQL_ERR_CUDA;
       grid = g2;
     }
   }
