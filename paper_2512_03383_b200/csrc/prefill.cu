@@ -753,17 +753,22 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
       conv_in_kernel = true;
     }
   }
-  // stream-K for the last round when whole tiles would leave many SMs idle in it, the share of every block
-  // is long enough to amortise the hand-over of a partial tile, and the partial tiles fit in the workspace
+  // stream-K for the tiles left over when whole tiles would leave SMs idle in their last round and the partial
+  // tiles fit in the workspace.  It pays when the k-blocks a block no longer waits for outweigh the hand-over:
+  // measured on B200, a k-block takes about 0.65 us, and the hand-over (zeroing the sums, the additions, the
+  // read-back by the finishing block) about 24 us for tiles of 256 tokens when whole tiles follow and hide
+  // most of it, 28 us when every tile is split; both shrink with the tile's width.
   {
     int g2 = sms;
     if (const char* g = getenv("UNIQL_PREFILL_GRID")) { const int v = atoi(g); if (v >= 1 && v <= sms) g2 = v; }
     const int left = c.n_tiles % g2;
-    const long share = left ? (long)left * c.n_kb / g2 : 0;            // k-blocks per block in the last round
+    const double share = (double)left * c.n_kb / g2;                   // k-blocks per block of the split tiles
+    const double hand_over = c.n_tiles < g2 ? 10.0 + 18.0 * c.bn / 256.0 : 24.0 * c.bn / 256.0;
+    const bool pays = ((double)c.n_kb - share) * 0.65 > hand_over;
     const size_t sums = (size_t)left * c.bn * BMW * 4;                 // one fp32 tile per left-over tile
     const size_t need = ws_used + sums;
     const char* force = getenv("UNIQL_PREFILL_STREAMK");
-    const bool want = force ? (force[0] == '1') : (left != 0 && left * 10 < g2 * 9 && share >= 48);
+    const bool want = force ? (force[0] == '1') : (left != 0 && pays);
     if (want && left != 0 && cfg.ws_bytes >= need && c.n_tiles <= (1 << 16)) {
       c.streamk = 1;
       c.partials = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(cfg.workspace) + ws_used);
