@@ -137,10 +137,15 @@ int uniql_embed_rows(const uint8_t* packed, const void* scales, const void* zero
  * must be 256-byte aligned, at least uniql_workspace_bytes() large, and prepared once by
  * uniql_workspace_init (zeroes the counters; they return to zero after every call).
  * Calls that share a workspace must not overlap on the device. */
-/* For M > 16 (tensor-core path) the workspace only carries the status word and, for bf16 activations,
+/* For M > 16 (tensor-core path) the workspace carries the status word, for bf16 activations
  * an fp16 copy of x (M x K x 2 bytes): the tensor cores run on fp16 operands, because weights rounded
  * to bf16 would alone spend the 2e-3 error budget; bf16 magnitudes beyond 65504 saturate.  When the
- * workspace is too small for the copy the tiles are converted inside the kernel (same result, slower). */
+ * workspace is too small for the copy the tiles are converted inside the kernel (same result, slower).
+ * It also carries the fp32 sums of output tiles whose contraction is split over several thread blocks
+ * (at most 147 tiles of 128 rows x 256 tokens): the parts of such a tile are added in the order in
+ * which the blocks finish, so with more than two blocks on a tile the last bit of an fp32 sum, and
+ * rarely of the rounded output, can differ between two runs on the same input.  Without room for the
+ * sums every tile is computed by one block (reproducible, slower for shapes that fill few SMs). */
 size_t uniql_workspace_bytes(int M, int K, int N_total);
 int uniql_workspace_init(void* workspace, size_t bytes, void* stream);
 /* Every wait inside the kernels is bounded.  When one expires the kernel stops early and writes
