@@ -250,10 +250,6 @@ __device__ inline RowInfo tile_row(const JobDev& jb, int tl, int r) {
   }
   return o;
 }
-__device__ inline int job_tiles_p(const JobDev& j) {
-  if (j.rope.enabled) return (j.rope.n_heads * (j.rope.head_keep / 2) + BMW / 2 - 1) / (BMW / 2);
-  return (j.k_out + BMW - 1) / BMW;
-}
 
 // Two bf16 values of a word as two fp16 values (exact for magnitudes in fp16's normal range, which
 // holds LLM activations; larger magnitudes saturate at +-65504 instead of becoming infinite).
@@ -346,7 +342,6 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int n_wtiles = c.wtile_begin[p.n_jobs];
   auto job_of_wt = [&](int wt) { int j = 0; while (j + 1 < p.n_jobs && wt >= c.wtile_begin[j + 1]) ++j; return j; };
   bool failed = false;
 
