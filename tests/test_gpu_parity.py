@@ -400,12 +400,13 @@ def test_multi_job(B):
 
 
 # ---------------------------------------------------------------- fused Q/K projection + pruned RoPE
-def run_rope(B, rng, M, K, Hq, Hkv, D, keep, theta, dtype, idx_kind="perm", bias=False, inv_freq=None, v_keep=None):
+def run_rope(B, rng, M, K, Hq, Hkv, D, keep, theta, dtype, idx_kind="perm", bias=False, inv_freq=None, v_keep=None,
+             max_pos=8192):
     """Q and K projection with the rotary epilogue; with v_keep also the V projection in the same launch."""
     wq, wk = synth.draw_qweight(rng, Hq * D, K), synth.draw_qweight(rng, Hkv * D, K)
     dq, dk = dev_weight(wq), dev_weight(wk)
     x = synth.draw_x(rng, M, K, dtype)
-    pos = synth.draw_pos(rng, M)
+    pos = synth.draw_pos(rng, M, max_pos)
     idx = synth.draw_idx(rng, Hkv, D, keep, kind=idx_kind)
     bq = bk = None
     if bias:
@@ -474,6 +475,24 @@ def test_qk_rope_bf16_table_and_split(B):
     os.environ["UNIQL_DECODE_KP"], os.environ["UNIQL_DECODE_RP"] = "2", "7"
     for (g, ref) in run_rope(B, rng, 3, 512, 4, 4, 128, 108, 1e6, "bf16", inv_freq=invf):
         check_output(g, ref, "bf16", TIGHT, "rope bf16 table")
+
+
+@pytest.mark.parametrize("path", ["auto", "generic"])
+@pytest.mark.parametrize("M", [2, 40])
+def test_rope_long_context_and_odd_tables(B, path, M):
+    """The angle pos * inv_freq is reduced modulo one turn in 64-bit fixed point: positions up to a million
+    tokens, and caller tables whose frequencies exceed one turn per token, are zero, tiny or negative, must
+    still meet the fp64 oracle (M = 2 decode kernel, M = 40 tensor-core kernel, and the generic kernel)."""
+    B.set_path(B.PATH_AUTO if path == "auto" else B.PATH_GENERIC)
+    rng = np.random.default_rng(75 + M)
+    tol = TIGHT if M < 17 else 5e-4
+    for (g, ref) in run_rope(B, rng, M, 256, 4, 2, 128, 96, 500000.0, "f16", max_pos=1 << 20):
+        check_output(g, ref, "f16", tol, "rope, positions to 2^20, M=%d" % M)
+    invf = 1e4 ** (-np.arange(64) / 64.0)
+    invf[:6] = [10.0, 2.0 * np.pi, 7.25, 0.0, 1e-9, -0.75]
+    for (g, ref) in run_rope(B, rng, M, 256, 4, 2, 128, 128, 1e4, "f16", idx_kind="identity", inv_freq=invf, max_pos=1 << 20):
+        check_output(g, ref, "f16", tol, "rope, odd table, M=%d" % M)
+    assert B.workspace_status() == 0
 
 
 @pytest.mark.parametrize("M", [1, 16])
