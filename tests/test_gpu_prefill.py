@@ -221,6 +221,42 @@ def test_qwen_gate_down_full_size_sampled(B, M):
     assert B.workspace_status() == 0
 
 
+def test_llama_gate_few_split_tiles_full_grid(B):
+    """Llama-3-8B gate projection at M = 1024 on the full grid: 448 tiles are three rounds of 148 plus 4 tiles
+    whose k-blocks are spread over all blocks (about 37 blocks add their part to each of those tiles, ahead of
+    their whole tiles).  Sampled token rows, all output columns, so the split tiles (the last ones) are covered;
+    likewise the q|k projection with the rotary epilogue at M = 1024 (160 tiles: 12 split twelve ways)."""
+    rng = np.random.default_rng(45)
+    M, K, N = 1024, 4096, 14336
+    w = synth.random_qweight_fast(rng, N, K)
+    d = dev_weight(w)
+    x = synth.draw_x(rng, M, K, "f16")
+    xd = dev_x(x, "f16")
+    y = torch.zeros((M, N), dtype=torch.float16, device="cuda")
+    B.qlinear_ex(xd, K, d[1], d[2], d[3], None, M, K, N, None, K, None, N, y, N)
+    torch.cuda.synchronize()
+    rows = _sampled_rows(M)[::2] + [M - 300]
+    ref = oracle.qlinear(x, d[0], w.scales, w.zeros, oracle.leading(N), oracle.leading(K), rows=rows)
+    check_output(y[rows], ref, "f16", TOL["f16"], "llama gate M=1024, few split tiles")
+    del d, w
+    Hq, Hkv, D, keep, theta = 32, 8, 128, 128, 5e5
+    wq, wk = synth.random_qweight_fast(rng, Hq * D, K), synth.random_qweight_fast(rng, Hkv * D, K)
+    dq, dk = dev_weight(wq), dev_weight(wk)
+    pos = synth.draw_pos(rng, M)
+    idx = synth.draw_idx(rng, Hkv, D, keep)
+    qo = torch.zeros((M, Hq * keep), dtype=torch.float16, device="cuda")
+    ko = torch.zeros((M, Hkv * keep), dtype=torch.float16, device="cuda")
+    B.qk_rope_proj(xd, K, dq[1], dq[2], dq[3], dk[1], dk[2], dk[3], None, None, M, K, Hq, Hkv, D, keep,
+                   torch.from_numpy(idx).cuda(), torch.from_numpy(pos).cuda(), theta, None, qo, Hq * keep, ko, Hkv * keep)
+    torch.cuda.synchronize()
+    for (wt, dv, nh, g) in ((wq, dq, Hq, qo), (wk, dk, Hkv, ko)):
+        O = oracle.expand_map(oracle.qk_halfhead_map(nh, D, keep))
+        acc = oracle.qlinear(x, dv[0], wt.scales, wt.zeros, O, oracle.leading(K), rows=rows)
+        ref = oracle.rope(acc, nh, Hkv, D, keep, idx, pos[rows], theta)
+        check_output(g[rows], ref, "f16", TOL["f16"], "llama q/k rope M=1024, split tiles")
+    assert B.workspace_status() == 0
+
+
 def test_qwen_qk_rope_full_size_sampled(B):
     """Configuration 4's attention projections with the fused pruned RoPE at M = 512 (theta 1e6, 28 Q / 4 KV heads)."""
     rng = np.random.default_rng(44)
