@@ -279,7 +279,11 @@ __device__ inline uint4 dequant_word(uint32_t w, __half2 s2, __half2 cz2) {
 
 // bf16 activations -> fp16 copy in the workspace, once per call (every weight tile re-reads the tile of
 // activations, so converting there would repeat the work once per 128 weight rows).
-__global__ void x_to_f16_kernel(const __nv_bfloat16* __restrict__ x, int ldx, int M, int k_in, __half* __restrict__ o, int ldo) {
+// The same pass zeroes `zero_units` 16-byte units at `zero` (the stream-K sums of the launch that follows).
+__global__ void x_to_f16_kernel(const __nv_bfloat16* __restrict__ x, int ldx, int M, int k_in, __half* __restrict__ o, int ldo,
+                                uint4* __restrict__ zero, long zero_units) {
+  for (long i = (long)blockIdx.x * blockDim.x + threadIdx.x; i < zero_units; i += (long)gridDim.x * blockDim.x)
+    zero[i] = make_uint4(0, 0, 0, 0);
   const int units = ldo / 8;                         // 16-byte units per output row (ldo is a multiple of 8)
   const long total = (long)M * units;
   for (long i = (long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
@@ -729,18 +733,16 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   const void* xsrc = p.x;
   int ldxs = p.ldx;
   bool conv_in_kernel = false;
+  __half* x16 = nullptr;              // fp16 copy to be written by the pre-pass
+  int x16_ld = 0;
   if (p.dt == UNIQL_BF16) {
     const int ldo = (p.k_in + 7) / 8 * 8;
     const size_t off = ws_used;
     const size_t need = off + (size_t)p.M * ldo * 2;
     const char* force = getenv("UNIQL_PREFILL_CONVERT");
     if (cfg.ws_bytes >= need && !(force && force[0] == 'k')) {
-      __half* x16 = reinterpret_cast<__half*>(reinterpret_cast<unsigned char*>(cfg.workspace) + off);
-      const long units = (long)p.M * (ldo / 8);
-      long blocks = (units + 255) / 256;
-      if (blocks > 148 * 8) blocks = 148 * 8;
-      x_to_f16_kernel<<<(int)blocks, 256, 0, cfg.stream>>>(reinterpret_cast<const __nv_bfloat16*>(p.x), p.ldx, p.M, p.k_in, x16, ldo);
-      if (cudaGetLastError() != cudaSuccess) return UNIQL_ERR_CUDA;
+      x16 = reinterpret_cast<__half*>(reinterpret_cast<unsigned char*>(cfg.workspace) + off);
+      x16_ld = ldo;
       xsrc = x16;
       ldxs = ldo;
       ws_used = (need + 255) & ~(size_t)255;
@@ -767,8 +769,18 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
     if (want && left != 0 && cfg.ws_bytes >= need && c.n_tiles <= (1 << 16)) {
       c.streamk = 1;
       c.partials = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(cfg.workspace) + ws_used);
-      if (cudaMemsetAsync(c.partials, 0, sums, cfg.stream) != cudaSuccess) return UNIQL_ERR_CUDA;
       grid = g2;
+    }
+    // the sums start at zero: the conversion pre-pass clears them where there is one, else a memset node
+    if (x16) {
+      const long units = (long)p.M * (x16_ld / 8) + (c.streamk ? (long)(sums / 16) : 0);
+      long blocks = (units + 255) / 256;
+      if (blocks > 148 * 8) blocks = 148 * 8;
+      x_to_f16_kernel<<<(int)blocks, 256, 0, cfg.stream>>>(reinterpret_cast<const __nv_bfloat16*>(p.x), p.ldx, p.M, p.k_in, x16, x16_ld,
+                                                           reinterpret_cast<uint4*>(c.partials), c.streamk ? (long)(sums / 16) : 0);
+      if (cudaGetLastError() != cudaSuccess) return UNIQL_ERR_CUDA;
+    } else if (c.streamk) {
+      if (cudaMemsetAsync(c.partials, 0, sums, cfg.stream) != cudaSuccess) return UNIQL_ERR_CUDA;
     }
   }
   {
