@@ -236,7 +236,7 @@ int uniql_qkv_rope_proj(const void* x, int ldx, int dt, const uint8_t* wq, const
                         const double* inv_freq, void* q_out, int ldq, void* k_out, int ldk, void* v_out,
                         int ldv, void* workspace, size_t ws_bytes, void* stream);
 
-/* ---- SwiGLU MLP block at decode:  y = ( silu(x Wg^T) * (x Wu^T) ) Wd^T ----
+/* ---- SwiGLU MLP block:  y = ( silu(x Wg^T) * (x Wu^T) ) Wd^T ----
  * (Section 3.2, MLP paragraph: f_MLP(X) = (sigma(X W_g) . X W_u) W_d with sigma(t) = t / (1 + exp(-t)),
  * the gate of the Llama / Qwen blocks the paper compresses; Section 3.4: after sorting, pruning the
  * intermediate dimension keeps the leading k_int channels.)
@@ -249,8 +249,13 @@ int uniql_qkv_rope_proj(const void* x, int ldx, int dt, const uint8_t* wq, const
  *   activations do not fit in shared memory.  fuse = 0: two launches (gate|up with the gated product as
  *   epilogue, then down).  fuse = -1: the faster of the two on this hardware (two launches: the boundary
  *   between dependent launches costs less than the grid-wide barrier).  M in 9..16 runs as two halves.
- * Limits: fp16; 1 <= M <= 16; hidden, inter multiples of 256; k_int a multiple of 8; ldx, ldh multiples of 8;
- * x and h 16-byte aligned.  Other shapes: UNIQL_ERR_UNSUPPORTED (compose uniql_qlinear_multi calls).
+ * Limits at 1 <= M <= 16: fp16; hidden, inter multiples of 256; k_int a multiple of 8; ldx, ldh multiples
+ * of 8; x and h 16-byte aligned.  Other shapes: UNIQL_ERR_UNSUPPORTED (compose uniql_qlinear_multi calls).
+ * M > 16 (the name is historical): two launches of the tensor-core kernel.  The first takes Wg and Wu as a
+ *   pair, retained row i of each in neighbouring rows of every tile, and stores silu(g) * u as h; the second
+ *   is the down projection over the leading k_int channels of h (on the generic kernel when ldh is not a
+ *   multiple of 8 or h is not 16-byte aligned).  fp16; hidden, inter multiples of 128; any k_int in
+ *   [1, inter]; ldx a multiple of 8 and x 16-byte aligned; fuse = 1 is UNIQL_ERR_UNSUPPORTED.
  * workspace: NULL (library buffer) or uniql_mlp_workspace_bytes(M, hidden, inter) bytes, zeroed once by
  * uniql_workspace_init; after a UNIQL_ERR_TIMEOUT status it must be zeroed again before reuse. */
 size_t uniql_mlp_workspace_bytes(int M, int hidden, int inter);

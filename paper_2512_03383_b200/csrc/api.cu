@@ -337,7 +337,8 @@ extern "C" int uniql_qkv_rope_proj(const void* x, int ldx, int dt, const uint8_t
 
 extern "C" size_t uniql_mlp_workspace_bytes(int M, int hidden, int inter) {
   if (M < 1 || hidden < 1 || inter < 1) return 0;
-  return mlp_decode_workspace_bytes(M > 16 ? 16 : M, hidden, inter);
+  if (M > 16) return prefill_workspace_bytes(M, hidden > inter ? hidden : inter);     // tensor-core kernel, two launches
+  return mlp_decode_workspace_bytes(M, hidden, inter);
 }
 
 extern "C" int uniql_mlp_swiglu_decode(const void* x, int ldx, const uint8_t* wg, const void* sg, const void* zg,
@@ -360,6 +361,40 @@ extern "C" int uniql_mlp_swiglu_decode(const void* x, int ldx, const uint8_t* wg
   if (!cfg.workspace) {
     rc = lib_workspace(&cfg.workspace, &cfg.ws_bytes, cfg.stream);
     if (rc != UNIQL_OK) return rc;
+  }
+  if (M > 16) {
+    // More than 16 rows: two launches of the tensor-core kernel.  The first takes gate and up as a pair (their
+    // retained rows interleaved in every tile) and writes h = silu(x Wg^T) * (x Wu^T); the second is the plain
+    // down projection over the leading k_int channels of h.
+    if (fuse == 1) return UNIQL_ERR_UNSUPPORTED;
+    if ((hidden % kGroup) != 0 || (inter % kGroup) != 0) return UNIQL_ERR_SHAPE;
+    Params a;
+    memset(&a, 0, sizeof(a));
+    compile_map(nullptr, hidden, hidden, &a.imap);
+    a.x = x; a.ldx = ldx; a.dt = UNIQL_F16; a.M = M; a.K = hidden; a.k_in = hidden;
+    a.n_jobs = 2;
+    for (int j = 0; j < 2; ++j) {
+      JobDev& jd = a.job[j];
+      compile_map(nullptr, k_int, inter, &jd.omap);
+      jd.w = j == 0 ? wg : wu;
+      jd.scales = (const __half*)(j == 0 ? sg : su);
+      jd.zeros = (const __half*)(j == 0 ? zg : zu);
+      jd.y = h; jd.ldy = ldh; jd.N = inter; jd.k_out = k_int;
+      jd.pair = j + 1;
+    }
+    if (!prefill_supported(a)) return UNIQL_ERR_UNSUPPORTED;
+    rc = launch_prefill(a, cfg);
+    if (rc != UNIQL_OK) return rc;
+    Params b;
+    memset(&b, 0, sizeof(b));
+    compile_map(nullptr, k_int, inter, &b.imap);
+    b.x = h; b.ldx = ldh; b.dt = UNIQL_F16; b.M = M; b.K = inter; b.k_in = k_int;
+    b.n_jobs = 1;
+    JobDev& jd = b.job[0];
+    compile_map(nullptr, hidden, hidden, &jd.omap);
+    jd.w = wd; jd.scales = (const __half*)sd; jd.zeros = (const __half*)zd;
+    jd.y = y; jd.ldy = ldy; jd.N = hidden; jd.k_out = hidden;
+    return dispatch(b, cfg.workspace, cfg.ws_bytes, stream);
   }
   MlpDecode d;
   memset(&d, 0, sizeof(d));

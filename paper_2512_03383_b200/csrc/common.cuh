@@ -44,6 +44,10 @@ struct JobDev {
   int k_out;          // retained rows
   ChanMap omap;       // ignored when rope.enabled (rows follow the half-head rule)
   RopeDesc rope;
+  int pair;           // tensor-core kernel only.  1: the gate matrix of a SwiGLU pair (Section 3.2, MLP paragraph):
+                      // rows 2i, 2i+1 of a tile are retained row i of this matrix and of the NEXT job's (the up
+                      // matrix), and the epilogue stores silu(g_i) * u_i at column i of this job's output.
+                      // 2: that next job (it has no tiles of its own).
 };
 
 struct Params {

@@ -228,7 +228,8 @@ __device__ inline uint32_t pand_or(uint32_t a, uint32_t mask, uint32_t magic) {
 // ---------------------------------------------------------------------------------------- tile rows
 // Row r (0..127) of local weight tile `tl` of a job: stored weight row, or -1 when the row is empty.
 // Rope jobs: rows 2i and 2i + 1 are the two members of rotation pair i (first-half member, then its partner),
-// so that the two sit in neighbouring lanes of the epilogue warp that rotates them.
+// so that the two sit in neighbouring lanes of the epilogue warp that rotates them.  SwiGLU pairs (pair == 1)
+// likewise: rows 2i and 2i + 1 are retained row i of the gate matrix and of the up matrix.
 struct RowInfo { int stored; int out_col; int pair_c; int head; };
 __device__ inline RowInfo tile_row(const JobDev& jb, int tl, int r) {
   RowInfo o;
@@ -241,6 +242,13 @@ __device__ inline RowInfo tile_row(const JobDev& jb, int tl, int r) {
     o.stored = h * jb.rope.head_dim + hi * (jb.rope.head_dim >> 1) + cc;
     o.out_col = h * jb.rope.head_keep + hi * half + cc;
     o.pair_c = cc; o.head = h;
+  } else if (jb.pair == 1) {
+    const int j = tl * (BMW / 2) + (r >> 1);
+    if (j >= jb.k_out) return o;
+    o.stored = (jb.omap.n_fam == 1 && jb.omap.fam[0].count == 1) ? jb.omap.fam[0].start + j
+                                                                  : map_compact_to_stored(jb.omap, j);
+    o.out_col = j;
+    o.pair_c = r & 1;          // 0: row of the gate matrix, 1: row of the up matrix
   } else {
     const int j = tl * BMW + r;
     if (j >= jb.k_out) return o;
@@ -417,9 +425,10 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
       const JobDev& jb = p.job[jn];
       const RowInfo ri = tile_row(jb, wt - c.wtile_begin[jn], r);
       const bool live = ri.stored >= 0;
-      const uint8_t* wrow = jb.w + (size_t)(live ? ri.stored : 0) * (p.K / 2) + hf * 16;
-      const __half* srow = jb.scales + (size_t)(live ? ri.stored : 0) * G;
-      const __half* zrow = jb.zeros + (size_t)(live ? ri.stored : 0) * G;
+      const JobDev& src = (jb.pair == 1 && (r & 1)) ? p.job[jn + 1] : jb;      // odd rows of a SwiGLU pair: the up matrix
+      const uint8_t* wrow = src.w + (size_t)(live ? ri.stored : 0) * (p.K / 2) + hf * 16;
+      const __half* srow = src.scales + (size_t)(live ? ri.stored : 0) * G;
+      const __half* zrow = src.zeros + (size_t)(live ? ri.stored : 0) * G;
       const int kb0 = ((done & 1) == team) ? sg.kb0 : sg.kb0 + 1;
       // codes and scale / zero-point of this team's next two k-blocks are kept in registers
       uint4 q0 = make_uint4(0, 0, 0, 0), q1 = q0;
@@ -504,8 +513,10 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
       const RowInfo ri = tile_row(jb, tl, etid);
       float b_own = 0.f;
       unsigned long long turn = 0;
+      const bool swiglu = jb.pair == 1;
       if (ri.stored >= 0) {
-        if (bias) b_own = DT<T>::to_f(bias[ri.stored]);
+        const T* bias_own = (swiglu && (etid & 1)) ? reinterpret_cast<const T*>(p.job[jn + 1].bias) : bias;
+        if (bias_own) b_own = DT<T>::to_f(bias_own[ri.stored]);
         if (rope) {
           const int half = jb.rope.head_keep >> 1;
           int pidx = p.idx[(ri.head / jb.rope.rep) * half + ri.pair_c];
@@ -537,6 +548,21 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
               y_lo[(size_t)m * jb.ldy] = DT<T>::from_f(fmaf(-hi, sn, lo * cs));
               y_lo[(size_t)m * jb.ldy + half] = DT<T>::from_f(fmaf(lo, sn, hi * cs));
             }
+          }
+        } else if (swiglu) {
+          // as for a rotation pair: the even lane (gate row) takes the even tokens, the odd lane (up row) the odd
+          // ones, one exchange gives each the other matrix's sum of its token; h = silu(g) * u, one rounding
+          const bool second = (lane & 1) != 0;
+          const float b_other = __shfl_xor_sync(0xffffffffu, b_own, 1);
+          const float b_g = second ? b_other : b_own, b_u = second ? b_own : b_other;
+          T* yr = y + ri.out_col;
+#pragma unroll
+          for (int k = 0; k < NV; k += 2) {
+            if (m0 + k >= p.M) break;
+            const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
+            const int m = m0 + k + (second ? 1 : 0);
+            const float g = (second ? got : val[k]) + b_g, u = (second ? val[k + 1] : got) + b_u;
+            if (ri.stored >= 0 && m < p.M) yr[(size_t)m * jb.ldy] = DT<T>::from_f(g / (1.f + __expf(-g)) * u);
           }
         } else {
           if (ri.stored < 0) return;
@@ -655,6 +681,8 @@ int p_sm_count() {
 }
 
 int host_job_tiles(const JobDev& j) {
+  if (j.pair == 2) return 0;                                       // its rows ride in the tiles of the job before
+  if (j.pair == 1) return (j.k_out + BMW / 2 - 1) / (BMW / 2);
   if (j.rope.enabled) return (j.rope.n_heads * (j.rope.head_keep / 2) + BMW / 2 - 1) / (BMW / 2);
   return (j.k_out + BMW - 1) / BMW;
 }

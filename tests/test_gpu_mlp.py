@@ -1,5 +1,6 @@
-"""GPU parity of the SwiGLU MLP block at decode (gate|up with the gated product as epilogue, down projection;
-one launch with a grid-wide barrier, or two launches) against the CPU oracle."""
+"""GPU parity of the SwiGLU MLP block (gate|up with the gated product as epilogue, down projection; at decode
+sizes one launch with a grid-wide barrier or two launches, above 16 rows two launches of the tensor-core kernel)
+against the CPU oracle."""
 import numpy as np
 import pytest
 import torch
@@ -68,6 +69,22 @@ def test_small_mlp(B, small, M, k_int, fuse):
     check_output(y, y_ref, "f16", TOL_Y, "y M=%d k_int=%d fuse=%d" % (M, k_int, fuse))
 
 
+@pytest.mark.parametrize("M", [17, 64, 200, 300])
+@pytest.mark.parametrize("k_int", [1024, 872, 200, 8])
+def test_batches_on_the_tensor_cores(B, small, M, k_int):
+    """More than 16 rows: gate and up as a pair of matrices in one launch of the tensor-core kernel (their
+    retained rows interleaved in every tile, silu(g) * u in the epilogue), then the down projection over the
+    leading k_int channels of h.  Tile tails in rows (k_int not a multiple of 64) and in tokens, padded pitches.
+    Weights are rounded to fp16 on this path: 5e-4 for h as for the other tensor-core tests."""
+    _, qs, ds = small
+    x = synth.draw_x(np.random.default_rng(300 + M + k_int), M, 512, "f16", outlier_frac=0.01)
+    h, h_ref, y, y_ref = run_mlp(B, qs, ds, x, k_int, -1, pad=8 if M % 2 else 0)
+    check_output(h, h_ref, "f16", 5e-4, "h M=%d k_int=%d" % (M, k_int))
+    check_output(y, y_ref, "f16", TOL_Y, "y M=%d k_int=%d" % (M, k_int))
+    with pytest.raises(RuntimeError):                      # no single-launch form above 16 rows
+        run_mlp(B, qs, ds, x, k_int, 1)
+
+
 @pytest.mark.parametrize("M", [9, 11, 16])
 def test_batches_above_eight(B, small, M):
     _, qs, ds = small
@@ -113,8 +130,12 @@ def test_rejects_bad_arguments(B, small):
     for k_int in (0, 1028, 100):            # empty, beyond the stored rows, not a multiple of 8
         with pytest.raises(RuntimeError):
             run_mlp(B, qs, ds, x, k_int, -1)
-    with pytest.raises(RuntimeError):
-        run_mlp(B, qs, ds, synth.draw_x(np.random.default_rng(9), 17, 512, "f16"), 1024, -1)
+    # above 16 rows the keep count need not be a multiple of 8 (the down projection then reads an h whose row
+    # pitch the tensor-core kernel cannot take, and runs on the generic kernel)
+    x17 = synth.draw_x(np.random.default_rng(9), 17, 512, "f16")
+    h, h_ref, y, y_ref = run_mlp(B, qs, ds, x17, 100, -1)
+    check_output(h, h_ref, "f16", 5e-4, "h M=17 k_int=100")
+    check_output(y, y_ref, "f16", TOL_Y, "y M=17 k_int=100")
 
 
 # ---------------------------------------------------------------- full size: Llama-3-8B MLP, sampled outputs
