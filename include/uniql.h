@@ -259,6 +259,14 @@ int uniql_qkv_rope_proj(const void* x, int ldx, int dt, const uint8_t* wq, const
  * workspace: NULL (library buffer) or uniql_mlp_workspace_bytes(M, hidden, inter) bytes, zeroed once by
  * uniql_workspace_init; after a UNIQL_ERR_TIMEOUT status it must be zeroed again before reuse. */
 size_t uniql_mlp_workspace_bytes(int M, int hidden, int inter);
+/* The same block for either activation type and any M: dt = UNIQL_F16 with M <= 16 is
+ * uniql_mlp_swiglu_decode(fuse = -1); everything else (M > 16, and bf16 at any M) takes the two launches of
+ * the tensor-core kernel described above, x, h and y all of type dt (bf16: the tensor cores run on an fp16
+ * copy of x and of h, as for uniql_qlinear; h is rounded to bf16 once).  Same argument meaning and errors. */
+int uniql_mlp_swiglu(const void* x, int ldx, int dt, const uint8_t* wg, const void* sg, const void* zg,
+                     const uint8_t* wu, const void* su, const void* zu, const uint8_t* wd, const void* sd,
+                     const void* zd, int M, int hidden, int inter, int k_int, void* h, int ldh, void* y,
+                     int ldy, void* workspace, size_t ws_bytes, void* stream);
 int uniql_mlp_swiglu_decode(const void* x, int ldx, const uint8_t* wg, const void* sg, const void* zg,
                             const uint8_t* wu, const void* su, const void* zu, const uint8_t* wd,
                             const void* sd, const void* zd, int M, int hidden, int inter, int k_int,

@@ -188,19 +188,28 @@ def swiglu(g, u) -> np.ndarray:
     return out
 
 
+def round_bf16(a: np.ndarray) -> np.ndarray:
+    """Nearest bfloat16 (8 significand bits, ties to even) of every element, returned in fp64: the value is
+    first taken to fp32, whose upper 16 bits are the bfloat16 format, then rounded on the integer pattern."""
+    u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).astype(np.float64)
+
+
 def mlp_swiglu(x, wg, sg, zg, wu, su, zu, wd, sd, zd, k_int: int,
-               out_rows: Optional[Sequence[int]] = None) -> Tuple[np.ndarray, np.ndarray]:
+               out_rows: Optional[Sequence[int]] = None, h_dtype: str = "f16") -> Tuple[np.ndarray, np.ndarray]:
     """The pruned SwiGLU MLP block, one call of the oracle per step:
     g = x Wg[:k_int]^T, u = x Wu[:k_int]^T, h = silu(g) * u, y = fp16(h) Wd[:, :k_int]^T.
     The gated activations are a stored fp16 tensor of the model, so they are rounded to
-    fp16 (a type conversion, no arithmetic) before the down projection.
+    fp16 (a type conversion, no arithmetic) before the down projection; h_dtype = "bf16"
+    for a model whose activations are stored in bfloat16.
     Returns (h in fp64 before that rounding, y in fp64); `out_rows` samples output channels of y."""
     hidden = 2 * np.asarray(wg).shape[1]
     O, I = leading(k_int), leading(hidden)
     g = qlinear(x, wg, sg, zg, O, I)
     u = qlinear(x, wu, su, zu, O, I)
     h = swiglu(g, u)
-    h16 = h.astype(np.float16).astype(np.float64)
+    h16 = h.astype(np.float16).astype(np.float64) if h_dtype == "f16" else round_bf16(h)
     n_out = np.asarray(wd).shape[0]
     Od = leading(n_out) if out_rows is None else np.ascontiguousarray(out_rows, dtype=np.int32)
     y = qlinear(h16, wd, sd, zd, Od, leading(k_int))

@@ -69,6 +69,8 @@ _lib.uniql_mlp_workspace_bytes.restype = _sz
 _lib.uniql_mlp_workspace_bytes.argtypes = [_i, _i, _i]
 _lib.uniql_mlp_swiglu_decode.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i,
                                          _vp, _i, _vp, _i, _i, _vp, _sz, _vp]
+_lib.uniql_mlp_swiglu.argtypes = [_vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i,
+                                  _vp, _i, _vp, _i, _vp, _sz, _vp]
 _lib.uniql_qlinear_noalloc.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp]
 _lib.uniql_qlinear_ex.argtypes = [_vp, _i, _i, _vp, _vp, _vp, _vp, _i, _i, _i, ctypes.POINTER(_ChanMap), _i,
                                   ctypes.POINTER(_ChanMap), _i, _vp, _i, _vp, _sz, _vp]
@@ -78,7 +80,7 @@ _lib.uniql_qk_rope_proj.argtypes = [_vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _
                                     _vp, _vp, _d, ctypes.POINTER(_d), _vp, _i, _vp, _i, _vp, _sz, _vp]
 for _n in ("uniql_set_path", "uniql_pack_u4", "uniql_unpack_u4", "uniql_dequant", "uniql_workspace_init",
            "uniql_workspace_status", "uniql_qlinear", "uniql_qlinear_noalloc", "uniql_qlinear_ex", "uniql_qlinear_multi", "uniql_qk_rope_proj",
-           "uniql_mlp_swiglu_decode", "uniql_qkv_rope_proj", "uniql_embed_rows"):
+           "uniql_mlp_swiglu_decode", "uniql_mlp_swiglu", "uniql_qkv_rope_proj", "uniql_embed_rows"):
     getattr(_lib, _n).restype = _i
 
 
@@ -237,6 +239,17 @@ def mlp_swiglu_decode(x, ldx, wg, sg, zg, wu, su, zu, wd, sd, zd, M, hidden, int
                                         _ptr(wd), _ptr(sd), _ptr(zd), M, hidden, inter, k_int, _ptr(h), ldh,
                                         _ptr(y), ldy, int(fuse), _ptr(workspace), ws_bytes, _stream(stream)),
            "uniql_mlp_swiglu_decode")
+
+
+def mlp_swiglu(x, ldx, wg, sg, zg, wu, su, zu, wd, sd, zd, M, hidden, inter, k_int, h, ldh, y, ldy,
+               workspace=None, stream=None) -> None:
+    """uniql_mlp_swiglu: the SwiGLU MLP block for fp16 or bf16 activations and any M (x, h, y of one type)."""
+    if h.dtype != x.dtype or y.dtype != x.dtype:
+        raise TypeError("x, h and y must have the same type")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.uniql_mlp_swiglu(_ptr(x), ldx, _dt(x), _ptr(wg), _ptr(sg), _ptr(zg), _ptr(wu), _ptr(su), _ptr(zu),
+                                 _ptr(wd), _ptr(sd), _ptr(zd), M, hidden, inter, k_int, _ptr(h), ldh, _ptr(y), ldy,
+                                 _ptr(workspace), ws_bytes, _stream(stream)), "uniql_mlp_swiglu")
 
 
 def qkv_rope_proj(x, ldx, wq, sq, zq, wk, sk, zk, wv, sv, zv, bq, bk, bv, M, K, n_q_heads, n_kv_heads, head_dim,

@@ -335,10 +335,52 @@ extern "C" int uniql_qkv_rope_proj(const void* x, int ldx, int dt, const uint8_t
                        v_out, ldv, workspace, ws_bytes, stream);
 }
 
+namespace {
+
+// SwiGLU MLP on the tensor-core kernel, two launches.  The first takes gate and up as a pair (their retained
+// rows interleaved in every tile) and writes h = silu(x Wg^T) * (x Wu^T); the second is the plain down
+// projection over the leading k_int channels of h.
+int mlp_tensor_core(const void* x, int ldx, int dt, const uint8_t* wg, const void* sg, const void* zg, const uint8_t* wu,
+                    const void* su, const void* zu, const uint8_t* wd, const void* sd, const void* zd, int M, int hidden,
+                    int inter, int k_int, void* h, int ldh, void* y, int ldy, const LaunchCfg& cfg) {
+  if ((hidden % kGroup) != 0 || (inter % kGroup) != 0) return UNIQL_ERR_SHAPE;
+  Params a;
+  memset(&a, 0, sizeof(a));
+  compile_map(nullptr, hidden, hidden, &a.imap);
+  a.x = x; a.ldx = ldx; a.dt = dt; a.M = M; a.K = hidden; a.k_in = hidden;
+  a.n_jobs = 2;
+  for (int j = 0; j < 2; ++j) {
+    JobDev& jd = a.job[j];
+    compile_map(nullptr, k_int, inter, &jd.omap);
+    jd.w = j == 0 ? wg : wu;
+    jd.scales = (const __half*)(j == 0 ? sg : su);
+    jd.zeros = (const __half*)(j == 0 ? zg : zu);
+    jd.y = h; jd.ldy = ldh; jd.N = inter; jd.k_out = k_int;
+    jd.pair = j + 1;
+  }
+  if (!prefill_supported(a)) return UNIQL_ERR_UNSUPPORTED;
+  int rc = launch_prefill(a, cfg);
+  if (rc != UNIQL_OK) return rc;
+  Params b;
+  memset(&b, 0, sizeof(b));
+  compile_map(nullptr, k_int, inter, &b.imap);
+  b.x = h; b.ldx = ldh; b.dt = dt; b.M = M; b.K = inter; b.k_in = k_int;
+  b.n_jobs = 1;
+  JobDev& jd = b.job[0];
+  compile_map(nullptr, hidden, hidden, &jd.omap);
+  jd.w = wd; jd.scales = (const __half*)sd; jd.zeros = (const __half*)zd;
+  jd.y = y; jd.ldy = ldy; jd.N = hidden; jd.k_out = hidden;
+  return dispatch(b, cfg.workspace, cfg.ws_bytes, cfg.stream);
+}
+
+}  // namespace
+
 extern "C" size_t uniql_mlp_workspace_bytes(int M, int hidden, int inter) {
   if (M < 1 || hidden < 1 || inter < 1) return 0;
   if (M > 16) return prefill_workspace_bytes(M, hidden > inter ? hidden : inter);     // tensor-core kernel, two launches
-  return mlp_decode_workspace_bytes(M, hidden, inter);
+  // (16 rows or fewer in bf16 also run on the tensor-core kernel: room for its fp16 copy of the activations)
+  const size_t a = mlp_decode_workspace_bytes(M, hidden, inter), b = prefill_workspace_bytes(M, hidden > inter ? hidden : inter);
+  return a > b ? a : b;
 }
 
 extern "C" int uniql_mlp_swiglu_decode(const void* x, int ldx, const uint8_t* wg, const void* sg, const void* zg,
@@ -363,38 +405,8 @@ extern "C" int uniql_mlp_swiglu_decode(const void* x, int ldx, const uint8_t* wg
     if (rc != UNIQL_OK) return rc;
   }
   if (M > 16) {
-    // More than 16 rows: two launches of the tensor-core kernel.  The first takes gate and up as a pair (their
-    // retained rows interleaved in every tile) and writes h = silu(x Wg^T) * (x Wu^T); the second is the plain
-    // down projection over the leading k_int channels of h.
     if (fuse == 1) return UNIQL_ERR_UNSUPPORTED;
-    if ((hidden % kGroup) != 0 || (inter % kGroup) != 0) return UNIQL_ERR_SHAPE;
-    Params a;
-    memset(&a, 0, sizeof(a));
-    compile_map(nullptr, hidden, hidden, &a.imap);
-    a.x = x; a.ldx = ldx; a.dt = UNIQL_F16; a.M = M; a.K = hidden; a.k_in = hidden;
-    a.n_jobs = 2;
-    for (int j = 0; j < 2; ++j) {
-      JobDev& jd = a.job[j];
-      compile_map(nullptr, k_int, inter, &jd.omap);
-      jd.w = j == 0 ? wg : wu;
-      jd.scales = (const __half*)(j == 0 ? sg : su);
-      jd.zeros = (const __half*)(j == 0 ? zg : zu);
-      jd.y = h; jd.ldy = ldh; jd.N = inter; jd.k_out = k_int;
-      jd.pair = j + 1;
-    }
-    if (!prefill_supported(a)) return UNIQL_ERR_UNSUPPORTED;
-    rc = launch_prefill(a, cfg);
-    if (rc != UNIQL_OK) return rc;
-    Params b;
-    memset(&b, 0, sizeof(b));
-    compile_map(nullptr, k_int, inter, &b.imap);
-    b.x = h; b.ldx = ldh; b.dt = UNIQL_F16; b.M = M; b.K = inter; b.k_in = k_int;
-    b.n_jobs = 1;
-    JobDev& jd = b.job[0];
-    compile_map(nullptr, hidden, hidden, &jd.omap);
-    jd.w = wd; jd.scales = (const __half*)sd; jd.zeros = (const __half*)zd;
-    jd.y = y; jd.ldy = ldy; jd.N = hidden; jd.k_out = hidden;
-    return dispatch(b, cfg.workspace, cfg.ws_bytes, stream);
+    return mlp_tensor_core(x, ldx, UNIQL_F16, wg, sg, zg, wu, su, zu, wd, sd, zd, M, hidden, inter, k_int, h, ldh, y, ldy, cfg);
   }
   MlpDecode d;
   memset(&d, 0, sizeof(d));
@@ -422,4 +434,30 @@ extern "C" int uniql_mlp_swiglu_decode(const void* x, int ldx, const uint8_t* wg
     return rc ? rc : run(b);
   }
   return run(d);
+}
+
+extern "C" int uniql_mlp_swiglu(const void* x, int ldx, int dt, const uint8_t* wg, const void* sg, const void* zg,
+                                const uint8_t* wu, const void* su, const void* zu, const uint8_t* wd, const void* sd,
+                                const void* zd, int M, int hidden, int inter, int k_int, void* h, int ldh, void* y,
+                                int ldy, void* workspace, size_t ws_bytes, void* stream) {
+  if (dt != UNIQL_F16 && dt != UNIQL_BF16) return UNIQL_ERR_DTYPE;
+  if (dt == UNIQL_F16 && M <= 16)
+    return uniql_mlp_swiglu_decode(x, ldx, wg, sg, zg, wu, su, zu, wd, sd, zd, M, hidden, inter, k_int, h, ldh, y, ldy,
+                                   -1, workspace, ws_bytes, stream);
+  if (!x || !h || !y) return UNIQL_ERR_NULL;
+  if (M < 1 || hidden < kGroup || inter < kGroup || k_int < 1 || k_int > inter) return UNIQL_ERR_SHAPE;
+  if (ldx < hidden || ldh < k_int || ldy < hidden) return UNIQL_ERR_SHAPE;
+  int rc = check_weight(wg, sg, zg, inter);
+  if (!rc) rc = check_weight(wu, su, zu, inter);
+  if (!rc) rc = check_weight(wd, sd, zd, hidden);
+  if (rc) return rc;
+  if ((((uintptr_t)x) | ((uintptr_t)h) | ((uintptr_t)y)) & 1) return UNIQL_ERR_ALIGN;
+  if (workspace && (((uintptr_t)workspace) & 255)) return UNIQL_ERR_ALIGN;
+  if (cudaPeekAtLastError() != cudaSuccess) return UNIQL_ERR_CUDA;
+  LaunchCfg cfg{workspace, ws_bytes, (cudaStream_t)stream};
+  if (!cfg.workspace) {
+    rc = lib_workspace(&cfg.workspace, &cfg.ws_bytes, cfg.stream);
+    if (rc != UNIQL_OK) return rc;
+  }
+  return mlp_tensor_core(x, ldx, dt, wg, sg, zg, wu, su, zu, wd, sd, zd, M, hidden, inter, k_int, h, ldh, y, ldy, cfg);
 }

@@ -85,6 +85,31 @@ def test_batches_on_the_tensor_cores(B, small, M, k_int):
         run_mlp(B, qs, ds, x, k_int, 1)
 
 
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("M", [3, 16, 40, 200])
+def test_typed_entry_point(B, small, M, dtype):
+    """uniql_mlp_swiglu: fp16 at 16 rows or fewer is the decode path; everything else (bf16 at any M, M > 16)
+    the two launches of the tensor-core kernel, with x, h and y of the activation type."""
+    _, (qg, qu, qd), ((pg, wg, sg, zg), (pu, wu, su, zu), (pd, wd, sd, zd)) = small
+    k_int, hidden, inter = 872, 512, 1024
+    x = synth.draw_x(np.random.default_rng(400 + M), M, hidden, dtype, outlier_frac=0.01)
+    xd = dev_x(x, dtype)
+    h = torch.full((M, k_int + 8), -55.0, device="cuda", dtype=xd.dtype)
+    y = torch.full((M, hidden + 8), -77.0, device="cuda", dtype=xd.dtype)
+    B.mlp_swiglu(xd, xd.stride(0), wg, sg, zg, wu, su, zu, wd, sd, zd, M, hidden, inter, k_int, h, h.stride(0), y, y.stride(0))
+    torch.cuda.synchronize()
+    assert B.workspace_status() == 0
+    assert (h[:, k_int:] == -55.0).all() and (y[:, hidden:] == -77.0).all(), "wrote outside the output columns"
+    h_ref, y_ref = oracle.mlp_swiglu(x, pg, qg.scales, qg.zeros, pu, qu.scales, qu.zeros, pd, qd.scales, qd.zeros, k_int,
+                                     h_dtype=dtype)
+    check_output(h[:, :k_int], h_ref, dtype, 5e-4, "h %s M=%d" % (dtype, M))
+    # bf16: h is stored with 8 significand bits.  Where the two sides' h (5e-4 of the scale apart before the
+    # rounding) fall on different sides of a rounding boundary the stored values differ by a whole bf16 step
+    # (2^-8 of the element): per element an rms of sqrt(5e-4 * 2^-8) = 1.4e-3 of its size, which the down
+    # projection sums with random signs.  Measured 1.1e-3 of max|y|; held to the 2e-3 bar itself.
+    check_output(y[:, :hidden], y_ref, dtype, TOL_Y if dtype == "f16" else 2e-3, "y %s M=%d" % (dtype, M))
+
+
 @pytest.mark.parametrize("M", [9, 11, 16])
 def test_batches_above_eight(B, small, M):
     _, qs, ds = small

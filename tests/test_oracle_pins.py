@@ -323,3 +323,20 @@ def test_mlp_swiglu_equals_dense_definition():
     ys = oracle.mlp_swiglu(x, pg, qg.scales, qg.zeros, pu, qu.scales, qu.zeros, pd, qd.scales, qd.zeros, k_int,
                            out_rows=[5, 77, 255])[1]
     assert np.array_equal(ys, y[:, [5, 77, 255]])
+    # a bfloat16 model: the stored activations are the library's bfloat16 conversion of h
+    import torch
+    hb = torch.from_numpy(hd.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    yb = oracle.mlp_swiglu(x, pg, qg.scales, qg.zeros, pu, qu.scales, qu.zeros, pd, qd.scales, qd.zeros, k_int,
+                           h_dtype="bf16")[1]
+    assert np.allclose(yb, hb @ Wd[:, :k_int].T, rtol=1e-11, atol=1e-12) and not np.allclose(yb, y, rtol=1e-6)
+
+
+def test_round_bf16_against_the_library_conversion_and_ties():
+    import torch
+    rng = np.random.default_rng(13)
+    a = np.concatenate([rng.standard_normal(20000) * 10.0 ** rng.integers(-6, 6, 20000), [0.0, -0.0, 1.0, -1.0]])
+    want = torch.from_numpy(a.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(oracle.round_bf16(a), want)
+    # ties go to the even pattern: 1 + 2^-8 lies half-way between 1 and 1 + 2^-7; 1 + 3 * 2^-8 between 1 + 2^-7 and 1 + 2^-6
+    assert np.array_equal(oracle.round_bf16(np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20])),
+                          np.array([1.0, 1.0 + 2.0 ** -6, 1.0 + 2.0 ** -7]))
