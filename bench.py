@@ -486,6 +486,45 @@ def prefill_tables(B, torch):
             out["prefill_qwen_%s_M%d" % (name, M)] = rows
         del q
         torch.cuda.empty_cache()
+    # the whole Llama-3-8B SwiGLU block through its entry point (gate and up as a pair job with the gated product
+    # in the epilogue, then down), bf16 and fp16
+    from paper_2512_03383_b200 import synth
+    rng = np.random.default_rng(11)
+    ws = []
+    for N, K in ((INTER, HIDDEN), (INTER, HIDDEN), (HIDDEN, INTER)):
+        m = synth.random_qweight_fast(rng, N, K)
+        cd = torch.from_numpy(m.codes).cuda()
+        pw = torch.empty((N, K // 2), dtype=torch.uint8, device="cuda")
+        B.pack_u4(cd, pw)
+        del cd
+        ws.append((pw, torch.from_numpy(m.scales).cuda(), torch.from_numpy(m.zeros).cuda()))
+    (wg, sg, zg), (wu, su, zu), (wd, sd, zd) = ws
+    for M in (512, 2048):
+        for dt, dname in ((torch.bfloat16, "bf16"), (torch.float16, "f16")):
+            rows = {}
+            x = torch.randn((M, HIDDEN), device="cuda").to(dt)
+            for r in (1.0, 0.85, 0.65):
+                k = keep_count(r, INTER) // 8 * 8
+                h = torch.zeros((M, k), dtype=dt, device="cuda")
+                y = torch.zeros((M, HIDDEN), dtype=dt, device="cuda")
+
+                def one():
+                    B.mlp_swiglu(x, HIDDEN, wg, sg, zg, wu, su, zu, wd, sd, zd, M, HIDDEN, INTER, k, h, k, y, HIDDEN)
+                for _ in range(3):
+                    one()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                a.record()
+                for _ in range(10):
+                    one()
+                b.record()
+                torch.cuda.synchronize()
+                sec = a.elapsed_time(b) * 1e-3 / 10
+                flops = 2.0 * M * HIDDEN * k * 3
+                rows["%.2f" % r] = {"us": round(sec * 1e6, 1), "TFLOPs": round(flops / sec / 1e12, 1),
+                                    "frac_bf16_%s" % which: round(flops / sec / 1e12 / tf, 3),
+                                    "tokens_per_s": round(M / sec, 1)}
+            out["prefill_llama_mlp_swiglu_%s_M%d" % (dname, M)] = rows
     return out
 
 
