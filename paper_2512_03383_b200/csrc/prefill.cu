@@ -552,6 +552,8 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         } else if (swiglu) {
           // as for a rotation pair: the even lane (gate row) takes the even tokens, the odd lane (up row) the odd
           // ones, one exchange gives each the other matrix's sum of its token; h = silu(g) * u, one rounding
+          // (the approximate division: two instructions instead of ten in warps that share the issue slots
+          //  with the de-quantisers; exp(-g) beyond fp32 gives a quotient of zero, the limit of silu)
           const bool second = (lane & 1) != 0;
           const float b_other = __shfl_xor_sync(0xffffffffu, b_own, 1);
           const float b_g = second ? b_other : b_own, b_u = second ? b_own : b_other;
@@ -562,7 +564,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
             const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
             const int m = m0 + k + (second ? 1 : 0);
             const float g = (second ? got : val[k]) + b_g, u = (second ? val[k + 1] : got) + b_u;
-            if (ri.stored >= 0 && m < p.M) yr[(size_t)m * jb.ldy] = DT<T>::from_f(g / (1.f + __expf(-g)) * u);
+            if (ri.stored >= 0 && m < p.M) yr[(size_t)m * jb.ldy] = DT<T>::from_f(__fdividef(g, 1.f + __expf(-g)) * u);
           }
         } else {
           if (ri.stored < 0) return;
