@@ -568,12 +568,18 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
           }
         } else {
           if (ri.stored < 0) return;
-          T* yr = y + ri.out_col;
+          T* yr = y + ri.out_col + (size_t)m0 * jb.ldy;
+          const int left = p.M - m0;
+          if (left >= NV) {                       // a whole chunk of tokens: no test per token
 #pragma unroll
-          for (int k = 0; k < NV; ++k) {
-            const int m = m0 + k;
-            if (m >= p.M) break;
-            yr[(size_t)m * jb.ldy] = DT<T>::from_f(val[k] + b_own);
+            for (int k = 0; k < NV; ++k) { *yr = DT<T>::from_f(val[k] + b_own); yr += jb.ldy; }
+          } else {
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+              if (k >= left) break;
+              *yr = DT<T>::from_f(val[k] + b_own);
+              yr += jb.ldy;
+            }
           }
         }
       };
