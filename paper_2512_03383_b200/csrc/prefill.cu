@@ -535,18 +535,37 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
           const int half = jb.rope.head_keep >> 1;
           const float b_other = __shfl_xor_sync(0xffffffffu, b_own, 1);
           const float b_lo = second ? b_other : b_own, b_hi = second ? b_own : b_other;
-          T* y_lo = y + (ri.out_col - (second ? half : 0));
+          const bool live = ri.stored >= 0;
+          const int left = p.M - m0, odd = second ? 1 : 0;
+          T* yp = y + (live ? ri.out_col - (second ? half : 0) : 0) + (size_t)(m0 + odd) * jb.ldy;   // this lane's first token
+          const size_t step = 2 * (size_t)jb.ldy;
+          const int32_t* pp = p.pos + m0 + odd;
+          if (left >= NV) {                       // a whole chunk of tokens: no test per token
 #pragma unroll
-          for (int k = 0; k < NV; k += 2) {
-            if (m0 + k >= p.M) break;
-            const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
-            const int m = m0 + k + (second ? 1 : 0);
-            const float lo = (second ? got : val[k]) + b_lo, hi = (second ? val[k + 1] : got) + b_hi;
-            if (ri.stored >= 0 && m < p.M) {
+            for (int k = 0; k < NV; k += 2) {
+              const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
+              const float lo = (second ? got : val[k]) + b_lo, hi = (second ? val[k + 1] : got) + b_hi;
               float cs, sn;
-              rope_cos_sin(p.pos[m], turn, cs, sn);
-              y_lo[(size_t)m * jb.ldy] = DT<T>::from_f(fmaf(-hi, sn, lo * cs));
-              y_lo[(size_t)m * jb.ldy + half] = DT<T>::from_f(fmaf(lo, sn, hi * cs));
+              rope_cos_sin(pp[k], turn, cs, sn);
+              if (live) {
+                yp[0] = DT<T>::from_f(fmaf(-hi, sn, lo * cs));
+                yp[half] = DT<T>::from_f(fmaf(lo, sn, hi * cs));
+              }
+              yp += step;
+            }
+          } else {
+#pragma unroll
+            for (int k = 0; k < NV; k += 2) {
+              if (k >= left) break;
+              const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
+              const float lo = (second ? got : val[k]) + b_lo, hi = (second ? val[k + 1] : got) + b_hi;
+              if (live && k + odd < left) {
+                float cs, sn;
+                rope_cos_sin(pp[k], turn, cs, sn);
+                yp[0] = DT<T>::from_f(fmaf(-hi, sn, lo * cs));
+                yp[half] = DT<T>::from_f(fmaf(lo, sn, hi * cs));
+              }
+              yp += step;
             }
           }
         } else if (swiglu) {
@@ -557,14 +576,27 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
           const bool second = (lane & 1) != 0;
           const float b_other = __shfl_xor_sync(0xffffffffu, b_own, 1);
           const float b_g = second ? b_other : b_own, b_u = second ? b_own : b_other;
-          T* yr = y + ri.out_col;
+          const bool live = ri.stored >= 0;
+          const int left = p.M - m0, odd = second ? 1 : 0;
+          T* yp = y + (live ? ri.out_col : 0) + (size_t)(m0 + odd) * jb.ldy;          // this lane's first token
+          const size_t step = 2 * (size_t)jb.ldy;
+          if (left >= NV) {                       // a whole chunk of tokens: no test per token
 #pragma unroll
-          for (int k = 0; k < NV; k += 2) {
-            if (m0 + k >= p.M) break;
-            const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
-            const int m = m0 + k + (second ? 1 : 0);
-            const float g = (second ? got : val[k]) + b_g, u = (second ? val[k + 1] : got) + b_u;
-            if (ri.stored >= 0 && m < p.M) yr[(size_t)m * jb.ldy] = DT<T>::from_f(__fdividef(g, 1.f + __expf(-g)) * u);
+            for (int k = 0; k < NV; k += 2) {
+              const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
+              const float g = (second ? got : val[k]) + b_g, u = (second ? val[k + 1] : got) + b_u;
+              if (live) *yp = DT<T>::from_f(__fdividef(g, 1.f + __expf(-g)) * u);
+              yp += step;
+            }
+          } else {
+#pragma unroll
+            for (int k = 0; k < NV; k += 2) {
+              if (k >= left) break;
+              const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
+              const float g = (second ? got : val[k]) + b_g, u = (second ? val[k + 1] : got) + b_u;
+              if (live && k + odd < left) *yp = DT<T>::from_f(__fdividef(g, 1.f + __expf(-g)) * u);
+              yp += step;
+            }
           }
         } else {
           if (ri.stored < 0) return;
