@@ -27,7 +27,7 @@
  *    workspace, bias, positions, indices) is touched only after it has completed.  Packed weights,
  *    scales and zero-points must not be written by a decode call's immediate predecessor on the stream
  *    unless that predecessor is a plain kernel (which completes before its successor starts).
- *    UNIQL_PDL=0 in the environment turns the attribute off.
+ *    uniql_set_option("pdl", 0) (or UNIQL_PDL=0 in the environment at load time) turns the attribute off.
  *
  * Weight format (the interchange format; benchmark configuration 1)
  *  - W is stored in nn.Linear orientation, W[N][K]: N output channels (rows),
@@ -70,12 +70,17 @@ typedef enum {
 
 typedef enum { UNIQL_F16 = 0, UNIQL_BF16 = 1 } uniql_dtype;
 
-/* Kernel selection, for A/B tests.  AUTO: fp16 batches of M <= 16 take the decode kernel; everything
+/* Kernel selection, for A/B tests.  AUTO: fp16 batches of M <= 16 take the persistent decode kernel
+ * (UNIQL_PATH_DECODE); batches of M <= 4 whose input map lies on 4- but not on 8-channel boundaries (head dims 108
+ * and 84 on the input side of o_proj, 1740 of 2048 leading channels) take the streaming kernel (UNIQL_PATH_GEMV:
+ * every warp copies its own share of the codes through a private shared-memory ring) when its rules hold (one
+ * input family, every start / keep / period a multiple of 4, K a multiple of 512, x 8-byte aligned with ldx a
+ * multiple of 4, scale and zero-point arrays 8-byte aligned); everything
  * else (M > 16, bf16) the tensor-core (prefill) kernel when its alignment rules hold (activations 16-byte
  * aligned with a row pitch that is a multiple of 8, input map a leading block or one family of per-head
  * blocks on 64-channel boundaries with keep % 8 == 0), otherwise the generic kernel. */
 typedef enum { UNIQL_PATH_AUTO = 0, UNIQL_PATH_GENERIC = 1, UNIQL_PATH_DECODE = 2,
-               UNIQL_PATH_PREFILL = 3 } uniql_path;
+               UNIQL_PATH_PREFILL = 3, UNIQL_PATH_GEMV = 4 } uniql_path;
 
 /* Channel map (host struct, copied by value at call time).
  * On-device pruning keeps the leading sorted channels of D_int, of every head's
@@ -112,6 +117,20 @@ const char* uniql_status_string(int status);
 /* Force a kernel path for subsequent calls of this process (tests / A-B timing). */
 int uniql_set_path(int path);
 
+/* Tuning and test options of the process (one table of atomics, read by every launch; each option takes its
+ * initial value from the environment variable UNIQL_<NAME IN CAPITALS> when the library is loaded).
+ * UNIQL_ERR_SHAPE for an unknown name.  Options a caller may want:
+ *   "pdl"              1 / 0: programmatic stream serialization on decode launches (default 1)
+ *   "prefill_streamk"  -1 automatic, 0 never, 1 always: split the contraction of the output tiles of the last,
+ *                      partly filled round of the tensor-core kernel over several thread blocks.  0 makes the
+ *                      results of that kernel reproducible bit for bit (every tile is summed by one block).
+ *   "decode_split_batch" 1 / 0: batches of 9..16 rows as two launches over half the batch (default 1)
+ * The others steer the work split of the kernels and exist for the tests: "decode_kp", "decode_rp",
+ * "decode_stages", "decode_narrow", "decode_xstream", "decode_xcluster", "decode_i8", "prefill_grid",
+ * "prefill_convert", "gemv_first", "gemv_depth", and "wait_shift" (the poll limit of the barrier between the two
+ * phases of the one-launch MLP is divided by 2^wait_shift, so that a test can make that wait run out). */
+int uniql_set_option(const char* name, int value);
+
 /* ---- storage helpers (Section 3.4: 4-bit codes; bit-exact integer work) ----
  * codes: uint8 [N][K], one code (0..15) per byte.  packed: uint8 [N][K/2].  K even. */
 int uniql_pack_u4(const uint8_t* codes, int64_t N, int64_t K, uint8_t* packed, void* stream);
@@ -144,7 +163,9 @@ int uniql_embed_rows(const uint8_t* packed, const void* scales, const void* zero
  * It also carries the fp32 sums of output tiles whose contraction is split over several thread blocks
  * (at most 147 tiles of 128 rows x 256 tokens): the parts of such a tile are added in the order in
  * which the blocks finish, so with more than two blocks on a tile the last bit of an fp32 sum, and
- * rarely of the rounded output, can differ between two runs on the same input.  Without room for the
+ * rarely of the rounded output, can differ between two runs on the same input; uniql_set_option("prefill_streamk", 0)
+ * switches the splitting off.  Activations below fp16's range are affected too: bf16 values under 2^-24 become zero
+ * and those under 2^-14 lose significand bits in the fp16 copy.  Without room for the
  * sums every tile is computed by one block (reproducible, slower for shapes that fill few SMs). */
 size_t uniql_workspace_bytes(int M, int K, int N_total);
 int uniql_workspace_init(void* workspace, size_t bytes, void* stream);
@@ -173,7 +194,8 @@ int uniql_qlinear(const void* x, const uint8_t* packed_w, const void* scales, co
  *    UNIQL_ERR_UNSUPPORTED.  A problem whose split-K partial sums do not fit the fixed array returns
  *    UNIQL_ERR_WORKSPACE and launches nothing.  The need is 256 KB plus roughly 512 bytes per 64
  *    retained rows and batch row (more when large M * K splits the input channels over several
- *    groups of thread blocks); the Llama-3-8B MLP matrices fit for every M <= 16.
+ *    groups of thread blocks); the Llama-3-8B MLP matrices fit for every M <= 16.  Unlike uniql_qlinear, which
+ *    runs batches of 9..16 rows as two launches over half the batch, this call always is one launch.
  *  - The first call on a device looks up the array's device address (once per device, with that
  *    device current); make that first call outside any stream capture.
  *  - All calls share the one array, and it keeps what the previous call left: each call clears the
@@ -182,6 +204,14 @@ int uniql_qlinear(const void* x, const uint8_t* packed_w, const void* scales, co
 #define UNIQL_NOALLOC_SCRATCH_BYTES (8u << 20)
 int uniql_qlinear_noalloc(const void* x, const uint8_t* packed_w, const void* scales, const void* zeros,
                           int M, int K, int N, int k_in, int k_out, void* y, void* stream);
+/* Status of the uniql_qlinear_noalloc calls made so far on the current device (no counterpart in the paper
+ * either: it belongs to the entry point above).  Every wait inside the kernel is bounded; a call whose wait
+ * expired leaves UNIQL_ERR_TIMEOUT in a status word inside the fixed array and an incomplete y, while the call
+ * itself, which only enqueues work, has long returned UNIQL_OK.  uniql_workspace_status cannot see that word.
+ * This call waits for the device, copies the word to *status (host) and allocates nothing.  The next
+ * uniql_qlinear_noalloc call clears the word before it launches: read it after the calls whose outcome matters
+ * and before issuing more of them. */
+int uniql_noalloc_status(int* status);
 
 /* General form: dtype, leading dimensions, bias, channel maps (NULL map = leading k).
  * x and y must be 4-byte aligned with even ldx / ldy; every family's start and keep must be
@@ -211,7 +241,7 @@ int uniql_qlinear_multi(const void* x, int ldx, int dt, int M, int K, const uniq
  *   retained_idx: device int32 [n_kv_heads][head_keep/2], values in [0, head_dim/2)
  *   pos:          device int32 [M]
  *   inv_freq:     HOST double [head_dim/2] or NULL
- * head_dim even, <= 256; head_keep % 4 == 0; n_q_heads % n_kv_heads == 0.
+ * head_dim even, <= 256; head_keep even, 2 <= head_keep <= head_dim; n_q_heads % n_kv_heads == 0.
  * Index values are not range-checked on the host (they live on the device); the kernels
  * clamp them into [0, head_dim/2). */
 int uniql_qk_rope_proj(const void* x, int ldx, int dt, const uint8_t* wq, const void* sq,

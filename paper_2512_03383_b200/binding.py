@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libuniql.so")
 
 UNIQL_F16, UNIQL_BF16 = 0, 1
-PATH_AUTO, PATH_GENERIC, PATH_DECODE, PATH_PREFILL = 0, 1, 2, 3
+PATH_AUTO, PATH_GENERIC, PATH_DECODE, PATH_PREFILL, PATH_GEMV = 0, 1, 2, 3, 4
 MAX_FAMILIES, MAX_JOBS = 8, 4
 
 Family = Tuple[int, int, int, int]
@@ -79,9 +79,29 @@ _lib.uniql_qlinear_multi.argtypes = [_vp, _i, _i, _i, _i, ctypes.POINTER(_ChanMa
 _lib.uniql_qk_rope_proj.argtypes = [_vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i,
                                     _vp, _vp, _d, ctypes.POINTER(_d), _vp, _i, _vp, _i, _vp, _sz, _vp]
 for _n in ("uniql_set_path", "uniql_pack_u4", "uniql_unpack_u4", "uniql_dequant", "uniql_workspace_init",
-           "uniql_workspace_status", "uniql_qlinear", "uniql_qlinear_noalloc", "uniql_qlinear_ex", "uniql_qlinear_multi", "uniql_qk_rope_proj",
+           "uniql_workspace_status", "uniql_qlinear", "uniql_qlinear_noalloc", "uniql_noalloc_status", "uniql_qlinear_ex", "uniql_qlinear_multi", "uniql_qk_rope_proj",
            "uniql_mlp_swiglu_decode", "uniql_mlp_swiglu", "uniql_qkv_rope_proj", "uniql_embed_rows"):
     getattr(_lib, _n).restype = _i
+
+
+_lib.uniql_set_option.argtypes = [ctypes.c_char_p, _i]
+_lib.uniql_set_option.restype = _i
+_lib.uniql_noalloc_status.argtypes = [ctypes.POINTER(_i)]
+
+OPTION_DEFAULTS = {"pdl": 1, "decode_kp": 0, "decode_rp": 0, "decode_stages": 0, "decode_narrow": -1,
+                   "decode_xstream": -1, "decode_xcluster": -1, "decode_i8": 1, "decode_split_batch": 1,
+                   "prefill_grid": 0, "prefill_convert": 0, "prefill_streamk": -1, "gemv_first": 0, "gemv_depth": 0,
+                   "wait_shift": 0}
+
+
+def set_option(name: str, value: int) -> None:
+    """uniql_set_option: a tuning / test option of the process (see include/uniql.h)."""
+    _check(_lib.uniql_set_option(name.encode(), int(value)), "uniql_set_option")
+
+
+def reset_options() -> None:
+    for k, v in OPTION_DEFAULTS.items():
+        set_option(k, v)
 
 
 def lib() -> ctypes.CDLL:
@@ -181,6 +201,13 @@ def qlinear_noalloc(x, packed_w, scales, zeros, M, K, N, k_in, k_out, y, stream=
     array inside the library (decode sizes only, M <= 16)."""
     _check(_lib.uniql_qlinear_noalloc(_ptr(x), _ptr(packed_w), _ptr(scales), _ptr(zeros), M, K, N, k_in, k_out,
                                       _ptr(y), _stream(stream)), "uniql_qlinear_noalloc")
+
+
+def noalloc_status() -> int:
+    """Status word of the uniql_qlinear_noalloc calls made so far (synchronises the device; allocates nothing)."""
+    v = ctypes.c_int(0)
+    _check(_lib.uniql_noalloc_status(ctypes.byref(v)), "uniql_noalloc_status")
+    return int(v.value)
 
 
 def qlinear_ex(x, ldx, packed_w, scales, zeros, bias, M, K, N, in_map, k_in, out_map, k_out, y, ldy,

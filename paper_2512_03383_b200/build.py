@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libuniql.so")
-SOURCES = ["api.cu", "util_kernels.cu", "generic.cu", "decode.cu", "prefill.cu", "noalloc.cu"]
+SOURCES = ["api.cu", "util_kernels.cu", "generic.cu", "decode.cu", "gemv.cu", "prefill.cu", "noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 

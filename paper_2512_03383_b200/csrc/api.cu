@@ -5,6 +5,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "common.cuh"
@@ -13,7 +14,35 @@ using namespace uniql;
 
 namespace {
 
-int g_path = UNIQL_PATH_AUTO;
+std::atomic<int> g_path{UNIQL_PATH_AUTO};
+
+// name, environment variable read once at load, default
+struct OptDesc { const char* name; const char* env; int dflt; };
+const OptDesc kOpts[kOptCount] = {
+    {"pdl", "UNIQL_PDL", 1},                            // programmatic stream serialization on decode launches
+    {"decode_kp", "UNIQL_DECODE_KP", 0},                // groups of blocks over the input channels (0: automatic)
+    {"decode_rp", "UNIQL_DECODE_RP", 0},                // blocks per group (0: one per SM)
+    {"decode_stages", "UNIQL_DECODE_STAGES", 0},        // ring stages (0: automatic)
+    {"decode_narrow", "UNIQL_DECODE_NARROW", -1},       // narrow tiles: -1 automatic, 0 off, 1 on
+    {"decode_xstream", "UNIQL_DECODE_XSTREAM", -1},     // streamed activations: -1 automatic, 0 off, 1 on
+    {"decode_xcluster", "UNIQL_DECODE_XCLUSTER", -1},   // shared staging in clusters of two: -1 automatic, 0 off, 1 on
+    {"decode_i8", "UNIQL_DECODE_I8", 1},                // integer path (0: fp16 MMAs)
+    {"decode_split_batch", "UNIQL_DECODE_SPLIT_BATCH", 1},   // batches of 9..16 as two launches
+    {"prefill_grid", "UNIQL_PREFILL_GRID", 0},          // blocks of the tensor-core kernel (0: one per SM)
+    {"prefill_convert", "UNIQL_PREFILL_CONVERT_IN_KERNEL", 0},   // 1: bf16 tiles converted inside the kernel
+    {"prefill_streamk", "UNIQL_PREFILL_STREAMK", -1},   // split tiles: -1 automatic, 0 never (reproducible sums), 1 always
+    {"gemv_first", "UNIQL_GEMV_FIRST", 0},              // 1: the streaming kernel wherever it applies (M <= 4)
+    {"gemv_depth", "UNIQL_GEMV_DEPTH", 0},              // ring slots per warp of the streaming kernel (0: automatic)
+    {"wait_shift", "UNIQL_WAIT_SHIFT", 0},              // bounded device waits: limits divided by 2^shift (tests)
+};
+std::atomic<int> g_opt[kOptCount];
+const bool g_opt_init = [] {
+  for (int i = 0; i < kOptCount; ++i) {
+    const char* e = getenv(kOpts[i].env);
+    g_opt[i].store(e ? atoi(e) : kOpts[i].dflt);
+  }
+  return true;
+}();
 
 constexpr int kMaxDevices = 64;
 constexpr size_t kLibWorkspaceBytes = (size_t)192 << 20;
@@ -85,13 +114,27 @@ int check_weight(const uint8_t* w, const void* s, const void* z, int N) {
 int dispatch(const Params& p, void* workspace, size_t ws_bytes, void* stream) {
   if (cudaPeekAtLastError() != cudaSuccess) return UNIQL_ERR_CUDA;
   LaunchCfg cfg{workspace, ws_bytes, (cudaStream_t)stream};
-  int path = g_path;
+  int path = g_path.load();
   bool dec_ok = p.M <= 16 && decode_supported(p);
   // every batch the decode kernel does not take (more than 16 rows, bf16) goes to the tensor cores when the maps
   // allow it: at 17..63 rows the generic kernel measured 13 to 26 times slower (930 us against 71 us for the
   // Llama-3-8B gate|up at M = 17)
   bool pre_ok = prefill_supported(p);
-  if (path == UNIQL_PATH_AUTO) path = dec_ok ? UNIQL_PATH_DECODE : (pre_ok ? UNIQL_PATH_PREFILL : UNIQL_PATH_GENERIC);
+  if (path == UNIQL_PATH_AUTO) {
+    // one to four rows whose input map is on 4- but not 8-channel boundaries (head dims 108 and 84, 1740 of 2048
+    // channels): the streaming kernel; the persistent kernel would stage those activations element by element
+    const bool gemv_first = opt(kOptGemvFirst) == 1;
+    const bool gv = gemv_supported(p) && (gemv_first || !(dec_ok && decode_integer_path(p)));
+    path = gv ? UNIQL_PATH_GEMV : dec_ok ? UNIQL_PATH_DECODE : (pre_ok ? UNIQL_PATH_PREFILL : UNIQL_PATH_GENERIC);
+  }
+  if (path == UNIQL_PATH_GEMV) {
+    if (!gemv_supported(p)) return UNIQL_ERR_UNSUPPORTED;
+    if (!cfg.workspace) {
+      int rc = lib_workspace(&cfg.workspace, &cfg.ws_bytes, cfg.stream);
+      if (rc != UNIQL_OK) return rc;
+    }
+    return launch_gemv(p, cfg);
+  }
   if (path == UNIQL_PATH_DECODE) {
     if (!(p.M <= 16 && decode_supported(p))) return UNIQL_ERR_UNSUPPORTED;
     if (!cfg.workspace) {
@@ -102,7 +145,7 @@ int dispatch(const Params& p, void* workspace, size_t ws_bytes, void* stream) {
     // force the input channels to be split over two groups of blocks and every tile through a hand-over.
     // Two launches over half the batch each re-read the weights but run more than twice as fast
     // (UNIQL_DECODE_SPLIT_BATCH=0: one launch).
-    static const bool split_batch = []{ const char* e = getenv("UNIQL_DECODE_SPLIT_BATCH"); return !(e && e[0] == '0'); }();
+    const bool split_batch = opt(kOptDecodeSplitBatch) != 0;
     if (p.M > 8 && split_batch) {
       const int m1 = (p.M + 1) / 2;
       const size_t esz = 2;                               // fp16 / bf16
@@ -132,6 +175,15 @@ int dispatch(const Params& p, void* workspace, size_t ws_bytes, void* stream) {
 
 }  // namespace
 
+int uniql::opt(int id) { return g_opt[id].load(std::memory_order_relaxed); }
+
+extern "C" int uniql_set_option(const char* name, int value) {
+  if (!name) return UNIQL_ERR_NULL;
+  for (int i = 0; i < kOptCount; ++i)
+    if (strcmp(name, kOpts[i].name) == 0) { g_opt[i].store(value); return UNIQL_OK; }
+  return UNIQL_ERR_SHAPE;
+}
+
 extern "C" int uniql_version(void) { return 100; }
 
 extern "C" const char* uniql_status_string(int s) {
@@ -150,14 +202,16 @@ extern "C" const char* uniql_status_string(int s) {
 }
 
 extern "C" int uniql_set_path(int path) {
-  if (path < UNIQL_PATH_AUTO || path > UNIQL_PATH_PREFILL) return UNIQL_ERR_SHAPE;
-  g_path = path;
+  if (path < UNIQL_PATH_AUTO || path > UNIQL_PATH_GEMV) return UNIQL_ERR_SHAPE;
+  g_path.store(path);
   return UNIQL_OK;
 }
 
 extern "C" size_t uniql_workspace_bytes(int M, int K, int N_total) {
   if (M < 1 || K < 1 || N_total < 1) return 0;
-  return M <= 16 ? decode_workspace_bytes(M, K, N_total) : prefill_workspace_bytes(M, K);
+  if (M > 16) return prefill_workspace_bytes(M, K);
+  const size_t a = decode_workspace_bytes(M, K, N_total), b = M <= 4 ? gemv_workspace_bytes(M, K, N_total) : 0;
+  return a > b ? a : b;
 }
 
 extern "C" int uniql_workspace_init(void* workspace, size_t bytes, void* stream) {
@@ -380,7 +434,12 @@ extern "C" size_t uniql_mlp_workspace_bytes(int M, int hidden, int inter) {
   if (M > 16) return prefill_workspace_bytes(M, hidden > inter ? hidden : inter);     // tensor-core kernel, two launches
   // (16 rows or fewer in bf16 also run on the tensor-core kernel: room for its fp16 copy of the activations)
   const size_t a = mlp_decode_workspace_bytes(M, hidden, inter), b = prefill_workspace_bytes(M, hidden > inter ? hidden : inter);
-  return a > b ? a : b;
+  size_t c = 0;
+  if (M <= 4) {
+    const size_t c0 = gemv_workspace_bytes(M, hidden, 2 * inter), c1 = gemv_workspace_bytes(M, inter, hidden);
+    c = c0 > c1 ? c0 : c1;
+  }
+  return a > b ? (a > c ? a : c) : (b > c ? b : c);
 }
 
 extern "C" int uniql_mlp_swiglu_decode(const void* x, int ldx, const uint8_t* wg, const void* sg, const void* zg,
@@ -415,6 +474,12 @@ extern "C" int uniql_mlp_swiglu_decode(const void* x, int ldx, const uint8_t* wg
   d.sg = (const __half*)sg; d.zg = (const __half*)zg; d.su = (const __half*)su; d.zu = (const __half*)zu;
   d.sd = (const __half*)sd; d.zd = (const __half*)zd;
   d.h = h; d.ldh = ldh; d.y = y; d.ldy = ldy;
+  // one to four rows: two launches of the streaming kernel (unless one launch or the persistent kernel is asked for)
+  if (fuse != 1 && gemv_mlp_supported(d) &&
+      (g_path.load() == UNIQL_PATH_GEMV ||
+       (g_path.load() == UNIQL_PATH_AUTO && (opt(kOptGemvFirst) == 1 || !mlp_decode_supported(d)))))
+    return launch_gemv_mlp(d, cfg);
+  if (g_path.load() == UNIQL_PATH_GEMV) return UNIQL_ERR_UNSUPPORTED;
   if (!mlp_decode_supported(d)) return UNIQL_ERR_UNSUPPORTED;
   auto run = [&](const MlpDecode& q) -> int {
     // fuse = -1 takes two launches: on B200 the launch boundary (programmatic dependent launch) costs less

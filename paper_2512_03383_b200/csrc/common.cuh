@@ -139,15 +139,26 @@ __device__ inline void rope_cos_sin(int pos, unsigned long long turn, float& c, 
   s = __sinf(af);
 }
 
+// Tuning / test options of the process (uniql_set_option); every launch reads them from one table of atomics.
+enum OptId {
+  kOptPdl = 0, kOptDecodeKp, kOptDecodeRp, kOptDecodeStages, kOptDecodeNarrow, kOptDecodeXstream, kOptDecodeXcluster,
+  kOptDecodeI8, kOptDecodeSplitBatch, kOptPrefillGrid, kOptPrefillConvert, kOptPrefillStreamk, kOptGemvFirst,
+  kOptGemvDepth, kOptWaitShift, kOptCount
+};
+int opt(int id);
+
 // host launchers (one per kernel file) --------------------------------------------------
 struct LaunchCfg {
   void* workspace;
   size_t ws_bytes;
   cudaStream_t stream;
+  int clear_header;      // decode kernel: zero the arrival counters of the launch and the status block on `stream`
+                         // once the launch is certain (a workspace that may hold what an unfinished call left)
 };
 int launch_generic(const Params& p, const LaunchCfg& cfg);
 int launch_decode(const Params& p, const LaunchCfg& cfg);
 int decode_supported(const Params& p);
+int decode_integer_path(const Params& p);   // its int8 path takes the input map (8-channel boundaries)
 size_t decode_workspace_bytes(int M, int K, int N_total);
 int decode_status_offset();   // byte offset of the device status word inside a workspace
 size_t decode_workspace_header_bytes();   // counters + status word: the part that must start at zero
@@ -166,6 +177,12 @@ struct MlpDecode {
 int launch_mlp_decode(const MlpDecode& d, int fuse, const LaunchCfg& cfg);
 int mlp_decode_supported(const MlpDecode& d);
 size_t mlp_decode_workspace_bytes(int M, int hidden, int inter);
+// streaming kernel for one to four rows (csrc/gemv.cu)
+int launch_gemv(const Params& p, const LaunchCfg& cfg);
+int gemv_supported(const Params& p);
+size_t gemv_workspace_bytes(int M, int K, int N_total);
+int launch_gemv_mlp(const MlpDecode& d, const LaunchCfg& cfg);
+int gemv_mlp_supported(const MlpDecode& d);
 int launch_prefill(const Params& p, const LaunchCfg& cfg);
 int prefill_supported(const Params& p);
 size_t prefill_workspace_bytes(int M, int K);

@@ -37,6 +37,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "quant.cuh"
 
 namespace uniql {
 namespace {
@@ -136,6 +137,7 @@ struct DecodeCfg {
   float* partials;
   int* status;
   int* grid_sync;        // two ints: epilogue warps that finished phase 0, blocks that saw all of them
+  int grid_wait_limit;   // polls of the barrier between the phases before the block gives up
   // Streamed activations (rows too long to stage whole beside the ring): a small kernel quantises x once
   // into the layout the consumers read, [group][virtual row][128 bytes] plus (integer sum, 2^-e) per (group,
   // batch row), and every stage of the ring carries the eight groups of its unit beside the weights.
@@ -294,52 +296,7 @@ __device__ inline float2 lds64f(uint32_t addr) {
   asm volatile("ld.shared.v2.f32 {%0,%1}, [%2+%3];" : "=f"(v.x), "=f"(v.y) : "r"(addr), "n"(OFF));
   return v;
 }
-// exact int -> float for |v| < 2^22 without the conversion unit
-__device__ inline float small_int_to_float(int v) { return __int_as_float(v + 0x4B400000) - 12582912.f; }
 
-// Sixteen consecutive lanes hold the 128 activations of one (batch row, group), eight each (`in`): 16-bit fixed
-// point against the group's maximum, x_i = rint(x * 2^e) = 256 * hi + lo with both bytes signed.  Returns this
-// lane's bytes in the order the nibbles leave a weight word (even codes first), the group's integer sum and
-// 2^-e.  Every lane of the warp must call it (shuffles over the sixteen lanes).
-__device__ inline void quantise16(const uint4& in, uint2& hi2, uint2& lo2, int& isum_out, float& inv_scale_out) {
-  const __half2* h2 = reinterpret_cast<const __half2*>(&in);
-  float f[8];
-  float amax = 0.f;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float2 v = __half22float2(h2[i]);
-    f[2 * i] = v.x; f[2 * i + 1] = v.y;
-    amax = fmaxf(amax, fmaxf(fabsf(v.x), fabsf(v.y)));
-  }
-#pragma unroll
-  for (int o2 = 8; o2 >= 1; o2 >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o2));
-  int e = 0;
-  if (amax > 0.f && amax < 3.0e38f) {
-    e = 14 - ((int)((__float_as_uint(amax) >> 23) & 255u) - 127);
-    if (amax * __uint_as_float((uint32_t)(127 + e) << 23) > 32639.f) --e;     // keep the high byte of x_i + 128 signed
-  }
-  const float scale = __uint_as_float((uint32_t)(127 + e) << 23), inv_scale = __uint_as_float((uint32_t)(127 - e) << 23);
-  // t_k = x_i + 128 through the float adder: x * 2^e + (1.5 * 2^23 + 128) is rounded to an integer (nearest even,
-  // as rint) whose low mantissa bits are t_k.  Byte 1 of t_k is hi, byte 0 of t_k xor 0x80 is lo; the bytes are
-  // gathered with byte permutes.
-  int tk[8];
-  int isum = -8 * 128;
-#pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    tk[k] = __float_as_int(fmaf(f[k], scale, 12582912.f + 128.f)) - 0x4B400000;
-    isum += tk[k];
-  }
-  const uint32_t hi_e = __byte_perm(__byte_perm(tk[0], tk[2], 0x0051), __byte_perm(tk[4], tk[6], 0x0051), 0x5410);
-  const uint32_t hi_o = __byte_perm(__byte_perm(tk[1], tk[3], 0x0051), __byte_perm(tk[5], tk[7], 0x0051), 0x5410);
-  const uint32_t lo_e = __byte_perm(__byte_perm(tk[0], tk[2], 0x0040), __byte_perm(tk[4], tk[6], 0x0040), 0x5410) ^ 0x80808080u;
-  const uint32_t lo_o = __byte_perm(__byte_perm(tk[1], tk[3], 0x0040), __byte_perm(tk[5], tk[7], 0x0040), 0x5410) ^ 0x80808080u;
-#pragma unroll
-  for (int o2 = 8; o2 >= 1; o2 >>= 1) isum += __shfl_xor_sync(0xffffffffu, isum, o2);
-  hi2 = make_uint2(hi_e, hi_o);
-  lo2 = make_uint2(lo_e, lo_o);
-  isum_out = isum;
-  inv_scale_out = inv_scale;
-}
 
 // stored input channel (a multiple of 8) -> compact activation column, or -1 when the channel is pruned
 __device__ inline int compact_channel(const Phase& P, int ch) {
@@ -1121,7 +1078,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       if (warp == 0 && lane == 0) {
         const int target = (int)gridDim.x * EW;
         bool seen = false;
-        for (int i = 0; i < kGridWaitLimit && !seen; ++i) {
+        for (int i = 0; i < c.grid_wait_limit && !seen; ++i) {
           int v;
           asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(c.grid_sync) : "memory");
           seen = v >= target;
@@ -1138,10 +1095,12 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
             __threadfence();
           }
         } else {
+          // the wait ran out: the whole block leaves (the other roles see the flag in their own bounded waits)
           *abort_flag = 1;
+          atomicExch(c.status, UNIQL_ERR_TIMEOUT);
         }
       }
-      if (!consumer_sync()) return;
+      if (!consumer_sync() || *abort_flag) return;
     }
     if (wk.n_units == 0) continue;
     if (!xstream && !stage_x(ph, pc)) return;
@@ -1385,11 +1344,6 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
 }
 
 // -------------------------------------------------------------------------------- host side
-int env_int(const char* name, int dflt) {
-  const char* s = getenv(name);
-  return s ? atoi(s) : dflt;
-}
-
 int sm_count() {
   static int n = 0;
   if (n == 0) {
@@ -1540,7 +1494,7 @@ int launch_t(const Params& p, const DecodeCfg& c, size_t smem, cudaStream_t stre
   } else {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    lc.numAttrs = env_int("UNIQL_PDL", 1) ? 1 : 0;
+    lc.numAttrs = opt(kOptPdl) ? 1 : 0;
   }
   DecodeCfg cc = c;
   const bool as_clusters = XC && c.x_cluster != 0;
@@ -1582,8 +1536,8 @@ void visited_range(const ChanMap& m, int gran, int* first, int* total) {
 size_t plan_split(DecodeCfg* c, int M, int g_total, int gran, bool i8) {
   const int MT = M <= 8 ? 1 : 2;
   const int part_bufs = M <= 8 ? 2 : 1;
-  int n_kp = env_int("UNIQL_DECODE_KP", 0);
-  const int stages = env_int("UNIQL_DECODE_STAGES", 0);
+  int n_kp = opt(kOptDecodeKp);
+  const int stages = opt(kOptDecodeStages);
   const int want = (stages >= 2 && stages <= MAX_STAGES) ? stages : 4;
   size_t smem = 0;
   bool fits = false;
@@ -1608,7 +1562,7 @@ size_t plan_split(DecodeCfg* c, int M, int g_total, int gran, bool i8) {
   c->g_total = g_total;
   c->gran = gran;
   c->n_kp = (g_total + c->gp - 1) / c->gp;
-  int n_rp = env_int("UNIQL_DECODE_RP", 0);
+  int n_rp = opt(kOptDecodeRp);
   if (n_rp < 1) n_rp = sm_count() / c->n_kp;
   if (n_rp < 1) n_rp = 1;
   c->n_rp = n_rp;
@@ -1639,7 +1593,7 @@ size_t plan_stream(DecodeCfg* c, int M, int g_total, int gran) {
     c->g_total = g_total;
     c->gran = gran;
     c->n_kp = 1;
-    int n_rp = env_int("UNIQL_DECODE_RP", 0);
+    int n_rp = opt(kOptDecodeRp);
     if (n_rp < 1) n_rp = sm_count();
     c->n_rp = n_rp;
     if ((long long)n_rp * n_rp * ((c->gp + CG - 1) / CG) >= (1ll << 31)) return 0;
@@ -1661,6 +1615,13 @@ int decode_supported(const Params& p) {
     if (((uintptr_t)p.job[j].scales | (uintptr_t)p.job[j].zeros) & (uintptr_t)(gran * 2 - 1)) return 0;
   }
   return 1;
+}
+
+// The integer path of this kernel applies: one input family, everything on 8-channel boundaries, 128-bit loads.
+int decode_integer_path(const Params& p) {
+  return p.imap.n_fam == 1 && (p.imap.fam[0].start % 8) == 0 && (p.imap.fam[0].keep % 8) == 0 &&
+         (p.imap.fam[0].count == 1 || (p.imap.fam[0].period % 8) == 0) && (p.ldx % 8) == 0 &&
+         ((((uintptr_t)p.x) & 15) == 0);
 }
 
 size_t decode_workspace_bytes(int M, int K, int N_total) {
@@ -1689,13 +1650,11 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   visited_range(p.imap, gran, &v_first, &g_total);
   const int MT = p.M <= 8 ? 1 : 2;
   // 128-bit staging: one leading family, everything 8-element aligned
-  c.x_vec = p.imap.n_fam == 1 && (p.imap.fam[0].start % 8) == 0 && (p.imap.fam[0].keep % 8) == 0 &&
-            (p.imap.fam[0].count == 1 || (p.imap.fam[0].period % 8) == 0) && (p.ldx % 8) == 0 &&
-            ((((uintptr_t)p.x) & 15) == 0);
+  c.x_vec = decode_integer_path(p);
   if (count_tile_fams(p) > kMaxTF) return UNIQL_ERR_UNSUPPORTED;
 
   // integer path: fp16 activations staged with 128-bit loads (a leading input block); UNIQL_DECODE_I8=0: fp16 MMAs
-  const bool i8 = c.x_vec && env_int("UNIQL_DECODE_I8", 1) != 0;
+  const bool i8 = c.x_vec && opt(kOptDecodeI8) != 0;
   // Streamed activations for rows too long to stage whole beside the ring (which would otherwise split the input
   // channels over several groups of blocks and hand every tile over); UNIQL_DECODE_XSTREAM=0/1 forces.  Where the
   // staged copy fits the quantising kernel in front costs more than the staging it saves (measured 3.5 us), and
@@ -1704,7 +1663,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   size_t smem = 0;
   c.stage_bytes = STAGE_BYTES;
   {
-    const int force = env_int("UNIQL_DECODE_XSTREAM", -1);
+    const int force = opt(kOptDecodeXstream);
     if (i8 && p.M <= 8 && force != 0) {
       DecodeCfg t = c;
       const size_t s0 = plan_split(&t, p.M, g_total, gran, true);
@@ -1739,7 +1698,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
       //  the smaller boxes of the narrow tiles cost more than a better balance of many tiles gains)
       narrow = c.n_kp == 1 && t64 < c.n_rp &&
                schedule_cost(t32, (Gk0 + 2 * CG - 1) / (2 * CG), c.n_rp) < schedule_cost(t64, (Gk0 + CG - 1) / CG, c.n_rp);
-      const int force = env_int("UNIQL_DECODE_NARROW", -1);
+      const int force = opt(kOptDecodeNarrow);
       if (force == 0) narrow = false;
       if (force == 1) narrow = true;
     }
@@ -1798,7 +1757,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
     // small launches), so it is used where the staging is long: seven or eight rows and eight or more 16-byte units
     // per thread (smaller batches would alternate between two kernel functions within a layer, which costs more
     // than the staging saved).
-    const int force_xc = env_int("UNIQL_DECODE_XCLUSTER", -1);
+    const int force_xc = opt(kOptDecodeXcluster);
     c.x_cluster = i8 && !c.x_stream && c.n_kp == 1 && (c.n_rp % 2) == 0 && p.M <= 8 && all_stage_everything &&
                   pairs_alike && force_xc != 0 && (force_xc == 1 || (p.M >= 7 && g_total * p.M >= 256));
   }
@@ -1818,6 +1777,15 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   c.status = reinterpret_cast<int*>(ws + kStatusOff);
   c.partials = reinterpret_cast<float*>(ws + kWsHeader);
   c.grid_sync = reinterpret_cast<int*>(ws + kGridSyncOff);
+  if (cfg.clear_header) {
+    // every check has passed: only now is anything put on the stream.  What must start at zero: the counters of
+    // this launch's tiles, the status word and the two counters of the barrier between phases.
+    if (cudaMemsetAsync(ws, 0, (size_t)tiles * EW * sizeof(int), cfg.stream) != cudaSuccess ||
+        cudaMemsetAsync(ws + kStatusOff, 0, 256, cfg.stream) != cudaSuccess) {
+      cudaGetLastError();
+      return UNIQL_ERR_CUDA;
+    }
+  }
   if (c.x_stream) {
     EncodeTiledFn enc = encoder();
     if (!enc) return UNIQL_ERR_CUDA;
@@ -1840,7 +1808,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
-    lc.numAttrs = env_int("UNIQL_PDL", 1) ? 1 : 0;
+    lc.numAttrs = opt(kOptPdl) ? 1 : 0;
     if (cudaLaunchKernelEx(&lc, xquant_kernel, c.ph[0], p.M, c.vr, g_total, ws + xq_off,
                            reinterpret_cast<float2*>(ws + xg_off)) != cudaSuccess) {
       cudaGetLastError();
@@ -1933,7 +1901,7 @@ int launch_mlp_phases(const MlpDecode& d, int first, int count, const LaunchCfg&
     narrow = c.n_kp == 1 && (d.hidden + RB - 1) / RB < c.n_rp &&
              schedule_cost((d.hidden + RB / 2 - 1) / (RB / 2), (Gk0 + 2 * CG - 1) / (2 * CG), c.n_rp) <
                  schedule_cost((d.hidden + RB - 1) / RB, (Gk0 + CG - 1) / CG, c.n_rp);
-    const int force = env_int("UNIQL_DECODE_NARROW", -1);
+    const int force = opt(kOptDecodeNarrow);
     if (force == 0) narrow = false;
     if (force == 1) narrow = true;
   }
@@ -1984,6 +1952,10 @@ int launch_mlp_phases(const MlpDecode& d, int first, int count, const LaunchCfg&
   c.status = reinterpret_cast<int*>(ws + kStatusOff);
   c.partials = reinterpret_cast<float*>(ws + kWsHeader);
   c.grid_sync = reinterpret_cast<int*>(ws + kGridSyncOff);
+  {
+    const int shift = opt(kOptWaitShift);
+    c.grid_wait_limit = shift > 0 ? (shift >= 21 ? 1 : kGridWaitLimit >> shift) : kGridWaitLimit;
+  }
   if (count > 1) {
     if (d.M <= 4) return launch_t<1, false, 1, 2>(p, c, smem, cfg.stream);
     return launch_t<1, false, 2, 2>(p, c, smem, cfg.stream);
@@ -1992,7 +1964,7 @@ int launch_mlp_phases(const MlpDecode& d, int first, int count, const LaunchCfg&
   if (d.M <= 8) {
     // shared staging under the rule of the plain launches (every block of the gate|up launch has whole tiles)
     const Phase& P = c.ph[0];
-    const int force_xc = env_int("UNIQL_DECODE_XCLUSTER", -1);
+    const int force_xc = opt(kOptDecodeXcluster);
     c.x_cluster = c.n_kp == 1 && (c.n_rp % 2) == 0 && P.base > 0 && force_xc != 0 && d.M >= 7 && P.g_total * d.M >= 256;
     int rc = launch_t<1, false, 2, 1, true, true>(p, c, smem, cfg.stream);
     if (rc == UNIQL_ERR_UNSUPPORTED && c.x_cluster) {

@@ -68,10 +68,25 @@ extern "C" int uniql_qlinear_noalloc(const void* x, const uint8_t* packed_w, con
   void* scratch = nullptr;
   int rc = scratch_address(&scratch);
   if (rc != UNIQL_OK) return rc;
-  // The array keeps whatever the previous call left.  Counters and the status word must start at zero
-  // (they do return to zero after a call that ran to its end, but not after one that gave up).
-  if (cudaMemsetAsync(scratch, 0, decode_workspace_header_bytes(), (cudaStream_t)stream) != cudaSuccess)
-    return UNIQL_ERR_CUDA;
-  LaunchCfg cfg{scratch, (size_t)UNIQL_NOALLOC_SCRATCH_BYTES, (cudaStream_t)stream};
+  // The array keeps whatever the previous call left.  Counters and the status word must start at zero (they do
+  // return to zero after a call that ran to its end, but not after one that gave up): the launcher clears them
+  // on `stream`, after its own checks, so a call that is turned down puts nothing on the stream.
+  LaunchCfg cfg{scratch, (size_t)UNIQL_NOALLOC_SCRATCH_BYTES, (cudaStream_t)stream, 1};
   return launch_decode(p, cfg);      // UNIQL_ERR_WORKSPACE when the problem needs more than the fixed array
+}
+
+// The status word of the calls above lives inside the fixed array, where uniql_workspace_status cannot see it.
+extern "C" int uniql_noalloc_status(int* status) {
+  if (!status) return UNIQL_ERR_NULL;
+  void* scratch = nullptr;
+  const int rc = scratch_address(&scratch);
+  if (rc != UNIQL_OK) return rc;
+  int v = 0;
+  // (a blocking copy on the legacy stream: it waits for the work in flight and allocates nothing)
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(&v, reinterpret_cast<unsigned char*>(scratch) + decode_status_offset(), sizeof(int),
+                 cudaMemcpyDeviceToHost) != cudaSuccess)
+    return UNIQL_ERR_CUDA;
+  *status = v;
+  return UNIQL_OK;
 }

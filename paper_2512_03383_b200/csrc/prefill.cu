@@ -766,7 +766,8 @@ int prefill_supported(const Params& p) {
 int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   PEncodeFn enc = p_encoder();
   if (!enc) return UNIQL_ERR_CUDA;
-  if (!cfg.workspace) return UNIQL_ERR_WORKSPACE;
+  if (!cfg.workspace || cfg.ws_bytes < decode_workspace_header_bytes()) return UNIQL_ERR_WORKSPACE;   // status word
+  const int env_grid = opt(kOptPrefillGrid), env_streamk = opt(kOptPrefillStreamk);
   PrefillCfg c;
   memset(&c, 0, sizeof(c));
   c.bn = p.M <= 64 ? 64 : (p.M <= 128 ? 128 : 256);
@@ -790,10 +791,7 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   c.status = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(cfg.workspace) + decode_status_offset());
   const int sms = p_sm_count();
   int grid = c.n_tiles < sms ? c.n_tiles : sms;
-  if (const char* g = getenv("UNIQL_PREFILL_GRID")) {          // tests: odd splits on small problems
-    const int v = atoi(g);
-    if (v >= 1 && v <= sms) grid = v;
-  }
+  if (env_grid >= 1 && env_grid <= sms) grid = env_grid;          // tests: odd splits on small problems
   // workspace: [header: counters, status][fp16 copy of bf16 activations][stream-K partial tiles]
   size_t ws_used = (decode_workspace_header_bytes() + 255) & ~(size_t)255;
   c.counters = reinterpret_cast<int*>(cfg.workspace);
@@ -807,8 +805,7 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
     const int ldo = (p.k_in + 7) / 8 * 8;
     const size_t off = ws_used;
     const size_t need = off + (size_t)p.M * ldo * 2;
-    const char* force = getenv("UNIQL_PREFILL_CONVERT");
-    if (cfg.ws_bytes >= need && !(force && force[0] == 'k')) {
+    if (cfg.ws_bytes >= need && opt(kOptPrefillConvert) != 1) {
       x16 = reinterpret_cast<__half*>(reinterpret_cast<unsigned char*>(cfg.workspace) + off);
       x16_ld = ldo;
       xsrc = x16;
@@ -825,15 +822,14 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   // most of it, 28 us when every tile is split; both shrink with the tile's width.
   {
     int g2 = sms;
-    if (const char* g = getenv("UNIQL_PREFILL_GRID")) { const int v = atoi(g); if (v >= 1 && v <= sms) g2 = v; }
+    if (env_grid >= 1 && env_grid <= sms) g2 = env_grid;
     const int left = c.n_tiles % g2;
     const double share = (double)left * c.n_kb / g2;                   // k-blocks per block of the split tiles
     const double hand_over = c.n_tiles < g2 ? 10.0 + 18.0 * c.bn / 256.0 : 24.0 * c.bn / 256.0;
     const bool pays = ((double)c.n_kb - share) * 0.65 > hand_over;
     const size_t sums = (size_t)left * c.bn * BMW * 4;                 // one fp32 tile per left-over tile
     const size_t need = ws_used + sums;
-    const char* force = getenv("UNIQL_PREFILL_STREAMK");
-    const bool want = force ? (force[0] == '1') : (left != 0 && pays);
+    const bool want = env_streamk >= 0 ? (env_streamk == 1) : (left != 0 && pays);
     if (want && left != 0 && cfg.ws_bytes >= need && c.n_tiles <= (1 << 16)) {
       c.streamk = 1;
       c.partials = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(cfg.workspace) + ws_used);
@@ -843,7 +839,7 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
     if (x16) {
       const long units = (long)p.M * (x16_ld / 8) + (c.streamk ? (long)(sums / 16) : 0);
       long blocks = (units + 255) / 256;
-      if (blocks > 148 * 8) blocks = 148 * 8;
+      if (blocks > (long)sms * 8) blocks = (long)sms * 8;
       x_to_f16_kernel<<<(int)blocks, 256, 0, cfg.stream>>>(reinterpret_cast<const __nv_bfloat16*>(p.x), p.ldx, p.M, p.k_in, x16, x16_ld,
                                                            reinterpret_cast<uint4*>(c.partials), c.streamk ? (long)(sums / 16) : 0);
       if (cudaGetLastError() != cudaSuccess) return UNIQL_ERR_CUDA;
@@ -871,7 +867,7 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
 size_t prefill_workspace_bytes(int M, int K) {
   // status word and counters (shared header) + room for the fp16 copy of bf16 activations + stream-K partial tiles
   return ((decode_workspace_header_bytes() + 255) & ~(size_t)255) + (size_t)M * ((K + 7) / 8 * 8) * 2 + 256 +
-         (size_t)2 * 148 * MAXBN * BMW * 4;
+         (size_t)2 * p_sm_count() * MAXBN * BMW * 4;
 }
 
 }  // namespace uniql

@@ -76,9 +76,15 @@ __global__ void embed_kernel(const uint8_t* __restrict__ packed, const __half* _
 }
 
 inline int grid_for(int64_t n, int threads) {
+  static const int sms = [] {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+      return v;
+    return 148;
+  }();
   int64_t b = (n + threads - 1) / threads;
   if (b < 1) b = 1;
-  if (b > 148 * 16) b = 148 * 16;
+  if (b > (int64_t)sms * 16) b = (int64_t)sms * 16;
   return (int)b;
 }
 

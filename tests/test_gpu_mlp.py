@@ -152,9 +152,11 @@ def test_fused_equals_two_launches_bitwise(B, small):
 def test_rejects_bad_arguments(B, small):
     _, qs, ds = small
     x = synth.draw_x(np.random.default_rng(9), 1, 512, "f16")
-    for k_int in (0, 1028, 100):            # empty, beyond the stored rows, not a multiple of 8
+    for k_int in (0, 1028, 102):            # empty, beyond the stored rows, not a multiple of 4
         with pytest.raises(RuntimeError):
             run_mlp(B, qs, ds, x, k_int, -1)
+    with pytest.raises(RuntimeError):       # one launch: the persistent kernel wants a multiple of 8
+        run_mlp(B, qs, ds, x, 100, 1)
     # above 16 rows the keep count need not be a multiple of 8 (the down projection then reads an h whose row
     # pitch the tensor-core kernel cannot take, and runs on the generic kernel)
     x17 = synth.draw_x(np.random.default_rng(9), 17, 512, "f16")

@@ -31,8 +31,7 @@ def B():
 def _reset_path(B):
     yield
     B.set_path(B.PATH_AUTO)
-    for k in ("UNIQL_DECODE_KP", "UNIQL_DECODE_RP", "UNIQL_DECODE_NARROW", "UNIQL_DECODE_XSTREAM", "UNIQL_DECODE_XCLUSTER"):
-        os.environ.pop(k, None)
+    B.reset_options()
 
 
 def run_ex(B, qw, dw, x32, dtype, in_map, k_in, out_map, k_out, bias=None, ldx_pad=0, ldy_pad=0, workspace=None):
@@ -129,7 +128,7 @@ def test_m_sweep(B, M, dtype):
 @pytest.mark.parametrize("M", [1, 5, 16])
 def test_decode_split_configs(B, kp, rp, M):
     """Every way of cutting the work (k-parts x blocks per k-part) gives the same answer."""
-    os.environ["UNIQL_DECODE_KP"], os.environ["UNIQL_DECODE_RP"] = str(kp), str(rp)
+    B.set_option("decode_kp", kp); B.set_option("decode_rp", rp)
     B.set_path(B.PATH_DECODE)
     rng = np.random.default_rng(7)
     qw = synth.draw_qweight(rng, 144, 1536)
@@ -150,9 +149,9 @@ def test_tile_shapes(B, narrow, kp, rp, M):
     """Wide tiles (64 rows x 8 groups) and narrow tiles (32 rows x 16 groups) give the same answer for every
     split: ragged row counts, group counts that leave the second half of a narrow chunk empty or short,
     several families, bias, and both activation paths (128-bit staging and the generic one)."""
-    os.environ["UNIQL_DECODE_NARROW"] = str(narrow)
+    B.set_option("decode_narrow", narrow)
     if kp:
-        os.environ["UNIQL_DECODE_KP"], os.environ["UNIQL_DECODE_RP"] = str(kp), str(rp)
+        B.set_option("decode_kp", kp); B.set_option("decode_rp", rp)
     B.set_path(B.PATH_DECODE)
     rng = np.random.default_rng(70 + M)
     for (N, K, k_in, k_out) in [(200, 2304, 2304, 200), (200, 2304, 1100, 77), (96, 256, 256, 96), (70, 3328, 3072, 33)]:
@@ -179,9 +178,9 @@ def test_streamed_activations(B, stream, rp, M):
     """Activations quantised once by a small kernel and carried through the ring beside the weights (the default
     where a staged copy of x does not fit beside the ring) against the block-wide staging: the same results for plain, ragged and per-head shapes,
     several matrices in one launch and the rotary epilogue."""
-    os.environ["UNIQL_DECODE_XSTREAM"] = str(stream)
+    B.set_option("decode_xstream", stream)
     if rp:
-        os.environ["UNIQL_DECODE_RP"] = str(rp)
+        B.set_option("decode_rp", rp)
     B.set_path(B.PATH_DECODE)
     rng = np.random.default_rng(80 + M)
     for (N, K, k_in, k_out) in [(200, 2304, 2304, 200), (200, 2304, 1096, 77), (96, 256, 256, 96), (70, 3328, 3072, 33)]:
@@ -231,9 +230,9 @@ def test_tiny_and_ragged_shapes(B, M, dtype):
 def test_shared_staging_in_clusters(B, xc, rp, M):
     """Blocks launched as clusters of two, each quantising half of the activations into both blocks' shared memory
     (used by default where the staging is long), against every block staging everything."""
-    os.environ["UNIQL_DECODE_XCLUSTER"] = str(xc)
+    B.set_option("decode_xcluster", xc)
     if rp:
-        os.environ["UNIQL_DECODE_RP"] = str(rp)
+        B.set_option("decode_rp", rp)
     B.set_path(B.PATH_DECODE)
     rng = np.random.default_rng(500 + M)
     for (N, K, k_in, k_out) in [(300, 1024, 1024, 300), (200, 2304, 1096, 77), (96, 256, 256, 96), (640, 3328, 3072, 600)]:
@@ -257,7 +256,7 @@ def test_shared_staging_in_clusters(B, xc, rp, M):
 
 
 def test_caller_workspace(B):
-    os.environ["UNIQL_DECODE_KP"] = "2"
+    B.set_option("decode_kp", 2)
     rng = np.random.default_rng(8)
     qw = synth.draw_qweight(rng, 96, 1024)
     dw = dev_weight(qw)
@@ -472,7 +471,7 @@ def test_qkv_one_launch(B, path, M, keep, v_keep):
 def test_qk_rope_bf16_table_and_split(B):
     rng = np.random.default_rng(71)
     invf = (1e6 ** (-np.arange(64) / 64.0)) * 0.5          # a caller table (scaled-RoPE variants)
-    os.environ["UNIQL_DECODE_KP"], os.environ["UNIQL_DECODE_RP"] = "2", "7"
+    B.set_option("decode_kp", 2); B.set_option("decode_rp", 7)
     for (g, ref) in run_rope(B, rng, 3, 512, 4, 4, 128, 108, 1e6, "bf16", inv_freq=invf):
         check_output(g, ref, "bf16", TIGHT, "rope bf16 table")
 

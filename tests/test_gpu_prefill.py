@@ -28,6 +28,7 @@ def B():
 def _reset_path(B):
     yield
     B.set_path(B.PATH_AUTO)
+    B.reset_options()
 
 
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
@@ -98,7 +99,7 @@ def test_prefill_bf16_converted_in_kernel(B, monkeypatch):
     dw = dev_weight(qw)
     x = synth.draw_x(rng, 300, 652, "bf16")
     y1, ref = run_ex(B, qw, dw, x, "bf16", None, 652, None, 256, ldx_pad=4)
-    monkeypatch.setenv("UNIQL_PREFILL_CONVERT", "kernel")
+    B.set_option("prefill_convert", 1)
     y2, _ = run_ex(B, qw, dw, x, "bf16", None, 652, None, 256, ldx_pad=4)
     check_output(y2, ref, "bf16", TOL["bf16"], "bf16 converted in kernel")
     assert torch.equal(y1, y2)
@@ -113,8 +114,8 @@ def test_prefill_per_head_input_maps(B, monkeypatch, M, dtype, grid):
     inside its first (40, 8): a partly kept block reads the next head's activations against zero weights."""
     B.set_path(B.PATH_PREFILL)
     if grid:
-        monkeypatch.setenv("UNIQL_PREFILL_STREAMK", "1")
-        monkeypatch.setenv("UNIQL_PREFILL_GRID", str(grid))
+        B.set_option("prefill_streamk", 1)
+        B.set_option("prefill_grid", grid)
     rng = np.random.default_rng(950 + M)
     qw = synth.draw_qweight(rng, 200, 1024)
     dw = dev_weight(qw)
@@ -146,8 +147,8 @@ def test_prefill_stream_k(B, monkeypatch, grid, dtype):
     most two blocks repeats bit for bit (one addition, which commutes); with more blocks on a tile the order of
     the additions follows the order of arrival, so only the tolerance holds there."""
     B.set_path(B.PATH_PREFILL)
-    monkeypatch.setenv("UNIQL_PREFILL_STREAMK", "1")
-    monkeypatch.setenv("UNIQL_PREFILL_GRID", str(grid))
+    B.set_option("prefill_streamk", 1)
+    B.set_option("prefill_grid", grid)
     rng = np.random.default_rng(900 + grid)
     qw = synth.draw_qweight(rng, 300, 1024)
     dw = dev_weight(qw)
