@@ -111,22 +111,76 @@ int check_weight(const uint8_t* w, const void* s, const void* z, int N) {
   return UNIQL_OK;
 }
 
-int dispatch(const Params& p, void* workspace, size_t ws_bytes, void* stream) {
+// The activations re-laid so that the fast kernels can read them: one input family whose kept blocks (or whose row
+// pitch / base address) are not on 16-byte boundaries becomes the same family with every block padded to a multiple
+// of 8 channels, the padding zero (the extra channels then meet real weights with zero activations).  Fills `q` with
+// the parameters of the re-laid problem (x still to be set) and returns the padded block size, or 0 when the map
+// does not allow it.
+int relay_candidate(const Params& p, Params* q) {
+  if (p.imap.n_fam != 1) return 0;
+  const Fam& a = p.imap.fam[0];
+  const int keep8 = (a.keep + 7) / 8 * 8;
+  if ((a.start % 8) != 0) return 0;
+  if (a.count > 1 && ((a.period % 8) != 0 || keep8 > a.period)) return 0;
+  if (a.count == 1 && a.start + keep8 > p.K) return 0;
+  *q = p;
+  q->imap.fam[0].keep = keep8;
+  q->imap.total = keep8 * a.count;
+  q->imap.base[0] = 0;
+  q->k_in = q->imap.total;
+  q->ldx = q->imap.total;
+  q->x = reinterpret_cast<const void*>((uintptr_t)256);     // (aligned as the workspace region will be)
+  return keep8;
+}
+
+int dispatch(const Params& p_in, void* workspace, size_t ws_bytes, void* stream) {
   if (cudaPeekAtLastError() != cudaSuccess) return UNIQL_ERR_CUDA;
   LaunchCfg cfg{workspace, ws_bytes, (cudaStream_t)stream};
   int path = g_path.load();
+  Params p = p_in;
   bool dec_ok = p.M <= 16 && decode_supported(p);
   // every batch the decode kernel does not take (more than 16 rows, bf16) goes to the tensor cores when the maps
   // allow it: at 17..63 rows the generic kernel measured 13 to 26 times slower (930 us against 71 us for the
   // Llama-3-8B gate|up at M = 17)
   bool pre_ok = prefill_supported(p);
-  if (path == UNIQL_PATH_AUTO) {
-    // one to four rows whose input map is on 4- but not 8-channel boundaries (head dims 108 and 84, 1740 of 2048
-    // channels): the streaming kernel; the persistent kernel would stage those activations element by element
-    const bool gemv_first = opt(kOptGemvFirst) == 1;
-    const bool gv = gemv_supported(p) && (gemv_first || !(dec_ok && decode_integer_path(p)));
-    path = gv ? UNIQL_PATH_GEMV : dec_ok ? UNIQL_PATH_DECODE : (pre_ok ? UNIQL_PATH_PREFILL : UNIQL_PATH_GENERIC);
+  // one to four rows whose input map is on 4- but not 8-channel boundaries (head dims 108 and 84, 1740 of 2048
+  // channels): the streaming kernel, which stages activations in 8-byte units
+  const bool gv = path == UNIQL_PATH_GEMV ||
+                  (path == UNIQL_PATH_AUTO && gemv_supported(p) &&
+                   (opt(kOptGemvFirst) == 1 || !(dec_ok && decode_integer_path(p))));
+  // Everything else that misses a fast kernel only because of where its activations lie (blocks of 108 or 84
+  // channels, an odd row pitch) gets them re-laid in the workspace by a small kernel in front: 5..16 rows then run
+  // on the integer path of the decode kernel, larger batches and bf16 on the tensor cores.
+  if (!gv && path != UNIQL_PATH_GENERIC) {
+    const bool decode_size = p.M <= 16 && p.dt == UNIQL_F16 && path != UNIQL_PATH_PREFILL;
+    const bool slow = decode_size ? !(dec_ok && decode_integer_path(p)) : !pre_ok;
+    Params q;
+    int keep8 = 0;
+    if (slow && path != (decode_size ? UNIQL_PATH_PREFILL : UNIQL_PATH_DECODE) && (keep8 = relay_candidate(p, &q)) != 0 &&
+        (decode_size ? (decode_supported(q) && decode_integer_path(q)) : prefill_supported(q))) {
+      if (!cfg.workspace) {
+        int rc = lib_workspace(&cfg.workspace, &cfg.ws_bytes, cfg.stream);
+        if (rc != UNIQL_OK) return rc;
+      }
+      const size_t bytes = (((size_t)p.M * (size_t)q.ldx * 2) + 255) & ~(size_t)255;
+      const size_t floor_bytes = decode_size ? decode_workspace_bytes(p.M, p.K, 1) : decode_workspace_header_bytes();
+      if (cfg.ws_bytes >= bytes + floor_bytes + 256) {
+        // the copy lives at the end of the workspace; the kernels get what lies before it
+        const size_t off = (cfg.ws_bytes - bytes) & ~(size_t)255;
+        void* xr = reinterpret_cast<unsigned char*>(cfg.workspace) + off;
+        const Fam& a = p.imap.fam[0];
+        int rc = launch_relay_x(p.x, p.ldx, p.M, a.count, a.keep, keep8, xr, cfg.stream);
+        if (rc != UNIQL_OK) return rc;
+        q.x = xr;
+        p = q;
+        cfg.ws_bytes = off;
+        dec_ok = p.M <= 16 && decode_supported(p);
+        pre_ok = prefill_supported(p);
+      }
+    }
   }
+  if (path == UNIQL_PATH_AUTO)
+    path = gv ? UNIQL_PATH_GEMV : dec_ok ? UNIQL_PATH_DECODE : (pre_ok ? UNIQL_PATH_PREFILL : UNIQL_PATH_GENERIC);
   if (path == UNIQL_PATH_GEMV) {
     if (!gemv_supported(p)) return UNIQL_ERR_UNSUPPORTED;
     if (!cfg.workspace) {
@@ -144,7 +198,7 @@ int dispatch(const Params& p, void* workspace, size_t ws_bytes, void* stream) {
     // Batches of 9..16: the staged activations of 16 rows do not fit beside the stage ring, which would
     // force the input channels to be split over two groups of blocks and every tile through a hand-over.
     // Two launches over half the batch each re-read the weights but run more than twice as fast
-    // (UNIQL_DECODE_SPLIT_BATCH=0: one launch).
+    // (option "decode_split_batch" 0: one launch).
     const bool split_batch = opt(kOptDecodeSplitBatch) != 0;
     if (p.M > 8 && split_batch) {
       const int m1 = (p.M + 1) / 2;
@@ -209,9 +263,11 @@ extern "C" int uniql_set_path(int path) {
 
 extern "C" size_t uniql_workspace_bytes(int M, int K, int N_total) {
   if (M < 1 || K < 1 || N_total < 1) return 0;
-  if (M > 16) return prefill_workspace_bytes(M, K);
+  // (+ room for the activations re-laid on 8-channel boundaries, see dispatch())
+  const size_t relay = (((size_t)M * (size_t)(K + 8) * 2) + 255) / 256 * 256 + 512;
+  if (M > 16) return prefill_workspace_bytes(M, K) + relay;
   const size_t a = decode_workspace_bytes(M, K, N_total), b = M <= 4 ? gemv_workspace_bytes(M, K, N_total) : 0;
-  return a > b ? a : b;
+  return (a > b ? a : b) + relay;
 }
 
 extern "C" int uniql_workspace_init(void* workspace, size_t bytes, void* stream) {

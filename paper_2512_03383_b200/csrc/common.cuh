@@ -156,6 +156,8 @@ struct LaunchCfg {
                          // once the launch is certain (a workspace that may hold what an unfinished call left)
 };
 int launch_generic(const Params& p, const LaunchCfg& cfg);
+// out[m][h * keep8 + r] = r < keep ? x[m][h * keep + r] : 0  (2-byte elements; out 16-byte aligned, keep8 % 8 == 0)
+int launch_relay_x(const void* x, long long ldx, int M, int count, int keep, int keep8, void* out, cudaStream_t stream);
 int launch_decode(const Params& p, const LaunchCfg& cfg);
 int decode_supported(const Params& p);
 int decode_integer_path(const Params& p);   // its int8 path takes the input map (8-channel boundaries)

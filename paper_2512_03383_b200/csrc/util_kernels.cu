@@ -75,6 +75,32 @@ __global__ void embed_kernel(const uint8_t* __restrict__ packed, const __half* _
   }
 }
 
+// Activations re-laid with every kept block padded to a multiple of 8 channels (zeros in the padding): the fast
+// kernels read activations in 16-byte units, which blocks of 108 or 84 channels (multiples of 4) do not give.
+// One thread per 4 output channels (8 bytes); x needs 2-byte alignment only.
+__global__ void relay_x_kernel(const unsigned short* __restrict__ x, long long ldx, int M, int count, int keep, int keep8,
+                               unsigned short* __restrict__ out) {
+  const int units_row = count * (keep8 >> 2);
+  const long long total = (long long)M * units_row;
+  const bool vec = ((ldx & 3) == 0) && ((((uintptr_t)x) & 7) == 0) && ((keep & 3) == 0);
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const int m = (int)(i / units_row), u = (int)(i - (long long)m * units_row);
+    const int h = u / (keep8 >> 2), r = (u - h * (keep8 >> 2)) * 4;
+    const unsigned short* src = x + (size_t)m * ldx + (size_t)h * keep + r;
+    uint2 v = make_uint2(0u, 0u);
+    if (vec && r + 4 <= keep) {
+      v = *reinterpret_cast<const uint2*>(src);
+    } else {
+      unsigned short e[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) e[k] = r + k < keep ? src[k] : (unsigned short)0;
+      v.x = (uint32_t)e[0] | ((uint32_t)e[1] << 16);
+      v.y = (uint32_t)e[2] | ((uint32_t)e[3] << 16);
+    }
+    *reinterpret_cast<uint2*>(out + (size_t)m * ((size_t)count * keep8) + (size_t)h * keep8 + r) = v;
+  }
+}
+
 inline int grid_for(int64_t n, int threads) {
   static const int sms = [] {
     int dev = 0, v = 0;
@@ -90,6 +116,13 @@ inline int grid_for(int64_t n, int threads) {
 
 }  // namespace
 }  // namespace uniql
+
+int uniql::launch_relay_x(const void* x, long long ldx, int M, int count, int keep, int keep8, void* out, cudaStream_t stream) {
+  const int64_t units = (int64_t)M * count * (keep8 / 4);
+  relay_x_kernel<<<grid_for(units, 256), 256, 0, stream>>>(reinterpret_cast<const unsigned short*>(x), ldx, M, count, keep, keep8,
+                                                           reinterpret_cast<unsigned short*>(out));
+  return cudaGetLastError() == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
+}
 
 using namespace uniql;
 

@@ -39,7 +39,9 @@ def test_noalloc_matches_oracle_and_regular_entry_point_twice_in_a_row():
             assert B.noalloc_status() == 0
             o = oracle.qlinear(x32, packed, qw.scales, qw.zeros, oracle.leading(k), oracle.leading(k))
             check_output(y_new, o, "f16", TOL, "noalloc M=%d k=%d" % (M, k))
-            if M <= 8:      # the same kernel on the same plan (larger batches: one launch here, two halves there)
+            # the same kernel on the same plan: up to eight rows (larger batches: one launch here, two halves there)
+            # and channels in multiples of 8 (otherwise the regular entry point re-lays the activations first)
+            if M <= 8 and k % 8 == 0:
                 assert torch.equal(y_new, y_ref), "M=%d k=%d: not bitwise equal to uniql_qlinear" % (M, k)
     finally:
         B.set_path(B.PATH_AUTO)
