@@ -506,13 +506,14 @@ def test_qk_rope_llama_shape(B, M):
 
 
 # ---------------------------------------------------------------- configuration 2 at full size (sampled rows of the MLP)
-@pytest.mark.parametrize("M", [1, 16])
+@pytest.mark.parametrize("M", [1, 4, 16])
 def test_llama_mlp_full_size(B, M):
+    """Every batch size and every keep rate of configuration 2."""
     rng = np.random.default_rng(2)
     gate = synth.random_qweight_fast(rng, 14336, 4096)
     down = synth.random_qweight_fast(rng, 4096, 14336)
     dg, dd = dev_weight(gate), dev_weight(down)
-    for rate in (1.0, 0.65):
+    for rate in (1.0, 0.85, 0.75, 0.65):
         k = synth.keep_count(rate, 14336)
         x = synth.draw_x(rng, M, 4096, "f16")
         y, ref = run_ex(B, gate, dg, x, "f16", None, 4096, None, k)

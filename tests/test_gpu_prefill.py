@@ -196,7 +196,7 @@ def test_qwen_gate_down_full_size_sampled(B, M):
     rng = np.random.default_rng(4)
     gate = synth.random_qweight_fast(rng, 18944, 3584)
     dg = dev_weight(gate)
-    for rate in (1.0, 0.65):
+    for rate in (1.0, 0.85, 0.65):
         k = synth.keep_count(rate, 18944)
         x = synth.draw_x(rng, M, 3584, "bf16")
         xd = dev_x(x, "bf16")
@@ -209,7 +209,7 @@ def test_qwen_gate_down_full_size_sampled(B, M):
     del dg
     down = synth.random_qweight_fast(rng, 3584, 18944)
     dd = dev_weight(down)
-    for rate in (1.0, 0.65):
+    for rate in (1.0, 0.85, 0.65):
         k = synth.keep_count(rate, 18944)
         h = synth.draw_x(rng, M, k, "bf16")
         hd = dev_x(h, "bf16")
@@ -293,7 +293,7 @@ def test_mamba2_full_size(B, M):
     qout = synth.random_qweight_fast(rng, 2560, d_inner)
     din, dout = dev_weight(qin), dev_weight(qout)
     rows = _sampled_rows(M)
-    for keep in (64, 48):
+    for keep in (64, 56, 48):
         om = synth.map_mamba_in_proj(d_inner, headdim, keep, d_state, 1, nheads)
         n_out = synth.map_size(om)
         x = synth.draw_x(rng, M, 2560, "f16")
@@ -310,3 +310,78 @@ def test_mamba2_full_size(B, M):
         torch.cuda.synchronize()
         ref2 = oracle.qlinear(h, dout[0], qout.scales, qout.zeros, oracle.leading(2560), oracle.expand_map(im), rows=rows)
         check_output(y2[rows], ref2, "f16", TOL["f16"], "mamba out_proj keep %d M=%d" % (keep, M))
+
+
+@pytest.mark.parametrize("keep", [108, 96, 84])
+def test_llama_attention_m512_pruned_heads(B, keep):
+    """Configuration 3 at M = 512 with Llama-3-8B shapes and pruned heads: q|k|v in one launch with the rotary
+    epilogue on q and k, then o_proj over the kept channels of every head (108 and 84 are multiples of 4 only: the
+    activations are re-laid on 8-channel boundaries in front of the tensor-core kernel).  Sampled token rows."""
+    rng = np.random.default_rng(46 + keep)
+    M, K, Hq, Hkv, D, theta = 512, 4096, 32, 8, 128, 5e5
+    wq, wk, wv = (synth.random_qweight_fast(rng, Hq * D, K), synth.random_qweight_fast(rng, Hkv * D, K),
+                  synth.random_qweight_fast(rng, Hkv * D, K))
+    dq, dk, dv = dev_weight(wq), dev_weight(wk), dev_weight(wv)
+    x = synth.draw_x(rng, M, K, "f16")
+    xd = dev_x(x, "f16")
+    pos, idx = synth.draw_pos(rng, M), synth.draw_idx(rng, Hkv, D, keep)
+    rows = _sampled_rows(M)
+    qo = torch.zeros((M, Hq * keep), dtype=torch.float16, device="cuda")
+    ko = torch.zeros((M, Hkv * keep), dtype=torch.float16, device="cuda")
+    vo = torch.zeros((M, Hkv * keep), dtype=torch.float16, device="cuda")
+    B.qkv_rope_proj(xd, K, dq[1], dq[2], dq[3], dk[1], dk[2], dk[3], dv[1], dv[2], dv[3], None, None, None, M, K, Hq, Hkv,
+                    D, keep, keep, torch.from_numpy(idx).cuda(), torch.from_numpy(pos).cuda(), theta, None, qo, Hq * keep,
+                    ko, Hkv * keep, vo, Hkv * keep)
+    torch.cuda.synchronize()
+    for (w, d, nh, g) in ((wq, dq, Hq, qo), (wk, dk, Hkv, ko)):
+        O = oracle.expand_map(oracle.qk_halfhead_map(nh, D, keep))
+        acc = oracle.qlinear(x, d[0], w.scales, w.zeros, O, oracle.leading(K), rows=rows)
+        check_output(g[rows], oracle.rope(acc, nh, Hkv, D, keep, idx, pos[rows], theta), "f16", TOL["f16"],
+                     "llama q/k rope keep %d M=512" % keep)
+    Ov = oracle.expand_map(synth.map_per_head(Hkv, D, keep))
+    check_output(vo[rows], oracle.qlinear(x, dv[0], wv.scales, wv.zeros, Ov, oracle.leading(K), rows=rows), "f16",
+                 TOL["f16"], "llama v keep %d M=512" % keep)
+    del dq, dk, dv
+    wo = synth.random_qweight_fast(rng, K, Hq * D)
+    do = dev_weight(wo)
+    im = synth.map_per_head(Hq, D, keep)
+    a = synth.draw_x(rng, M, Hq * keep, "f16")
+    yo = torch.zeros((M, K), dtype=torch.float16, device="cuda")
+    B.set_path(B.PATH_PREFILL)                      # the tensor-core kernel must take it
+    B.qlinear_ex(dev_x(a, "f16"), Hq * keep, do[1], do[2], do[3], None, M, Hq * D, K, im, 0, None, K, yo, K)
+    torch.cuda.synchronize()
+    ref = oracle.qlinear(a, do[0], wo.scales, wo.zeros, oracle.leading(K), oracle.expand_map(im), rows=rows)
+    check_output(yo[rows], ref, "f16", TOL["f16"], "llama o_proj keep %d M=512" % keep)
+    assert B.workspace_status() == 0
+
+
+def test_bf16_activations_outside_fp16_range(B):
+    """The tensor cores run on an fp16 copy of bf16 activations.  Documented consequences: magnitudes above 65504
+    saturate, magnitudes under 2^-14 keep fewer significand bits and those under 2^-24 become zero.  A small
+    activation is therefore off by at most 2^-25 in absolute terms, and an output by at most sum |w| * 2^-25 (plus
+    the usual tolerance); a saturated activation contributes w * 65504 instead of w * x."""
+    B.set_path(B.PATH_PREFILL)
+    rng = np.random.default_rng(47)
+    qw = synth.draw_qweight(rng, 136, 512)
+    dw = dev_weight(qw)
+    M = 40
+    x = (rng.standard_normal((M, 512)) * 1e-5).astype(np.float32)
+    x = torch.from_numpy(x).to(torch.bfloat16).float().numpy()            # bf16 values, well under 2^-14
+    y = torch.zeros((M, 136), dtype=torch.bfloat16, device="cuda")
+    B.qlinear_ex(dev_x(x, "bf16"), 512, dw[1], dw[2], dw[3], None, M, 512, 136, None, 512, None, 136, y, 136)
+    torch.cuda.synchronize()
+    ref = oracle.qlinear(x, dw[0], qw.scales, qw.zeros, oracle.leading(136), oracle.leading(512))
+    wabs = np.abs(oracle.dequant(dw[0], qw.scales, qw.zeros)).sum(axis=1)  # sum |w| per output row
+    g = y.double().cpu().numpy()
+    bound = wabs[None, :] * 2.0 ** -25 + 5e-4 * np.abs(ref).max() + np.abs(ref) * 2.0 ** -8
+    assert np.isfinite(g).all() and (np.abs(g - ref) <= bound).all(), "small activations: beyond the flush bound"
+    # saturation: one activation of 1e6 acts as 65504
+    x2 = np.zeros((M, 512), dtype=np.float32)
+    x2[:, 7] = 999424.0                                                   # a bf16 value near 1e6
+    y2 = torch.zeros((M, 136), dtype=torch.bfloat16, device="cuda")
+    B.qlinear_ex(dev_x(x2, "bf16"), 512, dw[1], dw[2], dw[3], None, M, 512, 136, None, 512, None, 136, y2, 136)
+    torch.cuda.synchronize()
+    x2s = x2.copy()
+    x2s[:, 7] = 65504.0
+    ref2 = oracle.qlinear(x2s, dw[0], qw.scales, qw.zeros, oracle.leading(136), oracle.leading(512))
+    check_output(y2, ref2, "bf16", TOL["bf16"], "saturated activation")
