@@ -692,7 +692,7 @@ class QwenPrefill:
 
 def run_case(args):
     """A few plain (un-graphed) launches of one kernel on a small set-up, for ncu captures:
-    --case decode-gateup | decode-down | prefill-gate | prefill-down, with --M and --keep."""
+    --case decode-gateup | decode-down | decode-big | prefill-gate | prefill-down, with --M and --keep (and --gemv)."""
     import torch
     from paper_2512_03383_b200 import binding as B
     torch.cuda.set_device(0)
@@ -702,6 +702,20 @@ def run_case(args):
             (q.gate if args.case == "prefill-gate" else q.down)(args.keep)
         torch.cuda.synchronize()
         print("case %s M=%d keep=%.2f: %d launches done" % (args.case, args.M, args.keep, args.launches))
+        return 0
+    if args.gemv:
+        B.set_option("gemv_first", 1)           # the streaming kernel wherever it applies (M <= 4)
+    if args.case == "decode-big":
+        # one tall matrix (65536 x 4096, 140 MB: larger than L2), plain launches
+        N = 65536
+        ws = [dev_qweight(torch, N, HIDDEN, 50 + i) for i in range(2)]
+        x = dev_x(torch, args.M, HIDDEN, torch.float16, 5)
+        y = torch.zeros((args.M, N), dtype=torch.float16, device="cuda")
+        for i in range(args.launches):
+            w = ws[i % 2]
+            B.qlinear_ex(x, HIDDEN, w[0], w[1], w[2], None, args.M, HIDDEN, N, None, HIDDEN, None, N, y, N)
+        torch.cuda.synchronize()
+        print("case %s M=%d gemv=%d: %d launches done" % (args.case, args.M, int(args.gemv), args.launches))
         return 0
     w = MlpDecode(B, torch, args.M)
     k = keep_count(args.keep, INTER)
@@ -770,6 +784,7 @@ def main():
     ap.add_argument("--M", type=int, default=1)
     ap.add_argument("--keep", type=float, default=1.0)
     ap.add_argument("--launches", type=int, default=4)
+    ap.add_argument("--gemv", action="store_true", help="with --case: run the streaming kernel wherever it applies")
     args = ap.parse_args()
     if args.traffic_hash:
         print(kernel_source_hash())

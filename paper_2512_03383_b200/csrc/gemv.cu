@@ -6,18 +6,18 @@
 //
 // Work.  A tile is 16 MMA rows, a step is GCH quantisation groups (512 input channels) of a tile: 4 KB of codes and
 // their scales / zero-points.  The steps of all tiles form one sequence (tile after tile); it is cut into equal
-// contiguous ranges, one per WARP, so every warp streams the same number of bytes whatever the shape.  A warp is
-// its own pipeline: every lane copies the 16 bytes it will later use as an MMA fragment straight from global memory
-// into a private shared-memory ring with asynchronous copies (several steps ahead, no registers held, no barrier
-// and no other warp involved), and consumes them in order.  A tile whose steps fall into several warps' ranges is
-// finished by the last of them to arrive: each parks its fp32 partial sums in the workspace, and the last one adds
-// them in range order (deterministic).
+// contiguous ranges, one per WARP of a persistent grid (one block of eight warps per SM), so every warp streams the
+// same number of bytes whatever the shape.  A warp is its own pipeline: it copies its steps from global memory into
+// a private shared-memory ring with asynchronous 16-byte copies, four steps ahead (sixteen lanes fetch 256
+// contiguous bytes of a weight row; no registers held, no block-wide barrier, no other warp involved), and consumes
+// them in order.  A tile whose steps fall into several warps' ranges is finished by the last of them to arrive:
+// each parks its fp32 partial sums in the workspace, and the last one adds them in range order (deterministic).
 //
-// Activations.  A small kernel in front quantises x once per call to 16-bit fixed point per (batch row,
-// 128-channel group), split into a high and a low signed byte, in the order the nibbles leave a weight word; the
-// streaming kernel reads its B fragments from that copy (a few KB, served by L1).  The streaming kernel is
-// launched with programmatic stream serialization and fills its rings with weights, which no preceding kernel
-// produces, while the quantising kernel and the tail of the preceding call are still running.
+// Activations.  The rings are filled before the dependency wait (weights are never produced by the preceding
+// kernel); after it every block quantises the activations once into its shared memory: 16-bit fixed point per
+// (batch row, 128-channel group), split into a high and a low signed byte, in the order the nibbles leave a
+// weight word.  Activations are fetched in units of 4 channels, so kept blocks of 108 or 84 channels and blocks of
+// 1740 leading channels need no re-laying.
 //
 // On-device pruning (Section 3.4) is index arithmetic: a tile only addresses kept rows, a step only visited input
 // groups, and pruned input channels inside a visited group meet zero activations.
