@@ -818,14 +818,16 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   // stream-K for the tiles left over when whole tiles would leave SMs idle in their last round and the partial
   // tiles fit in the workspace.  It pays when the k-blocks a block no longer waits for outweigh the hand-over:
   // measured on B200, a k-block takes about 0.65 us, and the hand-over (zeroing the sums, the additions, the
-  // read-back by the finishing block) about 24 us for tiles of 256 tokens when whole tiles follow and hide
+  // read-back by the finishing block) about 14 us for tiles of 256 tokens when whole tiles follow and hide
   // most of it, 28 us when every tile is split; both shrink with the tile's width.
   {
     int g2 = sms;
     if (env_grid >= 1 && env_grid <= sms) g2 = env_grid;
     const int left = c.n_tiles % g2;
     const double share = (double)left * c.n_kb / g2;                   // k-blocks per block of the split tiles
-    const double hand_over = c.n_tiles < g2 ? 10.0 + 18.0 * c.bn / 256.0 : 24.0 * c.bn / 256.0;
+    // (whole tiles that follow hide most of the hand-over: forcing the split on the Qwen2.5-7B q projection at
+    //  M = 2048 and on the Mamba2 in_proj at M = 1024 saved 5.7 and 5.3 us where this rule's saving was 17.7 and 19.7 us)
+    const double hand_over = c.n_tiles < g2 ? 10.0 + 18.0 * c.bn / 256.0 : 14.0 * c.bn / 256.0;
     const bool pays = ((double)c.n_kb - share) * 0.65 > hand_over;
     const size_t sums = (size_t)left * c.bn * BMW * 4;                 // one fp32 tile per left-over tile
     const size_t need = ws_used + sums;
