@@ -385,3 +385,20 @@ def test_bf16_activations_outside_fp16_range(B):
     x2s[:, 7] = 65504.0
     ref2 = oracle.qlinear(x2s, dw[0], qw.scales, qw.zeros, oracle.leading(136), oracle.leading(512))
     check_output(y2, ref2, "bf16", TOL["bf16"], "saturated activation")
+
+
+def test_caller_workspace_smaller_than_the_header_is_refused(B):
+    """The tensor-core kernel keeps its status word in the workspace header: a caller workspace that cannot even
+    hold the header is turned down before anything is launched."""
+    B.set_path(B.PATH_PREFILL)
+    rng = np.random.default_rng(48)
+    qw = synth.draw_qweight(rng, 64, 256)
+    dw = dev_weight(qw)
+    x = dev_x(synth.draw_x(rng, 32, 256, "f16"), "f16")
+    y = torch.full((32, 64), -77.0, dtype=torch.float16, device="cuda")
+    tiny = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.UniqlError) as e:
+        B.qlinear_ex(x, 256, dw[1], dw[2], dw[3], None, 32, 256, 64, None, 256, None, 64, y, 64, workspace=tiny)
+    assert e.value.status == 6
+    torch.cuda.synchronize()
+    assert (y == -77.0).all()
