@@ -124,7 +124,9 @@ int uniql_set_path(int path);
  *   "prefill_streamk"  -1 automatic, 0 never, 1 always: split the contraction of the output tiles of the last,
  *                      partly filled round of the tensor-core kernel over several thread blocks.  0 makes the
  *                      results of that kernel reproducible bit for bit (every tile is summed by one block).
- *   "decode_split_batch" 1 / 0: batches of 9..16 rows as two launches over half the batch (default 1)
+ *   "decode_split_batch" batches of 9..16 rows: 2 (default) one launch that streams the quantised activations
+ *                      beside the weights, where the integer path applies, else two launches over half the batch;
+ *                      1 always two launches; 0 always one launch with the activations staged whole
  * The others steer the work split of the kernels and exist for the tests: "decode_kp", "decode_rp",
  * "decode_stages", "decode_narrow", "decode_xstream", "decode_xcluster", "decode_i8", "prefill_grid",
  * "prefill_convert", "gemv_first", "gemv_depth", and "wait_shift" (the poll limit of the barrier between the two
@@ -194,8 +196,9 @@ int uniql_qlinear(const void* x, const uint8_t* packed_w, const void* scales, co
  *    UNIQL_ERR_UNSUPPORTED.  A problem whose split-K partial sums do not fit the fixed array returns
  *    UNIQL_ERR_WORKSPACE and launches nothing.  The need is 256 KB plus roughly 512 bytes per 64
  *    retained rows and batch row (more when large M * K splits the input channels over several
- *    groups of thread blocks); the Llama-3-8B MLP matrices fit for every M <= 16.  Unlike uniql_qlinear, which
- *    runs batches of 9..16 rows as two launches over half the batch, this call always is one launch.
+ *    groups of thread blocks); the Llama-3-8B MLP matrices fit for every M <= 16.  Batches of 9..16 rows take
+ *    one launch here whatever option "decode_split_batch" says (streamed activations where they apply, else
+ *    staged ones), and the small kernel that quantises streamed activations writes into the same array.
  *  - The first call on a device looks up the array's device address (once per device, with that
  *    device current); make that first call outside any stream capture.
  *  - All calls share the one array, and it keeps what the previous call left: each call clears the
@@ -278,7 +281,8 @@ int uniql_qkv_rope_proj(const void* x, int ldx, int dt, const uint8_t* wq, const
  *   down projection are prefetched across the barrier); UNIQL_ERR_UNSUPPORTED when M > 8 or the staged
  *   activations do not fit in shared memory.  fuse = 0: two launches (gate|up with the gated product as
  *   epilogue, then down).  fuse = -1: the faster of the two on this hardware (two launches: the boundary
- *   between dependent launches costs less than the grid-wide barrier).  M in 9..16 runs as two halves.
+ *   between dependent launches costs less than the grid-wide barrier).  M in 9..16: each of the two launches
+ *   streams its quantised activations beside the weights (option "decode_split_batch" 1: two halves of the batch).
  * Limits at 1 <= M <= 16: fp16; hidden, inter multiples of 256; k_int a multiple of 8; ldx, ldh multiples
  * of 8; x and h 16-byte aligned.  Other shapes: UNIQL_ERR_UNSUPPORTED (compose uniql_qlinear_multi calls).
  * M > 16 (the name is historical): two launches of the tensor-core kernel.  The first takes Wg and Wu as a

@@ -27,7 +27,7 @@ const OptDesc kOpts[kOptCount] = {
     {"decode_xstream", "UNIQL_DECODE_XSTREAM", -1},     // streamed activations: -1 automatic, 0 off, 1 on
     {"decode_xcluster", "UNIQL_DECODE_XCLUSTER", -1},   // shared staging in clusters of two: -1 automatic, 0 off, 1 on
     {"decode_i8", "UNIQL_DECODE_I8", 1},                // integer path (0: fp16 MMAs)
-    {"decode_split_batch", "UNIQL_DECODE_SPLIT_BATCH", 1},   // batches of 9..16 as two launches
+    {"decode_split_batch", "UNIQL_DECODE_SPLIT_BATCH", 2},   // batches of 9..16: one streamed launch where it applies
     {"prefill_grid", "UNIQL_PREFILL_GRID", 0},          // blocks of the tensor-core kernel (0: one per SM)
     {"prefill_convert", "UNIQL_PREFILL_CONVERT_IN_KERNEL", 0},   // 1: bf16 tiles converted inside the kernel
     {"prefill_streamk", "UNIQL_PREFILL_STREAMK", -1},   // split tiles: -1 automatic, 0 never (reproducible sums), 1 always
@@ -197,9 +197,12 @@ int dispatch(const Params& p_in, void* workspace, size_t ws_bytes, void* stream)
     }
     // Batches of 9..16: the staged activations of 16 rows do not fit beside the stage ring, which would
     // force the input channels to be split over two groups of blocks and every tile through a hand-over.
-    // Two launches over half the batch each re-read the weights but run more than twice as fast
-    // (option "decode_split_batch" 0: one launch).
-    const bool split_batch = opt(kOptDecodeSplitBatch) != 0;
+    // The integer path streams the activations through the ring instead (one launch, the weights read once);
+    // elsewhere two launches over half the batch each re-read the weights but still run more than twice as fast
+    // as the split channels (option "decode_split_batch": 2 as described, 1 always two launches, 0 always one
+    // launch with staged activations).
+    const int sb = opt(kOptDecodeSplitBatch);
+    const bool split_batch = sb == 1 || (sb == 2 && !decode_streams_batch(p));
     if (p.M > 8 && split_batch) {
       const int m1 = (p.M + 1) / 2;
       const size_t esz = 2;                               // fp16 / bf16
@@ -542,7 +545,9 @@ extern "C" int uniql_mlp_swiglu_decode(const void* x, int ldx, const uint8_t* wg
     // than the grid-wide barrier of the single launch (measured 29.2 us against 32.6 us per Llama-3-8B layer)
     return launch_mlp_decode(q, fuse == 1 ? 1 : 0, cfg);
   };
-  if (M > 8 && fuse != 1) {      // as for the plain decode path: two halves of the batch
+  // (nine to sixteen rows: one pass with streamed activations, or under option "decode_split_batch" 0 / 1 as for
+  // the plain decode path)
+  if (M > 8 && fuse != 1 && !(opt(kOptDecodeSplitBatch) == 2 && opt(kOptDecodeXstream) != 0 && opt(kOptDecodeI8) != 0)) {
     const int m1 = (M + 1) / 2;
     MlpDecode a = d, b = d;
     a.M = m1;

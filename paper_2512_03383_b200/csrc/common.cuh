@@ -160,7 +160,8 @@ int launch_generic(const Params& p, const LaunchCfg& cfg);
 int launch_relay_x(const void* x, long long ldx, int M, int count, int keep, int keep8, void* out, cudaStream_t stream);
 int launch_decode(const Params& p, const LaunchCfg& cfg);
 int decode_supported(const Params& p);
-int decode_integer_path(const Params& p);   // its int8 path takes the input map (8-channel boundaries)
+int decode_integer_path(const Params& p);
+int decode_streams_batch(const Params& p);   // its int8 path takes the input map (8-channel boundaries)
 size_t decode_workspace_bytes(int M, int K, int N_total);
 int decode_status_offset();   // byte offset of the device status word inside a workspace
 size_t decode_workspace_header_bytes();   // counters + status word: the part that must start at zero

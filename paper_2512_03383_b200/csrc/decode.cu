@@ -245,6 +245,13 @@ __device__ inline void lds128_if(uint4& v, uint32_t addr, bool pred) {      // v
   asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %5, 0;\n\t@p ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+%6];\n\t}"
                : "+r"(v.x), "+r"(v.y), "+r"(v.z), "+r"(v.w) : "r"(addr), "r"((uint32_t)pred), "n"(OFF));
 }
+// line nt * 1024 bytes further on (the index is a constant once the caller's loop is unrolled)
+__device__ inline void lds128_line(uint4& v, uint32_t addr, int nt, bool pred) {
+  if (nt == 0) lds128_if<0>(v, addr, pred);
+  else if (nt == 1) lds128_if<1024>(v, addr, pred);
+  else if (nt == 2) lds128_if<2048>(v, addr, pred);
+  else lds128_if<3072>(v, addr, pred);
+}
 template <int OFF>
 __device__ inline float4 lds128f(uint32_t addr) {
   float4 v;
@@ -310,7 +317,7 @@ __device__ inline int compact_channel(const Phase& P, int ch) {
 // Quantises the activations of one launch once (streamed mode): half-warp (batch row m, visited group lv).
 // Rows m >= M of the vr / 2 row slots are written as zeros.
 __global__ void __launch_bounds__(256) xquant_kernel(const Phase P, int M, int vr, int g_total, unsigned char* xq,
-                                                     float2* xg) {
+                                                     float2* xg, int xg_stride) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");            // x may come from the preceding kernel
   const int rows = vr >> 1;
@@ -332,7 +339,7 @@ __global__ void __launch_bounds__(256) xquant_kernel(const Phase P, int M, int v
       const int off = (u16 >> 2) * 32 + (u16 & 3) * 8;
       *reinterpret_cast<uint2*>(xq + ((size_t)lv * vr + 2 * m) * 128 + off) = hi2;
       *reinterpret_cast<uint2*>(xq + ((size_t)lv * vr + 2 * m + 1) * 128 + off) = lo2;
-      if (u16 == 0) xg[lv * 8 + m] = make_float2((float)isum, inv_scale);
+      if (u16 == 0) xg[lv * xg_stride + m] = make_float2((float)isum, inv_scale);
     }
   }
 }
@@ -531,7 +538,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
   // XS / XC say what this instance can do; whether a launch streams its activations or shares their staging is a
   // flag of the launch (batches of five to eight rows always take the same instance: alternating between two
   // kernel functions costs about 1.5 us per switch)
-  const bool xs_on = XS && c.x_stream != 0, xc_on = XC && c.x_cluster != 0;
+  // (the instances for nine to sixteen rows each serve one kind of launch only)
+  const bool xs_on = XS && (NT == 4 || c.x_stream != 0), xc_on = XC && c.x_cluster != 0;
   // barriers: full[S], empty[S], consumer barrier, (spare), partials full[2] / free[2]; then the abort flag
   const uint32_t bar_full = sbase + c.off_bar, bar_empty = bar_full + 8 * MAX_STAGES;
   const uint32_t bar_cons = bar_full + 16 * MAX_STAGES, bar_epi = bar_cons + 8;
@@ -578,9 +586,9 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
     auto send_x = [&](int stage, int lv0) {                          // lane 31: arrival + the unit's activations
       const uint32_t full = bar_full + 8 * stage;
       const uint32_t st = sbase + (uint32_t)stage * (uint32_t)c.stage_bytes;
-      mbar_expect_tx(full, (uint32_t)(c.vr * CG * 128 + CG * 64));
+      mbar_expect_tx(full, (uint32_t)(c.vr * CG * 128 + CG * 64 * MT));
       tma_box3(st + STAGE_BYTES, &c.xmap, 0, 0, lv0, full);
-      bulk_copy(st + STAGE_BYTES + (uint32_t)(c.vr * CG * 128), c.xg_glob + (size_t)lv0 * 8, CG * 64, full);
+      bulk_copy(st + STAGE_BYTES + (uint32_t)(c.vr * CG * 128), c.xg_glob + (size_t)lv0 * 8 * MT, CG * 64 * MT, full);
     };
     auto flush_x = [&](int n_issued) {                               // after the first min(S, units) stages
       asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -1053,7 +1061,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       xs0[nt] = line + (uint32_t)(((2 * t) ^ (v & 7)) * 16);
       xs1[nt] = line + (uint32_t)(((2 * t + 1) ^ (v & 7)) * 16);
     }
-    const uint32_t xsg = (uint32_t)(STAGE_BYTES + c.vr * CG * 128 + kpw * 64 + t * 8);
+    const uint32_t xsg = (uint32_t)(STAGE_BYTES + c.vr * CG * 128 + kpw * 64 * MT + t * 8);
     const uint32_t wl_off = (uint32_t)((kpw >> 1) * BOX_BYTES + (rg * 32 + pg) * 128 + ((((kpw & 1) * 4 + t) ^ pg) * 16));
     const uint32_t sl_off = (uint32_t)(STAGE_W + (rg * 32 + pg) * (CG * 2) + kpw * 2);
     float out8[2][NT][2];
@@ -1115,6 +1123,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       if (gi < Gk) {
         const uint32_t st = sbase + (uint32_t)s * (xs_on ? (uint32_t)c.stage_bytes : (uint32_t)STAGE_BYTES);
         const uint32_t wp = st + wl_off, sp = st + sl_off;
+        if constexpr (NT <= 2) {
         uint4 wa[2], wb[2];
         wa[0] = lds128<0>(wp);
         wb[0] = lds128<8 * 128>(wp);
@@ -1164,6 +1173,53 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
             const float y1 = (float)(d[sub][nt][2] * 256 + d[sub][nt][3]);
             out8[sub][nt][0] = fmaf(sc[sub][0] * xs.y, fmaf(-zp[sub][0], xs.x, y0), out8[sub][nt][0]);
             out8[sub][nt][1] = fmaf(sc[sub][1] * xs.y, fmaf(-zp[sub][1], xs.x, y1), out8[sub][nt][1]);
+          }
+        }
+        } else {
+          // Four column tiles (nine to sixteen rows): the two halves of the warp's 32 weight rows one after the
+          // other; the nibbles of a half are split once (16 words) and each column tile then runs its chain of four
+          // MMAs and its scaling on its own, so that 4 accumulators and the activation bytes of one tile are live
+          // at a time (all four tiles at once need more registers than a thread of this block can have).
+          const uint32_t xga = xs_on ? st + xsg : xgaddr8 + (uint32_t)(gi * 8 * MT * 8);
+#pragma unroll
+          for (int sub = 0; sub < 2; ++sub) {
+            uint32_t lo0[4], lo1[4], hi0[4], hi1[4];
+            {
+              const uint4 wa = sub == 0 ? lds128<0>(wp) : lds128<16 * 128>(wp);
+              const uint4 wb = sub == 0 ? lds128<8 * 128>(wp) : lds128<24 * 128>(wp);
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const uint32_t w0 = j == 0 ? wa.x : j == 1 ? wa.y : j == 2 ? wa.z : wa.w;
+                const uint32_t w1 = j == 0 ? wb.x : j == 1 ? wb.y : j == 2 ? wb.z : wb.w;
+                lo0[j] = w0 & 0x0f0f0f0fu; hi0[j] = (w0 >> 4) & 0x0f0f0f0fu;
+                lo1[j] = w1 & 0x0f0f0f0fu; hi1[j] = (w1 >> 4) & 0x0f0f0f0fu;
+              }
+            }
+            const float sc0 = sub == 0 ? lds_h<0>(sp) : lds_h<16 * CG * 2>(sp);
+            const float sc1 = sub == 0 ? lds_h<8 * CG * 2>(sp) : lds_h<24 * CG * 2>(sp);
+            const float zp0 = sub == 0 ? lds_h<STAGE_SZ>(sp) : lds_h<STAGE_SZ + 16 * CG * 2>(sp);
+            const float zp1 = sub == 0 ? lds_h<STAGE_SZ + 8 * CG * 2>(sp) : lds_h<STAGE_SZ + 24 * CG * 2>(sp);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              uint4 xa = make_uint4(0, 0, 0, 0), xb = make_uint4(0, 0, 0, 0);
+              if (xs_on) {
+                lds128_line(xa, st + xs0[0], nt, true);
+                lds128_line(xb, st + xs1[0], nt, true);
+              } else {
+                lds128_if<0>(xa, xaddr8[nt] + (uint32_t)(gi * 128), xlive8[nt]);
+                lds128_if<16>(xb, xaddr8[nt] + (uint32_t)(gi * 128), xlive8[nt]);
+              }
+              const float2 xs = nt == 0 ? lds64f<0>(xga) : nt == 1 ? lds64f<32>(xga) : nt == 2 ? lds64f<64>(xga) : lds64f<96>(xga);
+              int d[4];
+              mma_s8_first(d, lo0[0], lo1[0], hi0[0], hi1[0], xa.x, xa.y);
+              mma_s8(d, lo0[1], lo1[1], hi0[1], hi1[1], xa.z, xa.w);
+              mma_s8(d, lo0[2], lo1[2], hi0[2], hi1[2], xb.x, xb.y);
+              mma_s8(d, lo0[3], lo1[3], hi0[3], hi1[3], xb.z, xb.w);
+              const float y0 = (float)(d[0] * 256 + d[1]);
+              const float y1 = (float)(d[2] * 256 + d[3]);
+              out8[sub][nt][0] = fmaf(sc0 * xs.y, fmaf(-zp0, xs.x, y0), out8[sub][nt][0]);
+              out8[sub][nt][1] = fmaf(sc1 * xs.y, fmaf(-zp1, xs.x, y1), out8[sub][nt][1]);
+            }
           }
         }
       }
@@ -1574,10 +1630,10 @@ size_t plan_split(DecodeCfg* c, int M, int g_total, int gran, bool i8) {
 // Shared-memory plan with streamed activations: no staged copy of x, every stage carries the unit's eight
 // groups of quantised activations.  One k-part.  Returns 0 when nothing fits.
 size_t plan_stream(DecodeCfg* c, int M, int g_total, int gran) {
-  c->vr = M <= 4 ? 8 : 16;
+  c->vr = M <= 4 ? 8 : (M <= 8 ? 16 : 32);
   c->stage_bytes = STAGE_BYTES + c->vr * CG * 128 + 1024;
-  const int tries[4][2] = {{4, 2}, {4, 1}, {3, 2}, {3, 1}};
-  for (int i = 0; i < 4; ++i) {
+  const int tries[6][2] = {{4, 2}, {4, 1}, {3, 2}, {3, 1}, {2, 2}, {2, 1}};
+  for (int i = 0; i < 6; ++i) {
     const int stages = tries[i][0], part_bufs = tries[i][1];
     size_t off = (size_t)stages * c->stage_bytes;
     c->off_bar = (int)off;
@@ -1602,7 +1658,57 @@ size_t plan_stream(DecodeCfg* c, int M, int g_total, int gran) {
   return 0;
 }
 
+// Streamed activations, host side.  The quantised copy sits in the workspace behind the partial sums:
+// [groups, padded to whole chunks][vr virtual rows][128 bytes], then one (sum, 1 / scale) pair per group and
+// batch-row slot (8 slots up to eight rows, 16 above).
+struct StreamWs { size_t xq_off, xg_off; int g_pad, slots; };
+size_t stream_need(const DecodeCfg& c, int M, int g_total, size_t need, StreamWs* o) {
+  o->g_pad = round_up(g_total, CG);
+  o->slots = M <= 8 ? 8 : 16;
+  o->xq_off = (need + 255) & ~(size_t)255;
+  o->xg_off = o->xq_off + (size_t)o->g_pad * c.vr * 128;
+  return o->xg_off + (size_t)o->g_pad * 8 * o->slots;
+}
+// The tensor map over the quantised copy, and the small kernel in front that writes it (once per launch).
+int stream_setup(DecodeCfg& c, const Phase& P, int M, int g_total, unsigned char* ws, const StreamWs& o,
+                 cudaStream_t stream) {
+  EncodeTiledFn enc = encoder();
+  if (!enc) return UNIQL_ERR_CUDA;
+  const cuuint64_t dims[3] = {128, (cuuint64_t)c.vr, (cuuint64_t)o.g_pad};
+  const cuuint64_t strides[2] = {128, (cuuint64_t)c.vr * 128};
+  const cuuint32_t box[3] = {128, (cuuint32_t)c.vr, (cuuint32_t)CG};
+  const cuuint32_t es[3] = {1, 1, 1};
+  if (enc(&c.xmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, ws + o.xq_off, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return UNIQL_ERR_CUDA;
+  c.xg_glob = reinterpret_cast<const float2*>(ws + o.xg_off);
+  cudaLaunchConfig_t lc;
+  memset(&lc, 0, sizeof(lc));
+  const int units = g_total * (c.vr / 2) * 16;
+  lc.gridDim = dim3((units + 255) / 256);
+  lc.blockDim = dim3(256);
+  lc.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr;
+  lc.numAttrs = opt(kOptPdl) ? 1 : 0;
+  if (cudaLaunchKernelEx(&lc, xquant_kernel, P, M, c.vr, g_total, ws + o.xq_off,
+                         reinterpret_cast<float2*>(ws + o.xg_off), o.slots) != cudaSuccess) {
+    cudaGetLastError();
+    return UNIQL_ERR_CUDA;
+  }
+  return UNIQL_OK;
+}
+
 }  // namespace
+
+// Nine to sixteen rows in one launch: the activations of so many rows never fit beside the ring, so they are
+// streamed through it; the integer path only (option "decode_split_batch" 2, the default).
+int decode_streams_batch(const Params& p) {
+  return p.M > 8 && p.M <= 16 && opt(kOptDecodeSplitBatch) == 2 && opt(kOptDecodeI8) != 0 &&
+         opt(kOptDecodeXstream) != 0 && decode_integer_path(p);
+}
 
 int decode_supported(const Params& p) {
   if (p.M < 1 || p.M > 16) return 0;
@@ -1637,8 +1743,10 @@ size_t decode_workspace_bytes(int M, int K, int N_total) {
   const size_t chunks = (size_t)(G + CG - 1) / CG;
   const size_t tiles = (size_t)(N_total + RB - 1) / RB + (size_t)N_total / 32 + 2 * kMaxJobs;
   const size_t slots = tiles * 2 * c.n_kp + (size_t)c.n_rp * c.n_kp * (chunks + 2 * c.n_kp);
-  // (+ the quantised activations of the streamed mode: 16 virtual rows of 128 bytes and 64 bytes per group)
-  return (size_t)kWsHeader + slots * (size_t)M * RB * 4 + (size_t)round_up(G, CG) * (16 * 128 + 64) + 512;
+  // (+ the quantised activations of the streamed mode: 16 virtual rows of 128 bytes and 64 bytes per group, twice
+  // that for more than eight rows)
+  const size_t xs_group = M > 8 ? 2 * (16 * 128 + 64) : (16 * 128 + 64);
+  return (size_t)kWsHeader + slots * (size_t)M * RB * 4 + (size_t)round_up(G, CG) * xs_group + 512;
 }
 
 int launch_decode(const Params& p, const LaunchCfg& cfg) {
@@ -1659,12 +1767,20 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   // channels over several groups of blocks and hand every tile over); UNIQL_DECODE_XSTREAM=0/1 forces.  Where the
   // staged copy fits the quantising kernel in front costs more than the staging it saves (measured 3.5 us), and
   // inside a sequence of launches it only pays for itself at eight rows (Llama-3-8B MLP: 51.7 against 53.9 us
-  // at M = 8, 93.8 against 105.1 us at M = 16 as two launches of eight; 46.6 against 43.0 us at M = 5).
+  // at M = 8; 46.6 against 43.0 us at M = 5).  Nine to sixteen rows are always streamed: their staged copy never
+  // fits beside a ring of more than two positions (Llama-3-8B MLP at M = 16: 55 us in one pass, 82 us as two
+  // launches of eight rows, 145 us with the input channels split over two groups of blocks).
   size_t smem = 0;
   c.stage_bytes = STAGE_BYTES;
   {
     const int force = opt(kOptDecodeXstream);
-    if (i8 && p.M <= 8 && force != 0) {
+    if (i8 && p.M > 8) {
+      if (decode_streams_batch(p)) {
+        smem = plan_stream(&c, p.M, g_total, gran);
+        c.x_stream = smem != 0;
+        if (!smem) c.stage_bytes = STAGE_BYTES;
+      }
+    } else if (i8 && force != 0) {
       DecodeCfg t = c;
       const size_t s0 = plan_split(&t, p.M, g_total, gran, true);
       if (force == 1 || !s0 || (t.n_kp > 1 && p.M >= 8)) {
@@ -1764,13 +1880,8 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   if (tiles < 1 || tiles * EW > kCounterInts) return UNIQL_ERR_UNSUPPORTED;
   c.max_slots = slots_needed(tiles, c.g_total, c.gp, c.n_rp, c.cgz);
   size_t need = (size_t)kWsHeader + (size_t)tiles * c.max_slots * p.M * RB * 4;
-  size_t xq_off = 0, xg_off = 0;
-  const int g_pad = round_up(g_total, CG);
-  if (c.x_stream) {
-    xq_off = (need + 255) & ~(size_t)255;
-    xg_off = xq_off + (size_t)g_pad * c.vr * 128;
-    need = xg_off + (size_t)g_pad * 64;
-  }
+  StreamWs sw;
+  if (c.x_stream) need = stream_need(c, p.M, g_total, need, &sw);
   if (!cfg.workspace || cfg.ws_bytes < need) return UNIQL_ERR_WORKSPACE;
   unsigned char* ws = reinterpret_cast<unsigned char*>(cfg.workspace);
   c.counters = reinterpret_cast<int*>(ws);
@@ -1787,33 +1898,8 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
     }
   }
   if (c.x_stream) {
-    EncodeTiledFn enc = encoder();
-    if (!enc) return UNIQL_ERR_CUDA;
-    const cuuint64_t dims[3] = {128, (cuuint64_t)c.vr, (cuuint64_t)g_pad};
-    const cuuint64_t strides[2] = {128, (cuuint64_t)c.vr * 128};
-    const cuuint32_t box[3] = {128, (cuuint32_t)c.vr, (cuuint32_t)CG};
-    const cuuint32_t es[3] = {1, 1, 1};
-    if (enc(&c.xmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, ws + xq_off, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return UNIQL_ERR_CUDA;
-    c.xg_glob = reinterpret_cast<const float2*>(ws + xg_off);
-    // the activations are quantised once, by a small kernel in front of the streaming one
-    cudaLaunchConfig_t lc;
-    memset(&lc, 0, sizeof(lc));
-    const int units = g_total * (c.vr / 2) * 16;
-    lc.gridDim = dim3((units + 255) / 256);
-    lc.blockDim = dim3(256);
-    lc.stream = cfg.stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    lc.attrs = attr;
-    lc.numAttrs = opt(kOptPdl) ? 1 : 0;
-    if (cudaLaunchKernelEx(&lc, xquant_kernel, c.ph[0], p.M, c.vr, g_total, ws + xq_off,
-                           reinterpret_cast<float2*>(ws + xg_off)) != cudaSuccess) {
-      cudaGetLastError();
-      return UNIQL_ERR_CUDA;
-    }
+    const int rc = stream_setup(c, c.ph[0], p.M, g_total, ws, sw, cfg.stream);
+    if (rc != UNIQL_OK) return rc;
   }
   if (i8 && p.M > 4 && p.M <= 8) {
     // five to eight rows: one instance that can stream and share, whatever this launch does
@@ -1824,6 +1910,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
     }
     return rc;
   }
+  if (c.x_stream && p.M > 8) return launch_t<2, false, 4, 1, true>(p, c, smem, cfg.stream);   // nine to sixteen rows, one launch
   if (c.x_stream) return launch_t<1, false, 1, 1, true>(p, c, smem, cfg.stream);      // (M <= 4: rows too long to stage)
   if (i8 && c.x_cluster) {                                                           // (M <= 4: forced only)
     const int rc = launch_t<1, false, 1, 1, false, true>(p, c, smem, cfg.stream);
@@ -1891,7 +1978,14 @@ int launch_mlp_phases(const MlpDecode& d, int first, int count, const LaunchCfg&
     const int gr = copy_granule((ph == 0 ? d.hidden : d.inter) / kGroup);
     if (gr < gran) gran = gr;
   }
-  const size_t smem = plan_split(&c, d.M, g_max, gran, true);
+  // (nine to sixteen rows: the gate|up launch on its own, activations streamed through the ring)
+  const bool stream = count == 1 && first == 0 && d.M > 8 && opt(kOptDecodeSplitBatch) == 2 && opt(kOptDecodeXstream) != 0;
+  size_t smem = stream ? plan_stream(&c, d.M, g_max, gran) : 0;
+  c.x_stream = smem != 0;
+  if (!smem) {
+    c.stage_bytes = STAGE_BYTES;
+    smem = plan_split(&c, d.M, g_max, gran, true);
+  }
   if (!smem) return UNIQL_ERR_UNSUPPORTED;
   if (count > 1 && (c.n_kp != 1 || d.M > 8)) return UNIQL_ERR_UNSUPPORTED;
   // the down projection on its own: narrow tiles under the same rule as any plain launch
@@ -1945,7 +2039,9 @@ int launch_mlp_phases(const MlpDecode& d, int first, int count, const LaunchCfg&
     const int sl = slots_needed(c.ph[i].tiles, c.ph[i].g_total, c.gp, c.n_rp, c.cgz);
     if (sl > c.max_slots) c.max_slots = sl;
   }
-  const size_t need = (size_t)kWsHeader + (size_t)tiles * c.max_slots * d.M * RB * 4;
+  size_t need = (size_t)kWsHeader + (size_t)tiles * c.max_slots * d.M * RB * 4;
+  StreamWs sw;
+  if (c.x_stream) need = stream_need(c, d.M, c.ph[0].g_total, need, &sw);
   if (!cfg.workspace || cfg.ws_bytes < need) return UNIQL_ERR_WORKSPACE;
   unsigned char* ws = reinterpret_cast<unsigned char*>(cfg.workspace);
   c.counters = reinterpret_cast<int*>(ws);
@@ -1955,6 +2051,11 @@ int launch_mlp_phases(const MlpDecode& d, int first, int count, const LaunchCfg&
   {
     const int shift = opt(kOptWaitShift);
     c.grid_wait_limit = shift > 0 ? (shift >= 21 ? 1 : kGridWaitLimit >> shift) : kGridWaitLimit;
+  }
+  if (c.x_stream) {
+    const int rc = stream_setup(c, c.ph[0], d.M, c.ph[0].g_total, ws, sw, cfg.stream);
+    if (rc != UNIQL_OK) return rc;
+    return launch_t<2, false, 4, 1, true>(p, c, smem, cfg.stream);
   }
   if (count > 1) {
     if (d.M <= 4) return launch_t<1, false, 1, 2>(p, c, smem, cfg.stream);

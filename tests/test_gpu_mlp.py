@@ -110,14 +110,19 @@ def test_typed_entry_point(B, small, M, dtype):
     check_output(y[:, :hidden], y_ref, dtype, TOL_Y if dtype == "f16" else 2e-3, "y %s M=%d" % (dtype, M))
 
 
+@pytest.mark.parametrize("mode", [2, 1, 0])
 @pytest.mark.parametrize("M", [9, 11, 16])
-def test_batches_above_eight(B, small, M):
+def test_batches_above_eight(B, small, M, mode):
+    """Nine to sixteen rows: one pass with streamed activations (2, the default), two passes over half the batch (1),
+    one pass with staged activations (0)."""
+    B.set_option("decode_split_batch", mode)
     _, qs, ds = small
     x = synth.draw_x(np.random.default_rng(200 + M), M, 512, "f16")
     for fuse in (-1, 0):
-        h, h_ref, y, y_ref = run_mlp(B, qs, ds, x, 872, fuse)
-        check_output(h, h_ref, "f16", TOL_H, "h M=%d" % M)
-        check_output(y, y_ref, "f16", TOL_Y, "y M=%d" % M)
+        for k_int in (872, 1024, 8):
+            h, h_ref, y, y_ref = run_mlp(B, qs, ds, x, k_int, fuse, pad=8)
+            check_output(h, h_ref, "f16", TOL_H, "h M=%d mode %d k_int %d" % (M, mode, k_int))
+            check_output(y, y_ref, "f16", TOL_Y, "y M=%d mode %d k_int %d" % (M, mode, k_int))
     with pytest.raises(RuntimeError):                      # one launch holds at most eight batch rows
         run_mlp(B, qs, ds, x, 872, 1)
 

@@ -204,6 +204,40 @@ def test_streamed_activations(B, stream, rp, M):
     assert B.workspace_status() == 0
 
 
+@pytest.mark.parametrize("mode", [2, 1, 0])
+@pytest.mark.parametrize("rp", [0, 1, 7])
+@pytest.mark.parametrize("M", [9, 12, 15, 16])
+def test_batches_of_nine_to_sixteen(B, mode, rp, M):
+    """Nine to sixteen rows in one launch with the quantised activations carried through the ring (2, the default),
+    as two launches over half the batch (1) and as one launch with staged activations (0): plain, ragged and
+    per-head shapes, bias, the rotary epilogue, more chunks than ring positions and fewer."""
+    B.set_option("decode_split_batch", mode)
+    if rp:
+        B.set_option("decode_rp", rp)
+    B.set_path(B.PATH_DECODE)
+    rng = np.random.default_rng(180 + M)
+    for (N, K, k_in, k_out) in [(200, 2304, 2304, 200), (200, 2304, 1096, 77), (96, 256, 256, 96), (70, 3328, 3072, 33),
+                                (330, 8192, 8192, 330)]:
+        qw = synth.draw_qweight(rng, N, K)
+        dw = dev_weight(qw)
+        bias = synth.to_dtype_values(rng.standard_normal(N).astype(np.float32), "f16")
+        x = synth.draw_x(rng, M, k_in, "f16")
+        y, ref = run_ex(B, qw, dw, x, "f16", None, k_in, None, k_out, bias=bias, ldy_pad=3)
+        check_output(y, ref, "f16", TIGHT, "mode=%d rp=%d M=%d %s" % (mode, rp, M, (N, K, k_in, k_out)))
+        y2, _ = run_ex(B, qw, dw, x, "f16", None, k_in, None, k_out, bias=bias, ldy_pad=3)
+        assert torch.equal(y, y2), "run-to-run results differ"
+    qw = synth.draw_qweight(rng, 512, 1024)
+    dw = dev_weight(qw)
+    for keep in (128, 96, 40):
+        in_map = synth.map_per_head(8, 128, keep)
+        x = synth.draw_x(rng, M, synth.map_size(in_map), "f16")
+        y, ref = run_ex(B, qw, dw, x, "f16", in_map, 0, synth.map_per_head(4, 128, 108), 0)
+        check_output(y, ref, "f16", TIGHT, "mode=%d per-head keep %d M=%d" % (mode, keep, M))
+    for (g, ref) in run_rope(B, rng, M, 512, 6, 2, 128, 96, 500000.0, "f16", bias=True, v_keep=104):
+        check_output(g, ref, "f16", TIGHT, "mode=%d q/k/v M=%d" % (mode, M))
+    assert B.workspace_status() == 0
+
+
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
 @pytest.mark.parametrize("M", [1, 7, 16, 17, 70])
 def test_tiny_and_ragged_shapes(B, M, dtype):
