@@ -1766,10 +1766,12 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
   // Streamed activations for rows too long to stage whole beside the ring (which would otherwise split the input
   // channels over several groups of blocks and hand every tile over); UNIQL_DECODE_XSTREAM=0/1 forces.  Where the
   // staged copy fits the quantising kernel in front costs more than the staging it saves (measured 3.5 us), and
-  // inside a sequence of launches it only pays for itself at eight rows (Llama-3-8B MLP: 51.7 against 53.9 us
-  // at M = 8; 46.6 against 43.0 us at M = 5).  Nine to sixteen rows are always streamed: their staged copy never
-  // fits beside a ring of more than two positions (Llama-3-8B MLP at M = 16: 55 us in one pass, 82 us as two
-  // launches of eight rows, 145 us with the input channels split over two groups of blocks).
+  // inside a sequence of launches it only pays for itself from five rows on, where the staged copy would split
+  // the input channels (Llama-3-8B gate|up + down at M = 5 / 6 / 7: 39.7 / 40.9 / 43.0 against 40.6 / 42.8 / 49.2 us;
+  // at M <= 4, and wherever the staged copy fits whole, staging is faster).  Nine to sixteen rows are always
+  // streamed: their staged copy never fits beside a ring of more than two positions (Llama-3-8B MLP at M = 16:
+  // 55 us in one pass, 82 us as two launches of eight rows, 145 us with the input channels split over two groups
+  // of blocks).
   size_t smem = 0;
   c.stage_bytes = STAGE_BYTES;
   {
@@ -1783,7 +1785,7 @@ int launch_decode(const Params& p, const LaunchCfg& cfg) {
     } else if (i8 && force != 0) {
       DecodeCfg t = c;
       const size_t s0 = plan_split(&t, p.M, g_total, gran, true);
-      if (force == 1 || !s0 || (t.n_kp > 1 && p.M >= 8)) {
+      if (force == 1 || !s0 || (t.n_kp > 1 && p.M >= 5)) {
         smem = plan_stream(&c, p.M, g_total, gran);
         c.x_stream = smem != 0;
         if (!smem) c.stage_bytes = STAGE_BYTES;
