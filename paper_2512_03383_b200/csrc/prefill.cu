@@ -45,10 +45,12 @@ namespace {
 constexpr int BMW = 128;            // weight rows per tile (MMA M)
 constexpr int BK = 64;              // k per stage: 128 bytes of fp16 / bf16, one swizzle row
 constexpr int MAXBN = 256;          // tokens per tile (MMA N), at most
-constexpr int PSTAGES = 4;
+constexpr int PSTAGES = 4;                   // ring of de-quantised weight stages (one k-block each)
+constexpr int BSLOTS = 4;                    // ring of activation boxes (one k-block of MAXBN tokens each)
 constexpr int A_BYTES = BMW * BK * 2;        // 16 KB
 constexpr int B_BYTES = MAXBN * BK * 2;      // 32 KB
-constexpr int PSTAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int RING_BYTES = PSTAGES * A_BYTES + BSLOTS * B_BYTES;
+constexpr int B_RING = PSTAGES * A_BYTES;    // the activation boxes follow the weight stages
 constexpr int EPI_TOK = 32;                  // tokens per epilogue pass
 constexpr int NWARPS = 24;
 constexpr int PTH = NWARPS * 32;
@@ -59,7 +61,8 @@ constexpr int kMaxPJobs = kMaxJobs;
 
 struct PrefillCfg {
   CUtensorMap xmap;          // activations: (k, token), box 64 x BN, 128-byte swizzle
-  int bn;                    // tokens per tile: 64, 128 or 256
+  int bn;                    // tokens per MMA and activation box: 64, 128 or 256
+  int nh;                    // boxes per tile: 2 when the tile takes both accumulators (512 tokens), else 1
   int n_ttiles;              // token tiles
   int wtile_begin[kMaxPJobs + 1];   // first weight tile of each job
   int n_tiles;               // weight tiles (all jobs) x token tiles
@@ -327,18 +330,22 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
   const uint32_t raw = (uint32_t)__cvta_generic_to_shared(psmem_raw);
   const uint32_t sbase = (raw + 1023u) & ~1023u;           // swizzled tiles need 1024-byte alignment
   unsigned char* smem = psmem_raw + (sbase - raw);
-  const uint32_t bars = sbase + PSTAGES * PSTAGE_BYTES;
-  const uint32_t full_a = bars, full_b = bars + 8 * PSTAGES, empty = bars + 16 * PSTAGES;
-  const uint32_t acc_full = bars + 24 * PSTAGES, acc_empty = acc_full + 16, epi_bar = acc_full + 32;
-  unsigned char* misc = smem + PSTAGES * PSTAGE_BYTES + 24 * PSTAGES + 40;
+  const uint32_t bars = sbase + RING_BYTES;
+  const uint32_t full_a = bars, empty_a = bars + 8 * PSTAGES;
+  const uint32_t full_b = bars + 16 * PSTAGES, empty_b = full_b + 8 * BSLOTS;
+  const uint32_t acc_full = full_b + 16 * BSLOTS, acc_empty = acc_full + 16, epi_bar = acc_full + 32;
+  unsigned char* misc = smem + RING_BYTES + 16 * PSTAGES + 16 * BSLOTS + 40;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
 
   if (tid == 0) {
     for (int s = 0; s < PSTAGES; ++s) {
       pmbar_init(full_a + 8 * s, DQ_WARPS);
+      pmbar_init(empty_a + 8 * s, 1);
+    }
+    for (int s = 0; s < BSLOTS; ++s) {
       pmbar_init(full_b + 8 * s, 1);
-      pmbar_init(empty + 8 * s, 1);
+      pmbar_init(empty_b + 8 * s, 1);
     }
     for (int b = 0; b < 2; ++b) { pmbar_init(acc_full + 8 * b, 1); pmbar_init(acc_empty + 8 * b, 4); }
     pmbar_init(epi_bar, 4);
@@ -360,46 +367,59 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
   if (warp == 0) {
     // ===================================================================== activations by TMA
     if (lane == 0) {
-      int s = 0; uint32_t par = 1; int it = 0;
+      int s = 0; uint32_t par = 1; int jb = 0;             // box slot, parity of its previous use, boxes so far
       SegIter si; si.init(c, blockIdx.x, gridDim.x);
       Seg sg;
       while (!failed && si.next(sg)) {
         const int tt = sg.tile % c.n_ttiles;
-        for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
-          if (it >= PSTAGES && !pmbar_wait(empty + 8 * s, par, abort_flag, true)) { failed = true; break; }
-          const uint32_t fb = full_b + 8 * s;
-          pmbar_expect_tx(fb, (uint32_t)(c.bn * BK * 2));
-          tma_box2(sbase + s * PSTAGE_BYTES + A_BYTES, &c.xmap, HEADS ? kblock_of(c, kb).xcol : kb * BK, tt * c.bn, fb);
-          if (++s == PSTAGES) { s = 0; par ^= 1; }
+        for (int kb = sg.kb0; kb < sg.kb1 && !failed; ++kb) {
+          const int xcol = HEADS ? kblock_of(c, kb).xcol : kb * BK;
+          for (int h = 0; h < c.nh; ++h, ++jb) {
+            if (jb >= BSLOTS && !pmbar_wait(empty_b + 8 * s, par, abort_flag, true)) { failed = true; break; }
+            const uint32_t fb = full_b + 8 * s;
+            pmbar_expect_tx(fb, (uint32_t)(c.bn * BK * 2));
+            // (a box that starts at or beyond the last token is all zeros: the tensor map ends at M)
+            tma_box2(sbase + B_RING + s * B_BYTES, &c.xmap, xcol, (tt * c.nh + h) * c.bn, fb);
+            if (++s == BSLOTS) { s = 0; par ^= 1; }
+          }
         }
       }
     }
   } else if (warp == 1) {
     // ===================================================================== MMA issue
     if (lane == 0) {
-      int s = 0; uint32_t par = 0; int tcount = 0;
+      int s = 0; uint32_t par = 0; int tcount = 0;         // weight stage and its parity
+      int sb = 0; uint32_t parb = 0;                       // activation box slot and its parity
       SegIter si; si.init(c, blockIdx.x, gridDim.x);
       Seg sg;
       for (; !failed && si.next(sg); ++tcount) {
-        const int buf = tcount & 1;
-        if (tcount >= 2 && !pmbar_wait(acc_empty + 8 * buf, ((tcount >> 1) - 1) & 1, abort_flag)) { failed = true; break; }
-        tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MAXBN);
-        for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
-          // (bf16: the de-quantisers waited for the activation tile themselves and converted it)
-          if (!pmbar_wait(full_a + 8 * s, par, abort_flag) ||
-              (!CONV && !pmbar_wait(full_b + 8 * s, par, abort_flag))) { failed = true; break; }
-          tc_fence_after();
-          const uint64_t adesc = smem_desc_sw128(sbase + s * PSTAGE_BYTES);
-          const uint64_t bdesc = smem_desc_sw128(sbase + s * PSTAGE_BYTES + A_BYTES);
+        // A tile of one box alternates between the two accumulators; a tile of two boxes holds both: the
+        // de-quantised weight stage then serves 512 tokens, and the accumulator of the first 256 is drained by
+        // the epilogue while the MMAs of the next tile already run on ... once it is free again (per-accumulator waits).
+        const int acc0 = c.nh == 2 ? 0 : (tcount & 1);
+        const int au = c.nh == 2 ? tcount : (tcount >> 1);   // earlier tiles that used this tile's accumulator(s)
+        for (int kb = sg.kb0; kb < sg.kb1 && !failed; ++kb) {
+          if (!pmbar_wait(full_a + 8 * s, par, abort_flag)) { failed = true; break; }
+          const uint64_t adesc = smem_desc_sw128(sbase + s * A_BYTES);
+          for (int h = 0; h < c.nh; ++h) {
+            if (kb == sg.kb0 && au >= 1 && !pmbar_wait(acc_empty + 8 * (acc0 + h), (au - 1) & 1, abort_flag)) { failed = true; break; }
+            // (bf16: the de-quantisers waited for the activation box themselves and converted it)
+            if (!CONV && !pmbar_wait(full_b + 8 * sb, parb, abort_flag)) { failed = true; break; }
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)((acc0 + h) * MAXBN);
+            const uint64_t bdesc = smem_desc_sw128(sbase + B_RING + sb * B_BYTES);
 #pragma unroll
-          for (int k16 = 0; k16 < BK / 16; ++k16)       // 32 bytes along K per MMA: +2 in the address field
-            umma_f16(d_tmem, adesc + 2 * k16, bdesc + 2 * k16, c.idesc, (kb > sg.kb0 || k16 > 0) ? 1u : 0u);
-          umma_commit(empty + 8 * s);                   // the stage is free once these MMAs have read it
+            for (int k16 = 0; k16 < BK / 16; ++k16)     // 32 bytes along K per MMA: +2 in the address field
+              umma_f16(d_tmem, adesc + 2 * k16, bdesc + 2 * k16, c.idesc, (kb > sg.kb0 || k16 > 0) ? 1u : 0u);
+            umma_commit(empty_b + 8 * sb);              // the box is free once these MMAs have read it
+            if (++sb == BSLOTS) { sb = 0; parb ^= 1; }
+          }
+          if (failed) break;
+          umma_commit(empty_a + 8 * s);                 // ... and the weight stage after the last of them
           if (++s == PSTAGES) { s = 0; par ^= 1; }
         }
         if (failed) break;
-        umma_commit(acc_full + 8 * buf);
+        for (int h = 0; h < c.nh; ++h) umma_commit(acc_full + 8 * (acc0 + h));
       }
     }
   } else if (warp >= DQ_WARP0) {
@@ -452,8 +472,8 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         uint4 q2 = make_uint4(0, 0, 0, 0);
         __half s2 = s1, z2 = z1;
         if (live && kb + 4 < sg.kb1) fetch(kb + 4, q2, s2, z2);
-        if (it >= PSTAGES && !pmbar_wait(empty + 8 * s, (use - 1) & 1, abort_flag)) { failed = true; break; }
-        const uint32_t a_st = sbase + s * PSTAGE_BYTES + row_off;
+        if (it >= PSTAGES && !pmbar_wait(empty_a + 8 * s, (use - 1) & 1, abort_flag)) { failed = true; break; }
+        const uint32_t a_st = sbase + s * A_BYTES + row_off;
         const __half2 sh2 = __half2half2(s0);
         const __half2 cz2 = __float2half2_rn((8.f - __half2float(z0)) * __half2float(s0));
         const uint32_t qw[4] = {q0.x, q0.y, q0.z, q0.w};
@@ -467,14 +487,19 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         if constexpr (CONV) {
           // bf16 activations: the tensor cores run on fp16 (8 more mantissa bits for the weights than bf16
           // would leave them); the activation tile that TMA delivered is converted in place
-          if (!pmbar_wait(full_b + 8 * s, use & 1, abort_flag)) { failed = true; break; }
-          const uint32_t b_st = sbase + s * PSTAGE_BYTES + A_BYTES;
-          for (int ci = dt; ci < c.bn * 8; ci += DQ_WARPS * 32) {
-            uint32_t v0, v1, v2, v3;
-            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(b_st + ci * 16));
-            v0 = bf16x2_to_f16x2(v0); v1 = bf16x2_to_f16x2(v1); v2 = bf16x2_to_f16x2(v2); v3 = bf16x2_to_f16x2(v3);
-            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(b_st + ci * 16), "r"(v0), "r"(v1), "r"(v2), "r"(v3) : "memory");
+          for (int h = 0; h < c.nh && !failed; ++h) {
+            const int jb = it * c.nh + h;                  // the k-block's boxes in the order the producer issued them
+            const int sb = jb % BSLOTS;
+            if (!pmbar_wait(full_b + 8 * sb, (uint32_t)(jb / BSLOTS) & 1, abort_flag)) { failed = true; break; }
+            const uint32_t b_st = sbase + B_RING + sb * B_BYTES;
+            for (int ci = dt; ci < c.bn * 8; ci += DQ_WARPS * 32) {
+              uint32_t v0, v1, v2, v3;
+              asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(b_st + ci * 16));
+              v0 = bf16x2_to_f16x2(v0); v1 = bf16x2_to_f16x2(v1); v2 = bf16x2_to_f16x2(v2); v3 = bf16x2_to_f16x2(v3);
+              asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(b_st + ci * 16), "r"(v0), "r"(v1), "r"(v2), "r"(v3) : "memory");
+            }
           }
+          if (failed) break;
         }
         fence_async_smem();            // generic-proxy writes must be visible to the tensor core (async proxy)
         __syncwarp();
@@ -500,7 +525,9 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
     SegIter si; si.init(c, blockIdx.x, gridDim.x);
     Seg sg;
     for (; !failed && si.next(sg); ++tcount) {
-      const int buf = tcount & 1;
+      const int acc0 = c.nh == 2 ? 0 : (tcount & 1);     // as in the MMA warp
+      const int au = c.nh == 2 ? tcount : (tcount >> 1);
+      const int ntok = c.bn * c.nh;                      // tokens of the tile
       const int t = sg.tile;
       const int wt = t / c.n_ttiles, tt = t - wt * c.n_ttiles;
       const int jn = job_of_wt(wt);
@@ -527,7 +554,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
       // bias, rotary embedding, rounding and store of 32 tokens of this row (all lanes of the warp call it)
       auto store_chunk = [&](int tok0, const auto& val) {
         constexpr int NV = (int)(sizeof(val) / sizeof(float));
-        const int m0 = tt * c.bn + tok0;
+        const int m0 = tt * ntok + tok0;
         if (rope) {
           // the even lane of a pair rotates the even tokens, the odd lane the odd ones: one exchange hands
           // each the other member's value of its token, and it stores both rotated members
@@ -615,42 +642,48 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
           }
         }
       };
-      if (!pmbar_wait(acc_full + 8 * buf, (tcount >> 1) & 1, abort_flag)) { failed = true; break; }
+      for (int h = 0; h < c.nh && !failed; ++h)
+        if (!pmbar_wait(acc_full + 8 * (acc0 + h), au & 1, abort_flag)) failed = true;
+      if (failed) break;
       tc_fence_after();
-      const uint32_t t_acc = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * MAXBN);
+      // (the two accumulators are neighbours in tensor memory: a tile of two boxes is 512 consecutive columns)
+      const uint32_t t_acc = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc0 * MAXBN);
       const int row = 32 * q + lane;
+      // this warp is done with the accumulator that holds token chunk `ch` once that chunk was its last
+      auto release_after = [&](int ch) {
+        if (((ch + 1) * EPI_TOK) % c.bn != 0) return;
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) pmbar_arrive(acc_empty + 8 * (acc0 + (ch * EPI_TOK) / c.bn));
+      };
       if (sg.kb0 == 0 && sg.kb1 == c.n_kb) {
         // ---- the whole contraction of this tile ran here
-        for (int ch = 0; ch < c.bn / EPI_TOK; ++ch) {
+        for (int ch = 0; ch < ntok / EPI_TOK; ++ch) {
           uint32_t v[32];
           tmem_ld32(t_acc + (uint32_t)(ch * EPI_TOK), v);
           tmem_ld_wait();
+          release_after(ch);                             // (the values are in registers)
           float val[32];
 #pragma unroll
           for (int k = 0; k < 32; ++k) val[k] = __uint_as_float(v[k]);
           store_chunk(ch * EPI_TOK, val);
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) pmbar_arrive(acc_empty + 8 * buf);
       } else {
         // ---- a part of the contraction (stream-K): the fp32 partial tile is added (reductions done in L2, a
         //      warp covers 32 consecutive rows of a token) to the tile's accumulation buffer [token][row] in the
         //      workspace (zero at launch); the last of the tile's blocks to arrive reads the sum and finishes the tile
-        const size_t slot_f = (size_t)c.bn * BMW;
+        const size_t slot_f = (size_t)ntok * BMW;
         const int T0 = (c.n_tiles / (int)gridDim.x) * (int)gridDim.x;          // first left-over tile
         float* sum = c.partials + (size_t)(t - T0) * slot_f;
-        for (int ch = 0; ch < c.bn / EPI_TOK; ++ch) {
+        for (int ch = 0; ch < ntok / EPI_TOK; ++ch) {
           uint32_t v[32];
           tmem_ld32(t_acc + (uint32_t)(ch * EPI_TOK), v);
           tmem_ld_wait();
+          release_after(ch);                                   // the accumulator is free for the next segment
           float* dst = sum + (size_t)(ch * EPI_TOK) * BMW + row;
 #pragma unroll
           for (int k = 0; k < 32; ++k) atomicAdd(dst + (size_t)k * BMW, __uint_as_float(v[k]));
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) pmbar_arrive(acc_empty + 8 * buf);      // the accumulator is free for the next segment
         __threadfence();                                       // this thread's additions are done before ...
         if (!epi_sync()) { failed = true; break; }
         const long U = (long)(c.n_tiles - T0) * c.n_kb, Bn = (long)gridDim.x < U ? (long)gridDim.x : U;
@@ -668,11 +701,11 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
           float nxt[16];
 #pragma unroll
           for (int k = 0; k < 16; ++k) nxt[k] = __ldcg(src + (size_t)k * BMW);
-          for (int tk = 0; tk < c.bn; tk += 16) {
+          for (int tk = 0; tk < ntok; tk += 16) {
             float val[16];
 #pragma unroll
             for (int k = 0; k < 16; ++k) val[k] = nxt[k];
-            if (tk + 16 < c.bn) {
+            if (tk + 16 < ntok) {
               const float* nx = src + (size_t)(tk + 16) * BMW;
 #pragma unroll
               for (int k = 0; k < 16; ++k) nxt[k] = __ldcg(nx + (size_t)k * BMW);
@@ -729,7 +762,7 @@ int host_job_tiles(const JobDev& j) {
 
 template <typename T, bool CONV, bool HEADS>
 int launch_pth(const Params& p, const PrefillCfg& c, int grid, cudaStream_t stream) {
-  const size_t smem = 1024 + (size_t)PSTAGES * PSTAGE_BYTES + 512;
+  const size_t smem = 1024 + (size_t)RING_BYTES + 512;
   auto kern = prefill_kernel<T, CONV, HEADS>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return UNIQL_ERR_CUDA;
@@ -771,12 +804,10 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   PrefillCfg c;
   memset(&c, 0, sizeof(c));
   c.bn = p.M <= 64 ? 64 : (p.M <= 128 ? 128 : 256);
-  c.n_ttiles = (p.M + c.bn - 1) / c.bn;
   int wt = 0;
   for (int j = 0; j < p.n_jobs; ++j) { c.wtile_begin[j] = wt; wt += host_job_tiles(p.job[j]); }
   for (int j = p.n_jobs; j <= kMaxPJobs; ++j) c.wtile_begin[j] = wt;
-  c.n_tiles = wt * c.n_ttiles;
-  if (c.n_tiles < 1) return UNIQL_ERR_SHAPE;
+  if (wt < 1) return UNIQL_ERR_SHAPE;
   {
     const Fam& a = p.imap.fam[0];
     c.km_start = a.start / BK;
@@ -790,8 +821,6 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   c.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(c.bn >> 3) << 17) | ((uint32_t)(BMW >> 4) << 24);
   c.status = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(cfg.workspace) + decode_status_offset());
   const int sms = p_sm_count();
-  int grid = c.n_tiles < sms ? c.n_tiles : sms;
-  if (env_grid >= 1 && env_grid <= sms) grid = env_grid;          // tests: odd splits on small problems
   // workspace: [header: counters, status][fp16 copy of bf16 activations][stream-K partial tiles]
   size_t ws_used = (decode_workspace_header_bytes() + 255) & ~(size_t)255;
   c.counters = reinterpret_cast<int*>(cfg.workspace);
@@ -815,24 +844,57 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
       conv_in_kernel = true;
     }
   }
-  // stream-K for the tiles left over when whole tiles would leave SMs idle in their last round and the partial
+  // The shape of the work: tokens per tile (one accumulator, or both = 512 tokens, so that a de-quantised weight
+  // stage serves twice the tokens) and whether the tiles left over after the whole rounds are split along K.
+  // Stream-K serves the tiles left over when whole tiles would leave SMs idle in their last round and the partial
   // tiles fit in the workspace.  It pays when the k-blocks a block no longer waits for outweigh the hand-over:
-  // measured on B200, a k-block takes about 0.65 us, and the hand-over (zeroing the sums, the additions, the
+  // measured on B200, a k-block takes about 0.65 us (1.07 us on both accumulators: 1.65 times the time for twice
+  // the work), and the hand-over (zeroing the sums, the additions, the
   // read-back by the finishing block) about 14 us for tiles of 256 tokens when whole tiles follow and hide
-  // most of it, 28 us when every tile is split; both shrink with the tile's width.
+  // most of it, 28 us when every tile is split; both grow with the tile's width.
+  // (whole tiles that follow hide most of the hand-over: forcing the split on the Qwen2.5-7B q projection at
+  //  M = 2048 and on the Mamba2 in_proj at M = 1024 saved 5.7 and 5.3 us where this rule's saving was 17.7 and 19.7 us)
+  // Both tile widths are costed with these figures and the cheaper one runs: wide tiles win where they still fill
+  // the SMs (Qwen2.5-7B gate at M = 512..4096: 17-22 % faster), narrow ones where wide tiles would leave most SMs
+  // without a tile (q / o projections at M = 512) or push a few left-over tiles into a round of their own.
+  int g2 = sms;
+  if (env_grid >= 1 && env_grid <= sms) g2 = env_grid;            // tests: odd splits on small problems
+  struct Plan { int nh, ttiles, tiles, left; bool streamk; size_t sums; double us; };
+  auto plan_for = [&](int nh) {
+    Plan q;
+    q.nh = nh;
+    const int ntok = c.bn * nh;
+    q.ttiles = (p.M + ntok - 1) / ntok;
+    const long tiles = (long)wt * q.ttiles;
+    q.tiles = tiles <= (1 << 24) ? (int)tiles : (1 << 24);
+    q.left = q.tiles % g2;
+    const double kcost = nh == 2 ? 1.07 : 0.65;
+    const double share = (double)q.left * c.n_kb / g2;                 // k-blocks per block of the split tiles
+    const double hand_over = q.tiles < g2 ? 10.0 + 18.0 * ntok / 256.0 : 14.0 * ntok / 256.0;
+    const bool pays = ((double)c.n_kb - share) * kcost > hand_over;
+    q.sums = (size_t)q.left * ntok * BMW * 4;                          // one fp32 tile per left-over tile
+    const bool want = env_streamk >= 0 ? (env_streamk == 1) : (q.left != 0 && pays);
+    q.streamk = want && q.left != 0 && cfg.ws_bytes >= ws_used + q.sums && q.tiles <= (1 << 16);
+    q.us = q.streamk ? (double)q.tiles / g2 * c.n_kb * kcost + hand_over
+                     : (double)((q.tiles + g2 - 1) / g2) * c.n_kb * kcost;
+    return q;
+  };
+  Plan pl = plan_for(1);
   {
-    int g2 = sms;
-    if (env_grid >= 1 && env_grid <= sms) g2 = env_grid;
-    const int left = c.n_tiles % g2;
-    const double share = (double)left * c.n_kb / g2;                   // k-blocks per block of the split tiles
-    // (whole tiles that follow hide most of the hand-over: forcing the split on the Qwen2.5-7B q projection at
-    //  M = 2048 and on the Mamba2 in_proj at M = 1024 saved 5.7 and 5.3 us where this rule's saving was 17.7 and 19.7 us)
-    const double hand_over = c.n_tiles < g2 ? 10.0 + 18.0 * c.bn / 256.0 : 14.0 * c.bn / 256.0;
-    const bool pays = ((double)c.n_kb - share) * 0.65 > hand_over;
-    const size_t sums = (size_t)left * c.bn * BMW * 4;                 // one fp32 tile per left-over tile
-    const size_t need = ws_used + sums;
-    const bool want = env_streamk >= 0 ? (env_streamk == 1) : (left != 0 && pays);
-    if (want && left != 0 && cfg.ws_bytes >= need && c.n_tiles <= (1 << 16)) {
+    const int dual = opt(kOptPrefillDual);                          // -1: by cost, 0: never, 1: wherever M > 256
+    if (p.M > MAXBN && dual != 0) {
+      const Plan p2 = plan_for(2);
+      if (dual == 1 || p2.us < pl.us) pl = p2;
+    }
+  }
+  c.nh = pl.nh;
+  c.n_ttiles = pl.ttiles;
+  c.n_tiles = pl.tiles;
+  if ((long)wt * pl.ttiles > (1 << 24)) return UNIQL_ERR_SHAPE;
+  int grid = c.n_tiles < g2 ? c.n_tiles : g2;
+  {
+    const size_t sums = pl.sums;
+    if (pl.streamk) {
       c.streamk = 1;
       c.partials = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(cfg.workspace) + ws_used);
       grid = g2;

@@ -149,6 +149,7 @@ def test_prefill_stream_k(B, monkeypatch, grid, dtype):
     B.set_path(B.PATH_PREFILL)
     B.set_option("prefill_streamk", 1)
     B.set_option("prefill_grid", grid)
+    B.set_option("prefill_dual", 0)                              # tiles of 256 tokens (the counts below assume them)
     rng = np.random.default_rng(900 + grid)
     qw = synth.draw_qweight(rng, 300, 1024)
     dw = dev_weight(qw)
@@ -162,6 +163,50 @@ def test_prefill_stream_k(B, monkeypatch, grid, dtype):
         check_output(y2, ref, dtype, TOL[dtype], "stream-K grid %d, second run" % grid)
     for (g, r) in run_rope(B, rng, 200, 512, 6, 2, 128, 84, 5e5, dtype):
         check_output(g, r, dtype, TOL[dtype], "stream-K rope grid %d" % grid)
+    assert B.workspace_status() == 0
+
+
+@pytest.mark.parametrize("grid", [0, 1, 2, 5])
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("M", [257, 300, 513, 700, 1100])
+def test_prefill_tiles_on_both_accumulators(B, M, dtype, grid):
+    """Above 256 tokens a tile may take both accumulators (512 tokens: two activation boxes per de-quantised weight
+    stage).  Forced on, against the oracle and against tiles of 256 tokens: token counts that end inside the first
+    box of a tile, inside the second and on a tile boundary; one block running many tiles in a row (accumulators
+    re-used tile after tile), whole tiles and tiles split along K; bias, ragged rows, the rotary epilogue,
+    per-head input maps, and bf16 activations converted inside the kernel."""
+    B.set_path(B.PATH_PREFILL)
+    if grid:
+        B.set_option("prefill_grid", grid)
+    B.set_option("prefill_streamk", 1 if grid == 5 else 0)
+    rng = np.random.default_rng(990 + M)
+    qw = synth.draw_qweight(rng, 300, 1024)
+    dw = dev_weight(qw)
+    bias = synth.to_dtype_values(rng.standard_normal(300).astype(np.float32), dtype)
+    outs = {}
+    for dual in (1, 0):
+        B.set_option("prefill_dual", dual)
+        for (k_in, k_out) in [(1024, 300), (652, 132)]:
+            x = synth.draw_x(np.random.default_rng(M + k_in), M, k_in, dtype)
+            y, ref = run_ex(B, qw, dw, x, dtype, None, k_in, None, k_out, bias=bias, ldx_pad=8 - k_in % 8 if k_in % 8 else 0,
+                            ldy_pad=3)
+            check_output(y, ref, dtype, TOL[dtype], "dual=%d M=%d %s k=(%d,%d) grid %d" % (dual, M, dtype, k_in, k_out, grid))
+            outs[(dual, k_in)] = y.clone()
+    if grid != 5:        # whole tiles: one block sums a tile's k-blocks in the same order, whatever the tile's width
+        for k_in in (1024, 652):
+            assert torch.equal(outs[(1, k_in)], outs[(0, k_in)]), "tile width changed the result"
+    B.set_option("prefill_dual", 1)
+    im = synth.map_per_head(8, 128, 104)
+    x = synth.draw_x(rng, M, synth.map_size(im), dtype)
+    y, ref = run_ex(B, qw, dw, x, dtype, im, 0, None, 200, ldx_pad=8)
+    check_output(y, ref, dtype, TOL[dtype], "dual per-head input map M=%d" % M)
+    for (g, r) in run_rope(B, rng, M, 512, 6, 2, 128, 84, 5e5, dtype, bias=True):
+        check_output(g, r, dtype, TOL[dtype], "dual rope M=%d grid %d" % (M, grid))
+    if dtype == "bf16":
+        B.set_option("prefill_convert", 1)
+        x = synth.draw_x(rng, M, 652, dtype)
+        y, ref = run_ex(B, qw, dw, x, dtype, None, 652, None, 256, ldx_pad=4)
+        check_output(y, ref, dtype, TOL[dtype], "dual, converted in kernel, M=%d" % M)
     assert B.workspace_status() == 0
 
 
