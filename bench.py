@@ -512,6 +512,47 @@ def tables(B, torch, work, reps=20):
     torch.cuda.empty_cache()
     out["mamba2_27b_fp16"] = mamba
 
+    # ---- Hybrid model (the Mamba2 mixer of a Bamba-v2-9B-shaped layer: d_model 4096, d_inner 8192, 128 SSM heads of
+    #      64 channels, one group of 128 states; shapes from the public model card, synthetic weights), fp16:
+    #      in_proj with z / x pruned per SSM head AND the state dimension D_s pruned (the leading rows of B and of C:
+    #      Section 3.2, SSM paragraph), out_proj with its input columns pruned per head.  Its attention and MLP
+    #      blocks have the Llama-3-8B shapes of the tables above.
+    d_model, d_inner, d_state, headdim, nheads = 4096, 8192, 128, 64, 128
+    rows_in = 2 * d_inner + 2 * d_state + nheads
+    n_cp = 3                                               # 3 x 53 MB > L2
+    hw = [(dev_qweight(torch, rows_in, d_model, 400 + c), dev_qweight(torch, d_model, d_inner, 420 + c)) for c in range(n_cp)]
+    hybrid = {}
+    for M in (1, 1024):
+        x = dev_x(torch, M, d_model, f16, 13)
+        rows = {}
+        for (keep, skeep) in ((64, 128), (56, 112), (48, 96), (40, 80)):
+            om = synth.map_mamba_in_proj(d_inner, headdim, keep, d_state, 1, nheads, state_keep=skeep)
+            im = synth.map_per_head(nheads, headdim, keep)
+            n_out = synth.map_size(om)
+            yin = torch.zeros((M, n_out), dtype=f16, device="cuda")
+            xo = dev_x(torch, M, nheads * keep, f16, 14)
+            yo = torch.zeros((M, d_model), dtype=f16, device="cuda")
+
+            def inp(i):
+                w = hw[i][0]
+                B.qlinear_ex(x, d_model, w[0], w[1], w[2], None, M, d_model, rows_in, None, d_model, om, 0, yin, n_out)
+
+            def outp(i):
+                w = hw[i][1]
+                B.qlinear_ex(xo, nheads * keep, w[0], w[1], w[2], None, M, d_inner, d_model, im, 0, None, d_model, yo, d_model)
+            w_in, w_out = n_out * d_model, d_model * nheads * keep
+            key = "hd%d_ds%d" % (keep, skeep)
+            if M == 1:
+                rows[key] = {"in_proj": rec_hbm(time_rotating(torch, inp, n_cp, reps), w_in, hbm, M),
+                             "out_proj": rec_hbm(time_rotating(torch, outp, n_cp, reps), w_out, hbm, M)}
+            else:
+                rows[key] = {"in_proj": rec_tc(time_plain(torch, inp, 10), 2.0 * M * w_in, tf, tf_sus, M),
+                             "out_proj": rec_tc(time_plain(torch, outp, 10), 2.0 * M * w_out, tf, tf_sus, M)}
+        hybrid["M%d" % M] = rows
+    del hw
+    torch.cuda.empty_cache()
+    out["hybrid_bamba_v2_9b_mixer_fp16"] = hybrid
+
     # derived per-model decode figure (layer counts are the public model-card values, not the paper's): the MLP
     # and attention-projection launches of one Llama-3-8B layer at M = 1, keep 1.0 and 0.65, times 32 layers
     try:
