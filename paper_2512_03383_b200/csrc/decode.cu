@@ -1123,7 +1123,7 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
       if (gi < Gk) {
         const uint32_t st = sbase + (uint32_t)s * (xs_on ? (uint32_t)c.stage_bytes : (uint32_t)STAGE_BYTES);
         const uint32_t wp = st + wl_off, sp = st + sl_off;
-        if constexpr (NT <= 2) {
+        if constexpr (NT <= 1) {
         uint4 wa[2], wb[2];
         wa[0] = lds128<0>(wp);
         wb[0] = lds128<8 * 128>(wp);
@@ -1176,10 +1176,12 @@ __global__ void __launch_bounds__(NTH, 1) decode_kernel(const __grid_constant__ 
           }
         }
         } else {
-          // Four column tiles (nine to sixteen rows): the two halves of the warp's 32 weight rows one after the
-          // other; the nibbles of a half are split once (16 words) and each column tile then runs its chain of four
-          // MMAs and its scaling on its own, so that 4 accumulators and the activation bytes of one tile are live
-          // at a time (all four tiles at once need more registers than a thread of this block can have).
+          // Two or four column tiles (five to sixteen rows): the two halves of the warp's 32 weight rows one after
+          // the other; the nibbles of a half are split once (16 words) and each column tile then runs its chain of
+          // four MMAs and its scaling on its own, so that 4 accumulators and the activation bytes of one tile are
+          // live at a time (all four tiles at once need more registers than a thread of this block can have:
+          // 284 bytes of spills inside this loop; with two tiles this order measured 3-4 % faster than all
+          // accumulators at once, with one tile slightly slower).
           const uint32_t xga = xs_on ? st + xsg : xgaddr8 + (uint32_t)(gi * 8 * MT * 8);
 #pragma unroll
           for (int sub = 0; sub < 2; ++sub) {
