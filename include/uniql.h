@@ -165,7 +165,7 @@ int uniql_embed_rows(const uint8_t* packed, const void* scales, const void* zero
  * to bf16 would alone spend the 2e-3 error budget; bf16 magnitudes beyond 65504 saturate.  When the
  * workspace is too small for the copy the tiles are converted inside the kernel (same result, slower).
  * It also carries the fp32 sums of output tiles whose contraction is split over several thread blocks
- * (at most 147 tiles of 128 rows x 256 tokens): the parts of such a tile are added in the order in
+ * (at most 147 tiles of 128 rows x 256 or 512 tokens): the parts of such a tile are added in the order in
  * which the blocks finish, so with more than two blocks on a tile the last bit of an fp32 sum, and
  * rarely of the rounded output, can differ between two runs on the same input; uniql_set_option("prefill_streamk", 0)
  * switches the splitting off.  Activations below fp16's range are affected too: bf16 values under 2^-24 become zero
