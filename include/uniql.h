@@ -126,6 +126,7 @@ int uniql_set_path(int path);
  *                      results of that kernel reproducible bit for bit (every tile is summed by one block).
  *   "prefill_dual"     -1 / 0: above 256 tokens a tile of the tensor-core kernel takes both accumulators (512
  *                      tokens per de-quantised weight stage); 0 keeps tiles of 256 tokens
+ *   "prefill_helpers"  1 / 0: the de-quantiser warps of the tensor-core kernel share the epilogue of a block's last tile
  *   "decode_split_batch" batches of 9..16 rows: 2 (default) one launch that streams the quantised activations
  *                      beside the weights, where the integer path applies, else two launches over half the batch;
  *                      1 always two launches; 0 always one launch with the activations staged whole

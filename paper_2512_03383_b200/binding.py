@@ -90,7 +90,7 @@ _lib.uniql_noalloc_status.argtypes = [ctypes.POINTER(_i)]
 
 OPTION_DEFAULTS = {"pdl": 1, "decode_kp": 0, "decode_rp": 0, "decode_stages": 0, "decode_narrow": -1,
                    "decode_xstream": -1, "decode_xcluster": -1, "decode_i8": 1, "decode_split_batch": 2,
-                   "prefill_grid": 0, "prefill_convert": 0, "prefill_streamk": -1, "prefill_dual": -1, "gemv_first": 0, "gemv_depth": 0,
+                   "prefill_grid": 0, "prefill_convert": 0, "prefill_streamk": -1, "prefill_dual": -1, "prefill_helpers": 1, "gemv_first": 0, "gemv_depth": 0,
                    "wait_shift": 0}
 
 

@@ -32,6 +32,7 @@ const OptDesc kOpts[kOptCount] = {
     {"prefill_convert", "UNIQL_PREFILL_CONVERT_IN_KERNEL", 0},   // 1: bf16 tiles converted inside the kernel
     {"prefill_streamk", "UNIQL_PREFILL_STREAMK", -1},   // split tiles: -1 automatic, 0 never (reproducible sums), 1 always
     {"prefill_dual", "UNIQL_PREFILL_DUAL", -1},         // tiles of 512 tokens on both accumulators: -1 where M > 256, 0 never
+    {"prefill_helpers", "UNIQL_PREFILL_HELPERS", 1},    // de-quantiser warps share the epilogue of a block's last tile
     {"gemv_first", "UNIQL_GEMV_FIRST", 0},              // 1: the streaming kernel wherever it applies (M <= 4)
     {"gemv_depth", "UNIQL_GEMV_DEPTH", 0},              // ring slots per warp of the streaming kernel (0: automatic)
     {"wait_shift", "UNIQL_WAIT_SHIFT", 0},              // bounded device waits: limits divided by 2^shift (tests)

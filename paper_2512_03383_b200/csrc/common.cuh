@@ -142,7 +142,7 @@ __device__ inline void rope_cos_sin(int pos, unsigned long long turn, float& c, 
 // Tuning / test options of the process (uniql_set_option); every launch reads them from one table of atomics.
 enum OptId {
   kOptPdl = 0, kOptDecodeKp, kOptDecodeRp, kOptDecodeStages, kOptDecodeNarrow, kOptDecodeXstream, kOptDecodeXcluster,
-  kOptDecodeI8, kOptDecodeSplitBatch, kOptPrefillGrid, kOptPrefillConvert, kOptPrefillStreamk, kOptPrefillDual, kOptGemvFirst,
+  kOptDecodeI8, kOptDecodeSplitBatch, kOptPrefillGrid, kOptPrefillConvert, kOptPrefillStreamk, kOptPrefillDual, kOptPrefillHelpers, kOptGemvFirst,
   kOptGemvDepth, kOptWaitShift, kOptCount
 };
 int opt(int id);

@@ -71,6 +71,7 @@ struct PrefillCfg {
   int km_kbh, km_keep;       // kept k-blocks per head (the last may be partly kept), kept channels per head
   uint32_t idesc;
   int streamk;               // 1: contiguous ranges of (tile, k-block) units per block; 0: whole tiles round-robin
+  int helpers;               // 1: the de-quantiser warps share the epilogue of the block's last tile
   int* status;
   int* counters;             // stream-K: arrivals per tile
   float* partials;           // stream-K: one accumulation tile [bn tokens][128 rows] fp32 per left-over tile
@@ -364,6 +365,214 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
   auto job_of_wt = [&](int wt) { int j = 0; while (j + 1 < p.n_jobs && wt >= c.wtile_begin[j + 1]) ++j; return j; };
   bool failed = false;
 
+  // ---- the epilogue of one segment, for the warp that calls it: accumulator -> bias, rotary embedding or gated
+  //      product, rounding, store.  A warp reaches the tensor-memory lanes 32 (warp % 4) .. + 31 (a lane is a tile
+  //      row); it takes the chunks ch0, ch0 + chs, ... of 32 tokens.  chs == 1: the epilogue warp on its own (it
+  //      also hands the accumulators back and runs the hand-over of a tile split along K).
+  const int q = warp & 3;                          // TMEM lanes 32q .. 32q+31
+  const int etid = 32 * q + lane;                  // tile row handled in the store phase
+  uint32_t epar = 0;
+  auto epi_sync = [&]() -> bool {
+    __syncwarp();
+    if (lane == 0) pmbar_arrive(epi_bar);
+    const bool ok = pmbar_wait(epi_bar, epar, abort_flag);
+    epar ^= 1;
+    return ok;
+  };
+  volatile int* last_flag = reinterpret_cast<volatile int*>(misc + 8);
+  auto epilogue_segment = [&](const Seg& sg, int tcount, int ch0, int chs) {
+      const int acc0 = c.nh == 2 ? 0 : (tcount & 1);     // as in the MMA warp
+      const int au = c.nh == 2 ? tcount : (tcount >> 1);
+      const int ntok = c.bn * c.nh;                      // tokens of the tile
+      const int t = sg.tile;
+      const int wt = t / c.n_ttiles, tt = t - wt * c.n_ttiles;
+      const int jn = job_of_wt(wt);
+      const JobDev& jb = p.job[jn];
+      const int tl = wt - c.wtile_begin[jn];
+      T* y = reinterpret_cast<T*>(jb.y);
+      const T* bias = reinterpret_cast<const T*>(jb.bias);
+      const bool rope = jb.rope.enabled != 0;
+      // this thread owns tile row etid (= its TMEM lane); a rope pair sits in lanes 2i, 2i + 1
+      const RowInfo ri = tile_row(jb, tl, etid);
+      float b_own = 0.f;
+      unsigned long long turn = 0;
+      const bool swiglu = jb.pair == 1;
+      if (ri.stored >= 0) {
+        const T* bias_own = (swiglu && (etid & 1)) ? reinterpret_cast<const T*>(p.job[jn + 1].bias) : bias;
+        if (bias_own) b_own = DT<T>::to_f(bias_own[ri.stored]);
+        if (rope) {
+          const int half = jb.rope.head_keep >> 1;
+          int pidx = p.idx[(ri.head / jb.rope.rep) * half + ri.pair_c];
+          pidx = min(max(pidx, 0), (jb.rope.head_dim >> 1) - 1);
+          turn = p.rope_turn[pidx];
+        }
+      }
+      // bias, rotary embedding, rounding and store of 32 tokens of this row (all lanes of the warp call it)
+      auto store_chunk = [&](int tok0, const auto& val) {
+        constexpr int NV = (int)(sizeof(val) / sizeof(float));
+        const int m0 = tt * ntok + tok0;
+        if (rope) {
+          // the even lane of a pair rotates the even tokens, the odd lane the odd ones: one exchange hands
+          // each the other member's value of its token, and it stores both rotated members
+          const bool second = (lane & 1) != 0;
+          const int half = jb.rope.head_keep >> 1;
+          const float b_other = __shfl_xor_sync(0xffffffffu, b_own, 1);
+          const float b_lo = second ? b_other : b_own, b_hi = second ? b_own : b_other;
+          const bool live = ri.stored >= 0;
+          const int left = p.M - m0, odd = second ? 1 : 0;
+          T* yp = y + (live ? ri.out_col - (second ? half : 0) : 0) + (size_t)(m0 + odd) * jb.ldy;   // this lane's first token
+          const size_t step = 2 * (size_t)jb.ldy;
+          const int32_t* pp = p.pos + m0 + odd;
+          if (left >= NV) {                       // a whole chunk of tokens: no test per token
+#pragma unroll
+            for (int k = 0; k < NV; k += 2) {
+              const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
+              const float lo = (second ? got : val[k]) + b_lo, hi = (second ? val[k + 1] : got) + b_hi;
+              float cs, sn;
+              rope_cos_sin(__ldg(pp + k), turn, cs, sn);
+              if (live) {
+                yp[0] = DT<T>::from_f(fmaf(-hi, sn, lo * cs));
+                yp[half] = DT<T>::from_f(fmaf(lo, sn, hi * cs));
+              }
+              yp += step;
+            }
+          } else {
+#pragma unroll
+            for (int k = 0; k < NV; k += 2) {
+              if (k >= left) break;
+              const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
+              const float lo = (second ? got : val[k]) + b_lo, hi = (second ? val[k + 1] : got) + b_hi;
+              if (live && k + odd < left) {
+                float cs, sn;
+                rope_cos_sin(__ldg(pp + k), turn, cs, sn);
+                yp[0] = DT<T>::from_f(fmaf(-hi, sn, lo * cs));
+                yp[half] = DT<T>::from_f(fmaf(lo, sn, hi * cs));
+              }
+              yp += step;
+            }
+          }
+        } else if (swiglu) {
+          // as for a rotation pair: the even lane (gate row) takes the even tokens, the odd lane (up row) the odd
+          // ones, one exchange gives each the other matrix's sum of its token; h = silu(g) * u, one rounding
+          // (the approximate division: two instructions instead of ten in warps that share the issue slots
+          //  with the de-quantisers; exp(-g) beyond fp32 gives a quotient of zero, the limit of silu)
+          const bool second = (lane & 1) != 0;
+          const float b_other = __shfl_xor_sync(0xffffffffu, b_own, 1);
+          const float b_g = second ? b_other : b_own, b_u = second ? b_own : b_other;
+          const bool live = ri.stored >= 0;
+          const int left = p.M - m0, odd = second ? 1 : 0;
+          T* yp = y + (live ? ri.out_col : 0) + (size_t)(m0 + odd) * jb.ldy;          // this lane's first token
+          const size_t step = 2 * (size_t)jb.ldy;
+          if (left >= NV) {                       // a whole chunk of tokens: no test per token
+#pragma unroll
+            for (int k = 0; k < NV; k += 2) {
+              const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
+              const float g = (second ? got : val[k]) + b_g, u = (second ? val[k + 1] : got) + b_u;
+              if (live) *yp = DT<T>::from_f(__fdividef(g, 1.f + __expf(-g)) * u);
+              yp += step;
+            }
+          } else {
+#pragma unroll
+            for (int k = 0; k < NV; k += 2) {
+              if (k >= left) break;
+              const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
+              const float g = (second ? got : val[k]) + b_g, u = (second ? val[k + 1] : got) + b_u;
+              if (live && k + odd < left) *yp = DT<T>::from_f(__fdividef(g, 1.f + __expf(-g)) * u);
+              yp += step;
+            }
+          }
+        } else {
+          if (ri.stored < 0) return;
+          T* yr = y + ri.out_col + (size_t)m0 * jb.ldy;
+          const int left = p.M - m0;
+          if (left >= NV) {                       // a whole chunk of tokens: no test per token
+#pragma unroll
+            for (int k = 0; k < NV; ++k) { *yr = DT<T>::from_f(val[k] + b_own); yr += jb.ldy; }
+          } else {
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+              if (k >= left) break;
+              *yr = DT<T>::from_f(val[k] + b_own);
+              yr += jb.ldy;
+            }
+          }
+        }
+      };
+      for (int h = 0; h < c.nh && !failed; ++h)
+        if (!pmbar_wait(acc_full + 8 * (acc0 + h), au & 1, abort_flag)) failed = true;
+      if (failed) return;
+      tc_fence_after();
+      // (the two accumulators are neighbours in tensor memory: a tile of two boxes is 512 consecutive columns)
+      const uint32_t t_acc = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc0 * MAXBN);
+      const int row = 32 * q + lane;
+      // this warp is done with the accumulator that holds token chunk `ch` once that chunk was its last
+      auto release_after = [&](int ch) {
+        if (((ch + 1) * EPI_TOK) % c.bn != 0) return;
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) pmbar_arrive(acc_empty + 8 * (acc0 + (ch * EPI_TOK) / c.bn));
+      };
+      if (sg.kb0 == 0 && sg.kb1 == c.n_kb) {
+        // ---- the whole contraction of this tile ran here (this warp takes every chs-th chunk of 32 tokens)
+        for (int ch = ch0; ch < ntok / EPI_TOK; ch += chs) {
+          uint32_t v[32];
+          tmem_ld32(t_acc + (uint32_t)(ch * EPI_TOK), v);
+          tmem_ld_wait();
+          if (chs == 1) release_after(ch);               // (the values are in registers)
+          float val[32];
+#pragma unroll
+          for (int k = 0; k < 32; ++k) val[k] = __uint_as_float(v[k]);
+          store_chunk(ch * EPI_TOK, val);
+        }
+      } else if (chs == 1) {
+        // ---- a part of the contraction (stream-K): the fp32 partial tile is added (reductions done in L2, a
+        //      warp covers 32 consecutive rows of a token) to the tile's accumulation buffer [token][row] in the
+        //      workspace (zero at launch); the last of the tile's blocks to arrive reads the sum and finishes the tile
+        const size_t slot_f = (size_t)ntok * BMW;
+        const int T0 = (c.n_tiles / (int)gridDim.x) * (int)gridDim.x;          // first left-over tile
+        float* sum = c.partials + (size_t)(t - T0) * slot_f;
+        for (int ch = 0; ch < ntok / EPI_TOK; ++ch) {
+          uint32_t v[32];
+          tmem_ld32(t_acc + (uint32_t)(ch * EPI_TOK), v);
+          tmem_ld_wait();
+          release_after(ch);                                   // the accumulator is free for the next segment
+          float* dst = sum + (size_t)(ch * EPI_TOK) * BMW + row;
+#pragma unroll
+          for (int k = 0; k < 32; ++k) atomicAdd(dst + (size_t)k * BMW, __uint_as_float(v[k]));
+        }
+        __threadfence();                                       // this thread's additions are done before ...
+        if (!epi_sync()) { failed = true; return; }
+        const long U = (long)(c.n_tiles - T0) * c.n_kb, Bn = (long)gridDim.x < U ? (long)gridDim.x : U;
+        const long tu = (long)(t - T0) * c.n_kb;                               // the tile's first left-over unit
+        const int first = sk_owner(tu, Bn, U), last = sk_owner(tu + c.n_kb - 1, Bn, U);
+        if (etid == 0) {
+          const int arrived = atomicAdd(&c.counters[t], 1);    // ... the block's arrival shows
+          *last_flag = arrived == last - first;
+          __threadfence();
+        }
+        if (!epi_sync()) { failed = true; return; }
+        if (*last_flag) {
+          // 16 tokens at a time: the loads of the next 16 are in flight while these are rotated and stored
+          const float* src = sum + row;
+          float nxt[16];
+#pragma unroll
+          for (int k = 0; k < 16; ++k) nxt[k] = __ldcg(src + (size_t)k * BMW);
+          for (int tk = 0; tk < ntok; tk += 16) {
+            float val[16];
+#pragma unroll
+            for (int k = 0; k < 16; ++k) val[k] = nxt[k];
+            if (tk + 16 < ntok) {
+              const float* nx = src + (size_t)(tk + 16) * BMW;
+#pragma unroll
+              for (int k = 0; k < 16; ++k) nxt[k] = __ldcg(nx + (size_t)k * BMW);
+            }
+            store_chunk(tk, val);
+          }
+          if (etid == 0) c.counters[t] = 0;              // ready for the next call
+        }
+      }
+  };
+
   if (warp == 0) {
     // ===================================================================== activations by TMA
     if (lane == 0) {
@@ -438,7 +647,9 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
     constexpr bool heads = HEADS;
     SegIter si; si.init(c, blockIdx.x, gridDim.x);
     Seg sg;
-    for (; !failed && si.next(sg); done += sg.kb1 - sg.kb0) {
+    Seg last_sg = {0, 0, 0};
+    int n_seg = 0;
+    for (; !failed && si.next(sg); done += sg.kb1 - sg.kb0, last_sg = sg, ++n_seg) {
       const int it0 = done - sg.kb0;   // stage iteration of k-block kb of this segment = it0 + kb
       const int wt = sg.tile / c.n_ttiles;
       const int jn = job_of_wt(wt);
@@ -508,213 +719,22 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         q1 = q2; s1 = s2; z1 = z2;
       }
     }
+    // the block's last tile, when it ran whole here: this warp takes a fifth of its chunks beside the epilogue warp
+    // of its tensor-memory quadrant (warps 8 + q, 12 + q, 16 + q, 20 + q: chunks 1, 2, 3, 4 of every five)
+    if (c.helpers && !failed && n_seg > 0 && last_sg.kb0 == 0 && last_sg.kb1 == c.n_kb)
+      epilogue_segment(last_sg, n_seg - 1, 1 + (warp - DQ_WARP0) / 4, 5);
   } else if (warp >= EPI_WARP0) {
     // ===================================================================== epilogue
-    const int q = warp - EPI_WARP0;                 // TMEM lanes 32q .. 32q+31
-    const int etid = tid - EPI_WARP0 * 32;          // 0..127 = tile row handled in the store phase
-    uint32_t epar = 0;
-    auto epi_sync = [&]() -> bool {
-      __syncwarp();
-      if (lane == 0) pmbar_arrive(epi_bar);
-      const bool ok = pmbar_wait(epi_bar, epar, abort_flag);
-      epar ^= 1;
-      return ok;
-    };
-    volatile int* last_flag = reinterpret_cast<volatile int*>(misc + 8);
     int tcount = 0;
     SegIter si; si.init(c, blockIdx.x, gridDim.x);
     Seg sg;
     for (; !failed && si.next(sg); ++tcount) {
-      const int acc0 = c.nh == 2 ? 0 : (tcount & 1);     // as in the MMA warp
-      const int au = c.nh == 2 ? tcount : (tcount >> 1);
-      const int ntok = c.bn * c.nh;                      // tokens of the tile
-      const int t = sg.tile;
-      const int wt = t / c.n_ttiles, tt = t - wt * c.n_ttiles;
-      const int jn = job_of_wt(wt);
-      const JobDev& jb = p.job[jn];
-      const int tl = wt - c.wtile_begin[jn];
-      T* y = reinterpret_cast<T*>(jb.y);
-      const T* bias = reinterpret_cast<const T*>(jb.bias);
-      const bool rope = jb.rope.enabled != 0;
-      // this thread owns tile row etid (= its TMEM lane); a rope pair sits in lanes 2i, 2i + 1
-      const RowInfo ri = tile_row(jb, tl, etid);
-      float b_own = 0.f;
-      unsigned long long turn = 0;
-      const bool swiglu = jb.pair == 1;
-      if (ri.stored >= 0) {
-        const T* bias_own = (swiglu && (etid & 1)) ? reinterpret_cast<const T*>(p.job[jn + 1].bias) : bias;
-        if (bias_own) b_own = DT<T>::to_f(bias_own[ri.stored]);
-        if (rope) {
-          const int half = jb.rope.head_keep >> 1;
-          int pidx = p.idx[(ri.head / jb.rope.rep) * half + ri.pair_c];
-          pidx = min(max(pidx, 0), (jb.rope.head_dim >> 1) - 1);
-          turn = p.rope_turn[pidx];
-        }
-      }
-      // bias, rotary embedding, rounding and store of 32 tokens of this row (all lanes of the warp call it)
-      auto store_chunk = [&](int tok0, const auto& val) {
-        constexpr int NV = (int)(sizeof(val) / sizeof(float));
-        const int m0 = tt * ntok + tok0;
-        if (rope) {
-          // the even lane of a pair rotates the even tokens, the odd lane the odd ones: one exchange hands
-          // each the other member's value of its token, and it stores both rotated members
-          const bool second = (lane & 1) != 0;
-          const int half = jb.rope.head_keep >> 1;
-          const float b_other = __shfl_xor_sync(0xffffffffu, b_own, 1);
-          const float b_lo = second ? b_other : b_own, b_hi = second ? b_own : b_other;
-          const bool live = ri.stored >= 0;
-          const int left = p.M - m0, odd = second ? 1 : 0;
-          T* yp = y + (live ? ri.out_col - (second ? half : 0) : 0) + (size_t)(m0 + odd) * jb.ldy;   // this lane's first token
-          const size_t step = 2 * (size_t)jb.ldy;
-          const int32_t* pp = p.pos + m0 + odd;
-          if (left >= NV) {                       // a whole chunk of tokens: no test per token
-#pragma unroll
-            for (int k = 0; k < NV; k += 2) {
-              const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
-              const float lo = (second ? got : val[k]) + b_lo, hi = (second ? val[k + 1] : got) + b_hi;
-              float cs, sn;
-              rope_cos_sin(pp[k], turn, cs, sn);
-              if (live) {
-                yp[0] = DT<T>::from_f(fmaf(-hi, sn, lo * cs));
-                yp[half] = DT<T>::from_f(fmaf(lo, sn, hi * cs));
-              }
-              yp += step;
-            }
-          } else {
-#pragma unroll
-            for (int k = 0; k < NV; k += 2) {
-              if (k >= left) break;
-              const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
-              const float lo = (second ? got : val[k]) + b_lo, hi = (second ? val[k + 1] : got) + b_hi;
-              if (live && k + odd < left) {
-                float cs, sn;
-                rope_cos_sin(pp[k], turn, cs, sn);
-                yp[0] = DT<T>::from_f(fmaf(-hi, sn, lo * cs));
-                yp[half] = DT<T>::from_f(fmaf(lo, sn, hi * cs));
-              }
-              yp += step;
-            }
-          }
-        } else if (swiglu) {
-          // as for a rotation pair: the even lane (gate row) takes the even tokens, the odd lane (up row) the odd
-          // ones, one exchange gives each the other matrix's sum of its token; h = silu(g) * u, one rounding
-          // (the approximate division: two instructions instead of ten in warps that share the issue slots
-          //  with the de-quantisers; exp(-g) beyond fp32 gives a quotient of zero, the limit of silu)
-          const bool second = (lane & 1) != 0;
-          const float b_other = __shfl_xor_sync(0xffffffffu, b_own, 1);
-          const float b_g = second ? b_other : b_own, b_u = second ? b_own : b_other;
-          const bool live = ri.stored >= 0;
-          const int left = p.M - m0, odd = second ? 1 : 0;
-          T* yp = y + (live ? ri.out_col : 0) + (size_t)(m0 + odd) * jb.ldy;          // this lane's first token
-          const size_t step = 2 * (size_t)jb.ldy;
-          if (left >= NV) {                       // a whole chunk of tokens: no test per token
-#pragma unroll
-            for (int k = 0; k < NV; k += 2) {
-              const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
-              const float g = (second ? got : val[k]) + b_g, u = (second ? val[k + 1] : got) + b_u;
-              if (live) *yp = DT<T>::from_f(__fdividef(g, 1.f + __expf(-g)) * u);
-              yp += step;
-            }
-          } else {
-#pragma unroll
-            for (int k = 0; k < NV; k += 2) {
-              if (k >= left) break;
-              const float got = __shfl_xor_sync(0xffffffffu, second ? val[k] : val[k + 1], 1);
-              const float g = (second ? got : val[k]) + b_g, u = (second ? val[k + 1] : got) + b_u;
-              if (live && k + odd < left) *yp = DT<T>::from_f(__fdividef(g, 1.f + __expf(-g)) * u);
-              yp += step;
-            }
-          }
-        } else {
-          if (ri.stored < 0) return;
-          T* yr = y + ri.out_col + (size_t)m0 * jb.ldy;
-          const int left = p.M - m0;
-          if (left >= NV) {                       // a whole chunk of tokens: no test per token
-#pragma unroll
-            for (int k = 0; k < NV; ++k) { *yr = DT<T>::from_f(val[k] + b_own); yr += jb.ldy; }
-          } else {
-#pragma unroll
-            for (int k = 0; k < NV; ++k) {
-              if (k >= left) break;
-              *yr = DT<T>::from_f(val[k] + b_own);
-              yr += jb.ldy;
-            }
-          }
-        }
-      };
-      for (int h = 0; h < c.nh && !failed; ++h)
-        if (!pmbar_wait(acc_full + 8 * (acc0 + h), au & 1, abort_flag)) failed = true;
-      if (failed) break;
-      tc_fence_after();
-      // (the two accumulators are neighbours in tensor memory: a tile of two boxes is 512 consecutive columns)
-      const uint32_t t_acc = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc0 * MAXBN);
-      const int row = 32 * q + lane;
-      // this warp is done with the accumulator that holds token chunk `ch` once that chunk was its last
-      auto release_after = [&](int ch) {
-        if (((ch + 1) * EPI_TOK) % c.bn != 0) return;
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) pmbar_arrive(acc_empty + 8 * (acc0 + (ch * EPI_TOK) / c.bn));
-      };
-      if (sg.kb0 == 0 && sg.kb1 == c.n_kb) {
-        // ---- the whole contraction of this tile ran here
-        for (int ch = 0; ch < ntok / EPI_TOK; ++ch) {
-          uint32_t v[32];
-          tmem_ld32(t_acc + (uint32_t)(ch * EPI_TOK), v);
-          tmem_ld_wait();
-          release_after(ch);                             // (the values are in registers)
-          float val[32];
-#pragma unroll
-          for (int k = 0; k < 32; ++k) val[k] = __uint_as_float(v[k]);
-          store_chunk(ch * EPI_TOK, val);
-        }
-      } else {
-        // ---- a part of the contraction (stream-K): the fp32 partial tile is added (reductions done in L2, a
-        //      warp covers 32 consecutive rows of a token) to the tile's accumulation buffer [token][row] in the
-        //      workspace (zero at launch); the last of the tile's blocks to arrive reads the sum and finishes the tile
-        const size_t slot_f = (size_t)ntok * BMW;
-        const int T0 = (c.n_tiles / (int)gridDim.x) * (int)gridDim.x;          // first left-over tile
-        float* sum = c.partials + (size_t)(t - T0) * slot_f;
-        for (int ch = 0; ch < ntok / EPI_TOK; ++ch) {
-          uint32_t v[32];
-          tmem_ld32(t_acc + (uint32_t)(ch * EPI_TOK), v);
-          tmem_ld_wait();
-          release_after(ch);                                   // the accumulator is free for the next segment
-          float* dst = sum + (size_t)(ch * EPI_TOK) * BMW + row;
-#pragma unroll
-          for (int k = 0; k < 32; ++k) atomicAdd(dst + (size_t)k * BMW, __uint_as_float(v[k]));
-        }
-        __threadfence();                                       // this thread's additions are done before ...
-        if (!epi_sync()) { failed = true; break; }
-        const long U = (long)(c.n_tiles - T0) * c.n_kb, Bn = (long)gridDim.x < U ? (long)gridDim.x : U;
-        const long tu = (long)(t - T0) * c.n_kb;                               // the tile's first left-over unit
-        const int first = sk_owner(tu, Bn, U), last = sk_owner(tu + c.n_kb - 1, Bn, U);
-        if (etid == 0) {
-          const int arrived = atomicAdd(&c.counters[t], 1);    // ... the block's arrival shows
-          *last_flag = arrived == last - first;
-          __threadfence();
-        }
-        if (!epi_sync()) { failed = true; break; }
-        if (*last_flag) {
-          // 16 tokens at a time: the loads of the next 16 are in flight while these are rotated and stored
-          const float* src = sum + row;
-          float nxt[16];
-#pragma unroll
-          for (int k = 0; k < 16; ++k) nxt[k] = __ldcg(src + (size_t)k * BMW);
-          for (int tk = 0; tk < ntok; tk += 16) {
-            float val[16];
-#pragma unroll
-            for (int k = 0; k < 16; ++k) val[k] = nxt[k];
-            if (tk + 16 < ntok) {
-              const float* nx = src + (size_t)(tk + 16) * BMW;
-#pragma unroll
-              for (int k = 0; k < 16; ++k) nxt[k] = __ldcg(nx + (size_t)k * BMW);
-            }
-            store_chunk(tk, val);
-          }
-          if (etid == 0) c.counters[t] = 0;              // ready for the next call
-        }
-      }
+      // The block's last tile: nothing is left to overlap its epilogue with, and the sixteen de-quantiser warps
+      // are idle by then, so the four of each tensor-memory quadrant take four fifths of its chunks.
+      SegIter peek = si;
+      Seg nxt;
+      const bool helped = c.helpers && sg.kb0 == 0 && sg.kb1 == c.n_kb && !peek.next(nxt);
+      epilogue_segment(sg, tcount, 0, helped ? 5 : 1);
     }
   }
 
@@ -887,6 +907,7 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
       if (dual == 1 || p2.us < pl.us) pl = p2;
     }
   }
+  c.helpers = opt(kOptPrefillHelpers) != 0;
   c.nh = pl.nh;
   c.n_ttiles = pl.ttiles;
   c.n_tiles = pl.tiles;
