@@ -7,15 +7,18 @@
 // k-block) and the tokens its N dimension (up to 256 per tile): D[row][token] += W[row][k] x[token][k].
 //
 // Roles inside a block (one persistent block per SM, tiles taken round-robin):
-//   warp 0       TMA producer: one box [64 k x BN tokens] of activations per stage (128-byte swizzle)
-//   warp 1       allocates tensor memory; one lane issues the MMAs of a stage (4 x K=16) and commits
-//                them to the stage's "empty" barrier and, at the end of a tile, to "accumulator full"
+//   warp 0       TMA producer: boxes [64 k x BN tokens] of activations into a ring of four (128-byte swizzle);
+//                one box per k-block, or two where a tile takes both accumulators (512 tokens)
+//   warp 1       allocates tensor memory; one lane issues the MMAs of a k-block (4 x K=16 per box) and commits
+//                them to the box's and the weight stage's "empty" barriers and, at the end of a tile, to
+//                "accumulator full"
 //   warps 4..7   epilogue: tcgen05.ld the fp32 accumulators (warp w owns TMEM lanes 32(w-4).., a lane
 //                is a tile row and holds 32 tokens of it per pass), bias, rotary embedding on the
 //                retained pair (Section 3.2; the pair's two rows are neighbouring lanes and swap
 //                values by shuffle), one rounding, stores of 32 consecutive outputs of a token per
 //                warp; two accumulator buffers of 256 columns let the epilogue of tile i overlap
-//                the MMAs of tile i+1
+//                the MMAs of tile i+1 (tiles of 512 tokens use both and hand them back one by one);
+//                the epilogue of a block's last tile is shared with the de-quantiser warps, idle by then
 //   warps 8..23  de-quantisers (two teams of eight warps on alternate stages): thread (row, half) converts 32 codes of its weight row per k-block --
 //                nibbles to fp16 by magic number, (q-8) exact, then one fp16 FMA (q-8)*s + fp16(s*(8-z))
 //                -- and writes them into the A-operand stage in the
