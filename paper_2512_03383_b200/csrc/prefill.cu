@@ -77,7 +77,7 @@ struct PrefillCfg {
   int helpers;               // 1: the de-quantiser warps share the epilogue of the block's last tile
   int* status;
   int* counters;             // stream-K: arrivals per tile
-  float* partials;           // stream-K: one accumulation tile [bn tokens][128 rows] fp32 per left-over tile
+  float* partials;           // stream-K: one slot [tokens / 32][128 rows][32 tokens] fp32 per (left-over tile, block) piece
 };
 
 // Work of a block as a sequence of segments (tile, k-blocks [kb0, kb1)): whole tiles t = b, b + grid, ...
@@ -294,11 +294,7 @@ __device__ inline uint4 dequant_word(uint32_t w, __half2 s2, __half2 cz2) {
 
 // bf16 activations -> fp16 copy in the workspace, once per call (every weight tile re-reads the tile of
 // activations, so converting there would repeat the work once per 128 weight rows).
-// The same pass zeroes `zero_units` 16-byte units at `zero` (the stream-K sums of the launch that follows).
-__global__ void x_to_f16_kernel(const __nv_bfloat16* __restrict__ x, int ldx, int M, int k_in, __half* __restrict__ o, int ldo,
-                                uint4* __restrict__ zero, long zero_units) {
-  for (long i = (long)blockIdx.x * blockDim.x + threadIdx.x; i < zero_units; i += (long)gridDim.x * blockDim.x)
-    zero[i] = make_uint4(0, 0, 0, 0);
+__global__ void x_to_f16_kernel(const __nv_bfloat16* __restrict__ x, int ldx, int M, int k_in, __half* __restrict__ o, int ldo) {
   const int units = ldo / 8;                         // 16-byte units per output row (ldo is a multiple of 8)
   const long total = (long)M * units;
   for (long i = (long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
@@ -338,7 +334,9 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
   const uint32_t full_a = bars, empty_a = bars + 8 * PSTAGES;
   const uint32_t full_b = bars + 16 * PSTAGES, empty_b = full_b + 8 * BSLOTS;
   const uint32_t acc_full = full_b + 16 * BSLOTS, acc_empty = acc_full + 16, epi_bar = acc_full + 32;
-  unsigned char* misc = smem + RING_BYTES + 16 * PSTAGES + 16 * BSLOTS + 40;
+  const uint32_t help_bar = acc_full + 40;         // the epilogue warps and the de-quantiser warps that help them
+  const uint32_t last_full = acc_full + 48;        // the MMAs of the block's last segment are complete (one phase only)
+  unsigned char* misc = smem + RING_BYTES + 16 * PSTAGES + 16 * BSLOTS + 56;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
 
@@ -353,6 +351,8 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
     }
     for (int b = 0; b < 2; ++b) { pmbar_init(acc_full + 8 * b, 1); pmbar_init(acc_empty + 8 * b, 4); }
     pmbar_init(epi_bar, 4);
+    pmbar_init(help_bar, 4 + 2 * DQ_WARPS);
+    pmbar_init(last_full, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -383,7 +383,15 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
     return ok;
   };
   volatile int* last_flag = reinterpret_cast<volatile int*>(misc + 8);
-  auto epilogue_segment = [&](const Seg& sg, int tcount, int ch0, int chs) {
+  uint32_t hpar = 0;
+  auto help_sync = [&]() -> bool {
+    __syncwarp();
+    if (lane == 0) pmbar_arrive(help_bar);
+    const bool ok = pmbar_wait(help_bar, hpar, abort_flag);
+    hpar ^= 1;
+    return ok;
+  };
+  auto epilogue_segment = [&](const Seg& sg, int tcount, int ch0, int chs, bool acc_known_full) {
       const int acc0 = c.nh == 2 ? 0 : (tcount & 1);     // as in the MMA warp
       const int au = c.nh == 2 ? tcount : (tcount >> 1);
       const int ntok = c.bn * c.nh;                      // tokens of the tile
@@ -501,7 +509,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
           }
         }
       };
-      for (int h = 0; h < c.nh && !failed; ++h)
+      for (int h = 0; h < c.nh && !failed && !acc_known_full; ++h)
         if (!pmbar_wait(acc_full + 8 * (acc0 + h), au & 1, abort_flag)) failed = true;
       if (failed) return;
       tc_fence_after();
@@ -527,51 +535,61 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
           for (int k = 0; k < 32; ++k) val[k] = __uint_as_float(v[k]);
           store_chunk(ch * EPI_TOK, val);
         }
-      } else if (chs == 1) {
-        // ---- a part of the contraction (stream-K): the fp32 partial tile is added (reductions done in L2, a
-        //      warp covers 32 consecutive rows of a token) to the tile's accumulation buffer [token][row] in the
-        //      workspace (zero at launch); the last of the tile's blocks to arrive reads the sum and finishes the tile
+      } else {
+        // ---- a part of the contraction (stream-K): the fp32 partial tile goes to a slot of its own in the
+        //      workspace, [token][row] (a warp writes and later reads 32 consecutive rows of a token: whole
+        //      128-byte lines); the last of the tile's blocks to arrive adds the slots of all of them in block
+        //      order (the same sum whatever the order of arrival) and finishes the tile.
+        //      The pieces (tile, block) of the cut unit line are numbered lt + block: both grow along the line and
+        //      one of them grows from each piece to the next, so no two pieces share a number.
+        //      chs > 1: the block's last segment, shared with the de-quantiser warps (twenty warps write, meet at a
+        //      barrier of their own, and -- in the last block to arrive -- read back and finish).
+        const bool main_lane = warp == EPI_WARP0 && lane == 0;
         const size_t slot_f = (size_t)ntok * BMW;
         const int T0 = (c.n_tiles / (int)gridDim.x) * (int)gridDim.x;          // first left-over tile
-        float* sum = c.partials + (size_t)(t - T0) * slot_f;
-        for (int ch = 0; ch < ntok / EPI_TOK; ++ch) {
+        float* mine = c.partials + ((size_t)(t - T0) + blockIdx.x) * slot_f;
+        for (int ch = ch0; ch < ntok / EPI_TOK; ch += chs) {
           uint32_t v[32];
           tmem_ld32(t_acc + (uint32_t)(ch * EPI_TOK), v);
           tmem_ld_wait();
-          release_after(ch);                                   // the accumulator is free for the next segment
-          float* dst = sum + (size_t)(ch * EPI_TOK) * BMW + row;
+          if (chs == 1) release_after(ch);                     // the accumulator is free for the next segment
+          float* dst = mine + (size_t)(ch * EPI_TOK) * BMW + row;
 #pragma unroll
-          for (int k = 0; k < 32; ++k) atomicAdd(dst + (size_t)k * BMW, __uint_as_float(v[k]));
+          for (int k = 0; k < 32; ++k) __stcg(dst + (size_t)k * BMW, __uint_as_float(v[k]));
         }
-        __threadfence();                                       // this thread's additions are done before ...
-        if (!epi_sync()) { failed = true; return; }
+        __threadfence();                                       // this thread's part is in place before ...
+        if (!(chs == 1 ? epi_sync() : help_sync())) { failed = true; return; }
         const long U = (long)(c.n_tiles - T0) * c.n_kb, Bn = (long)gridDim.x < U ? (long)gridDim.x : U;
         const long tu = (long)(t - T0) * c.n_kb;                               // the tile's first left-over unit
         const int first = sk_owner(tu, Bn, U), last = sk_owner(tu + c.n_kb - 1, Bn, U);
-        if (etid == 0) {
+        if (main_lane) {
           const int arrived = atomicAdd(&c.counters[t], 1);    // ... the block's arrival shows
           *last_flag = arrived == last - first;
           __threadfence();
         }
-        if (!epi_sync()) { failed = true; return; }
+        if (!(chs == 1 ? epi_sync() : help_sync())) { failed = true; return; }
         if (*last_flag) {
-          // 16 tokens at a time: the loads of the next 16 are in flight while these are rotated and stored
-          const float* src = sum + row;
-          float nxt[16];
-#pragma unroll
-          for (int k = 0; k < 16; ++k) nxt[k] = __ldcg(src + (size_t)k * BMW);
-          for (int tk = 0; tk < ntok; tk += 16) {
+          const float* base = c.partials + ((size_t)(t - T0) + first) * slot_f;
+          const int parts = last - first + 1;
+          // 16 tokens at a time, the loads of two slots in flight together (what the registers of a thread hold)
+          for (int tk = 16 * ch0; tk < ntok; tk += 16 * chs) {
             float val[16];
 #pragma unroll
-            for (int k = 0; k < 16; ++k) val[k] = nxt[k];
-            if (tk + 16 < ntok) {
-              const float* nx = src + (size_t)(tk + 16) * BMW;
+            for (int k = 0; k < 16; ++k) val[k] = 0.f;
+            const float* src = base + (size_t)tk * BMW + row;
+            for (int s2 = 0; s2 < parts; s2 += 2) {
+              const bool two = s2 + 1 < parts;
+              float a[16], b[16];
 #pragma unroll
-              for (int k = 0; k < 16; ++k) nxt[k] = __ldcg(nx + (size_t)k * BMW);
+              for (int k = 0; k < 16; ++k) a[k] = __ldcg(src + (size_t)s2 * slot_f + (size_t)k * BMW);
+#pragma unroll
+              for (int k = 0; k < 16; ++k) b[k] = two ? __ldcg(src + (size_t)(s2 + 1) * slot_f + (size_t)k * BMW) : 0.f;
+#pragma unroll
+              for (int k = 0; k < 16; ++k) val[k] = (val[k] + a[k]) + b[k];
             }
             store_chunk(tk, val);
           }
-          if (etid == 0) c.counters[t] = 0;              // ready for the next call
+          if (main_lane) c.counters[t] = 0;              // ready for the next call
         }
       }
   };
@@ -632,6 +650,12 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         }
         if (failed) break;
         for (int h = 0; h < c.nh; ++h) umma_commit(acc_full + 8 * (acc0 + h));
+        // (the de-quantiser warps that help with the last segment's epilogue cannot follow the phases of the
+        //  accumulator barriers -- a parity wait cannot tell "not yet" from "two phases ago" -- so the last
+        //  segment completes a barrier of its own, which has this one phase)
+        SegIter peek = si;
+        Seg nxt;
+        if (!peek.next(nxt)) umma_commit(last_full);
       }
     }
   } else if (warp >= DQ_WARP0) {
@@ -722,22 +746,24 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         q1 = q2; s1 = s2; z1 = z2;
       }
     }
-    // the block's last tile, when it ran whole here: this warp takes a fifth of its chunks beside the epilogue warp
-    // of its tensor-memory quadrant (warps 8 + q, 12 + q, 16 + q, 20 + q: chunks 1, 2, 3, 4 of every five)
-    if (c.helpers && !failed && n_seg > 0 && last_sg.kb0 == 0 && last_sg.kb1 == c.n_kb)
-      epilogue_segment(last_sg, n_seg - 1, 1 + (warp - DQ_WARP0) / 4, 5);
+    // the block's last segment: this warp takes a fifth of its chunks beside the epilogue warp of its tensor-memory
+    // quadrant (warps 8 + q, 12 + q, 16 + q, 20 + q: chunks 1, 2, 3, 4 of every five)
+    if (c.helpers && !failed && n_seg > 0) {
+      if (!pmbar_wait(last_full, 0, abort_flag, true)) failed = true;
+      if (!failed) epilogue_segment(last_sg, n_seg - 1, 1 + (warp - DQ_WARP0) / 4, 5, true);
+    }
   } else if (warp >= EPI_WARP0) {
     // ===================================================================== epilogue
     int tcount = 0;
     SegIter si; si.init(c, blockIdx.x, gridDim.x);
     Seg sg;
     for (; !failed && si.next(sg); ++tcount) {
-      // The block's last tile: nothing is left to overlap its epilogue with, and the sixteen de-quantiser warps
+      // The block's last segment: nothing is left to overlap its epilogue with, and the sixteen de-quantiser warps
       // are idle by then, so the four of each tensor-memory quadrant take four fifths of its chunks.
       SegIter peek = si;
       Seg nxt;
-      const bool helped = c.helpers && sg.kb0 == 0 && sg.kb1 == c.n_kb && !peek.next(nxt);
-      epilogue_segment(sg, tcount, 0, helped ? 5 : 1);
+      const bool helped = c.helpers && !peek.next(nxt);
+      epilogue_segment(sg, tcount, 0, helped ? 5 : 1, false);
     }
   }
 
@@ -895,7 +921,7 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
     const double share = (double)q.left * c.n_kb / g2;                 // k-blocks per block of the split tiles
     const double hand_over = q.tiles < g2 ? 10.0 + 18.0 * ntok / 256.0 : 14.0 * ntok / 256.0;
     const bool pays = ((double)c.n_kb - share) * kcost > hand_over;
-    q.sums = (size_t)q.left * ntok * BMW * 4;                          // one fp32 tile per left-over tile
+    q.sums = (size_t)(q.left + g2) * ntok * BMW * 4;                   // one fp32 slot per (left-over tile, block) piece
     const bool want = env_streamk >= 0 ? (env_streamk == 1) : (q.left != 0 && pays);
     q.streamk = want && q.left != 0 && cfg.ws_bytes >= ws_used + q.sums && q.tiles <= (1 << 16);
     q.us = q.streamk ? (double)q.tiles / g2 * c.n_kb * kcost + hand_over
@@ -917,22 +943,18 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   if ((long)wt * pl.ttiles > (1 << 24)) return UNIQL_ERR_SHAPE;
   int grid = c.n_tiles < g2 ? c.n_tiles : g2;
   {
-    const size_t sums = pl.sums;
     if (pl.streamk) {
       c.streamk = 1;
       c.partials = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(cfg.workspace) + ws_used);
       grid = g2;
     }
-    // the sums start at zero: the conversion pre-pass clears them where there is one, else a memset node
+    // (the slots of the split tiles are written before they are read: nothing to clear)
     if (x16) {
-      const long units = (long)p.M * (x16_ld / 8) + (c.streamk ? (long)(sums / 16) : 0);
+      const long units = (long)p.M * (x16_ld / 8);
       long blocks = (units + 255) / 256;
       if (blocks > (long)sms * 8) blocks = (long)sms * 8;
-      x_to_f16_kernel<<<(int)blocks, 256, 0, cfg.stream>>>(reinterpret_cast<const __nv_bfloat16*>(p.x), p.ldx, p.M, p.k_in, x16, x16_ld,
-                                                           reinterpret_cast<uint4*>(c.partials), c.streamk ? (long)(sums / 16) : 0);
+      x_to_f16_kernel<<<(int)blocks, 256, 0, cfg.stream>>>(reinterpret_cast<const __nv_bfloat16*>(p.x), p.ldx, p.M, p.k_in, x16, x16_ld);
       if (cudaGetLastError() != cudaSuccess) return UNIQL_ERR_CUDA;
-    } else if (c.streamk) {
-      if (cudaMemsetAsync(c.partials, 0, sums, cfg.stream) != cudaSuccess) return UNIQL_ERR_CUDA;
     }
   }
   {
@@ -953,9 +975,10 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
 }
 
 size_t prefill_workspace_bytes(int M, int K) {
-  // status word and counters (shared header) + room for the fp16 copy of bf16 activations + stream-K partial tiles
+  // status word and counters (shared header) + room for the fp16 copy of bf16 activations + the slots of tiles
+  // split along K: fewer than two per SM, of 256 tokens, or of 512 where tiles take both accumulators
   return ((decode_workspace_header_bytes() + 255) & ~(size_t)255) + (size_t)M * ((K + 7) / 8 * 8) * 2 + 256 +
-         (size_t)2 * p_sm_count() * MAXBN * BMW * 4;
+         (size_t)2 * p_sm_count() * (M > MAXBN ? 2 * MAXBN : MAXBN) * BMW * 4;
 }
 
 }  // namespace uniql
