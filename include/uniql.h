@@ -121,9 +121,12 @@ int uniql_set_path(int path);
  * initial value from the environment variable UNIQL_<NAME IN CAPITALS> when the library is loaded).
  * UNIQL_ERR_SHAPE for an unknown name.  Options a caller may want:
  *   "pdl"              1 / 0: programmatic stream serialization on decode launches (default 1)
- *   "prefill_streamk"  -1 automatic, 0 never, 1 always: split the contraction of the output tiles of the last,
- *                      partly filled round of the tensor-core kernel over several thread blocks.  0 makes the
- *                      results of that kernel reproducible bit for bit (every tile is summed by one block).
+ *   "prefill_streamk"  -1 automatic, 0 never, 1 / 2 always: split the contraction of the output tiles of the last,
+ *                      partly filled round of the tensor-core kernel over several thread blocks.  The parts of a tile
+ *                      go to slots of their own and are added in block order (1; bit-reproducible: the automatic
+ *                      choice where every tile is split), or into one sum per tile in the order in which the blocks
+ *                      finish (2; the automatic choice where whole tiles follow the split ones).  0 makes the results of
+ *                      that kernel reproducible bit for bit in every case (every tile is summed by one block).
  *   "prefill_dual"     -1 / 0: above 256 tokens a tile of the tensor-core kernel takes both accumulators (512
  *                      tokens per de-quantised weight stage); 0 keeps tiles of 256 tokens
  *   "prefill_helpers"  1 / 0: the de-quantiser warps of the tensor-core kernel share the epilogue of a block's last tile
@@ -165,11 +168,11 @@ int uniql_embed_rows(const uint8_t* packed, const void* scales, const void* zero
  * an fp16 copy of x (M x K x 2 bytes): the tensor cores run on fp16 operands, because weights rounded
  * to bf16 would alone spend the 2e-3 error budget; bf16 magnitudes beyond 65504 saturate.  When the
  * workspace is too small for the copy the tiles are converted inside the kernel (same result, slower).
- * It also carries the fp32 sums of output tiles whose contraction is split over several thread blocks
- * (at most 147 tiles of 128 rows x 256 or 512 tokens): the parts of such a tile are added in the order in
- * which the blocks finish, so with more than two blocks on a tile the last bit of an fp32 sum, and
- * rarely of the rounded output, can differ between two runs on the same input; uniql_set_option("prefill_streamk", 0)
- * switches the splitting off.  Activations below fp16's range are affected too: bf16 values under 2^-24 become zero
+ * It also carries the fp32 parts of output tiles whose contraction is split over several thread blocks
+ * (fewer than two slots of 128 rows x 256 or 512 tokens per SM).  Where every tile is split the parts are added in block order; where
+ * split tiles stand in front of whole tiles they are added in the order in which the blocks finish, and with more
+ * than two blocks on a tile the last bit of an fp32 sum, and rarely of the rounded output, can differ
+ * between two runs on the same input; uniql_set_option("prefill_streamk", 0) switches the splitting off.  Activations below fp16's range are affected too: bf16 values under 2^-24 become zero
  * and those under 2^-14 lose significand bits in the fp16 copy.  Without room for the
  * sums every tile is computed by one block (reproducible, slower for shapes that fill few SMs). */
 size_t uniql_workspace_bytes(int M, int K, int N_total);

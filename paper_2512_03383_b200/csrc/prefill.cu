@@ -75,6 +75,7 @@ struct PrefillCfg {
   uint32_t idesc;
   int streamk;               // 1: contiguous ranges of (tile, k-block) units per block; 0: whole tiles round-robin
   int helpers;               // 1: the de-quantiser warps share the epilogue of the block's last tile
+  int sk_atomic;             // stream-K hand-over: 1 = parts added into one sum per tile (reductions in L2), 0 = a slot per part
   int* status;
   int* counters;             // stream-K: arrivals per tile
   float* partials;           // stream-K: one slot [tokens / 32][128 rows][32 tokens] fp32 per (left-over tile, block) piece
@@ -544,18 +545,27 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         //      one of them grows from each piece to the next, so no two pieces share a number.
         //      chs > 1: the block's last segment, shared with the de-quantiser warps (twenty warps write, meet at a
         //      barrier of their own, and -- in the last block to arrive -- read back and finish).
+        //      Where a few split tiles in front of whole tiles have many parts each, reading all the slots back
+        //      would take the four epilogue warps longer than the tiles behind can hide: such launches add the parts
+        //      into ONE sum per tile instead (reductions done in L2, zero at launch; the last bit of a sum then
+        //      depends on the order of arrival when more than two blocks share a tile).
         const bool main_lane = warp == EPI_WARP0 && lane == 0;
         const size_t slot_f = (size_t)ntok * BMW;
         const int T0 = (c.n_tiles / (int)gridDim.x) * (int)gridDim.x;          // first left-over tile
-        float* mine = c.partials + ((size_t)(t - T0) + blockIdx.x) * slot_f;
+        float* mine = c.partials + ((size_t)(t - T0) + (c.sk_atomic ? 0 : blockIdx.x)) * slot_f;
         for (int ch = ch0; ch < ntok / EPI_TOK; ch += chs) {
           uint32_t v[32];
           tmem_ld32(t_acc + (uint32_t)(ch * EPI_TOK), v);
           tmem_ld_wait();
           if (chs == 1) release_after(ch);                     // the accumulator is free for the next segment
           float* dst = mine + (size_t)(ch * EPI_TOK) * BMW + row;
+          if (c.sk_atomic) {
 #pragma unroll
-          for (int k = 0; k < 32; ++k) __stcg(dst + (size_t)k * BMW, __uint_as_float(v[k]));
+            for (int k = 0; k < 32; ++k) atomicAdd(dst + (size_t)k * BMW, __uint_as_float(v[k]));
+          } else {
+#pragma unroll
+            for (int k = 0; k < 32; ++k) __stcg(dst + (size_t)k * BMW, __uint_as_float(v[k]));
+          }
         }
         __threadfence();                                       // this thread's part is in place before ...
         if (!(chs == 1 ? epi_sync() : help_sync())) { failed = true; return; }
@@ -569,8 +579,8 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         }
         if (!(chs == 1 ? epi_sync() : help_sync())) { failed = true; return; }
         if (*last_flag) {
-          const float* base = c.partials + ((size_t)(t - T0) + first) * slot_f;
-          const int parts = last - first + 1;
+          const float* base = c.partials + ((size_t)(t - T0) + (c.sk_atomic ? 0 : first)) * slot_f;
+          const int parts = c.sk_atomic ? 1 : last - first + 1;
           // 16 tokens at a time, the loads of two slots in flight together (what the registers of a thread hold)
           for (int tk = 16 * ch0; tk < ntok; tk += 16 * chs) {
             float val[16];
@@ -895,20 +905,20 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   }
   // The shape of the work: tokens per tile (one accumulator, or both = 512 tokens, so that a de-quantised weight
   // stage serves twice the tokens) and whether the tiles left over after the whole rounds are split along K.
-  // Stream-K serves the tiles left over when whole tiles would leave SMs idle in their last round and the partial
-  // tiles fit in the workspace.  It pays when the k-blocks a block no longer waits for outweigh the hand-over:
-  // measured on B200, a k-block takes about 0.65 us (1.07 us on both accumulators: 1.65 times the time for twice
-  // the work), and the hand-over (zeroing the sums, the additions, the
-  // read-back by the finishing block) about 14 us for tiles of 256 tokens when whole tiles follow and hide
-  // most of it, 28 us when every tile is split; both grow with the tile's width.
-  // (whole tiles that follow hide most of the hand-over: forcing the split on the Qwen2.5-7B q projection at
-  //  M = 2048 and on the Mamba2 in_proj at M = 1024 saved 5.7 and 5.3 us where this rule's saving was 17.7 and 19.7 us)
+  // Stream-K serves the tiles left over when whole tiles would leave SMs idle in their last round and the slots
+  // of the parts fit in the workspace.  It pays when the k-blocks a block no longer waits for outweigh the
+  // hand-over.  Measured on B200: a k-block takes about 0.65 us (1.07 us on both accumulators: 1.65 times the time
+  // for twice the work); a hand-over at the end of a block (every tile split) 20 - 40 us, growing with the number
+  // of blocks on a tile and the tile's width; a hand-over in front of whole tiles is hidden behind them unless a
+  // tile has so many parts that reading them back (11 us per part of 256 tokens) outlasts the whole tiles.
   // Both tile widths are costed with these figures and the cheaper one runs: wide tiles win where they still fill
   // the SMs (Qwen2.5-7B gate at M = 512..4096: 17-22 % faster), narrow ones where wide tiles would leave most SMs
   // without a tile (q / o projections at M = 512) or push a few left-over tiles into a round of their own.
   int g2 = sms;
   if (env_grid >= 1 && env_grid <= sms) g2 = env_grid;            // tests: odd splits on small problems
-  struct Plan { int nh, ttiles, tiles, left; bool streamk; size_t sums; double us; };
+  bool any_rope = false;
+  for (int j = 0; j < p.n_jobs; ++j) any_rope = any_rope || p.job[j].rope.enabled != 0;
+  struct Plan { int nh, ttiles, tiles, left; bool streamk, atomic; size_t sums; double us; };
   auto plan_for = [&](int nh) {
     Plan q;
     q.nh = nh;
@@ -918,14 +928,37 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
     q.tiles = tiles <= (1 << 24) ? (int)tiles : (1 << 24);
     q.left = q.tiles % g2;
     const double kcost = nh == 2 ? 1.07 : 0.65;
-    const double share = (double)q.left * c.n_kb / g2;                 // k-blocks per block of the split tiles
-    const double hand_over = q.tiles < g2 ? 10.0 + 18.0 * ntok / 256.0 : 14.0 * ntok / 256.0;
-    const bool pays = ((double)c.n_kb - share) * kcost > hand_over;
-    q.sums = (size_t)(q.left + g2) * ntok * BMW * 4;                   // one fp32 slot per (left-over tile, block) piece
-    const bool want = env_streamk >= 0 ? (env_streamk == 1) : (q.left != 0 && pays);
+    const double wide = ntok / 256.0;
+    // blocks on the split tile with the most of them: its finishing block reads that many slots back
+    const long units = (long)q.left * c.n_kb;
+    const long bt = units < g2 ? units : g2;
+    const double pmax = q.left ? (double)((bt + q.left - 1) / q.left + 1) : 0.0;
+    double hand_over;
+    q.atomic = false;
+    if (q.tiles < g2) {
+      // every tile is split and every block ends on a split tile: the hand-over is shared with the de-quantiser warps
+      hand_over = 24.0 + 2.0 * pmax * wide;
+    } else {
+      // The split tiles come first and whole tiles follow.  Reading a tile's slots back takes the four epilogue
+      // warps 11 us per slot of 256 tokens, and a split tile in front of whole tiles has three or more parts: that
+      // outlasts the first whole tile, whose epilogue then waits (measured 37 us lost on the Qwen2.5-7B gate at keep
+      // 0.65, M = 2048, three parts).  Here the parts are added into one sum per tile instead (reductions done in
+      // L2): 14 us per 256 tokens, measured, most of it hidden behind the whole tiles.
+      q.atomic = true;
+      hand_over = 14.0 * wide;
+    }
+    // (a tile with the rotary epilogue costs its finishing block about twice as long: measured on the Qwen2.5-7B
+    //  q|k launch at M = 2048, head dim 84, where the split forms lost 8 us against this estimate without it)
+    if (any_rope) hand_over += 12.0 * wide;
+    if (env_streamk == 1) q.atomic = false;                            // tests: the form of the hand-over forced
+    if (env_streamk == 2) q.atomic = true;
+    const double us_split = (double)q.tiles / g2 * c.n_kb * kcost + hand_over;
+    const double us_whole = (double)((q.tiles + g2 - 1) / g2) * c.n_kb * kcost;
+    // one fp32 slot per (left-over tile, block) piece, or one sum per left-over tile
+    q.sums = (size_t)(q.atomic ? q.left : q.left + g2) * ntok * BMW * 4;
+    const bool want = env_streamk >= 0 ? (env_streamk >= 1) : (q.left != 0 && us_split < us_whole);
     q.streamk = want && q.left != 0 && cfg.ws_bytes >= ws_used + q.sums && q.tiles <= (1 << 16);
-    q.us = q.streamk ? (double)q.tiles / g2 * c.n_kb * kcost + hand_over
-                     : (double)((q.tiles + g2 - 1) / g2) * c.n_kb * kcost;
+    q.us = q.streamk ? us_split : us_whole;
     return q;
   };
   Plan pl = plan_for(1);
@@ -945,10 +978,12 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   {
     if (pl.streamk) {
       c.streamk = 1;
+      c.sk_atomic = pl.atomic ? 1 : 0;
       c.partials = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(cfg.workspace) + ws_used);
       grid = g2;
+      // (slots are written before they are read; sums start at zero)
+      if (pl.atomic && cudaMemsetAsync(c.partials, 0, pl.sums, cfg.stream) != cudaSuccess) return UNIQL_ERR_CUDA;
     }
-    // (the slots of the split tiles are written before they are read: nothing to clear)
     if (x16) {
       const long units = (long)p.M * (x16_ld / 8);
       long blocks = (units + 255) / 256;
