@@ -19,11 +19,12 @@
 //                warp; two accumulator buffers of 256 columns let the epilogue of tile i overlap
 //                the MMAs of tile i+1 (tiles of 512 tokens use both and hand them back one by one);
 //                the epilogue of a block's last tile is shared with the de-quantiser warps, idle by then
-//   warps 8..23  de-quantisers (two teams of eight warps on alternate stages): thread (row, half) converts 32 codes of its weight row per k-block --
+//   warps 8..23  de-quantisers: the twelve of them whose scheduler does not host the MMA warp (warp % 4 != 1), two
+//                teams of six warps on alternate stages; a thread converts 32 codes of a weight row per item --
 //                nibbles to fp16 by magic number, (q-8) exact, then one fp16 FMA (q-8)*s + fp16(s*(8-z))
 //                -- and writes them into the A-operand stage in the
-//                canonical K-major 128-byte-swizzled layout; the packed codes of the next two k-blocks
-//                are already in registers
+//                canonical K-major 128-byte-swizzled layout; the packed codes of the next k-block
+//                are already in registers.  All sixteen share the epilogue of the block's last segment.
 // On-device pruning (Section 3.4) is index arithmetic: tile rows are compact output channels mapped to
 // stored rows per thread; the input side is the leading k_in channels (the TMA tensor ends at k_in, so
 // the tail of the last k-block is zero activations).
@@ -57,7 +58,8 @@ constexpr int B_RING = PSTAGES * A_BYTES;    // the activation boxes follow the 
 constexpr int EPI_TOK = 32;                  // tokens per epilogue pass
 constexpr int NWARPS = 24;
 constexpr int PTH = NWARPS * 32;
-constexpr int DQ_WARP0 = 8, DQ_WARPS = 8;      // two teams of DQ_WARPS warps: even and odd stages
+constexpr int DQ_WARP0 = 8, DQ_WARPS = 8;      // warps 8 .. 8 + 2 * DQ_WARPS - 1: the de-quantisers and epilogue helpers
+constexpr int DQ_TEAM_WARPS = 6;               // twelve of them convert: two teams of six warps on alternate stages
 constexpr int EPI_WARP0 = 4;
 constexpr int kPWait = 1 << 20;
 constexpr int kMaxPJobs = kMaxJobs;
@@ -343,7 +345,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
 
   if (tid == 0) {
     for (int s = 0; s < PSTAGES; ++s) {
-      pmbar_init(full_a + 8 * s, DQ_WARPS);
+      pmbar_init(full_a + 8 * s, DQ_TEAM_WARPS);
       pmbar_init(empty_a + 8 * s, 1);
     }
     for (int s = 0; s < BSLOTS; ++s) {
@@ -670,77 +672,103 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
     }
   } else if (warp >= DQ_WARP0) {
     // ===================================================================== de-quantisers
-    // Two teams of eight warps take alternate stages, so that each warp has two stage periods for the
-    // conversion of one stage and the schedulers always find a ready warp.
-    const int team = (warp - DQ_WARP0) / DQ_WARPS;
-    const int dt = tid - (DQ_WARP0 + team * DQ_WARPS) * 32;
-    const int r = dt >> 1, hf = dt & 1;
+    // Two teams of six warps take alternate stages (a team always meets the same ring slots again, so its parity
+    // waits are never more than one phase away from their barriers); a thread converts 32 codes of a weight row,
+    // the first 64 threads of a team a second such item (256 items on 192 threads).  The teams are the twelve
+    // warps on the three schedulers that do NOT host the MMA warp (warp % 4 != 1): the lane that issues the MMAs
+    // runs one dependent instruction after the other, and with four busy warps on its scheduler every one of them
+    // waited longer for its issue slot (measured with those four warps idle, results wrong by construction: Qwen
+    // gate at M = 2048 296 -> 266 us with tiles of 256 tokens, 251 -> 232 us with 512).  The four warps 9, 13, 17,
+    // 21 only help with the block's last epilogue (below).
+    const int sc = warp & 3;
+    if (sc != 1) {
+    const int pos = ((warp - DQ_WARP0) >> 2) * 3 + (sc == 0 ? 0 : sc - 1);      // 0..11 among the twelve
+    const int team = pos / DQ_TEAM_WARPS;
+    const int dt = (pos - team * DQ_TEAM_WARPS) * 32 + lane;                    // 0..191
+    constexpr int TEAM_TH = DQ_TEAM_WARPS * 32;
+    const int n_items = dt + TEAM_TH < 2 * BMW ? 2 : 1;                         // items dt and dt + 192 of 256
     const int G = p.K / kGroup;
-    const uint32_t row_off = (uint32_t)(r * 128);
-    uint32_t col_off[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) col_off[j] = (uint32_t)(((hf * 4 + j) ^ (r & 7)) * 16);
     int done = 0;                      // stage iterations before this segment
     constexpr bool heads = HEADS;
     SegIter si; si.init(c, blockIdx.x, gridDim.x);
     Seg sg;
-    Seg last_sg = {0, 0, 0};
-    int n_seg = 0;
-    for (; !failed && si.next(sg); done += sg.kb1 - sg.kb0, last_sg = sg, ++n_seg) {
+    for (; !failed && si.next(sg); done += sg.kb1 - sg.kb0) {
       const int it0 = done - sg.kb0;   // stage iteration of k-block kb of this segment = it0 + kb
       const int wt = sg.tile / c.n_ttiles;
       const int jn = job_of_wt(wt);
       const JobDev& jb = p.job[jn];
-      const RowInfo ri = tile_row(jb, wt - c.wtile_begin[jn], r);
-      const bool live = ri.stored >= 0;
-      const JobDev& src = (jb.pair == 1 && (r & 1)) ? p.job[jn + 1] : jb;      // odd rows of a SwiGLU pair: the up matrix
-      const uint8_t* wrow = src.w + (size_t)(live ? ri.stored : 0) * (p.K / 2) + hf * 16;
-      const __half* srow = src.scales + (size_t)(live ? ri.stored : 0) * G;
-      const __half* zrow = src.zeros + (size_t)(live ? ri.stored : 0) * G;
+      bool live[2];
+      const uint8_t* wrow[2];
+      const __half* srow[2];
+      const __half* zrow[2];
+      uint32_t st_off[2];              // row and half of the item inside a stage (the swizzle is applied per word)
+      int hf_of[2], r7[2];
+#pragma unroll
+      for (int m = 0; m < 2; ++m) {
+        const int item = dt + m * TEAM_TH;
+        const int r = (item >> 1) & (BMW - 1), hf = item & 1;
+        const RowInfo ri = tile_row(jb, wt - c.wtile_begin[jn], r);
+        live[m] = m < n_items && ri.stored >= 0;
+        const JobDev& src = (jb.pair == 1 && (r & 1)) ? p.job[jn + 1] : jb;    // odd rows of a SwiGLU pair: the up matrix
+        wrow[m] = src.w + (size_t)(live[m] ? ri.stored : 0) * (p.K / 2) + hf * 16;
+        srow[m] = src.scales + (size_t)(live[m] ? ri.stored : 0) * G;
+        zrow[m] = src.zeros + (size_t)(live[m] ? ri.stored : 0) * G;
+        st_off[m] = (uint32_t)(r * 128);
+        hf_of[m] = hf; r7[m] = r & 7;
+      }
       const int kb0 = ((done & 1) == team) ? sg.kb0 : sg.kb0 + 1;
-      // codes and scale / zero-point of this team's next two k-blocks are kept in registers
-      uint4 q0 = make_uint4(0, 0, 0, 0), q1 = q0;
-      __half s0 = __ushort_as_half(0), z0 = s0, s1 = s0, z1 = s0;
-      // codes, scale and zero-point of visited k-block v of this thread's row; `valid` channels of it are kept
+      // codes and scale / zero-point of this team's next k-block are kept in registers
+      uint4 q0[2];
+      __half s0[2], z0[2];
+#pragma unroll
+      for (int m = 0; m < 2; ++m) { q0[m] = make_uint4(0, 0, 0, 0); s0[m] = __ushort_as_half(0); z0[m] = s0[m]; }
+      // codes, scale and zero-point of visited k-block v of an item's row; `valid` channels of it are kept
       // (a leading block needs no mask: the activation tensor map ends at k_in, so the tail of its last k-block
       //  meets zeros)
-      auto fetch = [&](int v, uint4& q, __half& sc, __half& zr) {
+      auto fetch = [&](int m, int v, uint4& q, __half& sc2, __half& zr) {
         const int stored = heads ? kblock_of(c, v).stored : v;
-        q = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)stored * 32));
-        sc = __ldg(srow + (stored >> 1)); zr = __ldg(zrow + (stored >> 1));
+        q = __ldg(reinterpret_cast<const uint4*>(wrow[m] + (size_t)stored * 32));
+        sc2 = __ldg(srow[m] + (stored >> 1)); zr = __ldg(zrow[m] + (stored >> 1));
       };
-      if (live) {
-        if (kb0 < sg.kb1) fetch(kb0, q0, s0, z0);
-        if (kb0 + 2 < sg.kb1) fetch(kb0 + 2, q1, s1, z1);
-      }
+#pragma unroll
+      for (int m = 0; m < 2; ++m)
+        if (live[m] && kb0 < sg.kb1) fetch(m, kb0, q0[m], s0[m], z0[m]);
       for (int kb = kb0; kb < sg.kb1; kb += 2) {
         const int it = it0 + kb;
         const int s = it & (PSTAGES - 1);
         const uint32_t use = (uint32_t)(it / PSTAGES);
-        uint4 q2 = make_uint4(0, 0, 0, 0);
-        __half s2 = s1, z2 = z1;
-        if (live && kb + 4 < sg.kb1) fetch(kb + 4, q2, s2, z2);
+        uint4 q1[2];
+        __half s1[2], z1[2];
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+          q1[m] = make_uint4(0, 0, 0, 0); s1[m] = s0[m]; z1[m] = z0[m];
+          if (live[m] && kb + 2 < sg.kb1) fetch(m, kb + 2, q1[m], s1[m], z1[m]);
+        }
         if (it >= PSTAGES && !pmbar_wait(empty_a + 8 * s, (use - 1) & 1, abort_flag)) { failed = true; break; }
-        const uint32_t a_st = sbase + s * A_BYTES + row_off;
-        const __half2 sh2 = __half2half2(s0);
-        const __half2 cz2 = __float2half2_rn((8.f - __half2float(z0)) * __half2float(s0));
-        const uint32_t qw[4] = {q0.x, q0.y, q0.z, q0.w};
         const int v0 = heads ? kblock_of(c, kb).valid : BK;        // kept channels of this k-block
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          // (eight channels per word; keep counts are multiples of eight, so a word is kept or pruned whole)
-          const uint4 o = (live && (!HEADS || hf * 32 + j * 8 < v0)) ? dequant_word(qw[j], sh2, cz2) : make_uint4(0, 0, 0, 0);
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a_st + col_off[j]), "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w) : "memory");
+        for (int m = 0; m < 2; ++m) {
+          if (m >= n_items) break;
+          const uint32_t a_st = sbase + s * A_BYTES + st_off[m];
+          const __half2 sh2 = __half2half2(s0[m]);
+          const __half2 cz2 = __float2half2_rn((8.f - __half2float(z0[m])) * __half2float(s0[m]));
+          const uint32_t qw[4] = {q0[m].x, q0[m].y, q0[m].z, q0[m].w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            // (eight channels per word; keep counts are multiples of eight, so a word is kept or pruned whole)
+            const uint4 o = (live[m] && (!HEADS || hf_of[m] * 32 + j * 8 < v0)) ? dequant_word(qw[j], sh2, cz2) : make_uint4(0, 0, 0, 0);
+            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a_st + (uint32_t)(((hf_of[m] * 4 + j) ^ r7[m]) * 16)), "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w) : "memory");
+          }
         }
         if constexpr (CONV) {
           // bf16 activations: the tensor cores run on fp16 (8 more mantissa bits for the weights than bf16
           // would leave them); the activation tile that TMA delivered is converted in place
           for (int h = 0; h < c.nh && !failed; ++h) {
-            const int jb = it * c.nh + h;                  // the k-block's boxes in the order the producer issued them
-            const int sb = jb % BSLOTS;
-            if (!pmbar_wait(full_b + 8 * sb, (uint32_t)(jb / BSLOTS) & 1, abort_flag)) { failed = true; break; }
+            const int jb2 = it * c.nh + h;                 // the k-block's boxes in the order the producer issued them
+            const int sb = jb2 % BSLOTS;
+            if (!pmbar_wait(full_b + 8 * sb, (uint32_t)(jb2 / BSLOTS) & 1, abort_flag)) { failed = true; break; }
             const uint32_t b_st = sbase + B_RING + sb * B_BYTES;
-            for (int ci = dt; ci < c.bn * 8; ci += DQ_WARPS * 32) {
+            for (int ci = dt; ci < c.bn * 8; ci += TEAM_TH) {
               uint32_t v0, v1, v2, v3;
               asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(b_st + ci * 16));
               v0 = bf16x2_to_f16x2(v0); v1 = bf16x2_to_f16x2(v1); v2 = bf16x2_to_f16x2(v2); v3 = bf16x2_to_f16x2(v3);
@@ -752,9 +780,18 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         fence_async_smem();            // generic-proxy writes must be visible to the tensor core (async proxy)
         __syncwarp();
         if (lane == 0) pmbar_arrive(full_a + 8 * s);
-        q0 = q1; s0 = s1; z0 = z1;
-        q1 = q2; s1 = s2; z1 = z2;
+#pragma unroll
+        for (int m = 0; m < 2; ++m) { q0[m] = q1[m]; s0[m] = s1[m]; z0[m] = z1[m]; }
       }
+    }
+    }
+    // the block's segments, counted by every warp of this group (the idle four included)
+    Seg last_sg = {0, 0, 0};
+    int n_seg = 0;
+    {
+      SegIter sj; sj.init(c, blockIdx.x, gridDim.x);
+      Seg sgj;
+      while (sj.next(sgj)) { last_sg = sgj; ++n_seg; }
     }
     // the block's last segment: this warp takes a fifth of its chunks beside the epilogue warp of its tensor-memory
     // quadrant (warps 8 + q, 12 + q, 16 + q, 20 + q: chunks 1, 2, 3, 4 of every five)
