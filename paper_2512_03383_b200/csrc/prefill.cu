@@ -96,16 +96,16 @@ struct PrefillCfg {
 // One family {start, period, keep, count}: head h keeps channels [0, keep) of its period; a leading block is
 // the case count = 1.  The activation box of a partly kept block also covers the first columns of the next
 // head: the de-quantisers write zeros for the pruned channels of the block, so those columns do not count.
-struct KBlock { int stored, xcol, valid; };
-__device__ inline KBlock kblock_of(const PrefillCfg& c, int v) {
-  int h = 0, r = v;
-  if (v >= c.km_kbh) { h = v / c.km_kbh; r = v - h * c.km_kbh; }
-  KBlock k;
-  k.stored = c.km_start + h * c.km_period + r;
-  k.xcol = h * c.km_keep + r * BK;
-  k.valid = min(BK, c.km_keep - r * BK);
-  return k;
-}
+// Walked without a division per k-block (a division by the kept blocks per head cost the per-head launches 8 us
+// of 52): (head, kept block within the head) of a visited k-block, stepped.
+struct KWalk {
+  int h, r;
+  __device__ inline void start(const PrefillCfg& c, int v) { h = v / c.km_kbh; r = v - h * c.km_kbh; }
+  __device__ inline void step(const PrefillCfg& c, int n) { r += n; while (r >= c.km_kbh) { r -= c.km_kbh; ++h; } }
+  __device__ inline int stored(const PrefillCfg& c) const { return c.km_start + h * c.km_period + r; }
+  __device__ inline int xcol(const PrefillCfg& c) const { return h * c.km_keep + r * BK; }
+  __device__ inline int valid(const PrefillCfg& c) const { return min(BK, c.km_keep - r * BK); }
+};
 
 struct Seg { int tile, kb0, kb1; };
 struct SegIter {
@@ -614,8 +614,11 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
       Seg sg;
       while (!failed && si.next(sg)) {
         const int tt = sg.tile % c.n_ttiles;
+        KWalk kw;
+        if (HEADS) kw.start(c, sg.kb0);
         for (int kb = sg.kb0; kb < sg.kb1 && !failed; ++kb) {
-          const int xcol = HEADS ? kblock_of(c, kb).xcol : kb * BK;
+          const int xcol = HEADS ? kw.xcol(c) : kb * BK;
+          if (HEADS) kw.step(c, 1);
           for (int h = 0; h < c.nh; ++h, ++jb) {
             if (jb >= BSLOTS && !pmbar_wait(empty_b + 8 * s, par, abort_flag, true)) { failed = true; break; }
             const uint32_t fb = full_b + 8 * s;
@@ -725,27 +728,35 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
       // codes, scale and zero-point of visited k-block v of an item's row; `valid` channels of it are kept
       // (a leading block needs no mask: the activation tensor map ends at k_in, so the tail of its last k-block
       //  meets zeros)
-      auto fetch = [&](int m, int v, uint4& q, __half& sc2, __half& zr) {
-        const int stored = heads ? kblock_of(c, v).stored : v;
+      // (the stored k-block of a visited one costs a division with per-head maps: worked out once for both items)
+      auto fetch = [&](int m, int stored, uint4& q, __half& sc2, __half& zr) {
         q = __ldg(reinterpret_cast<const uint4*>(wrow[m] + (size_t)stored * 32));
         sc2 = __ldg(srow[m] + (stored >> 1)); zr = __ldg(zrow[m] + (stored >> 1));
       };
+      KWalk kw;                                            // this team's current k-block
+      if (heads && kb0 < sg.kb1) kw.start(c, kb0);
+      if (kb0 < sg.kb1) {
+        const int st0 = heads ? kw.stored(c) : kb0;
 #pragma unroll
-      for (int m = 0; m < 2; ++m)
-        if (live[m] && kb0 < sg.kb1) fetch(m, kb0, q0[m], s0[m], z0[m]);
+        for (int m = 0; m < 2; ++m)
+          if (live[m]) fetch(m, st0, q0[m], s0[m], z0[m]);
+      }
       for (int kb = kb0; kb < sg.kb1; kb += 2) {
         const int it = it0 + kb;
         const int s = it & (PSTAGES - 1);
         const uint32_t use = (uint32_t)(it / PSTAGES);
         uint4 q1[2];
         __half s1[2], z1[2];
+        const bool more = kb + 2 < sg.kb1;
+        const int v0 = heads ? kw.valid(c) : BK;           // kept channels of this k-block
+        if (heads) kw.step(c, 2);
+        const int st1 = (heads && more) ? kw.stored(c) : kb + 2;
 #pragma unroll
         for (int m = 0; m < 2; ++m) {
           q1[m] = make_uint4(0, 0, 0, 0); s1[m] = s0[m]; z1[m] = z0[m];
-          if (live[m] && kb + 2 < sg.kb1) fetch(m, kb + 2, q1[m], s1[m], z1[m]);
+          if (live[m] && more) fetch(m, st1, q1[m], s1[m], z1[m]);
         }
         if (it >= PSTAGES && !pmbar_wait(empty_a + 8 * s, (use - 1) & 1, abort_flag)) { failed = true; break; }
-        const int v0 = heads ? kblock_of(c, kb).valid : BK;        // kept channels of this k-block
 #pragma unroll
         for (int m = 0; m < 2; ++m) {
           if (m >= n_items) break;
