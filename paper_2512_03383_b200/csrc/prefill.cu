@@ -938,8 +938,11 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   __half* x16 = nullptr;              // fp16 copy to be written by the pre-pass
   int x16_ld = 0;
   if (p.dt == UNIQL_BF16) {
-    const int ldo = (p.k_in + 7) / 8 * 8;
+    // (a row pitch of whole 128-byte lines: a box row that straddles two lines costs a second L2 request, measured
+    //  as 1.09 instead of 0.85 us per k-block on the Qwen2.5-7B down projection at 12312 of 18944 input channels)
+    int ldo = (p.k_in + 63) / 64 * 64;
     const size_t off = ws_used;
+    if (cfg.ws_bytes < off + (size_t)p.M * ldo * 2) ldo = (p.k_in + 7) / 8 * 8;
     const size_t need = off + (size_t)p.M * ldo * 2;
     if (cfg.ws_bytes >= need && opt(kOptPrefillConvert) != 1) {
       x16 = reinterpret_cast<__half*>(reinterpret_cast<unsigned char*>(cfg.workspace) + off);
@@ -1000,8 +1003,16 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
     if (any_rope) hand_over += 12.0 * wide;
     if (env_streamk == 1) q.atomic = false;                            // tests: the form of the hand-over forced
     if (env_streamk == 2) q.atomic = true;
-    const double us_split = (double)q.tiles / g2 * c.n_kb * kcost + hand_over;
-    const double us_whole = (double)((q.tiles + g2 - 1) / g2) * c.n_kb * kcost;
+    // (a split is taken where it is estimated 5 % ahead: its hand-over varies more than a whole tile's time)
+    const double us_split = 1.05 * ((double)q.tiles / g2 * c.n_kb * kcost + hand_over);
+    // Whole tiles.  On both accumulators a k-block takes 0.84 us when every SM runs one and less when some have no
+    // tile (0.79 us with 28 busy SMs: they share the activation traffic out of L2), and between two tiles of a block
+    // the MMAs wait 7 - 10 us for the epilogue to drain the accumulators (in-kernel time stamps, Qwen2.5-7B gate at
+    // M = 2048); fitted over 48 launches (16 shapes at M = 512, 1024, 2048, every width and hand-over forced in turn).
+    const int rounds = (q.tiles + g2 - 1) / g2;
+    double us_whole = (double)rounds * c.n_kb * kcost;
+    if (nh == 2)
+      us_whole = (double)(q.tiles / g2) * c.n_kb * 0.96 + (q.left ? c.n_kb * (0.90 + 0.06 * q.left / g2) : 0.0) + 10.0 * (rounds - 1);
     // one fp32 slot per (left-over tile, block) piece, or one sum per left-over tile
     q.sums = (size_t)(q.atomic ? q.left : q.left + g2) * ntok * BMW * 4;
     const bool want = env_streamk >= 0 ? (env_streamk >= 1) : (q.left != 0 && us_split < us_whole);
@@ -1060,7 +1071,7 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
 size_t prefill_workspace_bytes(int M, int K) {
   // status word and counters (shared header) + room for the fp16 copy of bf16 activations + the slots of tiles
   // split along K: fewer than two per SM, of 256 tokens, or of 512 where tiles take both accumulators
-  return ((decode_workspace_header_bytes() + 255) & ~(size_t)255) + (size_t)M * ((K + 7) / 8 * 8) * 2 + 256 +
+  return ((decode_workspace_header_bytes() + 255) & ~(size_t)255) + (size_t)M * ((K + 63) / 64 * 64) * 2 + 256 +
          (size_t)2 * p_sm_count() * (M > MAXBN ? 2 * MAXBN : MAXBN) * BMW * 4;
 }
 
