@@ -19,7 +19,7 @@ std::atomic<int> g_path{UNIQL_PATH_AUTO};
 // name, environment variable read once at load, default
 struct OptDesc { const char* name; const char* env; int dflt; };
 const OptDesc kOpts[kOptCount] = {
-    {"pdl", "UNIQL_PDL", 1},                            // programmatic stream serialization on decode launches
+    {"pdl", "UNIQL_PDL", 1},                            // programmatic stream serialization (decode and tensor-core launches)
     {"decode_kp", "UNIQL_DECODE_KP", 0},                // groups of blocks over the input channels (0: automatic)
     {"decode_rp", "UNIQL_DECODE_RP", 0},                // blocks per group (0: one per SM)
     {"decode_stages", "UNIQL_DECODE_STAGES", 0},        // ring stages (0: automatic)

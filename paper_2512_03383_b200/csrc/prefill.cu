@@ -330,6 +330,11 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
                                                          const __grid_constant__ PrefillCfg c) {
   extern __shared__ unsigned char psmem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // Programmatic dependent launch: the next kernel of the stream may be set up while this one runs (its blocks
+  // become resident as ours leave).  What a block does before its own `griddepcontrol.wait` touches nothing a
+  // predecessor may still write or read: barriers, tensor memory, and the weights, which no kernel writes (the
+  // de-quantisers fill the ring ahead); activations, positions, outputs and workspace come after the wait.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const uint32_t raw = (uint32_t)__cvta_generic_to_shared(psmem_raw);
   const uint32_t sbase = (raw + 1023u) & ~1023u;           // swizzled tiles need 1024-byte alignment
   unsigned char* smem = psmem_raw + (sbase - raw);
@@ -609,6 +614,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
   if (warp == 0) {
     // ===================================================================== activations by TMA
     if (lane == 0) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");   // the activations may come from the preceding kernel
       int s = 0; uint32_t par = 1; int jb = 0;             // box slot, parity of its previous use, boxes so far
       SegIter si; si.init(c, blockIdx.x, gridDim.x);
       Seg sg;
@@ -807,11 +813,13 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
     // the block's last segment: this warp takes a fifth of its chunks beside the epilogue warp of its tensor-memory
     // quadrant (warps 8 + q, 12 + q, 16 + q, 20 + q: chunks 1, 2, 3, 4 of every five)
     if (c.helpers && !failed && n_seg > 0) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");   // outputs and workspace: after the preceding kernel
       if (!pmbar_wait(last_full, 0, abort_flag, true)) failed = true;
       if (!failed) epilogue_segment(last_sg, n_seg - 1, 1 + (warp - DQ_WARP0) / 4, 5, true);
     }
   } else if (warp >= EPI_WARP0) {
     // ===================================================================== epilogue
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // positions, outputs and workspace: after the preceding kernel
     int tcount = 0;
     SegIter si; si.init(c, blockIdx.x, gridDim.x);
     Seg sg;
@@ -873,8 +881,19 @@ int launch_pth(const Params& p, const PrefillCfg& c, int grid, cudaStream_t stre
   auto kern = prefill_kernel<T, CONV, HEADS>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return UNIQL_ERR_CUDA;
-  kern<<<grid, PTH, smem, stream>>>(p, c);
-  return cudaGetLastError() == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
+  cudaLaunchConfig_t lc;
+  memset(&lc, 0, sizeof(lc));
+  lc.gridDim = dim3(grid);
+  lc.blockDim = dim3(PTH);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr;
+  lc.numAttrs = opt(kOptPdl) ? 1 : 0;
+  if (cudaLaunchKernelEx(&lc, kern, p, c) != cudaSuccess) { cudaGetLastError(); return UNIQL_ERR_CUDA; }
+  return UNIQL_OK;
 }
 template <typename T, bool CONV>
 int launch_pt(const Params& p, const PrefillCfg& c, int grid, cudaStream_t stream) {

@@ -472,3 +472,48 @@ def test_caller_workspace_smaller_than_the_header_is_refused(B):
     assert e.value.status == 6
     torch.cuda.synchronize()
     assert (y == -77.0).all()
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("streamk", [0, 1])
+def test_chain_of_dependent_launches(B, dtype, streamk):
+    """Launches whose input is the previous launch's output, enqueued back to back with no host synchronisation:
+    with programmatic dependent launch the next kernel's blocks are set up (barriers, tensor memory, the first
+    weight stages) while the previous one still runs, and only its activation loads, stores and workspace traffic
+    wait for it.  The chain must give the same bits as with the attribute off, and its first link the oracle's
+    values.  With split tiles every launch also re-uses the previous one's slots in the workspace."""
+    B.set_path(B.PATH_PREFILL)
+    B.set_option("prefill_streamk", streamk)
+    if streamk:
+        B.set_option("prefill_grid", 5)
+    rng = np.random.default_rng(4242)
+    n = 768
+    qw = synth.draw_qweight(rng, n, n)
+    dw = dev_weight(qw)
+    M = 300
+    tdt = torch.float16 if dtype == "f16" else torch.bfloat16
+    xd = (torch.from_numpy(synth.draw_x(rng, M, n, dtype)).cuda() * 2.0 ** -6).to(tdt)     # small, so that six links stay finite
+    x0 = xd.float().cpu().numpy()
+
+    def chain(pdl, links):
+        B.set_option("pdl", pdl)
+        bufs = [torch.zeros((M, n), dtype=tdt, device="cuda") for _ in range(2)]
+        src = xd
+        first = None
+        for i in range(links):
+            dst = bufs[i & 1]
+            B.qlinear_ex(src, n, dw[1], dw[2], dw[3], None, M, n, n, None, n, None, n, dst, n)
+            if i == 0:
+                first = dst.clone()              # (enqueued on the same stream: ordered after the first launch)
+            src = dst
+        torch.cuda.synchronize()
+        return first, src.clone()
+
+    for rep in range(3):
+        f_off, y_off = chain(0, 6)
+        f_on, y_on = chain(1, 6)
+        assert torch.isfinite(y_off.float()).all()
+        assert torch.equal(f_on, f_off) and torch.equal(y_on, y_off), "repeat %d" % rep
+    ref = oracle.qlinear(x0, dw[0], qw.scales, qw.zeros, oracle.leading(n), oracle.leading(n))
+    check_output(f_on, ref, dtype, TOL[dtype], "first link of the chain")
+    assert B.workspace_status() == 0
