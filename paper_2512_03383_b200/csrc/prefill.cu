@@ -298,6 +298,10 @@ __device__ inline uint4 dequant_word(uint32_t w, __half2 s2, __half2 cz2) {
 // bf16 activations -> fp16 copy in the workspace, once per call (every weight tile re-reads the tile of
 // activations, so converting there would repeat the work once per 128 weight rows).
 __global__ void x_to_f16_kernel(const __nv_bfloat16* __restrict__ x, int ldx, int M, int k_in, __half* __restrict__ o, int ldo) {
+  // (programmatic dependent launch: the tensor-core kernel behind this one may set itself up meanwhile; this one
+  //  waits for its own predecessor before it reads x or overwrites the copy that predecessor may still read)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int units = ldo / 8;                         // 16-byte units per output row (ldo is a multiple of 8)
   const long total = (long)M * units;
   for (long i = (long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
@@ -1066,8 +1070,20 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
       const long units = (long)p.M * (x16_ld / 8);
       long blocks = (units + 255) / 256;
       if (blocks > (long)sms * 8) blocks = (long)sms * 8;
-      x_to_f16_kernel<<<(int)blocks, 256, 0, cfg.stream>>>(reinterpret_cast<const __nv_bfloat16*>(p.x), p.ldx, p.M, p.k_in, x16, x16_ld);
-      if (cudaGetLastError() != cudaSuccess) return UNIQL_ERR_CUDA;
+      cudaLaunchConfig_t lc;
+      memset(&lc, 0, sizeof(lc));
+      lc.gridDim = dim3((unsigned)blocks);
+      lc.blockDim = dim3(256);
+      lc.stream = cfg.stream;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      lc.attrs = attr;
+      lc.numAttrs = opt(kOptPdl) ? 1 : 0;
+      if (cudaLaunchKernelEx(&lc, x_to_f16_kernel, reinterpret_cast<const __nv_bfloat16*>(p.x), p.ldx, p.M, p.k_in, x16, x16_ld) != cudaSuccess) {
+        cudaGetLastError();
+        return UNIQL_ERR_CUDA;
+      }
     }
   }
   {

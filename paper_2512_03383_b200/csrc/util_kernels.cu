@@ -80,6 +80,10 @@ __global__ void embed_kernel(const uint8_t* __restrict__ packed, const __half* _
 // One thread per 4 output channels (8 bytes); x needs 2-byte alignment only.
 __global__ void relay_x_kernel(const unsigned short* __restrict__ x, long long ldx, int M, int count, int keep, int keep8,
                                unsigned short* __restrict__ out) {
+  // (programmatic dependent launch: the kernel behind this one may set itself up meanwhile; this one waits for its
+  //  own predecessor before it reads x or overwrites the copy that predecessor may still read)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int units_row = count * (keep8 >> 2);
   const long long total = (long long)M * units_row;
   const bool vec = ((ldx & 3) == 0) && ((((uintptr_t)x) & 7) == 0) && ((keep & 3) == 0);
@@ -119,9 +123,22 @@ inline int grid_for(int64_t n, int threads) {
 
 int uniql::launch_relay_x(const void* x, long long ldx, int M, int count, int keep, int keep8, void* out, cudaStream_t stream) {
   const int64_t units = (int64_t)M * count * (keep8 / 4);
-  relay_x_kernel<<<grid_for(units, 256), 256, 0, stream>>>(reinterpret_cast<const unsigned short*>(x), ldx, M, count, keep, keep8,
-                                                           reinterpret_cast<unsigned short*>(out));
-  return cudaGetLastError() == cudaSuccess ? UNIQL_OK : UNIQL_ERR_CUDA;
+  cudaLaunchConfig_t lc;
+  memset(&lc, 0, sizeof(lc));
+  lc.gridDim = dim3((unsigned)grid_for(units, 256));
+  lc.blockDim = dim3(256);
+  lc.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr;
+  lc.numAttrs = opt(kOptPdl) ? 1 : 0;
+  if (cudaLaunchKernelEx(&lc, relay_x_kernel, reinterpret_cast<const unsigned short*>(x), ldx, M, count, keep, keep8,
+                         reinterpret_cast<unsigned short*>(out)) != cudaSuccess) {
+    cudaGetLastError();
+    return UNIQL_ERR_CUDA;
+  }
+  return UNIQL_OK;
 }
 
 using namespace uniql;
