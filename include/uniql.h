@@ -134,7 +134,9 @@ int uniql_set_path(int path);
  *                      finish (2; the automatic choice where whole tiles follow the split ones).  0 makes the results of
  *                      that kernel reproducible bit for bit in every case (every tile is summed by one block).
  *   "prefill_dual"     -1 / 0: above 256 tokens a tile of the tensor-core kernel takes both accumulators (512
- *                      tokens per de-quantised weight stage); 0 keeps tiles of 256 tokens
+ *                      tokens per de-quantised weight stage); 0 keeps tiles of 256 tokens; 1 forces tiles of 512 tokens
+ *                      wherever M > 256 (tests: 2 the same without half tiles for the left-over round, 3 with them
+ *                      wherever they fit)
  *   "prefill_helpers"  1 / 0: the de-quantiser warps of the tensor-core kernel share the epilogue of a block's last tile
  *   "decode_split_batch" batches of 9..16 rows: 2 (default) one launch that streams the quantised activations
  *                      beside the weights, where the integer path applies, else two launches over half the batch;

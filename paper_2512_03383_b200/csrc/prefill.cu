@@ -78,6 +78,8 @@ struct PrefillCfg {
   int streamk;               // 1: contiguous ranges of (tile, k-block) units per block; 0: whole tiles round-robin
   int helpers;               // 1: the de-quantiser warps share the epilogue of the block's last tile
   int sk_atomic;             // stream-K hand-over: 1 = parts added into one sum per tile (reductions in L2), 0 = a slot per part
+  int halves;                // tiles on both accumulators: the tiles left over after the whole rounds run as half tiles
+                             // (one box of 256 tokens each, on twice as many blocks), every block's last segment
   int* status;
   int* counters;             // stream-K: arrivals per tile
   float* partials;           // stream-K: one slot [tokens / 32][128 rows][32 tokens] fp32 per (left-over tile, block) piece
@@ -107,12 +109,21 @@ struct KWalk {
   __device__ inline int valid(const PrefillCfg& c) const { return min(BK, c.km_keep - r * BK); }
 };
 
-struct Seg { int tile, kb0, kb1; };
+// half: -1 the whole tile; 0 / 1: only the first / second box of a tile of two boxes (into accumulator 0 / 1)
+struct Seg { int tile, kb0, kb1, half; };
 struct SegIter {
   long u, ue;
-  int t, t_end, n_kb, step, tail_tile0;
+  int t, t_end, n_kb, step, tail_tile0, half_tile, half;
   __device__ inline void init(const PrefillCfg& c, int b, int grid) {
     n_kb = c.n_kb; step = grid; t = b;
+    half_tile = -1; half = 0;
+    if (c.halves) {
+      // whole rounds of whole tiles, then tile (rounds * grid + b / 2) as two halves on blocks b and b + 1
+      const int full = (c.n_tiles / grid) * grid;
+      t_end = full; tail_tile0 = full; u = ue = 0;
+      if (full + b / 2 < c.n_tiles) { half_tile = full + b / 2; half = b & 1; }
+      return;
+    }
     const int base = c.streamk ? c.n_tiles / grid : (c.n_tiles + grid - 1) / grid;
     t_end = c.streamk ? base * grid : c.n_tiles;
     tail_tile0 = base * grid;
@@ -130,12 +141,18 @@ struct SegIter {
       sg.kb0 = (int)(u - (long)tt * n_kb);
       const long len = (n_kb - sg.kb0) < (ue - u) ? (n_kb - sg.kb0) : (ue - u);
       sg.kb1 = sg.kb0 + (int)len;
+      sg.half = -1;
       u += len;
       return true;
     }
     if (t < t_end) {
-      sg.tile = t; sg.kb0 = 0; sg.kb1 = n_kb;
+      sg.tile = t; sg.kb0 = 0; sg.kb1 = n_kb; sg.half = -1;
       t += step;
+      return true;
+    }
+    if (half_tile >= 0) {
+      sg.tile = half_tile; sg.kb0 = 0; sg.kb1 = n_kb; sg.half = half;
+      half_tile = -1;
       return true;
     }
     return false;
@@ -407,6 +424,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
       const int acc0 = c.nh == 2 ? 0 : (tcount & 1);     // as in the MMA warp
       const int au = c.nh == 2 ? tcount : (tcount >> 1);
       const int ntok = c.bn * c.nh;                      // tokens of the tile
+      const int h_lo = sg.half < 0 ? 0 : sg.half, h_hi = sg.half < 0 ? c.nh : sg.half + 1;   // boxes of this segment
       const int t = sg.tile;
       const int wt = t / c.n_ttiles, tt = t - wt * c.n_ttiles;
       const int jn = job_of_wt(wt);
@@ -521,7 +539,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
           }
         }
       };
-      for (int h = 0; h < c.nh && !failed && !acc_known_full; ++h)
+      for (int h = h_lo; h < h_hi && !failed && !acc_known_full; ++h)
         if (!pmbar_wait(acc_full + 8 * (acc0 + h), au & 1, abort_flag)) failed = true;
       if (failed) return;
       tc_fence_after();
@@ -536,8 +554,10 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         if (lane == 0) pmbar_arrive(acc_empty + 8 * (acc0 + (ch * EPI_TOK) / c.bn));
       };
       if (sg.kb0 == 0 && sg.kb1 == c.n_kb) {
-        // ---- the whole contraction of this tile ran here (this warp takes every chs-th chunk of 32 tokens)
-        for (int ch = ch0; ch < ntok / EPI_TOK; ch += chs) {
+        // ---- the whole contraction of this tile ran here (this warp takes every chs-th chunk of 32 tokens;
+        //      of a half tile only the chunks of its box)
+        const int cpb = c.bn / EPI_TOK;
+        for (int ch = h_lo * cpb + ch0; ch < h_hi * cpb; ch += chs) {
           uint32_t v[32];
           tmem_ld32(t_acc + (uint32_t)(ch * EPI_TOK), v);
           tmem_ld_wait();
@@ -629,7 +649,8 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         for (int kb = sg.kb0; kb < sg.kb1 && !failed; ++kb) {
           const int xcol = HEADS ? kw.xcol(c) : kb * BK;
           if (HEADS) kw.step(c, 1);
-          for (int h = 0; h < c.nh; ++h, ++jb) {
+          const int h_lo = sg.half < 0 ? 0 : sg.half, h_hi = sg.half < 0 ? c.nh : sg.half + 1;
+          for (int h = h_lo; h < h_hi; ++h, ++jb) {
             if (jb >= BSLOTS && !pmbar_wait(empty_b + 8 * s, par, abort_flag, true)) { failed = true; break; }
             const uint32_t fb = full_b + 8 * s;
             pmbar_expect_tx(fb, (uint32_t)(c.bn * BK * 2));
@@ -653,10 +674,11 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         // the epilogue while the MMAs of the next tile already run on ... once it is free again (per-accumulator waits).
         const int acc0 = c.nh == 2 ? 0 : (tcount & 1);
         const int au = c.nh == 2 ? tcount : (tcount >> 1);   // earlier tiles that used this tile's accumulator(s)
+        const int h_lo = sg.half < 0 ? 0 : sg.half, h_hi = sg.half < 0 ? c.nh : sg.half + 1;   // (a half tile is a block's last)
         for (int kb = sg.kb0; kb < sg.kb1 && !failed; ++kb) {
           if (!pmbar_wait(full_a + 8 * s, par, abort_flag)) { failed = true; break; }
           const uint64_t adesc = smem_desc_sw128(sbase + s * A_BYTES);
-          for (int h = 0; h < c.nh; ++h) {
+          for (int h = h_lo; h < h_hi; ++h) {
             if (kb == sg.kb0 && au >= 1 && !pmbar_wait(acc_empty + 8 * (acc0 + h), (au - 1) & 1, abort_flag)) { failed = true; break; }
             // (bf16: the de-quantisers waited for the activation box themselves and converted it)
             if (!CONV && !pmbar_wait(full_b + 8 * sb, parb, abort_flag)) { failed = true; break; }
@@ -674,7 +696,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
           if (++s == PSTAGES) { s = 0; par ^= 1; }
         }
         if (failed) break;
-        for (int h = 0; h < c.nh; ++h) umma_commit(acc_full + 8 * (acc0 + h));
+        for (int h = h_lo; h < h_hi; ++h) umma_commit(acc_full + 8 * (acc0 + h));
         // (the de-quantiser warps that help with the last segment's epilogue cannot follow the phases of the
         //  accumulator barriers -- a parity wait cannot tell "not yet" from "two phases ago" -- so the last
         //  segment completes a barrier of its own, which has this one phase)
@@ -807,7 +829,7 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
     }
     }
     // the block's segments, counted by every warp of this group (the idle four included)
-    Seg last_sg = {0, 0, 0};
+    Seg last_sg = {0, 0, 0, -1};
     int n_seg = 0;
     {
       SegIter sj; sj.init(c, blockIdx.x, gridDim.x);
@@ -992,7 +1014,7 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   if (env_grid >= 1 && env_grid <= sms) g2 = env_grid;            // tests: odd splits on small problems
   bool any_rope = false;
   for (int j = 0; j < p.n_jobs; ++j) any_rope = any_rope || p.job[j].rope.enabled != 0;
-  struct Plan { int nh, ttiles, tiles, left; bool streamk, atomic; size_t sums; double us; };
+  struct Plan { int nh, ttiles, tiles, left; bool streamk, atomic, halves; size_t sums; double us; };
   auto plan_for = [&](int nh) {
     Plan q;
     q.nh = nh;
@@ -1041,18 +1063,28 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
     const bool want = env_streamk >= 0 ? (env_streamk >= 1) : (q.left != 0 && us_split < us_whole);
     q.streamk = want && q.left != 0 && cfg.ws_bytes >= ws_used + q.sums && q.tiles <= (1 << 16);
     q.us = q.streamk ? us_split : us_whole;
+    // Tiles of two boxes left over after the whole rounds, when they are few: each runs as two half tiles (one box,
+    // 256 tokens) on two blocks, a block's last segment -- no hand-over, and the round takes a one-box tile's time
+    // (0.45 - 0.6 us per k-block by the number of busy SMs) instead of a two-box tile's on a few SMs.
+    q.halves = false;
+    if (nh == 2 && q.left != 0 && 2 * q.left <= g2 && q.tiles > g2 && !conv_in_kernel && env_streamk < 1 && opt(kOptPrefillDual) != 2) {
+      const double us_halves = (double)(q.tiles / g2) * (c.n_kb * 0.96 + 10.0) + c.n_kb * (0.45 + 0.15 * 2 * q.left / g2);
+      if (us_halves < q.us || opt(kOptPrefillDual) == 3) { q.halves = true; q.streamk = false; q.us = us_halves; }
+    }
     return q;
   };
   Plan pl = plan_for(1);
   {
-    const int dual = opt(kOptPrefillDual);                          // -1: by cost, 0: never, 1: wherever M > 256
+    // -1: by cost, 0: never, 1: wherever M > 256; tests: 2 the same without half tiles, 3 with them wherever they fit
+    const int dual = opt(kOptPrefillDual);
     if (p.M > MAXBN && dual != 0) {
       const Plan p2 = plan_for(2);
-      if (dual == 1 || p2.us < pl.us) pl = p2;
+      if (dual >= 1 || p2.us < pl.us) pl = p2;
     }
   }
   c.helpers = opt(kOptPrefillHelpers) != 0;
   c.nh = pl.nh;
+  c.halves = pl.halves ? 1 : 0;
   c.n_ttiles = pl.ttiles;
   c.n_tiles = pl.tiles;
   if ((long)wt * pl.ttiles > (1 << 24)) return UNIQL_ERR_SHAPE;

@@ -517,3 +517,39 @@ def test_chain_of_dependent_launches(B, dtype, streamk):
     ref = oracle.qlinear(x0, dw[0], qw.scales, qw.zeros, oracle.leading(n), oracle.leading(n))
     check_output(f_on, ref, dtype, TOL[dtype], "first link of the chain")
     assert B.workspace_status() == 0
+
+
+@pytest.mark.parametrize("grid", [2, 3, 4, 6, 7])
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("M", [513, 700, 1100])
+def test_left_over_wide_tiles_as_half_tiles(B, M, dtype, grid):
+    """Tiles of two boxes left over after the whole rounds run as half tiles (one box each, on two blocks, a block's
+    last segment on the accumulator of its box).  Forced wherever the rule allows, on grids that leave one to three
+    tiles over, against the oracle and bit for bit against tiles of 256 tokens (whole tiles either way: one block sums
+    a tile's k-blocks in the same order); plain rows with bias, a per-head input map and the rotary epilogue."""
+    B.set_path(B.PATH_PREFILL)
+    B.set_option("prefill_grid", grid)
+    B.set_option("prefill_streamk", 0)
+    rng = np.random.default_rng(3300 + M + grid)
+    qw = synth.draw_qweight(rng, 600, 512)                     # 5 weight tiles x 2 or 3 token tiles of 512
+    dw = dev_weight(qw)
+    bias = synth.to_dtype_values(rng.standard_normal(600).astype(np.float32), dtype)
+    outs = {}
+    for dual in (3, 0):
+        B.set_option("prefill_dual", dual)
+        for (k_in, k_out) in [(512, 600), (420, 388)]:
+            x = synth.draw_x(np.random.default_rng(M + k_in), M, k_in, dtype)
+            y, ref = run_ex(B, qw, dw, x, dtype, None, k_in, None, k_out, bias=bias, ldx_pad=8 - k_in % 8 if k_in % 8 else 0,
+                            ldy_pad=5)
+            check_output(y, ref, dtype, TOL[dtype], "half tiles=%d M=%d %s k=(%d,%d) grid %d" % (dual, M, dtype, k_in, k_out, grid))
+            outs[(dual, k_in)] = y.clone()
+    for k_in in (512, 420):
+        assert torch.equal(outs[(3, k_in)], outs[(0, k_in)]), "half tiles changed the result"
+    B.set_option("prefill_dual", 3)
+    im = synth.map_per_head(4, 128, 104)
+    x = synth.draw_x(rng, M, synth.map_size(im), dtype)
+    y, ref = run_ex(B, qw, dw, x, dtype, im, 0, None, 600, ldx_pad=8)
+    check_output(y, ref, dtype, TOL[dtype], "half tiles, per-head input map M=%d" % M)
+    for (g, r) in run_rope(B, rng, M, 512, 6, 2, 128, 84, 5e5, dtype, bias=True):
+        check_output(g, r, dtype, TOL[dtype], "half tiles, rope M=%d grid %d" % (M, grid))
+    assert B.workspace_status() == 0
