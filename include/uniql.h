@@ -77,8 +77,10 @@ typedef enum {
 typedef enum { UNIQL_F16 = 0, UNIQL_BF16 = 1 } uniql_dtype;
 
 /* Kernel selection, for A/B tests.  AUTO: fp16 batches of M <= 16 take the persistent decode kernel
- * (UNIQL_PATH_DECODE); batches of M <= 4 whose input map lies on 4- but not on 8-channel boundaries (head dims 108
- * and 84 on the input side of o_proj, 1740 of 2048 leading channels) take the streaming kernel (UNIQL_PATH_GEMV:
+ * (UNIQL_PATH_DECODE); where the input map lies on 4- but not on 8-channel boundaries (head dims 108 and 84 on the
+ * input side of o_proj, 1740 of 2048 leading channels) a small kernel in front re-lays the activations on
+ * 8-channel boundaries in the workspace, and batches of M <= 4 for which that is not possible (no room in the
+ * workspace, blocks that do not start on 8-channel boundaries) take the streaming kernel (UNIQL_PATH_GEMV:
  * every warp copies its own share of the codes through a private shared-memory ring) when its rules hold (one
  * input family, every start / keep / period a multiple of 4, K a multiple of 512, x 8-byte aligned with ldx a
  * multiple of 4, scale and zero-point arrays 8-byte aligned); everything

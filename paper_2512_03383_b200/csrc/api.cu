@@ -145,11 +145,13 @@ int dispatch(const Params& p_in, void* workspace, size_t ws_bytes, void* stream)
   // allow it: at 17..63 rows the generic kernel measured 13 to 26 times slower (930 us against 71 us for the
   // Llama-3-8B gate|up at M = 17)
   bool pre_ok = prefill_supported(p);
-  // one to four rows whose input map is on 4- but not 8-channel boundaries (head dims 108 and 84, 1740 of 2048
-  // channels): the streaming kernel, which stages activations in 8-byte units
-  const bool gv = path == UNIQL_PATH_GEMV ||
-                  (path == UNIQL_PATH_AUTO && gemv_supported(p) &&
-                   (opt(kOptGemvFirst) == 1 || !(dec_ok && decode_integer_path(p))));
+  // One to four rows whose input map is on 4- but not 8-channel boundaries (head dims 108 and 84, 1740 of 2048
+  // channels): re-laid on 8-channel boundaries for the decode kernel's integer path where that is possible (with
+  // the small kernel in front under programmatic dependent launch: Llama-3-8B o_proj at head dim 108, M = 1 / 4:
+  // 5.9 / 8.4 us), else the streaming kernel, which stages activations in 8-byte units (8.7 / 13.1 us).
+  bool gv = path == UNIQL_PATH_GEMV || (path == UNIQL_PATH_AUTO && gemv_supported(p) && opt(kOptGemvFirst) == 1);
+  const bool gv_else = path == UNIQL_PATH_AUTO && !gv && gemv_supported(p) && !(dec_ok && decode_integer_path(p));
+  bool relaid = false;
   // Everything else that misses a fast kernel only because of where its activations lie (blocks of 108 or 84
   // channels, an odd row pitch) gets them re-laid in the workspace by a small kernel in front: 5..16 rows then run
   // on the integer path of the decode kernel, larger batches and bf16 on the tensor cores.
@@ -175,12 +177,14 @@ int dispatch(const Params& p_in, void* workspace, size_t ws_bytes, void* stream)
         if (rc != UNIQL_OK) return rc;
         q.x = xr;
         p = q;
+        relaid = true;
         cfg.ws_bytes = off;
         dec_ok = p.M <= 16 && decode_supported(p);
         pre_ok = prefill_supported(p);
       }
     }
   }
+  if (gv_else && !relaid) gv = true;
   if (path == UNIQL_PATH_AUTO)
     path = gv ? UNIQL_PATH_GEMV : dec_ok ? UNIQL_PATH_DECODE : (pre_ok ? UNIQL_PATH_PREFILL : UNIQL_PATH_GENERIC);
   if (path == UNIQL_PATH_GEMV) {
