@@ -133,8 +133,11 @@ int uniql_set_path(int path);
  *                      partly filled round of the tensor-core kernel over several thread blocks.  The parts of a tile
  *                      go to slots of their own and are added in block order (1; bit-reproducible: the automatic
  *                      choice where every tile is split), or into one sum per tile in the order in which the blocks
- *                      finish (2; the automatic choice where whole tiles follow the split ones).  0 makes the results of
- *                      that kernel reproducible bit for bit in every case (every tile is summed by one block).
+ *                      finish (2; the automatic choice where whole tiles follow the split ones).  Launches with at most
+ *                      one tile for every two SMs may instead run a cluster of two blocks per tile, half of the
+ *                      contraction each, the second block's sums added in the first one's shared memory (3 forces it
+ *                      wherever it fits; bit-reproducible).  0 makes the results of that kernel reproducible bit for
+ *                      bit in every case (every tile is summed by one block).
  *   "prefill_dual"     -1 / 0: above 256 tokens a tile of the tensor-core kernel takes both accumulators (512
  *                      tokens per de-quantised weight stage); 0 keeps tiles of 256 tokens; 1 forces tiles of 512 tokens
  *                      wherever M > 256 (tests: 2 the same without half tiles for the left-over round, 3 with them

@@ -30,7 +30,7 @@ const OptDesc kOpts[kOptCount] = {
     {"decode_split_batch", "UNIQL_DECODE_SPLIT_BATCH", 2},   // batches of 9..16: one streamed launch where it applies
     {"prefill_grid", "UNIQL_PREFILL_GRID", 0},          // blocks of the tensor-core kernel (0: one per SM)
     {"prefill_convert", "UNIQL_PREFILL_CONVERT_IN_KERNEL", 0},   // 1: bf16 tiles converted inside the kernel
-    {"prefill_streamk", "UNIQL_PREFILL_STREAMK", -1},   // split tiles: -1 automatic, 0 never, 1 always (a slot per part), 2 always (one sum per tile)
+    {"prefill_streamk", "UNIQL_PREFILL_STREAMK", -1},   // split tiles: -1 automatic, 0 never, 1 always (a slot per part), 2 always (one sum per tile), 3 pairs of blocks
     {"prefill_dual", "UNIQL_PREFILL_DUAL", -1},         // tiles of 512 tokens on both accumulators: -1 by cost, 0 never, 1 always (2 / 3: without / with half tiles)
     {"prefill_helpers", "UNIQL_PREFILL_HELPERS", 1},    // de-quantiser warps share the epilogue of a block's last tile
     {"gemv_first", "UNIQL_GEMV_FIRST", 0},              // 1: the streaming kernel wherever it applies (M <= 4)

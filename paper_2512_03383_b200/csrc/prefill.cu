@@ -38,6 +38,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
 #include <mutex>
 #include <type_traits>
 
@@ -78,6 +79,8 @@ struct PrefillCfg {
   int streamk;               // 1: contiguous ranges of (tile, k-block) units per block; 0: whole tiles round-robin
   int helpers;               // 1: the de-quantiser warps share the epilogue of the block's last tile
   int sk_atomic;             // stream-K hand-over: 1 = parts added into one sum per tile (reductions in L2), 0 = a slot per part
+  int pair_split;            // clusters of two blocks on one tile, half of the contraction each; the second block's
+                             // fp32 sums go into the first one's shared memory (the rings, idle by then)
   int halves;                // tiles on both accumulators: the tiles left over after the whole rounds run as half tiles
                              // (one box of 256 tokens each, on twice as many blocks), every block's last segment
   int* status;
@@ -113,10 +116,20 @@ struct KWalk {
 struct Seg { int tile, kb0, kb1, half; };
 struct SegIter {
   long u, ue;
-  int t, t_end, n_kb, step, tail_tile0, half_tile, half;
+  int t, t_end, n_kb, step, tail_tile0, half_tile, half, ps_tile, ps_kb0, ps_kb1;
   __device__ inline void init(const PrefillCfg& c, int b, int grid) {
     n_kb = c.n_kb; step = grid; t = b;
     half_tile = -1; half = 0;
+    ps_tile = -1;
+    if (c.pair_split) {
+      // block 2t takes the first k-blocks of tile t and finishes it, block 2t + 1 the rest (the smaller half)
+      t_end = 0; tail_tile0 = 0; u = ue = 0; t = 1;
+      ps_tile = b >> 1;
+      const int mid = n_kb - n_kb / 2;
+      ps_kb0 = (b & 1) ? mid : 0;
+      ps_kb1 = (b & 1) ? n_kb : mid;
+      return;
+    }
     if (c.halves) {
       // whole rounds of whole tiles, then tile (rounds * grid + b / 2) as two halves on blocks b and b + 1
       const int full = (c.n_tiles / grid) * grid;
@@ -148,6 +161,11 @@ struct SegIter {
     if (t < t_end) {
       sg.tile = t; sg.kb0 = 0; sg.kb1 = n_kb; sg.half = -1;
       t += step;
+      return true;
+    }
+    if (ps_tile >= 0) {
+      sg.tile = ps_tile; sg.kb0 = ps_kb0; sg.kb1 = ps_kb1; sg.half = -1;
+      ps_tile = -1;
       return true;
     }
     if (half_tile >= 0) {
@@ -192,6 +210,51 @@ __device__ inline bool pmbar_wait(uint32_t bar, uint32_t parity, volatile int* a
   *abort_flag = 1;
   return false;
 }
+// ---- clusters of two (a tile's contraction split over a pair of blocks)
+__device__ inline uint32_t pcluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// address of `addr` (shared memory of this block) in block `rank` of the cluster
+__device__ inline uint32_t ppeer_addr(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+// generic address of `ptr` (shared memory of this block) in block `rank` of the cluster
+__device__ inline float* ppeer_generic(void* ptr, uint32_t rank) {
+  unsigned long long r;
+  asm volatile("mapa.u64 %0, %1, %2;" : "=l"(r) : "l"(reinterpret_cast<unsigned long long>(ptr)), "r"(rank));
+  return reinterpret_cast<float*>(r);
+}
+template <int STRIDE, int K = 0>
+__device__ inline void pld_add_f32x16(uint32_t base, const uint32_t (&v)[16], float (&val)[16]) {
+  if constexpr (K < 16) {
+    float o;
+    asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(o) : "r"(base), "n"(K * STRIDE) : "memory");
+    val[K] = __uint_as_float(v[K]) + o;
+    pld_add_f32x16<STRIDE, K + 1>(base, v, val);
+  }
+}
+__device__ inline void pmbar_arrive_peer(uint32_t addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(addr) : "memory");
+}
+__device__ inline bool pmbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (int i = 0; i < kPWait; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (ok) return true;
+    __nanosleep(100);
+    if ((i & 63) == 63 && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
 __device__ inline void tma_box2(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -229,6 +292,14 @@ __device__ inline void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
         "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ inline void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr) : "memory");
 }
 __device__ inline void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -365,7 +436,9 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
   const uint32_t acc_full = full_b + 16 * BSLOTS, acc_empty = acc_full + 16, epi_bar = acc_full + 32;
   const uint32_t help_bar = acc_full + 40;         // the epilogue warps and the de-quantiser warps that help them
   const uint32_t last_full = acc_full + 48;        // the MMAs of the block's last segment are complete (one phase only)
-  unsigned char* misc = smem + RING_BYTES + 16 * PSTAGES + 16 * BSLOTS + 56;
+  const uint32_t px_ready = acc_full + 56;         // pair split, second block: the first block's rings are idle
+  const uint32_t px_done = acc_full + 64;          // pair split, first block: the second block's sums have arrived
+  unsigned char* misc = smem + RING_BYTES + 16 * PSTAGES + 16 * BSLOTS + 72;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
 
@@ -382,6 +455,8 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
     pmbar_init(epi_bar, 4);
     pmbar_init(help_bar, 4 + 2 * DQ_WARPS);
     pmbar_init(last_full, 1);
+    pmbar_init(px_ready, 1);
+    pmbar_init(px_done, c.helpers ? 4 + 2 * DQ_WARPS : 4);       // one arrival per warp that sends
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -393,6 +468,11 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  const uint32_t crank = c.pair_split ? pcluster_rank() : 0u;
+  if (c.pair_split) {                   // the other block's barriers exist before anything is sent to it
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  }
 
   auto job_of_wt = [&](int wt) { int j = 0; while (j + 1 < p.n_jobs && wt >= c.wtile_begin[j + 1]) ++j; return j; };
   bool failed = false;
@@ -580,23 +660,61 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         //      would take the four epilogue warps longer than the tiles behind can hide: such launches add the parts
         //      into ONE sum per tile instead (reductions done in L2, zero at launch; the last bit of a sum then
         //      depends on the order of arrival when more than two blocks share a tile).
+        const bool pair_send = c.pair_split && crank != 0;
+        if (c.pair_split && !pair_send) {
+          // ---- the two blocks of a cluster each ran half of the contraction.  The second block waits until the
+          //      first one's MMAs are complete (its rings are idle then), writes its fp32 sums into them ([token][row]:
+          //      a warp stores 32 consecutive rows of a token) and arrives, one arrival per warp, at the first block's
+          //      barrier; the first block adds them to its own sums (always own + other: the same bits every run)
+          //      and finishes the tile.  No traffic through L2, no counter, nothing to clear.
+          {
+            if (!pmbar_wait_cluster(px_done, 0, abort_flag)) { failed = true; return; }
+            // (16 tokens at a time, as the read-back of the slots: what the registers of a thread hold)
+            for (int tk = 16 * ch0; tk < ntok; tk += 16 * chs) {
+              uint32_t v[16];
+              tmem_ld16(t_acc + (uint32_t)tk, v);
+              tmem_ld_wait();
+              const uint32_t src = sbase + (uint32_t)((tk * BMW + row) * 4);
+              float val[16];
+              pld_add_f32x16<BMW * 4>(src, v, val);
+              store_chunk(tk, val);
+            }
+          }
+          return;
+        }
         const bool main_lane = warp == EPI_WARP0 && lane == 0;
         const size_t slot_f = (size_t)ntok * BMW;
         const int T0 = (c.n_tiles / (int)gridDim.x) * (int)gridDim.x;          // first left-over tile
         float* mine = c.partials + ((size_t)(t - T0) + (c.sk_atomic ? 0 : blockIdx.x)) * slot_f;
+        if (pair_send) {
+          // (the second block of a pair: its "slot" is the first block's rings, once they are idle)
+          if (!pmbar_wait_cluster(px_ready, 0, abort_flag)) { failed = true; return; }
+          mine = ppeer_generic(smem, 0u);
+        }
         for (int ch = ch0; ch < ntok / EPI_TOK; ch += chs) {
           uint32_t v[32];
           tmem_ld32(t_acc + (uint32_t)(ch * EPI_TOK), v);
           tmem_ld_wait();
           if (chs == 1) release_after(ch);                     // the accumulator is free for the next segment
           float* dst = mine + (size_t)(ch * EPI_TOK) * BMW + row;
-          if (c.sk_atomic) {
+          if (pair_send) {
+#pragma unroll
+            for (int k = 0; k < 32; ++k) dst[(size_t)k * BMW] = __uint_as_float(v[k]);
+          } else if (c.sk_atomic) {
 #pragma unroll
             for (int k = 0; k < 32; ++k) atomicAdd(dst + (size_t)k * BMW, __uint_as_float(v[k]));
           } else {
 #pragma unroll
             for (int k = 0; k < 32; ++k) __stcg(dst + (size_t)k * BMW, __uint_as_float(v[k]));
           }
+        }
+        if (pair_send) {
+          __syncwarp();
+          if (lane == 0) {
+            asm volatile("fence.acq_rel.cluster;" ::: "memory");
+            pmbar_arrive_peer(ppeer_addr(px_done, 0u));
+          }
+          return;
         }
         __threadfence();                                       // this thread's part is in place before ...
         if (!(chs == 1 ? epi_sync() : help_sync())) { failed = true; return; }
@@ -703,6 +821,15 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
         SegIter peek = si;
         Seg nxt;
         if (!peek.next(nxt)) umma_commit(last_full);
+      }
+      if (c.pair_split && crank == 0 && !failed) {
+        // the first block of a pair: once its own MMAs are complete nothing reads its rings any more
+        if (pmbar_wait(last_full, 0, abort_flag)) {
+          asm volatile("fence.acq_rel.cluster;" ::: "memory");
+          pmbar_arrive_peer(ppeer_addr(px_ready, 1u));
+        } else {
+          failed = true;
+        }
       }
     }
   } else if (warp >= DQ_WARP0) {
@@ -864,6 +991,10 @@ __global__ void __launch_bounds__(PTH, 1) prefill_kernel(const __grid_constant__
   __syncthreads();
   tc_fence_after();
   if (warp == 1) tmem_dealloc(tmem_base, 512);
+  if (c.pair_split) {                   // neither block of a pair leaves while the other may still send to it
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  }
 }
 
 // -------------------------------------------------------------------------------- host side
@@ -913,12 +1044,25 @@ int launch_pth(const Params& p, const PrefillCfg& c, int grid, cudaStream_t stre
   lc.blockDim = dim3(PTH);
   lc.dynamicSmemBytes = smem;
   lc.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = attr;
   lc.numAttrs = opt(kOptPdl) ? 1 : 0;
-  if (cudaLaunchKernelEx(&lc, kern, p, c) != cudaSuccess) { cudaGetLastError(); return UNIQL_ERR_CUDA; }
+  if (c.pair_split) {
+    // clusters of two, only when every pair can be resident at once; else the caller plans without them
+    attr[lc.numAttrs].id = cudaLaunchAttributeClusterDimension;
+    attr[lc.numAttrs].val.clusterDim.x = 2;
+    attr[lc.numAttrs].val.clusterDim.y = 1;
+    attr[lc.numAttrs].val.clusterDim.z = 1;
+    ++lc.numAttrs;
+    int n_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&n_clusters, kern, &lc) != cudaSuccess || n_clusters * 2 < grid) {
+      cudaGetLastError();
+      return UNIQL_ERR_UNSUPPORTED;
+    }
+  }
+  if (cudaLaunchKernelEx(&lc, kern, p, c) != cudaSuccess) { cudaGetLastError(); return c.pair_split ? UNIQL_ERR_UNSUPPORTED : UNIQL_ERR_CUDA; }
   return UNIQL_OK;
 }
 template <typename T, bool CONV>
@@ -1014,7 +1158,8 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   if (env_grid >= 1 && env_grid <= sms) g2 = env_grid;            // tests: odd splits on small problems
   bool any_rope = false;
   for (int j = 0; j < p.n_jobs; ++j) any_rope = any_rope || p.job[j].rope.enabled != 0;
-  struct Plan { int nh, ttiles, tiles, left; bool streamk, atomic, halves; size_t sums; double us; };
+  struct Plan { int nh, ttiles, tiles, left; bool streamk, atomic, halves, pair; size_t sums; double us; };
+  static std::atomic<bool> pair_refused{false};       // a cluster launch was refused once: planned without from then on
   auto plan_for = [&](int nh) {
     Plan q;
     q.nh = nh;
@@ -1031,9 +1176,12 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
     const double pmax = q.left ? (double)((bt + q.left - 1) / q.left + 1) : 0.0;
     double hand_over;
     q.atomic = false;
+    // a k-block of a one-box tile by the number of busy SMs (0.45 us with 28 of them, 0.61 us with all)
+    auto kb1 = [&](int busy) { return 0.42 + 0.19 * (busy < g2 ? busy : g2) / g2; };
     if (q.tiles < g2) {
       // every tile is split and every block ends on a split tile: the hand-over is shared with the de-quantiser warps
-      hand_over = 24.0 + 2.0 * pmax * wide;
+      // (one-box tiles, measured at M = 64 .. 512 on seven layer shapes: 5 us per 64 tokens of the tile)
+      hand_over = nh == 2 ? 24.0 + 2.0 * pmax * wide : (14.0 + pmax) * wide;
     } else {
       // The split tiles come first and whole tiles follow.  Reading a tile's slots back takes the four epilogue
       // warps 11 us per slot of 256 tokens, and a split tile in front of whole tiles has three or more parts: that
@@ -1049,13 +1197,14 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
     if (env_streamk == 1) q.atomic = false;                            // tests: the form of the hand-over forced
     if (env_streamk == 2) q.atomic = true;
     // (a split is taken where it is estimated 5 % ahead: its hand-over varies more than a whole tile's time)
-    const double us_split = 1.05 * ((double)q.tiles / g2 * c.n_kb * kcost + hand_over);
+    const double us_split = 1.05 * ((double)q.tiles / g2 * c.n_kb * ((nh == 1 && q.tiles < g2) ? kb1(g2) : kcost) + hand_over);
     // Whole tiles.  On both accumulators a k-block takes 0.84 us when every SM runs one and less when some have no
     // tile (0.79 us with 28 busy SMs: they share the activation traffic out of L2), and between two tiles of a block
     // the MMAs wait 7 - 10 us for the epilogue to drain the accumulators (in-kernel time stamps, Qwen2.5-7B gate at
     // M = 2048); fitted over 48 launches (16 shapes at M = 512, 1024, 2048, every width and hand-over forced in turn).
     const int rounds = (q.tiles + g2 - 1) / g2;
     double us_whole = (double)rounds * c.n_kb * kcost;
+    if (nh == 1 && q.tiles <= g2) us_whole = c.n_kb * kb1(q.tiles);
     if (nh == 2)
       us_whole = (double)(q.tiles / g2) * c.n_kb * 0.96 + (q.left ? c.n_kb * (0.90 + 0.06 * q.left / g2) : 0.0) + 10.0 * (rounds - 1);
     // one fp32 slot per (left-over tile, block) piece, or one sum per left-over tile
@@ -1071,6 +1220,16 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
       const double us_halves = (double)(q.tiles / g2) * (c.n_kb * 0.96 + 10.0) + c.n_kb * (0.45 + 0.15 * 2 * q.left / g2);
       if (us_halves < q.us || opt(kOptPrefillDual) == 3) { q.halves = true; q.streamk = false; q.us = us_halves; }
     }
+    // Few tiles of one box (at most one for every two SMs): a cluster of two blocks per tile, half of the
+    // contraction each, the second block's sums handed over through the first one's shared memory (about 5 us
+    // against the 11 - 28 us of a hand-over through the workspace; a k-block takes the same 0.5 - 0.65 us).
+    q.pair = false;
+    if (nh == 1 && 2 * q.tiles <= sms && c.n_kb >= 4 && env_grid == 0 && !pair_refused.load() && (env_streamk < 0 || env_streamk == 3)) {
+      const double us_pair = (double)(c.n_kb - c.n_kb / 2) * kb1(2 * q.tiles) + 1.0 + 4.5 * wide + (any_rope ? 3.0 : 0.0);
+      // (against a split over all SMs it has to be 10 % ahead: with long contractions the two come out level and
+      //  the split measured ahead, Qwen2.5-7B down projection at M = 512)
+      if (us_pair * (q.streamk ? 1.10 : 1.0) < q.us || env_streamk == 3) { q.pair = true; q.streamk = false; q.us = us_pair; }
+    }
     return q;
   };
   Plan pl = plan_for(1);
@@ -1085,10 +1244,12 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
   c.helpers = opt(kOptPrefillHelpers) != 0;
   c.nh = pl.nh;
   c.halves = pl.halves ? 1 : 0;
+  c.pair_split = pl.pair ? 1 : 0;
   c.n_ttiles = pl.ttiles;
   c.n_tiles = pl.tiles;
   if ((long)wt * pl.ttiles > (1 << 24)) return UNIQL_ERR_SHAPE;
   int grid = c.n_tiles < g2 ? c.n_tiles : g2;
+  if (pl.pair) grid = 2 * c.n_tiles;
   {
     if (pl.streamk) {
       c.streamk = 1;
@@ -1129,10 +1290,18 @@ int launch_prefill(const Params& p, const LaunchCfg& cfg) {
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return UNIQL_ERR_CUDA;
   }
+  int rc;
   if (p.dt == UNIQL_BF16)
-    return conv_in_kernel ? launch_pt<__nv_bfloat16, true>(p, c, grid, cfg.stream)
-                          : launch_pt<__nv_bfloat16, false>(p, c, grid, cfg.stream);
-  return launch_pt<__half, false>(p, c, grid, cfg.stream);
+    rc = conv_in_kernel ? launch_pt<__nv_bfloat16, true>(p, c, grid, cfg.stream)
+                        : launch_pt<__nv_bfloat16, false>(p, c, grid, cfg.stream);
+  else
+    rc = launch_pt<__half, false>(p, c, grid, cfg.stream);
+  if (rc == UNIQL_ERR_UNSUPPORTED && c.pair_split) {
+    // the pairs cannot all be resident (or clusters cannot be launched here): planned again without them
+    pair_refused.store(true);
+    return launch_prefill(p, cfg);
+  }
+  return rc;
 }
 
 size_t prefill_workspace_bytes(int M, int K) {

@@ -553,3 +553,31 @@ def test_left_over_wide_tiles_as_half_tiles(B, M, dtype, grid):
     for (g, r) in run_rope(B, rng, M, 512, 6, 2, 128, 84, 5e5, dtype, bias=True):
         check_output(g, r, dtype, TOL[dtype], "half tiles, rope M=%d grid %d" % (M, grid))
     assert B.workspace_status() == 0
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("M", [17, 64, 100, 200, 256])
+def test_pairs_of_blocks_on_one_tile(B, M, dtype):
+    """Few tiles: a cluster of two blocks per tile, half of the contraction each; the second block's fp32 sums go
+    into the first one's shared memory and are added there (own + other, the same bits every run).  Forced, against
+    the oracle, twice for the bits; plain rows with bias, pruned inputs and outputs, a per-head input map and the
+    rotary epilogue; the library must come back clean."""
+    B.set_path(B.PATH_PREFILL)
+    B.set_option("prefill_streamk", 3)
+    rng = np.random.default_rng(8800 + M)
+    qw = synth.draw_qweight(rng, 300, 1024)
+    dw = dev_weight(qw)
+    bias = synth.to_dtype_values(rng.standard_normal(300).astype(np.float32), dtype)
+    for (k_in, k_out) in [(1024, 300), (652, 132), (256, 40)]:
+        x = synth.draw_x(np.random.default_rng(M + k_in), M, k_in, dtype)
+        y, ref = run_ex(B, qw, dw, x, dtype, None, k_in, None, k_out, bias=bias, ldx_pad=8 - k_in % 8 if k_in % 8 else 0, ldy_pad=3)
+        check_output(y, ref, dtype, TOL[dtype], "pairs M=%d %s k=(%d,%d)" % (M, dtype, k_in, k_out))
+        y2, _ = run_ex(B, qw, dw, x, dtype, None, k_in, None, k_out, bias=bias, ldx_pad=8 - k_in % 8 if k_in % 8 else 0, ldy_pad=3)
+        assert torch.equal(y, y2)
+    im = synth.map_per_head(8, 128, 104)
+    x = synth.draw_x(rng, M, synth.map_size(im), dtype)
+    y, ref = run_ex(B, qw, dw, x, dtype, im, 0, None, 200, ldx_pad=8)
+    check_output(y, ref, dtype, TOL[dtype], "pairs, per-head input map M=%d" % M)
+    for (g, r) in run_rope(B, rng, M, 512, 6, 2, 128, 84, 5e5, dtype, bias=True):
+        check_output(g, r, dtype, TOL[dtype], "pairs, rope M=%d" % M)
+    assert B.workspace_status() == 0
