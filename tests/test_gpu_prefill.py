@@ -581,3 +581,26 @@ def test_pairs_of_blocks_on_one_tile(B, M, dtype):
     for (g, r) in run_rope(B, rng, M, 512, 6, 2, 128, 84, 5e5, dtype, bias=True):
         check_output(g, r, dtype, TOL[dtype], "pairs, rope M=%d" % M)
     assert B.workspace_status() == 0
+
+
+def test_random_shapes_under_the_launcher_s_own_plan(B):
+    """Seeded random shapes with nothing forced: whatever the launcher picks on the full grid (whole tiles of either
+    width, pairs of blocks on a tile, split tiles in both forms, half tiles) must match the oracle, and launches
+    whose plan is reproducible by construction must repeat bit for bit."""
+    B.set_path(B.PATH_PREFILL)
+    rng = np.random.default_rng(20261130)
+    cases = []
+    for _ in range(28):
+        M = int(rng.choice([17, 40, 64, 100, 128, 200, 256, 257, 384, 512, 700, 1024, 1100]))
+        N = int(rng.integers(1, 9)) * 128 - int(rng.choice([0, 0, 28, 96]))
+        K = int(rng.integers(1, 9)) * 128
+        cases.append((M, N, K, K - int(rng.choice([0, 0, 0, 52, 120]))))
+    cases += [(4096, 2560, 256, 256), (2048, 9600, 128, 128), (1536, 2432, 384, 380)]   # more tiles than SMs: left-over rounds
+    for (M, N, K, k_in) in cases:
+        dtype = "bf16" if (M + N) % 3 == 0 else "f16"
+        qw = synth.draw_qweight(rng, N, K)
+        dw = dev_weight(qw)
+        x = synth.draw_x(rng, M, k_in, dtype)
+        y, ref = run_ex(B, qw, dw, x, dtype, None, k_in, None, N, ldx_pad=8 - k_in % 8 if k_in % 8 else 0)
+        check_output(y, ref, dtype, TOL[dtype], "auto plan M=%d N=%d K=%d k_in=%d %s" % (M, N, K, k_in, dtype))
+        assert B.workspace_status() == 0
