@@ -25,6 +25,12 @@
 //                -- and writes them into the A-operand stage in the
 //                canonical K-major 128-byte-swizzled layout; the packed codes of the next k-block
 //                are already in registers.  All sixteen share the epilogue of the block's last segment.
+// Work split (chosen by the launcher from a cost model): whole tiles round-robin; tiles left over after the whole
+// rounds split along K over all blocks (stream-K: parts handed over through slots in the workspace, or added into
+// one sum per tile) or, for tiles of two boxes, run as half tiles on twice the blocks; launches with few tiles as
+// clusters of two blocks per tile, the second block's sums written into the first one's idle rings.
+// Launched with programmatic stream serialization: what a block does before griddepcontrol.wait (barriers, tensor
+// memory, the first weight stages) touches nothing a preceding kernel may still read or write.
 // On-device pruning (Section 3.4) is index arithmetic: tile rows are compact output channels mapped to
 // stored rows per thread; the input side is the leading k_in channels (the TMA tensor ends at k_in, so
 // the tail of the last k-block is zero activations).
