@@ -1062,11 +1062,14 @@ int launch_pth(const Params& p, const PrefillCfg& c, int grid, cudaStream_t stre
     attr[lc.numAttrs].val.clusterDim.y = 1;
     attr[lc.numAttrs].val.clusterDim.z = 1;
     ++lc.numAttrs;
-    int n_clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&n_clusters, kern, &lc) != cudaSuccess || n_clusters * 2 < grid) {
-      cudaGetLastError();
-      return UNIQL_ERR_UNSUPPORTED;
+    // (asked once per kernel instance: the answer depends on the block's resources, which do not change)
+    static std::atomic<int> max_clusters{-1};
+    int n_clusters = max_clusters.load();
+    if (n_clusters < 0) {
+      if (cudaOccupancyMaxActiveClusters(&n_clusters, kern, &lc) != cudaSuccess) { cudaGetLastError(); n_clusters = 0; }
+      max_clusters.store(n_clusters);
     }
+    if (n_clusters * 2 < grid) return UNIQL_ERR_UNSUPPORTED;
   }
   if (cudaLaunchKernelEx(&lc, kern, p, c) != cudaSuccess) { cudaGetLastError(); return c.pair_split ? UNIQL_ERR_UNSUPPORTED : UNIQL_ERR_CUDA; }
   return UNIQL_OK;
